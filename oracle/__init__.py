@@ -1,0 +1,20 @@
+"""CPU oracle for the backward-state-policy operators and their per-use check.
+
+TEST INFRASTRUCTURE, NOT PRODUCT.  Plain numpy, float64 unless a step is pinned to FP32, slow
+and written to be checked against the paper by eye.  Only the tests, the smoke entry and the
+benchmark's CPU-baseline leg may import this package; the CUDA library never does, and this
+package imports nothing from it.  No blocking, fusion or reordering beyond what each definition
+states.
+
+Modules (each function cites the passage of the paper it follows):
+  philox     Philox4x32-10 and the (seed, tensor, use, draw, element) keying
+  fp8        E4M3 / E5M2 codec, round-to-nearest-even and stochastic rounding
+  norm       RMSNorm / LayerNorm store forward, the three reads, backward
+  linear     incoming gradient, weight gradient, input-gradient helper
+  attention  causal attention forward statistics and backward with the D use
+  mc         Monte-Carlo reduction, statistics z, R, Q', verdict
+
+Parity unpinned (no value of the paper fixes them; only GPU == oracle): the verdict
+thresholds of `mc.verdict`, and the quantisation points / P and dS scales of the FP8-operand
+attention mode.
+"""
