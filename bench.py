@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the per-use check (one JSON line on stdout).
+
+A step is one pass of the whole hot path over one batch of synthetic input: statistics and
+current-amax scale, forward store, incoming gradient to E5M2, du = dY W, then the six
+(use, policy) evaluations of the check -- gain use {U, R, N x K}, weight use {U, R, N x K}.
+Workload at every N: config 2, RMSNorm -> Linear at 390M-model shapes, replicated per GPU
+(the path has no exchange step, so N GPUs run N independent replicas: weak scaling).
+
+metric = per-use check elements/s: sum over use-evaluations of (saved-tensor elements x draws
+consumed) divided by the time of the step.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "per_use_check_elements_per_s"
+UNIT = "elements/s"
+WORKLOAD = "cfg2_rmsnorm_linear_390m"
+
+
+def check_elements(T, C, K):
+    """Saved-tensor elements x draws over the six use-evaluations (U, R: 1 draw; N: K draws)."""
+    return T * C * (2 * (1 + 1 + K))
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"], samples=0)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2] if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ----------------------------------------------------------------------------------- oracle arm
+
+
+def oracle_sample(inp, rows, k_gain, k_wgrad):
+    """The oracle as it stands on the first `rows` tokens of the workload: preparation, gain use
+    {U, R, N x k_gain}, weight use {U, R, N x k_wgrad}.  Returns (seconds, check elements)."""
+    from oracle import check, norm
+    kind = norm.RMS if inp.norm == "rms" else norm.LAYER
+    x, dY = inp.x[:rows], inp.dY[:rows]
+    t0 = time.perf_counter()
+    prep = check.prepare_norm_linear(x, inp.gamma, inp.beta, inp.W, dY, kind, inp.eps, inp.seed, inp.dtype)
+    for p in (0, 1, 2):
+        check.gain_use(x, inp.gamma, inp.beta, kind, inp.eps, prep, p, k_gain, inp.seed)
+    for p in (0, 1, 2):
+        check.wgrad_use(prep, p, k_wgrad, inp.seed)
+    dt = time.perf_counter() - t0
+    return dt, rows * inp.C * (2 + k_gain + 2 + k_wgrad)
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads") for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_39813_b200 import workloads
+    inp = workloads.config2()
+    # calibrate on a small slice, then size each step so the whole run stays within ~2.5 minutes
+    dt0, el0 = oracle_sample(inp, 64, 2, 2)
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    rows = int(max(64, min(inp.T, 64 * budget / max(dt0, 1e-3))))
+    rows = max(64, rows // 64 * 64)
+    for _ in range(args.warmup):
+        oracle_sample(inp, rows, 2, 2)
+    total_t, total_el = 0.0, 0
+    for _ in range(args.steps):
+        dt, el = oracle_sample(inp, rows, 2, 2)
+        total_t += dt
+        total_el += el
+    value = total_el / total_t
+    sample = "first %d of %d tokens, gain {U,R,N x2} + weight {U,R,N x2}, numpy float64" % (rows, inp.T)
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * total_t / max(1, args.steps), higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=WORKLOAD, T=inp.T, C=inp.C, O=inp.O, K=inp.K),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=blas_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------- CUDA arm
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_39813_b200 import binding as b
+    from paper_2609_39813_b200 import workloads
+    from paper_2609_39813_b200.harness import NormLinearGpu, up
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    b.lib()
+
+    inp = workloads.config2()
+    T, C, O, K = inp.T, inp.C, inp.O, inp.K
+    g = NormLinearGpu(inp)
+    desc = g.desc()
+    ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
+    diag = b.new_diag()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB of L2
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        return b.bsp_mc_check(desc, K, ws, diag)
+
+    for _ in range(max(args.warmup, 3)):
+        res = step()
+    verdicts = [r.verdict for r in res]
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    barrier()
+    n0 = b.bsp_launch_count()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)              # evict L2 between timed steps (not timed)
+        starts[i].record(stream)
+        step()
+        ends[i].record(stream)
+    barrier()
+    launches = b.bsp_launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    elements = check_elements(T, C, K)
+    value = world * elements * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end: host buffers in, host results out, through the same entry point
+    host = dict(x=g.x.cpu().pin_memory(), gamma=g.gamma.cpu().pin_memory(), W=g.W.cpu().pin_memory(),
+                dY=g.dY.cpu().pin_memory())
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = sum(min(592, (n + 255) // 256) * 64 for n in (C, C, C, O * C, O * C, O * C))
+    e2e_steps = max(3, min(args.steps, 20))
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        g.x.copy_(host["x"], non_blocking=True)
+        g.gamma.copy_(host["gamma"], non_blocking=True)
+        g.W.copy_(host["W"], non_blocking=True)
+        g.dY.copy_(host["dY"], non_blocking=True)
+        step()
+    e1.record(stream)
+    barrier()
+    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_value = world * elements * e2e_steps / (float(t2.item()) * 1e-3)
+
+    # ---- roofline of the dominant kernel: the FP8 weight-gradient contraction with the fused
+    # shifted-sum epilogue, timed alone with CUDA events on the launching stream
+    peaks = read_peaks()
+    fresh_t = torch.zeros(C * g.ld_t, dtype=torch.uint8, device="cuda")
+    qf = b.quant(inp.store_fmt, b.ROUND_STOCHASTIC, 1.0, g.scale)
+    b.bsp_norm_fwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, qf,
+                   b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, 0), None, fresh_t, g.ld_t)
+    ref = torch.zeros(O * C, device="cuda")
+    S1 = torch.zeros(O * C, device="cuda")
+    S2 = torch.zeros(O * C, device="cuda")
+    wsg = b.workspace(256)
+    reps = 32
+    for _ in range(3):
+        b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, b.READ_FRESH, fresh_t, qf, g.ld_t, None, ref, S1, S2, wsg, diag)
+    torch.cuda.synchronize()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record(stream)
+    for _ in range(reps):
+        b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, b.READ_FRESH, fresh_t, qf, g.ld_t, None, ref, S1, S2, wsg, diag)
+    r1.record(stream)
+    torch.cuda.synchronize()
+    gemm_ms = r0.elapsed_time(r1) / reps
+    flops = 2.0 * T * O * C
+    achieved = flops / (gemm_ms * 1e-3) / 1e12
+    peak = 2.0 * peaks["bf16_tflops"]        # FP8 dense = 2 x the measured BF16 burst figure
+    roofline = dict(bound="tensor", kernel="gemm_tc_kernel<fp8> (weight gradient, MC epilogue)",
+                    achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                    us_per_launch=gemm_ms * 1e3, peak_source="2 x bf16_tflops (%s)" % peaks["source"])
+    dstat = b.read_diag(diag)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        dt, el = oracle_sample(inp, 512, 2, 2)
+        cpu_baseline = dict(value=el / dt, unit=UNIT, cores=blas_threads(), kind="oracle",
+                            sample="first 512 of %d tokens, gain {U,R,N x2} + weight {U,R,N x2}, %.1f s" % (T, dt))
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                ms_per_step=ms_total / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f8e4m3/f8e5m2 operands, f32 accumulate", data="synthetic",
+                config=dict(workload=WORKLOAD, T=T, C=C, O=O, K=K, policies="gain{U,R,N} x weight{U,R,N}",
+                            l2="flushed between timed steps (256 MiB write, outside the timed spans)",
+                            replicas=world),
+                clocks=clocks,
+                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
+                gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
+                verdicts=verdicts, diag_status=dstat["status"])
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 100 and args.warmup == 5:
+            args.steps, args.warmup = 5, 1
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

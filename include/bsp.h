@@ -1,0 +1,279 @@
+/*
+ * bsp.h -- C ABI of the backward-state-policy operator library for NVIDIA B200 (sm_100a).
+ *
+ * The paper ("Backward-State Policy Is Part of the Learning Algorithm") studies what each
+ * backward *use* of a saved, rounded tensor reads: U the original, R the forward's rounding, N a
+ * new stochastic rounding from a separate generator stream (Introduction; Section "One tensor,
+ * two uses").  This library evaluates single operators under such a per-use policy and checks
+ * each use against the paper's reference -- the gradient of the forward as it ran, rounding
+ * passed straight through -- with a K-draw Monte-Carlo reduction, without any training.
+ *
+ * Conventions (all entry points):
+ *   - plain C, every function returns a bsp_status_t as int;
+ *   - every pointer is a CALLER-OWNED DEVICE pointer unless its comment says "host"; tensors are
+ *     row-major and contiguous, base addresses 16-byte aligned;
+ *   - the library allocates no device memory: scratch comes from the caller's workspace `ws` of
+ *     `ws_bytes` bytes (256-byte aligned); the needed size is returned by the matching
+ *     *_workspace_bytes() query; a too-small workspace returns BSP_ERR_WORKSPACE before launch;
+ *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     unless stated; outputs are valid after the caller synchronises that stream;
+ *   - argument errors are detected on the host and returned before anything is launched;
+ *   - device-detected conditions (non-finite inputs, saturated roundings, a bounded wait that
+ *     ran out) are accumulated into the caller's device-resident bsp_diag_t, never trapped; the
+ *     caller clears it (bsp_diag_clear) and reads it back after synchronising;
+ *   - no global mutable state: the same inputs give byte-identical outputs.
+ *
+ * FP8 codes are raw bit patterns (uint8): E4M3 = 1-4-3 bits, bias 7, no infinity, NaN 0x7F/0xFF,
+ * max 448; E5M2 = 1-5-2, bias 15, max 57344.  A code stands for decode(code) / scale.
+ */
+#ifndef BSP_H_
+#define BSP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  BSP_OK = 0,
+  BSP_ERR_ARG = 1,          /* NULL / negative / inconsistent argument                    */
+  BSP_ERR_ALIGN = 2,        /* pointer or leading dimension not 16-byte aligned           */
+  BSP_ERR_UNSUPPORTED = 3,  /* valid request this build does not implement                */
+  BSP_ERR_WORKSPACE = 4,    /* workspace missing or too small                             */
+  BSP_ERR_NONFINITE = 5,    /* (diag.status) NaN or infinity met in an input              */
+  BSP_ERR_TIMEOUT = 6,      /* (diag.status) a bounded device-side wait ran out           */
+  BSP_ERR_CUDA = 7          /* a CUDA runtime or driver call failed                       */
+} bsp_status_t;
+
+typedef enum { BSP_E4M3 = 0, BSP_E5M2 = 1 } bsp_format_t;
+typedef enum { BSP_ROUND_NEAREST = 0, BSP_ROUND_STOCHASTIC = 1 } bsp_round_mode_t;
+/* What a backward use reads (Section "One tensor, two uses"; Appendix table "Store policies"). */
+typedef enum { BSP_READ_ORIGINAL = 0 /* U */, BSP_READ_FORWARD = 1 /* R */, BSP_READ_FRESH = 2 /* N */ } bsp_policy_t;
+typedef enum { BSP_F32 = 0, BSP_BF16 = 1 } bsp_dtype_t;
+typedef enum { BSP_RMSNORM = 0, BSP_LAYERNORM = 1 } bsp_norm_t;
+typedef enum { BSP_HOLDS = 0, BSP_FAILS = 1, BSP_UNDECIDED = 2 } bsp_verdict_t;
+
+/* Generator streams: the `stream` field of bsp_key_t.  "The new rounding uses a separate stream
+ * of the same law" (Appendix "The forks"). */
+enum { BSP_STREAM_FORWARD = 0, BSP_STREAM_GAIN = 1, BSP_STREAM_WGRAD = 2, BSP_STREAM_DX = 3,
+       BSP_STREAM_ATTN_D = 4, BSP_STREAM_SHARED = 255 };
+
+/* Key of the counter-based generator (Philox4x32-10).  Element with row-major logical index e of
+ * tensor `tensor_id` uses word (e & 3) of
+ *   philox(counter = (lo32(e>>2), hi32(e>>2), draw, (tensor_id << 8) | stream),
+ *          key     = (lo32(seed), hi32(seed))).
+ * One 32-bit word per element, independent of layout, tiling and launch shape. */
+typedef struct {
+  uint64_t seed;
+  uint32_t tensor_id;   /* < 2^24 */
+  uint32_t stream;      /* < 256  */
+  uint32_t draw;
+  uint32_t reserved;    /* must be 0 */
+} bsp_key_t;
+
+/* How a tensor is rounded: code = round(fl32(x * scale)).  If scale_dev is not NULL the kernels
+ * read the scale from that device float (scale_dev[0]) and ignore `scale`; this lets a scale
+ * computed on the device (bsp_scale_from_amax) be used without a host round trip. */
+typedef struct {
+  int32_t fmt;              /* bsp_format_t     */
+  int32_t mode;             /* bsp_round_mode_t */
+  float scale;
+  const float* scale_dev;
+} bsp_quant_t;
+
+/* Device-resident diagnostics, accumulated with atomics by every kernel that is handed one. */
+typedef struct {
+  unsigned long long n_saturated;   /* finite magnitudes above the format's maximum          */
+  unsigned long long n_nonfinite;   /* NaN or infinite inputs                                 */
+  uint32_t amax_bits;               /* bit pattern of the largest finite |value| seen (float) */
+  int32_t status;                   /* BSP_OK, BSP_ERR_NONFINITE or BSP_ERR_TIMEOUT           */
+} bsp_diag_t;
+
+/* Result of one (use, output tensor) evaluation of the check; lives in HOST memory.
+ * Statistics: standard error over draws and z = (m - g*) / se (Appendix "Checkpointing");
+ * R = ||m - g*||^2 / sum_j se_j^2 (Appendix "The normalization store"); Q' = mean z^2 (K-3)/(K-1);
+ * rel = ||m - g*||_2 / ||g*||_2.  Verdict: deterministic read -> HOLDS iff rel <= 1e-4;
+ * fresh read -> HOLDS if Q' <= 2 and R <= 3, FAILS if Q' >= 4 or R >= 6, else UNDECIDED. */
+typedef struct {
+  int32_t use_id;            /* BSP_STREAM_* of the use                         */
+  int32_t output_id;         /* bsp_output_t                                    */
+  int32_t policy;            /* bsp_policy_t                                    */
+  int32_t K;                 /* draws (1 for U and R)                           */
+  int64_t n_elements;
+  double rel_l2_mean_err;
+  double R;
+  double Qprime;
+  double mean_z;
+  double rms_z;
+  double max_abs_z;
+  double frac_abs_z_gt3;
+  int32_t verdict;           /* bsp_verdict_t                                   */
+  int32_t reserved;
+} bsp_use_result_t;
+
+typedef enum { BSP_OUT_DGAMMA = 0, BSP_OUT_DBETA = 1, BSP_OUT_DW = 2, BSP_OUT_DX = 3,
+               BSP_OUT_D = 4, BSP_OUT_DQ = 5, BSP_OUT_DK = 6, BSP_OUT_DV = 7 } bsp_output_t;
+
+const char* bsp_status_string(int status);
+
+/* Number of kernels this library has launched in this process so far (a monotone counter kept for
+ * accounting; it influences no result). */
+unsigned long long bsp_launch_count(void);
+
+/* Clears a device bsp_diag_t (asynchronous memset). */
+int bsp_diag_clear(bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Rounding (Section "Same rounding distribution, opposite outcomes": stochastic rounding sends
+ * a bracketed value to one of its two neighbours with a zero-mean error; Appendix "The forks":
+ * entries at the top of the range round to nearest and are counted, generator keyed on seed and
+ * stream).
+ * ------------------------------------------------------------------------------------------ */
+
+/* out[i] = the 32-bit generator word of element i, i in [0, n).  For the bit-exact stream test. */
+int bsp_philox_fill(bsp_key_t key, size_t n, uint32_t* out, void* stream);
+
+/* amax[g] = max |x| over group g (n_groups contiguous groups of group_size elements); NaN and
+ * infinities are skipped and counted in diag (may be NULL).  Overwrites amax. */
+int bsp_amax(const void* x, int dt, size_t n_groups, size_t group_size, float* amax,
+             bsp_diag_t* diag, void* stream);
+
+/* scale[g] = fl32(fmax / amax[g]); 1 when amax is 0, non-finite, or the quotient overflows. */
+int bsp_scale_from_amax(const float* amax, size_t n, int fmt, float* scale, void* stream);
+
+/* codes[i] = round(fl32(x[i] * scale)), nearest-even saturating, or stochastic with the word of
+ * element `elem_offset + i` under `key`.  x: dt[n]; codes: uint8[n]. */
+int bsp_round(const void* x, int dt, size_t n, bsp_quant_t q, bsp_key_t key, uint64_t elem_offset,
+              uint8_t* codes, bsp_diag_t* diag, void* stream);
+
+/* Same with one scale per contiguous group: scales[n_groups] (device).  Element index is the
+ * position in the whole tensor. */
+int bsp_round_grouped(const void* x, int dt, size_t n_groups, size_t group_size, int fmt, int mode,
+                      const float* scales, bsp_key_t key, uint8_t* codes, bsp_diag_t* diag,
+                      void* stream);
+
+/* 2-D variant that can also write the transposed code matrix used by the weight-gradient
+ * contraction: codes[r*cols + c] (may be NULL) and codes_t[c*ld_t + r] (may be NULL), ld_t >= rows
+ * and a multiple of 16. */
+int bsp_round_2d(const void* x, int dt, int64_t rows, int64_t cols, bsp_quant_t q, bsp_key_t key,
+                 uint8_t* codes, uint8_t* codes_t, int64_t ld_t, bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Normalisation store (Appendix "The normalization store"; Eq. norm-uses): z, u = gamma o z
+ * (+ beta), u_q = round(u).  RMSNorm: rstd = 1/sqrt(mean x^2 + eps); LayerNorm: mean, biased
+ * variance.  The value handed to the rounding is a fixed chain of FP32 operations without FMA:
+ *   RMS  fl(fl(fl(x*rstd)*gamma)*scale);  LN  fl(fl(fl(fl(fl(x-mean)*rstd)*gamma)+beta)*scale).
+ * ------------------------------------------------------------------------------------------ */
+
+/* Row statistics and the largest |u| (for a current-amax scale).  rstd[T], mean[T] (LayerNorm
+ * only; may be NULL for RMSNorm), amax: one device float, overwritten (may be NULL). */
+int bsp_norm_stats(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                   const float* beta, float eps, float* rstd, float* mean, float* amax,
+                   bsp_diag_t* diag, void* stream);
+
+/* Rounds u from saved statistics.  Any of the outputs may be NULL:
+ *   u_codes[T*C], u_codes_t[C*ld_t] (transposed), u_f32[T*C] (the FP32 u before scaling),
+ *   u_bf16_t[C*ld_t] (u rounded to bf16, transposed: the U operand of the weight gradient).
+ * With key.stream = BSP_STREAM_FORWARD this is the forward's store; with another stream and
+ * mode stochastic it is the re-rounding pass that feeds a fresh read (policy N). */
+int bsp_norm_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                 const float* beta, const float* rstd, const float* mean, bsp_quant_t q,
+                 bsp_key_t key, uint8_t* u_codes, uint8_t* u_codes_t, int64_t ld_t, float* u_f32,
+                 void* u_bf16_t, bsp_diag_t* diag, void* stream);
+
+/* Backward of the normalisation with du passed through the rounding unchanged:
+ *   dgamma[C] = sum_t z_g o du, z_g = z (U) | (decode(u_codes)/scale - beta)/gamma (R) |
+ *               the same from a fresh rounding under `key` (N, one draw);
+ *   dbeta[C] = sum_t du (may be NULL);  dx[T*C] from unrounded values (may be NULL):
+ *   RMS dx = rstd (dz - z mean_j(dz o z)), LN dx = rstd (dz - mean_j dz - z mean_j(dz o z)),
+ *   dz = gamma o du.  du: du_dt[T*C].  Outputs FP32. */
+size_t bsp_norm_bwd_workspace_bytes(int64_t T, int64_t C);
+int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                 const float* beta, const float* rstd, const float* mean, const void* du, int du_dt,
+                 int gain_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key,
+                 float* dgamma, float* dbeta, float* dx, void* ws, size_t ws_bytes,
+                 bsp_diag_t* diag, void* stream);
+
+/* K fresh draws of the gain use in one pass over x and du: for draw k in [draw0, draw0+K) the
+ * gain gradient g_k is formed as in bsp_norm_bwd (policy N, key.draw = k) and the shifted sums
+ * S1[c] += sum_k (g_k[c] - g_ref[c]), S2[c] += sum_k (g_k[c] - g_ref[c])^2 are accumulated, so
+ * draw ranges can be split and merged by addition.  Never materialises the K gradients. */
+size_t bsp_norm_gain_mc_workspace_bytes(int64_t T, int64_t C, int K);
+int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                     const float* beta, const float* rstd, const float* mean, const void* du,
+                     int du_dt, bsp_quant_t q, bsp_key_t key, int draw0, int K, const float* g_ref,
+                     float* S1, float* S2, void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Linear layer after the store (Eq. norm-uses: dW = u_q^T dy; reading the original adds
+ * -r^T dy).  W is stored [O, C]; dW[O, C] = dY^T X with X the copy the weight use reads.
+ * Operands are "token-minor" (transposed) matrices: dy_t[O*ld_t], x_t[C*ld_t], entry (row, t) at
+ * row*ld_t + t, ld_t a multiple of 16 -- as written by bsp_round_2d / bsp_norm_fwd.
+ *   x_read = U: x_t is bf16 (u rounded to bf16), dy is decoded to bf16 in `ws`; BF16 tensor cores.
+ *   x_read = R or N: x_t is uint8 codes in q_x.fmt; FP8 tensor cores (E5M2 x E4M3).
+ * FP32 accumulation; dW = acc / (scale_dy * scale_x).
+ * If mc_ref is not NULL the epilogue does not store dW but accumulates the shifted sums
+ *   S1 += dW - mc_ref, S2 += (dW - mc_ref)^2          (all [O*C] FP32).
+ * ------------------------------------------------------------------------------------------ */
+size_t bsp_linear_wgrad_workspace_bytes(int64_t T, int64_t O, int64_t C, int x_read);
+int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy,
+                     int x_read, const void* x_t, bsp_quant_t q_x, int64_t ld_t, float* dW,
+                     const float* mc_ref, float* mc_S1, float* mc_S2, void* ws, size_t ws_bytes,
+                     bsp_diag_t* diag, void* stream);
+
+/* du[T*C] (du_dt) = dY W with dY = decode(dy_codes[T*O]) / scale and W w_dt[O*C]: the incoming
+ * gradient passed through the rounding unchanged.  BF16 tensor cores (W rounded to bf16). */
+size_t bsp_linear_dgrad_workspace_bytes(int64_t T, int64_t O, int64_t C);
+int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, bsp_quant_t q_dy,
+                     const void* W, int w_dt, void* du, int du_dt, void* ws, size_t ws_bytes,
+                     bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Monte-Carlo reduction (Section "Each use has a checkable requirement").
+ * ------------------------------------------------------------------------------------------ */
+
+/* Reduces per-element shifted sums to the statistics of bsp_use_result_t and the verdict.
+ * fresh = 0: deterministic read, `g` holds the gradient itself (S2 ignored, K = 1).
+ * fresh = 1: g = S1, with S2, over K draws.  ws: >= bsp_mc_stats_workspace_bytes(n).
+ * Synchronises `stream`; `result` is HOST memory; use_id/output_id/policy are left untouched. */
+size_t bsp_mc_stats_workspace_bytes(int64_t n);
+int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
+                 bsp_use_result_t* result, void* ws, size_t ws_bytes, void* stream);
+
+/* The whole per-use check of a normalisation -> linear workload, device-resident inputs.
+ * Once per call: statistics, current-amax scale, forward store (stream 0, `forward_mode`),
+ * incoming gradient dY -> E5M2 nearest at its own amax, du = dY W.  Then per use and policy:
+ *   gain use  (dgamma, reference read U):  U, R, N (K draws);
+ *   weight use (dW,    reference read R):  U, R, N (K draws: re-round + FP8 contraction + fused
+ *   shifted-sum epilogue).
+ * `policy_mask` bit (use*3 + policy) selects evaluations, use 0 = gain, 1 = weight.
+ * results: HOST array, filled in order gain U,R,N then weight U,R,N (selected ones only);
+ * *n_results returns the count.  Synchronises before returning. */
+typedef struct {
+  int32_t norm_kind;         /* bsp_norm_t  */
+  int32_t dtype;             /* bsp_dtype_t of x, W, dY (and of du) */
+  int64_t T, C, O;
+  const void* x;             /* [T, C] */
+  const float* gamma;        /* [C]    */
+  const float* beta;         /* [C] or NULL */
+  const void* W;             /* [O, C] */
+  const void* dY;            /* [T, O] */
+  float eps;
+  int32_t store_fmt;         /* bsp_format_t of the store (E4M3)      */
+  int32_t grad_fmt;          /* bsp_format_t of dY (E5M2)             */
+  int32_t forward_mode;      /* bsp_round_mode_t of the forward store */
+  uint64_t seed;
+  uint32_t tensor_id;
+  uint32_t policy_mask;
+} bsp_norm_linear_desc_t;
+
+size_t bsp_mc_check_workspace_bytes(const bsp_norm_linear_desc_t* op, int K);
+int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* results, int* n_results,
+                 void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BSP_H_ */

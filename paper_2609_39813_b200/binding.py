@@ -1,0 +1,303 @@
+"""ctypes binding of libbsp.so: the same names as the C ABI (include/bsp.h), argument marshalling
+only -- every step of the path runs in the CUDA kernels.  Tensors are torch CUDA tensors (or
+None for optional pointers); torch is used for device memory and streams, nothing else.
+
+There is no CPU fallback: loading fails loudly when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libbsp.so")
+
+OK, ERR_ARG, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA = range(8)
+E4M3, E5M2 = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+READ_ORIGINAL, READ_FORWARD, READ_FRESH = 0, 1, 2
+F32, BF16 = 0, 1
+RMSNORM, LAYERNORM = 0, 1
+HOLDS, FAILS, UNDECIDED = 0, 1, 2
+STREAM_FORWARD, STREAM_GAIN, STREAM_WGRAD, STREAM_DX, STREAM_ATTN_D, STREAM_SHARED = 0, 1, 2, 3, 4, 255
+OUT_DGAMMA, OUT_DBETA, OUT_DW, OUT_DX, OUT_D, OUT_DQ, OUT_DK, OUT_DV = range(8)
+
+
+class Key(C.Structure):
+    _fields_ = [("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("stream", C.c_uint32),
+                ("draw", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class Quant(C.Structure):
+    _fields_ = [("fmt", C.c_int32), ("mode", C.c_int32), ("scale", C.c_float), ("scale_dev", C.c_void_p)]
+
+
+class Diag(C.Structure):
+    _fields_ = [("n_saturated", C.c_ulonglong), ("n_nonfinite", C.c_ulonglong),
+                ("amax_bits", C.c_uint32), ("status", C.c_int32)]
+
+
+class UseResult(C.Structure):
+    _fields_ = [("use_id", C.c_int32), ("output_id", C.c_int32), ("policy", C.c_int32), ("K", C.c_int32),
+                ("n_elements", C.c_int64), ("rel_l2_mean_err", C.c_double), ("R", C.c_double),
+                ("Qprime", C.c_double), ("mean_z", C.c_double), ("rms_z", C.c_double),
+                ("max_abs_z", C.c_double), ("frac_abs_z_gt3", C.c_double), ("verdict", C.c_int32),
+                ("reserved", C.c_int32)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+
+
+class NormLinearDesc(C.Structure):
+    _fields_ = [("norm_kind", C.c_int32), ("dtype", C.c_int32), ("T", C.c_int64), ("C", C.c_int64),
+                ("O", C.c_int64), ("x", C.c_void_p), ("gamma", C.c_void_p), ("beta", C.c_void_p),
+                ("W", C.c_void_p), ("dY", C.c_void_p), ("eps", C.c_float), ("store_fmt", C.c_int32),
+                ("grad_fmt", C.c_int32), ("forward_mode", C.c_int32), ("seed", C.c_uint64),
+                ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
+
+
+class BspError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+_P, _SZ, _I, _I64, _U64, _F = C.c_void_p, C.c_size_t, C.c_int, C.c_int64, C.c_uint64, C.c_float
+
+_SIGNATURES = {
+    "bsp_status_string": (C.c_char_p, [_I]),
+    "bsp_launch_count": (C.c_ulonglong, []),
+    "bsp_diag_clear": (_I, [_P, _P]),
+    "bsp_philox_fill": (_I, [Key, _SZ, _P, _P]),
+    "bsp_amax": (_I, [_P, _I, _SZ, _SZ, _P, _P, _P]),
+    "bsp_scale_from_amax": (_I, [_P, _SZ, _I, _P, _P]),
+    "bsp_round": (_I, [_P, _I, _SZ, Quant, Key, _U64, _P, _P, _P]),
+    "bsp_round_grouped": (_I, [_P, _I, _SZ, _SZ, _I, _I, _P, Key, _P, _P, _P]),
+    "bsp_round_2d": (_I, [_P, _I, _I64, _I64, Quant, Key, _P, _P, _I64, _P, _P]),
+    "bsp_norm_stats": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _F, _P, _P, _P, _P, _P]),
+    "bsp_norm_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, Quant, Key, _P, _P, _I64, _P, _P, _P, _P]),
+    "bsp_norm_bwd_workspace_bytes": (_SZ, [_I64, _I64]),
+    "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
+                          _P, _SZ, _P, _P]),
+    "bsp_norm_gain_mc_workspace_bytes": (_SZ, [_I64, _I64, _I]),
+    "bsp_norm_gain_mc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, Quant, Key, _I, _I, _P, _P, _P,
+                              _P, _SZ, _P, _P]),
+    "bsp_linear_wgrad_workspace_bytes": (_SZ, [_I64, _I64, _I64, _I]),
+    "bsp_linear_wgrad": (_I, [_I64, _I64, _I64, _P, Quant, _I, _P, Quant, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
+    "bsp_linear_dgrad_workspace_bytes": (_SZ, [_I64, _I64, _I64]),
+    "bsp_linear_dgrad": (_I, [_I64, _I64, _I64, _P, Quant, _P, _I, _P, _I, _P, _SZ, _P, _P]),
+    "bsp_mc_stats_workspace_bytes": (_SZ, [_I64]),
+    "bsp_mc_stats": (_I, [_P, _P, _P, _I64, _I, _I, C.POINTER(UseResult), _P, _SZ, _P]),
+    "bsp_mc_check_workspace_bytes": (_SZ, [C.POINTER(NormLinearDesc), _I]),
+    "bsp_mc_check": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(UseResult), C.POINTER(_I), _P, _SZ, _P, _P]),
+}
+
+
+def exported_names():
+    """Every symbol include/bsp.h declares."""
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    """The loaded library.  Raises if it has not been built: there is no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libbsp.so is missing (%s): build it with `python -m paper_2609_39813_b200.build`; "
+                "this package has no CPU or PyTorch fallback" % LIB_PATH)
+        l = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().bsp_status_string(int(status)).decode()
+
+
+def check(status: int, where: str = "bsp"):
+    if status != OK:
+        raise BspError(status, where)
+
+
+def ptr(t):
+    """Device pointer of a torch tensor (must be contiguous), or NULL for None; ints pass through."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise ValueError("unsupported dtype %s" % t.dtype)
+
+
+def cur_stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def key(seed, tensor_id, stream, draw=0) -> Key:
+    return Key(int(seed) & 0xFFFFFFFFFFFFFFFF, int(tensor_id), int(stream), int(draw), 0)
+
+
+def quant(fmt, mode, scale=1.0, scale_dev=None) -> Quant:
+    return Quant(int(fmt), int(mode), float(scale), ptr(scale_dev))
+
+
+def new_diag():
+    """A zeroed device bsp_diag_t as a uint8 tensor."""
+    import torch
+    return torch.zeros(C.sizeof(Diag), dtype=torch.uint8, device="cuda")
+
+
+def read_diag(d) -> dict:
+    import torch
+    torch.cuda.synchronize()
+    raw = bytes(d.cpu().numpy().tobytes())
+    s = Diag.from_buffer_copy(raw)
+    import struct
+    amax = struct.unpack("<f", struct.pack("<I", s.amax_bits))[0]
+    return dict(n_saturated=s.n_saturated, n_nonfinite=s.n_nonfinite, amax=amax, status=s.status)
+
+
+def workspace(nbytes: int):
+    import torch
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device="cuda")
+
+
+# ----------------------------------------------------------------------------- entry points
+
+
+def bsp_launch_count() -> int:
+    return int(lib().bsp_launch_count())
+
+
+def bsp_diag_clear(diag, stream=None):
+    check(lib().bsp_diag_clear(ptr(diag), stream if stream is not None else cur_stream()), "bsp_diag_clear")
+
+
+def bsp_philox_fill(k: Key, n, out, stream=None):
+    check(lib().bsp_philox_fill(k, n, ptr(out), stream if stream is not None else cur_stream()), "bsp_philox_fill")
+
+
+def bsp_amax(x, n_groups, group_size, amax, diag=None, stream=None):
+    check(lib().bsp_amax(ptr(x), dtype_code(x), n_groups, group_size, ptr(amax), ptr(diag),
+                         stream if stream is not None else cur_stream()), "bsp_amax")
+
+
+def bsp_scale_from_amax(amax, n, fmt, scale, stream=None):
+    check(lib().bsp_scale_from_amax(ptr(amax), n, fmt, ptr(scale), stream if stream is not None else cur_stream()),
+          "bsp_scale_from_amax")
+
+
+def bsp_round(x, n, q: Quant, k: Key, elem_offset, codes, diag=None, stream=None):
+    check(lib().bsp_round(ptr(x), dtype_code(x), n, q, k, elem_offset, ptr(codes), ptr(diag),
+                          stream if stream is not None else cur_stream()), "bsp_round")
+
+
+def bsp_round_grouped(x, n_groups, group_size, fmt, mode, scales, k: Key, codes, diag=None, stream=None):
+    check(lib().bsp_round_grouped(ptr(x), dtype_code(x), n_groups, group_size, fmt, mode, ptr(scales), k,
+                                  ptr(codes), ptr(diag), stream if stream is not None else cur_stream()),
+          "bsp_round_grouped")
+
+
+def bsp_round_2d(x, rows, cols, q: Quant, k: Key, codes, codes_t, ld_t, diag=None, stream=None):
+    check(lib().bsp_round_2d(ptr(x), dtype_code(x), rows, cols, q, k, ptr(codes), ptr(codes_t), ld_t, ptr(diag),
+                             stream if stream is not None else cur_stream()), "bsp_round_2d")
+
+
+def bsp_norm_stats(kind, x, T, Cc, gamma, beta, eps, rstd, mean, amax, diag=None, stream=None):
+    check(lib().bsp_norm_stats(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), eps, ptr(rstd),
+                               ptr(mean), ptr(amax), ptr(diag), stream if stream is not None else cur_stream()),
+          "bsp_norm_stats")
+
+
+def bsp_norm_fwd(kind, x, T, Cc, gamma, beta, rstd, mean, q: Quant, k: Key, u_codes, u_codes_t, ld_t,
+                 u_f32=None, u_bf16_t=None, diag=None, stream=None):
+    check(lib().bsp_norm_fwd(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean), q, k,
+                             ptr(u_codes), ptr(u_codes_t), ld_t, ptr(u_f32), ptr(u_bf16_t), ptr(diag),
+                             stream if stream is not None else cur_stream()), "bsp_norm_fwd")
+
+
+def bsp_norm_bwd_workspace_bytes(T, Cc):
+    return lib().bsp_norm_bwd_workspace_bytes(T, Cc)
+
+
+def bsp_norm_bwd(kind, x, T, Cc, gamma, beta, rstd, mean, du, gain_read, u_codes, q: Quant, k: Key,
+                 dgamma, dbeta, dx, ws, diag=None, stream=None):
+    check(lib().bsp_norm_bwd(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
+                             ptr(du), dtype_code(du), gain_read, ptr(u_codes), q, k, ptr(dgamma), ptr(dbeta),
+                             ptr(dx), ptr(ws), ws.numel() if ws is not None else 0, ptr(diag),
+                             stream if stream is not None else cur_stream()), "bsp_norm_bwd")
+
+
+def bsp_norm_gain_mc_workspace_bytes(T, Cc, K):
+    return lib().bsp_norm_gain_mc_workspace_bytes(T, Cc, K)
+
+
+def bsp_norm_gain_mc(kind, x, T, Cc, gamma, beta, rstd, mean, du, q: Quant, k: Key, draw0, K, g_ref, S1, S2,
+                     ws, diag=None, stream=None):
+    check(lib().bsp_norm_gain_mc(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
+                                 ptr(du), dtype_code(du), q, k, draw0, K, ptr(g_ref), ptr(S1), ptr(S2), ptr(ws),
+                                 ws.numel() if ws is not None else 0, ptr(diag),
+                                 stream if stream is not None else cur_stream()), "bsp_norm_gain_mc")
+
+
+def bsp_linear_wgrad_workspace_bytes(T, O, Cc, x_read):
+    return lib().bsp_linear_wgrad_workspace_bytes(T, O, Cc, x_read)
+
+
+def bsp_linear_wgrad(T, O, Cc, dy_codes_t, q_dy: Quant, x_read, x_t, q_x: Quant, ld_t, dW, mc_ref=None,
+                     mc_S1=None, mc_S2=None, ws=None, diag=None, stream=None):
+    check(lib().bsp_linear_wgrad(T, O, Cc, ptr(dy_codes_t), q_dy, x_read, ptr(x_t), q_x, ld_t, ptr(dW),
+                                 ptr(mc_ref), ptr(mc_S1), ptr(mc_S2), ptr(ws), ws.numel() if ws is not None else 0,
+                                 ptr(diag), stream if stream is not None else cur_stream()), "bsp_linear_wgrad")
+
+
+def bsp_linear_dgrad_workspace_bytes(T, O, Cc):
+    return lib().bsp_linear_dgrad_workspace_bytes(T, O, Cc)
+
+
+def bsp_linear_dgrad(T, O, Cc, dy_codes, q_dy: Quant, W, du, ws, diag=None, stream=None):
+    check(lib().bsp_linear_dgrad(T, O, Cc, ptr(dy_codes), q_dy, ptr(W), dtype_code(W), ptr(du), dtype_code(du),
+                                 ptr(ws), ws.numel() if ws is not None else 0, ptr(diag),
+                                 stream if stream is not None else cur_stream()), "bsp_linear_dgrad")
+
+
+def bsp_mc_stats_workspace_bytes(n):
+    return lib().bsp_mc_stats_workspace_bytes(n)
+
+
+def bsp_mc_stats(g_ref, g, S2, n, K, fresh, ws, stream=None) -> UseResult:
+    r = UseResult()
+    check(lib().bsp_mc_stats(ptr(g_ref), ptr(g), ptr(S2), n, K, fresh, C.byref(r), ptr(ws), ws.numel(),
+                             stream if stream is not None else cur_stream()), "bsp_mc_stats")
+    return r
+
+
+def bsp_mc_check_workspace_bytes(desc: NormLinearDesc, K):
+    return lib().bsp_mc_check_workspace_bytes(C.byref(desc), K)
+
+
+def bsp_mc_check(desc: NormLinearDesc, K, ws, diag=None, stream=None):
+    """Returns the list of UseResult (gain U,R,N then weight U,R,N; selected ones only)."""
+    res = (UseResult * 8)()
+    n = C.c_int(0)
+    check(lib().bsp_mc_check(C.byref(desc), K, res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
+                             stream if stream is not None else cur_stream()), "bsp_mc_check")
+    return [res[i] for i in range(n.value)]

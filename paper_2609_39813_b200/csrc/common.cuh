@@ -1,0 +1,226 @@
+// Device-side building blocks shared by the kernels: Philox4x32-10, the FP8 codec, typed loads.
+// Everything here is written for sm_100a; integer paths are bit-exact by construction.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bsp.h"
+
+#define BSP_CHECK_CUDA(expr)                      \
+  do {                                            \
+    cudaError_t _e = (expr);                      \
+    if (_e != cudaSuccess) return BSP_ERR_CUDA;   \
+  } while (0)
+
+// Every kernel launch of the library is followed by this: it counts the launch (see
+// bsp_launch_count) and turns a launch error into BSP_ERR_CUDA.
+#define BSP_LAUNCH_CHECK()                   \
+  do {                                       \
+    ::bsp::count_launch();                   \
+    BSP_CHECK_CUDA(cudaGetLastError());      \
+  } while (0)
+
+namespace bsp {
+
+void count_launch();          // defined in mc.cu
+
+constexpr int kNumSMs = 148;
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
+
+// ------------------------------------------------------------------------------- Philox
+
+struct PhiloxKey {
+  uint32_t k0, k1;     // lo32(seed), hi32(seed)
+  uint32_t c2, c3;     // draw, (tensor_id << 8) | stream
+};
+
+static inline PhiloxKey make_key(const bsp_key_t& k) {
+  PhiloxKey p;
+  p.k0 = (uint32_t)(k.seed & 0xFFFFFFFFull);
+  p.k1 = (uint32_t)(k.seed >> 32);
+  p.c2 = k.draw;
+  p.c3 = (k.tensor_id << 8) | (k.stream & 0xFFu);
+  return p;
+}
+
+// Ten rounds; counter (c0, c1, c2, c3), key (k0, k1).  Returns the four output words.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += W0; k1 += W1;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// Words of elements 4q .. 4q+3 of a tensor (q = element index >> 2).
+__device__ __forceinline__ uint4 philox_block(const PhiloxKey& k, uint64_t q, uint32_t draw) {
+  return philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), draw, k.c3, k.k0, k.k1);
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& w, uint32_t lane) {
+  return lane == 0 ? w.x : lane == 1 ? w.y : lane == 2 ? w.z : w.w;
+}
+
+// ------------------------------------------------------------------------------- FP8 codec
+
+template <int FMT> struct F8;
+template <> struct F8<BSP_E4M3> {
+  static constexpr int MB = 3, EMIN = -6, BIAS = 7;
+  static constexpr uint32_t FMAX_BITS = 0x43E00000u;   // 448.0f
+  static constexpr uint32_t TOP = 0x7Eu;
+  static constexpr uint32_t EMASK = 0xFu;
+};
+template <> struct F8<BSP_E5M2> {
+  static constexpr int MB = 2, EMIN = -14, BIAS = 15;
+  static constexpr uint32_t FMAX_BITS = 0x47600000u;   // 57344.0f
+  static constexpr uint32_t TOP = 0x7Bu;
+  static constexpr uint32_t EMASK = 0x1Fu;
+};
+
+// Per-thread counters, flushed to bsp_diag_t once per thread.
+struct DiagCounters {
+  uint32_t sat = 0, nonfinite = 0;
+};
+
+// Round an FP32 value to an FP8 code.  e = max(floor(log2|v|), EMIN), ulp = 2^(e-MB),
+// n = floor(|v|/ulp), f = frac.  Nearest: up iff f > 1/2 or tie with n odd.  Stochastic: up iff
+// U < floor(f * 2^32).  Saturating; the sign bit is kept even when the magnitude rounds to zero.
+template <int FMT, bool STOCHASTIC>
+__device__ __forceinline__ uint32_t f8_encode(float v, uint32_t U, DiagCounters& dc) {
+  using F = F8<FMT>;
+  const uint32_t b = __float_as_uint(v);
+  const uint32_t sign = (b >> 24) & 0x80u;
+  const uint32_t a = b & 0x7FFFFFFFu;
+  if (a >= F::FMAX_BITS) {
+    if (a > 0x7F800000u) { dc.nonfinite++; return sign | 0x7Fu; }       // NaN -> canonical NaN
+    if (a == 0x7F800000u) dc.nonfinite++; else if (a > F::FMAX_BITS) dc.sat++;
+    return sign | F::TOP;
+  }
+  const uint32_t efield = a >> 23;
+  if (efield == 0) return sign;                                           // FP32 zero / denormal
+  const int E = (int)efield - 127;
+  const uint32_t sig = (a & 0x7FFFFFu) | 0x800000u;
+  uint32_t base, up;
+  if (E >= F::EMIN) {
+    constexpr int d = 23 - F::MB;
+    const uint32_t rem = sig & ((1u << d) - 1u);
+    const uint32_t n = sig >> d;                                           // in [2^MB, 2^(MB+1))
+    base = ((uint32_t)(E + F::BIAS) << F::MB) | (n & ((1u << F::MB) - 1u));
+    if (STOCHASTIC) {
+      up = U < (rem << (32 - d));
+    } else {
+      constexpr uint32_t half = 1u << (d - 1);
+      up = (rem > half) | ((rem == half) & (n & 1u));
+    }
+  } else {
+    int d = 23 - F::MB + (F::EMIN - E);
+    d = d > 60 ? 60 : d;
+    const uint64_t s64 = sig;
+    const uint64_t rem = s64 & ((1ull << d) - 1ull);
+    const uint32_t n = (uint32_t)(s64 >> d);
+    base = n;
+    if (STOCHASTIC) {
+      up = (uint64_t)U < ((rem << 32) >> d);
+    } else {
+      const uint64_t half = 1ull << (d - 1);
+      up = (rem > half) | ((rem == half) & (n & 1u));
+    }
+  }
+  return sign | (base + up);
+}
+
+// Exact FP32 value of a code.
+template <int FMT>
+__device__ __forceinline__ float f8_decode(uint32_t c) {
+  using F = F8<FMT>;
+  const uint32_t s = (c & 0x80u) << 24;
+  const uint32_t ef = (c >> F::MB) & F::EMASK;
+  const uint32_t m = c & ((1u << F::MB) - 1u);
+  if (FMT == BSP_E4M3) {
+    if ((c & 0x7Fu) == 0x7Fu) return __uint_as_float(s | 0x7FC00000u);
+  } else {
+    if (ef == 31u) return __uint_as_float(s | (m ? 0x7FC00000u : 0x7F800000u));
+  }
+  if (ef == 0) {
+    // subnormal: m * 2^(EMIN - MB); m < 8 is exact in FP32
+    const float mag = (float)m * __uint_as_float((uint32_t)(F::EMIN - F::MB + 127) << 23);
+    return __uint_as_float(s | __float_as_uint(mag));
+  }
+  return __uint_as_float(s | ((ef - F::BIAS + 127u) << 23) | (m << (23 - F::MB)));
+}
+
+__device__ __forceinline__ void diag_flush(bsp_diag_t* diag, const DiagCounters& dc) {
+  if (diag == nullptr) return;
+  if (dc.sat) atomicAdd(&diag->n_saturated, (unsigned long long)dc.sat);
+  if (dc.nonfinite) {
+    atomicAdd(&diag->n_nonfinite, (unsigned long long)dc.nonfinite);
+    atomicMax(&diag->status, (int)BSP_ERR_NONFINITE);
+  }
+}
+
+// Warp-aggregated flush: one atomic per warp.
+__device__ __forceinline__ void diag_flush_warp(bsp_diag_t* diag, DiagCounters dc) {
+  if (diag == nullptr) return;
+  uint32_t sat = dc.sat, nf = dc.nonfinite;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sat += __shfl_xor_sync(0xFFFFFFFFu, sat, o);
+    nf += __shfl_xor_sync(0xFFFFFFFFu, nf, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    DiagCounters t; t.sat = sat; t.nonfinite = nf;
+    diag_flush(diag, t);
+  }
+}
+
+// ------------------------------------------------------------------------------- typed loads
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+
+// Four consecutive elements starting at element index i (i % 4 == 0, pointer 16-byte aligned).
+template <int DT>
+__device__ __forceinline__ float4 load4(const void* p, size_t i) {
+  if (DT == BSP_F32) {
+    return __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + i));
+  } else {
+    const uint2 r = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(p) + i));
+    return make_float4(bf16_bits_to_float(r.x & 0xFFFFu), bf16_bits_to_float(r.x >> 16),
+                       bf16_bits_to_float(r.y & 0xFFFFu), bf16_bits_to_float(r.y >> 16));
+  }
+}
+
+template <int DT>
+__device__ __forceinline__ float load1(const void* p, size_t i) {
+  if (DT == BSP_F32) return __ldg(reinterpret_cast<const float*>(p) + i);
+  return bf16_bits_to_float(__ldg(reinterpret_cast<const uint16_t*>(p) + i));
+}
+
+// Round-to-nearest-even float -> bf16 bit pattern (finite inputs).
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+}  // namespace bsp

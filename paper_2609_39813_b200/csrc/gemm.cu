@@ -1,0 +1,637 @@
+// Dense contractions on the 5th-generation tensor cores: C[M,N] = alpha * A[M,K] B[N,K]^T with
+// both operands K-major (K contiguous), FP8 (kind::f8f6f4, E5M2/E4M3 in any combination) or BF16
+// (kind::f16) operands and FP32 accumulation in tensor memory.
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0      TMA producer   (cp.async.bulk.tensor, 128-byte swizzle, kStages-deep mbarrier ring)
+//   warp 1      MMA issuer     (one elected lane issues tcgen05.mma 128 x 256 x 32B; owns TMEM alloc)
+//   warps 2..5  epilogue       (tcgen05.ld 32 lanes x 32 columns -> registers -> global)
+// Two accumulator stages (2 x 256 TMEM columns) let the epilogue of one tile overlap the main loop
+// of the next.  Work items are (tile, batch): a CTA owns its tiles and walks all batches of a tile
+// in order, so the Monte-Carlo epilogue's read-modify-write of the shifted sums is race-free and
+// bit-reproducible.  Every wait is bounded; on time-out the kernel records BSP_ERR_TIMEOUT in the
+// diagnostics word and unwinds (TMEM is freed on every path).
+#include <cuda.h>
+#include <stdlib.h>
+
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace bsp {
+
+// ------------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait here
+
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit or another
+// role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <bool FP8>
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  if (FP8) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+  }
+}
+
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, K-major operand in the 128-byte-swizzle layout that TMA writes
+// (rows at a 128-byte pitch, 16-byte chunks XOR-ed with row % 8; 8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                                // leading byte offset: 1 (fixed) for swizzled K-major
+  d |= (uint64_t)(1024u >> 4) << 32;                     // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                                // descriptor version (sm_100)
+  d |= (uint64_t)2 << 61;                                // layout: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: FP32 accumulator, K-major A and B, M x N tile.
+// a_fmt / b_fmt: kind::f8f6f4 E4M3 = 0, E5M2 = 1; kind::f16 BF16 = 1.
+__host__ __device__ constexpr uint32_t make_idesc(uint32_t a_fmt, uint32_t b_fmt, uint32_t M, uint32_t N) {
+  return (1u << 4) | (a_fmt << 7) | (b_fmt << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------- the kernel
+
+constexpr int BM = 128, BN = 256, BKB = 128;      // tile; BKB = K extent of one stage in bytes
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BKB, kBBytes = BN * BKB, kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+struct GemmParams {
+  int M, N, K;            // K in elements
+  int nb;                 // batches of B (and of C in plain mode)
+  int elem_bytes;         // 1 (FP8) or 2 (BF16)
+  uint32_t idesc;
+  float sa, sb;           // operand scales; alpha = (1/sa) * (1/sb)
+  const float* sa_dev;
+  const float* sb_dev;
+  int mode;               // EPI_*
+  void* C;                // float or bf16 [nb][M][ldc]
+  int64_t ldc;
+  const float* ref;       // EPI_MC
+  float* S1;
+  float* S2;
+  bsp_diag_t* diag;
+};
+
+template <bool FP8>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                    // 1024-byte aligned operand ring
+  const uint32_t bars = tiles + kStages * kStageBytes;              // barriers after the ring
+  // barrier layout (8 bytes each): full[kStages], empty[kStages], tfull[2], tempty[2]; then tmem slot, abort flag
+  const uint32_t full0 = bars, empty0 = bars + 8 * kStages, tfull0 = bars + 16 * kStages, tempty0 = tfull0 + 16;
+  uint8_t* bars_gen = smem_raw + (bars - raw);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 16 * kStages + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 16 * kStages + 36);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = (p.K * p.elem_bytes + BKB - 1) / BKB;
+  const int bk_elems = BKB / p.elem_bytes;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_a);
+      tma_prefetch_desc(&tmap_b);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        const int tm = t / tiles_n, tn = t % tiles_n;
+        for (int b = 0; b < p.nb && ok; ++b) {
+          for (int kb = 0; kb < kblocks; ++kb, ++it) {
+            const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t sa = tiles + s * kStageBytes, sb = sa + kABytes;
+            mbar_expect_tx(full0 + 8 * s, kStageBytes);
+            tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * bk_elems, tm * BM);
+            tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * bk_elems, tn * BN, b);
+          }
+        }
+      }
+      if (!ok) {
+        // let copies already in flight land before the CTA's shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, tc = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        for (int b = 0; b < p.nb && ok; ++b, ++tc) {
+          const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
+          if (!mbar_wait(tempty0 + 8 * as, aph ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t tmem_d = tmem_base + as * BN;
+          for (int kb = 0; kb < kblocks; ++kb, ++it) {
+            const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
+            if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = tiles + s * kStageBytes, sb = sa + kABytes;
+            const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+#pragma unroll
+            for (int k = 0; k < BKB / 32; ++k) {
+              // advance 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
+              tc_mma<FP8>(tmem_d, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            tc_commit(empty0 + 8 * s);          // frees the stage when these MMAs have read it
+          }
+          if (ok) tc_commit(tfull0 + 8 * as);   // accumulator complete
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                      // TMEM lane quarter this warp may access
+    const float inv_a = __fdiv_rn(1.0f, p.sa_dev ? __ldg(p.sa_dev) : p.sa);
+    const float inv_b = __fdiv_rn(1.0f, p.sb_dev ? __ldg(p.sb_dev) : p.sb);
+    uint32_t tc = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+      const int tm = t / tiles_n, tn = t % tiles_n;
+      const int row = tm * BM + q * 32 + lane;
+      for (int b = 0; b < p.nb && ok; ++b, ++tc) {
+        const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
+        // every lane polls; the outcome is made warp-uniform before any .aligned instruction
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull0 + 8 * as, aph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + as * BN + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          const int col0 = tn * BN + ch * 32;
+          if (col0 >= p.N) break;                // warp-uniform
+          uint32_t r[32];
+          tmem_ld32(taddr + ch * 32, r);
+          if (row < p.M) {
+            const size_t off = (size_t)row * p.ldc + col0;
+            if (p.mode == EPI_STORE_F32) {
+              float* dst = reinterpret_cast<float*>(p.C) + (size_t)b * p.M * p.ldc + off;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                if (col0 + j < p.N) {
+                  float4 o;
+                  o.x = __uint_as_float(r[j]) * inv_a * inv_b; o.y = __uint_as_float(r[j + 1]) * inv_a * inv_b;
+                  o.z = __uint_as_float(r[j + 2]) * inv_a * inv_b; o.w = __uint_as_float(r[j + 3]) * inv_a * inv_b;
+                  *reinterpret_cast<float4*>(dst + j) = o;
+                }
+              }
+            } else if (p.mode == EPI_STORE_BF16) {
+              uint16_t* dst = reinterpret_cast<uint16_t*>(p.C) + (size_t)b * p.M * p.ldc + off;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                if (col0 + j < p.N) {
+                  const uint32_t lo = float_to_bf16_bits(__uint_as_float(r[j]) * inv_a * inv_b) |
+                                      (float_to_bf16_bits(__uint_as_float(r[j + 1]) * inv_a * inv_b) << 16);
+                  const uint32_t hi = float_to_bf16_bits(__uint_as_float(r[j + 2]) * inv_a * inv_b) |
+                                      (float_to_bf16_bits(__uint_as_float(r[j + 3]) * inv_a * inv_b) << 16);
+                  *reinterpret_cast<uint2*>(dst + j) = make_uint2(lo, hi);
+                }
+              }
+            } else {   // EPI_MC: shifted sums against the reference gradient
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                if (col0 + j < p.N) {
+                  const float4 g0 = *reinterpret_cast<const float4*>(p.ref + off + j);
+                  float4 s1 = *reinterpret_cast<float4*>(p.S1 + off + j);
+                  float4 s2 = *reinterpret_cast<float4*>(p.S2 + off + j);
+                  const float d0 = __uint_as_float(r[j]) * inv_a * inv_b - g0.x;
+                  const float d1 = __uint_as_float(r[j + 1]) * inv_a * inv_b - g0.y;
+                  const float d2 = __uint_as_float(r[j + 2]) * inv_a * inv_b - g0.z;
+                  const float d3 = __uint_as_float(r[j + 3]) * inv_a * inv_b - g0.w;
+                  s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
+                  s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y);
+                  s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
+                  *reinterpret_cast<float4*>(p.S1 + off + j) = s1;
+                  *reinterpret_cast<float4*>(p.S2 + off + j) = s2;
+                }
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.diag) atomicMax(&p.diag->status, (int)BSP_ERR_TIMEOUT);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------- diagnostic SIMT path
+
+// Plain shared-memory tiled contraction on the CUDA cores; selected only by BSP_GEMM_SIMT=1 in
+// the environment, to tell a tensor-core-path defect from a defect elsewhere.
+template <bool FP8>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(const void* __restrict__ A, const void* __restrict__ B, int a_fmt, int b_fmt, int64_t lda,
+                 int64_t ldb, int64_t b_batch_stride, GemmParams p) {
+  __shared__ float sa[16][17], sb[16][17];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int m = blockIdx.y * 16 + ty, n = blockIdx.x * 16 + tx;
+  const int b = blockIdx.z;
+  const float inv_a = __fdiv_rn(1.0f, p.sa_dev ? __ldg(p.sa_dev) : p.sa);
+  const float inv_b = __fdiv_rn(1.0f, p.sb_dev ? __ldg(p.sb_dev) : p.sb);
+  float acc = 0.f;
+  for (int k0 = 0; k0 < p.K; k0 += 16) {
+    const int ka = k0 + tx;
+    float av = 0.f, bv = 0.f;
+    const int mr = blockIdx.y * 16 + ty, nr = blockIdx.x * 16 + ty;
+    if (mr < p.M && ka < p.K) {
+      if (FP8) {
+        const uint32_t c = reinterpret_cast<const uint8_t*>(A)[(size_t)mr * lda + ka];
+        av = a_fmt == BSP_E4M3 ? f8_decode<BSP_E4M3>(c) : f8_decode<BSP_E5M2>(c);
+      } else {
+        av = bf16_bits_to_float(reinterpret_cast<const uint16_t*>(A)[(size_t)mr * lda + ka]);
+      }
+    }
+    if (nr < p.N && ka < p.K) {
+      const size_t idx = (size_t)b * b_batch_stride + (size_t)nr * ldb + ka;
+      if (FP8) {
+        const uint32_t c = reinterpret_cast<const uint8_t*>(B)[idx];
+        bv = b_fmt == BSP_E4M3 ? f8_decode<BSP_E4M3>(c) : f8_decode<BSP_E5M2>(c);
+      } else {
+        bv = bf16_bits_to_float(reinterpret_cast<const uint16_t*>(B)[idx]);
+      }
+    }
+    sa[ty][tx] = av;
+    sb[ty][tx] = bv;
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc = fmaf(sa[ty][k], sb[tx][k], acc);
+    __syncthreads();
+  }
+  if (m < p.M && n < p.N) {
+    const float v = acc * inv_a * inv_b;
+    const size_t off = (size_t)m * p.ldc + n;
+    if (p.mode == EPI_STORE_F32) {
+      reinterpret_cast<float*>(p.C)[(size_t)b * p.M * p.ldc + off] = v;
+    } else if (p.mode == EPI_STORE_BF16) {
+      reinterpret_cast<uint16_t*>(p.C)[(size_t)b * p.M * p.ldc + off] = (uint16_t)float_to_bf16_bits(v);
+    } else {
+      const float d = v - p.ref[off];
+      p.S1[off] += d;
+      p.S2[off] = fmaf(d, d, p.S2[off]);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Tensor map over a K-major matrix [batch][rows][K] (row pitch ld elements), box = 128 bytes x box_rows.
+static int make_operand_map(CUtensorMap* map, const void* base, int elem_bytes, int64_t K, int64_t rows, int64_t ld,
+                            int64_t nbatch, int64_t batch_stride_elems, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return BSP_ERR_CUDA;
+  const CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  cuuint64_t gdim[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)nbatch};
+  cuuint64_t gstr[2] = {(cuuint64_t)ld * elem_bytes, (cuuint64_t)batch_stride_elems * elem_bytes};
+  cuuint32_t box[3] = {(cuuint32_t)(BKB / elem_bytes), (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t rank = nbatch > 0 ? 3 : 2;
+  if (rank == 3 && nbatch == 1) gstr[1] = (cuuint64_t)rows * ld * elem_bytes;   // any valid stride
+  CUresult r = fn(map, dt, rank, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
+}
+
+static bool simt_forced() {
+  const char* e = getenv("BSP_GEMM_SIMT");
+  return e && e[0] == '1';
+}
+
+int gemm_run(const GemmArgs& g, cudaStream_t st) {
+  if (g.M <= 0 || g.N <= 0 || g.nb <= 0) return BSP_OK;
+  if (g.K <= 0) return BSP_ERR_ARG;
+  const int eb = g.fp8 ? 1 : 2;
+  if ((g.lda * eb) % 16 != 0 || (g.ldb * eb) % 16 != 0 || !aligned16(g.A) || !aligned16(g.B)) return BSP_ERR_ALIGN;
+  if (g.ldc % 4 != 0 || !aligned16(g.C) || !aligned16(g.ref) || !aligned16(g.S1) || !aligned16(g.S2))
+    return BSP_ERR_ALIGN;
+  if ((g.b_batch_stride * eb) % 16 != 0) return BSP_ERR_ALIGN;
+  GemmParams p;
+  p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K; p.nb = g.nb; p.elem_bytes = eb;
+  p.idesc = g.fp8 ? make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, BN)
+                  : make_idesc(1u, 1u, BM, BN);
+  p.sa = g.sa; p.sb = g.sb; p.sa_dev = g.sa_dev; p.sb_dev = g.sb_dev;
+  p.mode = g.mode; p.C = g.C; p.ldc = g.ldc; p.ref = g.ref; p.S1 = g.S1; p.S2 = g.S2; p.diag = g.diag;
+
+  if (simt_forced()) {
+    dim3 grid((unsigned)((g.N + 15) / 16), (unsigned)((g.M + 15) / 16), (unsigned)g.nb);
+    // the MC epilogue is a read-modify-write: batches must run one after another
+    if (g.mode == EPI_MC && g.nb > 1) {
+      for (int b = 0; b < g.nb; ++b) {
+        grid.z = 1;
+        const void* Bb = reinterpret_cast<const uint8_t*>(g.B) + (size_t)b * g.b_batch_stride * eb;
+        if (g.fp8) gemm_simt_kernel<true><<<grid, 256, 0, st>>>(g.A, Bb, g.a_fmt, g.b_fmt, g.lda, g.ldb, 0, p);
+        else gemm_simt_kernel<false><<<grid, 256, 0, st>>>(g.A, Bb, g.a_fmt, g.b_fmt, g.lda, g.ldb, 0, p);
+      }
+    } else {
+      if (g.fp8) gemm_simt_kernel<true><<<grid, 256, 0, st>>>(g.A, g.B, g.a_fmt, g.b_fmt, g.lda, g.ldb, g.b_batch_stride, p);
+      else gemm_simt_kernel<false><<<grid, 256, 0, st>>>(g.A, g.B, g.a_fmt, g.b_fmt, g.lda, g.ldb, g.b_batch_stride, p);
+    }
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  }
+
+  CUtensorMap ma, mb;
+  int rc = make_operand_map(&ma, g.A, eb, g.K, g.M, g.lda, 0, 0, BM);
+  if (rc != BSP_OK) return rc;
+  rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN);
+  if (rc != BSP_OK) return rc;
+  static bool attr_set[2] = {false, false};
+  if (!attr_set[g.fp8 ? 1 : 0]) {
+    if (g.fp8) BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
+    else BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
+    attr_set[g.fp8 ? 1 : 0] = true;
+  }
+  const int ntiles = (int)(((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN));
+  int nsm = kNumSMs;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) nsm = v;
+  }
+  const int grid = ntiles < nsm ? ntiles : nsm;
+  if (g.fp8) gemm_tc_kernel<true><<<grid, kGemmThreads, kGemmSmem, st>>>(ma, mb, p);
+  else gemm_tc_kernel<false><<<grid, kGemmThreads, kGemmSmem, st>>>(ma, mb, p);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+// ------------------------------------------------------------------------------- operand preparation
+
+// codes -> bf16 (exact: every FP8 value is a bf16 value), same layout.
+template <int FMT>
+__global__ void decode_to_bf16_kernel(const uint8_t* __restrict__ codes, size_t n16, uint16_t* __restrict__ out) {
+  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n16) return;
+  const uint4 c = __ldg(reinterpret_cast<const uint4*>(codes) + t);
+  const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t b0 = __float_as_uint(f8_decode<FMT>(w[i] & 0xFFu)) >> 16;
+    const uint32_t b1 = __float_as_uint(f8_decode<FMT>((w[i] >> 8) & 0xFFu)) >> 16;
+    const uint32_t b2 = __float_as_uint(f8_decode<FMT>((w[i] >> 16) & 0xFFu)) >> 16;
+    const uint32_t b3 = __float_as_uint(f8_decode<FMT>(w[i] >> 24)) >> 16;
+    o[2 * i] = b0 | (b1 << 16);
+    o[2 * i + 1] = b2 | (b3 << 16);
+  }
+  uint4* dst = reinterpret_cast<uint4*>(out) + 2 * t;
+  dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+// out[c*ld_out + r] = bf16(in[r*cols + c]); 32 x 32 tiles.
+template <int DT>
+__global__ void __launch_bounds__(256)
+to_bf16_transpose_kernel(const void* __restrict__ in, int64_t rows, int64_t cols, uint16_t* __restrict__ out,
+                         int64_t ld_out) {
+  __shared__ uint16_t tile[32][33];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;
+  for (int i = ty; i < 32; i += 8) {
+    const int64_t r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? (uint16_t)float_to_bf16_bits(load1<DT>(in, (size_t)r * cols + c)) : 0;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) {
+    const int64_t c = c0 + i, r = r0 + tx;
+    if (c < cols && r < ld_out) out[(size_t)c * ld_out + r] = r < rows ? tile[tx][i] : 0;
+  }
+}
+
+static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
+
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+size_t bsp_linear_wgrad_workspace_bytes(int64_t T, int64_t O, int64_t C, int x_read) {
+  (void)C;
+  if (T <= 0 || O <= 0) return 0;
+  if (x_read != BSP_READ_ORIGINAL) return 256;
+  return round_up((size_t)O * round_up((size_t)T, 16) * 2, 256);
+}
+
+int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy, int x_read,
+                     const void* x_t, bsp_quant_t q_x, int64_t ld_t, float* dW, const float* mc_ref, float* mc_S1,
+                     float* mc_S2, void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream) {
+  if (T < 0 || O < 0 || C < 0 || !valid_enum(x_read, 2) || !valid_enum(q_dy.fmt, 1) || !valid_enum(q_x.fmt, 1))
+    return BSP_ERR_ARG;
+  if (O == 0 || C == 0) return BSP_OK;
+  const bool mc = mc_ref != nullptr;
+  if (mc ? (!mc_S1 || !mc_S2) : !dW) return BSP_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (T == 0) {
+    if (!mc) BSP_CHECK_CUDA(cudaMemsetAsync(dW, 0, (size_t)O * C * sizeof(float), st));
+    return BSP_OK;
+  }
+  if (!dy_codes_t || !x_t) return BSP_ERR_ARG;
+  if (ld_t < T || ld_t % 16 != 0 || C % 4 != 0) return BSP_ERR_ALIGN;
+  GemmArgs g;
+  g.M = O; g.N = C; g.K = T; g.nb = 1;
+  g.lda = ld_t; g.ldb = ld_t; g.b_batch_stride = (int64_t)C * ld_t;
+  g.sa = q_dy.scale; g.sa_dev = q_dy.scale_dev; g.sb = q_x.scale; g.sb_dev = q_x.scale_dev;
+  g.mode = mc ? EPI_MC : EPI_STORE_F32;
+  g.C = dW; g.ldc = C; g.ref = mc_ref; g.S1 = mc_S1; g.S2 = mc_S2; g.diag = diag;
+  if (x_read == BSP_READ_ORIGINAL) {
+    // BF16 contraction: decode dY's codes to bf16 (exact) into the workspace; x_t is bf16 already
+    const size_t need = bsp_linear_wgrad_workspace_bytes(T, O, C, x_read);
+    if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return BSP_ERR_WORKSPACE;
+    const size_t n16 = (size_t)O * ld_t / 16;
+    uint16_t* dyb = reinterpret_cast<uint16_t*>(ws);
+    if (q_dy.fmt == BSP_E5M2)
+      decode_to_bf16_kernel<BSP_E5M2><<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(dy_codes_t, n16, dyb);
+    else
+      decode_to_bf16_kernel<BSP_E4M3><<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(dy_codes_t, n16, dyb);
+    BSP_LAUNCH_CHECK();
+    g.fp8 = false; g.A = dyb; g.B = x_t; g.a_fmt = 0; g.b_fmt = 0;
+    g.sb = 1.0f; g.sb_dev = nullptr;          // the original is unscaled
+  } else {
+    g.fp8 = true; g.A = dy_codes_t; g.B = x_t; g.a_fmt = q_dy.fmt; g.b_fmt = q_x.fmt;
+  }
+  return gemm_run(g, st);
+}
+
+size_t bsp_linear_dgrad_workspace_bytes(int64_t T, int64_t O, int64_t C) {
+  if (T <= 0 || O <= 0 || C <= 0) return 0;
+  const size_t ldo = round_up((size_t)O, 16);
+  return round_up((size_t)T * ldo * 2, 256) + round_up((size_t)C * ldo * 2, 256);
+}
+
+int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, bsp_quant_t q_dy, const void* W,
+                     int w_dt, void* du, int du_dt, void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream) {
+  if (T < 0 || O <= 0 || C < 0 || !valid_enum(q_dy.fmt, 1) || !valid_enum(w_dt, 1) || !valid_enum(du_dt, 1))
+    return BSP_ERR_ARG;
+  if (T == 0 || C == 0) return BSP_OK;
+  if (!dy_codes || !W || !du) return BSP_ERR_ARG;
+  if (O % 16 != 0 || C % 4 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < bsp_linear_dgrad_workspace_bytes(T, O, C) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  uint16_t* dyb = reinterpret_cast<uint16_t*>(ws);
+  uint16_t* wt = reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(ws) + round_up((size_t)T * O * 2, 256));
+  const size_t n16 = (size_t)T * O / 16;
+  if (q_dy.fmt == BSP_E5M2)
+    decode_to_bf16_kernel<BSP_E5M2><<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(dy_codes, n16, dyb);
+  else
+    decode_to_bf16_kernel<BSP_E4M3><<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(dy_codes, n16, dyb);
+  BSP_LAUNCH_CHECK();
+  dim3 tg((unsigned)((C + 31) / 32), (unsigned)((O + 31) / 32));
+  if (w_dt == BSP_F32) to_bf16_transpose_kernel<BSP_F32><<<tg, 256, 0, st>>>(W, O, C, wt, O);
+  else to_bf16_transpose_kernel<BSP_BF16><<<tg, 256, 0, st>>>(W, O, C, wt, O);
+  BSP_LAUNCH_CHECK();
+  GemmArgs g;
+  g.M = T; g.N = C; g.K = O; g.nb = 1; g.fp8 = false; g.a_fmt = 0; g.b_fmt = 0;
+  g.A = dyb; g.B = wt; g.lda = O; g.ldb = O; g.b_batch_stride = (int64_t)C * O;
+  g.sa = q_dy.scale; g.sa_dev = q_dy.scale_dev; g.sb = 1.0f; g.sb_dev = nullptr;
+  g.mode = du_dt == BSP_F32 ? EPI_STORE_F32 : EPI_STORE_BF16;
+  g.C = du; g.ldc = C; g.ref = nullptr; g.S1 = nullptr; g.S2 = nullptr; g.diag = diag;
+  return gemm_run(g, st);
+}
+
+}  // extern "C"

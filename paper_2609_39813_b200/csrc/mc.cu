@@ -1,0 +1,317 @@
+// Monte-Carlo statistics and the host-side orchestration of the per-use check.
+#include <math.h>
+#include <string.h>
+
+#include <atomic>
+
+#include "common.cuh"
+
+namespace bsp {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+constexpr int kStatBlocks = 592;     // 4 per SM
+constexpr int kStatFields = 8;       // err2, ref2, se2, z2, z, max|z|, count(|z|>3), unused
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_max_d(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+
+// Per element: err = mean - g*; fresh: mean - g* = S1/K, M2 = S2 - S1^2/K, se^2 = M2/(K-1)/K,
+// z = err/se (0 when both vanish).  Block partials in double, summed on the host in block order.
+__global__ void __launch_bounds__(256)
+mc_stats_kernel(const float* __restrict__ g_ref, const float* __restrict__ g, const float* __restrict__ S2,
+                int64_t n, int K, int fresh, double* __restrict__ partials) {
+  double err2 = 0, ref2 = 0, se2s = 0, z2 = 0, zs = 0, zmax = 0, cnt = 0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const double r = (double)g_ref[i];
+    ref2 += r * r;
+    if (!fresh) {
+      const double e = (double)g[i] - r;
+      err2 += e * e;
+    } else {
+      const double s1 = (double)g[i], s2 = (double)S2[i];
+      const double e = s1 / K;
+      double m2 = s2 - s1 * s1 / K;
+      if (m2 < 0) m2 = 0;
+      const double se2 = m2 / (K - 1) / K;
+      const double se = sqrt(se2);
+      const double z = (e == 0.0 && se == 0.0) ? 0.0 : e / se;
+      err2 += e * e;
+      se2s += se2;
+      z2 += z * z;
+      zs += z;
+      zmax = fmax(zmax, fabs(z));
+      cnt += fabs(z) > 3.0 ? 1.0 : 0.0;
+    }
+  }
+  __shared__ double sm[8][kStatFields];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  err2 = warp_sum_d(err2); ref2 = warp_sum_d(ref2); se2s = warp_sum_d(se2s); z2 = warp_sum_d(z2);
+  zs = warp_sum_d(zs); zmax = warp_max_d(zmax); cnt = warp_sum_d(cnt);
+  if (lane == 0) {
+    sm[warp][0] = err2; sm[warp][1] = ref2; sm[warp][2] = se2s; sm[warp][3] = z2;
+    sm[warp][4] = zs; sm[warp][5] = zmax; sm[warp][6] = cnt; sm[warp][7] = 0;
+  }
+  __syncthreads();
+  if (threadIdx.x < kStatFields) {
+    double a = 0;
+    for (int w = 0; w < 8; ++w) a = threadIdx.x == 5 ? fmax(a, sm[w][5]) : a + sm[w][threadIdx.x];
+    partials[(size_t)blockIdx.x * kStatFields + threadIdx.x] = a;
+  }
+}
+
+struct Bump {
+  char* base;
+  size_t off;
+  void* take(size_t bytes) {
+    void* p = base ? base + off : nullptr;
+    off += round_up(bytes ? bytes : 1, 256);
+    return p;
+  }
+};
+
+struct CheckBuffers {
+  float *rstd, *mean, *amax_u, *scale_u, *amax_dy, *scale_dy;
+  uint8_t *u_codes, *u_codes_t, *fresh_t, *dy_codes, *dy_codes_t;
+  uint16_t* u_bf16_t;
+  void* du;
+  float *dg_ref, *db_ref, *dg_pol, *S1g, *S2g, *dx;
+  float *dW_ref, *dW_pol, *S2w;
+  void *ws_bwd, *ws_gain, *ws_wgrad, *ws_dgrad, *ws_stats;
+  size_t b_bwd, b_gain, b_wgrad, b_dgrad, b_stats;
+  int64_t ld_t;
+};
+
+static size_t carve(const bsp_norm_linear_desc_t* op, int K, char* base, CheckBuffers* cb) {
+  Bump b{base, 0};
+  const size_t T = (size_t)op->T, C = (size_t)op->C, O = (size_t)op->O;
+  const size_t ld_t = round_up(T, 16);
+  const size_t eb = op->dtype == BSP_BF16 ? 2 : 4;
+  CheckBuffers c;
+  memset(&c, 0, sizeof(c));
+  c.ld_t = (int64_t)ld_t;
+  c.rstd = (float*)b.take(T * 4); c.mean = (float*)b.take(T * 4);
+  c.amax_u = (float*)b.take(4); c.scale_u = (float*)b.take(4);
+  c.amax_dy = (float*)b.take(4); c.scale_dy = (float*)b.take(4);
+  c.u_codes = (uint8_t*)b.take(T * C); c.u_codes_t = (uint8_t*)b.take(C * ld_t);
+  c.fresh_t = (uint8_t*)b.take(C * ld_t);
+  c.dy_codes = (uint8_t*)b.take(T * O); c.dy_codes_t = (uint8_t*)b.take(O * ld_t);
+  c.u_bf16_t = (uint16_t*)b.take(C * ld_t * 2);
+  c.du = b.take(T * C * eb);
+  c.dg_ref = (float*)b.take(C * 4); c.db_ref = (float*)b.take(C * 4); c.dg_pol = (float*)b.take(C * 4);
+  c.S1g = (float*)b.take(C * 4); c.S2g = (float*)b.take(C * 4);
+  c.dx = (float*)b.take(T * C * 4);
+  c.dW_ref = (float*)b.take(O * C * 4); c.dW_pol = (float*)b.take(O * C * 4); c.S2w = (float*)b.take(O * C * 4);
+  c.b_bwd = bsp_norm_bwd_workspace_bytes(op->T, op->C);
+  c.b_gain = bsp_norm_gain_mc_workspace_bytes(op->T, op->C, K > 0 ? K : 1);
+  c.b_wgrad = bsp_linear_wgrad_workspace_bytes(op->T, op->O, op->C, BSP_READ_ORIGINAL);
+  c.b_dgrad = bsp_linear_dgrad_workspace_bytes(op->T, op->O, op->C);
+  c.b_stats = bsp_mc_stats_workspace_bytes((int64_t)(O * C > C ? O * C : C));
+  c.ws_bwd = b.take(c.b_bwd); c.ws_gain = b.take(c.b_gain); c.ws_wgrad = b.take(c.b_wgrad);
+  c.ws_dgrad = b.take(c.b_dgrad); c.ws_stats = b.take(c.b_stats);
+  if (cb) *cb = c;
+  return b.off;
+}
+
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+const char* bsp_status_string(int status) {
+  switch (status) {
+    case BSP_OK: return "ok";
+    case BSP_ERR_ARG: return "invalid argument";
+    case BSP_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+    case BSP_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case BSP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case BSP_ERR_NONFINITE: return "non-finite value met in an input";
+    case BSP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case BSP_ERR_CUDA: return "CUDA runtime or driver call failed";
+    default: return "unknown status";
+  }
+}
+
+unsigned long long bsp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t bsp_mc_stats_workspace_bytes(int64_t n) {
+  (void)n;
+  return round_up((size_t)kStatBlocks * kStatFields * sizeof(double), 256);
+}
+
+int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
+                 bsp_use_result_t* result, void* ws, size_t ws_bytes, void* stream) {
+  if (!g_ref || !g || !result || n < 0 || (fresh && (!S2 || K < 2))) return BSP_ERR_ARG;
+  if (!ws || ws_bytes < bsp_mc_stats_workspace_bytes(n) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  double* partials = reinterpret_cast<double*>(ws);
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > kStatBlocks) blocks = kStatBlocks;
+  double host[kStatBlocks * kStatFields];
+  double f[kStatFields] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (blocks > 0) {
+    mc_stats_kernel<<<blocks, 256, 0, st>>>(g_ref, g, S2, n, K, fresh, partials);
+    BSP_LAUNCH_CHECK();
+    BSP_CHECK_CUDA(cudaMemcpyAsync(host, partials, (size_t)blocks * kStatFields * sizeof(double),
+                                   cudaMemcpyDeviceToHost, st));
+  }
+  BSP_CHECK_CUDA(cudaStreamSynchronize(st));
+  for (int b = 0; b < blocks; ++b)
+    for (int j = 0; j < kStatFields; ++j)
+      f[j] = j == 5 ? fmax(f[j], host[b * kStatFields + j]) : f[j] + host[b * kStatFields + j];
+  const double num = sqrt(f[0]), den = sqrt(f[1]);
+  result->n_elements = n;
+  result->rel_l2_mean_err = num == 0.0 ? 0.0 : (den > 0.0 ? num / den : INFINITY);
+  result->reserved = 0;
+  if (!fresh) {
+    result->K = 1;
+    result->R = result->Qprime = result->mean_z = result->rms_z = result->max_abs_z = result->frac_abs_z_gt3 = 0.0;
+    result->verdict = result->rel_l2_mean_err <= 1e-4 ? BSP_HOLDS : BSP_FAILS;
+    return BSP_OK;
+  }
+  const double nn = n > 0 ? (double)n : 1.0;
+  result->K = K;
+  result->R = f[0] == 0.0 ? 0.0 : (f[2] > 0.0 ? f[0] / f[2] : INFINITY);
+  result->Qprime = f[3] / nn * (double)(K - 3) / (double)(K - 1);
+  result->mean_z = f[4] / nn;
+  result->rms_z = sqrt(f[3] / nn);
+  result->max_abs_z = f[5];
+  result->frac_abs_z_gt3 = f[6] / nn;
+  if (result->Qprime >= 4.0 || result->R >= 6.0) result->verdict = BSP_FAILS;
+  else if (result->Qprime <= 2.0 && result->R <= 3.0) result->verdict = BSP_HOLDS;
+  else result->verdict = BSP_UNDECIDED;
+  return BSP_OK;
+}
+
+size_t bsp_mc_check_workspace_bytes(const bsp_norm_linear_desc_t* op, int K) {
+  if (!op || op->T <= 0 || op->C <= 0 || op->O <= 0) return 0;
+  return carve(op, K, nullptr, nullptr);
+}
+
+#define BSP_TRY(expr)            \
+  do {                           \
+    int _rc = (expr);            \
+    if (_rc != BSP_OK) return _rc; \
+  } while (0)
+
+int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* results, int* n_results, void* ws,
+                 size_t ws_bytes, bsp_diag_t* diag, void* stream) {
+  if (!op || !results || !n_results) return BSP_ERR_ARG;
+  if (op->T <= 0 || op->C <= 0 || op->O <= 0 || K < 2) return BSP_ERR_ARG;
+  if (!op->x || !op->gamma || !op->W || !op->dY || (op->norm_kind == BSP_LAYERNORM && !op->beta)) return BSP_ERR_ARG;
+  if (op->norm_kind < 0 || op->norm_kind > 1 || op->dtype < 0 || op->dtype > 1) return BSP_ERR_ARG;
+  if (op->C % 16 != 0 || op->O % 16 != 0 || op->C > 8192) return BSP_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < bsp_mc_check_workspace_bytes(op, K) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  CheckBuffers b;
+  carve(op, K, reinterpret_cast<char*>(ws), &b);
+  const int64_t T = op->T, C = op->C, O = op->O;
+  const int dt = op->dtype;
+  *n_results = 0;
+
+  // ---- once per call: statistics, scale, forward store, incoming gradient, du
+  BSP_TRY(bsp_norm_stats(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, op->eps, b.rstd, b.mean, b.amax_u,
+                         diag, st));
+  BSP_TRY(bsp_scale_from_amax(b.amax_u, 1, op->store_fmt, b.scale_u, st));
+  bsp_quant_t qu;
+  qu.fmt = op->store_fmt; qu.mode = op->forward_mode; qu.scale = 1.f; qu.scale_dev = b.scale_u;
+  bsp_key_t key;
+  key.seed = op->seed; key.tensor_id = op->tensor_id; key.stream = BSP_STREAM_FORWARD; key.draw = 0; key.reserved = 0;
+  const bool want_wu = (op->policy_mask >> 3) & 1u;
+  BSP_TRY(bsp_norm_fwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qu, key, b.u_codes,
+                       b.u_codes_t, b.ld_t, nullptr, want_wu ? b.u_bf16_t : nullptr, diag, st));
+  BSP_TRY(bsp_amax(op->dY, dt, 1, (size_t)T * O, b.amax_dy, diag, st));
+  BSP_TRY(bsp_scale_from_amax(b.amax_dy, 1, op->grad_fmt, b.scale_dy, st));
+  bsp_quant_t qdy;
+  qdy.fmt = op->grad_fmt; qdy.mode = BSP_ROUND_NEAREST; qdy.scale = 1.f; qdy.scale_dev = b.scale_dy;
+  bsp_key_t nokey;
+  memset(&nokey, 0, sizeof(nokey));
+  BSP_TRY(bsp_round_2d(op->dY, dt, T, O, qdy, nokey, b.dy_codes, b.dy_codes_t, b.ld_t, diag, st));
+  BSP_TRY(bsp_linear_dgrad(T, O, C, b.dy_codes, qdy, op->W, dt, b.du, dt, b.ws_dgrad, b.b_dgrad, diag, st));
+
+  int nres = 0;
+  auto emit = [&](int use, int out, int pol) -> bsp_use_result_t* {
+    bsp_use_result_t* r = &results[nres++];
+    memset(r, 0, sizeof(*r));
+    r->use_id = use; r->output_id = out; r->policy = pol;
+    return r;
+  };
+
+  // ---- gain use (reference: the original)
+  const uint32_t gain_mask = op->policy_mask & 7u;
+  if (gain_mask) {
+    key.stream = BSP_STREAM_GAIN;
+    BSP_TRY(bsp_norm_bwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt,
+                         BSP_READ_ORIGINAL, nullptr, qu, key, b.dg_ref, b.db_ref, b.dx, b.ws_bwd, b.b_bwd, diag, st));
+    if (gain_mask & 1u) {
+      bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_ORIGINAL);
+      BSP_TRY(bsp_mc_stats(b.dg_ref, b.dg_ref, nullptr, C, 1, 0, r, b.ws_stats, b.b_stats, st));
+    }
+    if (gain_mask & 2u) {
+      BSP_TRY(bsp_norm_bwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt,
+                           BSP_READ_FORWARD, b.u_codes, qu, key, b.dg_pol, nullptr, nullptr, b.ws_bwd, b.b_bwd,
+                           diag, st));
+      bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FORWARD);
+      BSP_TRY(bsp_mc_stats(b.dg_ref, b.dg_pol, nullptr, C, 1, 0, r, b.ws_stats, b.b_stats, st));
+    }
+    if (gain_mask & 4u) {
+      BSP_CHECK_CUDA(cudaMemsetAsync(b.S1g, 0, C * sizeof(float), st));
+      BSP_CHECK_CUDA(cudaMemsetAsync(b.S2g, 0, C * sizeof(float), st));
+      BSP_TRY(bsp_norm_gain_mc(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt, qu,
+                               key, 0, K, b.dg_ref, b.S1g, b.S2g, b.ws_gain, b.b_gain, diag, st));
+      bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FRESH);
+      BSP_TRY(bsp_mc_stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, r, b.ws_stats, b.b_stats, st));
+    }
+  }
+
+  // ---- weight use (reference: the rounded value the layer multiplied)
+  const uint32_t w_mask = (op->policy_mask >> 3) & 7u;
+  if (w_mask) {
+    BSP_TRY(bsp_linear_wgrad(T, O, C, b.dy_codes_t, qdy, BSP_READ_FORWARD, b.u_codes_t, qu, b.ld_t, b.dW_ref, nullptr,
+                             nullptr, nullptr, b.ws_wgrad, b.b_wgrad, diag, st));
+    if (w_mask & 1u) {
+      BSP_TRY(bsp_linear_wgrad(T, O, C, b.dy_codes_t, qdy, BSP_READ_ORIGINAL, b.u_bf16_t, qu, b.ld_t, b.dW_pol,
+                               nullptr, nullptr, nullptr, b.ws_wgrad, b.b_wgrad, diag, st));
+      bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_ORIGINAL);
+      BSP_TRY(bsp_mc_stats(b.dW_ref, b.dW_pol, nullptr, O * C, 1, 0, r, b.ws_stats, b.b_stats, st));
+    }
+    if (w_mask & 2u) {
+      bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FORWARD);
+      BSP_TRY(bsp_mc_stats(b.dW_ref, b.dW_ref, nullptr, O * C, 1, 0, r, b.ws_stats, b.b_stats, st));
+    }
+    if (w_mask & 4u) {
+      float* S1w = b.dW_pol;   // the U result has been reduced already
+      BSP_CHECK_CUDA(cudaMemsetAsync(S1w, 0, (size_t)O * C * sizeof(float), st));
+      BSP_CHECK_CUDA(cudaMemsetAsync(b.S2w, 0, (size_t)O * C * sizeof(float), st));
+      bsp_quant_t qf = qu;
+      qf.mode = BSP_ROUND_STOCHASTIC;
+      key.stream = BSP_STREAM_WGRAD;
+      for (int k = 0; k < K; ++k) {
+        key.draw = (uint32_t)k;
+        BSP_TRY(bsp_norm_fwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qf, key, nullptr,
+                             b.fresh_t, b.ld_t, nullptr, nullptr, nullptr, st));
+        BSP_TRY(bsp_linear_wgrad(T, O, C, b.dy_codes_t, qdy, BSP_READ_FRESH, b.fresh_t, qf, b.ld_t, nullptr, b.dW_ref,
+                                 S1w, b.S2w, b.ws_wgrad, b.b_wgrad, diag, st));
+      }
+      bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FRESH);
+      BSP_TRY(bsp_mc_stats(b.dW_ref, S1w, b.S2w, O * C, K, 1, r, b.ws_stats, b.b_stats, st));
+    }
+  }
+  *n_results = nres;
+  BSP_CHECK_CUDA(cudaStreamSynchronize(st));
+  return BSP_OK;
+}
+
+}  // extern "C"

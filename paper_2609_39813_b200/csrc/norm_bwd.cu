@@ -1,0 +1,443 @@
+// Normalisation backward under a per-use read policy, and the K-draw gain-use Monte-Carlo pass.
+//
+// norm_bwd_kernel: one row per block iteration; x and du are read once, dx is written once, the
+// column sums for dgamma / dbeta are kept in registers across the block's rows and reduced over
+// blocks by a second, deterministic kernel.  HBM-bound.
+// gain_mc_kernel: x and du are read once for all K draws; every draw costs one Philox block and
+// four stochastic roundings per four elements, all in registers.  ALU-bound.
+#include "common.cuh"
+
+namespace bsp {
+
+// Value of the stochastic rounding of v (scaled FP32 value) as FP32, i.e. decode(encode_SR(v)).
+template <int FMT>
+__device__ __forceinline__ float sr_value(float v, uint32_t U) {
+  using F = F8<FMT>;
+  const uint32_t b = __float_as_uint(v);
+  const uint32_t a = b & 0x7FFFFFFFu;
+  const int E = (int)(a >> 23) - 127;
+  if (a < F::FMAX_BITS && E >= F::EMIN) {
+    constexpr int d = 23 - F::MB;
+    const uint32_t rem = a & ((1u << d) - 1u);
+    const uint32_t up = U < (rem << (32 - d));
+    return __uint_as_float((b & 0x80000000u) | ((a - rem) + (up << d)));
+  }
+  DiagCounters dc;
+  return f8_decode<FMT>(f8_encode<FMT, true>(v, U, dc));
+}
+
+// ------------------------------------------------------------------------------- norm backward
+
+template <int DT, int DU_DT, int FMT, int JMAX>
+__global__ void __launch_bounds__(256)
+norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
+                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
+                const void* __restrict__ du, int gain_read, const uint8_t* __restrict__ u_codes, float scale_val,
+                const float* __restrict__ scale_dev, PhiloxKey key, float* __restrict__ part_g,
+                float* __restrict__ part_b, float* __restrict__ dx) {
+  __shared__ float red[2][2][8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float scale = scale_dev ? __ldg(scale_dev) : scale_val;
+  const float inv_scale = __fdiv_rn(1.0f, scale);
+  const float invC = 1.0f / (float)C;
+
+  float4 g4[JMAX], b4[JMAX], accg[JMAX], accb[JMAX];
+#pragma unroll
+  for (int j = 0; j < JMAX; ++j) {
+    const int64_t c = 4 * ((int64_t)tid + 256 * j);
+    g4[j] = make_float4(1.f, 1.f, 1.f, 1.f);
+    b4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < C) {
+      g4[j] = __ldg(reinterpret_cast<const float4*>(gamma + c));
+      if (kind == BSP_LAYERNORM) b4[j] = __ldg(reinterpret_cast<const float4*>(beta + c));
+    }
+    accg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    accb[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+
+  int it = 0;
+  for (int64_t r = blockIdx.x; r < T; r += gridDim.x, ++it) {
+    const float rs = __ldg(rstd + r);
+    const float mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+    float4 z[JMAX], dz[JMAX], d4[JMAX];
+    float p1 = 0.f, p2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < JMAX; ++j) {
+      const int64_t c = 4 * ((int64_t)tid + 256 * j);
+      z[j] = dz[j] = d4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c < C) {
+        const size_t i0 = (size_t)r * C + c;
+        const float4 xv = load4<DT>(x, i0);
+        d4[j] = load4<DU_DT>(du, i0);
+        if (kind == BSP_RMSNORM) {
+          z[j] = make_float4(__fmul_rn(xv.x, rs), __fmul_rn(xv.y, rs), __fmul_rn(xv.z, rs), __fmul_rn(xv.w, rs));
+        } else {
+          z[j] = make_float4(__fmul_rn(__fsub_rn(xv.x, mu), rs), __fmul_rn(__fsub_rn(xv.y, mu), rs),
+                             __fmul_rn(__fsub_rn(xv.z, mu), rs), __fmul_rn(__fsub_rn(xv.w, mu), rs));
+        }
+        dz[j] = make_float4(g4[j].x * d4[j].x, g4[j].y * d4[j].y, g4[j].z * d4[j].z, g4[j].w * d4[j].w);
+        p1 += (dz[j].x * z[j].x + dz[j].y * z[j].y) + (dz[j].z * z[j].z + dz[j].w * z[j].w);
+        p2 += (dz[j].x + dz[j].y) + (dz[j].z + dz[j].w);
+
+        // ---- gain use: z_g under the policy
+        float4 zg = z[j];
+        if (gain_read != BSP_READ_ORIGINAL) {
+          float dec[4];
+          if (gain_read == BSP_READ_FORWARD) {
+            const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(u_codes + i0));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) dec[e] = f8_decode<FMT>((pk >> (8 * e)) & 0xFFu);
+          } else {
+            const uint4 w = philox_block(key, (uint64_t)i0 >> 2, key.c2);
+            const float u[4] = {z[j].x, z[j].y, z[j].z, z[j].w};
+            const float gg[4] = {g4[j].x, g4[j].y, g4[j].z, g4[j].w};
+            const float bb[4] = {b4[j].x, b4[j].y, b4[j].z, b4[j].w};
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float uu = __fmul_rn(u[e], gg[e]);
+              if (kind == BSP_LAYERNORM) uu = __fadd_rn(uu, bb[e]);
+              dec[e] = sr_value<FMT>(__fmul_rn(uu, scale), ww[e]);
+            }
+          }
+          zg.x = __fdiv_rn(__fsub_rn(__fmul_rn(dec[0], inv_scale), b4[j].x), g4[j].x);
+          zg.y = __fdiv_rn(__fsub_rn(__fmul_rn(dec[1], inv_scale), b4[j].y), g4[j].y);
+          zg.z = __fdiv_rn(__fsub_rn(__fmul_rn(dec[2], inv_scale), b4[j].z), g4[j].z);
+          zg.w = __fdiv_rn(__fsub_rn(__fmul_rn(dec[3], inv_scale), b4[j].w), g4[j].w);
+        }
+        accg[j].x = fmaf(zg.x, d4[j].x, accg[j].x); accg[j].y = fmaf(zg.y, d4[j].y, accg[j].y);
+        accg[j].z = fmaf(zg.z, d4[j].z, accg[j].z); accg[j].w = fmaf(zg.w, d4[j].w, accg[j].w);
+        accb[j].x += d4[j].x; accb[j].y += d4[j].y; accb[j].z += d4[j].z; accb[j].w += d4[j].w;
+      }
+    }
+    if (dx) {
+      const int buf = it & 1;
+      p1 = warp_sum(p1);
+      p2 = warp_sum(p2);
+      if (lane == 0) { red[buf][0][warp] = p1; red[buf][1][warp] = p2; }
+      __syncthreads();
+      float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) { s1 += red[buf][0][w]; s2 += red[buf][1][w]; }
+      const float m1 = s1 * invC;
+      const float m2 = kind == BSP_LAYERNORM ? s2 * invC : 0.f;
+#pragma unroll
+      for (int j = 0; j < JMAX; ++j) {
+        const int64_t c = 4 * ((int64_t)tid + 256 * j);
+        if (c < C) {
+          float4 o;
+          o.x = rs * ((dz[j].x - m2) - z[j].x * m1);
+          o.y = rs * ((dz[j].y - m2) - z[j].y * m1);
+          o.z = rs * ((dz[j].z - m2) - z[j].z * m1);
+          o.w = rs * ((dz[j].w - m2) - z[j].w * m1);
+          *reinterpret_cast<float4*>(dx + (size_t)r * C + c) = o;
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < JMAX; ++j) {
+    const int64_t c = 4 * ((int64_t)tid + 256 * j);
+    if (c < C) {
+      *reinterpret_cast<float4*>(part_g + (size_t)blockIdx.x * C + c) = accg[j];
+      if (part_b) *reinterpret_cast<float4*>(part_b + (size_t)blockIdx.x * C + c) = accb[j];
+    }
+  }
+}
+
+// out[c] = sum over nparts of part[p*C + c], in order.  grid: C/32 blocks of 256 = 8 x 32 threads.
+__global__ void __launch_bounds__(256)
+column_reduce_kernel(const float* __restrict__ part, int nparts, int64_t C, float* __restrict__ out) {
+  __shared__ float sm[8][33];
+  const int cl = threadIdx.x & 31, pl = threadIdx.x >> 5;
+  const int64_t c = (int64_t)blockIdx.x * 32 + cl;
+  float s = 0.f;
+  if (c < C)
+    for (int p = pl; p < nparts; p += 8) s += part[(size_t)p * C + c];
+  sm[pl][cl] = s;
+  __syncthreads();
+  if (pl == 0 && c < C) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += sm[w][cl];
+    out[c] = t;
+  }
+}
+
+// ------------------------------------------------------------------------------- gain-use Monte Carlo
+
+constexpr int kMcRows = 8;              // rows per thread
+constexpr int kMcSlab = 8 * kMcRows;    // rows per block (8 warps)
+constexpr int kMcCols = 128;            // columns per block (32 lanes x 4)
+constexpr int kMcChunk = 64;            // draws per launch
+
+template <int DT, int DU_DT, int FMT>
+__global__ void __launch_bounds__(256)
+gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
+               const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
+               const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
+               int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */) {
+  __shared__ __align__(16) float red[2][8][kMcCols];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t c = (int64_t)blockIdx.x * kMcCols + lane * 4;
+  const int64_t slab = blockIdx.y, nslabs = gridDim.y;
+  const float scale = scale_dev ? __ldg(scale_dev) : scale_val;
+  const float inv_scale = __fdiv_rn(1.0f, scale);
+  const bool col_ok = c < C;
+
+  float4 g4 = make_float4(1.f, 1.f, 1.f, 1.f), b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (col_ok) {
+    g4 = __ldg(reinterpret_cast<const float4*>(gamma + c));
+    if (kind == BSP_LAYERNORM) b4 = __ldg(reinterpret_cast<const float4*>(beta + c));
+  }
+  float v[kMcRows][4], wgt[kMcRows][4];
+  uint64_t q[kMcRows];
+#pragma unroll
+  for (int i = 0; i < kMcRows; ++i) {
+    const int64_t r = slab * kMcSlab + warp + 8 * i;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { v[i][e] = 0.f; wgt[i][e] = 0.f; }
+    q[i] = 0;
+    if (r < T && col_ok) {
+      const size_t i0 = (size_t)r * C + c;
+      q[i] = (uint64_t)i0 >> 2;
+      const float4 xv = load4<DT>(x, i0);
+      const float4 dv = load4<DU_DT>(du, i0);
+      const float rs = __ldg(rstd + r);
+      const float mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+      const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
+      const float ds[4] = {dv.x, dv.y, dv.z, dv.w};
+      const float gg[4] = {g4.x, g4.y, g4.z, g4.w};
+      const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float u;
+        if (kind == BSP_RMSNORM) u = __fmul_rn(__fmul_rn(xs[e], rs), gg[e]);
+        else u = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xs[e], mu), rs), gg[e]), bb[e]);
+        v[i][e] = __fmul_rn(u, scale);
+        wgt[i][e] = __fdiv_rn(ds[e], gg[e]);
+      }
+    }
+  }
+  const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+  for (int k = 0; k < ndraws; ++k) {
+    const uint32_t draw = (uint32_t)(draw_begin + k);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < kMcRows; ++i) {
+      const uint4 w = philox_block(key, q[i], draw);
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float val = sr_value<FMT>(v[i][e], ww[e]);
+        acc[e] = fmaf(fmaf(val, inv_scale, -bb[e]), wgt[i][e], acc[e]);
+      }
+    }
+    const int buf = k & 1;
+    *reinterpret_cast<float4*>(&red[buf][warp][lane * 4]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    __syncthreads();
+    if (tid < kMcCols) {
+      float s = 0.f;
+#pragma unroll
+      for (int w8 = 0; w8 < 8; ++w8) s += red[buf][w8][tid];
+      const int64_t cc = (int64_t)blockIdx.x * kMcCols + tid;
+      if (cc < C) partial[((size_t)k * nslabs + slab) * C + cc] = s;
+    }
+  }
+}
+
+// gk[k*C + c] = sum over slabs of partial[k][slab][c] in a fixed order.
+__global__ void __launch_bounds__(256)
+gain_mc_slab_reduce_kernel(const float* __restrict__ partial, int nslabs, int64_t C, float* __restrict__ gk) {
+  __shared__ float sm[8][33];
+  const int cl = threadIdx.x & 31, pl = threadIdx.x >> 5;
+  const int64_t c = (int64_t)blockIdx.x * 32 + cl;
+  const size_t k = blockIdx.y;
+  float s = 0.f;
+  if (c < C)
+    for (int p = pl; p < nslabs; p += 8) s += partial[(k * nslabs + p) * C + c];
+  sm[pl][cl] = s;
+  __syncthreads();
+  if (pl == 0 && c < C) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += sm[w][cl];
+    gk[k * C + c] = t;
+  }
+}
+
+// S1[c] += sum_k (gk - ref), S2[c] += sum_k (gk - ref)^2.
+__global__ void gain_mc_accumulate_kernel(const float* __restrict__ gk, int ndraws, int64_t C,
+                                          const float* __restrict__ ref, float* __restrict__ S1,
+                                          float* __restrict__ S2) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const float g0 = ref[c];
+  float s1 = 0.f, s2 = 0.f;
+  for (int k = 0; k < ndraws; ++k) {
+    const float d = gk[(size_t)k * C + c] - g0;
+    s1 += d;
+    s2 = fmaf(d, d, s2);
+  }
+  S1[c] += s1;
+  S2[c] += s2;
+}
+
+static int bwd_grid(int64_t T) {
+  const int64_t want = (int64_t)kNumSMs * 4;
+  return (int)(T < want ? T : want);
+}
+
+template <int DT, int DU_DT, int FMT>
+static int launch_norm_bwd(int jmax, int grid, cudaStream_t st, int kind, const void* x, int64_t T, int64_t C,
+                           const float* gamma, const float* beta, const float* rstd, const float* mean,
+                           const void* du, int gain_read, const uint8_t* u_codes, bsp_quant_t q, PhiloxKey key,
+                           float* part_g, float* part_b, float* dx) {
+#define BSP_NB(J)                                                                                           \
+  norm_bwd_kernel<DT, DU_DT, FMT, J><<<grid, 256, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,      \
+                                                            gain_read, u_codes, q.scale, q.scale_dev, key,  \
+                                                            part_g, part_b, dx)
+  switch (jmax) {
+    case 1: BSP_NB(1); break;
+    case 2: BSP_NB(2); break;
+    case 4: BSP_NB(4); break;
+    default: BSP_NB(8); break;
+  }
+#undef BSP_NB
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
+
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+size_t bsp_norm_bwd_workspace_bytes(int64_t T, int64_t C) {
+  if (T <= 0 || C <= 0) return 0;
+  return round_up((size_t)bwd_grid(T) * (size_t)C * sizeof(float), 256) * 2;
+}
+
+int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
+                 const float* rstd, const float* mean, const void* du, int du_dt, int gain_read,
+                 const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key, float* dgamma, float* dbeta, float* dx,
+                 void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream) {
+  (void)diag;
+  if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(gain_read, 2) ||
+      !valid_enum(q.fmt, 1))
+    return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (T < 0 || C <= 0) return BSP_ERR_ARG;
+  if (!dgamma) return BSP_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (T == 0) {
+    BSP_CHECK_CUDA(cudaMemsetAsync(dgamma, 0, C * sizeof(float), st));
+    if (dbeta) BSP_CHECK_CUDA(cudaMemsetAsync(dbeta, 0, C * sizeof(float), st));
+    return BSP_OK;
+  }
+  if (!x || !gamma || !rstd || !du || (kind == BSP_LAYERNORM && (!beta || !mean))) return BSP_ERR_ARG;
+  if (gain_read == BSP_READ_FORWARD && !u_codes) return BSP_ERR_ARG;
+  if (C % 4 != 0 || C > 8192) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(du) || !aligned16(gamma) || !aligned16(beta) || !aligned16(dx) ||
+      (reinterpret_cast<uintptr_t>(u_codes) & 3u))
+    return BSP_ERR_ALIGN;
+  if (!ws || ws_bytes < bsp_norm_bwd_workspace_bytes(T, C) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  const int grid = bwd_grid(T);
+  float* part_g = reinterpret_cast<float*>(ws);
+  float* part_b = dbeta ? reinterpret_cast<float*>(reinterpret_cast<char*>(ws) +
+                                                   round_up((size_t)grid * C * sizeof(float), 256))
+                        : nullptr;
+  const int64_t groups = (C / 4 + 255) / 256;
+  const int jmax = groups <= 1 ? 1 : groups <= 2 ? 2 : groups <= 4 ? 4 : 8;
+  const PhiloxKey pk = make_key(key);
+  int rc;
+#define BSP_CALL(DT, DU, FMT)                                                                              \
+  rc = launch_norm_bwd<DT, DU, FMT>(jmax, grid, st, kind, x, T, C, gamma, beta, rstd, mean, du, gain_read, \
+                                    u_codes, q, pk, part_g, part_b, dx)
+  if (q.fmt == BSP_E4M3) {
+    if (dt == BSP_F32 && du_dt == BSP_F32) BSP_CALL(BSP_F32, BSP_F32, BSP_E4M3);
+    else if (dt == BSP_F32) BSP_CALL(BSP_F32, BSP_BF16, BSP_E4M3);
+    else if (du_dt == BSP_F32) BSP_CALL(BSP_BF16, BSP_F32, BSP_E4M3);
+    else BSP_CALL(BSP_BF16, BSP_BF16, BSP_E4M3);
+  } else {
+    if (dt == BSP_F32 && du_dt == BSP_F32) BSP_CALL(BSP_F32, BSP_F32, BSP_E5M2);
+    else if (dt == BSP_F32) BSP_CALL(BSP_F32, BSP_BF16, BSP_E5M2);
+    else if (du_dt == BSP_F32) BSP_CALL(BSP_BF16, BSP_F32, BSP_E5M2);
+    else BSP_CALL(BSP_BF16, BSP_BF16, BSP_E5M2);
+  }
+#undef BSP_CALL
+  if (rc != BSP_OK) return rc;
+  const unsigned rb = (unsigned)((C + 31) / 32);
+  column_reduce_kernel<<<rb, 256, 0, st>>>(part_g, grid, C, dgamma);
+  BSP_LAUNCH_CHECK();
+  if (dbeta) {
+    column_reduce_kernel<<<rb, 256, 0, st>>>(part_b, grid, C, dbeta);
+    BSP_LAUNCH_CHECK();
+  }
+  return BSP_OK;
+}
+
+size_t bsp_norm_gain_mc_workspace_bytes(int64_t T, int64_t C, int K) {
+  if (T <= 0 || C <= 0 || K <= 0) return 0;
+  const size_t nslabs = (size_t)((T + kMcSlab - 1) / kMcSlab);
+  const size_t kc = (size_t)(K < kMcChunk ? K : kMcChunk);
+  return round_up(kc * nslabs * (size_t)C * sizeof(float), 256) + round_up(kc * (size_t)C * sizeof(float), 256);
+}
+
+int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
+                     const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q, bsp_key_t key,
+                     int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
+                     bsp_diag_t* diag, void* stream) {
+  (void)diag;
+  if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(q.fmt, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (T < 0 || C <= 0 || K < 0 || draw0 < 0) return BSP_ERR_ARG;
+  if (!g_ref || !S1 || !S2) return BSP_ERR_ARG;
+  if (K == 0) return BSP_OK;
+  if (T > 0 && (!x || !gamma || !rstd || !du || (kind == BSP_LAYERNORM && (!beta || !mean)))) return BSP_ERR_ARG;
+  if (C % 4 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(du) || !aligned16(gamma) || !aligned16(beta)) return BSP_ERR_ALIGN;
+  if (!ws || ws_bytes < bsp_norm_gain_mc_workspace_bytes(T, C, K) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int nslabs = (int)((T + kMcSlab - 1) / kMcSlab);
+  const int kc_max = K < kMcChunk ? K : kMcChunk;
+  float* partial = reinterpret_cast<float*>(ws);
+  float* gk = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) +
+                                       round_up((size_t)kc_max * (nslabs > 0 ? nslabs : 1) * C * sizeof(float), 256));
+  const PhiloxKey pk = make_key(key);
+  for (int kb = 0; kb < K; kb += kMcChunk) {
+    const int nd = (K - kb) < kMcChunk ? (K - kb) : kMcChunk;
+    if (nslabs > 0) {
+      dim3 grid((unsigned)((C + kMcCols - 1) / kMcCols), (unsigned)nslabs);
+#define BSP_GM(DT, DU, FMT)                                                                                     \
+  gain_mc_kernel<DT, DU, FMT><<<grid, 256, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du, q.scale,        \
+                                                     q.scale_dev, pk, draw0 + kb, nd, partial)
+      if (q.fmt == BSP_E4M3) {
+        if (dt == BSP_F32 && du_dt == BSP_F32) BSP_GM(BSP_F32, BSP_F32, BSP_E4M3);
+        else if (dt == BSP_F32) BSP_GM(BSP_F32, BSP_BF16, BSP_E4M3);
+        else if (du_dt == BSP_F32) BSP_GM(BSP_BF16, BSP_F32, BSP_E4M3);
+        else BSP_GM(BSP_BF16, BSP_BF16, BSP_E4M3);
+      } else {
+        if (dt == BSP_F32 && du_dt == BSP_F32) BSP_GM(BSP_F32, BSP_F32, BSP_E5M2);
+        else if (dt == BSP_F32) BSP_GM(BSP_F32, BSP_BF16, BSP_E5M2);
+        else if (du_dt == BSP_F32) BSP_GM(BSP_BF16, BSP_F32, BSP_E5M2);
+        else BSP_GM(BSP_BF16, BSP_BF16, BSP_E5M2);
+      }
+#undef BSP_GM
+      BSP_LAUNCH_CHECK();
+    }
+    dim3 rgrid((unsigned)((C + 31) / 32), (unsigned)nd);
+    gain_mc_slab_reduce_kernel<<<rgrid, 256, 0, st>>>(partial, nslabs, C, gk);
+    BSP_LAUNCH_CHECK();
+    gain_mc_accumulate_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(gk, nd, C, g_ref, S1, S2);
+    BSP_LAUNCH_CHECK();
+  }
+  return BSP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,512 @@
+// Rounding kernels: raw generator words, group amax, scales, flat / grouped / 2-D rounding, and
+// the normalisation store's rounding pass (forward store and fresh re-rounding).
+//
+// All of these are streaming kernels: every element is read once and one byte is written, with
+// 128-bit loads and stores; stochastic rounding costs one Philox4x32-10 block per four elements.
+#include "common.cuh"
+
+namespace bsp {
+
+// ------------------------------------------------------------------------------- philox fill
+
+__global__ void philox_fill_kernel(PhiloxKey key, size_t n, uint32_t* __restrict__ out) {
+  const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t i = q * 4;
+  if (i >= n) return;
+  const uint4 w = philox_block(key, q, key.c2);
+  if (i + 4 <= n) {
+    reinterpret_cast<uint4*>(out)[q] = w;
+  } else {
+    for (uint32_t l = 0; i + l < n; ++l) out[i + l] = word_of(w, l);
+  }
+}
+
+// ------------------------------------------------------------------------------- amax
+
+template <int DT>
+__global__ void amax_kernel(const void* __restrict__ x, size_t group_size, uint32_t* __restrict__ amax_bits,
+                            bsp_diag_t* diag) {
+  // grid: (blocks_per_group, n_groups); amax_bits pre-cleared to 0.
+  const size_t g = blockIdx.y;
+  const size_t base = g * group_size;
+  float m = 0.f;
+  uint32_t nf = 0;
+  const size_t nvec = group_size / 4;
+  const bool vec_ok = ((base & 3) == 0);
+  if (vec_ok) {
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (size_t)gridDim.x * blockDim.x) {
+      const float4 f = load4<DT>(x, base + v * 4);
+      const float a[4] = {fabsf(f.x), fabsf(f.y), fabsf(f.z), fabsf(f.w)};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (a[j] <= 3.4028234663852886e38f) m = fmaxf(m, a[j]); else nf++;
+      }
+    }
+    for (size_t i = nvec * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < group_size;
+         i += (size_t)gridDim.x * blockDim.x) {
+      const float a = fabsf(load1<DT>(x, base + i));
+      if (a <= 3.4028234663852886e38f) m = fmaxf(m, a); else nf++;
+    }
+  } else {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < group_size; i += (size_t)gridDim.x * blockDim.x) {
+      const float a = fabsf(load1<DT>(x, base + i));
+      if (a <= 3.4028234663852886e38f) m = fmaxf(m, a); else nf++;
+    }
+  }
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0) atomicMax(&amax_bits[g], __float_as_uint(m));
+  DiagCounters dc; dc.nonfinite = nf;
+  diag_flush_warp(diag, dc);
+}
+
+__global__ void scale_from_amax_kernel(const float* __restrict__ amax, size_t n, int fmt, float* __restrict__ scale) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float a = amax[i];
+  const float fmax = fmt == BSP_E4M3 ? 448.f : 57344.f;
+  float s = 1.f;
+  if (a > 0.f && a <= 3.4028234663852886e38f) {
+    s = __fdiv_rn(fmax, a);
+    if (!(s <= 3.4028234663852886e38f)) s = 1.f;
+  }
+  scale[i] = s;
+}
+
+// ------------------------------------------------------------------------------- flat rounding
+
+// Encodes 16 consecutive values whose first element has logical index e0 (e0 % 4 == 0).
+template <int FMT, int MODE>
+__device__ __forceinline__ uint4 encode16(const float (&v)[16], const PhiloxKey& key, uint64_t e0, DiagCounters& dc) {
+  uint32_t packed[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    uint4 w = make_uint4(0, 0, 0, 0);
+    if (MODE == BSP_ROUND_STOCHASTIC) w = philox_block(key, (e0 >> 2) + b, key.c2);
+    const uint32_t c0 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 0], w.x, dc);
+    const uint32_t c1 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 1], w.y, dc);
+    const uint32_t c2 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 2], w.z, dc);
+    const uint32_t c3 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 3], w.w, dc);
+    packed[b] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+  }
+  return make_uint4(packed[0], packed[1], packed[2], packed[3]);
+}
+
+// One thread per 16 elements; group_size % 16 == 0 and elem_offset % 4 == 0 on this path.
+template <int DT, int FMT, int MODE>
+__global__ void __launch_bounds__(256)
+round_vec_kernel(const void* __restrict__ x, size_t n16, size_t group_size, float scale_val,
+                 const float* __restrict__ scales, PhiloxKey key, uint64_t elem_offset,
+                 uint8_t* __restrict__ codes, bsp_diag_t* diag) {
+  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  DiagCounters dc;
+  if (t < n16) {
+    const size_t i0 = t * 16;
+    const float s = scales ? __ldg(scales + (group_size ? i0 / group_size : 0)) : scale_val;
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 f = load4<DT>(x, i0 + 4 * j);
+      v[4 * j + 0] = __fmul_rn(f.x, s); v[4 * j + 1] = __fmul_rn(f.y, s);
+      v[4 * j + 2] = __fmul_rn(f.z, s); v[4 * j + 3] = __fmul_rn(f.w, s);
+    }
+    reinterpret_cast<uint4*>(codes)[t] = encode16<FMT, MODE>(v, key, elem_offset + i0, dc);
+  }
+  diag_flush_warp(diag, dc);
+}
+
+// General path: one thread per element (tails, odd group sizes, unaligned offsets).
+template <int DT, int FMT, int MODE>
+__global__ void round_scalar_kernel(const void* __restrict__ x, size_t i_begin, size_t n, size_t group_size,
+                                    float scale_val, const float* __restrict__ scales, PhiloxKey key,
+                                    uint64_t elem_offset, uint8_t* __restrict__ codes, bsp_diag_t* diag) {
+  const size_t i = i_begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  DiagCounters dc;
+  if (i < n) {
+    const float s = scales ? __ldg(scales + (group_size ? i / group_size : 0)) : scale_val;
+    const float v = __fmul_rn(load1<DT>(x, i), s);
+    uint32_t U = 0;
+    if (MODE == BSP_ROUND_STOCHASTIC) {
+      const uint64_t e = elem_offset + i;
+      U = word_of(philox_block(key, e >> 2, key.c2), (uint32_t)(e & 3));
+    }
+    codes[i] = (uint8_t)f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v, U, dc);
+  }
+  diag_flush_warp(diag, dc);
+}
+
+// ------------------------------------------------------------------------------- 2-D tile rounding
+
+// Produces the FP32 value *before scaling* of element (r, c) from the loaded input value.
+struct PlainProducer {
+  __device__ __forceinline__ void row(int64_t) {}
+  __device__ __forceinline__ float value(float xin, int64_t) const { return xin; }
+};
+
+struct NormProducer {
+  int kind;
+  const float* __restrict__ gamma;
+  const float* __restrict__ beta;
+  const float* __restrict__ rstd;
+  const float* __restrict__ mean;
+  float r_, m_;
+  __device__ __forceinline__ void row(int64_t r) {
+    r_ = __ldg(rstd + r);
+    m_ = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+  }
+  // RMS: fl(fl(x*rstd)*gamma).  LN: fl(fl(fl(fl(x-mean)*rstd)*gamma)+beta).
+  __device__ __forceinline__ float value(float xin, int64_t c) const {
+    if (kind == BSP_RMSNORM) return __fmul_rn(__fmul_rn(xin, r_), __ldg(gamma + c));
+    return __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xin, m_), r_), __ldg(gamma + c)), __ldg(beta + c));
+  }
+};
+
+constexpr int kTile = 64;   // 64 x 64 tile, 256 threads, 16 consecutive columns per thread
+
+// Requires cols % 16 == 0.  Outputs may each be NULL.
+template <class Producer, int DT, int FMT, int MODE>
+__global__ void __launch_bounds__(256)
+quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64_t cols, float scale_val,
+                  const float* __restrict__ scale_dev, PhiloxKey key, uint8_t* __restrict__ codes,
+                  uint8_t* __restrict__ codes_t, int64_t ld_t, float* __restrict__ u_f32,
+                  uint16_t* __restrict__ u_bf16_t, bsp_diag_t* diag) {
+  __shared__ __align__(16) uint8_t s_codes[kTile][kTile + 4];
+  __shared__ __align__(16) uint16_t s_bf16[kTile][kTile + 2];
+  const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
+  const int tr = threadIdx.x >> 2, tc = (threadIdx.x & 3) * 16;
+  const int64_t r = r0 + tr, c = c0 + tc;
+  const float s = scale_dev ? __ldg(scale_dev) : scale_val;
+  DiagCounters dc;
+  const bool active = (r < rows) && (c < cols);
+  if (active) {
+    prod.row(r);
+    const size_t i0 = (size_t)r * cols + c;
+    float u[16], v[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 f = load4<DT>(x, i0 + 4 * j);
+      u[4 * j + 0] = prod.value(f.x, c + 4 * j + 0); u[4 * j + 1] = prod.value(f.y, c + 4 * j + 1);
+      u[4 * j + 2] = prod.value(f.z, c + 4 * j + 2); u[4 * j + 3] = prod.value(f.w, c + 4 * j + 3);
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(u[j], s);
+    if (u_f32) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        reinterpret_cast<float4*>(u_f32 + i0)[j] = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
+    }
+    if (codes || codes_t) {
+      const uint4 pk = encode16<FMT, MODE>(v, key, (uint64_t)i0, dc);
+      if (codes) *reinterpret_cast<uint4*>(codes + i0) = pk;
+      if (codes_t) {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&s_codes[tr][tc]);
+        dst[0] = pk.x; dst[1] = pk.y; dst[2] = pk.z; dst[3] = pk.w;
+      }
+    }
+    if (u_bf16_t) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) s_bf16[tr][tc + j] = (uint16_t)float_to_bf16_bits(u[j]);
+    }
+  }
+  if (codes_t || u_bf16_t) {
+    __syncthreads();
+    // transposed write: thread -> column tcol, 16 consecutive rows
+    const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
+    const int64_t cc = c0 + tcol, rr = r0 + trow;
+    if (cc < cols && rr < rows) {
+      const int nvalid = (int)((rows - rr) < 16 ? (rows - rr) : 16);
+      if (codes_t) {
+        uint32_t pk[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t b = j < nvalid ? s_codes[trow + j][tcol] : 0u;
+          pk[j >> 2] |= b << (8 * (j & 3));
+        }
+        // ld_t is a multiple of 16 and >= rows rounded up, so the 16-byte store stays in the row
+        *reinterpret_cast<uint4*>(codes_t + (size_t)cc * ld_t + rr) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+      if (u_bf16_t) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t lo = (2 * j) < nvalid ? s_bf16[trow + 2 * j][tcol] : 0u;
+          const uint32_t hi = (2 * j + 1) < nvalid ? s_bf16[trow + 2 * j + 1][tcol] : 0u;
+          pk[j] = lo | (hi << 16);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(u_bf16_t + (size_t)cc * ld_t + rr);
+        dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+      }
+    }
+  }
+  diag_flush_warp(diag, dc);
+}
+
+// ------------------------------------------------------------------------------- norm statistics
+
+// One warp per row.  RMS: rstd = 1/sqrt(mean x^2 + eps).  LN: mean, biased variance.
+// Optionally the largest |u| with u from the same FP32 chain the rounding pass uses.
+template <int DT>
+__global__ void __launch_bounds__(256)
+norm_stats_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
+                  const float* __restrict__ beta, float eps, float* __restrict__ rstd, float* __restrict__ mean,
+                  uint32_t* __restrict__ amax_bits, bsp_diag_t* diag) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  float amax = 0.f;
+  uint32_t nf = 0;
+  if (row < T) {
+    const size_t base = (size_t)row * C;
+    const int64_t nvec = C / 4;
+    float mu = 0.f;
+    if (kind == BSP_LAYERNORM) {
+      float s = 0.f;
+      for (int64_t v = lane; v < nvec; v += 32) {
+        const float4 f = load4<DT>(x, base + v * 4);
+        s += (f.x + f.y) + (f.z + f.w);
+      }
+      mu = __fdiv_rn(warp_sum(s), (float)C);
+    }
+    float ss = 0.f;
+    for (int64_t v = lane; v < nvec; v += 32) {
+      const float4 f = load4<DT>(x, base + v * 4);
+      const float a = f.x - mu, b = f.y - mu, c = f.z - mu, d = f.w - mu;
+      ss += (a * a + b * b) + (c * c + d * d);
+      nf += !(fabsf(f.x) <= 3.4028234663852886e38f) + !(fabsf(f.y) <= 3.4028234663852886e38f) +
+            !(fabsf(f.z) <= 3.4028234663852886e38f) + !(fabsf(f.w) <= 3.4028234663852886e38f);
+    }
+    ss = warp_sum(ss);
+    const float rs = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, (float)C), eps)));
+    if (lane == 0) {
+      rstd[row] = rs;
+      if (mean && kind == BSP_LAYERNORM) mean[row] = mu;
+    }
+    if (amax_bits) {
+      for (int64_t v = lane; v < nvec; v += 32) {
+        const float4 f = load4<DT>(x, base + v * 4);
+        const float4 g = __ldg(reinterpret_cast<const float4*>(gamma) + v);
+        float u0, u1, u2, u3;
+        if (kind == BSP_RMSNORM) {
+          u0 = __fmul_rn(__fmul_rn(f.x, rs), g.x); u1 = __fmul_rn(__fmul_rn(f.y, rs), g.y);
+          u2 = __fmul_rn(__fmul_rn(f.z, rs), g.z); u3 = __fmul_rn(__fmul_rn(f.w, rs), g.w);
+        } else {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(beta) + v);
+          u0 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.x, mu), rs), g.x), b.x);
+          u1 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.y, mu), rs), g.y), b.y);
+          u2 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.z, mu), rs), g.z), b.z);
+          u3 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.w, mu), rs), g.w), b.w);
+        }
+        const float a[4] = {fabsf(u0), fabsf(u1), fabsf(u2), fabsf(u3)};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (a[j] <= 3.4028234663852886e38f) amax = fmaxf(amax, a[j]);
+      }
+    }
+  }
+  if (amax_bits) {
+    amax = warp_max(amax);
+    if (lane == 0 && amax > 0.f) atomicMax(amax_bits, __float_as_uint(amax));
+  }
+  DiagCounters dc; dc.nonfinite = nf;
+  diag_flush_warp(diag, dc);
+}
+
+// ------------------------------------------------------------------------------- dispatch helpers
+
+template <class Producer, int DT, int FMT>
+static void launch_tile_mode(int mode, dim3 grid, cudaStream_t st, Producer prod, const void* x, int64_t rows,
+                             int64_t cols, float scale, const float* scale_dev, PhiloxKey key, uint8_t* codes,
+                             uint8_t* codes_t, int64_t ld_t, float* u_f32, uint16_t* u_bf16_t, bsp_diag_t* diag) {
+  if (mode == BSP_ROUND_STOCHASTIC)
+    quant_tile_kernel<Producer, DT, FMT, BSP_ROUND_STOCHASTIC><<<grid, 256, 0, st>>>(
+        prod, x, rows, cols, scale, scale_dev, key, codes, codes_t, ld_t, u_f32, u_bf16_t, diag);
+  else
+    quant_tile_kernel<Producer, DT, FMT, BSP_ROUND_NEAREST><<<grid, 256, 0, st>>>(
+        prod, x, rows, cols, scale, scale_dev, key, codes, codes_t, ld_t, u_f32, u_bf16_t, diag);
+}
+
+template <class Producer>
+static int launch_tile(int dt, int fmt, int mode, cudaStream_t st, Producer prod, const void* x, int64_t rows,
+                       int64_t cols, float scale, const float* scale_dev, PhiloxKey key, uint8_t* codes,
+                       uint8_t* codes_t, int64_t ld_t, float* u_f32, uint16_t* u_bf16_t, bsp_diag_t* diag) {
+  dim3 grid((unsigned)((cols + kTile - 1) / kTile), (unsigned)((rows + kTile - 1) / kTile));
+#define BSP_TILE_CASE(DT, FMT)                                                                              \
+  launch_tile_mode<Producer, DT, FMT>(mode, grid, st, prod, x, rows, cols, scale, scale_dev, key, codes,   \
+                                      codes_t, ld_t, u_f32, u_bf16_t, diag)
+  if (dt == BSP_F32 && fmt == BSP_E4M3) BSP_TILE_CASE(BSP_F32, BSP_E4M3);
+  else if (dt == BSP_F32 && fmt == BSP_E5M2) BSP_TILE_CASE(BSP_F32, BSP_E5M2);
+  else if (dt == BSP_BF16 && fmt == BSP_E4M3) BSP_TILE_CASE(BSP_BF16, BSP_E4M3);
+  else BSP_TILE_CASE(BSP_BF16, BSP_E5M2);
+#undef BSP_TILE_CASE
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+template <int DT, int FMT, int MODE>
+static int launch_round_flat(const void* x, size_t n, size_t group_size, float scale, const float* scales,
+                             PhiloxKey key, uint64_t elem_offset, uint8_t* codes, bsp_diag_t* diag,
+                             cudaStream_t st) {
+  const bool vec_ok = (elem_offset % 4 == 0) && (group_size == 0 || group_size % 16 == 0);
+  size_t n16 = vec_ok ? n / 16 : 0;
+  if (n16) {
+    const unsigned blocks = (unsigned)((n16 + 255) / 256);
+    round_vec_kernel<DT, FMT, MODE><<<blocks, 256, 0, st>>>(x, n16, group_size, scale, scales, key, elem_offset,
+                                                           codes, diag);
+    BSP_LAUNCH_CHECK();
+  }
+  const size_t done = n16 * 16;
+  if (done < n) {
+    const unsigned blocks = (unsigned)((n - done + 255) / 256);
+    round_scalar_kernel<DT, FMT, MODE><<<blocks, 256, 0, st>>>(x, done, n, group_size, scale, scales, key,
+                                                              elem_offset, codes, diag);
+    BSP_LAUNCH_CHECK();
+  }
+  return BSP_OK;
+}
+
+static int dispatch_round_flat(int dt, int fmt, int mode, const void* x, size_t n, size_t group_size, float scale,
+                               const float* scales, PhiloxKey key, uint64_t elem_offset, uint8_t* codes,
+                               bsp_diag_t* diag, cudaStream_t st) {
+#define BSP_FLAT(DT, FMT, MODE) \
+  return launch_round_flat<DT, FMT, MODE>(x, n, group_size, scale, scales, key, elem_offset, codes, diag, st)
+  if (dt == BSP_F32) {
+    if (fmt == BSP_E4M3) { if (mode) BSP_FLAT(BSP_F32, BSP_E4M3, 1); else BSP_FLAT(BSP_F32, BSP_E4M3, 0); }
+    else { if (mode) BSP_FLAT(BSP_F32, BSP_E5M2, 1); else BSP_FLAT(BSP_F32, BSP_E5M2, 0); }
+  } else {
+    if (fmt == BSP_E4M3) { if (mode) BSP_FLAT(BSP_BF16, BSP_E4M3, 1); else BSP_FLAT(BSP_BF16, BSP_E4M3, 0); }
+    else { if (mode) BSP_FLAT(BSP_BF16, BSP_E5M2, 1); else BSP_FLAT(BSP_BF16, BSP_E5M2, 0); }
+  }
+#undef BSP_FLAT
+}
+
+static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
+
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+int bsp_diag_clear(bsp_diag_t* diag, void* stream) {
+  if (!diag) return BSP_ERR_ARG;
+  BSP_CHECK_CUDA(cudaMemsetAsync(diag, 0, sizeof(bsp_diag_t), (cudaStream_t)stream));
+  return BSP_OK;
+}
+
+int bsp_philox_fill(bsp_key_t key, size_t n, uint32_t* out, void* stream) {
+  if (!out && n) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (!aligned16(out)) return BSP_ERR_ALIGN;
+  if (n == 0) return BSP_OK;
+  const size_t nq = (n + 3) / 4;
+  philox_fill_kernel<<<(unsigned)((nq + 255) / 256), 256, 0, (cudaStream_t)stream>>>(make_key(key), n, out);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_amax(const void* x, int dt, size_t n_groups, size_t group_size, float* amax, bsp_diag_t* diag,
+             void* stream) {
+  if (!amax || !valid_enum(dt, 1)) return BSP_ERR_ARG;
+  if (n_groups == 0) return BSP_OK;
+  if (!x && group_size) return BSP_ERR_ARG;
+  if (!aligned16(x)) return BSP_ERR_ALIGN;
+  if (n_groups > 65535) return BSP_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  BSP_CHECK_CUDA(cudaMemsetAsync(amax, 0, n_groups * sizeof(float), st));
+  if (group_size == 0) return BSP_OK;
+  size_t per = (group_size / 4 + 255) / 256;
+  size_t want = (size_t)kNumSMs * 8 / n_groups + 1;
+  unsigned bx = (unsigned)(per < want ? (per ? per : 1) : want);
+  dim3 grid(bx, (unsigned)n_groups);
+  if (dt == BSP_F32) amax_kernel<BSP_F32><<<grid, 256, 0, st>>>(x, group_size, reinterpret_cast<uint32_t*>(amax), diag);
+  else amax_kernel<BSP_BF16><<<grid, 256, 0, st>>>(x, group_size, reinterpret_cast<uint32_t*>(amax), diag);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_scale_from_amax(const float* amax, size_t n, int fmt, float* scale, void* stream) {
+  if (!amax || !scale || !valid_enum(fmt, 1)) return BSP_ERR_ARG;
+  if (n == 0) return BSP_OK;
+  scale_from_amax_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(amax, n, fmt, scale);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_round(const void* x, int dt, size_t n, bsp_quant_t q, bsp_key_t key, uint64_t elem_offset,
+              uint8_t* codes, bsp_diag_t* diag, void* stream) {
+  if (!valid_enum(dt, 1) || !valid_enum(q.fmt, 1) || !valid_enum(q.mode, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (n == 0) return BSP_OK;
+  if (!x || !codes) return BSP_ERR_ARG;
+  if (!aligned16(x) || !aligned16(codes)) return BSP_ERR_ALIGN;
+  // a device scale is a scale array with group size 0: every element reads entry 0
+  return dispatch_round_flat(dt, q.fmt, q.mode, x, n, 0, q.scale, q.scale_dev,
+                             make_key(key), elem_offset, codes, diag, (cudaStream_t)stream);
+}
+
+int bsp_round_grouped(const void* x, int dt, size_t n_groups, size_t group_size, int fmt, int mode,
+                      const float* scales, bsp_key_t key, uint8_t* codes, bsp_diag_t* diag, void* stream) {
+  if (!valid_enum(dt, 1) || !valid_enum(fmt, 1) || !valid_enum(mode, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (n_groups == 0 || group_size == 0) return BSP_OK;
+  if (!x || !codes || !scales) return BSP_ERR_ARG;
+  if (!aligned16(x) || !aligned16(codes)) return BSP_ERR_ALIGN;
+  return dispatch_round_flat(dt, fmt, mode, x, n_groups * group_size, group_size, 1.f, scales, make_key(key), 0,
+                             codes, diag, (cudaStream_t)stream);
+}
+
+int bsp_round_2d(const void* x, int dt, int64_t rows, int64_t cols, bsp_quant_t q, bsp_key_t key,
+                 uint8_t* codes, uint8_t* codes_t, int64_t ld_t, bsp_diag_t* diag, void* stream) {
+  if (!valid_enum(dt, 1) || !valid_enum(q.fmt, 1) || !valid_enum(q.mode, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (rows < 0 || cols < 0) return BSP_ERR_ARG;
+  if (rows == 0 || cols == 0) return BSP_OK;
+  if (!x || (!codes && !codes_t)) return BSP_ERR_ARG;
+  if (cols % 16 != 0) return BSP_ERR_UNSUPPORTED;
+  if (codes_t && (ld_t < rows || ld_t % 16 != 0)) return BSP_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(codes_t)) return BSP_ERR_ALIGN;
+  return launch_tile(dt, q.fmt, q.mode, (cudaStream_t)stream, PlainProducer(), x, rows, cols, q.scale, q.scale_dev,
+                     make_key(key), codes, codes_t, ld_t, nullptr, nullptr, diag);
+}
+
+int bsp_norm_stats(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
+                   float eps, float* rstd, float* mean, float* amax, bsp_diag_t* diag, void* stream) {
+  if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || T < 0 || C <= 0) return BSP_ERR_ARG;
+  if (T == 0) return BSP_OK;
+  if (!x || !rstd || (kind == BSP_LAYERNORM && !mean)) return BSP_ERR_ARG;
+  if (amax && (!gamma || (kind == BSP_LAYERNORM && !beta))) return BSP_ERR_ARG;
+  if (C % 4 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(gamma) || !aligned16(beta)) return BSP_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (amax) BSP_CHECK_CUDA(cudaMemsetAsync(amax, 0, sizeof(float), st));
+  const unsigned blocks = (unsigned)((T + 7) / 8);
+  if (dt == BSP_F32)
+    norm_stats_kernel<BSP_F32><<<blocks, 256, 0, st>>>(kind, x, T, C, gamma, beta, eps, rstd, mean,
+                                                       reinterpret_cast<uint32_t*>(amax), diag);
+  else
+    norm_stats_kernel<BSP_BF16><<<blocks, 256, 0, st>>>(kind, x, T, C, gamma, beta, eps, rstd, mean,
+                                                        reinterpret_cast<uint32_t*>(amax), diag);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_norm_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
+                 const float* rstd, const float* mean, bsp_quant_t q, bsp_key_t key, uint8_t* u_codes,
+                 uint8_t* u_codes_t, int64_t ld_t, float* u_f32, void* u_bf16_t, bsp_diag_t* diag, void* stream) {
+  if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(q.fmt, 1) || !valid_enum(q.mode, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (T < 0 || C <= 0) return BSP_ERR_ARG;
+  if (T == 0) return BSP_OK;
+  if (!x || !gamma || !rstd || (kind == BSP_LAYERNORM && (!beta || !mean))) return BSP_ERR_ARG;
+  if (!u_codes && !u_codes_t && !u_f32 && !u_bf16_t) return BSP_ERR_ARG;
+  if (C % 16 != 0) return BSP_ERR_UNSUPPORTED;
+  if ((u_codes_t || u_bf16_t) && (ld_t < T || ld_t % 16 != 0)) return BSP_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(u_codes) || !aligned16(u_codes_t) || !aligned16(u_f32) || !aligned16(u_bf16_t))
+    return BSP_ERR_ALIGN;
+  NormProducer prod;
+  prod.kind = kind; prod.gamma = gamma; prod.beta = beta; prod.rstd = rstd; prod.mean = mean;
+  prod.r_ = 0.f; prod.m_ = 0.f;
+  return launch_tile(dt, q.fmt, q.mode, (cudaStream_t)stream, prod, x, T, C, q.scale, q.scale_dev, make_key(key),
+                     u_codes, u_codes_t, ld_t, u_f32, reinterpret_cast<uint16_t*>(u_bf16_t), diag);
+}
+
+}  // extern "C"
