@@ -85,8 +85,9 @@ def encode(v32, fmt: int, mode: int = RN, words=None):
     f = t - n.  Nearest: up iff f > 1/2 or (f == 1/2 and n odd).  Stochastic: P = floor(f 2^32),
     up iff U < P with U the element's 32-bit random word, so P(up) = f and the mean is v.
     The result magnitude is (n + up) * ulp; the sign bit of v is kept even when that is zero.
-    a >= fmax gives +-fmax (counted as saturated when a > fmax); NaN gives the canonical NaN
-    code 0x7F | sign; infinities saturate and are counted as non-finite.
+    a >= fmax gives +-fmax (counted as saturated when a > fmax); NaN gives the NaN code
+    0x7F whatever its sign bit (IEEE 754 leaves the sign of a NaN produced by the scaling multiply
+    unspecified); infinities saturate and are counted as non-finite.
 
     Returns (codes uint8, n_saturated, n_nonfinite).
     """
@@ -127,8 +128,8 @@ def encode(v32, fmt: int, mode: int = RN, words=None):
     if not np.array_equal(vals[idx][~isnan], mag[~isnan]):
         raise AssertionError("rounded magnitude is not representable")
     codes = poscodes[idx].astype(np.uint8)
-    codes = np.where(isnan, np.uint8(0x7F), codes)
     codes = codes | (sign.astype(np.uint8) << np.uint8(7))
+    codes = np.where(isnan, np.uint8(0x7F), codes)       # one NaN code, whatever the NaN's sign bit
     return codes.reshape(shape).astype(np.uint8), n_sat, n_nonfinite
 
 

@@ -103,7 +103,7 @@ __device__ __forceinline__ uint32_t f8_encode(float v, uint32_t U, DiagCounters&
   const uint32_t sign = (b >> 24) & 0x80u;
   const uint32_t a = b & 0x7FFFFFFFu;
   if (a >= F::FMAX_BITS) {
-    if (a > 0x7F800000u) { dc.nonfinite++; return sign | 0x7Fu; }       // NaN -> canonical NaN
+    if (a > 0x7F800000u) { dc.nonfinite++; return 0x7Fu; }              // any NaN -> the one NaN code
     if (a == 0x7F800000u) dc.nonfinite++; else if (a > F::FMAX_BITS) dc.sat++;
     return sign | F::TOP;
   }

@@ -298,7 +298,7 @@ def test_mc_statistics_match_oracle(b):
     rng = np.random.default_rng(12)
     n, K = 50000, 24
     ref = rng.standard_normal(n).astype(np.float32)
-    gk = ref[None, :].astype(np.float64) + 0.05 * rng.standard_normal((K, n)) + 0.01
+    gk = ref[None, :].astype(np.float64) + 0.05 * rng.standard_normal((K, n)) + 0.03
     d = gk - ref.astype(np.float64)
     S1 = d.sum(0).astype(np.float32)
     S2 = (d * d).sum(0).astype(np.float32)
