@@ -183,6 +183,16 @@ int bsp_norm_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
                  bsp_key_t key, uint8_t* u_codes, uint8_t* u_codes_t, int64_t ld_t, float* u_f32,
                  void* u_bf16_t, bsp_diag_t* diag, void* stream);
 
+/* The re-rounding pass for n_draws consecutive draws [draw0, draw0 + n_draws) of a fresh read
+ * (policy N; "a new rounding draws separate random numbers the same way", Section "Same rounding
+ * distribution, opposite outcomes"): the FP32 value of each element is formed once and rounded
+ * stochastically once per draw (key.draw is ignored).  Writes only the transposed code matrices,
+ * draw d at u_codes_t_draws + d * C * ld_t, each [C * ld_t]. */
+int bsp_norm_fwd_draws(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                       const float* beta, const float* rstd, const float* mean, bsp_quant_t q,
+                       bsp_key_t key, int draw0, int n_draws, uint8_t* u_codes_t_draws, int64_t ld_t,
+                       void* stream);
+
 /* Backward of the normalisation with du passed through the rounding unchanged:
  *   dgamma[C] = sum_t z_g o du, z_g = z (U) | (decode(u_codes)/scale - beta)/gamma (R) |
  *               the same from a fresh rounding under `key` (N, one draw);
@@ -222,6 +232,18 @@ int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t,
                      int x_read, const void* x_t, bsp_quant_t q_x, int64_t ld_t, float* dW,
                      const float* mc_ref, float* mc_S1, float* mc_S2, void* ws, size_t ws_bytes,
                      bsp_diag_t* diag, void* stream);
+
+/* The weight use under n_draws fresh roundings in one launch (Section "Each use has a checkable
+ * requirement": the substitute's own draw is averaged with the forward and the incoming gradient
+ * held fixed).  x_t_draws holds n_draws code matrices [C * ld_t] back to back (as written by
+ * bsp_norm_fwd_draws).  For every draw d: dW_d = dY^T X_d, and
+ *   S1 += dW_d - g_ref,  S2 += (dW_d - g_ref)^2      (all [O*C] FP32; S1, S2 are read, updated,
+ * written back, so draw ranges can be chained).  The per-draw gradients are never written: the
+ * running sums of an output tile stay in tensor memory while the kernel walks the draws.
+ * C must be a multiple of 16. */
+int bsp_linear_wgrad_mc(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy,
+                        const uint8_t* x_t_draws, bsp_quant_t q_x, int64_t ld_t, int n_draws,
+                        const float* g_ref, float* S1, float* S2, bsp_diag_t* diag, void* stream);
 
 /* du[T*C] (du_dt) = dY W with dY = decode(dy_codes[T*O]) / scale and W w_dt[O*C]: the incoming
  * gradient passed through the rounding unchanged.  BF16 tensor cores (W rounded to bf16). */

@@ -78,6 +78,8 @@ _SIGNATURES = {
     "bsp_round_2d": (_I, [_P, _I, _I64, _I64, Quant, Key, _P, _P, _I64, _P, _P]),
     "bsp_norm_stats": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _F, _P, _P, _P, _P, _P]),
     "bsp_norm_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, Quant, Key, _P, _P, _I64, _P, _P, _P, _P]),
+    "bsp_norm_fwd_draws": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, Quant, Key, _I, _I, _P, _I64, _P]),
+    "bsp_linear_wgrad_mc": (_I, [_I64, _I64, _I64, _P, Quant, _P, Quant, _I64, _I, _P, _P, _P, _P, _P]),
     "bsp_norm_bwd_workspace_bytes": (_SZ, [_I64, _I64]),
     "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
                           _P, _SZ, _P, _P]),
@@ -232,6 +234,20 @@ def bsp_norm_fwd(kind, x, T, Cc, gamma, beta, rstd, mean, q: Quant, k: Key, u_co
     check(lib().bsp_norm_fwd(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean), q, k,
                              ptr(u_codes), ptr(u_codes_t), ld_t, ptr(u_f32), ptr(u_bf16_t), ptr(diag),
                              stream if stream is not None else cur_stream()), "bsp_norm_fwd")
+
+
+def bsp_norm_fwd_draws(kind, x, T, Cc, gamma, beta, rstd, mean, q: Quant, k: Key, draw0, n_draws,
+                       u_codes_t_draws, ld_t, stream=None):
+    check(lib().bsp_norm_fwd_draws(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
+                                   q, k, draw0, n_draws, ptr(u_codes_t_draws), ld_t,
+                                   stream if stream is not None else cur_stream()), "bsp_norm_fwd_draws")
+
+
+def bsp_linear_wgrad_mc(T, O, Cc, dy_codes_t, q_dy: Quant, x_t_draws, q_x: Quant, ld_t, n_draws, g_ref, S1, S2,
+                        diag=None, stream=None):
+    check(lib().bsp_linear_wgrad_mc(T, O, Cc, ptr(dy_codes_t), q_dy, ptr(x_t_draws), q_x, ld_t, n_draws,
+                                    ptr(g_ref), ptr(S1), ptr(S2), ptr(diag),
+                                    stream if stream is not None else cur_stream()), "bsp_linear_wgrad_mc")
 
 
 def bsp_norm_bwd_workspace_bytes(T, Cc):

@@ -303,30 +303,222 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                   *reinterpret_cast<uint2*>(dst + j) = make_uint2(lo, hi);
                 }
               }
-            } else {   // EPI_MC: shifted sums against the reference gradient
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                if (col0 + j < p.N) {
-                  const float4 g0 = *reinterpret_cast<const float4*>(p.ref + off + j);
-                  float4 s1 = *reinterpret_cast<float4*>(p.S1 + off + j);
-                  float4 s2 = *reinterpret_cast<float4*>(p.S2 + off + j);
-                  const float d0 = __uint_as_float(r[j]) * inv_a * inv_b - g0.x;
-                  const float d1 = __uint_as_float(r[j + 1]) * inv_a * inv_b - g0.y;
-                  const float d2 = __uint_as_float(r[j + 2]) * inv_a * inv_b - g0.z;
-                  const float d3 = __uint_as_float(r[j + 3]) * inv_a * inv_b - g0.w;
-                  s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
-                  s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y);
-                  s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
-                  *reinterpret_cast<float4*>(p.S1 + off + j) = s1;
-                  *reinterpret_cast<float4*>(p.S2 + off + j) = s2;
-                }
-              }
             }
           }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.diag) atomicMax(&p.diag->status, (int)BSP_ERR_TIMEOUT);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------- Monte-Carlo contraction
+
+// FP8 contraction over nb draws of B with the per-element shifted sums kept in tensor memory:
+// for every output tile the CTA walks all draws b and accumulates
+//   S1 += alpha*acc_b - ref,   S2 += (alpha*acc_b - ref)^2
+// without ever writing a per-draw gradient.  Tile 128 x 128; TMEM columns: two accumulator stages
+// [0,128) and [128,256), S1 in [256,384), S2 in [384,512).  The reference tile sits in the
+// epilogue threads' registers for the whole tile; S1/S2 are read from global memory once per tile
+// (so calls can be chained over draw ranges) and written back once.
+// 320 threads: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue (two warps per TMEM lane quarter, each
+// owning 64 of the 128 columns).
+constexpr int MC_BN = 128;
+constexpr int kMcStages = 6;
+constexpr int kMcABytes = BM * BKB, kMcBBytes = MC_BN * BKB, kMcStageBytes = kMcABytes + kMcBBytes;
+constexpr int kMcThreads = 320;
+constexpr size_t kMcSmem = (size_t)kMcStages * kMcStageBytes + 1024 + 256;
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kMcThreads, 1)
+gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  const uint32_t bars = tiles + kMcStages * kMcStageBytes;
+  const uint32_t full0 = bars, empty0 = bars + 8 * kMcStages, tfull0 = bars + 16 * kMcStages, tempty0 = tfull0 + 16;
+  uint8_t* bars_gen = smem_raw + (bars - raw);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 16 * kMcStages + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 16 * kMcStages + 36);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + MC_BN - 1) / MC_BN;
+  const int ntiles = tiles_m * tiles_n;
+  const int kblocks = (p.K + BKB - 1) / BKB;          // FP8: one byte per element
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kMcStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 8); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tmap_a);
+      tma_prefetch_desc(&tmap_b);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        const int tm = t / tiles_n, tn = t % tiles_n;
+        for (int b = 0; b < p.nb && ok; ++b) {
+          for (int kb = 0; kb < kblocks; ++kb, ++it) {
+            const uint32_t s = it % kMcStages, ph = (it / kMcStages) & 1u;
+            if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
+            mbar_expect_tx(full0 + 8 * s, kMcStageBytes);
+            tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * BKB, tm * BM);
+            tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b);
+          }
+        }
+      }
+      if (!ok) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, tc = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        for (int b = 0; b < p.nb && ok; ++b, ++tc) {
+          const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
+          if (!mbar_wait(tempty0 + 8 * as, aph ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t tmem_d = tmem_base + as * MC_BN;
+          for (int kb = 0; kb < kblocks; ++kb, ++it) {
+            const uint32_t s = it % kMcStages, ph = (it / kMcStages) & 1u;
+            if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
+            const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+#pragma unroll
+            for (int k = 0; k < BKB / 32; ++k)
+              tc_mma<true>(tmem_d, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+            tc_commit(empty0 + 8 * s);
+          }
+          if (ok) tc_commit(tfull0 + 8 * as);
+        }
+      }
+    }
+  } else {
+    const int q = warp & 3;                  // TMEM lane quarter
+    const int h = (warp - 2) >> 2;           // column half
+    const float inv_a = __fdiv_rn(1.0f, p.sa_dev ? __ldg(p.sa_dev) : p.sa);
+    const float inv_b = __fdiv_rn(1.0f, p.sb_dev ? __ldg(p.sb_dev) : p.sb);
+    const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+    const uint32_t s1_base = lane_base + 2 * MC_BN + h * 64, s2_base = lane_base + 3 * MC_BN + h * 64;
+    uint32_t tc = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+      const int tm = t / tiles_n, tn = t % tiles_n;
+      const int row = tm * BM + q * 32 + lane;
+      const int colbase = tn * MC_BN + h * 64;
+      float refv[64];
+      // ---- tile start: reference into registers, running sums into tensor memory
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = colbase + c * 16;
+        uint32_t a1[16], a2[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { a1[j] = 0u; a2[j] = 0u; refv[c * 16 + j] = 0.f; }
+        if (row < p.M && col < p.N) {
+          const size_t off = (size_t)row * p.ldc + col;
+#pragma unroll
+          for (int j = 0; j < 16; j += 4) {
+            const float4 g0 = *reinterpret_cast<const float4*>(p.ref + off + j);
+            const uint4 v1 = *reinterpret_cast<const uint4*>(p.S1 + off + j);
+            const uint4 v2 = *reinterpret_cast<const uint4*>(p.S2 + off + j);
+            refv[c * 16 + j] = g0.x; refv[c * 16 + j + 1] = g0.y; refv[c * 16 + j + 2] = g0.z; refv[c * 16 + j + 3] = g0.w;
+            a1[j] = v1.x; a1[j + 1] = v1.y; a1[j + 2] = v1.z; a1[j + 3] = v1.w;
+            a2[j] = v2.x; a2[j + 1] = v2.y; a2[j + 2] = v2.z; a2[j + 3] = v2.w;
+          }
+        }
+        tmem_st16(s1_base + c * 16, a1);
+        tmem_st16(s2_base + c * 16, a2);
+      }
+      tmem_wait_st();
+      // ---- every draw of this tile
+      for (int b = 0; b < p.nb && ok; ++b, ++tc) {
+        const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull0 + 8 * as, aph, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t acc_base = lane_base + as * MC_BN + h * 64;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t acc[16], a1[16], a2[16];
+          tmem_ld16(acc_base + c * 16, acc);
+          tmem_ld16(s1_base + c * 16, a1);
+          tmem_ld16(s2_base + c * 16, a2);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float d = __uint_as_float(acc[j]) * inv_a * inv_b - refv[c * 16 + j];
+            a1[j] = __float_as_uint(__uint_as_float(a1[j]) + d);
+            a2[j] = __float_as_uint(fmaf(d, d, __uint_as_float(a2[j])));
+          }
+          tmem_st16(s1_base + c * 16, a1);
+          tmem_st16(s2_base + c * 16, a2);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+      }
+      if (!ok) break;
+      // ---- tile end: running sums back to global memory
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = colbase + c * 16;
+        uint32_t a1[16], a2[16];
+        tmem_ld16(s1_base + c * 16, a1);
+        tmem_ld16(s2_base + c * 16, a2);
+        tmem_wait_ld();
+        if (row < p.M && col < p.N) {
+          const size_t off = (size_t)row * p.ldc + col;
+#pragma unroll
+          for (int j = 0; j < 16; j += 4) {
+            *reinterpret_cast<uint4*>(p.S1 + off + j) = make_uint4(a1[j], a1[j + 1], a1[j + 2], a1[j + 3]);
+            *reinterpret_cast<uint4*>(p.S2 + off + j) = make_uint4(a2[j], a2[j + 1], a2[j + 2], a2[j + 3]);
+          }
+        }
       }
     }
   }
@@ -474,9 +666,36 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     return BSP_OK;
   }
 
+  int nsm = kNumSMs;
+  {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      nsm = v;
+  }
   CUtensorMap ma, mb;
   int rc = make_operand_map(&ma, g.A, eb, g.K, g.M, g.lda, 0, 0, BM);
   if (rc != BSP_OK) return rc;
+
+  if (g.mode == EPI_MC) {
+    // shifted sums resident in tensor memory over all draws of a tile
+    if (!g.fp8) return BSP_ERR_UNSUPPORTED;
+    if (g.N % 16 != 0 || !g.ref || !g.S1 || !g.S2) return BSP_ERR_ARG;
+    rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, MC_BN);
+    if (rc != BSP_OK) return rc;
+    p.idesc = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, MC_BN);
+    static bool mc_attr_set = false;
+    if (!mc_attr_set) {
+      BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
+      mc_attr_set = true;
+    }
+    const int ntiles_mc = (int)(((g.M + BM - 1) / BM) * ((g.N + MC_BN - 1) / MC_BN));
+    const int grid_mc = ntiles_mc < nsm ? ntiles_mc : nsm;
+    gemm_mc_kernel<<<grid_mc, kMcThreads, kMcSmem, st>>>(ma, mb, p);
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  }
+
   rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN);
   if (rc != BSP_OK) return rc;
   static bool attr_set[2] = {false, false};
@@ -486,12 +705,6 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     attr_set[g.fp8 ? 1 : 0] = true;
   }
   const int ntiles = (int)(((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN));
-  int nsm = kNumSMs;
-  int dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) {
-    int v = 0;
-    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) nsm = v;
-  }
   const int grid = ntiles < nsm ? ntiles : nsm;
   if (g.fp8) gemm_tc_kernel<true><<<grid, kGemmThreads, kGemmSmem, st>>>(ma, mb, p);
   else gemm_tc_kernel<false><<<grid, kGemmThreads, kGemmSmem, st>>>(ma, mb, p);
@@ -595,6 +808,24 @@ int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t,
     g.fp8 = true; g.A = dy_codes_t; g.B = x_t; g.a_fmt = q_dy.fmt; g.b_fmt = q_x.fmt;
   }
   return gemm_run(g, st);
+}
+
+int bsp_linear_wgrad_mc(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy,
+                        const uint8_t* x_t_draws, bsp_quant_t q_x, int64_t ld_t, int n_draws, const float* g_ref,
+                        float* S1, float* S2, bsp_diag_t* diag, void* stream) {
+  if (T < 0 || O < 0 || C < 0 || n_draws < 0 || !valid_enum(q_dy.fmt, 1) || !valid_enum(q_x.fmt, 1)) return BSP_ERR_ARG;
+  if (O == 0 || C == 0 || n_draws == 0) return BSP_OK;
+  if (!g_ref || !S1 || !S2) return BSP_ERR_ARG;
+  if (T == 0) return BSP_ERR_UNSUPPORTED;       // every draw would add (0 - ref): not a case the check produces
+  if (!dy_codes_t || !x_t_draws) return BSP_ERR_ARG;
+  if (ld_t < T || ld_t % 16 != 0 || C % 16 != 0) return BSP_ERR_ALIGN;
+  GemmArgs g;
+  g.M = O; g.N = C; g.K = T; g.nb = n_draws; g.fp8 = true;
+  g.A = dy_codes_t; g.B = x_t_draws; g.a_fmt = q_dy.fmt; g.b_fmt = q_x.fmt;
+  g.lda = ld_t; g.ldb = ld_t; g.b_batch_stride = (int64_t)C * ld_t;
+  g.sa = q_dy.scale; g.sa_dev = q_dy.scale_dev; g.sb = q_x.scale; g.sb_dev = q_x.scale_dev;
+  g.mode = EPI_MC; g.C = nullptr; g.ldc = C; g.ref = g_ref; g.S1 = S1; g.S2 = S2; g.diag = diag;
+  return gemm_run(g, (cudaStream_t)stream);
 }
 
 size_t bsp_linear_dgrad_workspace_bytes(int64_t T, int64_t O, int64_t C) {

@@ -79,6 +79,17 @@ struct Bump {
   }
 };
 
+// Draws per re-round + contraction launch pair: as many as fit a 1 GiB code buffer, balanced so
+// that the chunks are of near-equal size.
+static int draw_chunk(int64_t C, int64_t ld_t, int K) {
+  const int64_t per = C * ld_t;
+  int64_t fit = ((int64_t)1 << 30) / (per > 0 ? per : 1);
+  if (fit < 1) fit = 1;
+  if (fit >= K) return K > 0 ? K : 1;
+  const int64_t nchunks = (K + fit - 1) / fit;
+  return (int)((K + nchunks - 1) / nchunks);
+}
+
 struct CheckBuffers {
   float *rstd, *mean, *amax_u, *scale_u, *amax_dy, *scale_dy;
   uint8_t *u_codes, *u_codes_t, *fresh_t, *dy_codes, *dy_codes_t;
@@ -103,7 +114,7 @@ static size_t carve(const bsp_norm_linear_desc_t* op, int K, char* base, CheckBu
   c.amax_u = (float*)b.take(4); c.scale_u = (float*)b.take(4);
   c.amax_dy = (float*)b.take(4); c.scale_dy = (float*)b.take(4);
   c.u_codes = (uint8_t*)b.take(T * C); c.u_codes_t = (uint8_t*)b.take(C * ld_t);
-  c.fresh_t = (uint8_t*)b.take(C * ld_t);
+  c.fresh_t = (uint8_t*)b.take(C * ld_t * (size_t)draw_chunk((int64_t)C, (int64_t)ld_t, K > 0 ? K : 1));
   c.dy_codes = (uint8_t*)b.take(T * O); c.dy_codes_t = (uint8_t*)b.take(O * ld_t);
   c.u_bf16_t = (uint16_t*)b.take(C * ld_t * 2);
   c.du = b.take(T * C * eb);
@@ -298,12 +309,16 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
       bsp_quant_t qf = qu;
       qf.mode = BSP_ROUND_STOCHASTIC;
       key.stream = BSP_STREAM_WGRAD;
-      for (int k = 0; k < K; ++k) {
-        key.draw = (uint32_t)k;
-        BSP_TRY(bsp_norm_fwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qf, key, nullptr,
-                             b.fresh_t, b.ld_t, nullptr, nullptr, nullptr, st));
-        BSP_TRY(bsp_linear_wgrad(T, O, C, b.dy_codes_t, qdy, BSP_READ_FRESH, b.fresh_t, qf, b.ld_t, nullptr, b.dW_ref,
-                                 S1w, b.S2w, b.ws_wgrad, b.b_wgrad, diag, st));
+      // draws in chunks: one re-rounding launch writes the chunk's code matrices, one contraction
+      // launch walks them with the running sums resident in tensor memory
+      const int chunk = draw_chunk(C, b.ld_t, K);
+      key.draw = 0;
+      for (int k0 = 0; k0 < K; k0 += chunk) {
+        const int nd = (K - k0) < chunk ? (K - k0) : chunk;
+        BSP_TRY(bsp_norm_fwd_draws(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qf, key, k0,
+                                   nd, b.fresh_t, b.ld_t, st));
+        BSP_TRY(bsp_linear_wgrad_mc(T, O, C, b.dy_codes_t, qdy, b.fresh_t, qf, b.ld_t, nd, b.dW_ref, S1w, b.S2w, diag,
+                                    st));
       }
       bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FRESH);
       BSP_TRY(bsp_mc_stats(b.dW_ref, S1w, b.S2w, O * C, K, 1, r, b.ws_stats, b.b_stats, st));

@@ -76,12 +76,13 @@ __global__ void scale_from_amax_kernel(const float* __restrict__ amax, size_t n,
 
 // Encodes 16 consecutive values whose first element has logical index e0 (e0 % 4 == 0).
 template <int FMT, int MODE>
-__device__ __forceinline__ uint4 encode16(const float (&v)[16], const PhiloxKey& key, uint64_t e0, DiagCounters& dc) {
+__device__ __forceinline__ uint4 encode16(const float (&v)[16], const PhiloxKey& key, uint32_t draw, uint64_t e0,
+                                          DiagCounters& dc) {
   uint32_t packed[4];
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
     uint4 w = make_uint4(0, 0, 0, 0);
-    if (MODE == BSP_ROUND_STOCHASTIC) w = philox_block(key, (e0 >> 2) + b, key.c2);
+    if (MODE == BSP_ROUND_STOCHASTIC) w = philox_block(key, (e0 >> 2) + b, draw);
     const uint32_t c0 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 0], w.x, dc);
     const uint32_t c1 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 1], w.y, dc);
     const uint32_t c2 = f8_encode<FMT, MODE == BSP_ROUND_STOCHASTIC>(v[4 * b + 2], w.z, dc);
@@ -109,7 +110,7 @@ round_vec_kernel(const void* __restrict__ x, size_t n16, size_t group_size, floa
       v[4 * j + 0] = __fmul_rn(f.x, s); v[4 * j + 1] = __fmul_rn(f.y, s);
       v[4 * j + 2] = __fmul_rn(f.z, s); v[4 * j + 3] = __fmul_rn(f.w, s);
     }
-    reinterpret_cast<uint4*>(codes)[t] = encode16<FMT, MODE>(v, key, elem_offset + i0, dc);
+    reinterpret_cast<uint4*>(codes)[t] = encode16<FMT, MODE>(v, key, key.c2, elem_offset + i0, dc);
   }
   diag_flush_warp(diag, dc);
 }
@@ -195,7 +196,7 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
         reinterpret_cast<float4*>(u_f32 + i0)[j] = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
     }
     if (codes || codes_t) {
-      const uint4 pk = encode16<FMT, MODE>(v, key, (uint64_t)i0, dc);
+      const uint4 pk = encode16<FMT, MODE>(v, key, key.c2, (uint64_t)i0, dc);
       if (codes) *reinterpret_cast<uint4*>(codes + i0) = pk;
       if (codes_t) {
         uint32_t* dst = reinterpret_cast<uint32_t*>(&s_codes[tr][tc]);
@@ -239,6 +240,60 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
     }
   }
   diag_flush_warp(diag, dc);
+}
+
+// Fresh re-roundings of the normalisation output for `ndraws` consecutive draws in one pass: the
+// FP32 value of every element is formed once, then rounded stochastically once per draw; only the
+// transposed code matrices are written: codes_t[d][c][r], d-th matrix at d * cols * ld_t.
+template <int DT, int FMT>
+__global__ void __launch_bounds__(256)
+reround_draws_kernel(NormProducer prod, const void* __restrict__ x, int64_t rows, int64_t cols, float scale_val,
+                     const float* __restrict__ scale_dev, PhiloxKey key, int draw0, int ndraws,
+                     uint8_t* __restrict__ codes_t, int64_t ld_t) {
+  __shared__ __align__(16) uint8_t s_codes[2][kTile][kTile + 4];
+  const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
+  const int tr = threadIdx.x >> 2, tc = (threadIdx.x & 3) * 16;
+  const int64_t r = r0 + tr, c = c0 + tc;
+  const float s = scale_dev ? __ldg(scale_dev) : scale_val;
+  const bool active = (r < rows) && (c < cols);
+  const size_t i0 = (size_t)r * cols + c;
+  float v[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] = 0.f;
+  if (active) {
+    prod.row(r);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 f = load4<DT>(x, i0 + 4 * j);
+      v[4 * j + 0] = __fmul_rn(prod.value(f.x, c + 4 * j + 0), s);
+      v[4 * j + 1] = __fmul_rn(prod.value(f.y, c + 4 * j + 1), s);
+      v[4 * j + 2] = __fmul_rn(prod.value(f.z, c + 4 * j + 2), s);
+      v[4 * j + 3] = __fmul_rn(prod.value(f.w, c + 4 * j + 3), s);
+    }
+  }
+  const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
+  const int64_t cc = c0 + tcol, rr = r0 + trow;
+  const bool wr = cc < cols && rr < rows;
+  const int nvalid = wr ? (int)((rows - rr) < 16 ? (rows - rr) : 16) : 0;
+  DiagCounters dc;
+  for (int d = 0; d < ndraws; ++d) {
+    const int buf = d & 1;
+    if (active) {
+      const uint4 pk = encode16<FMT, BSP_ROUND_STOCHASTIC>(v, key, (uint32_t)(draw0 + d), (uint64_t)i0, dc);
+      uint32_t* dst = reinterpret_cast<uint32_t*>(&s_codes[buf][tr][tc]);
+      dst[0] = pk.x; dst[1] = pk.y; dst[2] = pk.z; dst[3] = pk.w;
+    }
+    __syncthreads();
+    if (wr) {
+      uint32_t pk[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t b = j < nvalid ? s_codes[buf][trow + j][tcol] : 0u;
+        pk[j >> 2] |= b << (8 * (j & 3));
+      }
+      *reinterpret_cast<uint4*>(codes_t + ((size_t)d * cols + cc) * ld_t + rr) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------- norm statistics
@@ -507,6 +562,35 @@ int bsp_norm_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
   prod.r_ = 0.f; prod.m_ = 0.f;
   return launch_tile(dt, q.fmt, q.mode, (cudaStream_t)stream, prod, x, T, C, q.scale, q.scale_dev, make_key(key),
                      u_codes, u_codes_t, ld_t, u_f32, reinterpret_cast<uint16_t*>(u_bf16_t), diag);
+}
+
+int bsp_norm_fwd_draws(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
+                       const float* rstd, const float* mean, bsp_quant_t q, bsp_key_t key, int draw0, int n_draws,
+                       uint8_t* u_codes_t_draws, int64_t ld_t, void* stream) {
+  if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(q.fmt, 1)) return BSP_ERR_ARG;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
+  if (T < 0 || C <= 0 || draw0 < 0 || n_draws < 0) return BSP_ERR_ARG;
+  if (T == 0 || n_draws == 0) return BSP_OK;
+  if (!x || !gamma || !rstd || !u_codes_t_draws || (kind == BSP_LAYERNORM && (!beta || !mean))) return BSP_ERR_ARG;
+  if (C % 16 != 0) return BSP_ERR_UNSUPPORTED;
+  if (ld_t < T || ld_t % 16 != 0) return BSP_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(u_codes_t_draws)) return BSP_ERR_ALIGN;
+  NormProducer prod;
+  prod.kind = kind; prod.gamma = gamma; prod.beta = beta; prod.rstd = rstd; prod.mean = mean;
+  prod.r_ = 0.f; prod.m_ = 0.f;
+  dim3 grid((unsigned)((C + kTile - 1) / kTile), (unsigned)((T + kTile - 1) / kTile));
+  cudaStream_t st = (cudaStream_t)stream;
+  const PhiloxKey pk = make_key(key);
+#define BSP_RR(DT, FMT)                                                                                          \
+  reround_draws_kernel<DT, FMT><<<grid, 256, 0, st>>>(prod, x, T, C, q.scale, q.scale_dev, pk, draw0, n_draws,   \
+                                                      u_codes_t_draws, ld_t)
+  if (dt == BSP_F32 && q.fmt == BSP_E4M3) BSP_RR(BSP_F32, BSP_E4M3);
+  else if (dt == BSP_F32) BSP_RR(BSP_F32, BSP_E5M2);
+  else if (q.fmt == BSP_E4M3) BSP_RR(BSP_BF16, BSP_E4M3);
+  else BSP_RR(BSP_BF16, BSP_E5M2);
+#undef BSP_RR
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
 }
 
 }  // extern "C"

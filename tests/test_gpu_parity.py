@@ -266,18 +266,36 @@ def test_weight_gradient_fused_monte_carlo_epilogue(b, case):
     refd = up(ref32.ravel())
     S1 = torch.zeros(O * C, device="cuda")
     S2 = torch.zeros(O * C, device="cuda")
-    fresh_t = torch.zeros(C * g.ld_t, dtype=torch.uint8, device="cuda")
+    fresh_t = torch.zeros(4 * C * g.ld_t, dtype=torch.uint8, device="cuda")
     q = b.quant(inp.store_fmt, b.ROUND_STOCHASTIC, 1.0, g.scale)
-    ws = b.workspace(256)
+    key = b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, 0)
+    diag = b.new_diag()
     acc = mc.Welford(ref.shape)
+    want_codes = []
     for k in range(K):
-        b.bsp_norm_fwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, q,
-                       b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, k), None, fresh_t, g.ld_t)
-        b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, 2, fresh_t, q, g.ld_t, None, refd, S1, S2, ws=ws)
-        acc.add(linear.wgrad(prep["dy"]["value"], check.fresh_copy(prep, inp.seed, philox.STREAM_WGRAD, k)[0]))
+        copy, codes = check.fresh_copy(prep, inp.seed, philox.STREAM_WGRAD, k)
+        want_codes.append(codes)
+        acc.add(linear.wgrad(prep["dy"]["value"], copy))
+    # two chained draw ranges: 4 draws, then the remaining 2
+    for k0, nd in ((0, 4), (4, K - 4)):
+        b.bsp_norm_fwd_draws(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, q, key, k0, nd, fresh_t, g.ld_t)
+        got = fresh_t.cpu().numpy()[:nd * C * g.ld_t].reshape(nd, C, g.ld_t)
+        for d in range(nd):
+            assert np.array_equal(got[d, :, :T], want_codes[k0 + d].T)
+        b.bsp_linear_wgrad_mc(T, O, C, g.dy_codes_t, g.q_dy, fresh_t, q, g.ld_t, nd, refd, S1, S2, diag)
+    assert b.read_diag(diag)["status"] == 0
     mean_gpu, m2_gpu = mc.shifted_sums_to_moments(down(S1).reshape(O, C), down(S2).reshape(O, C), K, ref32)
     assert rel_l2(mean_gpu, acc.mean) <= TOL_TC
     assert rel_l2(m2_gpu, acc.m2) <= 1e-2
+    # the single-draw form of bsp_linear_wgrad takes the same path and gives the same sums
+    S1b = torch.zeros(O * C, device="cuda")
+    S2b = torch.zeros(O * C, device="cuda")
+    one = torch.zeros(C * g.ld_t, dtype=torch.uint8, device="cuda")
+    for k in range(K):
+        b.bsp_norm_fwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, q,
+                       b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, k), None, one, g.ld_t)
+        b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, 2, one, q, g.ld_t, None, refd, S1b, S2b, ws=b.workspace(256))
+    assert torch.equal(S1, S1b) and torch.equal(S2, S2b)
 
 
 def test_input_gradient_helper(b, case):
