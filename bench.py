@@ -162,7 +162,7 @@ def run_ours(args):
 
     from paper_2609_39813_b200 import binding as b
     from paper_2609_39813_b200 import workloads
-    from paper_2609_39813_b200.harness import NormLinearGpu, up
+    from paper_2609_39813_b200.harness import NormLinearGpu, max_over_ranks, replica_throughput
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -212,12 +212,9 @@ def run_ours(args):
     launches = b.bsp_launch_count() - n0
     clocks = sampler.stop() if rank == 0 else None
     ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms, device="cuda")
     elements = check_elements(T, C, K)
-    value = world * elements * args.steps / (ms_total * 1e-3)
+    value = replica_throughput(elements, args.steps, world, ms_total)
 
     # ---- end to end: host buffers in, host results out, through the same entry point
     host = dict(x=g.x.cpu().pin_memory(), gamma=g.gamma.cpu().pin_memory(), W=g.W.cpu().pin_memory(),
@@ -236,10 +233,7 @@ def run_ours(args):
         step()
     e1.record(stream)
     barrier()
-    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_value = world * elements * e2e_steps / (float(t2.item()) * 1e-3)
+    e2e_value = replica_throughput(elements, e2e_steps, world, max_over_ranks(e0.elapsed_time(e1), device="cuda"))
 
     # ---- roofline of the dominant kernel: the FP8 weight-gradient contraction with the fused
     # shifted-sum epilogue, timed alone with CUDA events on the launching stream

@@ -90,3 +90,23 @@ class NormLinearGpu:
         d.forward_mode = b.ROUND_STOCHASTIC if inp.forward_mode == "sr" else b.ROUND_NEAREST
         d.seed, d.tensor_id, d.policy_mask = inp.seed, self.tensor_id, policy_mask
         return d
+
+
+# ------------------------------------------------------------------ replica timing protocol
+
+
+def max_over_ranks(ms: float, device="cpu") -> float:
+    """Largest step time over all ranks (the job is as slow as its slowest replica).  Single
+    process: the value itself."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(elements_per_step: int, steps: int, world: int, ms_total_max: float) -> float:
+    """Whole-job throughput of `world` independent replicas, each doing `steps` steps of
+    `elements_per_step` units, when the slowest replica took `ms_total_max` milliseconds."""
+    return world * elements_per_step * steps / (ms_total_max * 1e-3)
