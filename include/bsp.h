@@ -44,7 +44,8 @@ typedef enum {
   BSP_ERR_WORKSPACE = 4,    /* workspace missing or too small                             */
   BSP_ERR_NONFINITE = 5,    /* (diag.status) NaN or infinity met in an input              */
   BSP_ERR_TIMEOUT = 6,      /* (diag.status) a bounded device-side wait ran out           */
-  BSP_ERR_CUDA = 7          /* a CUDA runtime or driver call failed                       */
+  BSP_ERR_CUDA = 7,         /* a CUDA runtime or driver call failed                       */
+  BSP_ERR_TOO_LARGE = 8     /* problem exceeds the fixed capacity of a no-allocation entry */
 } bsp_status_t;
 
 typedef enum { BSP_E4M3 = 0, BSP_E5M2 = 1 } bsp_format_t;
@@ -205,6 +206,39 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
                  int gain_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key,
                  float* dgamma, float* dbeta, float* dx, void* ws, size_t ws_bytes,
                  bsp_diag_t* diag, void* stream);
+
+/* bsp_norm_bwd for callers that cannot hand over a workspace.  (The paper has no counterpart: this
+ * is a packaging variant of the entry point above, same arithmetic, same results.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- a plug-in inside a host
+ * application that reserved the whole GPU for its own pool at start-up and gives extensions no
+ * allocator; a latency-critical loop where cudaMalloc's implicit device-wide synchronisation and
+ * unbounded duration are not acceptable; a process running under a hard device-memory quota fixed
+ * at launch.  Such callers still own their inputs and outputs, but have nowhere to get scratch.
+ *
+ * What it does instead: the column partials that bsp_norm_bwd keeps in `ws` go to a fixed 20 MiB
+ * array inside the library's device image (BSP_NORM_BWD_NOALLOC_CAPACITY_BYTES).  Every GPU on
+ * which the library is loaded holds that array until the process exits, used or not.  The call
+ * never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ * Limits and rules:
+ *  - the problem must satisfy bsp_norm_bwd_workspace_bytes(T, C) <= the capacity (true for every
+ *    T when C <= 4096, and for T <= 320 when C = 8192); otherwise BSP_ERR_TOO_LARGE is returned
+ *    before anything is launched and no output is touched;
+ *  - the first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress, with that device current) and caches it; make that first call during
+ *    set-up, before any stream capture is begun;
+ *  - the array is shared by all calls and keeps whatever the last call wrote.  This pass writes
+ *    every partial it later reads, so nothing needs clearing between calls -- but two calls that
+ *    overlap on the GPU (different streams, or threads issuing concurrently) race on it and
+ *    corrupt each other's sums.  Serialise them, or use bsp_norm_bwd with separate workspaces.
+ * Arguments, outputs and error behaviour are otherwise those of bsp_norm_bwd. */
+#define BSP_NORM_BWD_NOALLOC_CAPACITY_BYTES ((size_t)20 << 20)
+int bsp_norm_bwd_noalloc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                         const float* beta, const float* rstd, const float* mean, const void* du,
+                         int du_dt, int gain_read, const uint8_t* u_codes, bsp_quant_t q,
+                         bsp_key_t key, float* dgamma, float* dbeta, float* dx, bsp_diag_t* diag,
+                         void* stream);
 
 /* K fresh draws of the gain use in one pass over x and du: for draw k in [draw0, draw0+K) the
  * gain gradient g_k is formed as in bsp_norm_bwd (policy N, key.draw = k) and the shifted sums

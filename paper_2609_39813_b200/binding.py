@@ -12,7 +12,8 @@ import os
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libbsp.so")
 
-OK, ERR_ARG, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA = range(8)
+OK, ERR_ARG, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA, ERR_TOO_LARGE = range(9)
+NORM_BWD_NOALLOC_CAPACITY_BYTES = 20 << 20
 E4M3, E5M2 = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 READ_ORIGINAL, READ_FORWARD, READ_FRESH = 0, 1, 2
@@ -83,6 +84,8 @@ _SIGNATURES = {
     "bsp_norm_bwd_workspace_bytes": (_SZ, [_I64, _I64]),
     "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
                           _P, _SZ, _P, _P]),
+    "bsp_norm_bwd_noalloc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
+                                  _P, _P]),
     "bsp_norm_gain_mc_workspace_bytes": (_SZ, [_I64, _I64, _I]),
     "bsp_norm_gain_mc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, Quant, Key, _I, _I, _P, _P, _P,
                               _P, _SZ, _P, _P]),
@@ -260,6 +263,17 @@ def bsp_norm_bwd(kind, x, T, Cc, gamma, beta, rstd, mean, du, gain_read, u_codes
                              ptr(du), dtype_code(du), gain_read, ptr(u_codes), q, k, ptr(dgamma), ptr(dbeta),
                              ptr(dx), ptr(ws), ws.numel() if ws is not None else 0, ptr(diag),
                              stream if stream is not None else cur_stream()), "bsp_norm_bwd")
+
+
+def bsp_norm_bwd_noalloc(kind, x, T, Cc, gamma, beta, rstd, mean, du, gain_read, u_codes, q: Quant, k: Key,
+                         dgamma, dbeta, dx, diag=None, stream=None):
+    """bsp_norm_bwd without a workspace argument: scratch is the library's own fixed device array
+    (for callers that may not allocate device memory).  Raises BspError(ERR_TOO_LARGE) when the
+    problem does not fit NORM_BWD_NOALLOC_CAPACITY_BYTES.  Calls that overlap on the GPU race."""
+    check(lib().bsp_norm_bwd_noalloc(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd),
+                                     ptr(mean), ptr(du), dtype_code(du), gain_read, ptr(u_codes), q, k,
+                                     ptr(dgamma), ptr(dbeta), ptr(dx), ptr(diag),
+                                     stream if stream is not None else cur_stream()), "bsp_norm_bwd_noalloc")
 
 
 def bsp_norm_gain_mc_workspace_bytes(T, Cc, K):

@@ -149,6 +149,7 @@ const char* bsp_status_string(int status) {
     case BSP_ERR_NONFINITE: return "non-finite value met in an input";
     case BSP_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case BSP_ERR_CUDA: return "CUDA runtime or driver call failed";
+    case BSP_ERR_TOO_LARGE: return "problem exceeds the fixed scratch capacity of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -5,6 +5,8 @@
 // blocks by a second, deterministic kernel.  HBM-bound.
 // gain_mc_kernel: x and du are read once for all K draws; every draw costs one Philox block and
 // four stochastic roundings per four elements, all in registers.  ALU-bound.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace bsp {
@@ -438,6 +440,59 @@ int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, cons
     BSP_LAUNCH_CHECK();
   }
   return BSP_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------- no-allocation variant
+
+namespace bsp {
+
+// Fixed scratch of bsp_norm_bwd_noalloc: lives in the library's device image, so every GPU that
+// loads the library carries these 20 MiB until the process exits.  In host code the symbol below is
+// only a handle; its device address is resolved with cudaGetSymbolAddress once per device.
+constexpr size_t kNoAllocScratchBytes = BSP_NORM_BWD_NOALLOC_CAPACITY_BYTES;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_noalloc_ptr[kMaxDevices];          // resolved device addresses, by device ordinal
+static std::mutex g_noalloc_mutex;
+
+// Device address of the scratch array on the current device (resolved on first use).
+static int noalloc_scratch(void** out) {
+  int dev = -1;
+  BSP_CHECK_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return BSP_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    BSP_CHECK_CUDA(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (p == nullptr || (reinterpret_cast<uintptr_t>(p) & 255u)) return BSP_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return BSP_OK;
+}
+
+}  // namespace bsp
+
+extern "C" {
+
+int bsp_norm_bwd_noalloc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                         const float* beta, const float* rstd, const float* mean, const void* du, int du_dt,
+                         int gain_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key, float* dgamma,
+                         float* dbeta, float* dx, bsp_diag_t* diag, void* stream) {
+  // size check first: pure host arithmetic, nothing is touched when the problem does not fit
+  if (T < 0 || C <= 0) return BSP_ERR_ARG;
+  const size_t need = bsp_norm_bwd_workspace_bytes(T, C);
+  if (need > bsp::kNoAllocScratchBytes) return BSP_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  const int rc = bsp::noalloc_scratch(&scratch);
+  if (rc != BSP_OK) return rc;
+  // The column partials this pass keeps in scratch are written in full before they are read, so
+  // whatever an earlier call left in the array is harmless and nothing has to be cleared.
+  return bsp_norm_bwd(kind, x, dt, T, C, gamma, beta, rstd, mean, du, du_dt, gain_read, u_codes, q, key, dgamma,
+                      dbeta, dx, scratch, bsp::kNoAllocScratchBytes, diag, stream);
 }
 
 }  // extern "C"
