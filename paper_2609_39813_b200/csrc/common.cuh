@@ -53,12 +53,12 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
   constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
 #pragma unroll
   for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
-    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ k0;
-    const uint32_t n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += W0; k1 += W1;
+    // one 32x32->64 multiply per lane pair (mul.wide.u32), one three-input XOR per new word
+    const uint64_t p0 = (uint64_t)M0 * c0;
+    const uint64_t p1 = (uint64_t)M1 * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ (k0 + (uint32_t)r * W0);
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ (k1 + (uint32_t)r * W1);
+    c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
 }
@@ -78,12 +78,14 @@ template <int FMT> struct F8;
 template <> struct F8<BSP_E4M3> {
   static constexpr int MB = 3, EMIN = -6, BIAS = 7;
   static constexpr uint32_t FMAX_BITS = 0x43E00000u;   // 448.0f
+  static constexpr uint32_t MINNORM_BITS = 0x3C800000u;   // 2^-6
   static constexpr uint32_t TOP = 0x7Eu;
   static constexpr uint32_t EMASK = 0xFu;
 };
 template <> struct F8<BSP_E5M2> {
   static constexpr int MB = 2, EMIN = -14, BIAS = 15;
   static constexpr uint32_t FMAX_BITS = 0x47600000u;   // 57344.0f
+  static constexpr uint32_t MINNORM_BITS = 0x38800000u;   // 2^-14
   static constexpr uint32_t TOP = 0x7Bu;
   static constexpr uint32_t EMASK = 0x1Fu;
 };
@@ -107,16 +109,13 @@ __device__ __forceinline__ uint32_t f8_encode(float v, uint32_t U, DiagCounters&
     if (a == 0x7F800000u) dc.nonfinite++; else if (a > F::FMAX_BITS) dc.sat++;
     return sign | F::TOP;
   }
-  const uint32_t efield = a >> 23;
-  if (efield == 0) return sign;                                           // FP32 zero / denormal
-  const int E = (int)efield - 127;
-  const uint32_t sig = (a & 0x7FFFFFu) | 0x800000u;
   uint32_t base, up;
-  if (E >= F::EMIN) {
+  if (a >= F::MINNORM_BITS) {
+    // normal range of the format: drop d low mantissa bits of the FP32 pattern
     constexpr int d = 23 - F::MB;
-    const uint32_t rem = sig & ((1u << d) - 1u);
-    const uint32_t n = sig >> d;                                           // in [2^MB, 2^(MB+1))
-    base = ((uint32_t)(E + F::BIAS) << F::MB) | (n & ((1u << F::MB) - 1u));
+    const uint32_t rem = a & ((1u << d) - 1u);
+    const uint32_t n = a >> d;                                             // exponent and kept mantissa
+    base = n - ((uint32_t)(127 - F::BIAS) << F::MB);                       // re-bias the exponent
     if (STOCHASTIC) {
       up = U < (rem << (32 - d));
     } else {
@@ -124,20 +123,45 @@ __device__ __forceinline__ uint32_t f8_encode(float v, uint32_t U, DiagCounters&
       up = (rem > half) | ((rem == half) & (n & 1u));
     }
   } else {
-    int d = 23 - F::MB + (F::EMIN - E);
-    d = d > 60 ? 60 : d;
-    const uint64_t s64 = sig;
-    const uint64_t rem = s64 & ((1ull << d) - 1ull);
-    const uint32_t n = (uint32_t)(s64 >> d);
+    // subnormal range: uniform grid of step 2^(EMIN-MB).  t = |v| / step is an exact FP32 product
+    // (a power-of-two scaling), n = floor(t) < 2^MB, f = t - n exact, floor(f * 2^32) exact.
+    const float t = __uint_as_float(a) * __uint_as_float((uint32_t)(F::MB - F::EMIN + 127) << 23);
+    const uint32_t n = (uint32_t)t;
+    const float f = t - (float)n;
     base = n;
     if (STOCHASTIC) {
-      up = (uint64_t)U < ((rem << 32) >> d);
+      up = U < __float2uint_rd(f * 4294967296.0f);
     } else {
-      const uint64_t half = 1ull << (d - 1);
-      up = (rem > half) | ((rem == half) & (n & 1u));
+      up = (f > 0.5f) | ((f == 0.5f) & (n & 1u));
     }
   }
   return sign | (base + up);
+}
+
+// Value of the stochastic rounding of v as FP32, i.e. decode(encode_SR(v)) without the detour
+// through the code: in the normal range the FP32 pattern is truncated and bumped in place.
+template <int FMT>
+__device__ __forceinline__ float f8_sr_value(float v, uint32_t U) {
+  using F = F8<FMT>;
+  const uint32_t b = __float_as_uint(v);
+  const uint32_t a = b & 0x7FFFFFFFu;
+  const uint32_t s = b & 0x80000000u;
+  if (a >= F::FMAX_BITS) {
+    if (a > 0x7F800000u) return __uint_as_float(0x7FC00000u);
+    return __uint_as_float(s | F::FMAX_BITS);
+  }
+  if (a >= F::MINNORM_BITS) {
+    constexpr int d = 23 - F::MB;
+    const uint32_t rem = a & ((1u << d) - 1u);
+    const uint32_t up = U < (rem << (32 - d));
+    return __uint_as_float(s | ((a - rem) + (up << d)));
+  }
+  const float t = __uint_as_float(a) * __uint_as_float((uint32_t)(F::MB - F::EMIN + 127) << 23);
+  const uint32_t n = (uint32_t)t;
+  const float f = t - (float)n;
+  const uint32_t up = U < __float2uint_rd(f * 4294967296.0f);
+  const float mag = (float)(n + up) * __uint_as_float((uint32_t)(F::EMIN - F::MB + 127) << 23);
+  return __uint_as_float(s | __float_as_uint(mag));
 }
 
 // Exact FP32 value of a code.

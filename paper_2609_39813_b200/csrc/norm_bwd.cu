@@ -11,22 +11,8 @@
 
 namespace bsp {
 
-// Value of the stochastic rounding of v (scaled FP32 value) as FP32, i.e. decode(encode_SR(v)).
 template <int FMT>
-__device__ __forceinline__ float sr_value(float v, uint32_t U) {
-  using F = F8<FMT>;
-  const uint32_t b = __float_as_uint(v);
-  const uint32_t a = b & 0x7FFFFFFFu;
-  const int E = (int)(a >> 23) - 127;
-  if (a < F::FMAX_BITS && E >= F::EMIN) {
-    constexpr int d = 23 - F::MB;
-    const uint32_t rem = a & ((1u << d) - 1u);
-    const uint32_t up = U < (rem << (32 - d));
-    return __uint_as_float((b & 0x80000000u) | ((a - rem) + (up << d)));
-  }
-  DiagCounters dc;
-  return f8_decode<FMT>(f8_encode<FMT, true>(v, U, dc));
-}
+__device__ __forceinline__ float sr_value(float v, uint32_t U) { return f8_sr_value<FMT>(v, U); }
 
 // ------------------------------------------------------------------------------- norm backward
 
@@ -172,13 +158,20 @@ constexpr int kMcRows = 8;              // rows per thread
 constexpr int kMcSlab = 8 * kMcRows;    // rows per block (8 warps)
 constexpr int kMcCols = 128;            // columns per block (32 lanes x 4)
 constexpr int kMcChunk = 64;            // draws per launch
+constexpr size_t kMcSmemBytes = (size_t)2 * kMcRows * 256 * sizeof(float4);   // values + weights of a slab
 
 template <int DT, int DU_DT, int FMT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
                int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */) {
+  // The slab's scaled values and weights live in shared memory (each thread reads back only what
+  // it wrote), which keeps the register count low enough for three blocks per SM: the draw loop
+  // is a chain of dependent integer multiplies, and it is occupancy that hides their latency.
+  extern __shared__ __align__(16) float4 mc_smem[];
+  float4* sv = mc_smem;                         // [kMcRows][256]
+  float4* sw = mc_smem + kMcRows * 256;         // [kMcRows][256]
   __shared__ __align__(16) float red[2][8][kMcCols];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t c = (int64_t)blockIdx.x * kMcCols + lane * 4;
@@ -192,17 +185,16 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
     g4 = __ldg(reinterpret_cast<const float4*>(gamma + c));
     if (kind == BSP_LAYERNORM) b4 = __ldg(reinterpret_cast<const float4*>(beta + c));
   }
-  float v[kMcRows][4], wgt[kMcRows][4];
-  uint64_t q[kMcRows];
-#pragma unroll
+  // generator block index of this thread's four columns in row (slab*kMcSlab + warp + 8*i) is
+  // q0 + i*qstep; rows beyond T keep v = wgt = 0 and contribute nothing whatever word they draw
+  const uint64_t q0 = (uint64_t)((slab * kMcSlab + warp) * C + (col_ok ? c : 0)) >> 2;
+  const uint64_t qstep = (uint64_t)(2 * C);
+#pragma unroll 1
   for (int i = 0; i < kMcRows; ++i) {
     const int64_t r = slab * kMcSlab + warp + 8 * i;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { v[i][e] = 0.f; wgt[i][e] = 0.f; }
-    q[i] = 0;
+    float v[4] = {0.f, 0.f, 0.f, 0.f}, wgt[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < T && col_ok) {
       const size_t i0 = (size_t)r * C + c;
-      q[i] = (uint64_t)i0 >> 2;
       const float4 xv = load4<DT>(x, i0);
       const float4 dv = load4<DU_DT>(du, i0);
       const float rs = __ldg(rstd + r);
@@ -216,23 +208,28 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
         float u;
         if (kind == BSP_RMSNORM) u = __fmul_rn(__fmul_rn(xs[e], rs), gg[e]);
         else u = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xs[e], mu), rs), gg[e]), bb[e]);
-        v[i][e] = __fmul_rn(u, scale);
-        wgt[i][e] = __fdiv_rn(ds[e], gg[e]);
+        v[e] = __fmul_rn(u, scale);
+        wgt[e] = __fdiv_rn(ds[e], gg[e]);
       }
     }
+    sv[i * 256 + tid] = make_float4(v[0], v[1], v[2], v[3]);
+    sw[i * 256 + tid] = make_float4(wgt[0], wgt[1], wgt[2], wgt[3]);
   }
   const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
   for (int k = 0; k < ndraws; ++k) {
     const uint32_t draw = (uint32_t)(draw_begin + k);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
+#pragma unroll 2
     for (int i = 0; i < kMcRows; ++i) {
-      const uint4 w = philox_block(key, q[i], draw);
+      const uint4 w = philox_block(key, q0 + (uint64_t)i * qstep, draw);
+      const float4 v4 = sv[i * 256 + tid], w4 = sw[i * 256 + tid];
       const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+      const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+      const float wg[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float val = sr_value<FMT>(v[i][e], ww[e]);
-        acc[e] = fmaf(fmaf(val, inv_scale, -bb[e]), wgt[i][e], acc[e]);
+        const float val = sr_value<FMT>(vv[e], ww[e]);
+        acc[e] = fmaf(fmaf(val, inv_scale, -bb[e]), wg[e], acc[e]);
       }
     }
     const int buf = k & 1;
@@ -417,8 +414,13 @@ int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, cons
     if (nslabs > 0) {
       dim3 grid((unsigned)((C + kMcCols - 1) / kMcCols), (unsigned)nslabs);
 #define BSP_GM(DT, DU, FMT)                                                                                     \
-  gain_mc_kernel<DT, DU, FMT><<<grid, 256, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du, q.scale,        \
-                                                     q.scale_dev, pk, draw0 + kb, nd, partial)
+  do {                                                                                                          \
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(gain_mc_kernel<DT, DU, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                        (int)kMcSmemBytes));                                                    \
+    gain_mc_kernel<DT, DU, FMT><<<grid, 256, kMcSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
+                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd,      \
+                                                                 partial);                                      \
+  } while (0)
       if (q.fmt == BSP_E4M3) {
         if (dt == BSP_F32 && du_dt == BSP_F32) BSP_GM(BSP_F32, BSP_F32, BSP_E4M3);
         else if (dt == BSP_F32) BSP_GM(BSP_F32, BSP_BF16, BSP_E4M3);
