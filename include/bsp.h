@@ -267,6 +267,17 @@ int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t,
                      const float* mc_ref, float* mc_S1, float* mc_S2, void* ws, size_t ws_bytes,
                      bsp_diag_t* diag, void* stream);
 
+/* The contraction primitive behind the weight gradient, the input gradient and the attention
+ * products (helper, not an operator of the paper): C[M,N] (FP32, pitch ldc) = alpha * A * B^T on
+ * the tensor cores with FP32 accumulation.  elem = 1: FP8 codes (a_fmt / b_fmt = bsp_format_t,
+ * any combination), elem = 2: bf16.  An operand is either K-major -- stored [rows][K], pitch ld --
+ * or, with its *_mn flag set, MN-major -- stored [K][rows], pitch ld -- so a product over the
+ * leading dimension of two row-major matrices (dW = dY^T X) needs no transposed copy.  Pitches are
+ * in elements; pitch * elem must be a multiple of 16 bytes; ldc a multiple of 4. */
+int bsp_gemm(int64_t M, int64_t N, int64_t K, int elem, const void* A, int64_t lda, int a_mn, int a_fmt,
+             const void* B, int64_t ldb, int b_mn, int b_fmt, float alpha, float* C, int64_t ldc,
+             bsp_diag_t* diag, void* stream);
+
 /* The weight use under n_draws fresh roundings in one launch (Section "Each use has a checkable
  * requirement": the substitute's own draw is averaged with the forward and the incoming gradient
  * held fixed).  x_t_draws holds n_draws code matrices [C * ld_t] back to back (as written by

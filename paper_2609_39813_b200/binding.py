@@ -80,6 +80,7 @@ _SIGNATURES = {
     "bsp_norm_stats": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _F, _P, _P, _P, _P, _P]),
     "bsp_norm_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, Quant, Key, _P, _P, _I64, _P, _P, _P, _P]),
     "bsp_norm_fwd_draws": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, Quant, Key, _I, _I, _P, _I64, _P]),
+    "bsp_gemm": (_I, [_I64, _I64, _I64, _I, _P, _I64, _I, _I, _P, _I64, _I, _I, _F, _P, _I64, _P, _P]),
     "bsp_linear_wgrad_mc": (_I, [_I64, _I64, _I64, _P, Quant, _P, Quant, _I64, _I, _P, _P, _P, _P, _P]),
     "bsp_norm_bwd_workspace_bytes": (_SZ, [_I64, _I64]),
     "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
@@ -244,6 +245,11 @@ def bsp_norm_fwd_draws(kind, x, T, Cc, gamma, beta, rstd, mean, q: Quant, k: Key
     check(lib().bsp_norm_fwd_draws(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
                                    q, k, draw0, n_draws, ptr(u_codes_t_draws), ld_t,
                                    stream if stream is not None else cur_stream()), "bsp_norm_fwd_draws")
+
+
+def bsp_gemm(M, N, K, elem, A, lda, a_mn, a_fmt, B, ldb, b_mn, b_fmt, alpha, Cout, ldc, diag=None, stream=None):
+    check(lib().bsp_gemm(M, N, K, elem, ptr(A), lda, int(a_mn), a_fmt, ptr(B), ldb, int(b_mn), b_fmt, alpha,
+                         ptr(Cout), ldc, ptr(diag), stream if stream is not None else cur_stream()), "bsp_gemm")
 
 
 def bsp_linear_wgrad_mc(T, O, Cc, dy_codes_t, q_dy: Quant, x_t_draws, q_x: Quant, ld_t, n_draws, g_ref, S1, S2,

@@ -138,6 +138,19 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
   return d;
 }
 
+// The same for an MN-major operand, i.e. a tile of a matrix stored [K rows][MN columns]: TMA writes
+// one atom per 128 bytes of MN ([k rows][128 B], 128-byte swizzle); atoms follow each other
+// `atom_bytes` apart (leading byte offset), groups of eight k rows are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t smem_addr, uint32_t atom_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((atom_bytes >> 4) & 0x3FFFu) << 16;    // leading byte offset: next 128 B of MN
+  d |= (uint64_t)(1024u >> 4) << 32;                     // stride byte offset: next eight k rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
 // Instruction descriptor: FP32 accumulator, K-major A and B, M x N tile.
 // a_fmt / b_fmt: kind::f8f6f4 E4M3 = 0, E5M2 = 1; kind::f16 BF16 = 1.
 __host__ __device__ constexpr uint32_t make_idesc(uint32_t a_fmt, uint32_t b_fmt, uint32_t M, uint32_t N) {
@@ -157,6 +170,7 @@ struct GemmParams {
   int M, N, K;            // K in elements
   int nb;                 // batches of B (and of C in plain mode)
   int elem_bytes;         // 1 (FP8) or 2 (BF16)
+  int a_mn, b_mn;         // operand stored [K][M] / [K][N] (MN-major) instead of [M][K] / [N][K]
   uint32_t idesc;
   float sa, sb;           // operand scales; alpha = (1/sa) * (1/sb)
   const float* sa_dev;
@@ -217,8 +231,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t sa = tiles + s * kStageBytes, sb = sa + kABytes;
             mbar_expect_tx(full0 + 8 * s, kStageBytes);
-            tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * bk_elems, tm * BM);
-            tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * bk_elems, tn * BN, b);
+            if (!p.a_mn) {
+              tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * bk_elems, tm * BM);
+            } else {
+              // one box per 128 bytes of M: [bk_elems k rows][128 B]
+              for (int a = 0; a < BM * p.elem_bytes / 128; ++a)
+                tma_load_2d(sa + a * bk_elems * 128, &tmap_a, full0 + 8 * s, tm * BM + a * (128 / p.elem_bytes),
+                            kb * bk_elems);
+            }
+            if (!p.b_mn) {
+              tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * bk_elems, tn * BN, b);
+            } else {
+              for (int a = 0; a < BN * p.elem_bytes / 128; ++a)
+                tma_load_3d(sb + a * bk_elems * 128, &tmap_b, full0 + 8 * s, tn * BN + a * (128 / p.elem_bytes),
+                            kb * bk_elems, b);
+            }
           }
         }
       }
@@ -243,12 +270,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = tiles + s * kStageBytes, sb = sa + kABytes;
-            const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+            // K-major: one MMA advances 32 bytes along K inside the swizzle atom (+2 in 16-byte
+            // units).  MN-major: it advances 32/elem_bytes k rows of 128 bytes.
+            const uint32_t atom_bytes = (uint32_t)bk_elems * 128u;
+            const uint32_t mn_step = (32u / (uint32_t)p.elem_bytes) * 128u >> 4;
+            const uint64_t adesc = p.a_mn ? make_smem_desc_mn(sa, atom_bytes) : make_smem_desc(sa);
+            const uint64_t bdesc = p.b_mn ? make_smem_desc_mn(sb, atom_bytes) : make_smem_desc(sb);
+            const uint32_t astep = p.a_mn ? mn_step : 2u, bstep = p.b_mn ? mn_step : 2u;
 #pragma unroll
-            for (int k = 0; k < BKB / 32; ++k) {
-              // advance 32 bytes along K inside the swizzle atom: +2 in 16-byte address units
-              tc_mma<FP8>(tmem_d, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
-            }
+            for (int k = 0; k < BKB / 32; ++k)
+              tc_mma<FP8>(tmem_d, adesc + astep * k, bdesc + bstep * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
             tc_commit(empty0 + 8 * s);          // frees the stage when these MMAs have read it
           }
           if (ok) tc_commit(tfull0 + 8 * as);   // accumulator complete
@@ -611,9 +642,11 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// Tensor map over a K-major matrix [batch][rows][K] (row pitch ld elements), box = 128 bytes x box_rows.
+// Tensor map over an operand.  K-major: matrix [batch][rows][K] (row pitch ld elements), box =
+// 128 bytes of K x box_rows.  MN-major: matrix [batch][K][rows] (pitch ld), box = 128 bytes of MN x
+// (128 / elem_bytes) k rows.
 static int make_operand_map(CUtensorMap* map, const void* base, int elem_bytes, int64_t K, int64_t rows, int64_t ld,
-                            int64_t nbatch, int64_t batch_stride_elems, int box_rows) {
+                            int64_t nbatch, int64_t batch_stride_elems, int box_rows, bool mn_major = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return BSP_ERR_CUDA;
   const CUtensorMapDataType dt = elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
@@ -622,7 +655,11 @@ static int make_operand_map(CUtensorMap* map, const void* base, int elem_bytes, 
   cuuint32_t box[3] = {(cuuint32_t)(BKB / elem_bytes), (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   const cuuint32_t rank = nbatch > 0 ? 3 : 2;
-  if (rank == 3 && nbatch == 1) gstr[1] = (cuuint64_t)rows * ld * elem_bytes;   // any valid stride
+  if (mn_major) {
+    gdim[0] = (cuuint64_t)rows; gdim[1] = (cuuint64_t)K;
+    box[0] = (cuuint32_t)(128 / elem_bytes); box[1] = (cuuint32_t)(BKB / elem_bytes);
+  }
+  if (rank == 3 && nbatch == 1) gstr[1] = (cuuint64_t)gdim[1] * ld * elem_bytes;   // any valid stride
   CUresult r = fn(map, dt, rank, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
@@ -643,8 +680,11 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
   if ((g.b_batch_stride * eb) % 16 != 0) return BSP_ERR_ALIGN;
   GemmParams p;
   p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K; p.nb = g.nb; p.elem_bytes = eb;
+  p.a_mn = g.a_mn ? 1 : 0; p.b_mn = g.b_mn ? 1 : 0;
   p.idesc = g.fp8 ? make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, BN)
                   : make_idesc(1u, 1u, BM, BN);
+  p.idesc |= (g.a_mn ? 1u << 15 : 0u) | (g.b_mn ? 1u << 16 : 0u);     // operand major bits
+  if ((g.a_mn || g.b_mn) && (g.mode == EPI_MC || simt_forced())) return BSP_ERR_UNSUPPORTED;
   p.sa = g.sa; p.sb = g.sb; p.sa_dev = g.sa_dev; p.sb_dev = g.sb_dev;
   p.mode = g.mode; p.C = g.C; p.ldc = g.ldc; p.ref = g.ref; p.S1 = g.S1; p.S2 = g.S2; p.diag = g.diag;
 
@@ -674,7 +714,7 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
       nsm = v;
   }
   CUtensorMap ma, mb;
-  int rc = make_operand_map(&ma, g.A, eb, g.K, g.M, g.lda, 0, 0, BM);
+  int rc = make_operand_map(&ma, g.A, eb, g.K, g.M, g.lda, 0, 0, BM, g.a_mn);
   if (rc != BSP_OK) return rc;
 
   if (g.mode == EPI_MC) {
@@ -696,7 +736,7 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     return BSP_OK;
   }
 
-  rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN);
+  rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN, g.b_mn);
   if (rc != BSP_OK) return rc;
   static bool attr_set[2] = {false, false};
   if (!attr_set[g.fp8 ? 1 : 0]) {
@@ -808,6 +848,21 @@ int bsp_linear_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t,
     g.fp8 = true; g.A = dy_codes_t; g.B = x_t; g.a_fmt = q_dy.fmt; g.b_fmt = q_x.fmt;
   }
   return gemm_run(g, st);
+}
+
+int bsp_gemm(int64_t M, int64_t N, int64_t K, int elem, const void* A, int64_t lda, int a_mn, int a_fmt,
+             const void* B, int64_t ldb, int b_mn, int b_fmt, float alpha, float* C, int64_t ldc, bsp_diag_t* diag,
+             void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || (elem != 1 && elem != 2) || !valid_enum(a_fmt, 1) || !valid_enum(b_fmt, 1))
+    return BSP_ERR_ARG;
+  if (M == 0 || N == 0) return BSP_OK;
+  if (!A || !B || !C || alpha == 0.f) return BSP_ERR_ARG;
+  GemmArgs g;
+  g.M = M; g.N = N; g.K = K; g.nb = 1; g.fp8 = elem == 1; g.a_fmt = a_fmt; g.b_fmt = b_fmt;
+  g.A = A; g.B = B; g.a_mn = a_mn != 0; g.b_mn = b_mn != 0; g.lda = lda; g.ldb = ldb;
+  g.b_batch_stride = (b_mn ? K : N) * ldb;
+  g.sa = 1.0f / alpha; g.sb = 1.0f; g.mode = EPI_STORE_F32; g.C = C; g.ldc = ldc; g.diag = diag;
+  return gemm_run(g, (cudaStream_t)stream);
 }
 
 int bsp_linear_wgrad_mc(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy,

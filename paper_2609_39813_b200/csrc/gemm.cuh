@@ -20,6 +20,7 @@ struct GemmArgs {
   int a_fmt = 0, b_fmt = 0;            // bsp_format_t of A and B when fp8
   const void* A = nullptr;
   const void* B = nullptr;
+  bool a_mn = false, b_mn = false;     // operand stored [K][M] / [K][N] (pitch lda / ldb) instead
   int64_t lda = 0, ldb = 0;            // row pitch in elements
   int64_t b_batch_stride = 0;          // elements between batches of B
   float sa = 1.f, sb = 1.f;
