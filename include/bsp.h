@@ -298,8 +298,52 @@ int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, b
                      bsp_diag_t* diag, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Causal softmax attention (Section "Same rounding distribution, opposite outcomes"):
+ * P = softmax(c Q K^T), O = P V; dV = P^T dO, dP = dO V^T, dS = P o (dP - D),
+ * D = rowsum(P o dP) = rowsum(dO o O); dQ = c dS K, dK = c dS^T Q.  The forward rounds O before the
+ * next layer consumes it; the correction term D is the one use of the saved output, and reading a
+ * copy O + E adds rowsum(dO o E) (Eq. dterm).  Tensors are [B, H, S, Dh] row-major, bf16 inputs
+ * (dt = BSP_BF16), Dh = 64, FP32 outputs; lse, D are [B, H, S].  BF16 tensor-core operands (P and
+ * dS are rounded to bf16 for their products); the FP8-operand variant of Appendix "The forks" is
+ * not built (fp8_operands != 0 returns BSP_ERR_UNSUPPORTED).
+ * ------------------------------------------------------------------------------------------ */
+
+/* Forward statistics from the operands exactly as the backward will see them: o = P V (FP32, the
+ * "original" output the store rounds) and lse = log sum_j exp(c q.k_j). */
+int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                       const void* k, const void* v, int dt, float* o, float* lse, bsp_diag_t* diag,
+                       void* stream);
+
+/* The D use: d_out[d][b,h,i] = sum_j dO[b,h,i,j] * O_copy[b,h,i,j] for n_draws draws, with
+ * O_copy = o_orig (U), decode(o_codes)/o_scales[b,h] (R), or a fresh stochastic rounding of
+ * fl32(o_orig * o_scales[b,h]) in o_fmt under (key, draw0 + d) (N).  U and R write one draw.
+ * dO: dt[B,H,S,Dh]; o_scales: one scale per (b,h) slice. */
+int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig,
+                   const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key,
+                   int draw0, int n_draws, float* d_out, bsp_diag_t* diag, void* stream);
+
+/* Backward given D (dterm[B,H,S]).  dk and dv are produced together (both NULL or both set);
+ * dq may be NULL. */
+int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                       const void* k, const void* v, const void* dO, int dt, const float* lse,
+                       const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
+                       void* stream);
+
+/* Backward under a read policy at the D use: bsp_attn_dterm (draw key.draw) into d_out[B,H,S]
+ * (required), then bsp_attn_bwd_dterm. */
+int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands,
+                 const void* q, const void* k, const void* v, const void* dO, int dt, const float* lse,
+                 const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt,
+                 int d_read, bsp_key_t key, float* dq, float* dk, float* dv, float* d_out,
+                 bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Monte-Carlo reduction (Section "Each use has a checkable requirement").
  * ------------------------------------------------------------------------------------------ */
+
+/* One draw's contribution to the shifted sums, elementwise: S1 += g - g_ref, S2 += (g - g_ref)^2
+ * (n a multiple of 4).  Used where the producing kernel has no fused accumulation. */
+int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, size_t n, void* stream);
 
 /* Reduces per-element shifted sums to the statistics of bsp_use_result_t and the verdict.
  * fresh = 0: deterministic read, `g` holds the gradient itself (S2 ignored, K = 1).

@@ -60,10 +60,13 @@ def forward_output(q, k, v, c: float, causal: bool = True):
 
 
 def backward(q, k, v, dO, c: float, o_copy, causal: bool = True, fp8_operands: bool = False,
-             scale_p: float = 256.0, scale_ds=None):
+             scale_p: float = 256.0, scale_ds=None, operand_round=None):
     """Attention backward for one slice with D = rowsum(dO o o_copy).
 
     BF16-operand mode (fp8_operands False): every product in float64 on the given operands.
+    `operand_round` (e.g. rounding to bf16), when given, is applied to the two computed operands
+    of the last three products -- P before dV = P^T dO, dS before dQ = c dS K and dK = c dS^T Q --
+    as a tensor-core contraction in that operand type does; None keeps them unrounded.
     FP8-operand mode: q, k, v must already be the dequantised E4M3 operands and dO the
     dequantised E5M2 gradient; P_q = RN_E4M3(P scale_p) / scale_p feeds dV, and
     dS_q = RN_E5M2(dS scale_ds) / scale_ds feeds dQ and dK.
@@ -82,6 +85,8 @@ def backward(q, k, v, dO, c: float, o_copy, causal: bool = True, fp8_operands: b
         if scale_ds is None:
             raise ValueError("the FP8-operand mode needs the caller's dS scale")
         dS_mm, _, _, _ = quantise_rn(dS, fp8.E5M2, scale=scale_ds)
+    elif operand_round is not None:
+        p_dv, dS_mm = operand_round(p), operand_round(dS)
     else:
         p_dv, dS_mm = p, dS
     dv = p_dv.T @ dO

@@ -142,20 +142,24 @@ def attention_d_copy(prep, policy, seed, draw, stream=philox.STREAM_ATTN_D):
     return norm.read_value(codes, prep["store_fmt"], prep["inv_scale"])
 
 
-def attention_d_use(q, k, v, dO, c, prep, policy, K, seed, causal=True, outputs=("D", "dq", "dk", "dv")):
+def attention_d_use(q, k, v, dO, c, prep, policy, K, seed, causal=True, outputs=("D", "dq", "dk", "dv"),
+                    operand_round=None):
     """Attention backward (BF16-operand mode) under one read at the D use, against the
     reference (D reads the original output).  Returns {name: dict(ref, mean, m2, stats)}."""
-    ref = attention.backward(q, k, v, dO, c, attention_d_copy(prep, U, seed, 0), causal)
+    ref = attention.backward(q, k, v, dO, c, attention_d_copy(prep, U, seed, 0), causal,
+                             operand_round=operand_round)
     out = {}
     if policy in (U, R):
-        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, policy, seed, 0), causal)
+        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, policy, seed, 0), causal,
+                               operand_round=operand_round)
         for name in outputs:
             out[name] = dict(ref=ref[name], mean=g[name], m2=None,
                              stats=mc.statistics(g[name], None, 1, ref[name], False))
         return out
     accs = {name: mc.Welford(ref[name].shape) for name in outputs}
     for kk in range(K):
-        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, N, seed, kk), causal)
+        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, N, seed, kk), causal,
+                               operand_round=operand_round)
         for name in outputs:
             accs[name].add(g[name])
     for name in outputs:

@@ -94,6 +94,12 @@ _SIGNATURES = {
     "bsp_linear_wgrad": (_I, [_I64, _I64, _I64, _P, Quant, _I, _P, Quant, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
     "bsp_linear_dgrad_workspace_bytes": (_SZ, [_I64, _I64, _I64]),
     "bsp_linear_dgrad": (_I, [_I64, _I64, _I64, _P, Quant, _P, _I, _P, _I, _P, _SZ, _P, _P]),
+    "bsp_attn_fwd_stats": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _I, _P, _P, _P, _P]),
+    "bsp_attn_dterm": (_I, [_I, _I, _I, _I, _P, _I, _P, _P, _P, _I, _I, Key, _I, _I, _P, _P, _P]),
+    "bsp_attn_bwd_dterm": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P]),
+    "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, _P, _P, _P, _P, _I, _I, Key, _P, _P, _P,
+                          _P, _P, _P]),
+    "bsp_mc_accumulate": (_I, [_P, _P, _P, _P, _SZ, _P]),
     "bsp_mc_stats_workspace_bytes": (_SZ, [_I64]),
     "bsp_mc_stats": (_I, [_P, _P, _P, _I64, _I, _I, C.POINTER(UseResult), _P, _SZ, _P]),
     "bsp_mc_check_workspace_bytes": (_SZ, [C.POINTER(NormLinearDesc), _I]),
@@ -313,6 +319,40 @@ def bsp_linear_dgrad(T, O, Cc, dy_codes, q_dy: Quant, W, du, ws, diag=None, stre
     check(lib().bsp_linear_dgrad(T, O, Cc, ptr(dy_codes), q_dy, ptr(W), dtype_code(W), ptr(du), dtype_code(du),
                                  ptr(ws), ws.numel() if ws is not None else 0, ptr(diag),
                                  stream if stream is not None else cur_stream()), "bsp_linear_dgrad")
+
+
+def _st(stream):
+    return stream if stream is not None else cur_stream()
+
+
+def bsp_attn_fwd_stats(B, H, S, Dh, causal, softmax_scale, q, k, v, o, lse, diag=None, stream=None):
+    check(lib().bsp_attn_fwd_stats(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), dtype_code(q),
+                                   ptr(o), ptr(lse), ptr(diag), _st(stream)), "bsp_attn_fwd_stats")
+
+
+def bsp_attn_dterm(B, H, S, Dh, dO, o_orig, o_codes, o_scales, o_fmt, d_read, k: Key, draw0, n_draws, d_out,
+                   diag=None, stream=None):
+    check(lib().bsp_attn_dterm(B, H, S, Dh, ptr(dO), dtype_code(dO), ptr(o_orig), ptr(o_codes), ptr(o_scales), o_fmt,
+                               d_read, k, draw0, n_draws, ptr(d_out), ptr(diag), _st(stream)), "bsp_attn_dterm")
+
+
+def bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, lse, dterm, dq, dk, dv, diag=None,
+                       stream=None):
+    check(lib().bsp_attn_bwd_dterm(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), ptr(dO),
+                                   dtype_code(q), ptr(lse), ptr(dterm), ptr(dq), ptr(dk), ptr(dv), ptr(diag),
+                                   _st(stream)), "bsp_attn_bwd_dterm")
+
+
+def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, lse, o_orig, o_codes, o_scales,
+                 o_fmt, d_read, key_: Key, dq, dk, dv, d_out, diag=None, stream=None):
+    check(lib().bsp_attn_bwd(B, H, S, Dh, int(causal), softmax_scale, int(fp8_operands), ptr(q), ptr(k), ptr(v),
+                             ptr(dO), dtype_code(q), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales), o_fmt,
+                             d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
+          "bsp_attn_bwd")
+
+
+def bsp_mc_accumulate(g, g_ref, S1, S2, n, stream=None):
+    check(lib().bsp_mc_accumulate(ptr(g), ptr(g_ref), ptr(S1), ptr(S2), n, _st(stream)), "bsp_mc_accumulate")
 
 
 def bsp_mc_stats_workspace_bytes(n):

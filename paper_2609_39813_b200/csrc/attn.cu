@@ -1,0 +1,550 @@
+// Causal softmax attention on the tensor cores: forward statistics and the backward whose
+// correction term D = rowsum(dO o O_copy) reads a copy of the saved output chosen by policy.
+//
+//   P = softmax(c Q K^T), O = P V;  dV = P^T dO, dP = dO V^T, dS = P o (dP - D),
+//   dQ = c dS K, dK = c dS^T Q.
+//
+// One kernel template, three modes, one CTA per (batch*head, 128-row block):
+//   AT_DKV  the CTA owns key block j: K_j, V_j resident, streams (Q_i, dO_i) for i >= j,
+//           accumulates dV_j and dK_j in tensor memory;
+//   AT_DQ   the CTA owns query block i: Q_i, dO_i resident, streams (K_j, V_j) for j <= i,
+//           accumulates dQ_i;
+//   AT_FWD  the CTA owns query block i: pass 1 over j gives the row log-sum-exp, pass 2 forms
+//           O_i = sum_j exp(S - LSE) V_j.
+// No cross-CTA reduction exists in any mode, so results are bit-reproducible.
+//
+// Per inner step: S = Q K^T and dP = dO V^T (128x128x64 each) land in TMEM columns [0,128) and
+// [128,256); eight softmax warps (two per TMEM lane quarter, 64 keys each) turn them into P and dS,
+// written as bf16 into shared memory in the 128-byte-swizzle layout; the products with P / dS then
+// read those buffers directly (MN-major A for dV and dK, K-major A for dQ and O) and the TMA-loaded
+// 128 x 64 tiles as MN-major B.  320 threads: warp 0 TMA, warp 1 MMA, warps 2..9 softmax + epilogue.
+// Head dimension 64, bf16 inputs, FP32 outputs.  Every wait is bounded.
+#include "common.cuh"
+#include "tc.cuh"
+
+namespace bsp {
+
+enum { AT_DKV = 0, AT_DQ = 1, AT_FWD = 2 };
+
+constexpr int AT_BLK = 128, AT_D = 64;
+constexpr int kAtTile = AT_BLK * AT_D * 2;        // 16 KB: one 128 x 64 bf16 tile
+constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
+constexpr int kAtThreads = 320;
+// shared memory: res0, res1, str[2][2], P, dS, barriers
+constexpr int kAtSmem = 2 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct AttnParams {
+  int BH, S, nblk;
+  int causal;
+  float c;                       // softmax scale
+  const float* lse;              // [BH*S]  (DKV, DQ: input; FWD: unused)
+  const float* dterm;            // [BH*S]  (DKV, DQ)
+  float* out0;                   // DKV: dV   DQ: dQ   FWD: O      [BH*S*64]
+  float* out1;                   // DKV: dK                         [BH*S*64]
+  float* lse_out;                // FWD
+  bsp_diag_t* diag;
+};
+
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kAtThreads, 1)
+attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  const uint32_t res0 = base, res1 = base + kAtTile;
+  const uint32_t str0 = base + 2 * kAtTile;                 // stage s: str0 + s*2*kAtTile (+kAtTile for the 2nd tile)
+  const uint32_t pbuf = base + 6 * kAtTile, dsbuf = pbuf + kAtPBytes;
+  const uint32_t bars = dsbuf + kAtPBytes;
+  // barriers: res_full, str_full[2], str_empty[2], sdp_full, sdp_free, pds_ready, pds_free, acc_full
+  const uint32_t b_res = bars, b_sfull = bars + 8, b_sempty = bars + 24, b_sdp_full = bars + 40,
+                 b_sdp_free = bars + 48, b_pds_ready = bars + 56, b_pds_free = bars + 64, b_acc = bars + 72;
+  uint8_t* gen = smem_raw + (base - raw);
+  uint8_t* bars_gen = gen + 6 * kAtTile + 2 * kAtPBytes;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 80);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 84);
+  float* xchg = reinterpret_cast<float*>(bars_gen + 96);    // FWD: [2][2][...] not used; see below
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // heavy blocks first: block rank 0 is the one with most inner steps
+  const int rank = blockIdx.x / p.BH, bh = blockIdx.x % p.BH;
+  int blk, it_begin, it_end;                                 // inner index range [it_begin, it_end)
+  if (MODE == AT_DKV) {
+    blk = rank;                                              // key block j: steps i = j .. nblk-1 (causal)
+    it_begin = p.causal ? blk : 0; it_end = p.nblk;
+  } else {
+    blk = p.nblk - 1 - rank;                                 // query block i: steps j = 0 .. i (causal)
+    it_begin = 0; it_end = p.causal ? blk + 1 : p.nblk;
+  }
+  const int nsteps = it_end - it_begin;
+  const int npass = MODE == AT_FWD ? 2 : 1;
+  const int total = nsteps * npass;
+
+  if (threadIdx.x == 0) {
+    mbar_init(b_res, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
+    mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
+    mbar_init(b_acc, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t t_s = tmem, t_dp = tmem + 128, t_acc0 = tmem + 256, t_acc1 = tmem + 320;
+
+  // instruction descriptors (bf16 operands, FP32 accumulation)
+  const uint32_t id_sdp = make_idesc(1u, 1u, 128, 128);                                   // A, B K-major
+  const uint32_t id_mn = make_idesc(1u, 1u, 128, 64) | (1u << 15) | (1u << 16);           // A, B MN-major
+  const uint32_t id_kmn = make_idesc(1u, 1u, 128, 64) | (1u << 16);                       // A K-major, B MN-major
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
+      // resident tiles
+      mbar_expect_tx(b_res, (MODE == AT_FWD ? 1 : 2) * kAtTile);
+      if (MODE == AT_DKV) {
+        tma_load_3d(res0, &tm_k, b_res, 0, blk * AT_BLK, bh);
+        tma_load_3d(res1, &tm_v, b_res, 0, blk * AT_BLK, bh);
+      } else {
+        tma_load_3d(res0, &tm_q, b_res, 0, blk * AT_BLK, bh);
+        if (MODE == AT_DQ) tma_load_3d(res1, &tm_do, b_res, 0, blk * AT_BLK, bh);
+      }
+      bool ok = true;
+      for (int it = 0; it < total && ok; ++it) {
+        const int step = it_begin + (it % nsteps);
+        const uint32_t s = it & 1u, ph = (it >> 1) & 1u;
+        if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
+        mbar_expect_tx(b_sfull + 8 * s, 2 * kAtTile);
+        if (MODE == AT_DKV) {
+          tma_load_3d(d0, &tm_q, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          tma_load_3d(d1, &tm_do, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+        } else {
+          tma_load_3d(d0, &tm_k, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          tma_load_3d(d1, &tm_v, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+        }
+      }
+      if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = mbar_wait(b_res, 0, abort_flag);
+      for (int it = 0; it < total && ok; ++it) {
+        const bool pass2 = it >= nsteps;                      // FWD only
+        const uint32_t s = it & 1u, ph = (it >> 1) & 1u, ip = it & 1u;
+        if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(b_sdp_free, ip ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
+        // S = Q K^T  (and dP = dO V^T): both operands K-major, 64 = 4 x 16 along K
+        const uint32_t q_t = MODE == AT_DKV ? st0 : res0, k_t = MODE == AT_DKV ? res0 : st0;
+        const uint32_t do_t = MODE == AT_DKV ? st1 : res1, v_t = MODE == AT_DKV ? res1 : st1;
+        {
+          const uint64_t a = make_smem_desc(q_t), b = make_smem_desc(k_t);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) tc_mma<false>(t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+        }
+        if (MODE != AT_FWD) {
+          const uint64_t a = make_smem_desc(do_t), b = make_smem_desc(v_t);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+        }
+        tc_commit(b_sdp_full);
+        if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t first = (MODE == AT_FWD ? it == nsteps : it == 0) ? 0u : 1u;   // overwrite on the first product
+        if (MODE == AT_DKV) {
+          // dV += P^T dO, dK += dS^T Q : A MN-major from the P / dS buffers (two 64-key atoms, 16 KB
+          // apart), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
+          const uint64_t ap = make_smem_desc_mn(pbuf, 16384u), ads = make_smem_desc_mn(dsbuf, 16384u);
+          const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) tc_mma<false>(t_acc0, ap + 128u * k, bdo + 128u * k, id_mn, first | (k != 0));
+#pragma unroll
+          for (int k = 0; k < 8; ++k) tc_mma<false>(t_acc1, ads + 128u * k, bq + 128u * k, id_mn, first | (k != 0));
+        } else if (MODE == AT_DQ || pass2) {
+          // dQ += dS K  (O += P V): A K-major from the dS (P) buffer, B MN-major = streamed K (V)
+          const uint32_t abuf = MODE == AT_DQ ? dsbuf : pbuf;
+          const uint64_t bk = make_smem_desc_mn(MODE == AT_DQ ? st0 : st1, 16384u);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t a = make_smem_desc(abuf + (k >> 2) * 16384u + (k & 3) * 32u);
+            tc_mma<false>(t_acc0, a, bk + 128u * k, id_kmn, first | (k != 0));
+          }
+        }
+        tc_commit(b_pds_free);
+        tc_commit(b_sempty + 8 * s);
+      }
+      if (ok) tc_commit(b_acc);
+    }
+  } else {
+    // ------------------------------------------------ softmax / dS warps, then the epilogue
+    const int q4 = warp & 3, h = (warp - 2) >> 2;
+    const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
+    const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    const float c2 = p.c * kLog2e;
+    bool ok = true;
+    float lse2 = 0.f, dq = 0.f;                               // this row's LSE*log2e and D
+    int qrow = 0;                                             // global query index of this thread's row
+    if (MODE != AT_DKV) {
+      qrow = blk * AT_BLK + r;
+      if (MODE == AT_DQ && qrow < p.S) {
+        lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
+        dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
+      }
+    }
+    float run_m = -INFINITY, run_l = 0.f;                     // FWD pass 1: running max and sum (this half)
+    for (int it = 0; it < total && ok; ++it) {
+      const bool pass2 = it >= nsteps;
+      const int step = it_begin + (it % nsteps);
+      const uint32_t ip = it & 1u;
+      int kblk;                                               // key block of this step
+      if (MODE == AT_DKV) {
+        kblk = blk;
+        qrow = step * AT_BLK + r;
+        lse2 = 0.f; dq = 0.f;
+        if (qrow < p.S) {
+          lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
+          dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
+        }
+      } else {
+        kblk = step;
+      }
+      if (MODE == AT_FWD && it == nsteps) {
+        // between the passes: combine the two column halves of every row into the row's LSE
+        float* xm = xchg;                                     // [2][128] max, then [2][128] sum
+        xm[h * 128 + r] = run_m;
+        xm[256 + h * 128 + r] = run_l;
+        named_bar_sync(1, 256);
+        const float m0 = xm[r], m1 = xm[128 + r], l0 = xm[256 + r], l1 = xm[384 + r];
+        const float m = fmaxf(m0, m1);
+        float l = 0.f;
+        if (m0 > -INFINITY) l += l0 * exp2f(m0 - m);
+        if (m1 > -INFINITY) l += l1 * exp2f(m1 - m);
+        lse2 = m + log2f(l);                                  // in units of log2: LSE * log2(e)
+        if (h == 0 && qrow < p.S) p.lse_out[(size_t)bh * p.S + qrow] = lse2 / kLog2e;
+        named_bar_sync(1, 256);
+      }
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sdp_full, ip, abort_flag));
+      if (!ok) break;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const int key0 = kblk * AT_BLK + h * 64;
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t sv[32], dv[32];
+        tmem_ld32(t_s + lane_off + h * 64 + ch * 32, sv);
+        if (MODE != AT_FWD) tmem_ld32(t_dp + lane_off + h * 64 + ch * 32, dv);
+        if (MODE == AT_FWD && !pass2) {
+          // running max / sum of exp2(c2 * s) over the valid keys of this half
+          float mloc = run_m;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int key = key0 + ch * 32 + j;
+            const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
+            if (valid) mloc = fmaxf(mloc, __uint_as_float(sv[j]) * c2);
+          }
+          if (mloc > -INFINITY) {
+            float add = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int key = key0 + ch * 32 + j;
+              const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
+              if (valid) add += exp2f(__uint_as_float(sv[j]) * c2 - mloc);
+            }
+            run_l = run_l * (run_m > -INFINITY ? exp2f(run_m - mloc) : 0.f) + add;
+            run_m = mloc;
+          }
+        } else {
+          uint32_t pk[16], dk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            float pv[2], dsv[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int key = key0 + ch * 32 + j + e;
+              const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
+              const float pr = valid ? exp2f(__uint_as_float(sv[j + e]) * c2 - lse2) : 0.f;
+              pv[e] = pr;
+              dsv[e] = MODE != AT_FWD ? pr * (__uint_as_float(dv[j + e]) - dq) : 0.f;
+            }
+            pk[j >> 1] = float_to_bf16_bits(pv[0]) | (float_to_bf16_bits(pv[1]) << 16);
+            dk[j >> 1] = float_to_bf16_bits(dsv[0]) | (float_to_bf16_bits(dsv[1]) << 16);
+          }
+          // 32 keys = 4 chunks of 16 bytes in row r of half h: chunk index (ch*4 + t) ^ (r & 7)
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)((ch * 4 + t) ^ (r & 7)) << 4);
+            if (MODE != AT_DQ)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
+                           "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
+            if (MODE != AT_FWD)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsbuf + off), "r"(dk[4 * t]), "r"(dk[4 * t + 1]),
+                           "r"(dk[4 * t + 2]), "r"(dk[4 * t + 3]) : "memory");
+          }
+        }
+      }
+      tc_fence_before();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(b_sdp_free); mbar_arrive(b_pds_ready); }
+    }
+    // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise)
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc, 0, abort_flag));
+    if (ok) {
+      tc_fence_after();
+      const int grow = blk * AT_BLK + r;
+      if (MODE == AT_DKV) {
+        // h = 0 warps write dV (acc0), h = 1 warps write dK (acc1, times the softmax scale)
+        float* dst = (h == 0 ? p.out0 : p.out1) + ((size_t)bh * p.S + grow) * AT_D;
+        const float mul = h == 0 ? 1.f : p.c;
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t a[32];
+          tmem_ld32((h == 0 ? t_acc0 : t_acc1) + lane_off + ch * 32, a);
+          if (grow < p.S) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(dst + ch * 32 + j) =
+                  make_float4(__uint_as_float(a[j]) * mul, __uint_as_float(a[j + 1]) * mul,
+                              __uint_as_float(a[j + 2]) * mul, __uint_as_float(a[j + 3]) * mul);
+          }
+        }
+      } else {
+        // each column half writes 32 of the 64 output columns
+        float* dst = p.out0 + ((size_t)bh * p.S + grow) * AT_D + h * 32;
+        const float mul = MODE == AT_DQ ? p.c : 1.f;
+        uint32_t a[32];
+        tmem_ld32(t_acc0 + lane_off + h * 32, a);
+        if (grow < p.S) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(dst + j) =
+                make_float4(__uint_as_float(a[j]) * mul, __uint_as_float(a[j + 1]) * mul,
+                            __uint_as_float(a[j + 2]) * mul, __uint_as_float(a[j + 3]) * mul);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && p.diag) atomicMax(&p.diag->status, (int)BSP_ERR_TIMEOUT);
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ------------------------------------------------------------------------------- D pre-pass
+
+// D[d][row] = sum_j dO[row][j] * O_copy[row][j] for n_draws draws (one for U and R).  16 threads per
+// row of 64, four elements each; U reads the FP32 original, R the forward's codes, N a fresh
+// stochastic rounding of fl32(O * scale[bh]) keyed by the element's index in the whole tensor.
+template <int DT, int FMT>
+__global__ void __launch_bounds__(256)
+attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig, const uint8_t* __restrict__ o_codes,
+                  const float* __restrict__ o_scales, int64_t rows, int S, int policy, PhiloxKey key, int draw0,
+                  int n_draws, float* __restrict__ D) {
+  const int64_t row = (int64_t)blockIdx.x * 16 + (threadIdx.x >> 4);
+  const int sub = threadIdx.x & 15;
+  const bool active = row < rows;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), o = g;
+  float scale = 1.f, inv = 1.f;
+  const size_t i0 = (size_t)(active ? row : 0) * AT_D + sub * 4;
+  if (active) {
+    g = load4<DT>(dO, i0);
+    if (policy != BSP_READ_ORIGINAL || true) {
+      scale = o_scales ? __ldg(o_scales + row / S) : 1.f;
+      inv = __fdiv_rn(1.0f, scale);
+    }
+    if (policy == BSP_READ_FORWARD) {
+      const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(o_codes + i0));
+      o = make_float4(f8_decode<FMT>(pk & 0xFFu) * inv, f8_decode<FMT>((pk >> 8) & 0xFFu) * inv,
+                      f8_decode<FMT>((pk >> 16) & 0xFFu) * inv, f8_decode<FMT>(pk >> 24) * inv);
+    } else {
+      o = __ldg(reinterpret_cast<const float4*>(o_orig + i0));
+    }
+  }
+  for (int d = 0; d < n_draws; ++d) {
+    float4 c = o;
+    if (policy == BSP_READ_FRESH) {
+      const uint4 w = philox_block(key, (uint64_t)i0 >> 2, (uint32_t)(draw0 + d));
+      c.x = f8_sr_value<FMT>(__fmul_rn(o.x, scale), w.x) * inv;
+      c.y = f8_sr_value<FMT>(__fmul_rn(o.y, scale), w.y) * inv;
+      c.z = f8_sr_value<FMT>(__fmul_rn(o.z, scale), w.z) * inv;
+      c.w = f8_sr_value<FMT>(__fmul_rn(o.w, scale), w.w) * inv;
+    }
+    float s = (g.x * c.x + g.y * c.y) + (g.z * c.z + g.w * c.w);
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+    if (active && sub == 0) D[(size_t)d * rows + row] = s;
+  }
+}
+
+// S1 += g - ref, S2 += (g - ref)^2, elementwise.
+__global__ void mc_accumulate_kernel(const float* __restrict__ g, const float* __restrict__ ref, float* __restrict__ S1,
+                                     float* __restrict__ S2, size_t n4) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 a = __ldg(reinterpret_cast<const float4*>(g) + i), r = __ldg(reinterpret_cast<const float4*>(ref) + i);
+  float4 s1 = reinterpret_cast<float4*>(S1)[i], s2 = reinterpret_cast<float4*>(S2)[i];
+  const float d0 = a.x - r.x, d1 = a.y - r.y, d2 = a.z - r.z, d3 = a.w - r.w;
+  s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
+  s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y); s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
+  reinterpret_cast<float4*>(S1)[i] = s1;
+  reinterpret_cast<float4*>(S2)[i] = s2;
+}
+
+// ------------------------------------------------------------------------------- host side
+
+static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return BSP_ERR_CUDA;
+  cuuint64_t gdim[3] = {(cuuint64_t)AT_D, (cuuint64_t)S, (cuuint64_t)BH};
+  cuuint64_t gstr[2] = {(cuuint64_t)AT_D * 2, (cuuint64_t)S * AT_D * 2};
+  cuuint32_t box[3] = {(cuuint32_t)AT_D, (cuuint32_t)AT_BLK, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
+}
+
+template <int MODE>
+static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
+  CUtensorMap mq, mk, mv, mdo;
+  int rc;
+  if ((rc = make_head_map(&mq, q, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
+  static bool attr_set = false;
+  if (!attr_set) {
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    attr_set = true;
+  }
+  const unsigned grid = (unsigned)p.nblk * (unsigned)p.BH;
+  attn_kernel<MODE><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, p);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
+
+static int check_attn_shape(int B, int H, int S, int Dh, int dt) {
+  if (B <= 0 || H <= 0 || S <= 0) return BSP_ERR_ARG;
+  if (Dh != AT_D || dt != BSP_BF16) return BSP_ERR_UNSUPPORTED;
+  if ((int64_t)B * H > 65535 * 16) return BSP_ERR_UNSUPPORTED;
+  return BSP_OK;
+}
+
+}  // namespace bsp
+
+using namespace bsp;
+
+extern "C" {
+
+int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                       const void* v, int dt, float* o, float* lse, bsp_diag_t* diag, void* stream) {
+  int rc = check_attn_shape(B, H, S, Dh, dt);
+  if (rc != BSP_OK) return rc;
+  if (!q || !k || !v || !o || !lse) return BSP_ERR_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
+  AttnParams p;
+  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
+  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag;
+  return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
+}
+
+int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig, const uint8_t* o_codes,
+                   const float* o_scales, int o_fmt, int d_read, bsp_key_t key, int draw0, int n_draws, float* d_out,
+                   bsp_diag_t* diag, void* stream) {
+  (void)diag;
+  if (B <= 0 || H <= 0 || S <= 0 || !valid_enum(dt, 1) || !valid_enum(o_fmt, 1) || !valid_enum(d_read, 2)) return BSP_ERR_ARG;
+  if (Dh != AT_D) return BSP_ERR_UNSUPPORTED;
+  if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0 || draw0 < 0 || n_draws < 0) return BSP_ERR_ARG;
+  if (n_draws == 0) return BSP_OK;
+  if (!dO || !d_out) return BSP_ERR_ARG;
+  if (d_read == BSP_READ_FORWARD ? (!o_codes || !o_scales) : !o_orig) return BSP_ERR_ARG;
+  if (d_read == BSP_READ_FRESH && !o_scales) return BSP_ERR_ARG;
+  if (d_read != BSP_READ_FRESH) n_draws = 1;
+  if (!aligned16(dO) || !aligned16(o_orig) || (reinterpret_cast<uintptr_t>(o_codes) & 3u)) return BSP_ERR_ALIGN;
+  const int64_t rows = (int64_t)B * H * S;
+  const unsigned grid = (unsigned)((rows + 15) / 16);
+  cudaStream_t st = (cudaStream_t)stream;
+  const PhiloxKey pk = make_key(key);
+#define BSP_DT(DT, FMT)                                                                                          \
+  attn_dterm_kernel<DT, FMT><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, rows, S, d_read, pk, draw0,    \
+                                                   n_draws, d_out)
+  if (dt == BSP_F32 && o_fmt == BSP_E4M3) BSP_DT(BSP_F32, BSP_E4M3);
+  else if (dt == BSP_F32) BSP_DT(BSP_F32, BSP_E5M2);
+  else if (o_fmt == BSP_E4M3) BSP_DT(BSP_BF16, BSP_E4M3);
+  else BSP_DT(BSP_BF16, BSP_E5M2);
+#undef BSP_DT
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                       const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq,
+                       float* dk, float* dv, bsp_diag_t* diag, void* stream) {
+  int rc = check_attn_shape(B, H, S, Dh, dt);
+  if (rc != BSP_OK) return rc;
+  if (!q || !k || !v || !dO || !lse || !dterm) return BSP_ERR_ARG;
+  if ((dk == nullptr) != (dv == nullptr) || (!dq && !dk)) return BSP_ERR_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) ||
+      !aligned16(dv))
+    return BSP_ERR_ALIGN;
+  AttnParams p;
+  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
+  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dk) {
+    p.out0 = dv; p.out1 = dk;
+    if ((rc = launch_attn<AT_DKV>(q, k, v, dO, p, st)) != BSP_OK) return rc;
+  }
+  if (dq) {
+    p.out0 = dq; p.out1 = nullptr;
+    if ((rc = launch_attn<AT_DQ>(q, k, v, dO, p, st)) != BSP_OK) return rc;
+  }
+  return BSP_OK;
+}
+
+int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands, const void* q,
+                 const void* k, const void* v, const void* dO, int dt, const float* lse, const float* o_orig,
+                 const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key, float* dq,
+                 float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
+  if (fp8_operands) return BSP_ERR_UNSUPPORTED;
+  if (!d_out) return BSP_ERR_ARG;
+  int rc = bsp_attn_dterm(B, H, S, Dh, dO, dt, o_orig, o_codes, o_scales, o_fmt, d_read, key, (int)key.draw, 1, d_out,
+                          diag, stream);
+  if (rc != BSP_OK) return rc;
+  return bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, lse, d_out, dq, dk, dv, diag, stream);
+}
+
+int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, size_t n, void* stream) {
+  if (!g || !g_ref || !S1 || !S2) return BSP_ERR_ARG;
+  if (n % 4 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(g) || !aligned16(g_ref) || !aligned16(S1) || !aligned16(S2)) return BSP_ERR_ALIGN;
+  if (n == 0) return BSP_OK;
+  const size_t n4 = n / 4;
+  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(g, g_ref, S1, S2, n4);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+}  // extern "C"

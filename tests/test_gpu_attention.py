@@ -1,0 +1,179 @@
+"""Attention on the GPU (forward statistics, the D use under the three reads, backward) against
+the float64 oracle.  Tensor-core products: <= 2e-3 relative L2 per tensor; D is CUDA-core FP32:
+<= 1e-5; codes of the output store bit-exact."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from conftest import golden_path
+from oracle import attention, check, fp8, linear, philox
+from paper_2609_39813_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL_TC = 2e-3
+TOL_FP32 = 1e-5
+
+
+@pytest.fixture(scope="module")
+def b():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39813_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _rel(a, ref):
+    a, ref = np.asarray(a, np.float64).ravel(), np.asarray(ref, np.float64).ravel()
+    return float(np.linalg.norm(a - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+class AttnGpu:
+    def __init__(self, b, inp, causal=True):
+        from paper_2609_39813_b200.harness import up
+        self.inp, self.causal = inp, causal
+        B, H, S, D = inp.B, inp.H, inp.S, inp.D
+        self.q, self.k, self.v, self.dO = (up(a, "bf16") for a in (inp.q, inp.k, inp.v, inp.dO))
+        self.o = torch.zeros(B * H * S * D, device="cuda")
+        self.lse = torch.zeros(B * H * S, device="cuda")
+        self.diag = b.new_diag()
+        b.bsp_attn_fwd_stats(B, H, S, D, causal, inp.softmax_scale, self.q, self.k, self.v, self.o, self.lse, self.diag)
+        # the output store: per-(b,h) amax scale, E4M3 stochastic rounding, stream 0
+        self.amax = torch.zeros(B * H, device="cuda")
+        self.scales = torch.zeros(B * H, device="cuda")
+        b.bsp_amax(self.o, B * H, S * D, self.amax)
+        b.bsp_scale_from_amax(self.amax, B * H, fp8.E4M3, self.scales)
+        self.codes = torch.zeros(B * H * S * D, dtype=torch.uint8, device="cuda")
+        b.bsp_round_grouped(self.o, B * H, S * D, fp8.E4M3, fp8.SR, self.scales,
+                            b.key(inp.seed, check.TENSOR_O, b.STREAM_FORWARD, 0), self.codes)
+        torch.cuda.synchronize()
+
+
+CASES = {
+    "two_blocks_ragged": dict(B=1, H=2, S=200, causal=True),
+    "three_blocks": dict(B=2, H=1, S=384, causal=True),
+    "noncausal": dict(B=1, H=1, S=256, causal=False),
+    "one_short_block": dict(B=1, H=3, S=72, causal=True),
+}
+
+
+@pytest.fixture(scope="module", params=list(CASES), ids=list(CASES))
+def case(request, b):
+    cfg = CASES[request.param]
+    inp = workloads.config3(B=cfg["B"], H=cfg["H"], S=cfg["S"], D=64, K=4, seed=1003 + cfg["S"])
+    g = AttnGpu(b, inp, cfg["causal"])
+    return inp, g
+
+
+def _slices(inp):
+    for bi in range(inp.B):
+        for hi in range(inp.H):
+            yield bi * inp.H + hi, inp.q[bi, hi], inp.k[bi, hi], inp.v[bi, hi], inp.dO[bi, hi]
+
+
+def test_forward_statistics_and_store(b, case):
+    inp, g = case
+    S, D = inp.S, inp.D
+    assert b.read_diag(g.diag)["status"] == 0
+    o = g.o.cpu().numpy().reshape(inp.B * inp.H, S, D)
+    lse = g.lse.cpu().numpy().reshape(inp.B * inp.H, S)
+    codes = g.codes.cpu().numpy().reshape(inp.B * inp.H, S, D)
+    for idx, q, k, v, dO in _slices(inp):
+        want_o, want_lse = attention.forward_output(q, k, v, inp.softmax_scale, g.causal)
+        assert _rel(o[idx], want_o) <= TOL_TC
+        assert np.max(np.abs(lse[idx] - want_lse)) <= 1e-4
+        # codes are bit-exact given the FP32 output the GPU stored
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, g.causal, o32=o[idx])
+        assert g.scales.cpu().numpy()[idx] == prep["scale"]
+        assert np.array_equal(codes[idx], prep["codes"])
+
+
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_dterm_three_reads(b, case, policy):
+    inp, g = case
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    ndraw = 3 if policy == 2 else 1
+    d_out = torch.zeros(ndraw * B * H * S, device="cuda")
+    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, g.codes, g.scales, fp8.E4M3, policy,
+                     b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0), 5, ndraw, d_out)
+    got = d_out.cpu().numpy().reshape(ndraw, B * H, S)
+    o = g.o.cpu().numpy().reshape(B * H, S, D)
+    for idx, q, k, v, dO in _slices(inp):
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, g.causal, o32=o[idx])
+        for d in range(ndraw):
+            copy = check.attention_d_copy(prep, policy, inp.seed, 5 + d)
+            want = np.sum(dO.astype(np.float64) * copy, axis=1)
+            assert _rel(got[d, idx], want) <= TOL_FP32
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_backward_against_oracle(b, case, policy):
+    inp, g = case
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    n = B * H * S * D
+    dq, dk, dv = (torch.full((n,), float("nan"), device="cuda") for _ in range(3))
+    d_out = torch.zeros(B * H * S, device="cuda")
+    diag = b.new_diag()
+    b.bsp_attn_bwd(B, H, S, D, g.causal, inp.softmax_scale, 0, g.q, g.k, g.v, g.dO, g.lse, g.o, g.codes, g.scales,
+                   fp8.E4M3, policy, b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0), dq, dk, dv, d_out, diag)
+    assert b.read_diag(diag)["status"] == 0
+    o = g.o.cpu().numpy().reshape(B * H, S, D)
+    got = {n_: t.cpu().numpy().reshape(B * H, S, D) for n_, t in (("dq", dq), ("dk", dk), ("dv", dv))}
+    for idx, q, k, v, dO in _slices(inp):
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, g.causal, o32=o[idx])
+        copy = check.attention_d_copy(prep, policy, inp.seed, 0)
+        # P and dS enter their products as bf16 tensor-core operands: the oracle rounds them alike
+        want = attention.backward(q, k, v, dO, inp.softmax_scale, copy, g.causal,
+                                  operand_round=linear.bf16_round)
+        for name in ("dq", "dk", "dv"):
+            assert np.isfinite(got[name][idx]).all(), name
+            assert _rel(got[name][idx], want[name]) <= TOL_TC, (name, idx)
+
+
+def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
+    inp, g = case
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    n = B * H * S * D
+    outs = []
+    for policy in (0, 0, 1):
+        dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
+        d_out = torch.zeros(B * H * S, device="cuda")
+        b.bsp_attn_bwd(B, H, S, D, g.causal, inp.softmax_scale, 0, g.q, g.k, g.v, g.dO, g.lse, g.o, g.codes,
+                       g.scales, fp8.E4M3, policy, b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0), dq, dk, dv,
+                       d_out)
+        outs.append((dq, dk, dv))
+    assert all(torch.equal(a, c) for a, c in zip(outs[0], outs[1]))      # byte-identical repeat
+    assert torch.equal(outs[0][2], outs[2][2])                             # dV never reads the saved output
+    assert not torch.equal(outs[0][0], outs[2][0])                         # dQ does
+
+
+def test_attention_row_case_of_the_paper(b):
+    """One causal row of 64 keys with uniform attention; saved entry x = 5/4 +- 1/4, dO = h at that
+    entry: dQ[63, 0] = c h (s - x).  In BF16-operand mode P = exp(S - LSE) is exact only to FP32
+    rounding, so the eight cells are reproduced to 1e-6 relative, not bit for bit."""
+    from paper_2609_39813_b200.harness import up
+    S, D, a, s, c = 64, 64, 0.25, 1.25, 0.125
+    q = np.zeros((1, 1, S, D), np.float32); q[..., 1] = 1.0
+    k = np.zeros((1, 1, S, D), np.float32); k[..., 0] = 1.0
+    v = np.zeros((1, 1, S, D), np.float32); v[0, 0, :, 0] = np.where(np.arange(S) % 2 == 0, 1.0, 1.5)
+    qd, kd, vd = up(q, "bf16"), up(k, "bf16"), up(v, "bf16")
+    o = torch.zeros(S * D, device="cuda"); lse = torch.zeros(S, device="cuda")
+    b.bsp_attn_fwd_stats(1, 1, S, D, True, c, qd, kd, vd, o, lse)
+    assert abs(o.cpu().numpy().reshape(S, D)[63, 0] - s) < 1e-5
+    cells = [l.split() for l in open(golden_path("attention_row_cells.txt")) if l[0] in "+-"]
+
+    def dq_at(x, h):
+        dO = np.zeros((1, 1, S, D), np.float32); dO[0, 0, 63, 0] = h
+        saved = o.clone(); saved[63 * D] = x
+        dq = torch.zeros(S * D, device="cuda"); d_out = torch.zeros(S, device="cuda")
+        b.bsp_attn_bwd(1, 1, S, D, True, c, 0, qd, kd, vd, up(dO, "bf16"), lse, saved, None, None, fp8.E4M3, 0,
+                       b.key(0, 2, 4, 0), dq, None, None, d_out)
+        return float(dq.cpu().numpy().reshape(S, D)[63, 0])
+
+    for sig, tau, t_dev, t_fixed in cells:
+        sig, tau = float(sig), float(tau)
+        for h, want in ((sig * a, float(t_dev)), (a, float(t_fixed))):
+            T = (dq_at(s + tau * a, h) - dq_at(s + sig * a, h)) / c
+            assert abs(T - want) <= 1e-6, (sig, tau, h, T, want)

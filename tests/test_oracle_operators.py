@@ -307,3 +307,20 @@ def test_attention_check_expected_verdicts():
     w_full = philox.tensor_words(inp.seed, check.TENSOR_O, 0, 0, 2 * 48 * 16)
     assert np.array_equal(philox.element_words(inp.seed, check.TENSOR_O, 0, 0, prep["elem"]).ravel(),
                           w_full[48 * 16:])
+
+
+def test_attention_operand_rounding_option():
+    """Rounding P and dS to bf16 before their products (what a BF16 tensor-core contraction does)
+    moves the gradients by about 2^-9, leaves D untouched, and is the identity when the rounding
+    is the identity."""
+    q, k, v, dO = _tiny_attention(11, 40, 8)
+    c = 0.3
+    O, _ = attention.forward_output(q, k, v, c)
+    exact = attention.backward(q, k, v, dO, c, O)
+    same = attention.backward(q, k, v, dO, c, O, operand_round=lambda a: a)
+    rounded = attention.backward(q, k, v, dO, c, O, operand_round=linear.bf16_round)
+    for n in ("dq", "dk", "dv"):
+        assert np.array_equal(same[n], exact[n])
+        rel = np.linalg.norm(rounded[n] - exact[n]) / np.linalg.norm(exact[n])
+        assert 1e-5 < rel < 4e-3, (n, rel)
+    assert np.array_equal(rounded["D"], exact["D"])
