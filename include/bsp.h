@@ -384,6 +384,32 @@ size_t bsp_mc_check_workspace_bytes(const bsp_norm_linear_desc_t* op, int K);
 int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* results, int* n_results,
                  void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
 
+/* The per-use check of the attention D use (Section "Same rounding distribution, opposite
+ * outcomes"; Eq. dterm), device-resident inputs.  Once per call: O = P V and LSE, the output store
+ * (per-(b,h) amax scale, `forward_mode`, stream 0).  Reference: D reads the original output.  Then
+ * for each selected policy (policy_mask bit p = bsp_policy_t p) the backward is evaluated with D
+ * read under that policy -- U and R once, N for K draws -- and four results are written per policy
+ * in the order D, dQ, dK, dV.  `results` is a HOST array (up to 12 entries).  Synchronises. */
+typedef struct {
+  int32_t B, H, S, Dh;
+  int32_t causal;
+  float softmax_scale;
+  int32_t dtype;             /* bsp_dtype_t of q, k, v, dO (BSP_BF16) */
+  const void* q;             /* [B, H, S, Dh] */
+  const void* k;
+  const void* v;
+  const void* dO;
+  int32_t store_fmt;         /* bsp_format_t of the output store (E4M3) */
+  int32_t forward_mode;      /* bsp_round_mode_t of the forward's store   */
+  uint64_t seed;
+  uint32_t tensor_id;
+  uint32_t policy_mask;
+} bsp_attn_desc_t;
+
+size_t bsp_mc_check_attn_workspace_bytes(const bsp_attn_desc_t* op, int K);
+int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* results, int* n_results,
+                      void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -57,6 +57,13 @@ class NormLinearDesc(C.Structure):
                 ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
 
 
+class AttnDesc(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("S", C.c_int32), ("Dh", C.c_int32), ("causal", C.c_int32),
+                ("softmax_scale", C.c_float), ("dtype", C.c_int32), ("q", C.c_void_p), ("k", C.c_void_p),
+                ("v", C.c_void_p), ("dO", C.c_void_p), ("store_fmt", C.c_int32), ("forward_mode", C.c_int32),
+                ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
+
+
 class BspError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
@@ -100,6 +107,8 @@ _SIGNATURES = {
     "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, _P, _P, _P, _P, _I, _I, Key, _P, _P, _P,
                           _P, _P, _P]),
     "bsp_mc_accumulate": (_I, [_P, _P, _P, _P, _SZ, _P]),
+    "bsp_mc_check_attn_workspace_bytes": (_SZ, [C.POINTER(AttnDesc), _I]),
+    "bsp_mc_check_attn": (_I, [C.POINTER(AttnDesc), _I, C.POINTER(UseResult), C.POINTER(_I), _P, _SZ, _P, _P]),
     "bsp_mc_stats_workspace_bytes": (_SZ, [_I64]),
     "bsp_mc_stats": (_I, [_P, _P, _P, _I64, _I, _I, C.POINTER(UseResult), _P, _SZ, _P]),
     "bsp_mc_check_workspace_bytes": (_SZ, [C.POINTER(NormLinearDesc), _I]),
@@ -353,6 +362,19 @@ def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, 
 
 def bsp_mc_accumulate(g, g_ref, S1, S2, n, stream=None):
     check(lib().bsp_mc_accumulate(ptr(g), ptr(g_ref), ptr(S1), ptr(S2), n, _st(stream)), "bsp_mc_accumulate")
+
+
+def bsp_mc_check_attn_workspace_bytes(desc: AttnDesc, K):
+    return lib().bsp_mc_check_attn_workspace_bytes(C.byref(desc), K)
+
+
+def bsp_mc_check_attn(desc: AttnDesc, K, ws, diag=None, stream=None):
+    """Returns the list of UseResult: per selected policy (U, R, N) the four outputs D, dQ, dK, dV."""
+    res = (UseResult * 12)()
+    n = C.c_int(0)
+    check(lib().bsp_mc_check_attn(C.byref(desc), K, res, C.byref(n), ptr(ws), ws.numel(), ptr(diag), _st(stream)),
+          "bsp_mc_check_attn")
+    return [res[i] for i in range(n.value)]
 
 
 def bsp_mc_stats_workspace_bytes(n):

@@ -19,6 +19,8 @@
 // read those buffers directly (MN-major A for dV and dK, K-major A for dQ and O) and the TMA-loaded
 // 128 x 64 tiles as MN-major B.  320 threads: warp 0 TMA, warp 1 MMA, warps 2..9 softmax + epilogue.
 // Head dimension 64, bf16 inputs, FP32 outputs.  Every wait is bounded.
+#include <string.h>
+
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -544,6 +546,145 @@ int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, 
   const size_t n4 = n / 4;
   mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(g, g_ref, S1, S2, n4);
   BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------- per-use check, attention
+
+namespace bsp {
+
+struct AttnCheckBuffers {
+  float *o, *lse, *amax, *scales, *d_ref, *d_pol, *d_draws;
+  uint8_t* codes;
+  float *g_ref[3], *g_pol[3], *S1[3], *S2[3], *S1d, *S2d;
+  void* ws_stats;
+  size_t b_stats;
+};
+
+static size_t attn_carve(const bsp_attn_desc_t* op, int K, char* base, AttnCheckBuffers* out) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> void* {
+    void* p = base ? base + off : nullptr;
+    off += round_up(bytes ? bytes : 1, 256);
+    return p;
+  };
+  const size_t BH = (size_t)op->B * op->H, rows = BH * op->S, n = rows * op->Dh;
+  AttnCheckBuffers c;
+  c.o = (float*)take(n * 4); c.lse = (float*)take(rows * 4);
+  c.amax = (float*)take(BH * 4); c.scales = (float*)take(BH * 4);
+  c.d_ref = (float*)take(rows * 4); c.d_pol = (float*)take(rows * 4);
+  c.d_draws = (float*)take(rows * 4 * (size_t)(K > 0 ? K : 1));
+  c.codes = (uint8_t*)take(n);
+  for (int t = 0; t < 3; ++t) {
+    c.g_ref[t] = (float*)take(n * 4); c.g_pol[t] = (float*)take(n * 4);
+    c.S1[t] = (float*)take(n * 4); c.S2[t] = (float*)take(n * 4);
+  }
+  c.S1d = (float*)take(rows * 4); c.S2d = (float*)take(rows * 4);
+  c.b_stats = bsp_mc_stats_workspace_bytes((int64_t)n);
+  c.ws_stats = take(c.b_stats);
+  if (out) *out = c;
+  return off;
+}
+
+}  // namespace bsp
+
+extern "C" {
+
+size_t bsp_mc_check_attn_workspace_bytes(const bsp_attn_desc_t* op, int K) {
+  if (!op || op->B <= 0 || op->H <= 0 || op->S <= 0 || op->Dh <= 0) return 0;
+  return bsp::attn_carve(op, K, nullptr, nullptr);
+}
+
+#define BSP_TRY(expr)              \
+  do {                             \
+    int _rc = (expr);              \
+    if (_rc != BSP_OK) return _rc; \
+  } while (0)
+
+int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* results, int* n_results, void* ws,
+                      size_t ws_bytes, bsp_diag_t* diag, void* stream) {
+  using namespace bsp;
+  if (!op || !results || !n_results || K < 2) return BSP_ERR_ARG;
+  if (!op->q || !op->k || !op->v || !op->dO) return BSP_ERR_ARG;
+  int rc = check_attn_shape(op->B, op->H, op->S, op->Dh, op->dtype);
+  if (rc != BSP_OK) return rc;
+  if (!ws || ws_bytes < bsp_mc_check_attn_workspace_bytes(op, K) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return BSP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  AttnCheckBuffers b;
+  attn_carve(op, K, reinterpret_cast<char*>(ws), &b);
+  const int B = op->B, H = op->H, S = op->S, Dh = op->Dh, dt = op->dtype;
+  const size_t BH = (size_t)B * H, rows = BH * S, n = rows * Dh;
+  const float c = op->softmax_scale;
+  *n_results = 0;
+
+  // ---- once: forward output and LSE, the output store (per-(b,h) amax scale, stream 0)
+  BSP_TRY(bsp_attn_fwd_stats(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, dt, b.o, b.lse, diag, st));
+  BSP_TRY(bsp_amax(b.o, BSP_F32, BH, (size_t)S * Dh, b.amax, diag, st));
+  BSP_TRY(bsp_scale_from_amax(b.amax, BH, op->store_fmt, b.scales, st));
+  bsp_key_t key;
+  key.seed = op->seed; key.tensor_id = op->tensor_id; key.stream = BSP_STREAM_FORWARD; key.draw = 0; key.reserved = 0;
+  BSP_TRY(bsp_round_grouped(b.o, BSP_F32, BH, (size_t)S * Dh, op->store_fmt, op->forward_mode, b.scales, key, b.codes,
+                            diag, st));
+  key.stream = BSP_STREAM_ATTN_D;
+
+  // ---- reference: D reads the original output
+  BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_ORIGINAL, key, 0, 1,
+                         b.d_ref, diag, st));
+  BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, b.d_ref, b.g_ref[0],
+                             b.g_ref[1], b.g_ref[2], diag, st));
+  int nres = 0;
+  const int out_ids[4] = {BSP_OUT_D, BSP_OUT_DQ, BSP_OUT_DK, BSP_OUT_DV};
+  auto emit = [&](int out, int pol) -> bsp_use_result_t* {
+    bsp_use_result_t* r = &results[nres++];
+    memset(r, 0, sizeof(*r));
+    r->use_id = BSP_STREAM_ATTN_D; r->output_id = out; r->policy = pol;
+    return r;
+  };
+  for (int pol = 0; pol < 2; ++pol) {
+    if (!((op->policy_mask >> pol) & 1u)) continue;
+    const float* dsrc = b.d_ref;
+    float* const* gsrc = b.g_ref;
+    if (pol == BSP_READ_FORWARD) {
+      BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_FORWARD, key, 0,
+                             1, b.d_pol, diag, st));
+      BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, b.d_pol,
+                                 b.g_pol[0], b.g_pol[1], b.g_pol[2], diag, st));
+      dsrc = b.d_pol;
+      gsrc = b.g_pol;
+    }
+    BSP_TRY(bsp_mc_stats(b.d_ref, dsrc, nullptr, (int64_t)rows, 1, 0, emit(out_ids[0], pol), b.ws_stats, b.b_stats, st));
+    for (int t = 0; t < 3; ++t)
+      BSP_TRY(bsp_mc_stats(b.g_ref[t], gsrc[t], nullptr, (int64_t)n, 1, 0, emit(out_ids[t + 1], pol), b.ws_stats,
+                           b.b_stats, st));
+  }
+  if ((op->policy_mask >> 2) & 1u) {
+    // fresh read: all K correction terms in one pass, then one backward per draw
+    BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_FRESH, key, 0, K,
+                           b.d_draws, diag, st));
+    BSP_CHECK_CUDA(cudaMemsetAsync(b.S1d, 0, rows * 4, st));
+    BSP_CHECK_CUDA(cudaMemsetAsync(b.S2d, 0, rows * 4, st));
+    for (int t = 0; t < 3; ++t) {
+      BSP_CHECK_CUDA(cudaMemsetAsync(b.S1[t], 0, n * 4, st));
+      BSP_CHECK_CUDA(cudaMemsetAsync(b.S2[t], 0, n * 4, st));
+    }
+    for (int k = 0; k < K; ++k) {
+      const float* dk_ = b.d_draws + (size_t)k * rows;
+      BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
+      BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],
+                                 b.g_pol[1], b.g_pol[2], diag, st));
+      for (int t = 0; t < 3; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
+    }
+    BSP_TRY(bsp_mc_stats(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH), b.ws_stats,
+                         b.b_stats, st));
+    for (int t = 0; t < 3; ++t)
+      BSP_TRY(bsp_mc_stats(b.g_ref[t], b.S1[t], b.S2[t], (int64_t)n, K, 1, emit(out_ids[t + 1], BSP_READ_FRESH),
+                           b.ws_stats, b.b_stats, st));
+  }
+  *n_results = nres;
+  BSP_CHECK_CUDA(cudaStreamSynchronize(st));
   return BSP_OK;
 }
 

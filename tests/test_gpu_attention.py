@@ -149,6 +149,51 @@ def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
     assert not torch.equal(outs[0][0], outs[2][0])                         # dQ does
 
 
+def test_mc_check_attention_verdicts(b):
+    """The whole per-use check of the D use on a small workload: verdicts identical to the oracle's
+    (U holds exactly, R fails, N holds on average; dV is untouched by the read), statistics close."""
+    from oracle import mc
+    inp = workloads.config3(B=1, H=2, S=192, D=64, K=24, seed=77)
+    g = AttnGpu(b, inp, True)
+    d = b.AttnDesc()
+    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = inp.B, inp.H, inp.S, inp.D, 1, inp.softmax_scale, b.BF16
+    d.q, d.k, d.v, d.dO = b.ptr(g.q), b.ptr(g.k), b.ptr(g.v), b.ptr(g.dO)
+    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, 7
+    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, inp.K))
+    diag = b.new_diag()
+    res = b.bsp_mc_check_attn(d, inp.K, ws, diag)
+    assert len(res) == 12 and b.read_diag(diag)["status"] == 0
+    assert [(r.policy, r.output_id) for r in res] == [(p, o) for p in (0, 1, 2) for o in (b.OUT_D, b.OUT_DQ, b.OUT_DK, b.OUT_DV)]
+    H_, F_ = mc.HOLDS, mc.FAILS
+    # U: everything exact.  R: D, dQ, dK fail, dV is untouched.  N: the use's own output D holds on
+    # average and dV is untouched.  (dQ and dK under N are compared with the oracle below: their
+    # products round dS to bf16, which is not linear in D, so their fresh-draw means carry a
+    # quantisation bias that is not the D use's fault -- the D-use verdict is the one on D.)
+    got = [r.verdict for r in res]
+    assert got[:8] == [H_, H_, H_, H_, F_, F_, F_, H_] and got[8] == H_ and got[11] == H_
+    for r in res[:4]:
+        assert r.rel_l2_mean_err == 0.0
+    assert res[7].rel_l2_mean_err == 0.0 and res[11].rel_l2_mean_err == 0.0 and res[11].R == 0.0     # dV
+    # the oracle on the same stored output (slice by slice; statistics pooled over the slices for D)
+    o = g.o.cpu().numpy().reshape(inp.B * inp.H, inp.S, inp.D)
+    for idx, q, k, v, dO in _slices(inp):
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, True, o32=o[idx])
+        for pol in (0, 1, 2):
+            want = check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, pol, inp.K, inp.seed,
+                                         operand_round=linear.bf16_round)
+            for j, name in enumerate(("D", "dq", "dk", "dv")):
+                assert want[name]["stats"].verdict == res[4 * pol + j].verdict, (pol, name)
+        # with unrounded operands the fresh read holds on average for dQ and dK too (the paper's
+        # statement about the D use); the bias above is the bf16 operand format's, not the read's
+        exact = check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, 2, inp.K, inp.seed)
+        assert [exact[n_]["stats"].verdict for n_ in ("D", "dq", "dk", "dv")] == [H_, H_, H_, H_]
+    # R's error on D is the size of the store's rounding error, as for the norm store
+    assert 0.005 < res[4].rel_l2_mean_err < 0.5
+    # determinism
+    res2 = b.bsp_mc_check_attn(d, inp.K, ws, diag)
+    assert [bytes(r) for r in res] == [bytes(r) for r in res2]
+
+
 def test_attention_row_case_of_the_paper(b):
     """One causal row of 64 keys with uniform attention; saved entry x = 5/4 +- 1/4, dO = h at that
     entry: dQ[63, 0] = c h (s - x).  In BF16-operand mode P = exp(S - LSE) is exact only to FP32
