@@ -156,6 +156,68 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------- CUDA arm
 
 
+def attention_section(b, peaks, steps=3):
+    """Config 3 (causal attention backward, B=8 H=16 S=2048 d=64, K=32): the per-use check of the D
+    use, timed as a whole, and the two backward kernels timed alone.  Extra information beside the
+    headline number; inputs are drawn on the device (same distributions as the seeded recipe)."""
+    import torch
+    B, H, S, D, K = 8, 16, 2048, 64, 32
+    tensor_o = 2                                              # generator tensor id of the attention output store
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1003)
+    n = B * H * S * D
+    q, k, v = (torch.randn(n, device="cuda", generator=gen).mul_(0.125).bfloat16() for _ in range(3))
+    dO = torch.randn(n, device="cuda", generator=gen).bfloat16()
+    d = b.AttnDesc()
+    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, 0.125, b.BF16
+    d.q, d.k, d.v, d.dO = b.ptr(q), b.ptr(k), b.ptr(v), b.ptr(dO)
+    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = b.E4M3, b.ROUND_STOCHASTIC, 1003, tensor_o, 7
+    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+    diag = b.new_diag()
+    stream = torch.cuda.current_stream()
+    res = b.bsp_mc_check_attn(d, K, ws, diag)                 # warm-up
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        res = b.bsp_mc_check_attn(d, K, ws, diag)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    elements = n * (1 + 1 + K)
+    # the backward kernels alone
+    o = torch.zeros(n, device="cuda"); lse = torch.zeros(B * H * S, device="cuda")
+    dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
+    dterm = torch.zeros(B * H * S, device="cuda")
+    b.bsp_attn_fwd_stats(B, H, S, D, True, 0.125, q, k, v, o, lse, diag)
+    b.bsp_attn_dterm(B, H, S, D, dO, o, None, None, b.E4M3, b.READ_ORIGINAL, b.key(0, 2, 4), 0, 1, dterm)
+
+    def timed(fn, reps=5):
+        fn(); fn()
+        torch.cuda.synchronize()
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        c.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(c) / reps
+
+    ms_dkv = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, None, dk, dv, diag))
+    ms_dq = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, dq, None, None, diag))
+    prod = 2.0 * B * H * S * S * D / 2                         # one causal S x S x d product over all heads
+    tf_dkv, tf_dq = 4 * prod / (ms_dkv * 1e-3) / 1e12, 3 * prod / (ms_dq * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, ms_per_check=ms,
+                check_elements_per_s=elements / (ms * 1e-3), verdicts=[r.verdict for r in res],
+                bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3,
+                roofline=dict(bound="tensor", kernel="attn_kernel<dK/dV> + attn_kernel<dQ> (bf16 operands)",
+                              achieved=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
+                              frac=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
+                              dkv_tflops=tf_dkv, dq_tflops=tf_dq,
+                              note="7 causal products of 2*S*S*d/2 flop per head; exp on the SFU co-bounds it"),
+                diag_status=b.read_diag(diag)["status"])
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -173,6 +235,11 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     b.lib()
+
+    if args.attention_only:
+        if rank == 0:
+            print(json.dumps(dict(attention=attention_section(b, read_peaks(), steps=args.attention_steps))), flush=True)
+        return
 
     inp = workloads.config2()
     T, C, O, K = inp.T, inp.C, inp.O, inp.K
@@ -288,6 +355,10 @@ def run_ours(args):
                 e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
                 gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
                 verdicts=verdicts, diag_status=dstat["status"])
+    if not args.no_attention and world == 1:
+        del ws, flush, fresh_t
+        torch.cuda.empty_cache()
+        line["attention"] = attention_section(b, peaks, steps=args.attention_steps)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -300,6 +371,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-attention", action="store_true", help="skip the config-3 attention section")
+    ap.add_argument("--attention-only", action="store_true", help="run only the config-3 attention section")
+    ap.add_argument("--attention-steps", type=int, default=3)
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 100 and args.warmup == 5:

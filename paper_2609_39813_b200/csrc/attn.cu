@@ -52,6 +52,34 @@ __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// 2^x on the special-function unit (2^-inf = 0): one instruction per probability.
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Two floats to one packed bf16 pair (round to nearest even): `lo` in bits 0..15, `hi` in 16..31.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// tcgen05.ld of 32 columns without the wait, so several loads can be in flight before one wait.
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -142,14 +170,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = mbar_wait(b_res, 0, abort_flag);
-      for (int it = 0; it < total && ok; ++it) {
-        const bool pass2 = it >= nsteps;                      // FWD only
-        const uint32_t s = it & 1u, ph = (it >> 1) & 1u, ip = it & 1u;
-        if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(b_sdp_free, ip ^ 1u, abort_flag)) { ok = false; break; }
+      // S = Q K^T (and dP = dO V^T) of step `jt`: both operands K-major, 64 = 4 x 16 along K.
+      // Issued one step ahead: the softmax warps release the S / dP columns as soon as they hold
+      // them in registers, so these products overlap the softmax arithmetic of the step before.
+      auto issue_sdp = [&](int jt) -> bool {
+        const uint32_t s = jt & 1u, ph = (jt >> 1) & 1u;
+        if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) return false;
+        if (!mbar_wait(b_sdp_free, (jt & 1u) ^ 1u, abort_flag)) return false;
         tc_fence_after();
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
-        // S = Q K^T  (and dP = dO V^T): both operands K-major, 64 = 4 x 16 along K
         const uint32_t q_t = MODE == AT_DKV ? st0 : res0, k_t = MODE == AT_DKV ? res0 : st0;
         const uint32_t do_t = MODE == AT_DKV ? st1 : res1, v_t = MODE == AT_DKV ? res1 : st1;
         {
@@ -163,6 +192,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
         }
         tc_commit(b_sdp_full);
+        return true;
+      };
+      if (ok && total > 0) ok = issue_sdp(0);
+      for (int it = 0; it < total && ok; ++it) {
+        const bool pass2 = it >= nsteps;                      // FWD only
+        const uint32_t s = it & 1u, ip = it & 1u;
+        const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
+        if (it + 1 < total && !issue_sdp(it + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t first = (MODE == AT_FWD ? it == nsteps : it == 0) ? 0u : 1u;   // overwrite on the first product
@@ -240,68 +277,89 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sdp_full, ip, abort_flag));
       if (!ok) break;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
-      if (!ok) break;
       tc_fence_after();
+      // this thread's 64 scores (and 64 dP values) into registers, then hand the TMEM columns back
+      // at once: the next step's S and dP are computed while this step's softmax runs
+      uint32_t sv[64], dv[64];
+      tmem_ld32_nowait(t_s + lane_off + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld32_nowait(t_s + lane_off + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      if (MODE != AT_FWD) {
+        tmem_ld32_nowait(t_dp + lane_off + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&dv[0]));
+        tmem_ld32_nowait(t_dp + lane_off + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&dv[32]));
+      }
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_sdp_free);
+
       const int key0 = kblk * AT_BLK + h * 64;
+      // masking is needed only on the diagonal block and where the sequence ends inside the block
+      const bool edge = (p.causal && kblk * AT_BLK + AT_BLK - 1 > (qrow - r)) || (kblk + 1) * AT_BLK > p.S ||
+                        (qrow - r) + AT_BLK > p.S;
+      if (MODE == AT_FWD && !pass2) {
+        // running max / sum of exp2(c2 * s) over the valid keys of this half
+        float mloc = run_m;
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t sv[32], dv[32];
-        tmem_ld32(t_s + lane_off + h * 64 + ch * 32, sv);
-        if (MODE != AT_FWD) tmem_ld32(t_dp + lane_off + h * 64 + ch * 32, dv);
-        if (MODE == AT_FWD && !pass2) {
-          // running max / sum of exp2(c2 * s) over the valid keys of this half
-          float mloc = run_m;
+        for (int j = 0; j < 64; ++j) {
+          const int key = key0 + j;
+          const bool valid = !edge || (key < p.S && qrow < p.S && (!p.causal || key <= qrow));
+          if (valid) mloc = fmaxf(mloc, __uint_as_float(sv[j]) * c2);
+        }
+        if (mloc > -INFINITY) {
+          float add = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int key = key0 + ch * 32 + j;
-            const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
-            if (valid) mloc = fmaxf(mloc, __uint_as_float(sv[j]) * c2);
+          for (int j = 0; j < 64; ++j) {
+            const int key = key0 + j;
+            const bool valid = !edge || (key < p.S && qrow < p.S && (!p.causal || key <= qrow));
+            add += ex2_approx(valid ? fmaf(__uint_as_float(sv[j]), c2, -mloc) : -INFINITY);
           }
-          if (mloc > -INFINITY) {
-            float add = 0.f;
+          run_l = run_l * (run_m > -INFINITY ? ex2_approx(run_m - mloc) : 0.f) + add;
+          run_m = mloc;
+        }
+      } else {
+        uint32_t pk[32], dk[32];
+        if (!edge) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int key = key0 + ch * 32 + j;
-              const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
-              if (valid) add += exp2f(__uint_as_float(sv[j]) * c2 - mloc);
-            }
-            run_l = run_l * (run_m > -INFINITY ? exp2f(run_m - mloc) : 0.f) + add;
-            run_m = mloc;
+          for (int j = 0; j < 64; j += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sv[j]), c2, -lse2));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sv[j + 1]), c2, -lse2));
+            pk[j >> 1] = pack_bf16x2(p0, p1);
+            if (MODE != AT_FWD)
+              dk[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(dv[j]) - dq), p1 * (__uint_as_float(dv[j + 1]) - dq));
           }
         } else {
-          uint32_t pk[16], dk[16];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float pv[2], dsv[2];
+          for (int j = 0; j < 64; j += 2) {
+            float pv[2];
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-              const int key = key0 + ch * 32 + j + e;
+              const int key = key0 + j + e;
               const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
-              const float pr = valid ? exp2f(__uint_as_float(sv[j + e]) * c2 - lse2) : 0.f;
-              pv[e] = pr;
-              dsv[e] = MODE != AT_FWD ? pr * (__uint_as_float(dv[j + e]) - dq) : 0.f;
+              pv[e] = ex2_approx(valid ? fmaf(__uint_as_float(sv[j + e]), c2, -lse2) : -INFINITY);
             }
-            pk[j >> 1] = float_to_bf16_bits(pv[0]) | (float_to_bf16_bits(pv[1]) << 16);
-            dk[j >> 1] = float_to_bf16_bits(dsv[0]) | (float_to_bf16_bits(dsv[1]) << 16);
-          }
-          // 32 keys = 4 chunks of 16 bytes in row r of half h: chunk index (ch*4 + t) ^ (r & 7)
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)((ch * 4 + t) ^ (r & 7)) << 4);
-            if (MODE != AT_DQ)
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
-                           "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
+            pk[j >> 1] = pack_bf16x2(pv[0], pv[1]);
             if (MODE != AT_FWD)
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsbuf + off), "r"(dk[4 * t]), "r"(dk[4 * t + 1]),
-                           "r"(dk[4 * t + 2]), "r"(dk[4 * t + 3]) : "memory");
+              dk[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(dv[j]) - dq), pv[1] * (__uint_as_float(dv[j + 1]) - dq));
           }
         }
+        // the P / dS buffers are free once the products of the previous step have read them
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+        if (!ok) break;
+        // 64 keys = 8 chunks of 16 bytes in row r of half h: chunk index t ^ (r & 7)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+          if (MODE != AT_DQ)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
+                         "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
+          if (MODE != AT_FWD)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsbuf + off), "r"(dk[4 * t]), "r"(dk[4 * t + 1]),
+                         "r"(dk[4 * t + 2]), "r"(dk[4 * t + 3]) : "memory");
+        }
       }
-      tc_fence_before();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) { mbar_arrive(b_sdp_free); mbar_arrive(b_pds_ready); }
+      if (lane == 0) mbar_arrive(b_pds_ready);
     }
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise)
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc, 0, abort_flag));
