@@ -1,0 +1,212 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py
+times, on outputs the oracle can compute one by one: all codes and all of dgamma / dbeta, sampled
+draws, sampled column blocks of dW, sampled (batch, head) slices of attention."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import attention, check, fp8, linear, mc, norm, philox
+from paper_2609_39813_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-5
+TOL_TC = 2e-3
+
+
+@pytest.fixture(scope="module")
+def b():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39813_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _rel(a, ref):
+    a, ref = np.asarray(a, np.float64).ravel(), np.asarray(ref, np.float64).ravel()
+    return float(np.linalg.norm(a - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+FULL = {
+    "cfg2": (workloads.config2, 64),
+    "cfg4": (workloads.config4, 32),      # K = 1024 in the config; 32 draws here keep the test short
+    "cfg5": (workloads.config5, 16),
+}
+
+
+@pytest.fixture(scope="module", params=list(FULL), ids=list(FULL))
+def full(request, b):
+    from paper_2609_39813_b200.harness import NormLinearGpu, down
+    make, K = FULL[request.param]
+    inp = make()
+    g = NormLinearGpu(inp)
+    kind = norm.RMS if inp.norm == "rms" else norm.LAYER
+    rng = np.random.default_rng(7)
+    cols = np.sort(rng.choice(inp.C, 128, replace=False))
+    rows = np.sort(rng.choice(inp.O, 192, replace=False))
+    # oracle side, restricted to what the sampled outputs need: the store on all of u, dY on the
+    # sampled output rows only (its amax over the whole tensor)
+    fw = norm.forward(inp.x, inp.gamma, inp.beta, kind, inp.eps)
+    rstd32, mean32 = down(g.rstd), down(g.mean)
+    u32 = norm.store_value_fp32(inp.x, inp.gamma, inp.beta, kind, rstd32, mean32, None)
+    amax = np.float32(np.max(np.abs(u32)))
+    scale, inv = fp8.scale_from_amax(amax, inp.store_fmt)
+    v32 = norm.store_value_fp32(inp.x, inp.gamma, inp.beta, kind, rstd32, mean32, scale)
+    codes, n_sat, _ = norm.store_codes(v32, inp.store_fmt, fp8.SR, inp.seed, check.TENSOR_U, philox.STREAM_FORWARD, 0)
+    amax_dy = np.float32(np.max(np.abs(inp.dY)))
+    s_dy, inv_dy = fp8.scale_from_amax(amax_dy, inp.grad_fmt)
+    dy_sub32 = (inp.dY[:, rows] * np.float32(s_dy)).astype(np.float32)
+    dy_codes_sub, _, _ = fp8.encode(dy_sub32, inp.grad_fmt, fp8.RN)
+    dy_sub = fp8.decode(dy_codes_sub, inp.grad_fmt) * float(inv_dy)
+    prep = dict(fw=fw, rstd32=rstd32, mean32=mean32, u32=u32, amax=amax, scale=np.float32(scale),
+                inv_scale=np.float32(inv), v32=v32, codes=codes, store_fmt=inp.store_fmt, n_saturated=n_sat)
+    return dict(inp=inp, g=g, kind=kind, K=K, cols=cols, rows=rows, prep=prep, dy_sub=dy_sub,
+                dy_codes_sub=dy_codes_sub, amax_dy=amax_dy, s_dy=s_dy)
+
+
+def test_full_store_and_incoming_gradient_codes(b, full):
+    from paper_2609_39813_b200.harness import down
+    inp, g, prep = full["inp"], full["g"], full["prep"]
+    assert np.max(np.abs(down(g.rstd) / prep["fw"]["rstd"] - 1)) < 1e-6
+    assert down(g.amax)[0] == prep["amax"] and down(g.scale)[0] == prep["scale"]
+    assert np.array_equal(g.u_codes.cpu().numpy().reshape(inp.T, inp.C), prep["codes"])
+    ct = g.u_codes_t.cpu().numpy().reshape(inp.C, g.ld_t)[full["cols"], :inp.T]
+    assert np.array_equal(ct, prep["codes"][:, full["cols"]].T)
+    assert down(g.amax_dy)[0] == full["amax_dy"] and down(g.scale_dy)[0] == full["s_dy"]
+    got_dy = g.dy_codes.cpu().numpy().reshape(inp.T, inp.O)[:, full["rows"]]
+    assert np.array_equal(got_dy, full["dy_codes_sub"])
+
+
+def test_full_gain_use(b, full):
+    from paper_2609_39813_b200.harness import down, up
+    inp, g, prep, kind = full["inp"], full["g"], full["prep"], full["kind"]
+    T, C = inp.T, inp.C
+    rng = np.random.default_rng(11)
+    du_np = rng.standard_normal((T, C)).astype(np.float32)
+    if inp.dtype == "bf16":
+        du_np = workloads.to_bf16_grid(du_np)
+    du = up(du_np, inp.dtype)
+    du64 = du_np.astype(np.float64)
+    ws = b.workspace(b.bsp_norm_bwd_workspace_bytes(T, C))
+    dg, db, dx = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda"), torch.zeros(T * C, device="cuda")
+    want_u = norm.backward(inp.x, inp.gamma, inp.beta, kind, inp.eps, du64)
+    key = b.key(inp.seed, g.tensor_id, b.STREAM_GAIN, 0)
+    b.bsp_norm_bwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, du, 0, g.u_codes, g.q, key, dg, db, dx, ws)
+    assert _rel(down(dg), want_u["dgamma"]) <= TOL_FP32 and _rel(down(db), want_u["dbeta"]) <= TOL_FP32
+    idx = np.random.default_rng(3).choice(T, 64, replace=False)
+    assert _rel(down(dx).reshape(T, C)[idx], want_u["dx"][idx]) <= TOL_FP32
+    ref32 = down(dg).copy()
+    b.bsp_norm_bwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, du, 1, g.u_codes, g.q, key, dg, None, None, ws)
+    copy_r = norm.read_value(prep["codes"], inp.store_fmt, prep["inv_scale"])
+    assert _rel(down(dg), norm.dgamma_from_copy(copy_r, inp.gamma, inp.beta, du64)) <= TOL_FP32
+    # fresh read: the last draw of the config, through the single-draw entry and through the MC pass
+    k_last = full["K"] - 1
+    copy_n, _ = check.fresh_copy(prep, inp.seed, philox.STREAM_GAIN, k_last)
+    want_n = norm.dgamma_from_copy(copy_n, inp.gamma, inp.beta, du64)
+    b.bsp_norm_bwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, du, 2, g.u_codes, g.q,
+                   b.key(inp.seed, g.tensor_id, b.STREAM_GAIN, k_last), dg, None, None, ws)
+    assert _rel(down(dg), want_n) <= TOL_FP32
+    S1, S2 = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda")
+    wsg = b.workspace(b.bsp_norm_gain_mc_workspace_bytes(T, C, 1))
+    b.bsp_norm_gain_mc(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, du,
+                       b.quant(inp.store_fmt, 1, 1.0, g.scale), key, k_last, 1, up(ref32), S1, S2, wsg)
+    d = want_n - ref32.astype(np.float64)
+    assert np.linalg.norm(down(S1) - d) <= TOL_FP32 * np.linalg.norm(want_n)
+    assert _rel(down(S2), d * d) <= 1e-3
+
+
+def test_full_weight_use(b, full):
+    from paper_2609_39813_b200.harness import down
+    inp, g, prep = full["inp"], full["g"], full["prep"]
+    T, C, O, cols, rows, dy = inp.T, inp.C, inp.O, full["cols"], full["rows"], full["dy_sub"]
+    pick = np.ix_(rows, cols)
+    dW = torch.zeros(O * C, device="cuda")
+    ws = b.workspace(b.bsp_linear_wgrad_workspace_bytes(T, O, C, 0))
+    diag = b.new_diag()
+    # R (the reference) and U on the sampled block
+    b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, 1, g.u_codes_t, g.q, g.ld_t, dW, ws=ws, diag=diag)
+    x_r = norm.read_value(prep["codes"][:, cols], inp.store_fmt, prep["inv_scale"])
+    ref = dy.T @ x_r
+    assert _rel(down(dW).reshape(O, C)[pick], ref) <= TOL_TC
+    ref_dev = dW.clone()
+    b.bsp_linear_wgrad(T, O, C, g.dy_codes_t, g.q_dy, 0, g.u_bf16_t, g.q, g.ld_t, dW, ws=ws, diag=diag)
+    x_u = linear.bf16_round(prep["u32"][:, cols].astype(np.float64))
+    assert _rel(down(dW).reshape(O, C)[pick], dy.T @ x_u) <= TOL_TC
+    # N: the two last draws through the batched re-rounding + Monte-Carlo contraction
+    K = full["K"]
+    q = b.quant(inp.store_fmt, 1, 1.0, g.scale)
+    fresh = torch.zeros(2 * C * g.ld_t, dtype=torch.uint8, device="cuda")
+    b.bsp_norm_fwd_draws(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, q,
+                         b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, 0), K - 2, 2, fresh, g.ld_t)
+    S1, S2 = torch.zeros(O * C, device="cuda"), torch.zeros(O * C, device="cuda")
+    b.bsp_linear_wgrad_mc(T, O, C, g.dy_codes_t, g.q_dy, fresh, q, g.ld_t, 2, ref_dev, S1, S2, diag)
+    assert b.read_diag(diag)["status"] == 0
+    got_codes = fresh.cpu().numpy().reshape(2, C, g.ld_t)
+    ref32 = down(ref_dev).reshape(O, C)[pick].astype(np.float64)
+    s1 = np.zeros_like(ref32)
+    s2 = np.zeros_like(ref32)
+    for d, k in enumerate((K - 2, K - 1)):
+        copy, codes = check.fresh_copy(prep, inp.seed, philox.STREAM_WGRAD, k, cols)
+        assert np.array_equal(got_codes[d][cols, :T], codes.T)
+        gk = dy.T @ copy
+        s1 += gk - ref32
+        s2 += (gk - ref32) ** 2
+    scale = np.linalg.norm(ref32)
+    assert np.linalg.norm(down(S1).reshape(O, C)[pick] - s1) <= TOL_TC * scale
+    assert _rel(down(S2).reshape(O, C)[pick], s2) <= 2e-2
+
+
+def test_full_mc_check_verdicts(b, full):
+    inp, g, K = full["inp"], full["g"], full["K"]
+    desc = g.desc()
+    ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
+    diag = b.new_diag()
+    res = b.bsp_mc_check(desc, K, ws, diag)
+    assert b.read_diag(diag)["status"] == 0
+    # gain use: U holds exactly, R fails, N holds on average; weight use: U fails, R holds exactly,
+    # N fails (its mean tends to the original's value)
+    assert [r.verdict for r in res] == [mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS]
+    assert res[0].rel_l2_mean_err == 0.0 and res[4].rel_l2_mean_err == 0.0
+    assert 0.005 < res[1].rel_l2_mean_err < 0.5 and 0.005 < res[3].rel_l2_mean_err < 0.5
+    assert res[2].Qprime < 1.6 and res[2].R < 2.0 and res[5].R > 6.0
+    assert [r.n_elements for r in res] == [inp.C] * 3 + [inp.O * inp.C] * 3
+
+
+def test_full_attention_sampled_heads(b):
+    """Config 3 at full size; the oracle evaluates two (batch, head) slices."""
+    from paper_2609_39813_b200.harness import up
+    inp = workloads.config3()
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    n = B * H * S * D
+    q, k, v, dO = (up(a, "bf16") for a in (inp.q, inp.k, inp.v, inp.dO))
+    o, lse = torch.zeros(n, device="cuda"), torch.zeros(B * H * S, device="cuda")
+    diag = b.new_diag()
+    b.bsp_attn_fwd_stats(B, H, S, D, True, inp.softmax_scale, q, k, v, o, lse, diag)
+    amax, scales = torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
+    b.bsp_amax(o, B * H, S * D, amax)
+    b.bsp_scale_from_amax(amax, B * H, fp8.E4M3, scales)
+    codes = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    b.bsp_round_grouped(o, B * H, S * D, fp8.E4M3, fp8.SR, scales, b.key(inp.seed, check.TENSOR_O, 0, 0), codes)
+    dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
+    d_out = torch.zeros(B * H * S, device="cuda")
+    pol, draw = 2, 31
+    b.bsp_attn_bwd(B, H, S, D, True, inp.softmax_scale, 0, q, k, v, dO, lse, o, codes, scales, fp8.E4M3, pol,
+                   b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, draw), dq, dk, dv, d_out, diag)
+    assert b.read_diag(diag)["status"] == 0
+    oh = o.cpu().numpy().reshape(B * H, S, D)
+    ch = codes.cpu().numpy().reshape(B * H, S, D)
+    for idx in (5, 127):
+        bi, hi = divmod(idx, H)
+        qs, ks, vs, dOs = inp.q[bi, hi], inp.k[bi, hi], inp.v[bi, hi], inp.dO[bi, hi]
+        want_o, want_lse = attention.forward_output(qs, ks, vs, inp.softmax_scale, True)
+        assert _rel(oh[idx], want_o) <= TOL_TC
+        assert np.max(np.abs(lse.cpu().numpy().reshape(B * H, S)[idx] - want_lse)) <= 1e-4
+        prep = check.prepare_attention_slice(qs, ks, vs, dOs, inp.softmax_scale, inp.seed, idx, True, o32=oh[idx])
+        assert np.array_equal(ch[idx], prep["codes"])
+        copy = check.attention_d_copy(prep, pol, inp.seed, draw)
+        want = attention.backward(qs, ks, vs, dOs, inp.softmax_scale, copy, True, operand_round=linear.bf16_round)
+        assert _rel(d_out.cpu().numpy().reshape(B * H, S)[idx], want["D"]) <= TOL_FP32
+        for name, t in (("dq", dq), ("dk", dk), ("dv", dv)):
+            assert _rel(t.cpu().numpy().reshape(B * H, S, D)[idx], want[name]) <= TOL_TC, (name, idx)
