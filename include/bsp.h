@@ -304,8 +304,9 @@ int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, b
  * next layer consumes it; the correction term D is the one use of the saved output, and reading a
  * copy O + E adds rowsum(dO o E) (Eq. dterm).  Tensors are [B, H, S, Dh] row-major, bf16 inputs
  * (dt = BSP_BF16), Dh = 64, FP32 outputs; lse, D are [B, H, S].  BF16 tensor-core operands (P and
- * dS are rounded to bf16 for their products); the FP8-operand variant of Appendix "The forks" is
- * not built (fp8_operands != 0 returns BSP_ERR_UNSUPPORTED).
+ * dS are rounded to bf16 for their products).  The FP8-operand variant of Appendix "The forks" has
+ * its own entry points (bsp_attn_*_fp8, below) because it needs the operand scales; in
+ * bsp_attn_bwd the flag fp8_operands must be 0 (otherwise BSP_ERR_UNSUPPORTED).
  * ------------------------------------------------------------------------------------------ */
 
 /* Forward statistics from the operands exactly as the backward will see them: o = P V (FP32, the
@@ -336,6 +337,45 @@ int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, i
                  const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt,
                  int d_read, bsp_key_t key, float* dq, float* dk, float* dv, float* d_out,
                  bsp_diag_t* diag, void* stream);
+
+/* FP8-operand mode, after the emulated FP8 attention backward of Appendix "The forks": Q, K, V are
+ * rounded to nearest onto E4M3 and dO onto E5M2, each at the per-(b,h) amax scale of its slice; P is
+ * recomputed (unrounded) from the dequantised Q and K; dV = P_q^T dO with P_q = RN_E4M3(P p_scale)
+ * / p_scale; dP = dO V^T; D from the assigned output copy; dS = P o (dP - D); dS_q = RN_E5M2(dS
+ * ds_scale) / ds_scale feeds dQ and dK (ds_scale supplied by the caller, like a delayed scale).
+ * The quantised operands travel as bf16 tensors holding the DECODED codes (every FP8 value is a
+ * bf16 value, so the tensor-core products are those of the FP8 operands exactly); their scales
+ * are folded back in the kernel.  The final E5M2 cast of the returned gradients is not applied
+ * (outputs FP32).  Quantisation points and the two scales are this library's reading of that
+ * appendix. */
+typedef struct {
+  const float* q_scale;      /* [B*H] device: scale of each slice of q8 (code = round(x * scale)) */
+  const float* k_scale;
+  const float* v_scale;
+  const float* do_scale;
+  float p_scale;             /* power of two; 256 keeps P * p_scale <= 256 < 448 */
+  float ds_scale;
+} bsp_attn_fp8_t;
+
+/* xq (bf16, same shape) = decode(RN_fmt(x * scale_g)) for each of n_groups contiguous groups of
+ * group_size bf16 elements, scale_g = fmax / amax_g; amax[n_groups] and scales[n_groups] are
+ * written too.  group_size a multiple of 8. */
+int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax,
+                      float* scales, bsp_diag_t* diag, void* stream);
+
+/* bsp_attn_fwd_stats on quantised operands (q8, k8, v8 from bsp_attn_quantize): o = P V_hat in
+ * FP32 with P unrounded, lse from the dequantised q and k. */
+int bsp_attn_fwd_stats_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8,
+                           const void* k8, const void* v8, int dt, const bsp_attn_fp8_t* fp8, float* o,
+                           float* lse, bsp_diag_t* diag, void* stream);
+
+/* bsp_attn_bwd in FP8-operand mode; dO8 holds the decoded E5M2 codes of dO, D = rowsum(dO_hat o
+ * O_copy) with dO_hat = dO8 / do_scale. */
+int bsp_attn_bwd_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8,
+                     const void* k8, const void* v8, const void* dO8, int dt, const bsp_attn_fp8_t* fp8,
+                     const float* lse, const float* o_orig, const uint8_t* o_codes, const float* o_scales,
+                     int o_fmt, int d_read, bsp_key_t key, float* dq, float* dk, float* dv, float* d_out,
+                     bsp_diag_t* diag, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Monte-Carlo reduction (Section "Each use has a checkable requirement").

@@ -64,6 +64,11 @@ class AttnDesc(C.Structure):
                 ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
 
 
+class AttnFp8(C.Structure):
+    _fields_ = [("q_scale", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
+                ("do_scale", C.c_void_p), ("p_scale", C.c_float), ("ds_scale", C.c_float)]
+
+
 class BspError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
@@ -106,6 +111,10 @@ _SIGNATURES = {
     "bsp_attn_bwd_dterm": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P]),
     "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, _P, _P, _P, _P, _I, _I, Key, _P, _P, _P,
                           _P, _P, _P]),
+    "bsp_attn_quantize": (_I, [_P, _I, _SZ, _I, _P, _P, _P, _P, _P]),
+    "bsp_attn_fwd_stats_fp8": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P]),
+    "bsp_attn_bwd_fp8": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _I, _I,
+                              Key, _P, _P, _P, _P, _P, _P]),
     "bsp_mc_accumulate": (_I, [_P, _P, _P, _P, _SZ, _P]),
     "bsp_mc_check_attn_workspace_bytes": (_SZ, [C.POINTER(AttnDesc), _I]),
     "bsp_mc_check_attn": (_I, [C.POINTER(AttnDesc), _I, C.POINTER(UseResult), C.POINTER(_I), _P, _SZ, _P, _P]),
@@ -358,6 +367,29 @@ def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, 
                              ptr(dO), dtype_code(q), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales), o_fmt,
                              d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
           "bsp_attn_bwd")
+
+
+def bsp_attn_quantize(x, n_groups, group_size, fmt, xq, amax, scales, diag=None, stream=None):
+    check(lib().bsp_attn_quantize(ptr(x), n_groups, group_size, fmt, ptr(xq), ptr(amax), ptr(scales), ptr(diag),
+                                  _st(stream)), "bsp_attn_quantize")
+
+
+def attn_fp8(q_scale, k_scale, v_scale, do_scale, p_scale=256.0, ds_scale=1.0) -> AttnFp8:
+    return AttnFp8(ptr(q_scale), ptr(k_scale), ptr(v_scale), ptr(do_scale), float(p_scale), float(ds_scale))
+
+
+def bsp_attn_fwd_stats_fp8(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, f: AttnFp8, o, lse, diag=None, stream=None):
+    check(lib().bsp_attn_fwd_stats_fp8(B, H, S, Dh, int(causal), softmax_scale, ptr(q8), ptr(k8), ptr(v8),
+                                       dtype_code(q8), C.byref(f), ptr(o), ptr(lse), ptr(diag), _st(stream)),
+          "bsp_attn_fwd_stats_fp8")
+
+
+def bsp_attn_bwd_fp8(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dO8, f: AttnFp8, lse, o_orig, o_codes, o_scales,
+                     o_fmt, d_read, key_: Key, dq, dk, dv, d_out, diag=None, stream=None):
+    check(lib().bsp_attn_bwd_fp8(B, H, S, Dh, int(causal), softmax_scale, ptr(q8), ptr(k8), ptr(v8), ptr(dO8),
+                                 dtype_code(q8), C.byref(f), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales),
+                                 o_fmt, d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
+          "bsp_attn_bwd_fp8")
 
 
 def bsp_mc_accumulate(g, g_ref, S1, S2, n, stream=None):

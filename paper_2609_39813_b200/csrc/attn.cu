@@ -46,6 +46,15 @@ struct AttnParams {
   float* out1;                   // DKV: dK                         [BH*S*64]
   float* lse_out;                // FWD
   bsp_diag_t* diag;
+  // FP8-operand mode: q, k, v, dO hold decoded FP8 codes (exact in bf16); their per-(b,h) scales
+  // are folded into the softmax argument, dP and the outputs; P and dS are rounded onto the E4M3 /
+  // E5M2 grids (at p_scale / ds_scale) before their products.  All NULL / 0 in BF16-operand mode.
+  int fp8;
+  const float* sc_q;             // [BH]
+  const float* sc_k;
+  const float* sc_v;
+  const float* sc_do;
+  float p_scale, ds_scale;
 };
 
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
@@ -232,7 +241,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const int q4 = warp & 3, h = (warp - 2) >> 2;
     const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
-    const float c2 = p.c * kLog2e;
+    float inv_q = 1.f, inv_k = 1.f, inv_v = 1.f, inv_do = 1.f;
+    if (p.fp8) {
+      inv_q = __fdiv_rn(1.0f, __ldg(p.sc_q + bh)); inv_k = __fdiv_rn(1.0f, __ldg(p.sc_k + bh));
+      inv_v = __fdiv_rn(1.0f, __ldg(p.sc_v + bh)); inv_do = __fdiv_rn(1.0f, __ldg(p.sc_do + bh));
+    }
+    const float c2 = p.c * kLog2e * inv_q * inv_k;            // scores arrive as products of decoded codes
+    const float dp_mul = inv_do * inv_v;                      // likewise dP
     bool ok = true;
     float lse2 = 0.f, dq = 0.f;                               // this row's LSE*log2e and D
     int qrow = 0;                                             // global query index of this thread's row
@@ -318,14 +333,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
       } else {
         uint32_t pk[32], dk[32];
+        // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
+        // first rounds P onto the E4M3 grid at p_scale and dS onto the E5M2 grid at ds_scale (the
+        // grid values are exact in bf16; the scales come back in the epilogue).
+        auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, uint32_t& po, uint32_t& dso) {
+          float s0 = 0.f, s1 = 0.f;
+          if (MODE != AT_FWD) {
+            s0 = p0 * (__uint_as_float(dp0) * dp_mul - dq);
+            s1 = p1 * (__uint_as_float(dp1) * dp_mul - dq);
+          }
+          if (p.fp8 && MODE != AT_FWD) {                    // the forward keeps P unrounded
+            p0 = f8_rn_value<BSP_E4M3>(p0 * p.p_scale); p1 = f8_rn_value<BSP_E4M3>(p1 * p.p_scale);
+            s0 = f8_rn_value<BSP_E5M2>(s0 * p.ds_scale); s1 = f8_rn_value<BSP_E5M2>(s1 * p.ds_scale);
+          }
+          po = pack_bf16x2(p0, p1);
+          if (MODE != AT_FWD) dso = pack_bf16x2(s0, s1);
+        };
         if (!edge) {
 #pragma unroll
           for (int j = 0; j < 64; j += 2) {
             const float p0 = ex2_approx(fmaf(__uint_as_float(sv[j]), c2, -lse2));
             const float p1 = ex2_approx(fmaf(__uint_as_float(sv[j + 1]), c2, -lse2));
-            pk[j >> 1] = pack_bf16x2(p0, p1);
-            if (MODE != AT_FWD)
-              dk[j >> 1] = pack_bf16x2(p0 * (__uint_as_float(dv[j]) - dq), p1 * (__uint_as_float(dv[j + 1]) - dq));
+            pack_pair(p0, p1, dv[j], dv[j + 1], pk[j >> 1], dk[j >> 1]);
           }
         } else {
 #pragma unroll
@@ -337,9 +366,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
               const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
               pv[e] = ex2_approx(valid ? fmaf(__uint_as_float(sv[j + e]), c2, -lse2) : -INFINITY);
             }
-            pk[j >> 1] = pack_bf16x2(pv[0], pv[1]);
-            if (MODE != AT_FWD)
-              dk[j >> 1] = pack_bf16x2(pv[0] * (__uint_as_float(dv[j]) - dq), pv[1] * (__uint_as_float(dv[j + 1]) - dq));
+            pack_pair(pv[0], pv[1], dv[j], dv[j + 1], pk[j >> 1], dk[j >> 1]);
           }
         }
         // the P / dS buffers are free once the products of the previous step have read them
@@ -369,7 +396,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (MODE == AT_DKV) {
         // h = 0 warps write dV (acc0), h = 1 warps write dK (acc1, times the softmax scale)
         float* dst = (h == 0 ? p.out0 : p.out1) + ((size_t)bh * p.S + grow) * AT_D;
-        const float mul = h == 0 ? 1.f : p.c;
+        const float mul = h == 0 ? (p.fp8 ? inv_do / p.p_scale : 1.f) : p.c * (p.fp8 ? inv_q / p.ds_scale : 1.f);
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           uint32_t a[32];
@@ -385,7 +412,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       } else {
         // each column half writes 32 of the 64 output columns
         float* dst = p.out0 + ((size_t)bh * p.S + grow) * AT_D + h * 32;
-        const float mul = MODE == AT_DQ ? p.c : 1.f;
+        const float mul = MODE == AT_DQ ? p.c * (p.fp8 ? inv_k / p.ds_scale : 1.f) : inv_v;
         uint32_t a[32];
         tmem_ld32(t_acc0 + lane_off + h * 32, a);
         if (grow < p.S) {
@@ -417,8 +444,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 template <int DT, int FMT>
 __global__ void __launch_bounds__(256)
 attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig, const uint8_t* __restrict__ o_codes,
-                  const float* __restrict__ o_scales, int64_t rows, int S, int policy, PhiloxKey key, int draw0,
-                  int n_draws, float* __restrict__ D) {
+                  const float* __restrict__ o_scales, const float* __restrict__ do_scales, int64_t rows, int S,
+                  int policy, PhiloxKey key, int draw0, int n_draws, float* __restrict__ D) {
   const int64_t row = (int64_t)blockIdx.x * 16 + (threadIdx.x >> 4);
   const int sub = threadIdx.x & 15;
   const bool active = row < rows;
@@ -427,10 +454,13 @@ attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig,
   const size_t i0 = (size_t)(active ? row : 0) * AT_D + sub * 4;
   if (active) {
     g = load4<DT>(dO, i0);
-    if (policy != BSP_READ_ORIGINAL || true) {
-      scale = o_scales ? __ldg(o_scales + row / S) : 1.f;
-      inv = __fdiv_rn(1.0f, scale);
+    if (do_scales) {
+      // dO holds decoded FP8 codes: bring back its per-(b,h) scale
+      const float inv_do = __fdiv_rn(1.0f, __ldg(do_scales + row / S));
+      g.x *= inv_do; g.y *= inv_do; g.z *= inv_do; g.w *= inv_do;
     }
+    scale = o_scales ? __ldg(o_scales + row / S) : 1.f;
+    inv = __fdiv_rn(1.0f, scale);
     if (policy == BSP_READ_FORWARD) {
       const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(o_codes + i0));
       o = make_float4(f8_decode<FMT>(pk & 0xFFu) * inv, f8_decode<FMT>((pk >> 8) & 0xFFu) * inv,
@@ -512,6 +542,38 @@ static int check_attn_shape(int B, int H, int S, int Dh, int dt) {
   return BSP_OK;
 }
 
+static int set_fp8(AttnParams& p, const bsp_attn_fp8_t* f) {
+  p.fp8 = f ? 1 : 0;
+  p.sc_q = f ? f->q_scale : nullptr; p.sc_k = f ? f->k_scale : nullptr;
+  p.sc_v = f ? f->v_scale : nullptr; p.sc_do = f ? f->do_scale : nullptr;
+  p.p_scale = f ? f->p_scale : 1.f; p.ds_scale = f ? f->ds_scale : 1.f;
+  if (f && (!f->q_scale || !f->k_scale || !f->v_scale || !f->do_scale || !(f->p_scale > 0.f) || !(f->ds_scale > 0.f)))
+    return BSP_ERR_ARG;
+  return BSP_OK;
+}
+
+static int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                         const void* v, int dt, const bsp_attn_fp8_t* f, float* o, float* lse, bsp_diag_t* diag,
+                         void* stream) {
+  int rc = check_attn_shape(B, H, S, Dh, dt);
+  if (rc != BSP_OK) return rc;
+  if (!q || !k || !v || !o || !lse) return BSP_ERR_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
+  AttnParams p;
+  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
+  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag;
+  if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
+  return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
+}
+
+static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
+                           const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
+                           bsp_key_t key, int draw0, int n_draws, float* d_out, void* stream);
+static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                               const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* f,
+                               const float* lse, const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
+                               void* stream);
+
 }  // namespace bsp
 
 using namespace bsp;
@@ -520,20 +582,24 @@ extern "C" {
 
 int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
                        const void* v, int dt, float* o, float* lse, bsp_diag_t* diag, void* stream) {
-  int rc = check_attn_shape(B, H, S, Dh, dt);
-  if (rc != BSP_OK) return rc;
-  if (!q || !k || !v || !o || !lse) return BSP_ERR_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
-  AttnParams p;
-  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag;
-  return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
+  return attn_fwd_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dt, nullptr, o, lse, diag, stream);
 }
 
 int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig, const uint8_t* o_codes,
                    const float* o_scales, int o_fmt, int d_read, bsp_key_t key, int draw0, int n_draws, float* d_out,
                    bsp_diag_t* diag, void* stream) {
   (void)diag;
+  return attn_dterm_impl(B, H, S, Dh, dO, dt, nullptr, o_orig, o_codes, o_scales, o_fmt, d_read, key, draw0, n_draws,
+                         d_out, stream);
+}
+
+}  // extern "C"
+
+namespace bsp {
+
+static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
+                           const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
+                           bsp_key_t key, int draw0, int n_draws, float* d_out, void* stream) {
   if (B <= 0 || H <= 0 || S <= 0 || !valid_enum(dt, 1) || !valid_enum(o_fmt, 1) || !valid_enum(d_read, 2)) return BSP_ERR_ARG;
   if (Dh != AT_D) return BSP_ERR_UNSUPPORTED;
   if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0 || draw0 < 0 || n_draws < 0) return BSP_ERR_ARG;
@@ -548,8 +614,8 @@ int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const fl
   cudaStream_t st = (cudaStream_t)stream;
   const PhiloxKey pk = make_key(key);
 #define BSP_DT(DT, FMT)                                                                                          \
-  attn_dterm_kernel<DT, FMT><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, rows, S, d_read, pk, draw0,    \
-                                                   n_draws, d_out)
+  attn_dterm_kernel<DT, FMT><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read,    \
+                                                   pk, draw0, n_draws, d_out)
   if (dt == BSP_F32 && o_fmt == BSP_E4M3) BSP_DT(BSP_F32, BSP_E4M3);
   else if (dt == BSP_F32) BSP_DT(BSP_F32, BSP_E5M2);
   else if (o_fmt == BSP_E4M3) BSP_DT(BSP_BF16, BSP_E4M3);
@@ -559,9 +625,10 @@ int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const fl
   return BSP_OK;
 }
 
-int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
-                       const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq,
-                       float* dk, float* dv, bsp_diag_t* diag, void* stream) {
+static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                               const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* f,
+                               const float* lse, const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
+                               void* stream) {
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !dO || !lse || !dterm) return BSP_ERR_ARG;
@@ -572,6 +639,7 @@ int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_sc
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
   p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag;
+  if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   if (dk) {
     p.out0 = dv; p.out1 = dk;
@@ -584,16 +652,89 @@ int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_sc
   return BSP_OK;
 }
 
+// x (bf16 [groups][group_size]) -> nearest FP8 codes at each group's own amax scale -> the decoded
+// codes as bf16 (exact), plus the scales.
+template <int FMT>
+__global__ void __launch_bounds__(256)
+quantize_decode_kernel(const uint16_t* __restrict__ x, size_t group_size, const float* __restrict__ scales,
+                       uint16_t* __restrict__ out, size_t n8) {
+  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n8) return;
+  const size_t i0 = t * 8;
+  const float s = __ldg(scales + i0 / group_size);
+  const uint4 raw = __ldg(reinterpret_cast<const uint4*>(x) + t);
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  uint32_t o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float a = f8_rn_value<FMT>(__fmul_rn(bf16_bits_to_float(w[i] & 0xFFFFu), s));
+    const float b = f8_rn_value<FMT>(__fmul_rn(bf16_bits_to_float(w[i] >> 16), s));
+    o[i] = (__float_as_uint(a) >> 16) | (__float_as_uint(b) & 0xFFFF0000u);     // FP8 values are exact in bf16
+  }
+  reinterpret_cast<uint4*>(out)[t] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+}  // namespace bsp
+
+extern "C" {
+
+int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                       const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq,
+                       float* dk, float* dv, bsp_diag_t* diag, void* stream) {
+  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, nullptr, lse, dterm, dq, dk, dv, diag,
+                             stream);
+}
+
 int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands, const void* q,
                  const void* k, const void* v, const void* dO, int dt, const float* lse, const float* o_orig,
                  const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key, float* dq,
                  float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
-  if (fp8_operands) return BSP_ERR_UNSUPPORTED;
+  if (fp8_operands) return BSP_ERR_UNSUPPORTED;      // that mode needs the operand scales: bsp_attn_bwd_fp8
   if (!d_out) return BSP_ERR_ARG;
   int rc = bsp_attn_dterm(B, H, S, Dh, dO, dt, o_orig, o_codes, o_scales, o_fmt, d_read, key, (int)key.draw, 1, d_out,
                           diag, stream);
   if (rc != BSP_OK) return rc;
   return bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, lse, d_out, dq, dk, dv, diag, stream);
+}
+
+int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax, float* scales,
+                      bsp_diag_t* diag, void* stream) {
+  if (!x || !xq || !amax || !scales || n_groups <= 0 || !valid_enum(fmt, 1)) return BSP_ERR_ARG;
+  if (group_size == 0 || group_size % 8 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(xq)) return BSP_ERR_ALIGN;
+  int rc = bsp_amax(x, BSP_BF16, (size_t)n_groups, group_size, amax, diag, stream);
+  if (rc != BSP_OK) return rc;
+  if ((rc = bsp_scale_from_amax(amax, (size_t)n_groups, fmt, scales, stream)) != BSP_OK) return rc;
+  const size_t n8 = (size_t)n_groups * group_size / 8;
+  const unsigned grid = (unsigned)((n8 + 255) / 256);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (fmt == BSP_E4M3)
+    quantize_decode_kernel<BSP_E4M3><<<grid, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), group_size, scales,
+                                                           reinterpret_cast<uint16_t*>(xq), n8);
+  else
+    quantize_decode_kernel<BSP_E5M2><<<grid, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), group_size, scales,
+                                                           reinterpret_cast<uint16_t*>(xq), n8);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
+
+int bsp_attn_fwd_stats_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8, const void* k8,
+                           const void* v8, int dt, const bsp_attn_fp8_t* fp8, float* o, float* lse, bsp_diag_t* diag,
+                           void* stream) {
+  if (!fp8) return BSP_ERR_ARG;
+  return attn_fwd_impl(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dt, fp8, o, lse, diag, stream);
+}
+
+int bsp_attn_bwd_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8, const void* k8,
+                     const void* v8, const void* dO8, int dt, const bsp_attn_fp8_t* fp8, const float* lse,
+                     const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
+                     bsp_key_t key, float* dq, float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
+  if (!fp8 || !d_out || !fp8->do_scale) return BSP_ERR_ARG;
+  int rc = attn_dterm_impl(B, H, S, Dh, dO8, dt, fp8->do_scale, o_orig, o_codes, o_scales, o_fmt, d_read, key,
+                           (int)key.draw, 1, d_out, stream);
+  if (rc != BSP_OK) return rc;
+  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dO8, dt, fp8, lse, d_out, dq, dk, dv, diag,
+                             stream);
 }
 
 int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, size_t n, void* stream) {

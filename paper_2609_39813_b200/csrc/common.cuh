@@ -164,6 +164,28 @@ __device__ __forceinline__ float f8_sr_value(float v, uint32_t U) {
   return __uint_as_float(s | __float_as_uint(mag));
 }
 
+// Value of the nearest-even rounding of v as FP32, i.e. decode(encode_RN(v)); saturating.
+template <int FMT>
+__device__ __forceinline__ float f8_rn_value(float v) {
+  using F = F8<FMT>;
+  const uint32_t b = __float_as_uint(v);
+  const uint32_t a = b & 0x7FFFFFFFu;
+  const uint32_t s = b & 0x80000000u;
+  if (a >= F::FMAX_BITS) {
+    if (a > 0x7F800000u) return __uint_as_float(0x7FC00000u);
+    return __uint_as_float(s | F::FMAX_BITS);
+  }
+  if (a >= F::MINNORM_BITS) {
+    constexpr int d = 23 - F::MB;
+    const uint32_t lsb = (a >> d) & 1u;
+    const uint32_t r = (a + ((1u << (d - 1)) - 1u) + lsb) & ~((1u << d) - 1u);   // ties to even
+    return __uint_as_float(s | r);
+  }
+  const float t = __uint_as_float(a) * __uint_as_float((uint32_t)(F::MB - F::EMIN + 127) << 23);
+  const float n = rintf(t);                                                      // ties to even, t < 2^MB
+  return __uint_as_float(s | __float_as_uint(n * __uint_as_float((uint32_t)(F::EMIN - F::MB + 127) << 23)));
+}
+
 // Exact FP32 value of a code.
 template <int FMT>
 __device__ __forceinline__ float f8_decode(uint32_t c) {

@@ -194,6 +194,60 @@ def test_mc_check_attention_verdicts(b):
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
 
 
+@pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks"])
+def test_fp8_operand_mode(b, name):
+    """The emulated FP8 attention backward: Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice, P rounded
+    to E4M3 at scale 256 before dV, dS rounded to E5M2 at a supplied scale before dQ and dK."""
+    from paper_2609_39813_b200.harness import up
+    cfg = CASES[name]
+    inp = workloads.config3(B=cfg["B"], H=cfg["H"], S=cfg["S"], D=64, K=4, seed=2000 + cfg["S"])
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    BH, n = B * H, B * H * S * D
+    dev = {}
+    for nm, arr, fmt in (("q", inp.q, fp8.E4M3), ("k", inp.k, fp8.E4M3), ("v", inp.v, fp8.E4M3), ("dO", inp.dO, fp8.E5M2)):
+        x = up(arr, "bf16")
+        xq = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+        amax, sc = torch.zeros(BH, device="cuda"), torch.zeros(BH, device="cuda")
+        b.bsp_attn_quantize(x, BH, S * D, fmt, xq, amax, sc)
+        dev[nm] = (xq, sc)
+    # quantised operands: bit-exact against the oracle's nearest rounding at the slice's amax scale
+    hat = {}
+    for nm, arr, fmt in (("q", inp.q, fp8.E4M3), ("k", inp.k, fp8.E4M3), ("v", inp.v, fp8.E4M3), ("dO", inp.dO, fp8.E5M2)):
+        got = dev[nm][0].float().cpu().numpy().reshape(BH, S, D)
+        scs = dev[nm][1].cpu().numpy()
+        vals = np.zeros((BH, S, D))
+        for idx in range(BH):
+            value, codes, s32, _ = attention.quantise_rn(arr.reshape(BH, S, D)[idx], fmt)
+            assert scs[idx] == s32
+            assert np.array_equal(got[idx], fp8.decode(codes, fmt).astype(np.float32))
+            vals[idx] = value
+        hat[nm] = vals
+    # one dS scale for the whole tensor, from the exact dS of the first slice (a "previous amax")
+    o0, _ = attention.forward_output(hat["q"][0], hat["k"][0], hat["v"][0], inp.softmax_scale, cfg["causal"])
+    ds0 = attention.backward(hat["q"][0], hat["k"][0], hat["v"][0], hat["dO"][0], inp.softmax_scale, o0, cfg["causal"])["dS"]
+    ds_scale = float(np.float32(2.0 ** np.floor(np.log2(57344.0 / (2.0 * np.max(np.abs(ds0)))))))
+    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale)
+    o, lse = torch.zeros(n, device="cuda"), torch.zeros(BH * S, device="cuda")
+    diag = b.new_diag()
+    b.bsp_attn_fwd_stats_fp8(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], f, o, lse, diag)
+    dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
+    d_out = torch.zeros(BH * S, device="cuda")
+    b.bsp_attn_bwd_fp8(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], dev["dO"][0],
+                       f, lse, o, None, None, fp8.E4M3, 0, b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0),
+                       dq, dk, dv, d_out, diag)
+    assert b.read_diag(diag)["status"] == 0
+    oh = o.cpu().numpy().reshape(BH, S, D)
+    for idx in range(BH):
+        want_o, want_lse = attention.forward_output(hat["q"][idx], hat["k"][idx], hat["v"][idx], inp.softmax_scale, cfg["causal"])
+        assert _rel(oh[idx], want_o) <= TOL_TC
+        assert np.max(np.abs(lse.cpu().numpy().reshape(BH, S)[idx] - want_lse)) <= 1e-4
+        want = attention.backward(hat["q"][idx], hat["k"][idx], hat["v"][idx], hat["dO"][idx], inp.softmax_scale,
+                                  oh[idx].astype(np.float64), cfg["causal"], True, 256.0, ds_scale)
+        assert _rel(d_out.cpu().numpy().reshape(BH, S)[idx], want["D"]) <= TOL_FP32
+        for nm, t in (("dq", dq), ("dk", dk), ("dv", dv)):
+            assert _rel(t.cpu().numpy().reshape(BH, S, D)[idx], want[nm]) <= TOL_TC, (nm, idx)
+
+
 def test_attention_row_case_of_the_paper(b):
     """One causal row of 64 keys with uniform attention; saved entry x = 5/4 +- 1/4, dO = h at that
     entry: dQ[63, 0] = c h (s - x).  In BF16-operand mode P = exp(S - LSE) is exact only to FP32
