@@ -164,6 +164,17 @@ __device__ __forceinline__ float f8_sr_value(float v, uint32_t U) {
   return __uint_as_float(s | __float_as_uint(mag));
 }
 
+// Nearest-even rounding of two in-range FP32 values (|v| below the format's maximum) to two codes
+// with the hardware conversion: `lo` in bits 0..7, `hi` in bits 8..15.  NaN, infinities and
+// magnitudes at or above the maximum never come here (the callers route those to f8_encode).
+template <int FMT>
+__device__ __forceinline__ uint32_t f8_encode_rn_pair_inrange(float lo, float hi) {
+  uint16_t r;
+  if (FMT == BSP_E4M3) asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  else asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return (uint32_t)r;
+}
+
 // Value of the nearest-even rounding of v as FP32, i.e. decode(encode_RN(v)); saturating.
 template <int FMT>
 __device__ __forceinline__ float f8_rn_value(float v) {
@@ -206,6 +217,25 @@ __device__ __forceinline__ float f8_decode(uint32_t c) {
   return __uint_as_float(s | ((ef - F::BIAS + 127u) << 23) | (m << (23 - F::MB)));
 }
 
+// Four codes (packed little-endian in one word) to FP32 with the hardware conversions: FP8 pair ->
+// f16 pair (exact: every E4M3 / E5M2 value is an f16 value) -> FP32.  NaN and infinity codes come
+// out as FP32 NaN / infinity.
+template <int FMT>
+__device__ __forceinline__ void f8_decode4(uint32_t packed, float (&out)[4]) {
+  uint32_t h01, h23;
+  const uint16_t lo = (uint16_t)(packed & 0xFFFFu), hi = (uint16_t)(packed >> 16);
+  if (FMT == BSP_E4M3) {
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"(lo));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"(hi));
+  } else {
+    asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h01) : "h"(lo));
+    asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h23) : "h"(hi));
+  }
+  const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+  const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+  out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+}
+
 __device__ __forceinline__ void diag_flush(bsp_diag_t* diag, const DiagCounters& dc) {
   if (diag == nullptr) return;
   if (dc.sat) atomicAdd(&diag->n_saturated, (unsigned long long)dc.sat);
@@ -243,6 +273,27 @@ __device__ __forceinline__ float4 load4(const void* p, size_t i) {
     const uint2 r = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(p) + i));
     return make_float4(bf16_bits_to_float(r.x & 0xFFFFu), bf16_bits_to_float(r.x >> 16),
                        bf16_bits_to_float(r.y & 0xFFFFu), bf16_bits_to_float(r.y >> 16));
+  }
+}
+
+// Sixteen consecutive elements starting at element index i (i % 16 == 0, pointer 16-byte aligned),
+// with 16-byte loads only: four for FP32, two for bf16.
+template <int DT>
+__device__ __forceinline__ void load16(const void* p, size_t i, float (&v)[16]) {
+  if (DT == BSP_F32) {
+    const float4* q = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + i);
+    const float4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2), d = __ldg(q + 3);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    v[8] = c.x; v[9] = c.y; v[10] = c.z; v[11] = c.w; v[12] = d.x; v[13] = d.y; v[14] = d.z; v[15] = d.w;
+  } else {
+    const uint4* q = reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(p) + i);
+    const uint4 a = __ldg(q), b = __ldg(q + 1);
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      v[2 * j] = bf16_bits_to_float(w[j] & 0xFFFFu);
+      v[2 * j + 1] = bf16_bits_to_float(w[j] >> 16);
+    }
   }
 }
 

@@ -30,29 +30,43 @@ __device__ __forceinline__ double warp_max_d(double v) {
 __global__ void __launch_bounds__(256)
 mc_stats_kernel(const float* __restrict__ g_ref, const float* __restrict__ g, const float* __restrict__ S2,
                 int64_t n, int K, int fresh, double* __restrict__ partials) {
-  double err2 = 0, ref2 = 0, se2s = 0, z2 = 0, zs = 0, zmax = 0, cnt = 0;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    const double r = (double)g_ref[i];
-    ref2 += r * r;
+  // Per-element arithmetic in FP32 (M2 = S2 - S1^2/K as one fused multiply-add), per-thread partial
+  // sums in FP32 over the few hundred elements a thread visits, everything above that in double:
+  // FP64 division and square root per element would make this pass compute-bound.
+  float f_err2 = 0.f, f_ref2 = 0.f, f_se2 = 0.f, f_z2 = 0.f, f_zs = 0.f, f_zmax = 0.f, f_cnt = 0.f;
+  const float invK = 1.0f / (float)K;
+  const float invKK = fresh ? 1.0f / ((float)(K - 1) * (float)K) : 0.f;
+  auto one = [&](float r, float a, float s2) {
+    f_ref2 = fmaf(r, r, f_ref2);
     if (!fresh) {
-      const double e = (double)g[i] - r;
-      err2 += e * e;
+      const float e = a - r;
+      f_err2 = fmaf(e, e, f_err2);
     } else {
-      const double s1 = (double)g[i], s2 = (double)S2[i];
-      const double e = s1 / K;
-      double m2 = s2 - s1 * s1 / K;
-      if (m2 < 0) m2 = 0;
-      const double se2 = m2 / (K - 1) / K;
-      const double se = sqrt(se2);
-      const double z = (e == 0.0 && se == 0.0) ? 0.0 : e / se;
-      err2 += e * e;
-      se2s += se2;
-      z2 += z * z;
-      zs += z;
-      zmax = fmax(zmax, fabs(z));
-      cnt += fabs(z) > 3.0 ? 1.0 : 0.0;
+      const float e = a * invK;
+      const float m2 = fmaxf(fmaf(-a, e, s2), 0.f);
+      const float se2 = m2 * invKK;
+      float z;
+      if (se2 > 0.f) z = e * rsqrtf(se2);
+      else z = e == 0.f ? 0.f : copysignf(INFINITY, e);
+      f_err2 = fmaf(e, e, f_err2);
+      f_se2 += se2;
+      f_z2 = fmaf(z, z, f_z2);
+      f_zs += z;
+      f_zmax = fmaxf(f_zmax, fabsf(z));
+      f_cnt += fabsf(z) > 3.0f ? 1.f : 0.f;
     }
+  };
+  const int64_t n4 = n / 4, stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const float4 r = __ldg(reinterpret_cast<const float4*>(g_ref) + i);
+    const float4 a = __ldg(reinterpret_cast<const float4*>(g) + i);
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (fresh) s = __ldg(reinterpret_cast<const float4*>(S2) + i);
+    one(r.x, a.x, s.x); one(r.y, a.y, s.y); one(r.z, a.z, s.z); one(r.w, a.w, s.w);
   }
+  for (int64_t i = n4 * 4 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    one(g_ref[i], g[i], fresh ? S2[i] : 0.f);
+  double err2 = f_err2, ref2 = f_ref2, se2s = f_se2, z2 = f_z2, zs = f_zs, zmax = f_zmax, cnt = f_cnt;
   __shared__ double sm[8][kStatFields];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   err2 = warp_sum_d(err2); ref2 = warp_sum_d(ref2); se2s = warp_sum_d(se2s); z2 = warp_sum_d(z2);
@@ -164,6 +178,7 @@ size_t bsp_mc_stats_workspace_bytes(int64_t n) {
 int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
                  bsp_use_result_t* result, void* ws, size_t ws_bytes, void* stream) {
   if (!g_ref || !g || !result || n < 0 || (fresh && (!S2 || K < 2))) return BSP_ERR_ARG;
+  if (!aligned16(g_ref) || !aligned16(g) || !aligned16(S2)) return BSP_ERR_ALIGN;
   if (!ws || ws_bytes < bsp_mc_stats_workspace_bytes(n) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return BSP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;

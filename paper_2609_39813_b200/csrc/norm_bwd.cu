@@ -16,14 +16,17 @@ __device__ __forceinline__ float sr_value(float v, uint32_t U) { return f8_sr_va
 
 // ------------------------------------------------------------------------------- norm backward
 
-template <int DT, int DU_DT, int FMT, int JMAX>
-__global__ void __launch_bounds__(256)
+// NT threads cover a row with JMAX groups of four columns each (NT * JMAX * 4 >= C).  Wide rows use
+// wide blocks rather than more columns per thread: the per-thread state (column sums, gains, the
+// current and the prefetched row) stays near 64 registers, which keeps 1024 threads resident.
+template <int DT, int DU_DT, int FMT, int JMAX, int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT)
 norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                 const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                 const void* __restrict__ du, int gain_read, const uint8_t* __restrict__ u_codes, float scale_val,
                 const float* __restrict__ scale_dev, PhiloxKey key, float* __restrict__ part_g,
                 float* __restrict__ part_b, float* __restrict__ dx) {
-  __shared__ float red[2][2][8];
+  __shared__ float red[2][2][NT / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float scale = scale_dev ? __ldg(scale_dev) : scale_val;
   const float inv_scale = __fdiv_rn(1.0f, scale);
@@ -32,7 +35,7 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
   float4 g4[JMAX], b4[JMAX], accg[JMAX], accb[JMAX];
 #pragma unroll
   for (int j = 0; j < JMAX; ++j) {
-    const int64_t c = 4 * ((int64_t)tid + 256 * j);
+    const int64_t c = 4 * ((int64_t)tid + NT * j);
     g4[j] = make_float4(1.f, 1.f, 1.f, 1.f);
     b4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < C) {
@@ -42,21 +45,44 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
     accg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
     accb[j] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  float4 rg4[JMAX];
+#pragma unroll
+  for (int j = 0; j < JMAX; ++j)
+    rg4[j] = make_float4(__fdiv_rn(1.0f, g4[j].x), __fdiv_rn(1.0f, g4[j].y), __fdiv_rn(1.0f, g4[j].z),
+                         __fdiv_rn(1.0f, g4[j].w));
 
+  // The next row's x and du are requested before this row's block-wide reduction, so the loads of
+  // one row overlap the arithmetic and the barrier of the row before.
+  float4 nx[JMAX], nd[JMAX];
+  float nrs = 0.f, nmu = 0.f;
+  auto fetch = [&](int64_t r) {
+    nrs = __ldg(rstd + r);
+    nmu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+#pragma unroll
+    for (int j = 0; j < JMAX; ++j) {
+      const int64_t c = 4 * ((int64_t)tid + NT * j);
+      if (c < C) {
+        nx[j] = load4<DT>(x, (size_t)r * C + c);
+        nd[j] = load4<DU_DT>(du, (size_t)r * C + c);
+      }
+    }
+  };
+  if (blockIdx.x < T) fetch(blockIdx.x);
   int it = 0;
   for (int64_t r = blockIdx.x; r < T; r += gridDim.x, ++it) {
-    const float rs = __ldg(rstd + r);
-    const float mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
-    float4 z[JMAX], dz[JMAX], d4[JMAX];
+    const float rs = nrs, mu = nmu;
+    float4 z[JMAX], dz[JMAX], d4[JMAX], xr[JMAX];
+#pragma unroll
+    for (int j = 0; j < JMAX; ++j) { xr[j] = nx[j]; d4[j] = nd[j]; }
+    if (r + gridDim.x < T) fetch(r + gridDim.x);
     float p1 = 0.f, p2 = 0.f;
 #pragma unroll
     for (int j = 0; j < JMAX; ++j) {
-      const int64_t c = 4 * ((int64_t)tid + 256 * j);
-      z[j] = dz[j] = d4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int64_t c = 4 * ((int64_t)tid + NT * j);
+      z[j] = dz[j] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (c < C) {
         const size_t i0 = (size_t)r * C + c;
-        const float4 xv = load4<DT>(x, i0);
-        d4[j] = load4<DU_DT>(du, i0);
+        const float4 xv = xr[j];
         if (kind == BSP_RMSNORM) {
           z[j] = make_float4(__fmul_rn(xv.x, rs), __fmul_rn(xv.y, rs), __fmul_rn(xv.z, rs), __fmul_rn(xv.w, rs));
         } else {
@@ -64,8 +90,10 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
                              __fmul_rn(__fsub_rn(xv.z, mu), rs), __fmul_rn(__fsub_rn(xv.w, mu), rs));
         }
         dz[j] = make_float4(g4[j].x * d4[j].x, g4[j].y * d4[j].y, g4[j].z * d4[j].z, g4[j].w * d4[j].w);
-        p1 += (dz[j].x * z[j].x + dz[j].y * z[j].y) + (dz[j].z * z[j].z + dz[j].w * z[j].w);
-        p2 += (dz[j].x + dz[j].y) + (dz[j].z + dz[j].w);
+        if (dx) {
+          p1 += (dz[j].x * z[j].x + dz[j].y * z[j].y) + (dz[j].z * z[j].z + dz[j].w * z[j].w);
+          p2 += (dz[j].x + dz[j].y) + (dz[j].z + dz[j].w);
+        }
 
         // ---- gain use: z_g under the policy
         float4 zg = z[j];
@@ -73,8 +101,7 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
           float dec[4];
           if (gain_read == BSP_READ_FORWARD) {
             const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(u_codes + i0));
-#pragma unroll
-            for (int e = 0; e < 4; ++e) dec[e] = f8_decode<FMT>((pk >> (8 * e)) & 0xFFu);
+            f8_decode4<FMT>(pk, dec);
           } else {
             const uint4 w = philox_block(key, (uint64_t)i0 >> 2, key.c2);
             const float u[4] = {z[j].x, z[j].y, z[j].z, z[j].w};
@@ -88,10 +115,13 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
               dec[e] = sr_value<FMT>(__fmul_rn(uu, scale), ww[e]);
             }
           }
-          zg.x = __fdiv_rn(__fsub_rn(__fmul_rn(dec[0], inv_scale), b4[j].x), g4[j].x);
-          zg.y = __fdiv_rn(__fsub_rn(__fmul_rn(dec[1], inv_scale), b4[j].y), g4[j].y);
-          zg.z = __fdiv_rn(__fsub_rn(__fmul_rn(dec[2], inv_scale), b4[j].z), g4[j].z);
-          zg.w = __fdiv_rn(__fsub_rn(__fmul_rn(dec[3], inv_scale), b4[j].w), g4[j].w);
+          // (copy - beta) / gamma as a multiplication by the per-column reciprocal (one rounding
+          // more than a division, far inside the FP32 tolerance; the division would cost ten
+          // instructions per element on a pass that has about that many to spend)
+          zg.x = (dec[0] * inv_scale - b4[j].x) * rg4[j].x;
+          zg.y = (dec[1] * inv_scale - b4[j].y) * rg4[j].y;
+          zg.z = (dec[2] * inv_scale - b4[j].z) * rg4[j].z;
+          zg.w = (dec[3] * inv_scale - b4[j].w) * rg4[j].w;
         }
         accg[j].x = fmaf(zg.x, d4[j].x, accg[j].x); accg[j].y = fmaf(zg.y, d4[j].y, accg[j].y);
         accg[j].z = fmaf(zg.z, d4[j].z, accg[j].z); accg[j].w = fmaf(zg.w, d4[j].w, accg[j].w);
@@ -104,14 +134,16 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
       p2 = warp_sum(p2);
       if (lane == 0) { red[buf][0][warp] = p1; red[buf][1][warp] = p2; }
       __syncthreads();
-      float s1 = 0.f, s2 = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) { s1 += red[buf][0][w]; s2 += red[buf][1][w]; }
+      // every warp re-reduces the per-warp partials: one shared load per lane, then shuffles
+      float s1 = lane < NT / 32 ? red[buf][0][lane] : 0.f;
+      float s2 = lane < NT / 32 ? red[buf][1][lane] : 0.f;
+      s1 = warp_sum(s1);
+      s2 = warp_sum(s2);
       const float m1 = s1 * invC;
       const float m2 = kind == BSP_LAYERNORM ? s2 * invC : 0.f;
 #pragma unroll
       for (int j = 0; j < JMAX; ++j) {
-        const int64_t c = 4 * ((int64_t)tid + 256 * j);
+        const int64_t c = 4 * ((int64_t)tid + NT * j);
         if (c < C) {
           float4 o;
           o.x = rs * ((dz[j].x - m2) - z[j].x * m1);
@@ -125,7 +157,7 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
   }
 #pragma unroll
   for (int j = 0; j < JMAX; ++j) {
-    const int64_t c = 4 * ((int64_t)tid + 256 * j);
+    const int64_t c = 4 * ((int64_t)tid + NT * j);
     if (c < C) {
       *reinterpret_cast<float4*>(part_g + (size_t)blockIdx.x * C + c) = accg[j];
       if (part_b) *reinterpret_cast<float4*>(part_b + (size_t)blockIdx.x * C + c) = accb[j];
@@ -292,16 +324,18 @@ static int launch_norm_bwd(int jmax, int grid, cudaStream_t st, int kind, const 
                            const float* gamma, const float* beta, const float* rstd, const float* mean,
                            const void* du, int gain_read, const uint8_t* u_codes, bsp_quant_t q, PhiloxKey key,
                            float* part_g, float* part_b, float* dx) {
-#define BSP_NB(J)                                                                                           \
-  norm_bwd_kernel<DT, DU_DT, FMT, J><<<grid, 256, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,      \
-                                                            gain_read, u_codes, q.scale, q.scale_dev, key,  \
-                                                            part_g, part_b, dx)
-  switch (jmax) {
-    case 1: BSP_NB(1); break;
-    case 2: BSP_NB(2); break;
-    case 4: BSP_NB(4); break;
-    default: BSP_NB(8); break;
-  }
+  // jmax encodes the launch shape: C/4 column groups over 256, 512 or 1024 threads, two groups per
+  // thread only beyond 4096 columns
+  (void)jmax;
+  const int64_t groups = C / 4;
+#define BSP_NB(J, NT)                                                                                        \
+  norm_bwd_kernel<DT, DU_DT, FMT, J, NT><<<grid, NT, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
+                                                               gain_read, u_codes, q.scale, q.scale_dev, key, \
+                                                               part_g, part_b, dx)
+  if (groups <= 256) BSP_NB(1, 256);
+  else if (groups <= 512) BSP_NB(1, 512);
+  else if (groups <= 1024) BSP_NB(1, 1024);
+  else BSP_NB(2, 1024);
 #undef BSP_NB
   BSP_LAUNCH_CHECK();
   return BSP_OK;

@@ -31,18 +31,37 @@ __global__ void amax_kernel(const void* __restrict__ x, size_t group_size, uint3
   const size_t base = g * group_size;
   float m = 0.f;
   uint32_t nf = 0;
-  const size_t nvec = group_size / 4;
-  const bool vec_ok = ((base & 3) == 0);
+  // 16-byte loads, four of them in flight per thread and iteration
+  constexpr int EPV = DT == BSP_F32 ? 4 : 8;                 // elements per 16-byte vector
+  const size_t nvec = group_size / EPV;
+  const bool vec_ok = ((base % EPV) == 0);
   if (vec_ok) {
-    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += (size_t)gridDim.x * blockDim.x) {
-      const float4 f = load4<DT>(x, base + v * 4);
-      const float a[4] = {fabsf(f.x), fabsf(f.y), fabsf(f.z), fabsf(f.w)};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (a[j] <= 3.4028234663852886e38f) m = fmaxf(m, a[j]); else nf++;
+    const uint4* xv = reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(x) + base * (16 / EPV));
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    auto take = [&](const uint4& r) {
+      float a[8];
+      if (DT == BSP_F32) {
+        a[0] = __uint_as_float(r.x); a[1] = __uint_as_float(r.y); a[2] = __uint_as_float(r.z); a[3] = __uint_as_float(r.w);
+      } else {
+        a[0] = bf16_bits_to_float(r.x & 0xFFFFu); a[1] = bf16_bits_to_float(r.x >> 16);
+        a[2] = bf16_bits_to_float(r.y & 0xFFFFu); a[3] = bf16_bits_to_float(r.y >> 16);
+        a[4] = bf16_bits_to_float(r.z & 0xFFFFu); a[5] = bf16_bits_to_float(r.z >> 16);
+        a[6] = bf16_bits_to_float(r.w & 0xFFFFu); a[7] = bf16_bits_to_float(r.w >> 16);
       }
+#pragma unroll
+      for (int j = 0; j < EPV; ++j) {
+        const float v = fabsf(a[j]);
+        if (v <= 3.4028234663852886e38f) m = fmaxf(m, v); else nf++;
+      }
+    };
+    size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; v + 3 * stride < nvec; v += 4 * stride) {
+      const uint4 r0 = __ldg(xv + v), r1 = __ldg(xv + v + stride), r2 = __ldg(xv + v + 2 * stride),
+                  r3 = __ldg(xv + v + 3 * stride);
+      take(r0); take(r1); take(r2); take(r3);
     }
-    for (size_t i = nvec * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < group_size;
+    for (; v < nvec; v += stride) take(__ldg(xv + v));
+    for (size_t i = nvec * EPV + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < group_size;
          i += (size_t)gridDim.x * blockDim.x) {
       const float a = fabsf(load1<DT>(x, base + i));
       if (a <= 3.4028234663852886e38f) m = fmaxf(m, a); else nf++;
@@ -79,6 +98,20 @@ template <int FMT, int MODE>
 __device__ __forceinline__ uint4 encode16(const float (&v)[16], const PhiloxKey& key, uint32_t draw, uint64_t e0,
                                           DiagCounters& dc) {
   uint32_t packed[4];
+  if (MODE == BSP_ROUND_NEAREST) {
+    // nearest-even: the hardware conversion, unless the chunk holds a value at or above the
+    // format's maximum (saturation, infinity, NaN), which goes through the counting encoder below
+    uint32_t amax_bits = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) amax_bits = max(amax_bits, __float_as_uint(v[j]) & 0x7FFFFFFFu);
+    if (amax_bits < F8<FMT>::FMAX_BITS) {
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        packed[b] = f8_encode_rn_pair_inrange<FMT>(v[4 * b], v[4 * b + 1]) |
+                    (f8_encode_rn_pair_inrange<FMT>(v[4 * b + 2], v[4 * b + 3]) << 16);
+      return make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    }
+  }
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
     uint4 w = make_uint4(0, 0, 0, 0);
@@ -98,19 +131,28 @@ __global__ void __launch_bounds__(256)
 round_vec_kernel(const void* __restrict__ x, size_t n16, size_t group_size, float scale_val,
                  const float* __restrict__ scales, PhiloxKey key, uint64_t elem_offset,
                  uint8_t* __restrict__ codes, bsp_diag_t* diag) {
-  const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // grid-stride over 16-element chunks, two chunks' loads in flight per thread
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
   DiagCounters dc;
-  if (t < n16) {
+  auto finish = [&](size_t t, float (&v)[16]) {
     const size_t i0 = t * 16;
     const float s = scales ? __ldg(scales + (group_size ? i0 / group_size : 0)) : scale_val;
-    float v[16];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float4 f = load4<DT>(x, i0 + 4 * j);
-      v[4 * j + 0] = __fmul_rn(f.x, s); v[4 * j + 1] = __fmul_rn(f.y, s);
-      v[4 * j + 2] = __fmul_rn(f.z, s); v[4 * j + 3] = __fmul_rn(f.w, s);
-    }
+    for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(v[j], s);
     reinterpret_cast<uint4*>(codes)[t] = encode16<FMT, MODE>(v, key, key.c2, elem_offset + i0, dc);
+  };
+  size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; t + stride < n16; t += 2 * stride) {
+    float a[16], b[16];
+    load16<DT>(x, t * 16, a);
+    load16<DT>(x, (t + stride) * 16, b);
+    finish(t, a);
+    finish(t + stride, b);
+  }
+  if (t < n16) {
+    float a[16];
+    load16<DT>(x, t * 16, a);
+    finish(t, a);
   }
   diag_flush_warp(diag, dc);
 }
@@ -182,12 +224,9 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
     prod.row(r);
     const size_t i0 = (size_t)r * cols + c;
     float u[16], v[16];
+    load16<DT>(x, i0, u);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float4 f = load4<DT>(x, i0 + 4 * j);
-      u[4 * j + 0] = prod.value(f.x, c + 4 * j + 0); u[4 * j + 1] = prod.value(f.y, c + 4 * j + 1);
-      u[4 * j + 2] = prod.value(f.z, c + 4 * j + 2); u[4 * j + 3] = prod.value(f.w, c + 4 * j + 3);
-    }
+    for (int j = 0; j < 16; ++j) u[j] = prod.value(u[j], c + j);
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(u[j], s);
     if (u_f32) {
@@ -262,14 +301,9 @@ reround_draws_kernel(NormProducer prod, const void* __restrict__ x, int64_t rows
   for (int j = 0; j < 16; ++j) v[j] = 0.f;
   if (active) {
     prod.row(r);
+    load16<DT>(x, i0, v);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float4 f = load4<DT>(x, i0 + 4 * j);
-      v[4 * j + 0] = __fmul_rn(prod.value(f.x, c + 4 * j + 0), s);
-      v[4 * j + 1] = __fmul_rn(prod.value(f.y, c + 4 * j + 1), s);
-      v[4 * j + 2] = __fmul_rn(prod.value(f.z, c + 4 * j + 2), s);
-      v[4 * j + 3] = __fmul_rn(prod.value(f.w, c + 4 * j + 3), s);
-    }
+    for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(prod.value(v[j], c + j), s);
   }
   const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
   const int64_t cc = c0 + tcol, rr = r0 + trow;
@@ -300,9 +334,12 @@ reround_draws_kernel(NormProducer prod, const void* __restrict__ x, int64_t rows
 
 // One warp per row.  RMS: rstd = 1/sqrt(mean x^2 + eps).  LN: mean, biased variance.
 // Optionally the largest |u| with u from the same FP32 chain the rounding pass uses.
-template <int DT>
+// Kept lean on purpose: at 2 bytes per element the HBM roofline leaves about ten instructions per
+// element, so non-finite inputs are detected once per row (a non-finite sum of squares), not per
+// element, and the norm kind is a template parameter.
+template <int DT, int kind>
 __global__ void __launch_bounds__(256)
-norm_stats_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
+norm_stats_kernel(const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                   const float* __restrict__ beta, float eps, float* __restrict__ rstd, float* __restrict__ mean,
                   uint32_t* __restrict__ amax_bits, bsp_diag_t* diag) {
   const int lane = threadIdx.x & 31;
@@ -312,24 +349,34 @@ norm_stats_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, co
   if (row < T) {
     const size_t base = (size_t)row * C;
     const int64_t nvec = C / 4;
+    // the first pass over the row sets the HBM traffic (later passes hit L1): four 16-byte loads in
+    // flight per lane.  Quads of four elements are visited in the same order by every pass.
+    auto first_pass = [&](auto&& fn) {
+      int64_t v = lane;
+      for (; v + 96 < nvec; v += 128) {
+        const float4 f0 = load4<DT>(x, base + v * 4), f1 = load4<DT>(x, base + (v + 32) * 4),
+                     f2 = load4<DT>(x, base + (v + 64) * 4), f3 = load4<DT>(x, base + (v + 96) * 4);
+        fn(f0); fn(f1); fn(f2); fn(f3);
+      }
+      for (; v < nvec; v += 32) fn(load4<DT>(x, base + v * 4));
+    };
     float mu = 0.f;
     if (kind == BSP_LAYERNORM) {
       float s = 0.f;
-      for (int64_t v = lane; v < nvec; v += 32) {
-        const float4 f = load4<DT>(x, base + v * 4);
-        s += (f.x + f.y) + (f.z + f.w);
-      }
+      first_pass([&](const float4& f) { s += (f.x + f.y) + (f.z + f.w); });
       mu = __fdiv_rn(warp_sum(s), (float)C);
     }
     float ss = 0.f;
-    for (int64_t v = lane; v < nvec; v += 32) {
-      const float4 f = load4<DT>(x, base + v * 4);
-      const float a = f.x - mu, b = f.y - mu, c = f.z - mu, d = f.w - mu;
-      ss += (a * a + b * b) + (c * c + d * d);
-      nf += !(fabsf(f.x) <= 3.4028234663852886e38f) + !(fabsf(f.y) <= 3.4028234663852886e38f) +
-            !(fabsf(f.z) <= 3.4028234663852886e38f) + !(fabsf(f.w) <= 3.4028234663852886e38f);
-    }
+    first_pass([&](const float4& f) {
+      if (kind == BSP_LAYERNORM) {
+        const float a = f.x - mu, b = f.y - mu, c = f.z - mu, d = f.w - mu;
+        ss += (a * a + b * b) + (c * c + d * d);
+      } else {
+        ss += (f.x * f.x + f.y * f.y) + (f.z * f.z + f.w * f.w);
+      }
+    });
     ss = warp_sum(ss);
+    if (lane == 0 && !(ss <= 3.4028234663852886e38f)) nf = 1;     // NaN, infinity or overflow in this row
     const float rs = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(ss, (float)C), eps)));
     if (lane == 0) {
       rstd[row] = rs;
@@ -350,10 +397,8 @@ norm_stats_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, co
           u2 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.z, mu), rs), g.z), b.z);
           u3 = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(f.w, mu), rs), g.w), b.w);
         }
-        const float a[4] = {fabsf(u0), fabsf(u1), fabsf(u2), fabsf(u3)};
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (a[j] <= 3.4028234663852886e38f) amax = fmaxf(amax, a[j]);
+        // fmaxf drops a NaN operand; an infinite |u| makes amax infinite and the scale falls back to 1
+        amax = fmaxf(fmaxf(amax, fabsf(u0)), fmaxf(fabsf(u1), fmaxf(fabsf(u2), fabsf(u3))));
       }
     }
   }
@@ -403,7 +448,9 @@ static int launch_round_flat(const void* x, size_t n, size_t group_size, float s
   const bool vec_ok = (elem_offset % 4 == 0) && (group_size == 0 || group_size % 16 == 0);
   size_t n16 = vec_ok ? n / 16 : 0;
   if (n16) {
-    const unsigned blocks = (unsigned)((n16 + 255) / 256);
+    const size_t want = (n16 + 511) / 512;                      // two chunks per thread
+    const size_t cap = (size_t)kNumSMs * 8;                     // eight 256-thread blocks per SM
+    const unsigned blocks = (unsigned)(want < cap ? want : cap);
     round_vec_kernel<DT, FMT, MODE><<<blocks, 256, 0, st>>>(x, n16, group_size, scale, scales, key, elem_offset,
                                                            codes, diag);
     BSP_LAUNCH_CHECK();
@@ -534,12 +581,11 @@ int bsp_norm_stats(int kind, const void* x, int dt, int64_t T, int64_t C, const 
   cudaStream_t st = (cudaStream_t)stream;
   if (amax) BSP_CHECK_CUDA(cudaMemsetAsync(amax, 0, sizeof(float), st));
   const unsigned blocks = (unsigned)((T + 7) / 8);
-  if (dt == BSP_F32)
-    norm_stats_kernel<BSP_F32><<<blocks, 256, 0, st>>>(kind, x, T, C, gamma, beta, eps, rstd, mean,
-                                                       reinterpret_cast<uint32_t*>(amax), diag);
-  else
-    norm_stats_kernel<BSP_BF16><<<blocks, 256, 0, st>>>(kind, x, T, C, gamma, beta, eps, rstd, mean,
-                                                        reinterpret_cast<uint32_t*>(amax), diag);
+  uint32_t* ab = reinterpret_cast<uint32_t*>(amax);
+#define BSP_NS(DT, KIND) norm_stats_kernel<DT, KIND><<<blocks, 256, 0, st>>>(x, T, C, gamma, beta, eps, rstd, mean, ab, diag)
+  if (dt == BSP_F32) { if (kind == BSP_RMSNORM) BSP_NS(BSP_F32, BSP_RMSNORM); else BSP_NS(BSP_F32, BSP_LAYERNORM); }
+  else { if (kind == BSP_RMSNORM) BSP_NS(BSP_BF16, BSP_RMSNORM); else BSP_NS(BSP_BF16, BSP_LAYERNORM); }
+#undef BSP_NS
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }

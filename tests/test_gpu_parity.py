@@ -325,7 +325,8 @@ def test_mc_statistics_match_oracle(b):
     mean, m2 = mc.shifted_sums_to_moments(S1, S2, K, ref)
     want = mc.statistics(mean, m2, K, ref, True)
     for name in ("rel_l2_mean_err", "R", "Qprime", "mean_z", "rms_z", "max_abs_z", "frac_abs_z_gt3"):
-        assert np.isclose(getattr(r, name), getattr(want, name), rtol=1e-6, atol=1e-9), name
+        # per-element arithmetic is FP32 on the GPU: agreement to 1e-4, far inside the verdict margins
+        assert np.isclose(getattr(r, name), getattr(want, name), rtol=1e-4, atol=1e-9), name
     assert r.verdict == want.verdict == mc.FAILS and r.K == K and r.n_elements == n
     r0 = b.bsp_mc_stats(up(ref), up(ref), None, n, 1, 0, ws)
     assert r0.rel_l2_mean_err == 0.0 and r0.verdict == mc.HOLDS
