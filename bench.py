@@ -218,6 +218,63 @@ def attention_section(b, peaks, steps=3):
                 diag_status=b.read_diag(diag)["status"])
 
 
+def kernel_table(b, peaks):
+    """The streaming kernels one by one at the large-MLP shape (T=16384, C=4096, O=11008, bf16):
+    microseconds per launch and algorithmic GB/s (bytes the method must move / time) against the
+    measured copy bandwidth.  Inputs are drawn on the device."""
+    import torch
+    T, C, O = 16384, 4096, 11008
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    x = torch.randn(T * C, device="cuda", generator=gen).bfloat16()
+    dY = (torch.randn(T * O, device="cuda", generator=gen) * 0.1).bfloat16()
+    du = torch.randn(T * C, device="cuda", generator=gen).bfloat16()
+    gamma = torch.ones(C, device="cuda")
+    rstd, mean = torch.zeros(T, device="cuda"), torch.zeros(T, device="cuda")
+    amax, scale = torch.zeros(1, device="cuda"), torch.ones(1, device="cuda")
+    codes = torch.zeros(T * C, dtype=torch.uint8, device="cuda")
+    codes_t = torch.zeros(C * T, dtype=torch.uint8, device="cuda")
+    dyc = torch.zeros(T * O, dtype=torch.uint8, device="cuda")
+    dyc_t = torch.zeros(O * T, dtype=torch.uint8, device="cuda")
+    dg, db, dx = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda"), torch.zeros(T * C, device="cuda")
+    ws = b.workspace(b.bsp_norm_bwd_workspace_bytes(T, C))
+    ref, S2 = torch.zeros(O * C, device="cuda"), torch.zeros(O * C, device="cuda")
+    wss = b.workspace(b.bsp_mc_stats_workspace_bytes(O * C))
+    stream = torch.cuda.current_stream()
+    q = b.quant(b.E4M3, b.ROUND_STOCHASTIC, 1.0, scale)
+    qrn = b.quant(b.E5M2, b.ROUND_NEAREST, 100.0)
+    k = b.key(1, 1, 0)
+    b.bsp_norm_stats(b.RMSNORM, x, T, C, gamma, None, 1e-6, rstd, mean, amax)
+    b.bsp_scale_from_amax(amax, 1, b.E4M3, scale)
+    rows = []
+
+    def t(name, bound, fn, nbytes, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        gbs = nbytes / us / 1e3
+        rows.append(dict(kernel=name, bound=bound, us=us, algorithmic_mb=nbytes / 1e6, gb_per_s=gbs,
+                         frac_of_hbm=gbs / peaks["hbm_gbs"]))
+
+    t("amax(dY)", "hbm", lambda: b.bsp_amax(dY, 1, T * O, amax), T * O * 2)
+    t("round dY -> E5M2 nearest", "hbm", lambda: b.bsp_round(dY, T * O, qrn, k, 0, dyc), T * O * 3)
+    t("round_2d dY -> E5M2 nearest, both layouts", "hbm", lambda: b.bsp_round_2d(dY, T, O, qrn, k, dyc, dyc_t, T), T * O * 4)
+    t("norm_stats + amax(u)", "hbm", lambda: b.bsp_norm_stats(b.RMSNORM, x, T, C, gamma, None, 1e-6, rstd, mean, amax), T * C * 2)
+    t("norm_fwd store, stochastic, codes", "alu", lambda: b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, None, T), T * C * 3)
+    t("norm_fwd store, stochastic, codes + transposed", "alu", lambda: b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, codes_t, T), T * C * 4)
+    t("norm_bwd read U: dgamma, dbeta, dx", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 0, codes, q, k, dg, db, dx, ws), T * C * 8)
+    t("norm_bwd read R: dgamma", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 1, codes, q, k, dg, None, None, ws), T * C * 5)
+    t("mc_stats (45 M elements, fresh)", "hbm", lambda: b.bsp_mc_stats(ref, ref, S2, O * C, 16, 1, wss), O * C * 12)
+    return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"], kernels=rows)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -236,6 +293,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     b.lib()
 
+    if args.kernel_table:
+        if rank == 0:
+            print(json.dumps(dict(kernel_table=kernel_table(b, read_peaks()))), flush=True)
+        return
     if args.attention_only:
         if rank == 0:
             print(json.dumps(dict(attention=attention_section(b, read_peaks(), steps=args.attention_steps))), flush=True)
@@ -374,6 +435,8 @@ def main():
     ap.add_argument("--no-attention", action="store_true", help="skip the config-3 attention section")
     ap.add_argument("--attention-only", action="store_true", help="run only the config-3 attention section")
     ap.add_argument("--attention-steps", type=int, default=3)
+    ap.add_argument("--kernel-table", action="store_true",
+                    help="time the streaming kernels one by one at the large-MLP shape and print their GB/s")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 100 and args.warmup == 5:

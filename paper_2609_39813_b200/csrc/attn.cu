@@ -33,7 +33,7 @@ constexpr int kAtTile = AT_BLK * AT_D * 2;        // 16 KB: one 128 x 64 bf16 ti
 constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
 constexpr int kAtThreads = 320;
 // shared memory: res0, res1, str[2][2], P, dS, barriers
-constexpr int kAtSmem = 2 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/;
+constexpr int kAtSmem = 4 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AttnParams {
@@ -96,39 +96,50 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
-  const uint32_t res0 = base, res1 = base + kAtTile;
-  const uint32_t str0 = base + 2 * kAtTile;                 // stage s: str0 + s*2*kAtTile (+kAtTile for the 2nd tile)
-  const uint32_t pbuf = base + 6 * kAtTile, dsbuf = pbuf + kAtPBytes;
+  // shared memory: resident tiles [2 buffers][2 tiles], streamed tiles [2 stages][2 tiles], P, dS
+  const uint32_t res_base = base;
+  const uint32_t str0 = base + 4 * kAtTile;                 // stage s: str0 + s*2*kAtTile (+kAtTile for the 2nd tile)
+  const uint32_t pbuf = base + 8 * kAtTile, dsbuf = pbuf + kAtPBytes;
   const uint32_t bars = dsbuf + kAtPBytes;
-  // barriers: res_full, str_full[2], str_empty[2], sdp_full, sdp_free, pds_ready, pds_free, acc_full
-  const uint32_t b_res = bars, b_sfull = bars + 8, b_sempty = bars + 24, b_sdp_full = bars + 40,
-                 b_sdp_free = bars + 48, b_pds_ready = bars + 56, b_pds_free = bars + 64, b_acc = bars + 72;
+  // barriers (8 bytes each): res_full[2], res_empty[2], str_full[2], str_empty[2], sdp_full, sdp_free,
+  // pds_ready, pds_free, acc_full[2], acc_free[2]
+  const uint32_t b_res = bars, b_res_empty = bars + 16, b_sfull = bars + 32, b_sempty = bars + 48,
+                 b_sdp_full = bars + 64, b_sdp_free = bars + 72, b_pds_ready = bars + 80, b_pds_free = bars + 88,
+                 b_acc = bars + 96, b_acc_free = bars + 112;
   uint8_t* gen = smem_raw + (base - raw);
-  uint8_t* bars_gen = gen + 6 * kAtTile + 2 * kAtPBytes;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 80);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 84);
-  float* xchg = reinterpret_cast<float*>(bars_gen + 96);    // FWD: [2][2][...] not used; see below
+  uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 132);
+  float* xchg = reinterpret_cast<float*>(bars_gen + 144);   // FWD: row max / sum exchange between column halves
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // heavy blocks first: block rank 0 is the one with most inner steps
-  const int rank = blockIdx.x / p.BH, bh = blockIdx.x % p.BH;
-  int blk, it_begin, it_end;                                 // inner index range [it_begin, it_end)
-  if (MODE == AT_DKV) {
-    blk = rank;                                              // key block j: steps i = j .. nblk-1 (causal)
-    it_begin = p.causal ? blk : 0; it_end = p.nblk;
-  } else {
-    blk = p.nblk - 1 - rank;                                 // query block i: steps j = 0 .. i (causal)
-    it_begin = 0; it_end = p.causal ? blk + 1 : p.nblk;
-  }
-  const int nsteps = it_end - it_begin;
-  const int npass = MODE == AT_FWD ? 2 : 1;
-  const int total = nsteps * npass;
+  // Persistent CTA: work items w = blockIdx.x, blockIdx.x + gridDim.x, ... of nblk * BH, heavy blocks
+  // first (item rank 0 is the block with most inner steps).  Resident tiles and accumulators are
+  // double-buffered across items, so the next item's loads and first products run under this
+  // item's tail and epilogue; barrier phases simply keep counting across items.
+  const int nitems = p.nblk * p.BH;
+  auto decode_item = [&](int w, int& blk, int& bh, int& it_begin, int& nsteps) {
+    const int rank = w / p.BH;
+    bh = w % p.BH;
+    int it_end;
+    if (MODE == AT_DKV) {
+      blk = rank;                                            // key block j: steps i = j .. nblk-1 (causal)
+      it_begin = p.causal ? blk : 0; it_end = p.nblk;
+    } else {
+      blk = p.nblk - 1 - rank;                               // query block i: steps j = 0 .. i (causal)
+      it_begin = 0; it_end = p.causal ? blk + 1 : p.nblk;
+    }
+    nsteps = it_end - it_begin;
+  };
+  constexpr int npass = MODE == AT_FWD ? 2 : 1;
 
   if (threadIdx.x == 0) {
-    mbar_init(b_res, 1);
-    for (int s = 0; s < 2; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(b_res + 8 * s, 1); mbar_init(b_res_empty + 8 * s, 1);
+      mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1);
+      mbar_init(b_acc + 8 * s, 1); mbar_init(b_acc_free + 8 * s, 8);
+    }
     mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
-    mbar_init(b_acc, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -138,7 +149,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t t_s = tmem, t_dp = tmem + 128, t_acc0 = tmem + 256, t_acc1 = tmem + 320;
+  // TMEM columns: S [0,128), dP [128,256), accumulator buffer ab at 256 + 128*ab (two 64-column halves)
+  const uint32_t t_s = tmem, t_dp = tmem + 128, t_accbase = tmem + 256;
 
   // instruction descriptors (bf16 operands, FP32 accumulation)
   const uint32_t id_sdp = make_idesc(1u, 1u, 128, 128);                                   // A, B K-major
@@ -149,28 +161,38 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
-      // resident tiles
-      mbar_expect_tx(b_res, (MODE == AT_FWD ? 1 : 2) * kAtTile);
-      if (MODE == AT_DKV) {
-        tma_load_3d(res0, &tm_k, b_res, 0, blk * AT_BLK, bh);
-        tma_load_3d(res1, &tm_v, b_res, 0, blk * AT_BLK, bh);
-      } else {
-        tma_load_3d(res0, &tm_q, b_res, 0, blk * AT_BLK, bh);
-        if (MODE == AT_DQ) tma_load_3d(res1, &tm_do, b_res, 0, blk * AT_BLK, bh);
-      }
       bool ok = true;
-      for (int it = 0; it < total && ok; ++it) {
-        const int step = it_begin + (it % nsteps);
-        const uint32_t s = it & 1u, ph = (it >> 1) & 1u;
-        if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-        const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
-        mbar_expect_tx(b_sfull + 8 * s, 2 * kAtTile);
+      uint32_t itg = 0;                                       // step counter across items
+      int item = 0;
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+        int blk, bh, it_begin, nsteps;
+        decode_item(w, blk, bh, it_begin, nsteps);
+        // resident tiles of this item, into the buffer the item before last has released
+        const uint32_t rb = item & 1u, rph = (item >> 1) & 1u;
+        if (!mbar_wait(b_res_empty + 8 * rb, rph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t r0 = res_base + rb * 2 * kAtTile, r1 = r0 + kAtTile;
+        mbar_expect_tx(b_res + 8 * rb, (MODE == AT_FWD ? 1 : 2) * kAtTile);
         if (MODE == AT_DKV) {
-          tma_load_3d(d0, &tm_q, b_sfull + 8 * s, 0, step * AT_BLK, bh);
-          tma_load_3d(d1, &tm_do, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          tma_load_3d(r0, &tm_k, b_res + 8 * rb, 0, blk * AT_BLK, bh);
+          tma_load_3d(r1, &tm_v, b_res + 8 * rb, 0, blk * AT_BLK, bh);
         } else {
-          tma_load_3d(d0, &tm_k, b_sfull + 8 * s, 0, step * AT_BLK, bh);
-          tma_load_3d(d1, &tm_v, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          tma_load_3d(r0, &tm_q, b_res + 8 * rb, 0, blk * AT_BLK, bh);
+          if (MODE == AT_DQ) tma_load_3d(r1, &tm_do, b_res + 8 * rb, 0, blk * AT_BLK, bh);
+        }
+        const int total = nsteps * npass;
+        for (int it = 0; it < total; ++it, ++itg) {
+          const int step = it_begin + (it % nsteps);
+          const uint32_t s = itg & 1u, ph = (itg >> 1) & 1u;
+          if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
+          mbar_expect_tx(b_sfull + 8 * s, 2 * kAtTile);
+          if (MODE == AT_DKV) {
+            tma_load_3d(d0, &tm_q, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+            tma_load_3d(d1, &tm_do, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          } else {
+            tma_load_3d(d0, &tm_k, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+            tma_load_3d(d1, &tm_v, b_sfull + 8 * s, 0, step * AT_BLK, bh);
+          }
         }
       }
       if (!ok) for (int i = 0; i < 200; ++i) __nanosleep(1000);
@@ -178,11 +200,22 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
-      bool ok = mbar_wait(b_res, 0, abort_flag);
-      // S = Q K^T (and dP = dO V^T) of step `jt`: both operands K-major, 64 = 4 x 16 along K.
+      bool ok = true;
+      uint32_t itg = 0;                                       // step counter across items
+      int item = 0;
+      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+      int blk, bh, it_begin, nsteps;
+      decode_item(w, blk, bh, it_begin, nsteps);
+      const int total = nsteps * npass;
+      const uint32_t rb = item & 1u, iph = (item >> 1) & 1u;  // resident / accumulator buffer and its phase
+      const uint32_t res0 = res_base + rb * 2 * kAtTile, res1 = res0 + kAtTile;
+      const uint32_t t_acc0 = t_accbase + rb * 128, t_acc1 = t_acc0 + 64;
+      if (!mbar_wait(b_res + 8 * rb, iph, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(b_acc_free + 8 * rb, iph ^ 1u, abort_flag)) { ok = false; break; }   // epilogue of item-2 done
+      // S = Q K^T (and dP = dO V^T) of global step `jt`: both operands K-major, 64 = 4 x 16 along K.
       // Issued one step ahead: the softmax warps release the S / dP columns as soon as they hold
       // them in registers, so these products overlap the softmax arithmetic of the step before.
-      auto issue_sdp = [&](int jt) -> bool {
+      auto issue_sdp = [&](uint32_t jt) -> bool {
         const uint32_t s = jt & 1u, ph = (jt >> 1) & 1u;
         if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) return false;
         if (!mbar_wait(b_sdp_free, (jt & 1u) ^ 1u, abort_flag)) return false;
@@ -203,12 +236,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_commit(b_sdp_full);
         return true;
       };
-      if (ok && total > 0) ok = issue_sdp(0);
+      if (ok && total > 0) ok = issue_sdp(itg);
       for (int it = 0; it < total && ok; ++it) {
         const bool pass2 = it >= nsteps;                      // FWD only
-        const uint32_t s = it & 1u, ip = it & 1u;
+        const uint32_t jg = itg + (uint32_t)it;
+        const uint32_t s = jg & 1u, ip = jg & 1u;
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
-        if (it + 1 < total && !issue_sdp(it + 1)) { ok = false; break; }
+        if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t first = (MODE == AT_FWD ? it == nsteps : it == 0) ? 0u : 1u;   // overwrite on the first product
@@ -234,13 +268,27 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_commit(b_pds_free);
         tc_commit(b_sempty + 8 * s);
       }
-      if (ok) tc_commit(b_acc);
+      itg += (uint32_t)total;
+      if (ok) {
+        tc_commit(b_acc + 8 * rb);          // this item's accumulators are complete
+        tc_commit(b_res_empty + 8 * rb);    // and its resident tiles are no longer read
+      }
+      }  // items
     }
   } else {
     // ------------------------------------------------ softmax / dS warps, then the epilogue
     const int q4 = warp & 3, h = (warp - 2) >> 2;
     const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    bool ok = true;
+    uint32_t itg = 0;                                         // step counter across items
+    int item = 0;
+    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+    int blk, bh, it_begin, nsteps;
+    decode_item(w, blk, bh, it_begin, nsteps);
+    const int total = nsteps * npass;
+    const uint32_t ab = item & 1u, iph = (item >> 1) & 1u;    // accumulator buffer of this item and its phase
+    const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
     float inv_q = 1.f, inv_k = 1.f, inv_v = 1.f, inv_do = 1.f;
     if (p.fp8) {
       inv_q = __fdiv_rn(1.0f, __ldg(p.sc_q + bh)); inv_k = __fdiv_rn(1.0f, __ldg(p.sc_k + bh));
@@ -248,7 +296,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     const float c2 = p.c * kLog2e * inv_q * inv_k;            // scores arrive as products of decoded codes
     const float dp_mul = inv_do * inv_v;                      // likewise dP
-    bool ok = true;
     float lse2 = 0.f, dq = 0.f;                               // this row's LSE*log2e and D
     int qrow = 0;                                             // global query index of this thread's row
     if (MODE != AT_DKV) {
@@ -262,7 +309,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     for (int it = 0; it < total && ok; ++it) {
       const bool pass2 = it >= nsteps;
       const int step = it_begin + (it % nsteps);
-      const uint32_t ip = it & 1u;
+      const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
       if (MODE == AT_DKV) {
         kblk = blk;
@@ -388,8 +435,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       __syncwarp();
       if (lane == 0) mbar_arrive(b_pds_ready);
     }
+    itg += (uint32_t)total;
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise)
-    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc, 0, abort_flag));
+    if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc + 8 * ab, iph, abort_flag));
     if (ok) {
       tc_fence_after();
       const int grow = blk * AT_BLK + r;
@@ -423,7 +471,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                             __uint_as_float(a[j + 2]) * mul, __uint_as_float(a[j + 3]) * mul);
         }
       }
+      // the accumulator buffer may be overwritten by the item after next
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_acc_free + 8 * ab);
     }
+    }  // items
   }
 
   tc_fence_before();
@@ -527,7 +580,13 @@ static int launch_attn(const void* q, const void* k, const void* v, const void* 
     BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;
   }
-  const unsigned grid = (unsigned)p.nblk * (unsigned)p.BH;
+  // persistent: one CTA per SM walks the (block, head) items, heaviest first
+  int nsm = kNumSMs, dev = 0, sm_count = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sm_count > 0)
+    nsm = sm_count;
+  const int64_t nitems = (int64_t)p.nblk * p.BH;
+  const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
   attn_kernel<MODE><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
