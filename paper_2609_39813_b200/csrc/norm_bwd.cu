@@ -2,12 +2,13 @@
 //
 // norm_bwd_kernel: one row per block iteration; x and du are read once, dx is written once, the
 // column sums for dgamma / dbeta are kept in registers across the block's rows and reduced over
-// blocks by a second, deterministic kernel.  HBM-bound.
+// blocks by a second, deterministic kernel.  HBM-bound.  Shapes made of whole 256-column stages
+// take norm_bwd_stream_kernel (same arithmetic, rows staged through shared memory by bulk copies).
 // gain_mc_kernel: x and du are read once for all K draws; every draw costs one Philox block and
 // four stochastic roundings per four elements, all in registers.  ALU-bound.
 #include <mutex>
 
-#include "common.cuh"
+#include "norm_bwd_stream.cuh"
 
 namespace bsp {
 
@@ -165,15 +166,27 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
   }
 }
 
-// out[c] = sum over nparts of part[p*C + c], in order.  grid: C/32 blocks of 256 = 8 x 32 threads.
+// out[c] = sum over nparts of part[p*C + c], in a fixed order.  grid: (C/32, 1 or 2) blocks of
+// 256 = 8 x 32 threads; blockIdx.y == 1 reduces the second pair (dbeta beside dgamma in one launch).
 __global__ void __launch_bounds__(256)
-column_reduce_kernel(const float* __restrict__ part, int nparts, int64_t C, float* __restrict__ out) {
+column_reduce_kernel(const float* __restrict__ part0, float* __restrict__ out0, const float* __restrict__ part1,
+                     float* __restrict__ out1, int nparts, int64_t C) {
   __shared__ float sm[8][33];
+  const float* __restrict__ part = blockIdx.y ? part1 : part0;
+  float* __restrict__ out = blockIdx.y ? out1 : out0;
   const int cl = threadIdx.x & 31, pl = threadIdx.x >> 5;
   const int64_t c = (int64_t)blockIdx.x * 32 + cl;
   float s = 0.f;
-  if (c < C)
-    for (int p = pl; p < nparts; p += 8) s += part[(size_t)p * C + c];
+  if (c < C) {
+    // four loads in flight per thread; the additions keep the order p = pl, pl + 8, ...
+    int p = pl;
+    for (; p + 24 < nparts; p += 32) {
+      const float a0 = __ldg(part + (size_t)p * C + c), a1 = __ldg(part + (size_t)(p + 8) * C + c);
+      const float a2 = __ldg(part + (size_t)(p + 16) * C + c), a3 = __ldg(part + (size_t)(p + 24) * C + c);
+      s += a0; s += a1; s += a2; s += a3;
+    }
+    for (; p < nparts; p += 8) s += __ldg(part + (size_t)p * C + c);
+  }
   sm[pl][cl] = s;
   __syncthreads();
   if (pl == 0 && c < C) {
@@ -186,7 +199,7 @@ column_reduce_kernel(const float* __restrict__ part, int nparts, int64_t C, floa
 
 // ------------------------------------------------------------------------------- gain-use Monte Carlo
 
-constexpr int kMcRows = 8;              // rows per thread
+constexpr int kMcRows = 8;             // rows per thread
 constexpr int kMcSlab = 8 * kMcRows;    // rows per block (8 warps)
 constexpr int kMcCols = 128;            // columns per block (32 lanes x 4)
 constexpr int kMcChunk = 64;            // draws per launch
@@ -358,7 +371,6 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
                  const float* rstd, const float* mean, const void* du, int du_dt, int gain_read,
                  const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key, float* dgamma, float* dbeta, float* dx,
                  void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream) {
-  (void)diag;
   if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(gain_read, 2) ||
       !valid_enum(q.fmt, 1))
     return BSP_ERR_ARG;
@@ -379,7 +391,9 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
     return BSP_ERR_ALIGN;
   if (!ws || ws_bytes < bsp_norm_bwd_workspace_bytes(T, C) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return BSP_ERR_WORKSPACE;
-  const int grid = bwd_grid(T);
+  // whole stages of 256-column multiples take the streamed kernel, every other shape the plain one
+  const StreamPlan plan = plan_stream(T, C, dt, du_dt, gain_read, x, du, u_codes);
+  const int grid = plan.ok ? plan.grid : bwd_grid(T);
   float* part_g = reinterpret_cast<float*>(ws);
   float* part_b = dbeta ? reinterpret_cast<float*>(reinterpret_cast<char*>(ws) +
                                                    round_up((size_t)grid * C * sizeof(float), 256))
@@ -388,9 +402,11 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
   const int jmax = groups <= 1 ? 1 : groups <= 2 ? 2 : groups <= 4 ? 4 : 8;
   const PhiloxKey pk = make_key(key);
   int rc;
-#define BSP_CALL(DT, DU, FMT)                                                                              \
-  rc = launch_norm_bwd<DT, DU, FMT>(jmax, grid, st, kind, x, T, C, gamma, beta, rstd, mean, du, gain_read, \
-                                    u_codes, q, pk, part_g, part_b, dx)
+#define BSP_CALL(DT, DU, FMT)                                                                                 \
+  rc = plan.ok ? launch_norm_bwd_stream<DT, DU, FMT>(plan, st, kind, x, T, C, gamma, beta, rstd, mean, du,    \
+                                                     gain_read, u_codes, q, pk, part_g, part_b, dx, diag)     \
+               : launch_norm_bwd<DT, DU, FMT>(jmax, grid, st, kind, x, T, C, gamma, beta, rstd, mean, du,     \
+                                              gain_read, u_codes, q, pk, part_g, part_b, dx)
   if (q.fmt == BSP_E4M3) {
     if (dt == BSP_F32 && du_dt == BSP_F32) BSP_CALL(BSP_F32, BSP_F32, BSP_E4M3);
     else if (dt == BSP_F32) BSP_CALL(BSP_F32, BSP_BF16, BSP_E4M3);
@@ -405,12 +421,8 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
 #undef BSP_CALL
   if (rc != BSP_OK) return rc;
   const unsigned rb = (unsigned)((C + 31) / 32);
-  column_reduce_kernel<<<rb, 256, 0, st>>>(part_g, grid, C, dgamma);
+  column_reduce_kernel<<<dim3(rb, dbeta ? 2 : 1), 256, 0, st>>>(part_g, dgamma, part_b, dbeta, grid, C);
   BSP_LAUNCH_CHECK();
-  if (dbeta) {
-    column_reduce_kernel<<<rb, 256, 0, st>>>(part_b, grid, C, dbeta);
-    BSP_LAUNCH_CHECK();
-  }
   return BSP_OK;
 }
 
