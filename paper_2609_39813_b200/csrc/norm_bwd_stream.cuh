@@ -154,7 +154,7 @@ norm_bwd_stream_kernel(const void* __restrict__ x, int64_t T, int64_t C, int64_t
     if (i + 1 < nst) fetch_stats(i + 1);
     const unsigned char* st = smem + (size_t)s * stage_bytes;
     // after a failed wait the stage's contents are arbitrary; the results are discarded below
-    const bool ok = mbar_wait(bar0 + 8 * s, par, abort_flag);
+    const bool ok = mbar_wait_suspend(bar0 + 8 * s, par, abort_flag);
 
     // ---- column sums and the stage's row sums; z and gamma*du stay in registers for dx
     float z[kRS][kNJ][4], dz[kRS][kNJ][4], p[NV];

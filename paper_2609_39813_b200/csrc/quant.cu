@@ -4,6 +4,7 @@
 // All of these are streaming kernels: every element is read once and one byte is written, with
 // 128-bit loads and stores; stochastic rounding costs one Philox4x32-10 block per four elements.
 #include "common.cuh"
+#include "norm_stats_stream.cuh"
 
 namespace bsp {
 
@@ -580,8 +581,24 @@ int bsp_norm_stats(int kind, const void* x, int dt, int64_t T, int64_t C, const 
   if (!aligned16(x) || !aligned16(gamma) || !aligned16(beta)) return BSP_ERR_ALIGN;
   cudaStream_t st = (cudaStream_t)stream;
   if (amax) BSP_CHECK_CUDA(cudaMemsetAsync(amax, 0, sizeof(float), st));
-  const unsigned blocks = (unsigned)((T + 7) / 8);
   uint32_t* ab = reinterpret_cast<uint32_t*>(amax);
+  // whole stages of 256-column multiples take the streamed kernel
+  const StatsPlan sp = plan_stats_stream(T, C, dt, x);
+  if (sp.ok) {
+#define BSP_NSS(DT, KIND)                                                                                    \
+  do {                                                                                                       \
+    auto kfn = norm_stats_stream_kernel<DT, KIND, kStatRS, kStatNJ>;                                                          \
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sp.smem));    \
+    kfn<<<sp.grid, sp.threads, sp.smem, st>>>(x, T, C, sp.rows_per_block, sp.ring, gamma, beta, eps, rstd,   \
+                                               mean, ab, diag);                                              \
+  } while (0)
+    if (dt == BSP_F32) { if (kind == BSP_RMSNORM) BSP_NSS(BSP_F32, BSP_RMSNORM); else BSP_NSS(BSP_F32, BSP_LAYERNORM); }
+    else { if (kind == BSP_RMSNORM) BSP_NSS(BSP_BF16, BSP_RMSNORM); else BSP_NSS(BSP_BF16, BSP_LAYERNORM); }
+#undef BSP_NSS
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  }
+  const unsigned blocks = (unsigned)((T + 7) / 8);
 #define BSP_NS(DT, KIND) norm_stats_kernel<DT, KIND><<<blocks, 256, 0, st>>>(x, T, C, gamma, beta, eps, rstd, mean, ab, diag)
   if (dt == BSP_F32) { if (kind == BSP_RMSNORM) BSP_NS(BSP_F32, BSP_RMSNORM); else BSP_NS(BSP_F32, BSP_LAYERNORM); }
   else { if (kind == BSP_RMSNORM) BSP_NS(BSP_BF16, BSP_RMSNORM); else BSP_NS(BSP_BF16, BSP_LAYERNORM); }

@@ -131,11 +131,12 @@ def test_round_2d_transposed_copy(b, rows, cols):
 
 def _small_cases():
     return [workloads.config1(),
-            workloads.config2(T=200, C=256, O=192, K=8),
+            workloads.config2(T=200, C=512, O=192, K=8),
             workloads.config4(T=150, C=320, O=128, K=8),
-            # whole 256-column stages and an even T: the LayerNorm / FP32 form of the streamed backward
-            # (cfg2_small is its RMSNorm / bf16 form; cfg1 and cfg4_small take the plain kernel)
-            workloads.config4(T=154, C=512, O=128, K=8)]
+            # whole 512-column stages and T a multiple of four: the LayerNorm / FP32 form of the streamed
+            # statistics and backward kernels (cfg2_small is their RMSNorm / bf16 form; cfg1 and
+            # cfg4_small take the plain kernels)
+            workloads.config4(T=156, C=512, O=128, K=8)]
 
 
 @pytest.fixture(scope="module", params=[0, 1, 2, 3], ids=["cfg1", "cfg2_small", "cfg4_small", "cfg4_stream"])
