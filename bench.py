@@ -214,7 +214,11 @@ def attention_section(b, peaks, steps=3):
                               achieved=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
                               frac=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
                               dkv_tflops=tf_dkv, dq_tflops=tf_dq,
-                              note="7 causal products of 2*S*S*d/2 flop per head; exp on the SFU co-bounds it"),
+                              # a backward needs 5 of those products; the two kernels form S and dP once each
+                              algorithmic_tflops=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12,
+                              algorithmic_frac=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
+                              note="achieved counts the 7 causal products of 2*S*S*d/2 flop per head that the two "
+                                   "kernels compute, algorithmic_* the 5 a backward needs; exp on the SFU co-bounds it"),
                 diag_status=b.read_diag(diag)["status"])
 
 
@@ -389,8 +393,14 @@ def run_ours(args):
     flops = 2.0 * T * O * C * K               # one launch contracts all K draws
     achieved = flops / (gemm_ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16_tflops"]        # FP8 dense = 2 x the measured BF16 burst figure
+    # DRAM bytes of one launch of this kernel at this shape, from one ncu capture of this command
+    # (dram__bytes_read.sum 604.6 MB + dram__bytes_write.sum 23.6 MB; profiles/gemm_mc_kernel_cfg2.md).
+    # The launch's operands are K x T x C = 268 MB of fresh codes, read once per column of output
+    # tiles that does not find them in L2, plus 16.8 MB of dY codes and 3 x 16.8 MB of sums.
+    traffic = 628.2e6 if (T, C, O, K) == (4096, 1024, 4096, 64) else None
     roofline = dict(bound="tensor", kernel="gemm_mc_kernel (FP8 weight gradient over K draws, TMEM-resident sums)",
-                    achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                    achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=traffic,
+                    traffic_unit="bytes per launch (ncu dram read + write, one capture)",
                     us_per_launch=gemm_ms * 1e3, draws_per_launch=K,
                     peak_source="2 x bf16_tflops (%s)" % peaks["source"])
     dstat = b.read_diag(diag)
