@@ -21,6 +21,7 @@
 // Head dimension 64, bf16 inputs, FP32 outputs.  Every wait is bounded.
 #include <string.h>
 
+
 #include "common.cuh"
 #include "tc.cuh"
 
@@ -96,21 +97,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
-  // shared memory: resident tiles [2 buffers][2 tiles], streamed tiles [2 stages][2 tiles], P, dS
+  // shared memory: resident tiles [2 buffers][2 tiles]; then FWD: streamed tiles [2 stages][2 tiles]
+  // and the P buffer; DKV / DQ: streamed tiles [4 stages][2 tiles] over the same 128 KB
   const uint32_t res_base = base;
   const uint32_t str0 = base + 4 * kAtTile;                 // stage s: str0 + s*2*kAtTile (+kAtTile for the 2nd tile)
   const uint32_t pbuf = base + 8 * kAtTile, dsbuf = pbuf + kAtPBytes;
   const uint32_t bars = dsbuf + kAtPBytes;
   // barriers (8 bytes each): res_full[2], res_empty[2], str_full[2], str_empty[2], sdp_full, sdp_free,
   // pds_ready, pds_free, acc_full[2], acc_free[2]
-  const uint32_t b_res = bars, b_res_empty = bars + 16, b_sfull = bars + 32, b_sempty = bars + 48,
-                 b_sdp_full = bars + 64, b_sdp_free = bars + 72, b_pds_ready = bars + 80, b_pds_free = bars + 88,
-                 b_acc = bars + 96, b_acc_free = bars + 112;
+  const uint32_t b_res = bars, b_res_empty = bars + 16, b_sfull = bars + 32, b_sempty = bars + 64,
+                 b_sdp_full = bars + 96, b_sdp_free = bars + 104, b_pds_ready = bars + 112, b_pds_free = bars + 120,
+                 b_acc = bars + 128, b_acc_free = bars + 144;
+  // streamed-tile ring: the backward modes have no P / dS buffers in shared memory (those operands
+  // live in tensor memory), so their ring takes that space too: four stages instead of two
+  constexpr uint32_t kStg = MODE == AT_FWD ? 2u : 4u;
   uint8_t* gen = smem_raw + (base - raw);
   uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 132);
-  float* xchg = reinterpret_cast<float*>(bars_gen + 144);   // FWD: row max / sum exchange between column halves
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 160);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
+  float* xchg = reinterpret_cast<float*>(bars_gen + 176);   // FWD: row max / sum exchange between column halves
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Persistent CTA: work items w = blockIdx.x, blockIdx.x + gridDim.x, ... of nblk * BH, heavy blocks
@@ -136,9 +141,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(b_res + 8 * s, 1); mbar_init(b_res_empty + 8 * s, 1);
-      mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1);
       mbar_init(b_acc + 8 * s, 1); mbar_init(b_acc_free + 8 * s, 8);
     }
+    for (uint32_t s = 0; s < kStg; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
     mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -149,12 +154,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  // TMEM columns: S [0,128), dP [128,256), accumulator buffer ab at 256 + 128*ab (two 64-column halves)
-  const uint32_t t_s = tmem, t_dp = tmem + 128, t_accbase = tmem + 256;
+  // TMEM columns: S [0,128), dP [128,256).  FWD: accumulator buffer ab at 256 + 128*ab.  DKV / DQ: the
+  // bf16 operands P and dS as the softmax warps write them back (64 columns each: two elements per
+  // column) at [256,320) and [320,384), and one accumulator buffer of two 64-column halves at 384.
+  const uint32_t t_s = tmem, t_dp = tmem + 128, t_p = tmem + 256, t_ds = tmem + 320;
+  const uint32_t t_accbase = MODE == AT_FWD ? tmem + 256 : tmem + 384;
+  constexpr bool kAccDouble = MODE == AT_FWD;   // accumulators double-buffered across items
 
   // instruction descriptors (bf16 operands, FP32 accumulation)
   const uint32_t id_sdp = make_idesc(1u, 1u, 128, 128);                                   // A, B K-major
-  const uint32_t id_mn = make_idesc(1u, 1u, 128, 64) | (1u << 15) | (1u << 16);           // A, B MN-major
   const uint32_t id_kmn = make_idesc(1u, 1u, 128, 64) | (1u << 16);                       // A K-major, B MN-major
 
   if (warp == 0) {
@@ -182,7 +190,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const int total = nsteps * npass;
         for (int it = 0; it < total; ++it, ++itg) {
           const int step = it_begin + (it % nsteps);
-          const uint32_t s = itg & 1u, ph = (itg >> 1) & 1u;
+          const uint32_t s = itg % kStg, ph = (itg / kStg) & 1u;
           if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
           mbar_expect_tx(b_sfull + 8 * s, 2 * kAtTile);
@@ -207,29 +215,36 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       int blk, bh, it_begin, nsteps;
       decode_item(w, blk, bh, it_begin, nsteps);
       const int total = nsteps * npass;
-      const uint32_t rb = item & 1u, iph = (item >> 1) & 1u;  // resident / accumulator buffer and its phase
+      const uint32_t rb = item & 1u, iph = (item >> 1) & 1u;  // resident buffer and its phase
+      // accumulator buffer and its phase: alternating with the items (FWD), else the one buffer
+      const uint32_t ab = kAccDouble ? rb : 0u, aph = kAccDouble ? iph : ((uint32_t)item & 1u);
       const uint32_t res0 = res_base + rb * 2 * kAtTile, res1 = res0 + kAtTile;
-      const uint32_t t_acc0 = t_accbase + rb * 128, t_acc1 = t_acc0 + 64;
+      const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
       if (!mbar_wait(b_res + 8 * rb, iph, abort_flag)) { ok = false; break; }
-      if (!mbar_wait(b_acc_free + 8 * rb, iph ^ 1u, abort_flag)) { ok = false; break; }   // epilogue of item-2 done
+      // the accumulators are free once the epilogue that last used them is done: with two buffers
+      // that is checked here, with one just before the item's first accumulating product, so the
+      // first S and dP of this item already run under the epilogue of the item before
+      if (kAccDouble && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
       // S = Q K^T (and dP = dO V^T) of global step `jt`: both operands K-major, 64 = 4 x 16 along K.
       // Issued one step ahead: the softmax warps release the S / dP columns as soon as they hold
       // them in registers, so these products overlap the softmax arithmetic of the step before.
       auto issue_sdp = [&](uint32_t jt) -> bool {
-        const uint32_t s = jt & 1u, ph = (jt >> 1) & 1u;
+        const uint32_t s = jt % kStg, ph = (jt / kStg) & 1u;
         if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) return false;
         if (!mbar_wait(b_sdp_free, (jt & 1u) ^ 1u, abort_flag)) return false;
         tc_fence_after();
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
         const uint32_t q_t = MODE == AT_DKV ? st0 : res0, k_t = MODE == AT_DKV ? res0 : st0;
         const uint32_t do_t = MODE == AT_DKV ? st1 : res1, v_t = MODE == AT_DKV ? res1 : st1;
+        // DKV forms the transposes, S^T = K Q^T and dP^T = V dO^T (rows = keys), so that P^T and dS^T
+        // come out of the softmax warps as the row-per-lane A operands of dV = P^T dO, dK = dS^T Q
         {
-          const uint64_t a = make_smem_desc(q_t), b = make_smem_desc(k_t);
+          const uint64_t a = make_smem_desc(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc(MODE == AT_DKV ? q_t : k_t);
 #pragma unroll
           for (int k = 0; k < 4; ++k) tc_mma<false>(t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
         }
         if (MODE != AT_FWD) {
-          const uint64_t a = make_smem_desc(do_t), b = make_smem_desc(v_t);
+          const uint64_t a = make_smem_desc(MODE == AT_DKV ? v_t : do_t), b = make_smem_desc(MODE == AT_DKV ? do_t : v_t);
 #pragma unroll
           for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
         }
@@ -240,28 +255,32 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int it = 0; it < total && ok; ++it) {
         const bool pass2 = it >= nsteps;                      // FWD only
         const uint32_t jg = itg + (uint32_t)it;
-        const uint32_t s = jg & 1u, ip = jg & 1u;
+        const uint32_t s = jg % kStg, ip = jg & 1u;
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
         if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t first = (MODE == AT_FWD ? it == nsteps : it == 0) ? 0u : 1u;   // overwrite on the first product
+        if (!kAccDouble && it == 0 && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
         if (MODE == AT_DKV) {
-          // dV += P^T dO, dK += dS^T Q : A MN-major from the P / dS buffers (two 64-key atoms, 16 KB
-          // apart), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
-          const uint64_t ap = make_smem_desc_mn(pbuf, 16384u), ads = make_smem_desc_mn(dsbuf, 16384u);
+          // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
+          // queries), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
           const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma<false>(t_acc0, ap + 128u * k, bdo + 128u * k, id_mn, first | (k != 0));
+          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma<false>(t_acc1, ads + 128u * k, bq + 128u * k, id_mn, first | (k != 0));
-        } else if (MODE == AT_DQ || pass2) {
-          // dQ += dS K  (O += P V): A K-major from the dS (P) buffer, B MN-major = streamed K (V)
-          const uint32_t abuf = MODE == AT_DQ ? dsbuf : pbuf;
-          const uint64_t bk = make_smem_desc_mn(MODE == AT_DQ ? st0 : st1, 16384u);
+          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
+        } else if (MODE == AT_DQ) {
+          // dQ += dS K : A from tensor memory (row = query, eight columns per 16 keys), B MN-major = streamed K
+          const uint64_t bk = make_smem_desc_mn(st0, 16384u);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_ds + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
+        } else if (pass2) {
+          // O += P V : A K-major from the P buffer in shared memory, B MN-major = streamed V
+          const uint64_t bk = make_smem_desc_mn(st1, 16384u);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const uint64_t a = make_smem_desc(abuf + (k >> 2) * 16384u + (k & 3) * 32u);
+            const uint64_t a = make_smem_desc(pbuf + (k >> 2) * 16384u + (k & 3) * 32u);
             tc_mma<false>(t_acc0, a, bk + 128u * k, id_kmn, first | (k != 0));
           }
         }
@@ -270,7 +289,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       itg += (uint32_t)total;
       if (ok) {
-        tc_commit(b_acc + 8 * rb);          // this item's accumulators are complete
+        tc_commit(b_acc + 8 * ab);          // this item's accumulators are complete
         tc_commit(b_res_empty + 8 * rb);    // and its resident tiles are no longer read
       }
       }  // items
@@ -287,8 +306,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     int blk, bh, it_begin, nsteps;
     decode_item(w, blk, bh, it_begin, nsteps);
     const int total = nsteps * npass;
-    const uint32_t ab = item & 1u, iph = (item >> 1) & 1u;    // accumulator buffer of this item and its phase
+    // accumulator buffer of this item and its phase (see the MMA issuer)
+    const uint32_t ab = kAccDouble ? (item & 1u) : 0u;
+    const uint32_t iph = kAccDouble ? ((item >> 1) & 1u) : ((uint32_t)item & 1u);
     const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
+    // DKV: a thread's row is a key and its 64 columns are queries, so the per-query LSE * log2(e) and
+    // D sit in shared memory, one 128 + 128 float vector per step, double-buffered: softmax thread ts
+    // fetches one value of the next step while this step computes.
+    const int ts = (int)threadIdx.x - 64;
+    float* colv = xchg;                                       // [2][256]
+    // the raw value only: nothing may depend on the load before the step's arithmetic is done, or
+    // the in-order warp would sit out the load's latency at the top of every step
+    const float* col_src = ts < 128 ? p.lse : p.dterm;
+    const float col_mul = ts < 128 ? kLog2e : 1.0f;
+    auto col_fetch = [&](int step) -> float {
+      const int q = step * AT_BLK + (ts & 127);
+      return __ldg(col_src + (size_t)bh * p.S + (q < p.S ? q : 0));
+    };
+    auto col_value = [&](int step, float raw) -> float {
+      return step * AT_BLK + (ts & 127) < p.S ? raw * col_mul : 0.f;
+    };
+    if (MODE == AT_DKV && total > 0) {
+      colv[ts] = col_value(it_begin, col_fetch(it_begin));
+      named_bar_sync(1, 256);
+    }
     float inv_q = 1.f, inv_k = 1.f, inv_v = 1.f, inv_do = 1.f;
     if (p.fp8) {
       inv_q = __fdiv_rn(1.0f, __ldg(p.sc_q + bh)); inv_k = __fdiv_rn(1.0f, __ldg(p.sc_k + bh));
@@ -311,17 +352,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
+      float col_next = 0.f;                                   // DKV: this thread's share of the next step's vector
       if (MODE == AT_DKV) {
         kblk = blk;
-        qrow = step * AT_BLK + r;
-        lse2 = 0.f; dq = 0.f;
-        if (qrow < p.S) {
-          lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
-          dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
-        }
       } else {
         kblk = step;
       }
+      const int qb0 = (MODE == AT_DKV ? step : blk) * AT_BLK;  // first query of this step's score tile
       if (MODE == AT_FWD && it == nsteps) {
         // between the passes: combine the two column halves of every row into the row's LSE
         float* xm = xchg;                                     // [2][128] max, then [2][128] sum
@@ -353,11 +390,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(b_sdp_free);
+      if (MODE == AT_DKV && it + 1 < total) col_next = col_fetch(step + 1);   // lands under this step's arithmetic
 
       const int key0 = kblk * AT_BLK + h * 64;
       // masking is needed only on the diagonal block and where the sequence ends inside the block
-      const bool edge = (p.causal && kblk * AT_BLK + AT_BLK - 1 > (qrow - r)) || (kblk + 1) * AT_BLK > p.S ||
-                        (qrow - r) + AT_BLK > p.S;
+      const bool edge = (p.causal && kblk * AT_BLK + AT_BLK - 1 > qb0) || (kblk + 1) * AT_BLK > p.S ||
+                        qb0 + AT_BLK > p.S;
       if (MODE == AT_FWD && !pass2) {
         // running max / sum of exp2(c2 * s) over the valid keys of this half
         float mloc = run_m;
@@ -383,11 +421,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
         // first rounds P onto the E4M3 grid at p_scale and dS onto the E5M2 grid at ds_scale (the
         // grid values are exact in bf16; the scales come back in the epilogue).
-        auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, uint32_t& po, uint32_t& dso) {
+        auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, float d0, float d1, uint32_t& po,
+                             uint32_t& dso) {
           float s0 = 0.f, s1 = 0.f;
           if (MODE != AT_FWD) {
-            s0 = p0 * (__uint_as_float(dp0) * dp_mul - dq);
-            s1 = p1 * (__uint_as_float(dp1) * dp_mul - dq);
+            s0 = p0 * (__uint_as_float(dp0) * dp_mul - d0);
+            s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
           }
           if (p.fp8 && MODE != AT_FWD) {                    // the forward keeps P unrounded
             p0 = f8_rn_value<BSP_E4M3>(p0 * p.p_scale); p1 = f8_rn_value<BSP_E4M3>(p1 * p.p_scale);
@@ -396,44 +435,68 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           po = pack_bf16x2(p0, p1);
           if (MODE != AT_FWD) dso = pack_bf16x2(s0, s1);
         };
+        // column j of this thread's row: a query (DKV, the row is a key) or a key (the row is a query)
+        const int col0 = (MODE == AT_DKV ? qb0 : kblk * AT_BLK) + h * 64;
+        const int myrow = MODE == AT_DKV ? blk * AT_BLK + r : qrow;
+        auto valid_at = [&](int j) {
+          const int cj = col0 + j;
+          const int key = MODE == AT_DKV ? myrow : cj, qy = MODE == AT_DKV ? cj : myrow;
+          return key < p.S && qy < p.S && (!p.causal || key <= qy);
+        };
+        const float* cv = colv + (it & 1) * 256 + h * 64;     // DKV: LSE * log2(e) of these 64 queries, D at +128
+        // Two columns per iteration on purpose: wider bodies made the compiler's schedule of the
+        // exponentials twice as slow.  `masked` adds the validity test that only the diagonal block
+        // and the blocks at the end of the sequence need.
+        auto pair_at = [&](int j, bool masked) {
+          float l0 = lse2, l1 = lse2, d0 = dq, d1 = dq;
+          if (MODE == AT_DKV) {
+            const float2 a = *reinterpret_cast<const float2*>(cv + j), b = *reinterpret_cast<const float2*>(cv + 128 + j);
+            l0 = a.x; l1 = a.y; d0 = b.x; d1 = b.y;
+          }
+          float a0 = fmaf(__uint_as_float(sv[j]), c2, -l0), a1 = fmaf(__uint_as_float(sv[j + 1]), c2, -l1);
+          if (masked) {
+            if (!valid_at(j)) a0 = -INFINITY;
+            if (!valid_at(j + 1)) a1 = -INFINITY;
+          }
+          pack_pair(ex2_approx(a0), ex2_approx(a1), dv[j], dv[j + 1], d0, d1, pk[j >> 1], dk[j >> 1]);
+        };
         if (!edge) {
 #pragma unroll
-          for (int j = 0; j < 64; j += 2) {
-            const float p0 = ex2_approx(fmaf(__uint_as_float(sv[j]), c2, -lse2));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(sv[j + 1]), c2, -lse2));
-            pack_pair(p0, p1, dv[j], dv[j + 1], pk[j >> 1], dk[j >> 1]);
-          }
+          for (int j = 0; j < 64; j += 2) pair_at(j, false);
         } else {
 #pragma unroll
-          for (int j = 0; j < 64; j += 2) {
-            float pv[2];
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int key = key0 + j + e;
-              const bool valid = key < p.S && qrow < p.S && (!p.causal || key <= qrow);
-              pv[e] = ex2_approx(valid ? fmaf(__uint_as_float(sv[j + e]), c2, -lse2) : -INFINITY);
-            }
-            pack_pair(pv[0], pv[1], dv[j], dv[j + 1], pk[j >> 1], dk[j >> 1]);
-          }
+          for (int j = 0; j < 64; j += 2) pair_at(j, true);
         }
-        // the P / dS buffers are free once the products of the previous step have read them
+        // the P / dS operands are free once the products of the previous step have read them
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
         if (!ok) break;
-        // 64 keys = 8 chunks of 16 bytes in row r of half h: chunk index t ^ (r & 7)
+        if (MODE == AT_FWD) {
+          // 64 keys = 8 chunks of 16 bytes in row r of half h of the shared P buffer: chunk index t ^ (r & 7)
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
-          if (MODE != AT_DQ)
+          for (int t = 0; t < 8; ++t) {
+            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
                          "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
-          if (MODE != AT_FWD)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dsbuf + off), "r"(dk[4 * t]), "r"(dk[4 * t + 1]),
-                         "r"(dk[4 * t + 2]), "r"(dk[4 * t + 3]) : "memory");
+          }
+        } else {
+          // back into tensor memory as the A operand of the next products: this row's 64 columns are
+          // 32 packed pairs, at columns h*32 .. h*32+31 of the operand
+          if (MODE == AT_DKV) tmem_st32(t_p + lane_off + h * 32, pk);
+          tmem_st32(t_ds + lane_off + h * 32, dk);
+          tmem_wait_st();
+          tc_fence_before();
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (MODE == AT_FWD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(b_pds_ready);
+      if (MODE == AT_DKV) {
+        // publish the next step's per-query vector; everyone is past this step's reads of the other one
+        // (the empty asm pins the first use of the fetched value here, after the step's arithmetic)
+        asm volatile("" : "+f"(col_next));
+        colv[((it + 1) & 1) * 256 + ts] = col_value(step + 1, col_next);
+        named_bar_sync(1, 256);
+      }
     }
     itg += (uint32_t)total;
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise)
