@@ -93,7 +93,8 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 template <int MODE>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, AttnParams p) {
+            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+            const __grid_constant__ CUtensorMap tm_o0, const __grid_constant__ CUtensorMap tm_o1, AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -109,8 +110,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                  b_sdp_full = bars + 96, b_sdp_free = bars + 104, b_pds_ready = bars + 112, b_pds_free = bars + 120,
                  b_acc = bars + 128, b_acc_free = bars + 144;
   // streamed-tile ring: the backward modes have no P / dS buffers in shared memory (those operands
-  // live in tensor memory), so their ring takes that space too: four stages instead of two
-  constexpr uint32_t kStg = MODE == AT_FWD ? 2u : 4u;
+  // live in tensor memory), so their ring takes a third stage there, and the last 32 KB of that
+  // space stage the second output of the dK/dV epilogue
+  constexpr uint32_t kStg = MODE == AT_FWD ? 2u : 3u;
+  const uint32_t stage2 = str0 + 3u * 2u * kAtTile;
   uint8_t* gen = smem_raw + (base - raw);
   uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 160);
@@ -118,11 +121,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   float* xchg = reinterpret_cast<float*>(bars_gen + 176);   // FWD: row max / sum exchange between column halves
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Persistent CTA: work items w = blockIdx.x, blockIdx.x + gridDim.x, ... of nblk * BH, heavy blocks
-  // first (item rank 0 is the block with most inner steps).  Resident tiles and accumulators are
+  // Persistent CTA: work items w = item_at(0), item_at(1), ... of nblk * BH, heavy blocks first
+  // (item rank 0 is the block with most inner steps).  Resident tiles and accumulators are
   // double-buffered across items, so the next item's loads and first products run under this
   // item's tail and epilogue; barrier phases simply keep counting across items.
   const int nitems = p.nblk * p.BH;
+  // the CTA's n-th item: rounds of gridDim.x items, walked forwards and backwards in turn, so the CTA
+  // that got the heaviest item of one round gets the lightest of the next
+  auto item_at = [&](int n) -> int {
+    const int b = (int)blockIdx.x, G = (int)gridDim.x;
+    return n * G + ((n & 1) ? G - 1 - b : b);
+  };
   auto decode_item = [&](int w, int& blk, int& bh, int& it_begin, int& nsteps) {
     const int rank = w / p.BH;
     bh = w % p.BH;
@@ -172,7 +181,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       bool ok = true;
       uint32_t itg = 0;                                       // step counter across items
       int item = 0;
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+      for (int w = item_at(0); w < nitems && ok; w = item_at(++item)) {
         int blk, bh, it_begin, nsteps;
         decode_item(w, blk, bh, it_begin, nsteps);
         // resident tiles of this item, into the buffer the item before last has released
@@ -211,7 +220,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       bool ok = true;
       uint32_t itg = 0;                                       // step counter across items
       int item = 0;
-      for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+      for (int w = item_at(0); w < nitems && ok; w = item_at(++item)) {
       int blk, bh, it_begin, nsteps;
       decode_item(w, blk, bh, it_begin, nsteps);
       const int total = nsteps * npass;
@@ -289,8 +298,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       itg += (uint32_t)total;
       if (ok) {
-        tc_commit(b_acc + 8 * ab);          // this item's accumulators are complete
-        tc_commit(b_res_empty + 8 * rb);    // and its resident tiles are no longer read
+        // this item's accumulators are complete (and its resident tiles no longer read: the epilogue
+        // stages the output through their buffer and releases it)
+        tc_commit(b_acc + 8 * ab);
       }
       }  // items
     }
@@ -300,9 +310,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     bool ok = true;
+    bool store_pending = false;                               // warp 2, lane 0: an epilogue's bulk stores are in flight
     uint32_t itg = 0;                                         // step counter across items
     int item = 0;
-    for (int w = blockIdx.x; w < nitems && ok; w += gridDim.x, ++item) {
+    for (int w = item_at(0); w < nitems && ok; w = item_at(++item)) {
     int blk, bh, it_begin, nsteps;
     decode_item(w, blk, bh, it_begin, nsteps);
     const int total = nsteps * npass;
@@ -490,6 +501,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (MODE == AT_FWD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(b_pds_ready);
+      if (it == 0 && warp == 2 && lane == 0 && store_pending) {
+        // the previous item's output has left its staging buffer by now: hand the resident-tile
+        // buffer it used back to the TMA producer
+        tma_store_wait_read();
+        mbar_arrive(b_res_empty + 8 * (((uint32_t)item & 1u) ^ 1u));
+        store_pending = false;
+      }
       if (MODE == AT_DKV) {
         // publish the next step's per-query vector; everyone is past this step's reads of the other one
         // (the empty asm pins the first use of the fetched value here, after the step's arithmetic)
@@ -499,47 +517,62 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
     }
     itg += (uint32_t)total;
-    // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise)
+    // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise), 32 KB at a
+    // time through the item's resident-tile buffer (no product reads it any more): every thread puts
+    // its row's 32 FP32 values of column half h into the 128-byte-swizzle box that a tiled bulk store
+    // then writes (whole 128-byte lines; rows beyond the sequence are clipped by the store).
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc + 8 * ab, iph, abort_flag));
     if (ok) {
       tc_fence_after();
-      const int grow = blk * AT_BLK + r;
-      if (MODE == AT_DKV) {
-        // h = 0 warps write dV (acc0), h = 1 warps write dK (acc1, times the softmax scale)
-        float* dst = (h == 0 ? p.out0 : p.out1) + ((size_t)bh * p.S + grow) * AT_D;
-        const float mul = h == 0 ? (p.fp8 ? inv_do / p.p_scale : 1.f) : p.c * (p.fp8 ? inv_q / p.ds_scale : 1.f);
+      const uint32_t rbi = (uint32_t)item & 1u;
+      constexpr int nout = MODE == AT_DKV ? 2 : 1;            // DKV: dV (acc0) and dK (acc1)
+      // the stores of the item before have long read their staging buffers; make that certain
+      if (warp == 2 && lane == 0 && store_pending) {
+        tma_store_wait_read();
+        mbar_arrive(b_res_empty + 8 * (rbi ^ 1u));
+        store_pending = false;
+      }
+      if (MODE == AT_DKV) named_bar_sync(3, 256);             // ... before anyone writes the second staging buffer again
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t a[32];
-          tmem_ld32((h == 0 ? t_acc0 : t_acc1) + lane_off + ch * 32, a);
-          if (grow < p.S) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(dst + ch * 32 + j) =
-                  make_float4(__uint_as_float(a[j]) * mul, __uint_as_float(a[j + 1]) * mul,
-                              __uint_as_float(a[j + 2]) * mul, __uint_as_float(a[j + 3]) * mul);
-          }
-        }
-      } else {
-        // each column half writes 32 of the 64 output columns
-        float* dst = p.out0 + ((size_t)bh * p.S + grow) * AT_D + h * 32;
-        const float mul = MODE == AT_DQ ? p.c * (p.fp8 ? inv_k / p.ds_scale : 1.f) : inv_v;
+      for (int o = 0; o < nout; ++o) {
+        const uint32_t stg = o == 0 ? res_base + rbi * 2 * kAtTile : stage2;
+        float mul;
+        if (MODE == AT_DKV) mul = o == 0 ? (p.fp8 ? inv_do / p.p_scale : 1.f) : p.c * (p.fp8 ? inv_q / p.ds_scale : 1.f);
+        else if (MODE == AT_DQ) mul = p.c * (p.fp8 ? inv_k / p.ds_scale : 1.f);
+        else mul = inv_v;
         uint32_t a[32];
-        tmem_ld32(t_acc0 + lane_off + h * 32, a);
-        if (grow < p.S) {
+        tmem_ld32((o == 0 ? t_acc0 : t_acc1) + lane_off + h * 32, a);
+        if (o == nout - 1) {
+          // the accumulators may be overwritten by the next item (FWD: the item after next)
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(b_acc_free + 8 * ab);
+        }
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *reinterpret_cast<float4*>(dst + j) =
-                make_float4(__uint_as_float(a[j]) * mul, __uint_as_float(a[j + 1]) * mul,
-                            __uint_as_float(a[j + 2]) * mul, __uint_as_float(a[j + 3]) * mul);
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(__uint_as_float(a[4 * t]) * mul),
+                       "f"(__uint_as_float(a[4 * t + 1]) * mul), "f"(__uint_as_float(a[4 * t + 2]) * mul),
+                       "f"(__uint_as_float(a[4 * t + 3]) * mul) : "memory");
         }
       }
-      // the accumulator buffer may be overwritten by the item after next
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(b_acc_free + 8 * ab);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      named_bar_sync(3, 256);
+      if (warp == 2 && lane == 0) {
+        // issue the stores and go on: their completion is only needed before the staging buffers are
+        // written again (next epilogue) or handed back (after the next item's first step)
+        tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
+        tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile + 16384u, 32, blk * AT_BLK, bh);
+        if (MODE == AT_DKV) {
+          tma_store_3d(&tm_o1, stage2, 0, blk * AT_BLK, bh);
+          tma_store_3d(&tm_o1, stage2 + 16384u, 32, blk * AT_BLK, bh);
+        }
+        tma_store_commit();
+        store_pending = true;
+      }
     }
     }  // items
+    if (warp == 2 && lane == 0) tma_store_wait_all();         // the bulk stores of this CTA have landed
   }
 
   tc_fence_before();
@@ -617,6 +650,20 @@ __global__ void mc_accumulate_kernel(const float* __restrict__ g, const float* _
 
 // ------------------------------------------------------------------------------- host side
 
+// FP32 output [BH][S][64] as two 32-column boxes per 128-row block (128-byte swizzle).
+static int make_out_map(CUtensorMap* map, const void* base, int BH, int S) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return BSP_ERR_CUDA;
+  cuuint64_t gdim[3] = {(cuuint64_t)AT_D, (cuuint64_t)S, (cuuint64_t)BH};
+  cuuint64_t gstr[2] = {(cuuint64_t)AT_D * 4, (cuuint64_t)S * AT_D * 4};
+  cuuint32_t box[3] = {32u, (cuuint32_t)AT_BLK, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
+}
+
 static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return BSP_ERR_CUDA;
@@ -632,8 +679,10 @@ static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
 
 template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
-  CUtensorMap mq, mk, mv, mdo;
+  CUtensorMap mq, mk, mv, mdo, mo0, mo1;
   int rc;
+  if ((rc = make_out_map(&mo0, p.out0, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_out_map(&mo1, p.out1 ? p.out1 : p.out0, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mq, q, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
@@ -650,7 +699,7 @@ static int launch_attn(const void* q, const void* k, const void* v, const void* 
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, p);
+  attn_kernel<MODE><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
