@@ -34,7 +34,10 @@ constexpr int kAtTile = AT_BLK * AT_D * 2;        // 16 KB: one 128 x 64 bf16 ti
 constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
 constexpr int kAtThreads = 320;
 // shared memory: res0, res1, str[2][2], P, dS, barriers
-constexpr int kAtSmem = 4 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/;
+constexpr int kAtBiasTile = AT_BLK * 16 * 2;      // 4 KB: one 128 x 16 bf16 tile of the extra K = 16 step (DKV)
+constexpr int kAtBias = 7 * kAtBiasTile;          // a tile of ones, then three buffers of (LSE tile, D tile)
+constexpr int kAtSmem = 4 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/ +
+                        kAtBias;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AttnParams {
@@ -119,6 +122,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   float* xchg = reinterpret_cast<float*>(bars_gen + 176);   // FWD: row max / sum exchange between column halves
+  // DKV: per-query terms enter the scores through the products themselves.  A thread of that mode
+  // owns a key row, so the query's -LSE and -D would be per-column values (a shared-memory load in
+  // front of every exponential: measured at twice the arithmetic time).  Instead S^T = K Q^T takes one
+  // more K = 16 step, ones[keys x 16] times X[queries x 16]^T, where row q of X holds
+  // -LSE[q] * log2(e) / c2 split into three bf16 terms (24 bits) and zeros, so the accumulator
+  // already is s - LSE/c; likewise dP^T with -D[q].  The tiles are K-major without swizzle: 8-row
+  // groups 256 bytes apart, the two 8-element halves of a row 128 bytes apart, 16 bytes per row.
+  const uint32_t b_bias = bars + 2240;                       // three barriers, one per buffer
+  const uint32_t bias0 = bars + 4096;                        // ones tile; buffer b: X_lse at 1 + 2b, X_d at 2 + 2b
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Persistent CTA: work items w = item_at(0), item_at(1), ... of nblk * BH, heavy blocks first
@@ -153,6 +165,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       mbar_init(b_acc + 8 * s, 1); mbar_init(b_acc_free + 8 * s, 8);
     }
     for (uint32_t s = 0; s < kStg; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
+    for (uint32_t s = 0; s < 3; ++s) mbar_init(b_bias + 8 * s, 8);
     mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -257,6 +270,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
           for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
         }
+        if (MODE == AT_DKV) {
+          // the extra K = 16 step: minus LSE/c into S^T, minus D into dP^T (see the X tiles)
+          const uint32_t bb = jt % 3u;
+          if (!mbar_wait(b_bias + 8 * bb, (jt / 3u) & 1u, abort_flag)) return false;
+          const uint64_t ones = make_smem_desc_k16(bias0);
+          tc_mma<false>(t_s, ones, make_smem_desc_k16(bias0 + (1u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
+          tc_mma<false>(t_dp, ones, make_smem_desc_k16(bias0 + (2u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
+        }
         tc_commit(b_sdp_full);
         return true;
       };
@@ -309,7 +330,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const int q4 = warp & 3, h = (warp - 2) >> 2;
     const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
+    if (MODE == AT_DKV) {
+      // the constant parts of the seven extra tiles: thread ts sets 16 bytes of each (row ts & 127,
+      // half ts >> 7): the first three columns of the ones tile to 1, everything else to 0
+      const int ts0 = (int)threadIdx.x - 64;
+      const uint32_t off = (uint32_t)((ts0 & 127) >> 3) * 256u + (uint32_t)(ts0 >> 7) * 128u + (uint32_t)(ts0 & 7) * 16u;
+#pragma unroll
+      for (uint32_t t = 0; t < 7; ++t) {
+        const bool one = t == 0 && ts0 < 128;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %3};" ::"r"(bias0 + t * kAtBiasTile + off),
+                     "r"(one ? 0x3F803F80u : 0u), "r"(one ? 0x00003F80u : 0u), "r"(0u) : "memory");
+      }
+      named_bar_sync(1, 256);   // before any thread overwrites a row's first half with a step's terms
+    }
     bool ok = true;
+    uint32_t bias_written = 0;                                // DKV: rows of the X tiles written so far (global steps)
     bool store_pending = false;                               // warp 2, lane 0: an epilogue's bulk stores are in flight
     uint32_t itg = 0;                                         // step counter across items
     int item = 0;
@@ -321,26 +356,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const uint32_t ab = kAccDouble ? (item & 1u) : 0u;
     const uint32_t iph = kAccDouble ? ((item >> 1) & 1u) : ((uint32_t)item & 1u);
     const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
-    // DKV: a thread's row is a key and its 64 columns are queries, so the per-query LSE * log2(e) and
-    // D sit in shared memory, one 128 + 128 float vector per step, double-buffered: softmax thread ts
-    // fetches one value of the next step while this step computes.
-    const int ts = (int)threadIdx.x - 64;
-    float* colv = xchg;                                       // [2][256]
-    // the raw value only: nothing may depend on the load before the step's arithmetic is done, or
-    // the in-order warp would sit out the load's latency at the top of every step
-    const float* col_src = ts < 128 ? p.lse : p.dterm;
-    const float col_mul = ts < 128 ? kLog2e : 1.0f;
-    auto col_fetch = [&](int step) -> float {
-      const int q = step * AT_BLK + (ts & 127);
-      return __ldg(col_src + (size_t)bh * p.S + (q < p.S ? q : 0));
-    };
-    auto col_value = [&](int step, float raw) -> float {
-      return step * AT_BLK + (ts & 127) < p.S ? raw * col_mul : 0.f;
-    };
-    if (MODE == AT_DKV && total > 0) {
-      colv[ts] = col_value(it_begin, col_fetch(it_begin));
-      named_bar_sync(1, 256);
-    }
     float inv_q = 1.f, inv_k = 1.f, inv_v = 1.f, inv_do = 1.f;
     if (p.fp8) {
       inv_q = __fdiv_rn(1.0f, __ldg(p.sc_q + bh)); inv_k = __fdiv_rn(1.0f, __ldg(p.sc_k + bh));
@@ -348,6 +363,64 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     const float c2 = p.c * kLog2e * inv_q * inv_k;            // scores arrive as products of decoded codes
     const float dp_mul = inv_do * inv_v;                      // likewise dP
+    // DKV: softmax thread ts owns row (ts & 127) of the X tiles: the LSE tile for ts < 128, the D tile
+    // above.  bias_fetch reads the raw value of a step's query (nothing may depend on that load
+    // before the step's arithmetic is done, or the in-order warp sits out its latency); bias_put
+    // writes the three-term row into buffer (global step) % 3 and signals the MMA issuer.
+    const int ts = (int)threadIdx.x - 64;
+    const float* bias_src = ts < 128 ? p.lse : p.dterm;
+    const float bias_mul = ts < 128 ? -kLog2e / c2 : -1.0f / dp_mul;
+    float nx_mul = bias_mul;                                  // the same factor for the next item's head
+    auto bias_fetch = [&](int tbh, int step) -> float {
+      const int q = step * AT_BLK + (ts & 127);
+      return __ldg(bias_src + (size_t)tbh * p.S + (q < p.S ? q : 0));
+    };
+    auto bias_put = [&](int step, uint32_t jt, float raw, float mul) {
+      const int q = ts & 127;
+      const float x = step * AT_BLK + q < p.S ? raw * mul : 0.f;
+      const __nv_bfloat16 h1 = __float2bfloat16_rn(x);
+      const float r1 = x - __bfloat162float(h1);
+      const __nv_bfloat16 h2 = __float2bfloat16_rn(r1);
+      const __nv_bfloat16 h3 = __float2bfloat16_rn(r1 - __bfloat162float(h2));
+      const uint32_t w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
+      const uint32_t w1 = (uint32_t)__bfloat16_as_ushort(h3);
+      const uint32_t tile = bias0 + (1u + 2u * (jt % 3u) + (ts < 128 ? 0u : 1u)) * kAtBiasTile;
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %3};" ::"r"(tile + (uint32_t)(q >> 3) * 256u + (uint32_t)(q & 7) * 16u),
+                   "r"(w0), "r"(w1), "r"(0u) : "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_bias + 8 * (jt % 3u));
+    };
+    // The rows are written two steps ahead of their use, in the order of the CTA's global step count
+    // (bias_written rows so far), across item boundaries: the last two steps of an item write the first
+    // two rows of the next one, so its first S and dP run under this item's epilogue.  Rows that are
+    // still missing at an item's start (the first item, or after a one-step item) are written here.
+    int nx_bh = 0, nx_begin = 0, nx_total = 0;                // DKV: the next item's head, first step, step count
+    if (MODE == AT_DKV) {
+      const int wn = item_at(item + 1);
+      if (wn < nitems) {
+        int nb, ns;
+        decode_item(wn, nb, nx_bh, nx_begin, ns);
+        nx_total = ns;
+        if (p.fp8) {                                          // per-head operand scales
+          const float nq = __fdiv_rn(1.0f, __ldg(p.sc_q + nx_bh)), nk = __fdiv_rn(1.0f, __ldg(p.sc_k + nx_bh));
+          const float nv = __fdiv_rn(1.0f, __ldg(p.sc_v + nx_bh)), ndo = __fdiv_rn(1.0f, __ldg(p.sc_do + nx_bh));
+          nx_mul = ts < 128 ? -kLog2e / (p.c * kLog2e * nq * nk) : -1.0f / (ndo * nv);
+        }
+      }
+      while (bias_written < itg + (uint32_t)(total < 2 ? total : 2)) {
+        const int l = (int)(bias_written - itg);
+        bias_put(it_begin + l, bias_written, bias_fetch(bh, it_begin + l), bias_mul);
+        ++bias_written;
+      }
+    }
+    // the row that step `it` of this item is to write: global step itg + it + 2
+    auto bias_target = [&](int it, int& tbh, int& tstep) -> bool {
+      const int t = it + 2;
+      if (t < total) { tbh = bh; tstep = it_begin + t; return true; }
+      if (t - total < nx_total) { tbh = nx_bh; tstep = nx_begin + (t - total); return true; }
+      return false;
+    };
     float lse2 = 0.f, dq = 0.f;                               // this row's LSE*log2e and D
     int qrow = 0;                                             // global query index of this thread's row
     if (MODE != AT_DKV) {
@@ -363,7 +436,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
-      float col_next = 0.f;                                   // DKV: this thread's share of the next step's vector
+      float bias_next = 0.f;                                  // DKV: this thread's raw value for the row two steps ahead
+      int bias_bh = 0, bias_step = 0;
+      const bool bias_due = MODE == AT_DKV && bias_written == itg + (uint32_t)it + 2u && bias_target(it, bias_bh, bias_step);
       if (MODE == AT_DKV) {
         kblk = blk;
       } else {
@@ -401,7 +476,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(b_sdp_free);
-      if (MODE == AT_DKV && it + 1 < total) col_next = col_fetch(step + 1);   // lands under this step's arithmetic
+      if (bias_due) bias_next = bias_fetch(bias_bh, bias_step);   // lands under this step's arithmetic
 
       const int key0 = kblk * AT_BLK + h * 64;
       // masking is needed only on the diagonal block and where the sequence ends inside the block
@@ -454,16 +529,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const int key = MODE == AT_DKV ? myrow : cj, qy = MODE == AT_DKV ? cj : myrow;
           return key < p.S && qy < p.S && (!p.causal || key <= qy);
         };
-        const float* cv = colv + (it & 1) * 256 + h * 64;     // DKV: LSE * log2(e) of these 64 queries, D at +128
         // Two columns per iteration on purpose: wider bodies made the compiler's schedule of the
         // exponentials twice as slow.  `masked` adds the validity test that only the diagonal block
         // and the blocks at the end of the sequence need.
         auto pair_at = [&](int j, bool masked) {
-          float l0 = lse2, l1 = lse2, d0 = dq, d1 = dq;
-          if (MODE == AT_DKV) {
-            const float2 a = *reinterpret_cast<const float2*>(cv + j), b = *reinterpret_cast<const float2*>(cv + 128 + j);
-            l0 = a.x; l1 = a.y; d0 = b.x; d1 = b.y;
-          }
+          // DKV: the accumulators already hold s - LSE/c and dP - D (see the X tiles)
+          const float l0 = MODE == AT_DKV ? 0.f : lse2, d0 = MODE == AT_DKV ? 0.f : dq;
+          const float l1 = l0, d1 = d0;
           float a0 = fmaf(__uint_as_float(sv[j]), c2, -l0), a1 = fmaf(__uint_as_float(sv[j + 1]), c2, -l1);
           if (masked) {
             if (!valid_at(j)) a0 = -INFINITY;
@@ -508,12 +580,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         mbar_arrive(b_res_empty + 8 * (((uint32_t)item & 1u) ^ 1u));
         store_pending = false;
       }
-      if (MODE == AT_DKV) {
-        // publish the next step's per-query vector; everyone is past this step's reads of the other one
+      if (bias_due) {
         // (the empty asm pins the first use of the fetched value here, after the step's arithmetic)
-        asm volatile("" : "+f"(col_next));
-        colv[((it + 1) & 1) * 256 + ts] = col_value(step + 1, col_next);
-        named_bar_sync(1, 256);
+        asm volatile("" : "+f"(bias_next));
+        bias_put(bias_step, bias_written, bias_next, bias_bh == bh && it + 2 < total ? bias_mul : nx_mul);
+        ++bias_written;
       }
     }
     itg += (uint32_t)total;

@@ -196,6 +196,18 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t smem_addr, uint32
   return d;
 }
 
+// A K-major operand of one K = 16 step (16-bit elements) without swizzle: rows of 16 bytes, eight
+// rows per 128-byte core matrix, the two 8-element halves of a row 128 bytes apart (leading byte
+// offset), 8-row groups 256 bytes apart (stride byte offset).
+__device__ __forceinline__ uint64_t make_smem_desc_k16(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(128u >> 4) << 16;
+  d |= (uint64_t)(256u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  return d;
+}
+
 // Instruction descriptor: FP32 accumulator, K-major A and B, M x N tile.
 // a_fmt / b_fmt: kind::f8f6f4 E4M3 = 0, E5M2 = 1; kind::f16 BF16 = 1.
 __host__ __device__ constexpr uint32_t make_idesc(uint32_t a_fmt, uint32_t b_fmt, uint32_t M, uint32_t N) {
