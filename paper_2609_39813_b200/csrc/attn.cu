@@ -33,6 +33,8 @@ constexpr int AT_BLK = 128, AT_D = 64;
 constexpr int kAtTile = AT_BLK * AT_D * 2;        // 16 KB: one 128 x 64 bf16 tile
 constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
 constexpr int kAtThreads = 320;
+constexpr int kAtSoftWarp0 = 2;                   // first softmax warp
+constexpr int kAtSoftThread0 = kAtSoftWarp0 * 32;
 // shared memory: res0, res1, str[2][2], P, dS, barriers
 constexpr int kAtBiasTile = AT_BLK * 16 * 2;      // 4 KB: one 128 x 16 bf16 tile of the extra K = 16 step (DKV)
 constexpr int kAtBias = 7 * kAtBiasTile;          // a tile of ones, then three buffers of (LSE tile, D tile)
@@ -93,7 +95,9 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
       : "memory");
 }
 
-template <int MODE>
+// FP8: the FP8-operand mode (per-head operand scales, P and dS rounded onto the FP8 grids); a
+// template parameter because its tests and extra multiplications sit in the innermost loop.
+template <int MODE, bool FP8>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -325,15 +329,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       }  // items
     }
-  } else {
+  } else if (warp >= kAtSoftWarp0) {
     // ------------------------------------------------ softmax / dS warps, then the epilogue
-    const int q4 = warp & 3, h = (warp - 2) >> 2;
+    const int q4 = warp & 3, h = (warp - kAtSoftWarp0) >> 2;
     const int r = q4 * 32 + lane;                             // row inside the 128-row block (a query)
     const uint32_t lane_off = (uint32_t)(q4 * 32) << 16;
     if (MODE == AT_DKV) {
       // the constant parts of the seven extra tiles: thread ts sets 16 bytes of each (row ts & 127,
       // half ts >> 7): the first three columns of the ones tile to 1, everything else to 0
-      const int ts0 = (int)threadIdx.x - 64;
+      const int ts0 = (int)threadIdx.x - kAtSoftThread0;
       const uint32_t off = (uint32_t)((ts0 & 127) >> 3) * 256u + (uint32_t)(ts0 >> 7) * 128u + (uint32_t)(ts0 & 7) * 16u;
 #pragma unroll
       for (uint32_t t = 0; t < 7; ++t) {
@@ -357,17 +361,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     const uint32_t iph = kAccDouble ? ((item >> 1) & 1u) : ((uint32_t)item & 1u);
     const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
     float inv_q = 1.f, inv_k = 1.f, inv_v = 1.f, inv_do = 1.f;
-    if (p.fp8) {
+    if (FP8) {
       inv_q = __fdiv_rn(1.0f, __ldg(p.sc_q + bh)); inv_k = __fdiv_rn(1.0f, __ldg(p.sc_k + bh));
       inv_v = __fdiv_rn(1.0f, __ldg(p.sc_v + bh)); inv_do = __fdiv_rn(1.0f, __ldg(p.sc_do + bh));
     }
-    const float c2 = p.c * kLog2e * inv_q * inv_k;            // scores arrive as products of decoded codes
-    const float dp_mul = inv_do * inv_v;                      // likewise dP
+    const float c2 = FP8 ? p.c * kLog2e * inv_q * inv_k : p.c * kLog2e;   // scores arrive as products of decoded codes
+    const float dp_mul = FP8 ? inv_do * inv_v : 1.0f;                     // likewise dP
     // DKV: softmax thread ts owns row (ts & 127) of the X tiles: the LSE tile for ts < 128, the D tile
     // above.  bias_fetch reads the raw value of a step's query (nothing may depend on that load
     // before the step's arithmetic is done, or the in-order warp sits out its latency); bias_put
     // writes the three-term row into buffer (global step) % 3 and signals the MMA issuer.
-    const int ts = (int)threadIdx.x - 64;
+    const int ts = (int)threadIdx.x - kAtSoftThread0;
     const float* bias_src = ts < 128 ? p.lse : p.dterm;
     const float bias_mul = ts < 128 ? -kLog2e / c2 : -1.0f / dp_mul;
     float nx_mul = bias_mul;                                  // the same factor for the next item's head
@@ -402,7 +406,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         int nb, ns;
         decode_item(wn, nb, nx_bh, nx_begin, ns);
         nx_total = ns;
-        if (p.fp8) {                                          // per-head operand scales
+        if (FP8) {                                            // per-head operand scales
           const float nq = __fdiv_rn(1.0f, __ldg(p.sc_q + nx_bh)), nk = __fdiv_rn(1.0f, __ldg(p.sc_k + nx_bh));
           const float nv = __fdiv_rn(1.0f, __ldg(p.sc_v + nx_bh)), ndo = __fdiv_rn(1.0f, __ldg(p.sc_do + nx_bh));
           nx_mul = ts < 128 ? -kLog2e / (p.c * kLog2e * nq * nk) : -1.0f / (ndo * nv);
@@ -514,7 +518,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             s0 = p0 * (__uint_as_float(dp0) * dp_mul - d0);
             s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
           }
-          if (p.fp8 && MODE != AT_FWD) {                    // the forward keeps P unrounded
+          if (FP8 && MODE != AT_FWD) {                      // the forward keeps P unrounded
             p0 = f8_rn_value<BSP_E4M3>(p0 * p.p_scale); p1 = f8_rn_value<BSP_E4M3>(p1 * p.p_scale);
             s0 = f8_rn_value<BSP_E5M2>(s0 * p.ds_scale); s1 = f8_rn_value<BSP_E5M2>(s1 * p.ds_scale);
           }
@@ -573,7 +577,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (MODE == AT_FWD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(b_pds_ready);
-      if (it == 0 && warp == 2 && lane == 0 && store_pending) {
+      if (it == 0 && warp == kAtSoftWarp0 && lane == 0 && store_pending) {
         // the previous item's output has left its staging buffer by now: hand the resident-tile
         // buffer it used back to the TMA producer
         tma_store_wait_read();
@@ -598,7 +602,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const uint32_t rbi = (uint32_t)item & 1u;
       constexpr int nout = MODE == AT_DKV ? 2 : 1;            // DKV: dV (acc0) and dK (acc1)
       // the stores of the item before have long read their staging buffers; make that certain
-      if (warp == 2 && lane == 0 && store_pending) {
+      if (warp == kAtSoftWarp0 && lane == 0 && store_pending) {
         tma_store_wait_read();
         mbar_arrive(b_res_empty + 8 * (rbi ^ 1u));
         store_pending = false;
@@ -608,8 +612,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int o = 0; o < nout; ++o) {
         const uint32_t stg = o == 0 ? res_base + rbi * 2 * kAtTile : stage2;
         float mul;
-        if (MODE == AT_DKV) mul = o == 0 ? (p.fp8 ? inv_do / p.p_scale : 1.f) : p.c * (p.fp8 ? inv_q / p.ds_scale : 1.f);
-        else if (MODE == AT_DQ) mul = p.c * (p.fp8 ? inv_k / p.ds_scale : 1.f);
+        if (MODE == AT_DKV) mul = o == 0 ? (FP8 ? inv_do / p.p_scale : 1.f) : p.c * (FP8 ? inv_q / p.ds_scale : 1.f);
+        else if (MODE == AT_DQ) mul = p.c * (FP8 ? inv_k / p.ds_scale : 1.f);
         else mul = inv_v;
         uint32_t a[32];
         tmem_ld32((o == 0 ? t_acc0 : t_acc1) + lane_off + h * 32, a);
@@ -629,7 +633,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       named_bar_sync(3, 256);
-      if (warp == 2 && lane == 0) {
+      if (warp == kAtSoftWarp0 && lane == 0) {
         // issue the stores and go on: their completion is only needed before the staging buffers are
         // written again (next epilogue) or handed back (after the next item's first step)
         tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
@@ -643,7 +647,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
     }
     }  // items
-    if (warp == 2 && lane == 0) tma_store_wait_all();         // the bulk stores of this CTA have landed
+    if (warp == kAtSoftWarp0 && lane == 0) tma_store_wait_all();         // the bulk stores of this CTA have landed
   }
 
   tc_fence_before();
@@ -748,8 +752,8 @@ static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
 }
 
-template <int MODE>
-static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
+template <int MODE, bool FP8>
+static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mdo, mo0, mo1;
   int rc;
   if ((rc = make_out_map(&mo0, p.out0, p.BH, p.S)) != BSP_OK) return rc;
@@ -760,7 +764,7 @@ static int launch_attn(const void* q, const void* k, const void* v, const void* 
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
   static bool attr_set = false;
   if (!attr_set) {
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
@@ -770,9 +774,14 @@ static int launch_attn(const void* q, const void* k, const void* v, const void* 
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
+  attn_kernel<MODE, FP8><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
+}
+
+template <int MODE>
+static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
+  return p.fp8 ? launch_attn_mode<MODE, true>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false>(q, k, v, dO, p, st);
 }
 
 static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
