@@ -547,17 +547,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           pack_pair(ex2_approx(a0), ex2_approx(a1), dv[j], dv[j + 1], d0, d1, pk[j >> 1], dk[j >> 1]);
         };
-        if (!edge) {
-#pragma unroll
-          for (int j = 0; j < 64; j += 2) pair_at(j, false);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 64; j += 2) pair_at(j, true);
-        }
-        // the P / dS operands are free once the products of the previous step have read them
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
-        if (!ok) break;
         if (MODE == AT_FWD) {
+          if (!edge) {
+#pragma unroll
+            for (int j = 0; j < 64; j += 2) pair_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 64; j += 2) pair_at(j, true);
+          }
+          // the P buffer is free once the product of the previous step has read it
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          if (!ok) break;
           // 64 keys = 8 chunks of 16 bytes in row r of half h of the shared P buffer: chunk index t ^ (r & 7)
 #pragma unroll
           for (int t = 0; t < 8; ++t) {
@@ -565,11 +565,47 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
                          "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
           }
-        } else {
-          // back into tensor memory as the A operand of the next products: this row's 64 columns are
-          // 32 packed pairs, at columns h*32 .. h*32+31 of the operand
-          if (MODE == AT_DKV) tmem_st32(t_p + lane_off + h * 32, pk);
+        } else if (MODE == AT_DQ) {
+          if (!edge) {
+#pragma unroll
+            for (int j = 0; j < 64; j += 2) pair_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 64; j += 2) pair_at(j, true);
+          }
+          // the dS operand is free once the product of the previous step has read it; then the row's
+          // 64 columns go back into tensor memory as 32 packed pairs (columns h*32 .. h*32+31)
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          if (!ok) break;
           tmem_st32(t_ds + lane_off + h * 32, dk);
+          tmem_wait_st();
+          tc_fence_before();
+        } else {
+          // DKV: P and dS go back into tensor memory as 32 packed pairs each (columns h*32 .. h*32+31
+          // of the operands), in two halves: the first half is stored while the second is computed,
+          // which also halves the registers the packed values hold.  The operands are free once the
+          // products of the previous step have read them: that wait sits between the halves, where it
+          // has long passed.
+          if (!edge) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair_at(j, true);
+          }
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          if (!ok) break;
+          tmem_st16(t_p + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+          tmem_st16(t_ds + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
+          if (!edge) {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair_at(j, true);
+          }
+          tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+          tmem_st16(t_ds + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
           tmem_wait_st();
           tc_fence_before();
         }
