@@ -56,6 +56,10 @@ CASES = {
     "three_blocks": dict(B=2, H=1, S=384, causal=True),
     "noncausal": dict(B=1, H=1, S=256, causal=False),
     "one_short_block": dict(B=1, H=3, S=72, causal=True),
+    # 450 (block, head) items on 148 persistent CTAs: every CTA walks three or four items of one, two
+    # and three steps, so the hand-overs between items (resident tiles, accumulators, the rows written
+    # two steps ahead, the deferred output stores) are all exercised, with a ragged last block
+    "many_items_ragged": dict(B=3, H=50, S=328, causal=True),
 }
 
 
@@ -194,7 +198,7 @@ def test_mc_check_attention_verdicts(b):
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
 
 
-@pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks"])
+@pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks", "many_items_ragged"])
 def test_fp8_operand_mode(b, name):
     """The emulated FP8 attention backward: Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice, P rounded
     to E4M3 at scale 256 before dV, dS rounded to E5M2 at a supplied scale before dQ and dK."""
