@@ -164,6 +164,25 @@ __device__ __forceinline__ float f8_sr_value(float v, uint32_t U) {
   return __uint_as_float(s | __float_as_uint(mag));
 }
 
+// The draw-independent part of the stochastic rounding of v: the threshold P such that the
+// element rounds up (away from zero, by one code) exactly when its generator word U < P.  The same
+// decision as f8_encode / f8_sr_value take: P = 0 when v is on the grid, saturates or is NaN.  With
+// it, K draws of one element cost one comparison each: value(U) = value(~0) + (U < P) * step, and
+// code(U) = code(~0) + (U < P).
+template <int FMT>
+__device__ __forceinline__ uint32_t f8_sr_threshold(float v) {
+  using F = F8<FMT>;
+  const uint32_t a = __float_as_uint(v) & 0x7FFFFFFFu;
+  if (a >= F::FMAX_BITS) return 0u;
+  if (a >= F::MINNORM_BITS) {
+    constexpr int d = 23 - F::MB;
+    return (a & ((1u << d) - 1u)) << (32 - d);
+  }
+  const float t = __uint_as_float(a) * __uint_as_float((uint32_t)(F::MB - F::EMIN + 127) << 23);
+  const float f = t - (float)(uint32_t)t;
+  return __float2uint_rd(f * 4294967296.0f);
+}
+
 // Nearest-even rounding of two in-range FP32 values (|v| below the format's maximum) to two codes
 // with the hardware conversion: `lo` in bits 0..7, `hi` in bits 8..15.  NaN, infinities and
 // magnitudes at or above the maximum never come here (the callers route those to f8_encode).

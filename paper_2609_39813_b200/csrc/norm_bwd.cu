@@ -211,12 +211,17 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
                int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */) {
-  // The slab's scaled values and weights live in shared memory (each thread reads back only what
-  // it wrote), which keeps the register count low enough for three blocks per SM: the draw loop
-  // is a chain of dependent integer multiplies, and it is occupancy that hides their latency.
+  // A fresh rounding of an element is its round-down value plus, with probability frac, one grid
+  // step: value(U) = lo + (U < P) * (hi - lo) with the threshold P of f8_sr_threshold.  So the
+  // gain-use sum of draw k is  sum_t (lo/scale - beta)/gamma * du  (the same for every draw, summed
+  // once) plus  sum_t [U_k,t < P_t] * (hi - lo)/scale/gamma * du : per element and draw one generator
+  // word, one comparison and one conditional add.  The slab's thresholds and step weights live in
+  // shared memory (each thread reads back only what it wrote), which keeps the register count low
+  // enough for three blocks per SM: the draw loop is a chain of dependent integer multiplies, and it
+  // is occupancy that hides their latency.
   extern __shared__ __align__(16) float4 mc_smem[];
-  float4* sv = mc_smem;                         // [kMcRows][256]
-  float4* sw = mc_smem + kMcRows * 256;         // [kMcRows][256]
+  uint4* sp = reinterpret_cast<uint4*>(mc_smem);   // [kMcRows][256] thresholds
+  float4* sw = mc_smem + kMcRows * 256;            // [kMcRows][256] step weights
   __shared__ __align__(16) float red[2][8][kMcCols];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t c = (int64_t)blockIdx.x * kMcCols + lane * 4;
@@ -234,10 +239,12 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
   // q0 + i*qstep; rows beyond T keep v = wgt = 0 and contribute nothing whatever word they draw
   const uint64_t q0 = (uint64_t)((slab * kMcSlab + warp) * C + (col_ok ? c : 0)) >> 2;
   const uint64_t qstep = (uint64_t)(2 * C);
+  float base[4] = {0.f, 0.f, 0.f, 0.f};                 // the draw-independent part of this thread's sums
 #pragma unroll 1
   for (int i = 0; i < kMcRows; ++i) {
     const int64_t r = slab * kMcSlab + warp + 8 * i;
-    float v[4] = {0.f, 0.f, 0.f, 0.f}, wgt[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t thr[4] = {0u, 0u, 0u, 0u};
+    float wgt[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < T && col_ok) {
       const size_t i0 = (size_t)r * C + c;
       const float4 xv = load4<DT>(x, i0);
@@ -253,29 +260,29 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
         float u;
         if (kind == BSP_RMSNORM) u = __fmul_rn(__fmul_rn(xs[e], rs), gg[e]);
         else u = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xs[e], mu), rs), gg[e]), bb[e]);
-        v[e] = __fmul_rn(u, scale);
-        wgt[e] = __fdiv_rn(ds[e], gg[e]);
+        const float v = __fmul_rn(u, scale);
+        const float w = __fdiv_rn(ds[e], gg[e]);
+        const float lo = sr_value<FMT>(v, 0xFFFFFFFFu), hi = sr_value<FMT>(v, 0u);   // never up / up whenever possible
+        thr[e] = f8_sr_threshold<FMT>(v);
+        base[e] = fmaf(fmaf(lo, inv_scale, -bb[e]), w, base[e]);
+        wgt[e] = thr[e] ? (hi - lo) * inv_scale * w : 0.f;      // (NaN has threshold 0: it stays in base)
       }
     }
-    sv[i * 256 + tid] = make_float4(v[0], v[1], v[2], v[3]);
+    sp[i * 256 + tid] = make_uint4(thr[0], thr[1], thr[2], thr[3]);
     sw[i * 256 + tid] = make_float4(wgt[0], wgt[1], wgt[2], wgt[3]);
   }
-  const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
   for (int k = 0; k < ndraws; ++k) {
     const uint32_t draw = (uint32_t)(draw_begin + k);
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[4] = {base[0], base[1], base[2], base[3]};
 #pragma unroll 2
     for (int i = 0; i < kMcRows; ++i) {
       const uint4 w = philox_block(key, q0 + (uint64_t)i * qstep, draw);
-      const float4 v4 = sv[i * 256 + tid], w4 = sw[i * 256 + tid];
-      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-      const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
-      const float wg[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float val = sr_value<FMT>(vv[e], ww[e]);
-        acc[e] = fmaf(fmaf(val, inv_scale, -bb[e]), wg[e], acc[e]);
-      }
+      const uint4 p4 = sp[i * 256 + tid];
+      const float4 w4 = sw[i * 256 + tid];
+      acc[0] += w.x < p4.x ? w4.x : 0.f;
+      acc[1] += w.y < p4.y ? w4.y : 0.f;
+      acc[2] += w.z < p4.z ? w4.z : 0.f;
+      acc[3] += w.w < p4.w ? w4.w : 0.f;
     }
     const int buf = k & 1;
     *reinterpret_cast<float4*>(&red[buf][warp][lane * 4]) = make_float4(acc[0], acc[1], acc[2], acc[3]);

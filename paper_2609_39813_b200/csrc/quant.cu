@@ -310,13 +310,35 @@ reround_draws_kernel(NormProducer prod, const void* __restrict__ x, int64_t rows
   const int64_t cc = c0 + tcol, rr = r0 + trow;
   const bool wr = cc < cols && rr < rows;
   const int nvalid = wr ? (int)((rows - rr) < 16 ? (rows - rr) : 16) : 0;
-  DiagCounters dc;
+  // A fresh rounding of an element is its round-down code plus one exactly when the element's
+  // generator word falls below the threshold of f8_sr_threshold: both are fixed across draws, so a
+  // draw costs one generator block, four comparisons and four conditional adds per four elements.
+  // (A code that can round up is below the format's top code, so the add never carries out of its byte.)
+  uint32_t thr[16], lo4[4] = {0u, 0u, 0u, 0u};
+  {
+    DiagCounters dc;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      thr[j] = f8_sr_threshold<FMT>(v[j]);
+      lo4[j >> 2] |= f8_encode<FMT, true>(v[j], 0xFFFFFFFFu, dc) << (8 * (j & 3));
+    }
+  }
   for (int d = 0; d < ndraws; ++d) {
     const int buf = d & 1;
     if (active) {
-      const uint4 pk = encode16<FMT, BSP_ROUND_STOCHASTIC>(v, key, (uint32_t)(draw0 + d), (uint64_t)i0, dc);
+      uint32_t pk[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const uint4 w = philox_block(key, ((uint64_t)i0 >> 2) + b, (uint32_t)(draw0 + d));
+        uint32_t c4 = lo4[b];
+        c4 += w.x < thr[4 * b + 0] ? 0x1u : 0u;
+        c4 += w.y < thr[4 * b + 1] ? 0x100u : 0u;
+        c4 += w.z < thr[4 * b + 2] ? 0x10000u : 0u;
+        c4 += w.w < thr[4 * b + 3] ? 0x1000000u : 0u;
+        pk[b] = c4;
+      }
       uint32_t* dst = reinterpret_cast<uint32_t*>(&s_codes[buf][tr][tc]);
-      dst[0] = pk.x; dst[1] = pk.y; dst[2] = pk.z; dst[3] = pk.w;
+      dst[0] = pk[0]; dst[1] = pk[1]; dst[2] = pk[2]; dst[3] = pk[3];
     }
     __syncthreads();
     if (wr) {
