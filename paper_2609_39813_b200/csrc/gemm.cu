@@ -35,6 +35,7 @@ struct GemmParams {
   int elem_bytes;         // 1 (FP8) or 2 (BF16)
   int a_mn, b_mn;         // operand stored [K][M] / [K][N] (MN-major) instead of [M][K] / [N][K]
   uint32_t idesc;
+  uint32_t idesc2;               // gemm_mc_kernel: the 128 x 256 product over a pair of draws
   float sa, sb;           // operand scales; alpha = (1/sa) * (1/sb)
   const float* sa_dev;
   const float* sb_dev;
@@ -229,8 +230,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // 320 threads: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue (two warps per TMEM lane quarter, each
 // owning 64 of the 128 columns).
 constexpr int MC_BN = 128;
-constexpr int kMcStages = 6;
-constexpr int kMcABytes = BM * BKB, kMcBBytes = MC_BN * BKB, kMcStageBytes = kMcABytes + kMcBBytes;
+// Draws are taken two at a time: a stage holds the A tile and the B tiles of both draws, one
+// after the other, so a single 128 x 256 product per K slice fills both accumulators and the A tile
+// is fetched (from L2 and from shared memory) once for two draws.
+constexpr int kMcStages = 4;
+constexpr int kMcABytes = BM * BKB, kMcBBytes = MC_BN * BKB, kMcStageBytes = kMcABytes + 2 * kMcBBytes;
 constexpr int kMcThreads = 320;
 constexpr size_t kMcSmem = (size_t)kMcStages * kMcStageBytes + 1024 + 256;
 
@@ -272,14 +276,16 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
         const int tm = t / tiles_n, tn = t % tiles_n;
-        for (int b = 0; b < p.nb && ok; ++b) {
+        for (int b = 0; b < p.nb && ok; b += 2) {
+          const bool two = b + 1 < p.nb;                       // an odd count ends with a single draw
           for (int kb = 0; kb < kblocks; ++kb, ++it) {
             const uint32_t s = it % kMcStages, ph = (it / kMcStages) & 1u;
             if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
-            mbar_expect_tx(full0 + 8 * s, kMcStageBytes);
+            mbar_expect_tx(full0 + 8 * s, kMcABytes + (two ? 2 : 1) * kMcBBytes);
             tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * BKB, tm * BM);
             tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b);
+            if (two) tma_load_3d(sb + kMcBBytes, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b + 1);
           }
         }
       }
@@ -292,23 +298,25 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t it = 0, tc = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        for (int b = 0; b < p.nb && ok; ++b, ++tc) {
-          const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
-          if (!mbar_wait(tempty0 + 8 * as, aph ^ 1u, abort_flag)) { ok = false; break; }
+        for (int b = 0; b < p.nb && ok; b += 2, ++tc) {
+          const bool two = b + 1 < p.nb;
+          // both accumulators (columns 0..127 and 128..255) belong to this pair of draws; the
+          // epilogue of the pair before must be through with them
+          if (!mbar_wait(tempty0, (tc & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t tmem_d = tmem_base + as * MC_BN;
+          const uint32_t idesc = two ? p.idesc2 : p.idesc;
           for (int kb = 0; kb < kblocks; ++kb, ++it) {
             const uint32_t s = it % kMcStages, ph = (it / kMcStages) & 1u;
             if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
-            const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+            const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);   // B: 128 or 256 rows
 #pragma unroll
             for (int k = 0; k < BKB / 32; ++k)
-              tc_mma<true>(tmem_d, adesc + 2u * k, bdesc + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+              tc_mma<true>(tmem_base, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
             tc_commit(empty0 + 8 * s);
           }
-          if (ok) tc_commit(tfull0 + 8 * as);
+          if (ok) tc_commit(tfull0);
         }
       }
     }
@@ -350,24 +358,32 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       tmem_wait_st();
       // ---- every draw of this tile
-      for (int b = 0; b < p.nb && ok; ++b, ++tc) {
-        const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull0 + 8 * as, aph, abort_flag));
+      for (int b = 0; b < p.nb && ok; b += 2, ++tc) {
+        const bool two = b + 1 < p.nb;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(tfull0, tc & 1u, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t acc_base = lane_base + as * MC_BN + h * 64;
+        const uint32_t acc_base = lane_base + h * 64;         // draw b; draw b + 1 is MC_BN columns further
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          uint32_t acc[16], a1[16], a2[16];
+          uint32_t acc[16], acc2[16], a1[16], a2[16];
           tmem_ld16(acc_base + c * 16, acc);
+          if (two) tmem_ld16(acc_base + MC_BN + c * 16, acc2);
           tmem_ld16(s1_base + c * 16, a1);
           tmem_ld16(s2_base + c * 16, a2);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
+            // the sums take the draws in order, as a one-draw-at-a-time pass would
             const float d = __uint_as_float(acc[j]) * inv_a * inv_b - refv[c * 16 + j];
-            a1[j] = __float_as_uint(__uint_as_float(a1[j]) + d);
-            a2[j] = __float_as_uint(fmaf(d, d, __uint_as_float(a2[j])));
+            float t1 = __uint_as_float(a1[j]) + d, t2 = fmaf(d, d, __uint_as_float(a2[j]));
+            if (two) {
+              const float e = __uint_as_float(acc2[j]) * inv_a * inv_b - refv[c * 16 + j];
+              t1 += e;
+              t2 = fmaf(e, e, t2);
+            }
+            a1[j] = __float_as_uint(t1);
+            a2[j] = __float_as_uint(t2);
           }
           tmem_st16(s1_base + c * 16, a1);
           tmem_st16(s2_base + c * 16, a2);
@@ -375,7 +391,7 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tmem_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty0 + 8 * as);
+        if (lane == 0) mbar_arrive(tempty0);
       }
       if (!ok) break;
       // ---- tile end: running sums back to global memory
@@ -550,6 +566,7 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, MC_BN);
     if (rc != BSP_OK) return rc;
     p.idesc = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, MC_BN);
+    p.idesc2 = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, 2 * MC_BN);
     static bool mc_attr_set = false;
     if (!mc_attr_set) {
       BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
