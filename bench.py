@@ -394,10 +394,10 @@ def run_ours(args):
     achieved = flops / (gemm_ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16_tflops"]        # FP8 dense = 2 x the measured BF16 burst figure
     # DRAM bytes of one launch of this kernel at this shape, from one ncu capture of this command
-    # (dram__bytes_read.sum 604.6 MB + dram__bytes_write.sum 23.6 MB; profiles/gemm_mc_kernel_cfg2.md).
+    # (dram__bytes_read.sum 604.7 MB + dram__bytes_write.sum 23.1 MB; profiles/gemm_mc_kernel_cfg2.md).
     # The launch's operands are K x T x C = 268 MB of fresh codes, read once per column of output
     # tiles that does not find them in L2, plus 16.8 MB of dY codes and 3 x 16.8 MB of sums.
-    traffic = 628.2e6 if (T, C, O, K) == (4096, 1024, 4096, 64) else None
+    traffic = 627.8e6 if (T, C, O, K) == (4096, 1024, 4096, 64) else None
     roofline = dict(bound="tensor", kernel="gemm_mc_kernel (FP8 weight gradient over K draws, TMEM-resident sums)",
                     achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=traffic,
                     traffic_unit="bytes per launch (ncu dram read + write, one capture)",
