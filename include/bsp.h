@@ -323,8 +323,9 @@ int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const fl
                    const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key,
                    int draw0, int n_draws, float* d_out, bsp_diag_t* diag, void* stream);
 
-/* Backward given D (dterm[B,H,S]).  dk and dv are produced together (both NULL or both set);
- * dq may be NULL. */
+/* Backward given D (dterm[B,H,S]).  dq may be NULL; dk and dv may both be NULL; dv may be NULL
+ * alone (dK only: dV does not read D, so the draws of a fresh read need it once); dv without dk
+ * is BSP_ERR_ARG. */
 int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
                        const void* k, const void* v, const void* dO, int dt, const float* lse,
                        const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,

@@ -97,7 +97,9 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 
 // FP8: the FP8-operand mode (per-head operand scales, P and dS rounded onto the FP8 grids); a
 // template parameter because its tests and extra multiplications sit in the innermost loop.
-template <int MODE, bool FP8>
+// DV (dK/dV mode only): false leaves dV out (its product, the P operand and its store): dV does
+// not read the correction term, so the draws of a fresh read need it once, not K times.
+template <int MODE, bool FP8, bool DV>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -300,8 +302,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
           // queries), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
           const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
+          if (DV) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
+            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
+          }
 #pragma unroll
           for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
         } else if (MODE == AT_DQ) {
@@ -595,7 +599,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
-          tmem_st16(t_p + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+          if (DV) tmem_st16(t_p + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
           tmem_st16(t_ds + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
           if (!edge) {
 #pragma unroll
@@ -604,7 +608,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair_at(j, true);
           }
-          tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+          if (DV) tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
           tmem_st16(t_ds + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
           tmem_wait_st();
           tc_fence_before();
@@ -645,7 +649,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       if (MODE == AT_DKV) named_bar_sync(3, 256);             // ... before anyone writes the second staging buffer again
 #pragma unroll
-      for (int o = 0; o < nout; ++o) {
+      for (int o = (MODE == AT_DKV && !DV) ? 1 : 0; o < nout; ++o) {
         const uint32_t stg = o == 0 ? res_base + rbi * 2 * kAtTile : stage2;
         float mul;
         if (MODE == AT_DKV) mul = o == 0 ? (FP8 ? inv_do / p.p_scale : 1.f) : p.c * (FP8 ? inv_q / p.ds_scale : 1.f);
@@ -672,8 +676,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (warp == kAtSoftWarp0 && lane == 0) {
         // issue the stores and go on: their completion is only needed before the staging buffers are
         // written again (next epilogue) or handed back (after the next item's first step)
-        tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
-        tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile + 16384u, 32, blk * AT_BLK, bh);
+        if (MODE != AT_DKV || DV) {
+          tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
+          tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile + 16384u, 32, blk * AT_BLK, bh);
+        }
         if (MODE == AT_DKV) {
           tma_store_3d(&tm_o1, stage2, 0, blk * AT_BLK, bh);
           tma_store_3d(&tm_o1, stage2 + 16384u, 32, blk * AT_BLK, bh);
@@ -745,16 +751,18 @@ attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig,
   }
 }
 
-// S1 += g - ref, S2 += (g - ref)^2, elementwise.
+// S1 += times * (g - ref), S2 += times * (g - ref)^2, elementwise (times = 1: one draw; K: a value
+// that is the same for K draws).
 __global__ void mc_accumulate_kernel(const float* __restrict__ g, const float* __restrict__ ref, float* __restrict__ S1,
-                                     float* __restrict__ S2, size_t n4) {
+                                     float* __restrict__ S2, size_t n4, float times) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n4) return;
   const float4 a = __ldg(reinterpret_cast<const float4*>(g) + i), r = __ldg(reinterpret_cast<const float4*>(ref) + i);
   float4 s1 = reinterpret_cast<float4*>(S1)[i], s2 = reinterpret_cast<float4*>(S2)[i];
   const float d0 = a.x - r.x, d1 = a.y - r.y, d2 = a.z - r.z, d3 = a.w - r.w;
-  s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
-  s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y); s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
+  s1.x = fmaf(times, d0, s1.x); s1.y = fmaf(times, d1, s1.y); s1.z = fmaf(times, d2, s1.z); s1.w = fmaf(times, d3, s1.w);
+  s2.x = fmaf(times * d0, d0, s2.x); s2.y = fmaf(times * d1, d1, s2.y);
+  s2.z = fmaf(times * d2, d2, s2.z); s2.w = fmaf(times * d3, d3, s2.w);
   reinterpret_cast<float4*>(S1)[i] = s1;
   reinterpret_cast<float4*>(S2)[i] = s2;
 }
@@ -788,11 +796,11 @@ static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
 }
 
-template <int MODE, bool FP8>
+template <int MODE, bool FP8, bool DV>
 static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mdo, mo0, mo1;
   int rc;
-  if ((rc = make_out_map(&mo0, p.out0, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_out_map(&mo0, p.out0 ? p.out0 : p.out1, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_out_map(&mo1, p.out1 ? p.out1 : p.out0, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mq, q, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
@@ -800,7 +808,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
   static bool attr_set = false;
   if (!attr_set) {
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
@@ -810,14 +818,16 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE, FP8><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
+  attn_kernel<MODE, FP8, DV><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
 
 template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
-  return p.fp8 ? launch_attn_mode<MODE, true>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false>(q, k, v, dO, p, st);
+  if (MODE == AT_DKV && p.out0 == nullptr)                   // dK only
+    return p.fp8 ? launch_attn_mode<MODE, true, false>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false, false>(q, k, v, dO, p, st);
+  return p.fp8 ? launch_attn_mode<MODE, true, true>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false, true>(q, k, v, dO, p, st);
 }
 
 static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
@@ -919,7 +929,7 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !dO || !lse || !dterm) return BSP_ERR_ARG;
-  if ((dk == nullptr) != (dv == nullptr) || (!dq && !dk)) return BSP_ERR_ARG;
+  if ((dv && !dk) || (!dq && !dk)) return BSP_ERR_ARG;          // dV comes with dK; dK may come alone
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return BSP_ERR_ALIGN;
@@ -1030,7 +1040,7 @@ int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, 
   if (!aligned16(g) || !aligned16(g_ref) || !aligned16(S1) || !aligned16(S2)) return BSP_ERR_ALIGN;
   if (n == 0) return BSP_OK;
   const size_t n4 = n / 4;
-  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(g, g_ref, S1, S2, n4);
+  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(g, g_ref, S1, S2, n4, 1.0f);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
@@ -1040,6 +1050,17 @@ int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, 
 // ------------------------------------------------------------------------------- per-use check, attention
 
 namespace bsp {
+
+// bsp_mc_accumulate for a value that is the same in `times` draws.
+static int mc_accumulate_times(const float* g, const float* g_ref, float* S1, float* S2, size_t n, float times,
+                               cudaStream_t st) {
+  if (n % 4 != 0) return BSP_ERR_UNSUPPORTED;
+  if (n == 0) return BSP_OK;
+  const size_t n4 = n / 4;
+  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(g, g_ref, S1, S2, n4, times);
+  BSP_LAUNCH_CHECK();
+  return BSP_OK;
+}
 
 struct AttnCheckBuffers {
   float *o, *lse, *amax, *scales, *d_ref, *d_pol, *d_draws;
@@ -1156,12 +1177,15 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S1[t], 0, n * 4, st));
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S2[t], 0, n * 4, st));
     }
+    // dV does not read the correction term: its value under the fresh read is the same for every
+    // draw, so it is computed with the first draw only and enters the sums K times
     for (int k = 0; k < K; ++k) {
       const float* dk_ = b.d_draws + (size_t)k * rows;
       BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
       BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],
-                                 b.g_pol[1], b.g_pol[2], diag, st));
-      for (int t = 0; t < 3; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
+                                 b.g_pol[1], k == 0 ? b.g_pol[2] : nullptr, diag, st));
+      for (int t = 0; t < 2; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
+      if (k == 0) BSP_TRY(mc_accumulate_times(b.g_pol[2], b.g_ref[2], b.S1[2], b.S2[2], n, (float)K, st));
     }
     BSP_TRY(bsp_mc_stats(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH), b.ws_stats,
                          b.b_stats, st));
