@@ -150,6 +150,18 @@ def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
         outs.append((dq, dk, dv))
     assert all(torch.equal(a, c) for a, c in zip(outs[0], outs[1]))      # byte-identical repeat
     assert torch.equal(outs[0][2], outs[2][2])                             # dV never reads the saved output
+    # the dK-only form of the backward (dV left out, as the draws after the first of a fresh read
+    # use it) gives the same dK bit for bit, and leaves a dV buffer it is not given untouched
+    dterm = torch.zeros(B * H * S, device="cuda")
+    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, None, None, fp8.E4M3, b.READ_ORIGINAL,
+                     b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0), 0, 1, dterm)
+    dk_full, dv_full, dk_only = (torch.zeros(n, device="cuda") for _ in range(3))
+    b.bsp_attn_bwd_dterm(B, H, S, D, g.causal, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, dterm, None,
+                         dk_full, dv_full)
+    b.bsp_attn_bwd_dterm(B, H, S, D, g.causal, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, dterm, None,
+                         dk_only, None)
+    assert torch.equal(dk_full, dk_only)
+    assert torch.equal(dk_full, outs[0][1]) and torch.equal(dv_full, outs[0][2])
     assert not torch.equal(outs[0][0], outs[2][0])                         # dQ does
 
 
