@@ -276,7 +276,51 @@ def kernel_table(b, peaks):
     t("norm_bwd read U: dgamma, dbeta, dx", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 0, codes, q, k, dg, db, dx, ws), T * C * 8)
     t("norm_bwd read R: dgamma", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 1, codes, q, k, dg, None, None, ws), T * C * 5)
     t("mc_stats (45 M elements, fresh)", "hbm", lambda: b.bsp_mc_stats(ref, ref, S2, O * C, 16, 1, wss), O * C * 12)
-    return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"], kernels=rows)
+    # ---- the K-draw kernels and the contractions at the same shape (K = 16 draws, as config 5)
+    Kd = 16
+    qf = b.quant(b.E4M3, b.ROUND_STOCHASTIC, 1.0, scale)
+    qdy = b.quant(b.E5M2, b.ROUND_NEAREST, 100.0)
+    fresh_t = torch.zeros(Kd * C * T, dtype=torch.uint8, device="cuda")
+    S1 = torch.zeros(O * C, device="cuda")
+    diag = b.new_diag()
+    b.bsp_round_2d(dY, T, O, qrn, k, dyc, dyc_t, T)
+    b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, codes_t, T)
+    g1, g2 = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda")
+    wsg = b.workspace(b.bsp_norm_gain_mc_workspace_bytes(T, C, Kd))
+    dW = torch.zeros(O * C, device="cuda")
+    wsw = b.workspace(max(b.bsp_linear_wgrad_workspace_bytes(T, O, C, b.READ_FORWARD), 256))
+    compute = []
+
+    def tc(name, bound, fn, work, unit, peak, reps=5):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        rate = work / (us * 1e-6)
+        compute.append(dict(kernel=name, bound=bound, us=us, achieved=rate / (1e9 if unit == "G element-draws/s" else 1e12),
+                            unit=unit, peak=peak, frac=(rate / (1e9 if unit == "G element-draws/s" else 1e12)) / peak))
+
+    alu_peak = 2650.0       # G element-draws/s: 37.2 T lane-instructions/s over ~14 per element-draw (derived)
+    tc("fresh code matrices, 16 draws (reround_draws)", "alu",
+       lambda: b.bsp_norm_fwd_draws(b.RMSNORM, x, T, C, gamma, None, rstd, mean, qf, b.key(1, 1, 2), 0, Kd, fresh_t, T),
+       float(T) * C * Kd, "G element-draws/s", alu_peak)
+    tc("gain use, 16 draws (gain_mc)", "alu",
+       lambda: b.bsp_norm_gain_mc(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, qf, b.key(1, 1, 1), 0, Kd, dg, g1, g2, wsg, diag),
+       float(T) * C * Kd, "G element-draws/s", alu_peak)
+    tc("weight gradient, read R (gemm_tc fp8)", "tensor",
+       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qdy, b.READ_FORWARD, codes_t, qf, T, dW, ws=wsw, diag=diag),
+       2.0 * T * O * C, "TFLOP/s", 2.0 * peaks["bf16_tflops"])
+    tc("weight gradient, 16 fresh draws with sums (gemm_mc)", "tensor",
+       lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qdy, fresh_t, qf, T, Kd, ref, S1, S2, diag),
+       2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], reps=3)
+    return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
+                kernels=rows, compute_kernels=compute, diag_status=b.read_diag(diag)["status"])
 
 
 def run_ours(args):
