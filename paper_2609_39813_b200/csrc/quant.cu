@@ -250,21 +250,32 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
   }
   if (codes_t || u_bf16_t) {
     __syncthreads();
-    // transposed write: thread -> column tcol, 16 consecutive rows
+    if (codes_t) {
+      // transposed codes: a thread takes a 4 x 4 block (rows 4*rb.., columns 4*g..) as four words,
+      // transposes it with eight byte permutes, and writes one word to each of its four columns;
+      // sixteen neighbouring lanes cover the 64 rows of a column (64 contiguous bytes)
+      const int rb = threadIdx.x & 15, g = threadIdx.x >> 4;
+      const int64_t rr = r0 + 4 * rb, cg = c0 + 4 * g;
+      // rows up to the next multiple of 16 past `rows` are written as zeros (ld_t covers them)
+      if (cg < cols && rr < ((rows + 15) & ~(int64_t)15)) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          w[i] = rr + i < rows ? *reinterpret_cast<const uint32_t*>(&s_codes[4 * rb + i][4 * g]) : 0u;
+        const uint32_t t0 = __byte_perm(w[0], w[1], 0x5140), t1 = __byte_perm(w[2], w[3], 0x5140);
+        const uint32_t t2 = __byte_perm(w[0], w[1], 0x7362), t3 = __byte_perm(w[2], w[3], 0x7362);
+        const uint32_t o[4] = {__byte_perm(t0, t1, 0x5410), __byte_perm(t0, t1, 0x7632),
+                               __byte_perm(t2, t3, 0x5410), __byte_perm(t2, t3, 0x7632)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          *reinterpret_cast<uint32_t*>(codes_t + (size_t)(cg + i) * ld_t + rr) = o[i];
+      }
+    }
+    // transposed bf16 copy: thread -> column tcol, 16 consecutive rows
     const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
     const int64_t cc = c0 + tcol, rr = r0 + trow;
     if (cc < cols && rr < rows) {
       const int nvalid = (int)((rows - rr) < 16 ? (rows - rr) : 16);
-      if (codes_t) {
-        uint32_t pk[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const uint32_t b = j < nvalid ? s_codes[trow + j][tcol] : 0u;
-          pk[j >> 2] |= b << (8 * (j & 3));
-        }
-        // ld_t is a multiple of 16 and >= rows rounded up, so the 16-byte store stays in the row
-        *reinterpret_cast<uint4*>(codes_t + (size_t)cc * ld_t + rr) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      }
       if (u_bf16_t) {
         uint32_t pk[8];
 #pragma unroll
