@@ -182,11 +182,13 @@ __global__ void round_scalar_kernel(const void* __restrict__ x, size_t i_begin, 
 
 // Produces the FP32 value *before scaling* of element (r, c) from the loaded input value.
 struct PlainProducer {
+  static constexpr bool kCopies = false;   // no FP32 / transposed-bf16 copies of the value on this path
   __device__ __forceinline__ void row(int64_t) {}
   __device__ __forceinline__ float value(float xin, int64_t) const { return xin; }
 };
 
 struct NormProducer {
+  static constexpr bool kCopies = true;
   int kind;
   const float* __restrict__ gamma;
   const float* __restrict__ beta;
@@ -214,7 +216,7 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
                   uint8_t* __restrict__ codes_t, int64_t ld_t, float* __restrict__ u_f32,
                   uint16_t* __restrict__ u_bf16_t, bsp_diag_t* diag) {
   __shared__ __align__(16) uint8_t s_codes[kTile][kTile + 4];
-  __shared__ __align__(16) uint16_t s_bf16[kTile][kTile + 2];
+  __shared__ __align__(16) uint16_t s_bf16[Producer::kCopies ? kTile : 1][kTile + 2];
   const int64_t r0 = (int64_t)blockIdx.y * kTile, c0 = (int64_t)blockIdx.x * kTile;
   const int tr = threadIdx.x >> 2, tc = (threadIdx.x & 3) * 16;
   const int64_t r = r0 + tr, c = c0 + tc;
@@ -230,7 +232,7 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
     for (int j = 0; j < 16; ++j) u[j] = prod.value(u[j], c + j);
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(u[j], s);
-    if (u_f32) {
+    if (Producer::kCopies && u_f32) {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
         reinterpret_cast<float4*>(u_f32 + i0)[j] = make_float4(u[4 * j], u[4 * j + 1], u[4 * j + 2], u[4 * j + 3]);
@@ -243,12 +245,12 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
         dst[0] = pk.x; dst[1] = pk.y; dst[2] = pk.z; dst[3] = pk.w;
       }
     }
-    if (u_bf16_t) {
+    if (Producer::kCopies && u_bf16_t) {
 #pragma unroll
       for (int j = 0; j < 16; ++j) s_bf16[tr][tc + j] = (uint16_t)float_to_bf16_bits(u[j]);
     }
   }
-  if (codes_t || u_bf16_t) {
+  if (codes_t || (Producer::kCopies && u_bf16_t)) {
     __syncthreads();
     if (codes_t) {
       // transposed codes: a thread takes a 4 x 4 block (rows 4*rb.., columns 4*g..) as four words,
@@ -276,7 +278,7 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
     const int64_t cc = c0 + tcol, rr = r0 + trow;
     if (cc < cols && rr < rows) {
       const int nvalid = (int)((rows - rr) < 16 ? (rows - rr) : 16);
-      if (u_bf16_t) {
+      if (Producer::kCopies && u_bf16_t) {
         uint32_t pk[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
