@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <vector>
 
 #include "common.cuh"
 
@@ -83,6 +84,61 @@ mc_stats_kernel(const float* __restrict__ g_ref, const float* __restrict__ g, co
   }
 }
 
+constexpr size_t kStatSlotDoubles = (size_t)kStatBlocks * kStatFields;
+
+// Launches the statistics pass over n elements into one slot of block partials; returns the number
+// of blocks whose partials the slot then holds.
+static int mc_stats_launch(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
+                           double* partials, cudaStream_t st, int* blocks_out) {
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > kStatBlocks) blocks = kStatBlocks;
+  *blocks_out = blocks;
+  if (blocks > 0) {
+    mc_stats_kernel<<<blocks, 256, 0, st>>>(g_ref, g, S2, n, K, fresh, partials);
+    BSP_LAUNCH_CHECK();
+  }
+  return BSP_OK;
+}
+
+// Sums a slot's block partials on the host, in block order, and fills the result of the use.
+static void mc_stats_finish(const double* host, int blocks, int64_t n, int K, int fresh, bsp_use_result_t* result) {
+  double f[kStatFields] = {0, 0, 0, 0, 0, 0, 0, 0};
+  for (int b = 0; b < blocks; ++b)
+    for (int j = 0; j < kStatFields; ++j)
+      f[j] = j == 5 ? fmax(f[j], host[b * kStatFields + j]) : f[j] + host[b * kStatFields + j];
+  const double num = sqrt(f[0]), den = sqrt(f[1]);
+  result->n_elements = n;
+  result->rel_l2_mean_err = num == 0.0 ? 0.0 : (den > 0.0 ? num / den : INFINITY);
+  result->reserved = 0;
+  if (!fresh) {
+    result->K = 1;
+    result->R = result->Qprime = result->mean_z = result->rms_z = result->max_abs_z = result->frac_abs_z_gt3 = 0.0;
+    result->verdict = result->rel_l2_mean_err <= 1e-4 ? BSP_HOLDS : BSP_FAILS;
+    return;
+  }
+  const double nn = n > 0 ? (double)n : 1.0;
+  result->K = K;
+  result->R = f[0] == 0.0 ? 0.0 : (f[2] > 0.0 ? f[0] / f[2] : INFINITY);
+  result->Qprime = f[3] / nn * (double)(K - 3) / (double)(K - 1);
+  result->mean_z = f[4] / nn;
+  result->rms_z = sqrt(f[3] / nn);
+  result->max_abs_z = f[5];
+  result->frac_abs_z_gt3 = f[6] / nn;
+  if (result->Qprime >= 4.0 || result->R >= 6.0) result->verdict = BSP_FAILS;
+  else if (result->Qprime <= 2.0 && result->R <= 3.0) result->verdict = BSP_HOLDS;
+  else result->verdict = BSP_UNDECIDED;
+}
+
+// The statistics passes of one check: each is launched into its own slot of partials as soon as its
+// inputs are queued, and all of them are brought to the host behind one synchronisation at the end.
+constexpr int kCheckStatSlots = 6;
+struct PendingStats {
+  bsp_use_result_t* result[kCheckStatSlots];
+  int blocks[kCheckStatSlots], K[kCheckStatSlots], fresh[kCheckStatSlots];
+  int64_t n[kCheckStatSlots];
+  int count = 0;
+};
+
 struct Bump {
   char* base;
   size_t off;
@@ -140,7 +196,7 @@ static size_t carve(const bsp_norm_linear_desc_t* op, int K, char* base, CheckBu
   c.b_gain = bsp_norm_gain_mc_workspace_bytes(op->T, op->C, K > 0 ? K : 1);
   c.b_wgrad = bsp_linear_wgrad_workspace_bytes(op->T, op->O, op->C, BSP_READ_ORIGINAL);
   c.b_dgrad = bsp_linear_dgrad_workspace_bytes(op->T, op->O, op->C);
-  c.b_stats = bsp_mc_stats_workspace_bytes((int64_t)(O * C > C ? O * C : C));
+  c.b_stats = kCheckStatSlots * bsp_mc_stats_workspace_bytes((int64_t)(O * C > C ? O * C : C));
   c.ws_bwd = b.take(c.b_bwd); c.ws_gain = b.take(c.b_gain); c.ws_wgrad = b.take(c.b_wgrad);
   c.ws_dgrad = b.take(c.b_dgrad); c.ws_stats = b.take(c.b_stats);
   if (cb) *cb = c;
@@ -183,41 +239,15 @@ int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n,
     return BSP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   double* partials = reinterpret_cast<double*>(ws);
-  int blocks = (int)((n + 255) / 256);
-  if (blocks > kStatBlocks) blocks = kStatBlocks;
-  double host[kStatBlocks * kStatFields];
-  double f[kStatFields] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (blocks > 0) {
-    mc_stats_kernel<<<blocks, 256, 0, st>>>(g_ref, g, S2, n, K, fresh, partials);
-    BSP_LAUNCH_CHECK();
+  int blocks = 0;
+  int rc = mc_stats_launch(g_ref, g, S2, n, K, fresh, partials, st, &blocks);
+  if (rc != BSP_OK) return rc;
+  double host[kStatSlotDoubles];
+  if (blocks > 0)
     BSP_CHECK_CUDA(cudaMemcpyAsync(host, partials, (size_t)blocks * kStatFields * sizeof(double),
                                    cudaMemcpyDeviceToHost, st));
-  }
   BSP_CHECK_CUDA(cudaStreamSynchronize(st));
-  for (int b = 0; b < blocks; ++b)
-    for (int j = 0; j < kStatFields; ++j)
-      f[j] = j == 5 ? fmax(f[j], host[b * kStatFields + j]) : f[j] + host[b * kStatFields + j];
-  const double num = sqrt(f[0]), den = sqrt(f[1]);
-  result->n_elements = n;
-  result->rel_l2_mean_err = num == 0.0 ? 0.0 : (den > 0.0 ? num / den : INFINITY);
-  result->reserved = 0;
-  if (!fresh) {
-    result->K = 1;
-    result->R = result->Qprime = result->mean_z = result->rms_z = result->max_abs_z = result->frac_abs_z_gt3 = 0.0;
-    result->verdict = result->rel_l2_mean_err <= 1e-4 ? BSP_HOLDS : BSP_FAILS;
-    return BSP_OK;
-  }
-  const double nn = n > 0 ? (double)n : 1.0;
-  result->K = K;
-  result->R = f[0] == 0.0 ? 0.0 : (f[2] > 0.0 ? f[0] / f[2] : INFINITY);
-  result->Qprime = f[3] / nn * (double)(K - 3) / (double)(K - 1);
-  result->mean_z = f[4] / nn;
-  result->rms_z = sqrt(f[3] / nn);
-  result->max_abs_z = f[5];
-  result->frac_abs_z_gt3 = f[6] / nn;
-  if (result->Qprime >= 4.0 || result->R >= 6.0) result->verdict = BSP_FAILS;
-  else if (result->Qprime <= 2.0 && result->R <= 3.0) result->verdict = BSP_HOLDS;
-  else result->verdict = BSP_UNDECIDED;
+  mc_stats_finish(host, blocks, n, K, fresh, result);
   return BSP_OK;
 }
 
@@ -268,6 +298,14 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
   BSP_TRY(bsp_round_2d(op->dY, dt, T, O, qdy, nokey, b.dy_codes, b.dy_codes_t, b.ld_t, diag, st));
   BSP_TRY(bsp_linear_dgrad(T, O, C, b.dy_codes, qdy, op->W, dt, b.du, dt, b.ws_dgrad, b.b_dgrad, diag, st));
 
+  PendingStats pend;
+  auto stats = [&](const float* g_ref, const float* g, const float* S2, int64_t n, int Kd, int fresh,
+                   bsp_use_result_t* r) -> int {
+    const int slot = pend.count++;
+    pend.result[slot] = r; pend.n[slot] = n; pend.K[slot] = Kd; pend.fresh[slot] = fresh;
+    return mc_stats_launch(g_ref, g, S2, n, Kd, fresh, reinterpret_cast<double*>(b.ws_stats) + slot * kStatSlotDoubles,
+                           st, &pend.blocks[slot]);
+  };
   int nres = 0;
   auto emit = [&](int use, int out, int pol) -> bsp_use_result_t* {
     bsp_use_result_t* r = &results[nres++];
@@ -284,14 +322,14 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
                          BSP_READ_ORIGINAL, nullptr, qu, key, b.dg_ref, b.db_ref, b.dx, b.ws_bwd, b.b_bwd, diag, st));
     if (gain_mask & 1u) {
       bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_ORIGINAL);
-      BSP_TRY(bsp_mc_stats(b.dg_ref, b.dg_ref, nullptr, C, 1, 0, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dg_ref, b.dg_ref, nullptr, C, 1, 0, r));
     }
     if (gain_mask & 2u) {
       BSP_TRY(bsp_norm_bwd(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt,
                            BSP_READ_FORWARD, b.u_codes, qu, key, b.dg_pol, nullptr, nullptr, b.ws_bwd, b.b_bwd,
                            diag, st));
       bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FORWARD);
-      BSP_TRY(bsp_mc_stats(b.dg_ref, b.dg_pol, nullptr, C, 1, 0, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dg_ref, b.dg_pol, nullptr, C, 1, 0, r));
     }
     if (gain_mask & 4u) {
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S1g, 0, C * sizeof(float), st));
@@ -299,7 +337,7 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
       BSP_TRY(bsp_norm_gain_mc(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt, qu,
                                key, 0, K, b.dg_ref, b.S1g, b.S2g, b.ws_gain, b.b_gain, diag, st));
       bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FRESH);
-      BSP_TRY(bsp_mc_stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, r));
     }
   }
 
@@ -312,11 +350,11 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
       BSP_TRY(bsp_linear_wgrad(T, O, C, b.dy_codes_t, qdy, BSP_READ_ORIGINAL, b.u_bf16_t, qu, b.ld_t, b.dW_pol,
                                nullptr, nullptr, nullptr, b.ws_wgrad, b.b_wgrad, diag, st));
       bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_ORIGINAL);
-      BSP_TRY(bsp_mc_stats(b.dW_ref, b.dW_pol, nullptr, O * C, 1, 0, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dW_ref, b.dW_pol, nullptr, O * C, 1, 0, r));
     }
     if (w_mask & 2u) {
       bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FORWARD);
-      BSP_TRY(bsp_mc_stats(b.dW_ref, b.dW_ref, nullptr, O * C, 1, 0, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dW_ref, b.dW_ref, nullptr, O * C, 1, 0, r));
     }
     if (w_mask & 4u) {
       float* S1w = b.dW_pol;   // the U result has been reduced already
@@ -337,11 +375,18 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
                                     st));
       }
       bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FRESH);
-      BSP_TRY(bsp_mc_stats(b.dW_ref, S1w, b.S2w, O * C, K, 1, r, b.ws_stats, b.b_stats, st));
+      BSP_TRY(stats(b.dW_ref, S1w, b.S2w, O * C, K, 1, r));
     }
   }
   *n_results = nres;
+  std::vector<double> host((size_t)(pend.count > 0 ? pend.count : 1) * kStatSlotDoubles);
+  if (pend.count > 0)
+    BSP_CHECK_CUDA(cudaMemcpyAsync(host.data(), b.ws_stats, (size_t)pend.count * kStatSlotDoubles * sizeof(double),
+                                   cudaMemcpyDeviceToHost, st));
   BSP_CHECK_CUDA(cudaStreamSynchronize(st));
+  for (int i = 0; i < pend.count; ++i)
+    mc_stats_finish(host.data() + (size_t)i * kStatSlotDoubles, pend.blocks[i], pend.n[i], pend.K[i], pend.fresh[i],
+                    pend.result[i]);
   return BSP_OK;
 }
 
