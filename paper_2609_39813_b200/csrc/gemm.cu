@@ -750,13 +750,21 @@ int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, b
   else
     decode_to_bf16_kernel<BSP_E4M3><<<(unsigned)((n16 + 255) / 256), 256, 0, st>>>(dy_codes, n16, dyb);
   BSP_LAUNCH_CHECK();
-  dim3 tg((unsigned)((C + 31) / 32), (unsigned)((O + 31) / 32));
-  if (w_dt == BSP_F32) to_bf16_transpose_kernel<BSP_F32><<<tg, 256, 0, st>>>(W, O, C, wt, O);
-  else to_bf16_transpose_kernel<BSP_BF16><<<tg, 256, 0, st>>>(W, O, C, wt, O);
-  BSP_LAUNCH_CHECK();
+  // W [O][C] is the B operand with the contraction index outermost: a bf16 W is read in place as
+  // an MN-major operand; an FP32 W (or a C that breaks the 16-byte pitch) goes through a bf16
+  // transposed copy
+  const bool w_in_place = w_dt == BSP_BF16 && C % 8 == 0 && aligned16(W) && !simt_forced();
+  if (!w_in_place) {
+    dim3 tg((unsigned)((C + 31) / 32), (unsigned)((O + 31) / 32));
+    if (w_dt == BSP_F32) to_bf16_transpose_kernel<BSP_F32><<<tg, 256, 0, st>>>(W, O, C, wt, O);
+    else to_bf16_transpose_kernel<BSP_BF16><<<tg, 256, 0, st>>>(W, O, C, wt, O);
+    BSP_LAUNCH_CHECK();
+  }
   GemmArgs g;
   g.M = T; g.N = C; g.K = O; g.nb = 1; g.fp8 = false; g.a_fmt = 0; g.b_fmt = 0;
-  g.A = dyb; g.B = wt; g.lda = O; g.ldb = O; g.b_batch_stride = (int64_t)C * O;
+  g.A = dyb; g.lda = O;
+  if (w_in_place) { g.B = W; g.b_mn = true; g.ldb = C; g.b_batch_stride = (int64_t)O * C; }
+  else { g.B = wt; g.ldb = O; g.b_batch_stride = (int64_t)C * O; }
   g.sa = q_dy.scale; g.sa_dev = q_dy.scale_dev; g.sb = 1.0f; g.sb_dev = nullptr;
   g.mode = du_dt == BSP_F32 ? EPI_STORE_F32 : EPI_STORE_BF16;
   g.C = du; g.ldc = C; g.ref = nullptr; g.S1 = nullptr; g.S2 = nullptr; g.diag = diag;
