@@ -51,6 +51,9 @@ struct AttnParams {
   float* out0;                   // DKV: dV   DQ: dQ   FWD: O      [BH*S*64]
   float* out1;                   // DKV: dK                         [BH*S*64]
   float* lse_out;                // FWD
+  // Monte-Carlo epilogue (DQ, and DKV without dV): instead of storing the gradient g, the kernel adds
+  // g - mc_ref to out0 and (g - mc_ref)^2 to out1 (the running sums S1, S2 of that gradient)
+  const float* mc_ref;           // [BH*S*64] or NULL
   bsp_diag_t* diag;
   // FP8-operand mode: q, k, v, dO hold decoded FP8 codes (exact in bf16); their per-(b,h) scales
   // are folded into the softmax argument, dP and the outputs; P and dS are rounded onto the E4M3 /
@@ -99,7 +102,9 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 // template parameter because its tests and extra multiplications sit in the innermost loop.
 // DV (dK/dV mode only): false leaves dV out (its product, the P operand and its store): dV does
 // not read the correction term, so the draws of a fresh read need it once, not K times.
-template <int MODE, bool FP8, bool DV>
+// MC: the Monte-Carlo epilogue (see AttnParams::mc_ref); a template parameter so that the plain
+// kernels carry none of its registers.
+template <int MODE, bool FP8, bool DV, bool MC>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -636,6 +641,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // time through the item's resident-tile buffer (no product reads it any more): every thread puts
     // its row's 32 FP32 values of column half h into the 128-byte-swizzle box that a tiled bulk store
     // then writes (whole 128-byte lines; rows beyond the sequence are clipped by the store).
+    constexpr bool mc = MC;
+    float rv[32];                                             // Monte-Carlo epilogue: the reference values of this thread's 32 outputs
+    if (mc) {
+      const int orow = blk * AT_BLK + r;
+      const float4* rp = reinterpret_cast<const float4*>(p.mc_ref + ((size_t)bh * p.S + (orow < p.S ? orow : 0)) * AT_D + h * 32);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const float4 v4 = __ldg(rp + t);
+        rv[4 * t] = v4.x; rv[4 * t + 1] = v4.y; rv[4 * t + 2] = v4.z; rv[4 * t + 3] = v4.w;
+      }
+    }
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc + 8 * ab, iph, abort_flag));
     if (ok) {
       tc_fence_after();
@@ -647,7 +663,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         mbar_arrive(b_res_empty + 8 * (rbi ^ 1u));
         store_pending = false;
       }
-      if (MODE == AT_DKV) named_bar_sync(3, 256);             // ... before anyone writes the second staging buffer again
+      if (MODE == AT_DKV || mc) named_bar_sync(3, 256);       // ... before anyone writes the second staging buffer again
 #pragma unroll
       for (int o = (MODE == AT_DKV && !DV) ? 1 : 0; o < nout; ++o) {
         const uint32_t stg = o == 0 ? res_base + rbi * 2 * kAtTile : stage2;
@@ -663,6 +679,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           __syncwarp();
           if (lane == 0) mbar_arrive(b_acc_free + 8 * ab);
         }
+        if (mc) {
+          // g - ref into this output's staging buffer, its square into the other one
+          const uint32_t stg2 = o == 0 ? stage2 : res_base + rbi * 2 * kAtTile;
+#pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+            const float d0 = __uint_as_float(a[4 * t]) * mul - rv[4 * t], d1 = __uint_as_float(a[4 * t + 1]) * mul - rv[4 * t + 1];
+            const float d2 = __uint_as_float(a[4 * t + 2]) * mul - rv[4 * t + 2], d3 = __uint_as_float(a[4 * t + 3]) * mul - rv[4 * t + 3];
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(d0), "f"(d1), "f"(d2), "f"(d3) : "memory");
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg2 + off), "f"(d0 * d0), "f"(d1 * d1), "f"(d2 * d2),
+                         "f"(d3 * d3) : "memory");
+          }
+          continue;
+        }
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
           const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
@@ -676,13 +706,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (warp == kAtSoftWarp0 && lane == 0) {
         // issue the stores and go on: their completion is only needed before the staging buffers are
         // written again (next epilogue) or handed back (after the next item's first step)
-        if (MODE != AT_DKV || DV) {
-          tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
-          tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile + 16384u, 32, blk * AT_BLK, bh);
-        }
-        if (MODE == AT_DKV) {
-          tma_store_3d(&tm_o1, stage2, 0, blk * AT_BLK, bh);
-          tma_store_3d(&tm_o1, stage2 + 16384u, 32, blk * AT_BLK, bh);
+        if (mc) {
+          // S1 += g - ref, S2 += (g - ref)^2: each element of the sums is added to once per launch
+          const uint32_t sx = MODE == AT_DKV ? stage2 : res_base + rbi * 2 * kAtTile;
+          const uint32_t sy = MODE == AT_DKV ? res_base + rbi * 2 * kAtTile : stage2;
+          tma_reduce_add_3d(&tm_o0, sx, 0, blk * AT_BLK, bh);
+          tma_reduce_add_3d(&tm_o0, sx + 16384u, 32, blk * AT_BLK, bh);
+          tma_reduce_add_3d(&tm_o1, sy, 0, blk * AT_BLK, bh);
+          tma_reduce_add_3d(&tm_o1, sy + 16384u, 32, blk * AT_BLK, bh);
+        } else {
+          if (MODE != AT_DKV || DV) {
+            tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile, 0, blk * AT_BLK, bh);
+            tma_store_3d(&tm_o0, res_base + rbi * 2 * kAtTile + 16384u, 32, blk * AT_BLK, bh);
+          }
+          if (MODE == AT_DKV) {
+            tma_store_3d(&tm_o1, stage2, 0, blk * AT_BLK, bh);
+            tma_store_3d(&tm_o1, stage2 + 16384u, 32, blk * AT_BLK, bh);
+          }
         }
         tma_store_commit();
         store_pending = true;
@@ -796,7 +836,7 @@ static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
 }
 
-template <int MODE, bool FP8, bool DV>
+template <int MODE, bool FP8, bool DV, bool MC = false>
 static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mdo, mo0, mo1;
   int rc;
@@ -808,7 +848,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
   static bool attr_set = false;
   if (!attr_set) {
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
@@ -818,13 +858,17 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE, FP8, DV><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
+  attn_kernel<MODE, FP8, DV, MC><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
 
 template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
+  if (MODE != AT_FWD && p.mc_ref != nullptr) {               // Monte-Carlo epilogue: BF16 operands, no dV
+    if (p.fp8) return BSP_ERR_UNSUPPORTED;
+    return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD>(q, k, v, dO, p, st);
+  }
   if (MODE == AT_DKV && p.out0 == nullptr)                   // dK only
     return p.fp8 ? launch_attn_mode<MODE, true, false>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false, false>(q, k, v, dO, p, st);
   return p.fp8 ? launch_attn_mode<MODE, true, true>(q, k, v, dO, p, st) : launch_attn_mode<MODE, false, true>(q, k, v, dO, p, st);
@@ -858,7 +902,7 @@ static int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag;
+  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
 }
@@ -935,7 +979,7 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
     return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag;
+  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag; p.mc_ref = nullptr;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   if (dk) {
@@ -947,6 +991,29 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
     if ((rc = launch_attn<AT_DQ>(q, k, v, dO, p, st)) != BSP_OK) return rc;
   }
   return BSP_OK;
+}
+
+// One fresh draw of the D use for dQ and dK with the Monte-Carlo epilogue: the two kernels add
+// g - ref and its square to the running sums of their gradient and write no gradient (BF16-operand
+// mode; dV is not computed).  The sums must not be touched by anything else while this runs.
+static int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                             const void* k, const void* v, const void* dO, int dt, const float* lse,
+                             const float* dterm, const float* ref_dq, float* S1q, float* S2q, const float* ref_dk,
+                             float* S1k, float* S2k, bsp_diag_t* diag, void* stream) {
+  int rc = check_attn_shape(B, H, S, Dh, dt);
+  if (rc != BSP_OK) return rc;
+  if (!q || !k || !v || !dO || !lse || !dterm || !ref_dq || !S1q || !S2q || !ref_dk || !S1k || !S2k) return BSP_ERR_ARG;
+  if (!aligned16(ref_dq) || !aligned16(ref_dk) || !aligned16(S1q) || !aligned16(S2q) || !aligned16(S1k) || !aligned16(S2k))
+    return BSP_ERR_ALIGN;
+  AttnParams p;
+  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
+  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag;
+  if ((rc = set_fp8(p, nullptr)) != BSP_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  p.mc_ref = ref_dk; p.out0 = S1k; p.out1 = S2k;
+  if ((rc = launch_attn<AT_DKV>(q, k, v, dO, p, st)) != BSP_OK) return rc;
+  p.mc_ref = ref_dq; p.out0 = S1q; p.out1 = S2q;
+  return launch_attn<AT_DQ>(q, k, v, dO, p, st);
 }
 
 // x (bf16 [groups][group_size]) -> nearest FP8 codes at each group's own amax scale -> the decoded
@@ -1182,10 +1249,16 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
     for (int k = 0; k < K; ++k) {
       const float* dk_ = b.d_draws + (size_t)k * rows;
       BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
+      if (k > 0) {
+        // the draws after the first: dQ and dK go from the accumulators straight into their sums
+        BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_ref[0],
+                                  b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
+        continue;
+      }
       BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],
-                                 b.g_pol[1], k == 0 ? b.g_pol[2] : nullptr, diag, st));
+                                 b.g_pol[1], b.g_pol[2], diag, st));
       for (int t = 0; t < 2; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
-      if (k == 0) BSP_TRY(mc_accumulate_times(b.g_pol[2], b.g_ref[2], b.S1[2], b.S2[2], n, (float)K, st));
+      BSP_TRY(mc_accumulate_times(b.g_pol[2], b.g_ref[2], b.S1[2], b.S2[2], n, (float)K, st));
     }
     BSP_TRY(bsp_mc_stats(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH), b.ws_stats,
                          b.b_stats, st));
