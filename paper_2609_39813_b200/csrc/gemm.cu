@@ -48,6 +48,21 @@ struct GemmParams {
   bsp_diag_t* diag;
 };
 
+// Tile t of the persistent walk -> (tm, tn).  The tile columns are taken in bands of kBandTiles: inside
+// a band the walk is row-major, so the CTAs of one wave (consecutive t) cover about 148 / 8 tile rows
+// by 8 tile columns, and the A and B panels they stream together stay within L2 (for a wide N, a
+// plain row-major walk has every CTA of a wave on its own B panel: 32 panels of 2 MB per draw at
+// T = 16384).  With at most kBandTiles tile columns this is the plain row-major order.
+constexpr int kBandTiles = 8;
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_band = kBandTiles * tiles_m;
+  const int band = t / per_band, idx = t - band * per_band;
+  const int c0 = band * kBandTiles;
+  const int wb = tiles_n - c0 < kBandTiles ? tiles_n - c0 : kBandTiles;
+  tm = idx / wb;
+  tn = c0 + idx - tm * wb;
+}
+
 template <bool FP8>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
@@ -88,7 +103,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        const int tm = t / tiles_n, tn = t % tiles_n;
+        int tm, tn;
+      tile_coords(t, tiles_m, tiles_n, tm, tn);
         for (int b = 0; b < p.nb && ok; ++b) {
           for (int kb = 0; kb < kblocks; ++kb, ++it) {
             const uint32_t s = it % kStages, ph = (it / kStages) & 1u;
@@ -158,7 +174,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t tc = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-      const int tm = t / tiles_n, tn = t % tiles_n;
+      int tm, tn;
+      tile_coords(t, tiles_m, tiles_n, tm, tn);
       const int row = tm * BM + q * 32 + lane;
       for (int b = 0; b < p.nb && ok; ++b, ++tc) {
         const uint32_t as = tc & 1u, aph = (tc >> 1) & 1u;
@@ -275,7 +292,8 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-        const int tm = t / tiles_n, tn = t % tiles_n;
+        int tm, tn;
+      tile_coords(t, tiles_m, tiles_n, tm, tn);
         for (int b = 0; b < p.nb && ok; b += 2) {
           const bool two = b + 1 < p.nb;                       // an odd count ends with a single draw
           for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -330,7 +348,8 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t tc = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-      const int tm = t / tiles_n, tn = t % tiles_n;
+      int tm, tn;
+      tile_coords(t, tiles_m, tiles_n, tm, tn);
       const int row = tm * BM + q * 32 + lane;
       const int colbase = tn * MC_BN + h * 64;
       float refv[64];

@@ -10,15 +10,24 @@ namespace bsp {
 
 // ------------------------------------------------------------------------------- philox fill
 
-__global__ void philox_fill_kernel(PhiloxKey key, size_t n, uint32_t* __restrict__ out) {
-  const size_t q = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const size_t i = q * 4;
-  if (i >= n) return;
-  const uint4 w = philox_block(key, q, key.c2);
-  if (i + 4 <= n) {
-    reinterpret_cast<uint4*>(out)[q] = w;
-  } else {
-    for (uint32_t l = 0; i + l < n; ++l) out[i + l] = word_of(w, l);
+// Four generator blocks per thread, a warp's 16-byte stores contiguous: the four chains of dependent
+// multiplies overlap, which is what the draw kernels also rely on.
+__global__ void __launch_bounds__(256)
+philox_fill_kernel(PhiloxKey key, size_t n, uint32_t* __restrict__ out) {
+  const size_t nq = (n + 3) / 4;
+  const size_t q0 = (size_t)blockIdx.x * (blockDim.x * 4) + threadIdx.x;
+  uint4 w[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) w[j] = philox_block(key, q0 + (size_t)j * blockDim.x, key.c2);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const size_t q = q0 + (size_t)j * blockDim.x, i = q * 4;
+    if (q >= nq) continue;
+    if (i + 4 <= n) {
+      reinterpret_cast<uint4*>(out)[q] = w[j];
+    } else {
+      for (uint32_t l = 0; i + l < n; ++l) out[i + l] = word_of(w[j], l);
+    }
   }
 }
 
@@ -536,7 +545,7 @@ int bsp_philox_fill(bsp_key_t key, size_t n, uint32_t* out, void* stream) {
   if (!aligned16(out)) return BSP_ERR_ALIGN;
   if (n == 0) return BSP_OK;
   const size_t nq = (n + 3) / 4;
-  philox_fill_kernel<<<(unsigned)((nq + 255) / 256), 256, 0, (cudaStream_t)stream>>>(make_key(key), n, out);
+  philox_fill_kernel<<<(unsigned)((nq + 1023) / 1024), 256, 0, (cudaStream_t)stream>>>(make_key(key), n, out);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
