@@ -326,6 +326,21 @@ def kernel_table(b, peaks):
     tc("weight gradient, read R (gemm_tc fp8)", "tensor",
        lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qdy, b.READ_FORWARD, codes_t, qf, T, dW, ws=wsw, diag=diag),
        2.0 * T * O * C, "TFLOP/s", 2.0 * peaks["bf16_tflops"])
+    # the two BF16 contractions of the path: the weight gradient reading the original u, and the
+    # incoming-gradient helper du = dY W (decoded dY codes; a bf16 W is read in place)
+    u_bf16_t = torch.zeros(C * T, dtype=torch.bfloat16, device="cuda")
+    b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, codes_t, T, None, u_bf16_t)
+    wsu = b.workspace(max(b.bsp_linear_wgrad_workspace_bytes(T, O, C, b.READ_ORIGINAL), 256))
+    tc("weight gradient, read U (decode + gemm_tc bf16)", "tensor",
+       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qdy, b.READ_ORIGINAL, u_bf16_t, qf, T, dW, ws=wsu, diag=diag),
+       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"])
+    Wb = (torch.randn(O * C, device="cuda") / 64).to(torch.bfloat16)
+    du_out = torch.zeros(T * C, dtype=torch.bfloat16, device="cuda")
+    wsd = b.workspace(b.bsp_linear_dgrad_workspace_bytes(T, O, C))
+    tc("incoming gradient du = dY W (decode + gemm_tc bf16)", "tensor",
+       lambda: b.bsp_linear_dgrad(T, O, C, dyc, qdy, Wb, du_out, wsd, diag),
+       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"])
+    del u_bf16_t, Wb, du_out, wsu, wsd
     tc("weight gradient, 16 fresh draws with sums (gemm_mc)", "tensor",
        lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qdy, fresh_t, qf, T, Kd, ref, S1, S2, diag),
        2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], reps=3)
