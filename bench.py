@@ -344,8 +344,31 @@ def kernel_table(b, peaks):
     tc("weight gradient, 16 fresh draws with sums (gemm_mc)", "tensor",
        lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qdy, fresh_t, qf, T, Kd, ref, S1, S2, diag),
        2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], reps=3)
+    # ---- the whole per-use check at this shape (K = 16, all six evaluations), as one call
+    del fresh_t, dyc, dyc_t, codes, codes_t, dx, du, dW, S1, S2, ref
+    torch.cuda.empty_cache()
+    Wc = (torch.randn(O * C, device="cuda", generator=gen) / 64).to(torch.bfloat16)
+    d = b.NormLinearDesc()
+    d.norm_kind, d.dtype = b.RMSNORM, b.BF16
+    d.T, d.C, d.O = T, C, O
+    d.x, d.gamma, d.beta, d.W, d.dY = b.ptr(x), b.ptr(gamma), None, b.ptr(Wc), b.ptr(dY)
+    d.eps = 1e-6
+    d.store_fmt, d.grad_fmt, d.forward_mode = b.E4M3, b.E5M2, b.ROUND_STOCHASTIC
+    d.seed, d.tensor_id, d.policy_mask = 1005, 1, 0x3F
+    wsc = b.workspace(b.bsp_mc_check_workspace_bytes(d, Kd))
+    for _ in range(2):
+        res = b.bsp_mc_check(d, Kd, wsc, diag)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(3):
+        res = b.bsp_mc_check(d, Kd, wsc, diag)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 3
+    whole = dict(K=Kd, ms_per_check=ms, check_elements_per_s=check_elements(T, C, Kd) / (ms * 1e-3),
+                 verdicts=[int(r.verdict) for r in res])
     return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
-                kernels=rows, compute_kernels=compute, diag_status=b.read_diag(diag)["status"])
+                kernels=rows, compute_kernels=compute, whole_check=whole, diag_status=b.read_diag(diag)["status"])
 
 
 def run_ours(args):
