@@ -54,6 +54,7 @@ struct AttnParams {
   // Monte-Carlo epilogue (DQ, and DKV without dV): instead of storing the gradient g, the kernel adds
   // g - mc_ref to out0 and (g - mc_ref)^2 to out1 (the running sums S1, S2 of that gradient)
   const float* mc_ref;           // [BH*S*64] or NULL
+  int nd;                        // draws per launch (1; 2 in the Monte-Carlo dQ kernel: dterm holds [2][BH*S])
   bsp_diag_t* diag;
   // FP8-operand mode: q, k, v, dO hold decoded FP8 codes (exact in bf16); their per-(b,h) scales
   // are folded into the softmax argument, dP and the outputs; P and dS are rounded onto the E4M3 /
@@ -104,7 +105,10 @@ __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[3
 // not read the correction term, so the draws of a fresh read need it once, not K times.
 // MC: the Monte-Carlo epilogue (see AttnParams::mc_ref); a template parameter so that the plain
 // kernels carry none of its registers.
-template <int MODE, bool FP8, bool DV, bool MC>
+// ND (Monte-Carlo dQ and dK kernels only): draws per launch.  S, dP and P do not depend on the correction
+// term, so with ND = 2 a step forms them once and builds two dS operands, one per draw's D (at
+// p.dterm and p.dterm + BH*S), into two accumulators; the epilogue adds both draws to the sums.
+template <int MODE, bool FP8, bool DV, bool MC, int ND>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -142,6 +146,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // groups 256 bytes apart, the two 8-element halves of a row 128 bytes apart, 16 bytes per row.
   const uint32_t b_bias = bars + 2240;                       // three barriers, one per buffer
   const uint32_t bias0 = bars + 4096;                        // ones tile; buffer b: X_lse at 1 + 2b, X_d at 2 + 2b
+
+  // dK kernel with two draws: the extra product step carries the first draw's -D; the second draw
+  // needs, per query (a column of S^T), delta = D_first - D_second, kept as FP32 in three buffers of
+  // 128 values that the threads writing the X tiles fill alongside them
+  const uint32_t delta0 = bars + 2304;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Persistent CTA: work items w = item_at(0), item_at(1), ... of nblk * BH, heavy blocks first
@@ -191,6 +200,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // bf16 operands P and dS as the softmax warps write them back (64 columns each: two elements per
   // column) at [256,320) and [320,384), and one accumulator buffer of two 64-column halves at 384.
   const uint32_t t_s = tmem, t_dp = tmem + 128, t_p = tmem + 256, t_ds = tmem + 320;
+  // two draws (dQ kernel): the second draw's dS operand takes the P columns (no product reads P
+  // there) and its accumulator the second half of the accumulator buffer
+  const uint32_t t_ds2 = tmem + 256;
   const uint32_t t_accbase = MODE == AT_FWD ? tmem + 256 : tmem + 384;
   constexpr bool kAccDouble = MODE == AT_FWD;   // accumulators double-buffered across items
 
@@ -313,11 +325,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
 #pragma unroll
           for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
+          if (ND == 2 && !DV) {
+            // second draw: its dS^T operand sits in the P columns, its dK in the dV accumulator
+#pragma unroll
+            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_ds2 + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
+          }
         } else if (MODE == AT_DQ) {
           // dQ += dS K : A from tensor memory (row = query, eight columns per 16 keys), B MN-major = streamed K
           const uint64_t bk = make_smem_desc_mn(st0, 16384u);
 #pragma unroll
           for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_ds + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
+          if (ND == 2) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
+          }
         } else if (pass2) {
           // O += P V : A K-major from the P buffer in shared memory, B MN-major = streamed V
           const uint64_t bk = make_smem_desc_mn(st1, 16384u);
@@ -388,8 +409,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int q = step * AT_BLK + (ts & 127);
       return __ldg(bias_src + (size_t)tbh * p.S + (q < p.S ? q : 0));
     };
-    auto bias_put = [&](int step, uint32_t jt, float raw, float mul) {
+    // the second draw's correction term of the same query (threads of the D tile only)
+    auto bias_fetch2 = [&](int tbh, int step) -> float {
+      if (ND != 2 || ts < 128) return 0.f;
+      const int q = step * AT_BLK + (ts & 127);
+      return __ldg(p.dterm + (size_t)p.BH * p.S + (size_t)tbh * p.S + (q < p.S ? q : 0));
+    };
+    auto bias_put = [&](int step, uint32_t jt, float raw, float mul, float raw2) {
       const int q = ts & 127;
+      if (ND == 2 && ts >= 128) {
+        const float dl = step * AT_BLK + q < p.S ? raw - raw2 : 0.f;
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(delta0 + ((jt % 3u) * 128u + (uint32_t)q) * 4u), "f"(dl) : "memory");
+      }
       const float x = step * AT_BLK + q < p.S ? raw * mul : 0.f;
       const __nv_bfloat16 h1 = __float2bfloat16_rn(x);
       const float r1 = x - __bfloat162float(h1);
@@ -423,7 +454,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       while (bias_written < itg + (uint32_t)(total < 2 ? total : 2)) {
         const int l = (int)(bias_written - itg);
-        bias_put(it_begin + l, bias_written, bias_fetch(bh, it_begin + l), bias_mul);
+        bias_put(it_begin + l, bias_written, bias_fetch(bh, it_begin + l), bias_mul, bias_fetch2(bh, it_begin + l));
         ++bias_written;
       }
     }
@@ -434,13 +465,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       if (t - total < nx_total) { tbh = nx_bh; tstep = nx_begin + (t - total); return true; }
       return false;
     };
-    float lse2 = 0.f, dq = 0.f;                               // this row's LSE*log2e and D
+    float lse2 = 0.f, dq = 0.f, dq2 = 0.f;                    // this row's LSE*log2e and D (dq2: the second draw's D)
     int qrow = 0;                                             // global query index of this thread's row
     if (MODE != AT_DKV) {
       qrow = blk * AT_BLK + r;
       if (MODE == AT_DQ && qrow < p.S) {
         lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
         dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
+        if (ND == 2) dq2 = __ldg(p.dterm + (size_t)p.BH * p.S + (size_t)bh * p.S + qrow);
       }
     }
     float run_m = -INFINITY, run_l = 0.f;                     // FWD pass 1: running max and sum (this half)
@@ -449,7 +481,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
-      float bias_next = 0.f;                                  // DKV: this thread's raw value for the row two steps ahead
+      float bias_next = 0.f, bias_next2 = 0.f;                // DKV: this thread's raw value(s) for the row two steps ahead
       int bias_bh = 0, bias_step = 0;
       const bool bias_due = MODE == AT_DKV && bias_written == itg + (uint32_t)it + 2u && bias_target(it, bias_bh, bias_step);
       if (MODE == AT_DKV) {
@@ -489,7 +521,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(b_sdp_free);
-      if (bias_due) bias_next = bias_fetch(bias_bh, bias_step);   // lands under this step's arithmetic
+      if (bias_due) {                                         // lands under this step's arithmetic
+        bias_next = bias_fetch(bias_bh, bias_step);
+        bias_next2 = bias_fetch2(bias_bh, bias_step);
+      }
 
       const int key0 = kblk * AT_BLK + h * 64;
       // masking is needed only on the diagonal block and where the sequence ends inside the block
@@ -574,6 +609,43 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
                          "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
           }
+        } else if (MODE == AT_DQ && ND == 2) {
+          // two draws: one exponential per element, two dS values; 32 columns at a time so that the
+          // packed operands of both draws stay within the register budget
+          uint32_t da[16], db[16];
+          auto pair2_at = [&](int j, bool masked) {
+            float a0 = fmaf(__uint_as_float(sv[j]), c2, -lse2), a1 = fmaf(__uint_as_float(sv[j + 1]), c2, -lse2);
+            if (masked) {
+              if (!valid_at(j)) a0 = -INFINITY;
+              if (!valid_at(j + 1)) a1 = -INFINITY;
+            }
+            const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+            const float x0 = __uint_as_float(dv[j]) * dp_mul, x1 = __uint_as_float(dv[j + 1]) * dp_mul;
+            da[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 - dq), p1 * (x1 - dq));
+            db[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 - dq2), p1 * (x1 - dq2));
+          };
+          if (!edge) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair2_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair2_at(j, true);
+          }
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          if (!ok) break;
+          tmem_st16(t_ds + lane_off + h * 32, da);
+          tmem_st16(t_ds2 + lane_off + h * 32, db);
+          if (!edge) {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair2_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair2_at(j, true);
+          }
+          tmem_st16(t_ds + lane_off + h * 32 + 16, da);
+          tmem_st16(t_ds2 + lane_off + h * 32 + 16, db);
+          tmem_wait_st();
+          tc_fence_before();
         } else if (MODE == AT_DQ) {
           if (!edge) {
 #pragma unroll
@@ -587,6 +659,46 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
           tmem_st32(t_ds + lane_off + h * 32, dk);
+          tmem_wait_st();
+          tc_fence_before();
+        } else if (MODE == AT_DKV && ND == 2) {
+          // dK kernel, two draws: the accumulators hold s - LSE/c and dP - D of the first draw; the
+          // second draw's dP - D is that plus delta of the column's query.  32 columns at a time.
+          uint32_t da[16], db[16];
+          const uint32_t dbase = delta0 + (((itg + (uint32_t)it) % 3u) * 128u + (uint32_t)h * 64u) * 4u;
+          auto pair2_at = [&](int j, bool masked) {
+            float a0 = __uint_as_float(sv[j]) * c2, a1 = __uint_as_float(sv[j + 1]) * c2;
+            if (masked) {
+              if (!valid_at(j)) a0 = -INFINITY;
+              if (!valid_at(j + 1)) a1 = -INFINITY;
+            }
+            const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+            float e0, e1;
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(e0), "=f"(e1) : "r"(dbase + (uint32_t)j * 4u));
+            const float x0 = __uint_as_float(dv[j]) * dp_mul, x1 = __uint_as_float(dv[j + 1]) * dp_mul;
+            da[(j & 31) >> 1] = pack_bf16x2(p0 * x0, p1 * x1);
+            db[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 + e0), p1 * (x1 + e1));
+          };
+          if (!edge) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair2_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) pair2_at(j, true);
+          }
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          if (!ok) break;
+          tmem_st16(t_ds + lane_off + h * 32, da);
+          tmem_st16(t_ds2 + lane_off + h * 32, db);
+          if (!edge) {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair2_at(j, false);
+          } else {
+#pragma unroll
+            for (int j = 32; j < 64; j += 2) pair2_at(j, true);
+          }
+          tmem_st16(t_ds + lane_off + h * 32 + 16, da);
+          tmem_st16(t_ds2 + lane_off + h * 32 + 16, db);
           tmem_wait_st();
           tc_fence_before();
         } else {
@@ -631,8 +743,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       if (bias_due) {
         // (the empty asm pins the first use of the fetched value here, after the step's arithmetic)
-        asm volatile("" : "+f"(bias_next));
-        bias_put(bias_step, bias_written, bias_next, bias_bh == bh && it + 2 < total ? bias_mul : nx_mul);
+        asm volatile("" : "+f"(bias_next), "+f"(bias_next2));
+        bias_put(bias_step, bias_written, bias_next, bias_bh == bh && it + 2 < total ? bias_mul : nx_mul, bias_next2);
         ++bias_written;
       }
     }
@@ -671,8 +783,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (MODE == AT_DKV) mul = o == 0 ? (FP8 ? inv_do / p.p_scale : 1.f) : p.c * (FP8 ? inv_q / p.ds_scale : 1.f);
         else if (MODE == AT_DQ) mul = p.c * (FP8 ? inv_k / p.ds_scale : 1.f);
         else mul = inv_v;
-        uint32_t a[32];
+        uint32_t a[32], a2[ND == 2 ? 32 : 1];
         tmem_ld32((o == 0 ? t_acc0 : t_acc1) + lane_off + h * 32, a);
+        if (ND == 2) tmem_ld32((o == 0 ? t_acc1 : t_acc0) + lane_off + h * 32, *reinterpret_cast<uint32_t(*)[32]>(&a2[0]));
         if (o == nout - 1) {
           // the accumulators may be overwritten by the next item (FWD: the item after next)
           tc_fence_before();
@@ -685,11 +798,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
           for (int t = 0; t < 8; ++t) {
             const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
-            const float d0 = __uint_as_float(a[4 * t]) * mul - rv[4 * t], d1 = __uint_as_float(a[4 * t + 1]) * mul - rv[4 * t + 1];
-            const float d2 = __uint_as_float(a[4 * t + 2]) * mul - rv[4 * t + 2], d3 = __uint_as_float(a[4 * t + 3]) * mul - rv[4 * t + 3];
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(d0), "f"(d1), "f"(d2), "f"(d3) : "memory");
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg2 + off), "f"(d0 * d0), "f"(d1 * d1), "f"(d2 * d2),
-                         "f"(d3 * d3) : "memory");
+            float d[4], q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              d[e] = __uint_as_float(a[4 * t + e]) * mul - rv[4 * t + e];
+              q[e] = d[e] * d[e];
+              if (ND == 2) {                                  // the second draw of this launch joins the first
+                const float e2 = __uint_as_float(a2[ND == 2 ? 4 * t + e : 0]) * mul - rv[4 * t + e];
+                d[e] += e2;
+                q[e] = fmaf(e2, e2, q[e]);
+              }
+            }
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(d[0]), "f"(d[1]), "f"(d[2]), "f"(d[3]) : "memory");
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg2 + off), "f"(q[0]), "f"(q[1]), "f"(q[2]), "f"(q[3]) : "memory");
           }
           continue;
         }
@@ -836,7 +957,7 @@ static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
 }
 
-template <int MODE, bool FP8, bool DV, bool MC = false>
+template <int MODE, bool FP8, bool DV, bool MC = false, int ND = 1>
 static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   CUtensorMap mq, mk, mv, mdo, mo0, mo1;
   int rc;
@@ -848,7 +969,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
   static bool attr_set = false;
   if (!attr_set) {
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC, ND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
@@ -858,7 +979,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE, FP8, DV, MC><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
+  attn_kernel<MODE, FP8, DV, MC, ND><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
@@ -867,6 +988,7 @@ template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   if (MODE != AT_FWD && p.mc_ref != nullptr) {               // Monte-Carlo epilogue: BF16 operands, no dV
     if (p.fp8) return BSP_ERR_UNSUPPORTED;
+    if (p.nd == 2) return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD, MODE != AT_FWD ? 2 : 1>(q, k, v, dO, p, st);
     return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD>(q, k, v, dO, p, st);
   }
   if (MODE == AT_DKV && p.out0 == nullptr)                   // dK only
@@ -902,7 +1024,7 @@ static int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr;
+  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
 }
@@ -979,7 +1101,7 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
     return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag; p.mc_ref = nullptr;
+  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   if (dk) {
@@ -993,23 +1115,27 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
   return BSP_OK;
 }
 
-// One fresh draw of the D use for dQ and dK with the Monte-Carlo epilogue: the two kernels add
+// nd (1 or 2) fresh draws of the D use for dQ and dK with the Monte-Carlo epilogue: the kernels add
 // g - ref and its square to the running sums of their gradient and write no gradient (BF16-operand
-// mode; dV is not computed).  The sums must not be touched by anything else while this runs.
+// mode; dV is not computed).  dterm holds the draws' correction terms back to back, [nd][B*H*S]; both
+// kernels take the two draws in one launch (S, dP and P are formed once per step).  The sums must not
+// be touched by anything else while this runs.
 static int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
                              const void* k, const void* v, const void* dO, int dt, const float* lse,
-                             const float* dterm, const float* ref_dq, float* S1q, float* S2q, const float* ref_dk,
-                             float* S1k, float* S2k, bsp_diag_t* diag, void* stream) {
+                             const float* dterm, int nd, const float* ref_dq, float* S1q, float* S2q,
+                             const float* ref_dk, float* S1k, float* S2k, bsp_diag_t* diag, void* stream) {
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !dO || !lse || !dterm || !ref_dq || !S1q || !S2q || !ref_dk || !S1k || !S2k) return BSP_ERR_ARG;
+  if (nd < 1 || nd > 2) return BSP_ERR_ARG;
   if (!aligned16(ref_dq) || !aligned16(ref_dk) || !aligned16(S1q) || !aligned16(S2q) || !aligned16(S1k) || !aligned16(S2k))
     return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag;
+  p.lse = lse; p.lse_out = nullptr; p.diag = diag;
   if ((rc = set_fp8(p, nullptr)) != BSP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
+  p.dterm = dterm; p.nd = nd;
   p.mc_ref = ref_dk; p.out0 = S1k; p.out1 = S2k;
   if ((rc = launch_attn<AT_DKV>(q, k, v, dO, p, st)) != BSP_OK) return rc;
   p.mc_ref = ref_dq; p.out0 = S1q; p.out1 = S2q;
@@ -1250,9 +1376,13 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
       const float* dk_ = b.d_draws + (size_t)k * rows;
       BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
       if (k > 0) {
-        // the draws after the first: dQ and dK go from the accumulators straight into their sums
-        BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_ref[0],
-                                  b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
+        // the draws after the first, two at a time: dQ and dK go from the accumulators straight into
+        // their sums
+        const int nd = k + 1 < K ? 2 : 1;
+        if (nd == 2) BSP_TRY(bsp_mc_accumulate(dk_ + rows, b.d_ref, b.S1d, b.S2d, rows, st));
+        BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, nd,
+                                  b.g_ref[0], b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
+        k += nd - 1;
         continue;
       }
       BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],

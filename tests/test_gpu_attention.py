@@ -210,6 +210,51 @@ def test_mc_check_attention_verdicts(b):
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
 
 
+def test_mc_check_attention_fused_sums_match_draw_by_draw(b):
+    """Inside the check the draws after the first go two at a time through kernels that add g - g*
+    and its square straight into the running sums.  The same statistics taken draw by draw through
+    the single-draw entry points (gradient written, then accumulated) must agree: same draws, same
+    per-draw arithmetic, only the order of a few FP32 additions differs.  K = 7: one plain draw,
+    two pairs, and a single draw left over; S = 328: three blocks, the last one ragged."""
+    inp = workloads.config3(B=2, H=3, S=328, D=64, K=7, seed=91)
+    g = AttnGpu(b, inp, True)
+    B, H, S, D, K = inp.B, inp.H, inp.S, inp.D, inp.K
+    rows, n = B * H * S, B * H * S * D
+    d = b.AttnDesc()
+    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, inp.softmax_scale, b.BF16
+    d.q, d.k, d.v, d.dO = b.ptr(g.q), b.ptr(g.k), b.ptr(g.v), b.ptr(g.dO)
+    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, 4
+    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+    diag = b.new_diag()
+    res = b.bsp_mc_check_attn(d, K, ws, diag)
+    assert b.read_diag(diag)["status"] == 0
+    assert [(r.policy, r.output_id) for r in res] == [(2, o) for o in (b.OUT_D, b.OUT_DQ, b.OUT_DK, b.OUT_DV)]
+    # draw by draw, through the public single-draw calls
+    key = b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0)
+    d_ref = torch.zeros(rows, device="cuda")
+    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, g.codes, g.scales, fp8.E4M3, b.READ_ORIGINAL, key, 0, 1, d_ref)
+    ref = [torch.zeros(n, device="cuda") for _ in range(3)]
+    b.bsp_attn_bwd_dterm(B, H, S, D, True, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, d_ref, *ref)
+    d_draws = torch.zeros(K * rows, device="cuda")
+    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, g.codes, g.scales, fp8.E4M3, b.READ_FRESH, key, 0, K, d_draws)
+    S1 = [torch.zeros(n, device="cuda") for _ in range(2)]
+    S2 = [torch.zeros(n, device="cuda") for _ in range(2)]
+    gk = [torch.zeros(n, device="cuda") for _ in range(2)]
+    for k in range(K):
+        b.bsp_attn_bwd_dterm(B, H, S, D, True, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse,
+                             d_draws[k * rows:(k + 1) * rows], gk[0], gk[1], None)
+        for t in range(2):
+            b.bsp_mc_accumulate(gk[t], ref[t], S1[t], S2[t], n)
+    wss = b.workspace(b.bsp_mc_stats_workspace_bytes(n))
+    for t in range(2):
+        want = b.bsp_mc_stats(ref[t], S1[t], S2[t], n, K, 1, wss)
+        got = res[1 + t]
+        assert got.verdict == want.verdict and got.K == want.K and got.n_elements == want.n_elements
+        for f in ("rel_l2_mean_err", "R", "Qprime", "mean_z", "rms_z", "max_abs_z", "frac_abs_z_gt3"):
+            x, y = getattr(got, f), getattr(want, f)
+            assert abs(x - y) <= 2e-3 * max(abs(y), 1e-3), (t, f, x, y)
+
+
 @pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks", "many_items_ragged"])
 def test_fp8_operand_mode(b, name):
     """The emulated FP8 attention backward: Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice, P rounded
