@@ -967,7 +967,8 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
-  static bool attr_set = false;
+  static bool attr_set_dev[kMaxDevices] = {};
+  bool& attr_set = attr_set_dev[device_slot()];
   if (!attr_set) {
     BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC, ND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set = true;

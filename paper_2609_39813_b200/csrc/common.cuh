@@ -28,6 +28,15 @@ void count_launch();          // defined in mc.cu
 
 constexpr int kNumSMs = 148;
 
+// Index of the current device into a per-device flag array of kMaxDevices entries (a function
+// attribute such as the dynamic shared-memory limit is set once per device, not once per process).
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+  return dev % kMaxDevices;
+}
+
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t round_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 

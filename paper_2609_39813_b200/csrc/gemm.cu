@@ -586,7 +586,8 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     if (rc != BSP_OK) return rc;
     p.idesc = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, MC_BN);
     p.idesc2 = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, 2 * MC_BN);
-    static bool mc_attr_set = false;
+    static bool mc_attr_set_dev[kMaxDevices] = {};
+    bool& mc_attr_set = mc_attr_set_dev[device_slot()];
     if (!mc_attr_set) {
       BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
       mc_attr_set = true;
@@ -600,7 +601,8 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
 
   rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN, g.b_mn);
   if (rc != BSP_OK) return rc;
-  static bool attr_set[2] = {false, false};
+  static bool attr_set_dev[kMaxDevices][2] = {};
+  bool* attr_set = attr_set_dev[device_slot()];
   if (!attr_set[g.fp8 ? 1 : 0]) {
     if (g.fp8) BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
     else BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));

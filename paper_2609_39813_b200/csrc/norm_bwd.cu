@@ -509,7 +509,6 @@ namespace bsp {
 constexpr size_t kNoAllocScratchBytes = BSP_NORM_BWD_NOALLOC_CAPACITY_BYTES;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
-constexpr int kMaxDevices = 64;
 static void* g_noalloc_ptr[kMaxDevices];          // resolved device addresses, by device ordinal
 static std::mutex g_noalloc_mutex;
 
