@@ -754,14 +754,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     // its row's 32 FP32 values of column half h into the 128-byte-swizzle box that a tiled bulk store
     // then writes (whole 128-byte lines; rows beyond the sequence are clipped by the store).
     constexpr bool mc = MC;
-    float rv[32];                                             // Monte-Carlo epilogue: the reference values of this thread's 32 outputs
+    // Monte-Carlo epilogue: the reference values of the warp's 32 rows x 32 columns, fetched by the
+    // warp together (load t: four rows of 128 contiguous bytes, lane -> row 4t + lane / 8, 16-byte
+    // chunk lane % 8) and handed to the row-owning threads through the staging buffer further down
+    float4 rc[8];
     if (mc) {
-      const int orow = blk * AT_BLK + r;
-      const float4* rp = reinterpret_cast<const float4*>(p.mc_ref + ((size_t)bh * p.S + (orow < p.S ? orow : 0)) * AT_D + h * 32);
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
-        const float4 v4 = __ldg(rp + t);
-        rv[4 * t] = v4.x; rv[4 * t + 1] = v4.y; rv[4 * t + 2] = v4.z; rv[4 * t + 3] = v4.w;
+        const int orow = blk * AT_BLK + q4 * 32 + 4 * t + (lane >> 3);
+        rc[t] = __ldg(reinterpret_cast<const float4*>(p.mc_ref + ((size_t)bh * p.S + (orow < p.S ? orow : 0)) * AT_D + h * 32) +
+                      (lane & 7));
       }
     }
     if (ok) ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_acc + 8 * ab, iph, abort_flag));
@@ -776,6 +778,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         store_pending = false;
       }
       if (MODE == AT_DKV || mc) named_bar_sync(3, 256);       // ... before anyone writes the second staging buffer again
+      float rv[32];                                           // this thread's 32 reference values
+      if (mc) {
+        // through the warp's own 4 KB of the (now free) second staging buffer: chunk (row, c) sits
+        // where the output boxes keep it, so every thread finds its row at its own output slots
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t row = (uint32_t)(q4 * 32 + 4 * t + (lane >> 3));
+          const uint32_t off = (uint32_t)h * 16384u + row * 128u + ((((uint32_t)lane & 7u) ^ (row & 7u)) << 4);
+          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage2 + off), "f"(rc[t].x), "f"(rc[t].y), "f"(rc[t].z),
+                       "f"(rc[t].w) : "memory");
+        }
+        __syncwarp();
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+          asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                       : "=f"(rv[4 * t]), "=f"(rv[4 * t + 1]), "=f"(rv[4 * t + 2]), "=f"(rv[4 * t + 3]) : "r"(stage2 + off));
+        }
+        __syncwarp();
+      }
 #pragma unroll
       for (int o = (MODE == AT_DKV && !DV) ? 1 : 0; o < nout; ++o) {
         const uint32_t stg = o == 0 ? res_base + rbi * 2 * kAtTile : stage2;
