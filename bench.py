@@ -115,6 +115,28 @@ def oracle_sample(inp, rows, k_gain, k_wgrad):
     return dt, rows * inp.C * (2 + k_gain + 2 + k_wgrad)
 
 
+def library_fp8_tflops(n=8192, reps=10):
+    """TFLOP/s of the library FP8 GEMM (torch._scaled_mm) at n^3; None where it is not available.
+    A measurement of the machine, not part of the path."""
+    import torch
+    try:
+        a = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn)
+        bt = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn).t()
+        one = torch.ones((), device="cuda")
+        for _ in range(3):
+            torch._scaled_mm(a, bt, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            torch._scaled_mm(a, bt, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+        e1.record()
+        torch.cuda.synchronize()
+        return 2.0 * n ** 3 * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    except Exception:
+        return None
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -514,6 +536,12 @@ def run_ours(args):
                     traffic_unit="bytes per launch (ncu dram read + write, one capture)",
                     us_per_launch=gemm_ms * 1e3, draws_per_launch=K,
                     peak_source="2 x bf16_tflops (%s)" % peaks["source"])
+    # Context beside that denominator: what the vendor library's own FP8 contraction reaches on this
+    # GPU in this run (8192^3, E4M3 x E4M3, a short burst), measured the way the BF16 figure was.
+    lib_fp8 = library_fp8_tflops() if rank == 0 else None
+    if lib_fp8:
+        roofline["library_fp8_tflops_this_run"] = lib_fp8
+        roofline["frac_of_library_fp8"] = achieved / lib_fp8
     dstat = b.read_diag(diag)
 
     if rank != 0:
