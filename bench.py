@@ -239,6 +239,7 @@ def attention_section(b, peaks, steps=3):
                               # a backward needs 5 of those products; the two kernels form S and dP once each
                               algorithmic_tflops=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12,
                               algorithmic_frac=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
+                              peak_nominal=2250.0, frac_of_nominal=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / 2250.0,
                               note="achieved counts the 7 causal products of 2*S*S*d/2 flop per head that the two "
                                    "kernels compute, algorithmic_* the 5 a backward needs; exp on the SFU co-bounds it"),
                 diag_status=b.read_diag(diag)["status"])
@@ -287,7 +288,7 @@ def kernel_table(b, peaks):
         us = e0.elapsed_time(e1) / reps * 1e3
         gbs = nbytes / us / 1e3
         rows.append(dict(kernel=name, bound=bound, us=us, algorithmic_mb=nbytes / 1e6, gb_per_s=gbs,
-                         frac_of_hbm=gbs / peaks["hbm_gbs"]))
+                         frac_of_hbm=gbs / peaks["hbm_gbs"], frac_of_nominal_hbm=gbs / 8000.0))
 
     t("amax(dY)", "hbm", lambda: b.bsp_amax(dY, 1, T * O, amax), T * O * 2)
     t("round dY -> E5M2 nearest", "hbm", lambda: b.bsp_round(dY, T * O, qrn, k, 0, dyc), T * O * 3)
@@ -535,7 +536,8 @@ def run_ours(args):
                     achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=traffic,
                     traffic_unit="bytes per launch (ncu dram read + write, one capture)",
                     us_per_launch=gemm_ms * 1e3, draws_per_launch=K,
-                    peak_source="2 x bf16_tflops (%s)" % peaks["source"])
+                    peak_source="2 x bf16_tflops (%s)" % peaks["source"],
+                    peak_nominal=4500.0, frac_of_nominal=achieved / 4500.0)
     # Context beside that denominator: what the vendor library's own FP8 contraction reaches on this
     # GPU in this run (8192^3, E4M3 x E4M3, a short burst), measured the way the BF16 figure was.
     lib_fp8 = library_fp8_tflops() if rank == 0 else None
