@@ -23,6 +23,7 @@
 
 
 #include "common.cuh"
+#include "mc_stats.cuh"
 #include "tc.cuh"
 
 namespace bsp {
@@ -1305,7 +1306,7 @@ static size_t attn_carve(const bsp_attn_desc_t* op, int K, char* base, AttnCheck
     c.S1[t] = (float*)take(n * 4); c.S2[t] = (float*)take(n * 4);
   }
   c.S1d = (float*)take(rows * 4); c.S2d = (float*)take(rows * 4);
-  c.b_stats = bsp_mc_stats_workspace_bytes((int64_t)n);
+  c.b_stats = kMaxPendingStats * kStatSlotBytes;
   c.ws_stats = take(c.b_stats);
   if (out) *out = c;
   return off;
@@ -1358,6 +1359,10 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
                          b.d_ref, diag, st));
   BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, b.d_ref, b.g_ref[0],
                              b.g_ref[1], b.g_ref[2], diag, st));
+  // the twelve statistics passes are read behind one synchronisation at the end
+  PendingStats pend;
+  pend.slots = reinterpret_cast<double*>(b.ws_stats);
+  pend.st = st;
   int nres = 0;
   const int out_ids[4] = {BSP_OUT_D, BSP_OUT_DQ, BSP_OUT_DK, BSP_OUT_DV};
   auto emit = [&](int out, int pol) -> bsp_use_result_t* {
@@ -1378,10 +1383,9 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
       dsrc = b.d_pol;
       gsrc = b.g_pol;
     }
-    BSP_TRY(bsp_mc_stats(b.d_ref, dsrc, nullptr, (int64_t)rows, 1, 0, emit(out_ids[0], pol), b.ws_stats, b.b_stats, st));
+    BSP_TRY(pend.add(b.d_ref, dsrc, nullptr, (int64_t)rows, 1, 0, emit(out_ids[0], pol)));
     for (int t = 0; t < 3; ++t)
-      BSP_TRY(bsp_mc_stats(b.g_ref[t], gsrc[t], nullptr, (int64_t)n, 1, 0, emit(out_ids[t + 1], pol), b.ws_stats,
-                           b.b_stats, st));
+      BSP_TRY(pend.add(b.g_ref[t], gsrc[t], nullptr, (int64_t)n, 1, 0, emit(out_ids[t + 1], pol)));
   }
   if ((op->policy_mask >> 2) & 1u) {
     // fresh read: all K correction terms in one pass, then one backward per draw
@@ -1413,15 +1417,12 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
       for (int t = 0; t < 2; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
       BSP_TRY(mc_accumulate_times(b.g_pol[2], b.g_ref[2], b.S1[2], b.S2[2], n, (float)K, st));
     }
-    BSP_TRY(bsp_mc_stats(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH), b.ws_stats,
-                         b.b_stats, st));
+    BSP_TRY(pend.add(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH)));
     for (int t = 0; t < 3; ++t)
-      BSP_TRY(bsp_mc_stats(b.g_ref[t], b.S1[t], b.S2[t], (int64_t)n, K, 1, emit(out_ids[t + 1], BSP_READ_FRESH),
-                           b.ws_stats, b.b_stats, st));
+      BSP_TRY(pend.add(b.g_ref[t], b.S1[t], b.S2[t], (int64_t)n, K, 1, emit(out_ids[t + 1], BSP_READ_FRESH)));
   }
   *n_results = nres;
-  BSP_CHECK_CUDA(cudaStreamSynchronize(st));
-  return BSP_OK;
+  return pend.flush();
 }
 
 }  // extern "C"

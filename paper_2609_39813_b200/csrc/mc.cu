@@ -6,14 +6,13 @@
 #include <vector>
 
 #include "common.cuh"
+#include "mc_stats.cuh"
 
 namespace bsp {
 
 static std::atomic<unsigned long long> g_launches{0};
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
-constexpr int kStatBlocks = 592;     // 4 per SM
-constexpr int kStatFields = 8;       // err2, ref2, se2, z2, z, max|z|, count(|z|>3), unused
 
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
@@ -84,11 +83,10 @@ mc_stats_kernel(const float* __restrict__ g_ref, const float* __restrict__ g, co
   }
 }
 
-constexpr size_t kStatSlotDoubles = (size_t)kStatBlocks * kStatFields;
 
 // Launches the statistics pass over n elements into one slot of block partials; returns the number
 // of blocks whose partials the slot then holds.
-static int mc_stats_launch(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
+int mc_stats_launch(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
                            double* partials, cudaStream_t st, int* blocks_out) {
   int blocks = (int)((n + 255) / 256);
   if (blocks > kStatBlocks) blocks = kStatBlocks;
@@ -101,7 +99,7 @@ static int mc_stats_launch(const float* g_ref, const float* g, const float* S2, 
 }
 
 // Sums a slot's block partials on the host, in block order, and fills the result of the use.
-static void mc_stats_finish(const double* host, int blocks, int64_t n, int K, int fresh, bsp_use_result_t* result) {
+void mc_stats_finish(const double* host, int blocks, int64_t n, int K, int fresh, bsp_use_result_t* result) {
   double f[kStatFields] = {0, 0, 0, 0, 0, 0, 0, 0};
   for (int b = 0; b < blocks; ++b)
     for (int j = 0; j < kStatFields; ++j)
@@ -128,16 +126,6 @@ static void mc_stats_finish(const double* host, int blocks, int64_t n, int K, in
   else if (result->Qprime <= 2.0 && result->R <= 3.0) result->verdict = BSP_HOLDS;
   else result->verdict = BSP_UNDECIDED;
 }
-
-// The statistics passes of one check: each is launched into its own slot of partials as soon as its
-// inputs are queued, and all of them are brought to the host behind one synchronisation at the end.
-constexpr int kCheckStatSlots = 6;
-struct PendingStats {
-  bsp_use_result_t* result[kCheckStatSlots];
-  int blocks[kCheckStatSlots], K[kCheckStatSlots], fresh[kCheckStatSlots];
-  int64_t n[kCheckStatSlots];
-  int count = 0;
-};
 
 struct Bump {
   char* base;
@@ -196,7 +184,7 @@ static size_t carve(const bsp_norm_linear_desc_t* op, int K, char* base, CheckBu
   c.b_gain = bsp_norm_gain_mc_workspace_bytes(op->T, op->C, K > 0 ? K : 1);
   c.b_wgrad = bsp_linear_wgrad_workspace_bytes(op->T, op->O, op->C, BSP_READ_ORIGINAL);
   c.b_dgrad = bsp_linear_dgrad_workspace_bytes(op->T, op->O, op->C);
-  c.b_stats = kCheckStatSlots * bsp_mc_stats_workspace_bytes((int64_t)(O * C > C ? O * C : C));
+  c.b_stats = kMaxPendingStats * kStatSlotBytes;
   c.ws_bwd = b.take(c.b_bwd); c.ws_gain = b.take(c.b_gain); c.ws_wgrad = b.take(c.b_wgrad);
   c.ws_dgrad = b.take(c.b_dgrad); c.ws_stats = b.take(c.b_stats);
   if (cb) *cb = c;
@@ -299,13 +287,10 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
   BSP_TRY(bsp_linear_dgrad(T, O, C, b.dy_codes, qdy, op->W, dt, b.du, dt, b.ws_dgrad, b.b_dgrad, diag, st));
 
   PendingStats pend;
+  pend.slots = reinterpret_cast<double*>(b.ws_stats);
+  pend.st = st;
   auto stats = [&](const float* g_ref, const float* g, const float* S2, int64_t n, int Kd, int fresh,
-                   bsp_use_result_t* r) -> int {
-    const int slot = pend.count++;
-    pend.result[slot] = r; pend.n[slot] = n; pend.K[slot] = Kd; pend.fresh[slot] = fresh;
-    return mc_stats_launch(g_ref, g, S2, n, Kd, fresh, reinterpret_cast<double*>(b.ws_stats) + slot * kStatSlotDoubles,
-                           st, &pend.blocks[slot]);
-  };
+                   bsp_use_result_t* r) -> int { return pend.add(g_ref, g, S2, n, Kd, fresh, r); };
   int nres = 0;
   auto emit = [&](int use, int out, int pol) -> bsp_use_result_t* {
     bsp_use_result_t* r = &results[nres++];
@@ -379,15 +364,7 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
     }
   }
   *n_results = nres;
-  std::vector<double> host((size_t)(pend.count > 0 ? pend.count : 1) * kStatSlotDoubles);
-  if (pend.count > 0)
-    BSP_CHECK_CUDA(cudaMemcpyAsync(host.data(), b.ws_stats, (size_t)pend.count * kStatSlotDoubles * sizeof(double),
-                                   cudaMemcpyDeviceToHost, st));
-  BSP_CHECK_CUDA(cudaStreamSynchronize(st));
-  for (int i = 0; i < pend.count; ++i)
-    mc_stats_finish(host.data() + (size_t)i * kStatSlotDoubles, pend.blocks[i], pend.n[i], pend.K[i], pend.fresh[i],
-                    pend.result[i]);
-  return BSP_OK;
+  return pend.flush();
 }
 
 }  // extern "C"
