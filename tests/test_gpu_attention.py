@@ -210,13 +210,15 @@ def test_mc_check_attention_verdicts(b):
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
 
 
-def test_mc_check_attention_fused_sums_match_draw_by_draw(b):
+@pytest.mark.parametrize("K", [4, 7, 8])
+def test_mc_check_attention_fused_sums_match_draw_by_draw(b, K):
     """Inside the check the draws after the first go two at a time through kernels that add g - g*
     and its square straight into the running sums.  The same statistics taken draw by draw through
     the single-draw entry points (gradient written, then accumulated) must agree: same draws, same
-    per-draw arithmetic, only the order of a few FP32 additions differs.  K = 7: one plain draw,
-    two pairs, and a single draw left over; S = 328: three blocks, the last one ragged."""
-    inp = workloads.config3(B=2, H=3, S=328, D=64, K=7, seed=91)
+    per-draw arithmetic, only the order of a few FP32 additions differs.  K = 4: one plain draw, a
+    pair and a single fused draw; K = 7: three pairs; K = 8: three pairs and a single draw left over.
+    S = 328: three blocks, the last one ragged."""
+    inp = workloads.config3(B=2, H=3, S=328, D=64, K=K, seed=91)
     g = AttnGpu(b, inp, True)
     B, H, S, D, K = inp.B, inp.H, inp.S, inp.D, inp.K
     rows, n = B * H * S, B * H * S * D
@@ -252,7 +254,7 @@ def test_mc_check_attention_fused_sums_match_draw_by_draw(b):
         assert got.verdict == want.verdict and got.K == want.K and got.n_elements == want.n_elements
         for f in ("rel_l2_mean_err", "R", "Qprime", "mean_z", "rms_z", "max_abs_z", "frac_abs_z_gt3"):
             x, y = getattr(got, f), getattr(want, f)
-            assert abs(x - y) <= 2e-3 * max(abs(y), 1e-3), (t, f, x, y)
+            assert x == y or abs(x - y) <= 2e-3 * max(abs(y), 1e-3), (t, f, x, y)
 
 
 @pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks", "many_items_ragged"])
