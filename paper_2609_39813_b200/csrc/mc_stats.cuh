@@ -33,6 +33,11 @@ struct PendingStats {
   cudaStream_t st = nullptr;
 
   int add(const float* g_ref, const float* g, const float* S2, int64_t n_, int K_, int fresh_, bsp_use_result_t* r) {
+    if (!fresh_ && g == g_ref) {
+      // a read that is the reference itself: its error is exactly zero, no pass needed
+      mc_stats_finish(nullptr, 0, n_, K_, 0, r);
+      return BSP_OK;
+    }
     if (count >= kMaxPendingStats) return BSP_ERR_ARG;
     const int slot = count++;
     result[slot] = r; n[slot] = n_; K[slot] = K_; fresh[slot] = fresh_;
