@@ -402,7 +402,11 @@ int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n,
  *   shifted-sum epilogue).
  * `policy_mask` bit (use*3 + policy) selects evaluations, use 0 = gain, 1 = weight.
  * results: HOST array, filled in order gain U,R,N then weight U,R,N (selected ones only);
- * *n_results returns the count.  Synchronises before returning. */
+ * *n_results returns the count.  Synchronises before returning.
+ * When both uses ask for N, the K-draw gain kernel runs beside the first K-draw contraction on a
+ * second, non-blocking stream that the library creates once per device and keeps; it is forked
+ * from and joined back into `stream` inside the call, and is idle when the call returns on any
+ * path.  Calls on one device may overlap in time only if they use different workspaces. */
 typedef struct {
   int32_t norm_kind;         /* bsp_norm_t  */
   int32_t dtype;             /* bsp_dtype_t of x, W, dY (and of du) */

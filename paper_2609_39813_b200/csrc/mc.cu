@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -127,6 +128,32 @@ void mc_stats_finish(const double* host, int blocks, int64_t n, int K, int fresh
   else result->verdict = BSP_UNDECIDED;
 }
 
+// A second stream per device for the one place where two independent kernels are worth running
+// side by side: the K-draw gain use (integer pipes) under the K-draw weight-gradient contraction
+// (tensor pipes).  Created on first use, kept until the process exits.
+static std::mutex g_side_mutex;
+static cudaStream_t g_side_stream[kMaxDevices];
+static int side_stream(cudaStream_t* out) {
+  const int slot = device_slot();
+  std::lock_guard<std::mutex> lock(g_side_mutex);
+  if (!g_side_stream[slot]) BSP_CHECK_CUDA(cudaStreamCreateWithFlags(&g_side_stream[slot], cudaStreamNonBlocking));
+  *out = g_side_stream[slot];
+  return BSP_OK;
+}
+
+// Fork / join of that stream inside one call; whatever path leaves the call, the side stream is
+// idle and the events are gone when this goes out of scope.
+struct SideWork {
+  cudaStream_t side = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool launched = false;
+  ~SideWork() {
+    if (launched) cudaStreamSynchronize(side);
+    if (fork) cudaEventDestroy(fork);
+    if (join) cudaEventDestroy(join);
+  }
+};
+
 struct Bump {
   char* base;
   size_t off;
@@ -181,7 +208,7 @@ static size_t carve(const bsp_norm_linear_desc_t* op, int K, char* base, CheckBu
   c.dx = (float*)b.take(T * C * 4);
   c.dW_ref = (float*)b.take(O * C * 4); c.dW_pol = (float*)b.take(O * C * 4); c.S2w = (float*)b.take(O * C * 4);
   c.b_bwd = bsp_norm_bwd_workspace_bytes(op->T, op->C);
-  c.b_gain = bsp_norm_gain_mc_workspace_bytes(op->T, op->C, K > 0 ? K : 1);
+  c.b_gain = norm_gain_mc_workspace(op->T, op->C, K > 0 ? K : 1, true);   // room for either kernel variant
   c.b_wgrad = bsp_linear_wgrad_workspace_bytes(op->T, op->O, op->C, BSP_READ_ORIGINAL);
   c.b_dgrad = bsp_linear_dgrad_workspace_bytes(op->T, op->O, op->C);
   c.b_stats = kMaxPendingStats * kStatSlotBytes;
@@ -299,6 +326,14 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
     return r;
   };
 
+  // When both uses ask for the fresh read, the K-draw gain kernel runs on a second stream beside the
+  // first K-draw contraction of the weight use: one is bound by the integer pipes, the other by the
+  // tensor pipes, and the thin variant of the gain kernel fits next to the contraction's CTA.
+  const bool overlap_gain = (op->policy_mask & 4u) && ((op->policy_mask >> 3) & 4u);
+  SideWork sw;
+  bsp_use_result_t* gain_n_result = nullptr;
+  bsp_key_t gain_key = key;
+
   // ---- gain use (reference: the original)
   const uint32_t gain_mask = op->policy_mask & 7u;
   if (gain_mask) {
@@ -319,10 +354,13 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
     if (gain_mask & 4u) {
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S1g, 0, C * sizeof(float), st));
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S2g, 0, C * sizeof(float), st));
-      BSP_TRY(bsp_norm_gain_mc(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt, qu,
-                               key, 0, K, b.dg_ref, b.S1g, b.S2g, b.ws_gain, b.b_gain, diag, st));
-      bsp_use_result_t* r = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FRESH);
-      BSP_TRY(stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, r));
+      gain_n_result = emit(BSP_STREAM_GAIN, BSP_OUT_DGAMMA, BSP_READ_FRESH);
+      gain_key = key;
+      if (!overlap_gain) {
+        BSP_TRY(bsp_norm_gain_mc(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt, qu,
+                                 gain_key, 0, K, b.dg_ref, b.S1g, b.S2g, b.ws_gain, b.b_gain, diag, st));
+        BSP_TRY(stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, gain_n_result));
+      }
     }
   }
 
@@ -356,8 +394,28 @@ int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* resu
         const int nd = (K - k0) < chunk ? (K - k0) : chunk;
         BSP_TRY(bsp_norm_fwd_draws(op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qf, key, k0,
                                    nd, b.fresh_t, b.ld_t, st));
+        if (overlap_gain && k0 == 0) {
+          // fork: everything the gain kernel reads (du, the statistics, the reference, the cleared
+          // sums) has been queued on the main stream before this point
+          BSP_TRY(side_stream(&sw.side));
+          BSP_CHECK_CUDA(cudaEventCreateWithFlags(&sw.fork, cudaEventDisableTiming));
+          BSP_CHECK_CUDA(cudaEventCreateWithFlags(&sw.join, cudaEventDisableTiming));
+          BSP_CHECK_CUDA(cudaEventRecord(sw.fork, st));
+        }
         BSP_TRY(bsp_linear_wgrad_mc(T, O, C, b.dy_codes_t, qdy, b.fresh_t, qf, b.ld_t, nd, b.dW_ref, S1w, b.S2w, diag,
                                     st));
+        if (overlap_gain && k0 == 0) {
+          // the contraction is queued first, so its CTAs take the SMs first; the gain blocks fill in
+          BSP_CHECK_CUDA(cudaStreamWaitEvent(sw.side, sw.fork, 0));
+          sw.launched = true;
+          BSP_TRY(norm_gain_mc_run(true, op->norm_kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, b.du, dt,
+                                   qu, gain_key, 0, K, b.dg_ref, b.S1g, b.S2g, b.ws_gain, b.b_gain, diag, sw.side));
+          BSP_CHECK_CUDA(cudaEventRecord(sw.join, sw.side));
+        }
+      }
+      if (overlap_gain) {
+        BSP_CHECK_CUDA(cudaStreamWaitEvent(st, sw.join, 0));
+        BSP_TRY(stats(b.dg_ref, b.S1g, b.S2g, C, K, 1, gain_n_result));
       }
       bsp_use_result_t* r = emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FRESH);
       BSP_TRY(stats(b.dW_ref, S1w, b.S2w, O * C, K, 1, r));

@@ -204,9 +204,11 @@ constexpr int kMcSlab = 8 * kMcRows;    // rows per block (8 warps)
 constexpr int kMcCols = 128;            // columns per block (32 lanes x 4)
 constexpr int kMcChunk = 64;            // draws per launch
 constexpr size_t kMcSmemBytes = (size_t)2 * kMcRows * 256 * sizeof(float4);   // values + weights of a slab
+constexpr int kMcThinWarps = 4, kMcThinRows = 4;     // the thin variant: 4 warps x 4 rows per thread
+constexpr size_t kMcThinSmemBytes = (size_t)2 * kMcThinRows * kMcThinWarps * 32 * sizeof(float4);
 
-template <int DT, int DU_DT, int FMT>
-__global__ void __launch_bounds__(256, 3)
+template <int DT, int DU_DT, int FMT, int NW, int ROWS>
+__global__ void __launch_bounds__(NW * 32, NW == 8 ? 3 : 4)
 gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
@@ -221,8 +223,9 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
   // is occupancy that hides their latency.
   extern __shared__ __align__(16) float4 mc_smem[];
   uint4* sp = reinterpret_cast<uint4*>(mc_smem);   // [kMcRows][256] thresholds
-  float4* sw = mc_smem + kMcRows * 256;            // [kMcRows][256] step weights
-  __shared__ __align__(16) float red[2][8][kMcCols];
+  constexpr int NT = NW * 32;
+  float4* sw = mc_smem + ROWS * NT;                // [ROWS][NT] step weights
+  __shared__ __align__(16) float red[2][NW][kMcCols];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t c = (int64_t)blockIdx.x * kMcCols + lane * 4;
   const int64_t slab = blockIdx.y, nslabs = gridDim.y;
@@ -235,14 +238,14 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
     g4 = __ldg(reinterpret_cast<const float4*>(gamma + c));
     if (kind == BSP_LAYERNORM) b4 = __ldg(reinterpret_cast<const float4*>(beta + c));
   }
-  // generator block index of this thread's four columns in row (slab*kMcSlab + warp + 8*i) is
+  // generator block index of this thread's four columns in row (slab*NW*ROWS + warp + NW*i) is
   // q0 + i*qstep; rows beyond T keep v = wgt = 0 and contribute nothing whatever word they draw
-  const uint64_t q0 = (uint64_t)((slab * kMcSlab + warp) * C + (col_ok ? c : 0)) >> 2;
-  const uint64_t qstep = (uint64_t)(2 * C);
+  const uint64_t q0 = (uint64_t)((slab * (NW * ROWS) + warp) * C + (col_ok ? c : 0)) >> 2;
+  const uint64_t qstep = (uint64_t)(NW * C) / 4;
   float base[4] = {0.f, 0.f, 0.f, 0.f};                 // the draw-independent part of this thread's sums
 #pragma unroll 1
-  for (int i = 0; i < kMcRows; ++i) {
-    const int64_t r = slab * kMcSlab + warp + 8 * i;
+  for (int i = 0; i < ROWS; ++i) {
+    const int64_t r = slab * (NW * ROWS) + warp + NW * i;
     uint32_t thr[4] = {0u, 0u, 0u, 0u};
     float wgt[4] = {0.f, 0.f, 0.f, 0.f};
     if (r < T && col_ok) {
@@ -268,17 +271,17 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
         wgt[e] = thr[e] ? (hi - lo) * inv_scale * w : 0.f;      // (NaN has threshold 0: it stays in base)
       }
     }
-    sp[i * 256 + tid] = make_uint4(thr[0], thr[1], thr[2], thr[3]);
-    sw[i * 256 + tid] = make_float4(wgt[0], wgt[1], wgt[2], wgt[3]);
+    sp[i * NT + tid] = make_uint4(thr[0], thr[1], thr[2], thr[3]);
+    sw[i * NT + tid] = make_float4(wgt[0], wgt[1], wgt[2], wgt[3]);
   }
   for (int k = 0; k < ndraws; ++k) {
     const uint32_t draw = (uint32_t)(draw_begin + k);
     float acc[4] = {base[0], base[1], base[2], base[3]};
 #pragma unroll 2
-    for (int i = 0; i < kMcRows; ++i) {
+    for (int i = 0; i < ROWS; ++i) {
       const uint4 w = philox_block(key, q0 + (uint64_t)i * qstep, draw);
-      const uint4 p4 = sp[i * 256 + tid];
-      const float4 w4 = sw[i * 256 + tid];
+      const uint4 p4 = sp[i * NT + tid];
+      const float4 w4 = sw[i * NT + tid];
       acc[0] += w.x < p4.x ? w4.x : 0.f;
       acc[1] += w.y < p4.y ? w4.y : 0.f;
       acc[2] += w.z < p4.z ? w4.z : 0.f;
@@ -290,7 +293,7 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
     if (tid < kMcCols) {
       float s = 0.f;
 #pragma unroll
-      for (int w8 = 0; w8 < 8; ++w8) s += red[buf][w8][tid];
+      for (int w8 = 0; w8 < NW; ++w8) s += red[buf][w8][tid];
       const int64_t cc = (int64_t)blockIdx.x * kMcCols + tid;
       if (cc < C) partial[((size_t)k * nslabs + slab) * C + cc] = s;
     }
@@ -434,15 +437,34 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
 }
 
 size_t bsp_norm_gain_mc_workspace_bytes(int64_t T, int64_t C, int K) {
-  if (T <= 0 || C <= 0 || K <= 0) return 0;
-  const size_t nslabs = (size_t)((T + kMcSlab - 1) / kMcSlab);
-  const size_t kc = (size_t)(K < kMcChunk ? K : kMcChunk);
-  return round_up(kc * nslabs * (size_t)C * sizeof(float), 256) + round_up(kc * (size_t)C * sizeof(float), 256);
+  return bsp::norm_gain_mc_workspace(T, C, K, false);
 }
 
 int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
                      const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q, bsp_key_t key,
                      int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
+                     bsp_diag_t* diag, void* stream) {
+  return bsp::norm_gain_mc_run(false, kind, x, dt, T, C, gamma, beta, rstd, mean, du, du_dt, q, key, draw0, K, g_ref, S1,
+                               S2, ws, ws_bytes, diag, stream);
+}
+
+}  // extern "C"
+
+namespace bsp {
+
+size_t norm_gain_mc_workspace(int64_t T, int64_t C, int K, bool thin) {
+  if (T <= 0 || C <= 0 || K <= 0) return 0;
+  const int slab_rows = thin ? kMcThinWarps * kMcThinRows : kMcSlab;
+  const size_t nslabs = (size_t)((T + slab_rows - 1) / slab_rows);
+  const size_t kc = (size_t)(K < kMcChunk ? K : kMcChunk);
+  return round_up(kc * nslabs * (size_t)C * sizeof(float), 256) + round_up(kc * (size_t)C * sizeof(float), 256);
+}
+
+// thin: the variant of the kernel made to run beside a kernel that fills the SMs (128 threads, 16 KB
+// of shared memory, 64 registers: one block fits next to a CTA of the Monte-Carlo contraction).
+int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                     const float* beta, const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q,
+                     bsp_key_t key, int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
                      bsp_diag_t* diag, void* stream) {
   (void)diag;
   if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(q.fmt, 1)) return BSP_ERR_ARG;
@@ -453,10 +475,11 @@ int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, cons
   if (T > 0 && (!x || !gamma || !rstd || !du || (kind == BSP_LAYERNORM && (!beta || !mean)))) return BSP_ERR_ARG;
   if (C % 4 != 0) return BSP_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(du) || !aligned16(gamma) || !aligned16(beta)) return BSP_ERR_ALIGN;
-  if (!ws || ws_bytes < bsp_norm_gain_mc_workspace_bytes(T, C, K) || (reinterpret_cast<uintptr_t>(ws) & 255u))
+  if (!ws || ws_bytes < norm_gain_mc_workspace(T, C, K, thin) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return BSP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
-  const int nslabs = (int)((T + kMcSlab - 1) / kMcSlab);
+  const int slab_rows = thin ? kMcThinWarps * kMcThinRows : kMcSlab;
+  const int nslabs = (int)((T + slab_rows - 1) / slab_rows);
   const int kc_max = K < kMcChunk ? K : kMcChunk;
   float* partial = reinterpret_cast<float*>(ws);
   float* gk = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) +
@@ -468,9 +491,14 @@ int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, cons
       dim3 grid((unsigned)((C + kMcCols - 1) / kMcCols), (unsigned)nslabs);
 #define BSP_GM(DT, DU, FMT)                                                                                     \
   do {                                                                                                          \
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(gain_mc_kernel<DT, DU, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+    if (thin) {                                                                                                 \
+      gain_mc_kernel<DT, DU, FMT, kMcThinWarps, kMcThinRows><<<grid, kMcThinWarps * 32, kMcThinSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du, \
+                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd, partial); \
+      break;                                                                                                    \
+    }                                                                                                           \
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(gain_mc_kernel<DT, DU, FMT, 8, kMcRows>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                         (int)kMcSmemBytes));                                                    \
-    gain_mc_kernel<DT, DU, FMT><<<grid, 256, kMcSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
+    gain_mc_kernel<DT, DU, FMT, 8, kMcRows><<<grid, 256, kMcSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
                                                                  q.scale, q.scale_dev, pk, draw0 + kb, nd,      \
                                                                  partial);                                      \
   } while (0)
@@ -497,7 +525,7 @@ int bsp_norm_gain_mc(int kind, const void* x, int dt, int64_t T, int64_t C, cons
   return BSP_OK;
 }
 
-}  // extern "C"
+}  // namespace bsp
 
 // ------------------------------------------------------------------------------- no-allocation variant
 
