@@ -951,6 +951,25 @@ __global__ void mc_accumulate_kernel(const float* __restrict__ g, const float* _
   reinterpret_cast<float4*>(S2)[i] = s2;
 }
 
+// The same over nd draws held back to back (g[d * stride + i]), in draw order: one launch instead of
+// nd for a tensor as small as the correction term.
+__global__ void mc_accumulate_draws_kernel(const float* __restrict__ g, size_t stride, int nd,
+                                           const float* __restrict__ ref, float* __restrict__ S1,
+                                           float* __restrict__ S2, size_t n4) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  const float4 r = __ldg(reinterpret_cast<const float4*>(ref) + i);
+  float4 s1 = reinterpret_cast<float4*>(S1)[i], s2 = reinterpret_cast<float4*>(S2)[i];
+  for (int d = 0; d < nd; ++d) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(g + (size_t)d * stride) + i);
+    const float d0 = a.x - r.x, d1 = a.y - r.y, d2 = a.z - r.z, d3 = a.w - r.w;
+    s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
+    s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y); s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
+  }
+  reinterpret_cast<float4*>(S1)[i] = s1;
+  reinterpret_cast<float4*>(S2)[i] = s2;
+}
+
 // ------------------------------------------------------------------------------- host side
 
 // FP32 output [BH][S][64] as two 32-column boxes per 128-row block (128-byte swizzle).
@@ -1399,14 +1418,21 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
     }
     // dV does not read the correction term: its value under the fresh read is the same for every
     // draw, so it is computed with the first draw only and enters the sums K times
+    // the sums of D itself over all K draws, in one launch (rows = B*H*S is a multiple of 4 or the
+    // draws go one by one)
+    if (rows % 4 == 0) {
+      mc_accumulate_draws_kernel<<<(unsigned)((rows / 4 + 255) / 256), 256, 0, st>>>(b.d_draws, rows, K, b.d_ref, b.S1d,
+                                                                                   b.S2d, rows / 4);
+      BSP_LAUNCH_CHECK();
+    }
     for (int k = 0; k < K; ++k) {
       const float* dk_ = b.d_draws + (size_t)k * rows;
-      BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
+      if (rows % 4 != 0) BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
       if (k > 0) {
         // the draws after the first, two at a time: dQ and dK go from the accumulators straight into
         // their sums
         const int nd = k + 1 < K ? 2 : 1;
-        if (nd == 2) BSP_TRY(bsp_mc_accumulate(dk_ + rows, b.d_ref, b.S1d, b.S2d, rows, st));
+        if (nd == 2 && rows % 4 != 0) BSP_TRY(bsp_mc_accumulate(dk_ + rows, b.d_ref, b.S1d, b.S2d, rows, st));
         BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, nd,
                                   b.g_ref[0], b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
         k += nd - 1;
