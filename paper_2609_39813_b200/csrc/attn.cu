@@ -1416,8 +1416,6 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S1[t], 0, n * 4, st));
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S2[t], 0, n * 4, st));
     }
-    // dV does not read the correction term: its value under the fresh read is the same for every
-    // draw, so it is computed with the first draw only and enters the sums K times
     // the sums of D itself over all K draws, in one launch (rows = B*H*S is a multiple of 4 or the
     // draws go one by one)
     if (rows % 4 == 0) {
@@ -1438,6 +1436,9 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* result
         k += nd - 1;
         continue;
       }
+      // the first draw: the whole backward, gradients written.  dV does not read the correction
+      // term, so its value under the fresh read is the same for every draw: it is computed here only
+      // and enters the sums K times
       BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],
                                  b.g_pol[1], b.g_pol[2], diag, st));
       for (int t = 0; t < 2; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
