@@ -308,7 +308,7 @@ quant_tile_kernel(Producer prod, const void* __restrict__ x, int64_t rows, int64
 // FP32 value of every element is formed once, then rounded stochastically once per draw; only the
 // transposed code matrices are written: codes_t[d][c][r], d-th matrix at d * cols * ld_t.
 template <int DT, int FMT>
-__global__ void __launch_bounds__(256, 2)
+__global__ void __launch_bounds__(256, 3)
 reround_draws_kernel(NormProducer prod, const void* __restrict__ x, int64_t rows, int64_t cols, float scale_val,
                      const float* __restrict__ scale_dev, PhiloxKey key, int draw0, int ndraws,
                      uint8_t* __restrict__ codes_t, int64_t ld_t) {
