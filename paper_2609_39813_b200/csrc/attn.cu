@@ -835,14 +835,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(d[0]), "f"(d[1]), "f"(d[2]), "f"(d[3]) : "memory");
             asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg2 + off), "f"(q[0]), "f"(q[1]), "f"(q[2]), "f"(q[3]) : "memory");
           }
-          continue;
-        }
+        } else {
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
-          asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(__uint_as_float(a[4 * t]) * mul),
-                       "f"(__uint_as_float(a[4 * t + 1]) * mul), "f"(__uint_as_float(a[4 * t + 2]) * mul),
-                       "f"(__uint_as_float(a[4 * t + 3]) * mul) : "memory");
+          for (int t = 0; t < 8; ++t) {
+            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + off), "f"(__uint_as_float(a[4 * t]) * mul),
+                         "f"(__uint_as_float(a[4 * t + 1]) * mul), "f"(__uint_as_float(a[4 * t + 2]) * mul),
+                         "f"(__uint_as_float(a[4 * t + 3]) * mul) : "memory");
+          }
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
