@@ -27,7 +27,8 @@ constexpr int kStages = 4;
 constexpr int kABytes = BM * BKB, kBBytes = BN * BKB, kStageBytes = kABytes + kBBytes;
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kEpiStage = 4 * 4096;              // one 32-row x 128-byte staging block per epilogue warp
+constexpr size_t kGemmSmem = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiStage;
 
 struct GemmParams {
   int M, N, K;            // K in elements
@@ -72,6 +73,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t bars = tiles + kStages * kStageBytes;              // barriers after the ring
   // barrier layout (8 bytes each): full[kStages], empty[kStages], tfull[2], tempty[2]; then tmem slot, abort flag
   const uint32_t full0 = bars, empty0 = bars + 8 * kStages, tfull0 = bars + 16 * kStages, tempty0 = tfull0 + 16;
+  const uint32_t epi_stage = bars + 256;                            // staging blocks of the epilogue warps
   uint8_t* bars_gen = smem_raw + (bars - raw);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 16 * kStages + 32);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 16 * kStages + 36);
@@ -190,19 +192,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           if (col0 >= p.N) break;                // warp-uniform
           uint32_t r[32];
           tmem_ld32(taddr + ch * 32, r);
+          if (p.mode == EPI_STORE_F32) {
+            // A lane holds 128 bytes of its own row; written as they are, a warp's store touches 32
+            // rows with 16 bytes each.  Through the warp's 4 KB staging block the warp instead writes
+            // four rows of 128 contiguous bytes per instruction (row 4 t + lane / 8, chunk lane % 8).
+            const uint32_t wb = epi_stage + (uint32_t)(warp - 2) * 4096u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(wb + (uint32_t)lane * 128u + ((uint32_t)(j ^ (lane & 7)) << 4)),
+                           "f"(__uint_as_float(r[4 * j]) * inv_a * inv_b), "f"(__uint_as_float(r[4 * j + 1]) * inv_a * inv_b),
+                           "f"(__uint_as_float(r[4 * j + 2]) * inv_a * inv_b), "f"(__uint_as_float(r[4 * j + 3]) * inv_a * inv_b)
+                           : "memory");
+            __syncwarp();
+            float* cbase = reinterpret_cast<float*>(p.C) + (size_t)b * p.M * p.ldc;
+#pragma unroll
+            for (int t8 = 0; t8 < 8; ++t8) {
+              const int rl = 4 * t8 + (lane >> 3), c4 = lane & 7;
+              float4 o;
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
+                           : "r"(wb + (uint32_t)rl * 128u + ((uint32_t)(c4 ^ (rl & 7)) << 4)));
+              const int orow = tm * BM + q * 32 + rl, ocol = col0 + 4 * c4;
+              if (orow < p.M && ocol < p.N) *reinterpret_cast<float4*>(cbase + (size_t)orow * p.ldc + ocol) = o;
+            }
+            __syncwarp();
+          }
           if (row < p.M) {
             const size_t off = (size_t)row * p.ldc + col0;
             if (p.mode == EPI_STORE_F32) {
-              float* dst = reinterpret_cast<float*>(p.C) + (size_t)b * p.M * p.ldc + off;
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                if (col0 + j < p.N) {
-                  float4 o;
-                  o.x = __uint_as_float(r[j]) * inv_a * inv_b; o.y = __uint_as_float(r[j + 1]) * inv_a * inv_b;
-                  o.z = __uint_as_float(r[j + 2]) * inv_a * inv_b; o.w = __uint_as_float(r[j + 3]) * inv_a * inv_b;
-                  *reinterpret_cast<float4*>(dst + j) = o;
-                }
-              }
+              // (stored above, by the warp together)
             } else if (p.mode == EPI_STORE_BF16) {
               uint16_t* dst = reinterpret_cast<uint16_t*>(p.C) + (size_t)b * p.M * p.ldc + off;
 #pragma unroll
