@@ -226,12 +226,29 @@ def attention_section(b, peaks, steps=3):
 
     ms_dkv = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, None, dk, dv, diag))
     ms_dq = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, dq, None, None, diag))
+    # the D pre-pass alone under its three reads (HBM-bound for U and R: dO read once, the copy of O
+    # read once; the fresh read is bound by the generator: one word per element and draw)
+    amax_o, scales_o = torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
+    codes_o = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    b.bsp_amax(o, B * H, S * D, amax_o)
+    b.bsp_scale_from_amax(amax_o, B * H, b.E4M3, scales_o)
+    b.bsp_round_grouped(o, B * H, S * D, b.E4M3, b.ROUND_STOCHASTIC, scales_o, b.key(1003, tensor_o, 0, 0), codes_o)
+    d_draws = torch.zeros(K * B * H * S, device="cuda")
+    kd = b.key(1003, tensor_o, b.STREAM_ATTN_D, 0)
+    ms_du = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_ORIGINAL, kd, 0, 1, dterm))
+    ms_dr = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FORWARD, kd, 0, 1, dterm))
+    ms_dn = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FRESH, kd, 0, K, d_draws))
+    hbm = peaks["hbm_gbs"]
+    dterm_rows = dict(
+        read_U=dict(us=ms_du * 1e3, algorithmic_mb=n * 6 / 1e6, gb_per_s=n * 6 / ms_du / 1e6, frac_of_hbm=n * 6 / ms_du / 1e6 / hbm),
+        read_R=dict(us=ms_dr * 1e3, algorithmic_mb=n * 3 / 1e6, gb_per_s=n * 3 / ms_dr / 1e6, frac_of_hbm=n * 3 / ms_dr / 1e6 / hbm),
+        read_N=dict(us=ms_dn * 1e3, draws=K, g_element_draws_per_s=n * K / ms_dn / 1e6))
     prod = 2.0 * B * H * S * S * D / 2                         # one causal S x S x d product over all heads
     tf_dkv, tf_dq = 4 * prod / (ms_dkv * 1e-3) / 1e12, 3 * prod / (ms_dq * 1e-3) / 1e12
     peak = peaks["bf16_tflops"]
     return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, ms_per_check=ms,
                 check_elements_per_s=elements / (ms * 1e-3), verdicts=[r.verdict for r in res],
-                bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3,
+                bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3, dterm=dterm_rows,
                 roofline=dict(bound="tensor", kernel="attn_kernel<dK/dV> + attn_kernel<dQ> (bf16 operands)",
                               achieved=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
                               frac=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,

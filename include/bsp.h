@@ -318,7 +318,8 @@ int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_sc
 /* The D use: d_out[d][b,h,i] = sum_j dO[b,h,i,j] * O_copy[b,h,i,j] for n_draws draws, with
  * O_copy = o_orig (U), decode(o_codes)/o_scales[b,h] (R), or a fresh stochastic rounding of
  * fl32(o_orig * o_scales[b,h]) in o_fmt under (key, draw0 + d) (N).  U and R write one draw.
- * dO: dt[B,H,S,Dh]; o_scales: one scale per (b,h) slice. */
+ * dO: dt[B,H,S,Dh]; o_scales: one scale per (b,h) slice.  dO and o_orig 16-byte aligned, o_codes
+ * 8-byte aligned (BSP_ERR_ALIGN otherwise). */
 int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig,
                    const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key,
                    int draw0, int n_draws, float* d_out, bsp_diag_t* diag, void* stream);

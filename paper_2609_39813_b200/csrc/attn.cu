@@ -888,50 +888,104 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 
 // ------------------------------------------------------------------------------- D pre-pass
 
-// D[d][row] = sum_j dO[row][j] * O_copy[row][j] for n_draws draws (one for U and R).  16 threads per
-// row of 64, four elements each; U reads the FP32 original, R the forward's codes, N a fresh
-// stochastic rounding of fl32(O * scale[bh]) keyed by the element's index in the whole tensor.
-template <int DT, int FMT>
+// D[d][row] = sum_j dO[row][j] * O_copy[row][j] for n_draws draws (one for U and R).  Eight lanes per
+// row of 64, eight elements each; a thread takes kDtRows rows (32 rows apart) and issues all their
+// loads before it uses any.  U reads the FP32 original, R the forward's codes, N a fresh stochastic
+// rounding of fl32(O * scale[bh]) keyed by the element's index in the whole tensor.  For N the
+// rounding of an element is its round-down value plus, when the generator word is below the
+// element's threshold (f8_sr_threshold), one grid step: per element the product of dO with the
+// round-down value goes into a sum shared by all draws, and a draw costs one comparison and one
+// conditional add of dO * step.
+template <int DT, int FMT, int kDtRows>
 __global__ void __launch_bounds__(256)
 attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig, const uint8_t* __restrict__ o_codes,
                   const float* __restrict__ o_scales, const float* __restrict__ do_scales, int64_t rows, int S,
                   int policy, PhiloxKey key, int draw0, int n_draws, float* __restrict__ D) {
-  const int64_t row = (int64_t)blockIdx.x * 16 + (threadIdx.x >> 4);
-  const int sub = threadIdx.x & 15;
-  const bool active = row < rows;
-  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), o = g;
-  float scale = 1.f, inv = 1.f;
-  const size_t i0 = (size_t)(active ? row : 0) * AT_D + sub * 4;
-  if (active) {
-    g = load4<DT>(dO, i0);
+  const int sub = threadIdx.x & 7;
+  const int64_t row0 = (int64_t)blockIdx.x * (32 * kDtRows) + (threadIdx.x >> 3);
+  float g[kDtRows][8], o[kDtRows][8], scale[kDtRows], inv[kDtRows];
+  bool active[kDtRows];
+  size_t i0[kDtRows];
+#pragma unroll
+  for (int m = 0; m < kDtRows; ++m) {
+    const int64_t row = row0 + 32 * m;
+    active[m] = row < rows;
+    i0[m] = (size_t)(active[m] ? row : 0) * AT_D + sub * 8;
+    const float4 g0 = load4<DT>(dO, i0[m]), g1 = load4<DT>(dO, i0[m] + 4);
+    g[m][0] = g0.x; g[m][1] = g0.y; g[m][2] = g0.z; g[m][3] = g0.w;
+    g[m][4] = g1.x; g[m][5] = g1.y; g[m][6] = g1.z; g[m][7] = g1.w;
+    if (policy == BSP_READ_FORWARD) {
+      const uint2 pk = __ldg(reinterpret_cast<const uint2*>(o_codes + i0[m]));
+      float d0[4], d1[4];
+      f8_decode4<FMT>(pk.x, d0);
+      f8_decode4<FMT>(pk.y, d1);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { o[m][j] = d0[j]; o[m][4 + j] = d1[j]; }
+    } else {
+      const float4 a0 = __ldg(reinterpret_cast<const float4*>(o_orig + i0[m]));
+      const float4 a1 = __ldg(reinterpret_cast<const float4*>(o_orig + i0[m] + 4));
+      o[m][0] = a0.x; o[m][1] = a0.y; o[m][2] = a0.z; o[m][3] = a0.w;
+      o[m][4] = a1.x; o[m][5] = a1.y; o[m][6] = a1.z; o[m][7] = a1.w;
+    }
+  }
+#pragma unroll
+  for (int m = 0; m < kDtRows; ++m) {
+    const int64_t row = active[m] ? row0 + 32 * m : 0;
+    scale[m] = o_scales ? __ldg(o_scales + row / S) : 1.f;
+    inv[m] = __fdiv_rn(1.0f, scale[m]);
     if (do_scales) {
       // dO holds decoded FP8 codes: bring back its per-(b,h) scale
       const float inv_do = __fdiv_rn(1.0f, __ldg(do_scales + row / S));
-      g.x *= inv_do; g.y *= inv_do; g.z *= inv_do; g.w *= inv_do;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) g[m][j] *= inv_do;
     }
-    scale = o_scales ? __ldg(o_scales + row / S) : 1.f;
-    inv = __fdiv_rn(1.0f, scale);
     if (policy == BSP_READ_FORWARD) {
-      const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(o_codes + i0));
-      o = make_float4(f8_decode<FMT>(pk & 0xFFu) * inv, f8_decode<FMT>((pk >> 8) & 0xFFu) * inv,
-                      f8_decode<FMT>((pk >> 16) & 0xFFu) * inv, f8_decode<FMT>(pk >> 24) * inv);
-    } else {
-      o = __ldg(reinterpret_cast<const float4*>(o_orig + i0));
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o[m][j] *= inv[m];
     }
   }
-  for (int d = 0; d < n_draws; ++d) {
-    float4 c = o;
-    if (policy == BSP_READ_FRESH) {
-      const uint4 w = philox_block(key, (uint64_t)i0 >> 2, (uint32_t)(draw0 + d));
-      c.x = f8_sr_value<FMT>(__fmul_rn(o.x, scale), w.x) * inv;
-      c.y = f8_sr_value<FMT>(__fmul_rn(o.y, scale), w.y) * inv;
-      c.z = f8_sr_value<FMT>(__fmul_rn(o.z, scale), w.z) * inv;
-      c.w = f8_sr_value<FMT>(__fmul_rn(o.w, scale), w.w) * inv;
-    }
-    float s = (g.x * c.x + g.y * c.y) + (g.z * c.z + g.w * c.w);
+  auto reduce_store = [&](int m, int d, float s) {
 #pragma unroll
-    for (int off = 8; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-    if (active && sub == 0) D[(size_t)d * rows + row] = s;
+    for (int off = 4; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+    if (active[m] && sub == 0) D[(size_t)d * rows + row0 + 32 * m] = s;
+  };
+  if (policy != BSP_READ_FRESH) {
+#pragma unroll
+    for (int m = 0; m < kDtRows; ++m) {
+      const float s = ((g[m][0] * o[m][0] + g[m][1] * o[m][1]) + (g[m][2] * o[m][2] + g[m][3] * o[m][3])) +
+                      ((g[m][4] * o[m][4] + g[m][5] * o[m][5]) + (g[m][6] * o[m][6] + g[m][7] * o[m][7]));
+      reduce_store(m, 0, s);
+    }
+    return;
+  }
+  // fresh read: per element the threshold and dO * step; the draw-independent part summed once
+  uint32_t thr[kDtRows][8];
+  float base[kDtRows];
+#pragma unroll
+  for (int m = 0; m < kDtRows; ++m) {
+    float bs = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float v = __fmul_rn(o[m][j], scale[m]);
+      const float lo = f8_sr_value<FMT>(v, 0xFFFFFFFFu) * inv[m], hi = f8_sr_value<FMT>(v, 0u) * inv[m];
+      thr[m][j] = f8_sr_threshold<FMT>(v);
+      bs = fmaf(g[m][j], lo, bs);
+      o[m][j] = thr[m][j] ? g[m][j] * (hi - lo) : 0.f;      // reuse: dO * step (a NaN stays in the shared sum)
+    }
+    base[m] = bs;
+  }
+  for (int d = 0; d < n_draws; ++d) {
+#pragma unroll
+    for (int m = 0; m < kDtRows; ++m) {
+      const uint4 w0 = philox_block(key, (uint64_t)i0[m] >> 2, (uint32_t)(draw0 + d));
+      const uint4 w1 = philox_block(key, ((uint64_t)i0[m] >> 2) + 1, (uint32_t)(draw0 + d));
+      float s = base[m];
+      s += w0.x < thr[m][0] ? o[m][0] : 0.f; s += w0.y < thr[m][1] ? o[m][1] : 0.f;
+      s += w0.z < thr[m][2] ? o[m][2] : 0.f; s += w0.w < thr[m][3] ? o[m][3] : 0.f;
+      s += w1.x < thr[m][4] ? o[m][4] : 0.f; s += w1.y < thr[m][5] ? o[m][5] : 0.f;
+      s += w1.z < thr[m][6] ? o[m][6] : 0.f; s += w1.w < thr[m][7] ? o[m][7] : 0.f;
+      reduce_store(m, d, s);
+    }
   }
 }
 
@@ -1114,14 +1168,21 @@ static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, 
   if (d_read == BSP_READ_FORWARD ? (!o_codes || !o_scales) : !o_orig) return BSP_ERR_ARG;
   if (d_read == BSP_READ_FRESH && !o_scales) return BSP_ERR_ARG;
   if (d_read != BSP_READ_FRESH) n_draws = 1;
-  if (!aligned16(dO) || !aligned16(o_orig) || (reinterpret_cast<uintptr_t>(o_codes) & 3u)) return BSP_ERR_ALIGN;
+  if (!aligned16(dO) || !aligned16(o_orig) || (reinterpret_cast<uintptr_t>(o_codes) & 7u)) return BSP_ERR_ALIGN;
   const int64_t rows = (int64_t)B * H * S;
-  const unsigned grid = (unsigned)((rows + 15) / 16);
+  const int nr = 2;                                  // (four rows per thread measured slower for U and R)
+  const unsigned grid = (unsigned)((rows + 32 * nr - 1) / (32 * nr));
   cudaStream_t st = (cudaStream_t)stream;
   const PhiloxKey pk = make_key(key);
 #define BSP_DT(DT, FMT)                                                                                          \
-  attn_dterm_kernel<DT, FMT><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read,    \
-                                                   pk, draw0, n_draws, d_out)
+  do {                                                                                                           \
+    if (nr == 2)                                                                                                 \
+      attn_dterm_kernel<DT, FMT, 2><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read, \
+                                                          pk, draw0, n_draws, d_out);                            \
+    else                                                                                                         \
+      attn_dterm_kernel<DT, FMT, 4><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read, \
+                                                          pk, draw0, n_draws, d_out);                            \
+  } while (0)
   if (dt == BSP_F32 && o_fmt == BSP_E4M3) BSP_DT(BSP_F32, BSP_E4M3);
   else if (dt == BSP_F32) BSP_DT(BSP_F32, BSP_E5M2);
   else if (o_fmt == BSP_E4M3) BSP_DT(BSP_BF16, BSP_E4M3);
