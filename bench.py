@@ -243,12 +243,30 @@ def attention_section(b, peaks, steps=3):
         read_U=dict(us=ms_du * 1e3, algorithmic_mb=n * 6 / 1e6, gb_per_s=n * 6 / ms_du / 1e6, frac_of_hbm=n * 6 / ms_du / 1e6 / hbm),
         read_R=dict(us=ms_dr * 1e3, algorithmic_mb=n * 3 / 1e6, gb_per_s=n * 3 / ms_dr / 1e6, frac_of_hbm=n * 3 / ms_dr / 1e6 / hbm),
         read_N=dict(us=ms_dn * 1e3, draws=K, g_element_draws_per_s=n * K / ms_dn / 1e6))
+    # the forward helper, and mode A of the config (FP8 operands: quantise Q, K, V, dO per (b,h) slice,
+    # then the whole backward with P and dS rounded onto the FP8 grids inside the kernels)
+    ms_fwd = timed(lambda: b.bsp_attn_fwd_stats(B, H, S, D, True, 0.125, q, k, v, o, lse, diag))
+    hatq, amq, scq = torch.zeros(n, dtype=torch.bfloat16, device="cuda"), torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
+    ms_quant = timed(lambda: b.bsp_attn_quantize(q, B * H, S * D, b.E4M3, hatq, amq, scq))
+    ops = {}
+    for nm, src, fmt in (("q", q, b.E4M3), ("k", k, b.E4M3), ("v", v, b.E4M3), ("dO", dO, b.E5M2)):
+        xq, am, sc = torch.zeros(n, dtype=torch.bfloat16, device="cuda"), torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
+        b.bsp_attn_quantize(src, B * H, S * D, fmt, xq, am, sc)
+        ops[nm] = (xq, sc)
+    f8 = b.attn_fp8(ops["q"][1], ops["k"][1], ops["v"][1], ops["dO"][1], 256.0, 1024.0)
+    o8, lse8 = torch.zeros(n, device="cuda"), torch.zeros(B * H * S, device="cuda")
+    b.bsp_attn_fwd_stats_fp8(B, H, S, D, True, 0.125, ops["q"][0], ops["k"][0], ops["v"][0], f8, o8, lse8, diag)
+    d8 = torch.zeros(B * H * S, device="cuda")
+    ms_fp8 = timed(lambda: b.bsp_attn_bwd_fp8(B, H, S, D, True, 0.125, ops["q"][0], ops["k"][0], ops["v"][0], ops["dO"][0],
+                                              f8, lse8, o8, None, None, b.E4M3, b.READ_ORIGINAL, kd, dq, dk, dv, d8, diag))
     prod = 2.0 * B * H * S * S * D / 2                         # one causal S x S x d product over all heads
     tf_dkv, tf_dq = 4 * prod / (ms_dkv * 1e-3) / 1e12, 3 * prod / (ms_dq * 1e-3) / 1e12
     peak = peaks["bf16_tflops"]
     return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, ms_per_check=ms,
                 check_elements_per_s=elements / (ms * 1e-3), verdicts=[r.verdict for r in res],
                 bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3, dterm=dterm_rows,
+                fwd_stats_us=ms_fwd * 1e3, quantize_one_tensor_us=ms_quant * 1e3,
+                bwd_fp8_operands_us=ms_fp8 * 1e3,   # D pre-pass + dK/dV + dQ kernels, FP8-operand mode
                 roofline=dict(bound="tensor", kernel="attn_kernel<dK/dV> + attn_kernel<dQ> (bf16 operands)",
                               achieved=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
                               frac=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,

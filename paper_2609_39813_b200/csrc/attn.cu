@@ -86,6 +86,19 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return d;
 }
 
+// Two floats rounded to the nearest FP8 grid value (ties to even, saturating: what f8_rn_value
+// gives) and packed as a bf16 pair, through the hardware conversions: f32 pair -> FP8 pair -> f16 pair
+// (every FP8 value is an f16 value) -> f32 -> bf16 pair (every FP8 value is a bf16 value too).
+template <int FMT>
+__device__ __forceinline__ uint32_t f8_grid_bf16x2(float lo, float hi) {
+  const uint16_t c = (uint16_t)f8_encode_rn_pair_inrange<FMT>(lo, hi);
+  uint32_t h2;
+  if (FMT == BSP_E4M3) asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(c));
+  else asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h2) : "h"(c));
+  const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+  return pack_bf16x2(f.x, f.y);
+}
+
 // tcgen05.ld of 32 columns without the wait, so several loads can be in flight before one wait.
 __device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -564,8 +577,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
           }
           if (FP8 && MODE != AT_FWD) {                      // the forward keeps P unrounded
-            p0 = f8_rn_value<BSP_E4M3>(p0 * p.p_scale); p1 = f8_rn_value<BSP_E4M3>(p1 * p.p_scale);
-            s0 = f8_rn_value<BSP_E5M2>(s0 * p.ds_scale); s1 = f8_rn_value<BSP_E5M2>(s1 * p.ds_scale);
+            po = f8_grid_bf16x2<BSP_E4M3>(p0 * p.p_scale, p1 * p.p_scale);
+            dso = f8_grid_bf16x2<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);
+            return;
           }
           po = pack_bf16x2(p0, p1);
           if (MODE != AT_FWD) dso = pack_bf16x2(s0, s1);
