@@ -333,6 +333,7 @@ def kernel_table(b, peaks):
     t("norm_fwd store, stochastic, codes + transposed", "alu", lambda: b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, codes_t, T), T * C * 4)
     t("norm_bwd read U: dgamma, dbeta, dx", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 0, codes, q, k, dg, db, dx, ws), T * C * 8)
     t("norm_bwd read R: dgamma", "hbm", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 1, codes, q, k, dg, None, None, ws), T * C * 5)
+    t("norm_bwd read N: dgamma, one fresh draw", "alu", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 2, codes, q, k, dg, None, None, ws), T * C * 4)
     t("mc_stats (45 M elements, fresh)", "hbm", lambda: b.bsp_mc_stats(ref, ref, S2, O * C, 16, 1, wss), O * C * 12)
     # ---- the K-draw kernels and the contractions at the same shape (K = 16 draws, as config 5)
     Kd = 16
