@@ -505,18 +505,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       const int qb0 = (MODE == AT_DKV ? step : blk) * AT_BLK;  // first query of this step's score tile
       if (MODE == AT_FWD && it == nsteps) {
-        // between the passes: combine the two column halves of every row into the row's LSE
+        // between the passes: the row's maximum over both column halves.  The second pass forms
+        // exp2(c2 s - max) (no exponential is spent in the first pass), sums it per row and divides
+        // the output by that sum at the end, where the LSE is written too.
         float* xm = xchg;                                     // [2][128] max, then [2][128] sum
         xm[h * 128 + r] = run_m;
-        xm[256 + h * 128 + r] = run_l;
         named_bar_sync(1, 256);
-        const float m0 = xm[r], m1 = xm[128 + r], l0 = xm[256 + r], l1 = xm[384 + r];
-        const float m = fmaxf(m0, m1);
-        float l = 0.f;
-        if (m0 > -INFINITY) l += l0 * exp2f(m0 - m);
-        if (m1 > -INFINITY) l += l1 * exp2f(m1 - m);
-        lse2 = m + log2f(l);                                  // in units of log2: LSE * log2(e)
-        if (h == 0 && qrow < p.S) p.lse_out[(size_t)bh * p.S + qrow] = lse2 / kLog2e;
+        lse2 = fmaxf(xm[r], xm[128 + r]);                     // the shift of the second pass, in units of log2
+        run_l = 0.f;
         named_bar_sync(1, 256);
       }
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sdp_full, ip, abort_flag));
@@ -545,7 +541,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const bool edge = (p.causal && kblk * AT_BLK + AT_BLK - 1 > qb0) || (kblk + 1) * AT_BLK > p.S ||
                         qb0 + AT_BLK > p.S;
       if (MODE == AT_FWD && !pass2) {
-        // running max / sum of exp2(c2 * s) over the valid keys of this half
+        // running max of c2 * s over the valid keys of this half
         float mloc = run_m;
 #pragma unroll
         for (int j = 0; j < 64; ++j) {
@@ -553,17 +549,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const bool valid = !edge || (key < p.S && qrow < p.S && (!p.causal || key <= qrow));
           if (valid) mloc = fmaxf(mloc, __uint_as_float(sv[j]) * c2);
         }
-        if (mloc > -INFINITY) {
-          float add = 0.f;
-#pragma unroll
-          for (int j = 0; j < 64; ++j) {
-            const int key = key0 + j;
-            const bool valid = !edge || (key < p.S && qrow < p.S && (!p.causal || key <= qrow));
-            add += ex2_approx(valid ? fmaf(__uint_as_float(sv[j]), c2, -mloc) : -INFINITY);
-          }
-          run_l = run_l * (run_m > -INFINITY ? ex2_approx(run_m - mloc) : 0.f) + add;
-          run_m = mloc;
-        }
+        run_m = mloc;
       } else {
         uint32_t pk[32], dk[32];
         // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
@@ -572,6 +558,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, float d0, float d1, uint32_t& po,
                              uint32_t& dso) {
           float s0 = 0.f, s1 = 0.f;
+          if (MODE == AT_FWD) run_l += p0 + p1;             // the row's normaliser, from the unrounded values
           if (MODE != AT_FWD) {
             s0 = p0 * (__uint_as_float(dp0) * dp_mul - d0);
             s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
@@ -764,6 +751,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
     }
     itg += (uint32_t)total;
+    float fwd_inv_l = 1.f;
+    if (MODE == AT_FWD) {
+      // the row's normaliser over both column halves; the LSE in natural-log units
+      float* xm = xchg;
+      xm[256 + h * 128 + r] = run_l;
+      named_bar_sync(1, 256);
+      const float l = xm[256 + r] + xm[384 + r];
+      fwd_inv_l = __fdividef(1.0f, l);
+      if (h == 0 && qrow < p.S) p.lse_out[(size_t)bh * p.S + qrow] = (lse2 + log2f(l)) / kLog2e;
+    }
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise), 32 KB at a
     // time through the item's resident-tile buffer (no product reads it any more): every thread puts
     // its row's 32 FP32 values of column half h into the 128-byte-swizzle box that a tiled bulk store
@@ -819,7 +816,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         float mul;
         if (MODE == AT_DKV) mul = o == 0 ? (FP8 ? inv_do / p.p_scale : 1.f) : p.c * (FP8 ? inv_q / p.ds_scale : 1.f);
         else if (MODE == AT_DQ) mul = p.c * (FP8 ? inv_k / p.ds_scale : 1.f);
-        else mul = inv_v;
+        else mul = inv_v * fwd_inv_l;
         uint32_t a[32], a2[ND == 2 ? 32 : 1];
         tmem_ld32((o == 0 ? t_acc0 : t_acc1) + lane_off + h * 32, a);
         if (ND == 2) tmem_ld32((o == 0 ? t_acc1 : t_acc0) + lane_off + h * 32, *reinterpret_cast<uint32_t(*)[32]>(&a2[0]));
