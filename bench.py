@@ -426,8 +426,28 @@ def kernel_table(b, peaks):
     ms = e0.elapsed_time(e1) / 3
     whole = dict(K=Kd, ms_per_check=ms, check_elements_per_s=check_elements(T, C, Kd) / (ms * 1e-3),
                  verdicts=[int(r.verdict) for r in res])
+    # ---- config 4 as it is defined (LayerNorm, FP32 inputs, Student-t values, K = 1024): the whole check
+    del wsc, Wc, x, dY
+    torch.cuda.empty_cache()
+    from paper_2609_39813_b200 import workloads
+    from paper_2609_39813_b200.harness import NormLinearGpu
+    inp4 = workloads.config4()
+    g4 = NormLinearGpu(inp4)
+    d4 = g4.desc()
+    ws4 = b.workspace(b.bsp_mc_check_workspace_bytes(d4, inp4.K))
+    res4 = b.bsp_mc_check(d4, inp4.K, ws4, diag)
+    e0.record(stream)
+    for _ in range(2):
+        res4 = b.bsp_mc_check(d4, inp4.K, ws4, diag)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms4 = e0.elapsed_time(e1) / 2
+    cfg4 = dict(T=inp4.T, C=inp4.C, O=inp4.O, K=inp4.K, ms_per_check=ms4,
+                check_elements_per_s=check_elements(inp4.T, inp4.C, inp4.K) / (ms4 * 1e-3),
+                verdicts=[int(r.verdict) for r in res4])
     return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
-                kernels=rows, compute_kernels=compute, whole_check=whole, diag_status=b.read_diag(diag)["status"])
+                kernels=rows, compute_kernels=compute, whole_check=whole, config4_check=cfg4,
+                diag_status=b.read_diag(diag)["status"])
 
 
 def run_ours(args):
