@@ -1181,19 +1181,13 @@ static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, 
   if (d_read != BSP_READ_FRESH) n_draws = 1;
   if (!aligned16(dO) || !aligned16(o_orig) || (reinterpret_cast<uintptr_t>(o_codes) & 7u)) return BSP_ERR_ALIGN;
   const int64_t rows = (int64_t)B * H * S;
-  const int nr = 2;                                  // (four rows per thread measured slower for U and R)
+  constexpr int nr = 2;                              // rows per thread (four measured slower for U and R)
   const unsigned grid = (unsigned)((rows + 32 * nr - 1) / (32 * nr));
   cudaStream_t st = (cudaStream_t)stream;
   const PhiloxKey pk = make_key(key);
 #define BSP_DT(DT, FMT)                                                                                          \
-  do {                                                                                                           \
-    if (nr == 2)                                                                                                 \
-      attn_dterm_kernel<DT, FMT, 2><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read, \
-                                                          pk, draw0, n_draws, d_out);                            \
-    else                                                                                                         \
-      attn_dterm_kernel<DT, FMT, 4><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read, \
-                                                          pk, draw0, n_draws, d_out);                            \
-  } while (0)
+  attn_dterm_kernel<DT, FMT, nr><<<grid, 256, 0, st>>>(dO, o_orig, o_codes, o_scales, do_scales, rows, S, d_read, \
+                                                       pk, draw0, n_draws, d_out)
   if (dt == BSP_F32 && o_fmt == BSP_E4M3) BSP_DT(BSP_F32, BSP_E4M3);
   else if (dt == BSP_F32) BSP_DT(BSP_F32, BSP_E5M2);
   else if (o_fmt == BSP_E4M3) BSP_DT(BSP_BF16, BSP_E4M3);
