@@ -143,23 +143,28 @@ def attention_d_copy(prep, policy, seed, draw, stream=philox.STREAM_ATTN_D):
 
 
 def attention_d_use(q, k, v, dO, c, prep, policy, K, seed, causal=True, outputs=("D", "dq", "dk", "dv"),
-                    operand_round=None):
-    """Attention backward (BF16-operand mode) under one read at the D use, against the
-    reference (D reads the original output).  Returns {name: dict(ref, mean, m2, stats)}."""
-    ref = attention.backward(q, k, v, dO, c, attention_d_copy(prep, U, seed, 0), causal,
-                             operand_round=operand_round)
+                    operand_round=None, fp8_operands=False, scale_p=256.0, scale_ds=None):
+    """Attention backward under one read at the D use, against the reference (D reads the original
+    output).  BF16-operand mode by default (every product in float64 on the given operands,
+    optionally with `operand_round` on P and dS); with `fp8_operands`, q, k, v, dO must be the
+    dequantised FP8 operands and the emulated backward of Appendix "The forks" is evaluated
+    (P rounded at scale_p before dV, dS rounded at scale_ds before dQ and dK).
+    Returns {name: dict(ref, mean, m2, stats)}."""
+    def bwd(copy):
+        return attention.backward(q, k, v, dO, c, copy, causal, fp8_operands=fp8_operands, scale_p=scale_p,
+                                  scale_ds=scale_ds, operand_round=operand_round)
+
+    ref = bwd(attention_d_copy(prep, U, seed, 0))
     out = {}
     if policy in (U, R):
-        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, policy, seed, 0), causal,
-                               operand_round=operand_round)
+        g = bwd(attention_d_copy(prep, policy, seed, 0))
         for name in outputs:
             out[name] = dict(ref=ref[name], mean=g[name], m2=None,
                              stats=mc.statistics(g[name], None, 1, ref[name], False))
         return out
     accs = {name: mc.Welford(ref[name].shape) for name in outputs}
     for kk in range(K):
-        g = attention.backward(q, k, v, dO, c, attention_d_copy(prep, N, seed, kk), causal,
-                               operand_round=operand_round)
+        g = bwd(attention_d_copy(prep, N, seed, kk))
         for name in outputs:
             accs[name].add(g[name])
     for name in outputs:

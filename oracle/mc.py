@@ -72,8 +72,9 @@ class UseStats:
 def statistics(mean, m2, K: int, g_ref, fresh: bool) -> UseStats:
     """Reduce per-element (mean, M2 = sum_k (g_k - mean)^2) against the reference gradient.
 
-    s^2 = M2 / (K - 1); se^2 = s^2 / K; z_j = (m_j - g*_j) / se_j, defined 0 when numerator and
-    se are both 0; R = sum_j (m_j - g*_j)^2 / sum_j se_j^2;
+    s^2 = M2 / (K - 1); se^2 = s^2 / K; z_j = (m_j - g*_j) / se_j; where se_j = 0 (every draw gave
+    the same value: the read is deterministic at that element) z_j = 0 if |m_j - g*_j| is within
+    the deterministic tolerance of |g*_j| and +-inf otherwise; R = sum_j (m_j - g*_j)^2 / sum_j se_j^2;
     Q' = mean_j z_j^2 (K - 3) / (K - 1)  (about one at zero bias: E t^2 of a t_{K-1} is
     (K-1)/(K-3)); rel = ||m - g*||_2 / ||g*||_2.
     A deterministic read (original or forward's rounding) has K_eff = 1 and only `rel`.
@@ -92,7 +93,10 @@ def statistics(mean, m2, K: int, g_ref, fresh: bool) -> UseStats:
     se2 = m2 / (K - 1) / K
     se = np.sqrt(se2)
     with np.errstate(divide="ignore", invalid="ignore"):
-        z = np.where((err == 0.0) & (se == 0.0), 0.0, err / se)
+        # an element whose draws all coincide is read deterministically: it is judged by the
+        # deterministic rule (z = 0 within REL_TOL_DETERMINISTIC of the reference, else +-inf)
+        flat = np.where(np.abs(err) <= REL_TOL_DETERMINISTIC * np.abs(g_ref), 0.0, np.sign(err) * np.inf)
+        z = np.where(se == 0.0, flat, err / se)
     sum_se2 = float(np.sum(se2))
     sum_err2 = float(np.sum(err * err))
     R = 0.0 if sum_err2 == 0.0 else (sum_err2 / sum_se2 if sum_se2 > 0 else float("inf"))
