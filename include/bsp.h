@@ -21,10 +21,20 @@
  *   - device-detected conditions (non-finite inputs, saturated roundings, a bounded wait that
  *     ran out) are accumulated into the caller's device-resident bsp_diag_t, never trapped; the
  *     caller clears it (bsp_diag_clear) and reads it back after synchronising;
- *   - no global mutable state: the same inputs give byte-identical outputs.
+ *   - the same inputs give byte-identical outputs.  State the library keeps per process, none of
+ *     which influences a result: the counters behind bsp_launch_count() and bsp_d2h_byte_count(), the record of which
+ *     kernels already have their shared-memory limit raised on which device, and the fixed scratch
+ *     array of bsp_norm_bwd_noalloc (a 20 MiB device array every GPU that loads the library holds).
+ *     No stream, event or allocation outlives a call.
  *
- * FP8 codes are raw bit patterns (uint8): E4M3 = 1-4-3 bits, bias 7, no infinity, NaN 0x7F/0xFF,
- * max 448; E5M2 = 1-5-2, bias 15, max 57344.  A code stands for decode(code) / scale.
+ * FP8 codes are raw bit patterns (uint8): E4M3 = 1-4-3 bits, bias 7, no infinity, max 448; E5M2 =
+ * 1-5-2, bias 15, max 57344.  Encoding maps every NaN input to the single code 0x7F (the sign of a
+ * NaN is not kept); decoding reads 0x7F / 0xFF (E4M3) and 0x7D..0x7F / 0xFD..0xFF (E5M2) as NaN.
+ * A code stands for decode(code) / scale.
+ *
+ * Shape limits (BSP_ERR_UNSUPPORTED beyond them): normalisation width C a multiple of 4 and at
+ * most 8192; the per-use check of a normalisation -> linear workload needs C and O multiples of
+ * 16; attention needs head dimension 64 and bf16 inputs (FP8-operand mode: uint8 codes).
  */
 #ifndef BSP_H_
 #define BSP_H_
@@ -95,8 +105,9 @@ typedef struct {
 /* Result of one (use, output tensor) evaluation of the check; lives in HOST memory.
  * Statistics: standard error over draws and z = (m - g*) / se (Appendix "Checkpointing");
  * R = ||m - g*||^2 / sum_j se_j^2 (Appendix "The normalization store"); Q' = mean z^2 (K-3)/(K-1);
- * rel = ||m - g*||_2 / ||g*||_2.  Verdict: deterministic read -> HOLDS iff rel <= 1e-4;
- * fresh read -> HOLDS if Q' <= 2 and R <= 3, FAILS if Q' >= 4 or R >= 6, else UNDECIDED. */
+ * rel = ||m - g*||_2 / ||g*||_2.  An element whose draws all coincide (se = 0) is judged as a
+ * deterministic read: z = 0 if its error is within the deterministic tolerance of |g*|, else
+ * +-infinity.  Verdict: see bsp_verdict_rule_t. */
 typedef struct {
   int32_t use_id;            /* BSP_STREAM_* of the use                         */
   int32_t output_id;         /* bsp_output_t                                    */
@@ -111,8 +122,24 @@ typedef struct {
   double max_abs_z;
   double frac_abs_z_gt3;
   int32_t verdict;           /* bsp_verdict_t                                   */
-  int32_t reserved;
+  int32_t informational;     /* 1: statistics reported for information; the use's verdict is the row
+                                of its own output (FP8-operand attention: dQ and dK pass through a
+                                nearest rounding of dS, which is not linear in D)  */
 } bsp_use_result_t;
+
+/* The decision rule of the check.  The paper registers a reading rule per test before measuring
+ * (Appendix "How the three tests were registered": nulls as "z < 2 and under x %", detections as
+ * "z > 5"); this is that template on the pooled statistics.  Deterministic read: HOLDS iff
+ * rel <= rel_tol_deterministic.  Fresh read: FAILS if Q' >= qprime_fail or R >= r_fail; HOLDS if
+ * Q' <= qprime_hold and R <= r_hold and (rel_hold == 0 or rel <= rel_hold); UNDECIDED otherwise.
+ * Passing NULL where a rule is expected selects {1e-4, 2, 3, 4, 6, 0}.  A rule with a hold
+ * threshold above its fail threshold, or a negative entry, is BSP_ERR_ARG. */
+typedef struct {
+  double rel_tol_deterministic;
+  double qprime_hold, r_hold;
+  double qprime_fail, r_fail;
+  double rel_hold;
+} bsp_verdict_rule_t;
 
 typedef enum { BSP_OUT_DGAMMA = 0, BSP_OUT_DBETA = 1, BSP_OUT_DW = 2, BSP_OUT_DX = 3,
                BSP_OUT_D = 4, BSP_OUT_DQ = 5, BSP_OUT_DK = 6, BSP_OUT_DV = 7 } bsp_output_t;
@@ -122,6 +149,10 @@ const char* bsp_status_string(int status);
 /* Number of kernels this library has launched in this process so far (a monotone counter kept for
  * accounting; it influences no result). */
 unsigned long long bsp_launch_count(void);
+
+/* Bytes this library has itself copied from the device to the host in this process so far (the
+ * block partials of the statistics passes: the only results a check brings back).  Accounting only. */
+unsigned long long bsp_d2h_byte_count(void);
 
 /* Clears a device bsp_diag_t (asynchronous memset). */
 int bsp_diag_clear(bsp_diag_t* diag, void* stream);
@@ -197,13 +228,17 @@ int bsp_norm_fwd_draws(int kind, const void* x, int dt, int64_t T, int64_t C, co
 /* Backward of the normalisation with du passed through the rounding unchanged:
  *   dgamma[C] = sum_t z_g o du, z_g = z (U) | (decode(u_codes)/scale - beta)/gamma (R) |
  *               the same from a fresh rounding under `key` (N, one draw);
- *   dbeta[C] = sum_t du (may be NULL);  dx[T*C] from unrounded values (may be NULL):
+ *   dbeta[C] = sum_t du (may be NULL);  dx[T*C] (may be NULL):
  *   RMS dx = rstd (dz - z mean_j(dz o z)), LN dx = rstd (dz - mean_j dz - z mean_j(dz o z)),
- *   dz = gamma o du.  du: du_dt[T*C].  Outputs FP32. */
+ *   dz = gamma o du, with z read under `dx_read`.  The paper's input gradient "uses unrounded
+ *   values" (Appendix "The normalization store"): that is dx_read = BSP_READ_ORIGINAL, the
+ *   reference and what every configuration uses; R and N read z as the gain use does, N under
+ *   generator stream BSP_STREAM_DX of the same key (dx is quadratic in z, so a fresh read leaves a
+ *   small bias: no verdict is put on it).  du: du_dt[T*C].  Outputs FP32. */
 size_t bsp_norm_bwd_workspace_bytes(int64_t T, int64_t C);
 int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                  const float* beta, const float* rstd, const float* mean, const void* du, int du_dt,
-                 int gain_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key,
+                 int gain_read, int dx_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key,
                  float* dgamma, float* dbeta, float* dx, void* ws, size_t ws_bytes,
                  bsp_diag_t* diag, void* stream);
 
@@ -229,14 +264,16 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
  *    cudaGetSymbolAddress, with that device current) and caches it; make that first call during
  *    set-up, before any stream capture is begun;
  *  - the array is shared by all calls and keeps whatever the last call wrote.  This pass writes
- *    every partial it later reads, so nothing needs clearing between calls -- but two calls that
- *    overlap on the GPU (different streams, or threads issuing concurrently) race on it and
- *    corrupt each other's sums.  Serialise them, or use bsp_norm_bwd with separate workspaces.
+ *    every partial it later reads, so nothing needs clearing between calls (a block whose bounded
+ *    wait ran out writes NaN partials and raises BSP_ERR_TIMEOUT in `diag`, so a failed call
+ *    cannot pass off the previous call's sums as its own) -- but two calls that overlap on the
+ *    GPU (different streams, or threads issuing concurrently) race on it and corrupt each
+ *    other's sums.  Serialise them, or use bsp_norm_bwd with separate workspaces.
  * Arguments, outputs and error behaviour are otherwise those of bsp_norm_bwd. */
 #define BSP_NORM_BWD_NOALLOC_CAPACITY_BYTES ((size_t)20 << 20)
 int bsp_norm_bwd_noalloc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                          const float* beta, const float* rstd, const float* mean, const void* du,
-                         int du_dt, int gain_read, const uint8_t* u_codes, bsp_quant_t q,
+                         int du_dt, int gain_read, int dx_read, const uint8_t* u_codes, bsp_quant_t q,
                          bsp_key_t key, float* dgamma, float* dbeta, float* dx, bsp_diag_t* diag,
                          void* stream);
 
@@ -302,56 +339,26 @@ int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, b
  * P = softmax(c Q K^T), O = P V; dV = P^T dO, dP = dO V^T, dS = P o (dP - D),
  * D = rowsum(P o dP) = rowsum(dO o O); dQ = c dS K, dK = c dS^T Q.  The forward rounds O before the
  * next layer consumes it; the correction term D is the one use of the saved output, and reading a
- * copy O + E adds rowsum(dO o E) (Eq. dterm).  Tensors are [B, H, S, Dh] row-major, bf16 inputs
- * (dt = BSP_BF16), Dh = 64, FP32 outputs; lse, D are [B, H, S].  BF16 tensor-core operands (P and
- * dS are rounded to bf16 for their products).  The FP8-operand variant of Appendix "The forks" has
- * its own entry points (bsp_attn_*_fp8, below) because it needs the operand scales; in
- * bsp_attn_bwd the flag fp8_operands must be 0 (otherwise BSP_ERR_UNSUPPORTED).
- * ------------------------------------------------------------------------------------------ */
-
-/* Forward statistics from the operands exactly as the backward will see them: o = P V (FP32, the
- * "original" output the store rounds) and lse = log sum_j exp(c q.k_j). */
-int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
-                       const void* k, const void* v, int dt, float* o, float* lse, bsp_diag_t* diag,
-                       void* stream);
-
-/* The D use: d_out[d][b,h,i] = sum_j dO[b,h,i,j] * O_copy[b,h,i,j] for n_draws draws, with
- * O_copy = o_orig (U), decode(o_codes)/o_scales[b,h] (R), or a fresh stochastic rounding of
- * fl32(o_orig * o_scales[b,h]) in o_fmt under (key, draw0 + d) (N).  U and R write one draw.
- * dO: dt[B,H,S,Dh]; o_scales: one scale per (b,h) slice.  dO and o_orig 16-byte aligned, o_codes
- * 8-byte aligned (BSP_ERR_ALIGN otherwise). */
-int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig,
-                   const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key,
-                   int draw0, int n_draws, float* d_out, bsp_diag_t* diag, void* stream);
-
-/* Backward given D (dterm[B,H,S]).  dq may be NULL; dk and dv may both be NULL; dv may be NULL
- * alone (dK only: dV does not read D, so the draws of a fresh read need it once); dv without dk
- * is BSP_ERR_ARG. */
-int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
-                       const void* k, const void* v, const void* dO, int dt, const float* lse,
-                       const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
-                       void* stream);
-
-/* Backward under a read policy at the D use: bsp_attn_dterm (draw key.draw) into d_out[B,H,S]
- * (required), then bsp_attn_bwd_dterm. */
-int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands,
-                 const void* q, const void* k, const void* v, const void* dO, int dt, const float* lse,
-                 const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt,
-                 int d_read, bsp_key_t key, float* dq, float* dk, float* dv, float* d_out,
-                 bsp_diag_t* diag, void* stream);
-
-/* FP8-operand mode, after the emulated FP8 attention backward of Appendix "The forks": Q, K, V are
+ * copy O + E adds rowsum(dO o E) (Eq. dterm).  Tensors are [B, H, S, Dh] row-major, bf16
+ * (dt = BSP_BF16), Dh = 64, FP32 outputs; lse, D are [B, H, S].
+ *
+ * Two operand modes.  BF16 operands (fp8 = NULL): the three products that consume a computed
+ * operand take P and dS rounded to bf16; against the plain definition that rounding alone is a
+ * relative distance of about 1.7e-3 per output tensor on the benchmark's inputs.  FP8 operands
+ * (fp8 != NULL), after the emulated FP8 attention backward of Appendix "The forks": Q, K, V are
  * rounded to nearest onto E4M3 and dO onto E5M2, each at the per-(b,h) amax scale of its slice; P is
  * recomputed (unrounded) from the dequantised Q and K; dV = P_q^T dO with P_q = RN_E4M3(P p_scale)
  * / p_scale; dP = dO V^T; D from the assigned output copy; dS = P o (dP - D); dS_q = RN_E5M2(dS
  * ds_scale) / ds_scale feeds dQ and dK (ds_scale supplied by the caller, like a delayed scale).
- * The quantised operands travel as bf16 tensors holding the DECODED codes (every FP8 value is a
- * bf16 value, so the tensor-core products are those of the FP8 operands exactly); their scales
- * are folded back in the kernel.  The final E5M2 cast of the returned gradients is not applied
- * (outputs FP32).  Quantisation points and the two scales are this library's reading of that
- * appendix. */
+ * In that mode q, k, v, dO are bf16 tensors holding the DECODED codes as written by
+ * bsp_attn_quantize (every FP8 value is a bf16 value, so the tensor-core products are those of the
+ * FP8 operands exactly); their scales are folded back in the kernel.  The final E5M2 cast of the
+ * returned gradients is not applied (outputs FP32).  Quantisation points and the two scales are
+ * this library's reading of that appendix.
+ * ------------------------------------------------------------------------------------------ */
+
 typedef struct {
-  const float* q_scale;      /* [B*H] device: scale of each slice of q8 (code = round(x * scale)) */
+  const float* q_scale;      /* [B*H] device: scale of each slice of q (code = round(x * scale)) */
   const float* k_scale;
   const float* v_scale;
   const float* do_scale;
@@ -365,19 +372,38 @@ typedef struct {
 int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax,
                       float* scales, bsp_diag_t* diag, void* stream);
 
-/* bsp_attn_fwd_stats on quantised operands (q8, k8, v8 from bsp_attn_quantize): o = P V_hat in
- * FP32 with P unrounded, lse from the dequantised q and k. */
-int bsp_attn_fwd_stats_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8,
-                           const void* k8, const void* v8, int dt, const bsp_attn_fp8_t* fp8, float* o,
-                           float* lse, bsp_diag_t* diag, void* stream);
+/* Forward statistics from the operands exactly as the backward will see them: o = P V (FP32, the
+ * "original" output the store rounds; P unrounded) and lse = log sum_j exp(c q.k_j). */
+int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                       const void* k, const void* v, int dt, const bsp_attn_fp8_t* fp8, float* o,
+                       float* lse, bsp_diag_t* diag, void* stream);
 
-/* bsp_attn_bwd in FP8-operand mode; dO8 holds the decoded E5M2 codes of dO, D = rowsum(dO_hat o
- * O_copy) with dO_hat = dO8 / do_scale. */
-int bsp_attn_bwd_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8,
-                     const void* k8, const void* v8, const void* dO8, int dt, const bsp_attn_fp8_t* fp8,
-                     const float* lse, const float* o_orig, const uint8_t* o_codes, const float* o_scales,
-                     int o_fmt, int d_read, bsp_key_t key, float* dq, float* dk, float* dv, float* d_out,
-                     bsp_diag_t* diag, void* stream);
+/* The D use: d_out[d][b,h,i] = sum_j dO[b,h,i,j] * O_copy[b,h,i,j] for n_draws draws, with
+ * O_copy = o_orig (U), decode(o_codes)/o_scales[b,h] (R), or a fresh stochastic rounding of
+ * fl32(o_orig * o_scales[b,h]) in o_fmt under (key, draw0 + d) (N).  U and R write one draw.
+ * dO: dt[B,H,S,Dh]; do_scales: NULL, or (FP8-operand mode) the per-(b,h) scales of a dO that holds
+ * decoded codes; o_scales: one scale per (b,h) slice.  dO and o_orig 16-byte aligned, o_codes
+ * 8-byte aligned (BSP_ERR_ALIGN otherwise). */
+int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
+                   const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt,
+                   int d_read, bsp_key_t key, int draw0, int n_draws, float* d_out, bsp_diag_t* diag,
+                   void* stream);
+
+/* Backward given D (dterm[B,H,S]).  dq may be NULL; dk and dv may both be NULL; dv may be NULL
+ * alone (dK only: dV does not read D); dv without dk is BSP_ERR_ARG. */
+int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                       const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* fp8,
+                       const float* lse, const float* dterm, float* dq, float* dk, float* dv,
+                       bsp_diag_t* diag, void* stream);
+
+/* Backward under a read policy at the D use: bsp_attn_dterm (draw key.draw) into d_out[B,H,S]
+ * (required), then bsp_attn_bwd_dterm.  fp8_operands = 0: fp8 must be NULL; fp8_operands = 1: fp8
+ * gives the operand scales (BSP_ERR_ARG when the flag and the pointer disagree). */
+int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands,
+                 const void* q, const void* k, const void* v, const void* dO, int dt,
+                 const bsp_attn_fp8_t* fp8, const float* lse, const float* o_orig, const uint8_t* o_codes,
+                 const float* o_scales, int o_fmt, int d_read, bsp_key_t key, float* dq, float* dk,
+                 float* dv, float* d_out, bsp_diag_t* diag, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Monte-Carlo reduction (Section "Each use has a checkable requirement").
@@ -387,27 +413,38 @@ int bsp_attn_bwd_fp8(int B, int H, int S, int Dh, int causal, float softmax_scal
  * (n a multiple of 4).  Used where the producing kernel has no fused accumulation. */
 int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, size_t n, void* stream);
 
+/* Per-element moments from the shifted sums of K draws (K >= 2): mean = g_ref + S1/K,
+ * var = (S2 - S1^2/K) / (K - 1) (clamped at 0), z = (S1/K) / sqrt(var/K) (0 when numerator and
+ * denominator both vanish, +-infinity when only the denominator does).  Any output may be NULL. */
+int bsp_mc_moments(const float* g_ref, const float* S1, const float* S2, size_t n, int K, float* mean,
+                   float* var, float* z, void* stream);
+
 /* Reduces per-element shifted sums to the statistics of bsp_use_result_t and the verdict.
  * fresh = 0: deterministic read, `g` holds the gradient itself (S2 ignored, K = 1).
- * fresh = 1: g = S1, with S2, over K draws.  ws: >= bsp_mc_stats_workspace_bytes(n).
+ * fresh = 1: g = S1, with S2, over K >= 4 draws.  ws: >= bsp_mc_stats_workspace_bytes(n).
  * Synchronises `stream`; `result` is HOST memory; use_id/output_id/policy are left untouched. */
 size_t bsp_mc_stats_workspace_bytes(int64_t n);
 int bsp_mc_stats(const float* g_ref, const float* g, const float* S2, int64_t n, int K, int fresh,
-                 bsp_use_result_t* result, void* ws, size_t ws_bytes, void* stream);
+                 const bsp_verdict_rule_t* rule, bsp_use_result_t* result, void* ws, size_t ws_bytes,
+                 void* stream);
 
 /* The whole per-use check of a normalisation -> linear workload, device-resident inputs.
  * Once per call: statistics, current-amax scale, forward store (stream 0, `forward_mode`),
  * incoming gradient dY -> E5M2 nearest at its own amax, du = dY W.  Then per use and policy:
- *   gain use  (dgamma, reference read U):  U, R, N (K draws);
+ *   gain use  (dgamma, reference read U):  U, R, N (K draws); each is followed by the result for
+ *   dbeta, which reads no saved tensor and so equals its reference under every read;
  *   weight use (dW,    reference read R):  U, R, N (K draws: re-round + FP8 contraction + fused
  *   shifted-sum epilogue).
  * `policy_mask` bit (use*3 + policy) selects evaluations, use 0 = gain, 1 = weight.
- * results: HOST array, filled in order gain U,R,N then weight U,R,N (selected ones only);
- * *n_results returns the count.  Synchronises before returning.
- * When both uses ask for N, the K-draw gain kernel runs beside the first K-draw contraction on a
- * second, non-blocking stream that the library creates once per device and keeps; it is forked
- * from and joined back into `stream` inside the call, and is idle when the call returns on any
- * path.  Calls on one device may overlap in time only if they use different workspaces. */
+ * K >= 4 (the factor (K-3)/(K-1) of Q' must be positive).
+ * results: HOST array of at least 9 entries, filled in order gain U (dgamma, dbeta), R, N, then
+ * weight U, R, N (selected ones only); *n_results returns the count.  Synchronises before
+ * returning.  The per-element results stay in `ws` at the offsets bsp_mc_check_layout gives.
+ * `side_stream` (a cudaStream_t, or NULL): when both uses ask for N, the K-draw gain kernel runs
+ * beside the first K-draw contraction on that stream, forked from and joined back into `stream`
+ * inside the call; with NULL the two run one after the other.  `draw_buffer_bytes` bounds the
+ * buffer of fresh code matrices (0 = 1 GiB): K draws are taken in chunks of as many draws as fit.
+ * Calls on one device may overlap in time only if they use different workspaces. */
 typedef struct {
   int32_t norm_kind;         /* bsp_norm_t  */
   int32_t dtype;             /* bsp_dtype_t of x, W, dY (and of du) */
@@ -424,18 +461,51 @@ typedef struct {
   uint64_t seed;
   uint32_t tensor_id;
   uint32_t policy_mask;
+  void* side_stream;
+  size_t draw_buffer_bytes;
 } bsp_norm_linear_desc_t;
 
+/* Byte offsets into the workspace of bsp_mc_check, of the FP32 arrays it leaves there.  With
+ * bsp_mc_moments they give the per-element mean, variance and z-score of every gradient
+ * (dgamma and dbeta: [C]; dW: [O*C]; under N: sums over K draws; dbeta has no sums, it equals its
+ * reference in every draw). */
+typedef struct {
+  size_t dgamma_ref, dbeta_ref;      /* [C]: the reference gradients (gain use reads U)          */
+  size_t dgamma_forward;             /* [C]: dgamma under read R                                 */
+  size_t dgamma_S1, dgamma_S2;       /* [C]: shifted sums of dgamma over the K draws of read N   */
+  size_t dW_ref;                     /* [O*C]: the reference (weight use reads R)                */
+  size_t dW_S1, dW_S2;               /* [O*C]: shifted sums of dW over the K draws of read N     */
+  size_t dx;                         /* [T*C]: the input gradient from unrounded values          */
+  size_t rstd, mean;                 /* [T]: saved statistics                                    */
+  size_t u_codes;                    /* [T*C] uint8: the forward's store                         */
+  size_t scale_u, scale_dy;          /* one float each                                           */
+  size_t du;                         /* [T*C] in the workload's dtype                            */
+} bsp_mc_layout_t;
+
 size_t bsp_mc_check_workspace_bytes(const bsp_norm_linear_desc_t* op, int K);
-int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, bsp_use_result_t* results, int* n_results,
-                 void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
+int bsp_mc_check_layout(const bsp_norm_linear_desc_t* op, int K, bsp_mc_layout_t* layout);
+int bsp_mc_check(const bsp_norm_linear_desc_t* op, int K, const bsp_verdict_rule_t* rule,
+                 bsp_use_result_t* results, int* n_results, void* ws, size_t ws_bytes, bsp_diag_t* diag,
+                 void* stream);
 
 /* The per-use check of the attention D use (Section "Same rounding distribution, opposite
- * outcomes"; Eq. dterm), device-resident inputs.  Once per call: O = P V and LSE, the output store
- * (per-(b,h) amax scale, `forward_mode`, stream 0).  Reference: D reads the original output.  Then
- * for each selected policy (policy_mask bit p = bsp_policy_t p) the backward is evaluated with D
- * read under that policy -- U and R once, N for K draws -- and four results are written per policy
- * in the order D, dQ, dK, dV.  `results` is a HOST array (up to 12 entries).  Synchronises. */
+ * outcomes"; Eq. dterm), device-resident inputs.  Once per call: (FP8-operand mode: the operands
+ * rounded per (b,h) slice), O = P V and LSE, the output store (per-(b,h) amax scale,
+ * `forward_mode`, stream 0).  Reference: D reads the original output.  Then for each selected
+ * policy (policy_mask bit p = bsp_policy_t p) the backward is evaluated with D read under that
+ * policy -- U and R once, N for K >= 4 draws -- and four results are written per policy in the
+ * order D, dQ, dK, dV.  `results` is a HOST array (up to 12 entries).  Synchronises.
+ *
+ * BF16-operand mode evaluates the fresh read through Eq. dterm itself: dS, dQ and dK are affine in
+ * D, so draw k differs from the reference by  dQ_k - dQ* = -c diag(D_k - D*) (P K)  and
+ * dK_k - dK* = -c P^T diag(D_k - D*) Q.  The kernels form these differences directly (the K draws
+ * of dQ collapse to one pass for P K and the sums of D_k - D*; dK takes one contraction per draw,
+ * four draws per pass of the probabilities), so the statistics are not blurred by the rounding of
+ * a full dS to the operand type, and no per-draw gradient is written.  dV does not read D: its
+ * difference is exactly zero in every draw.
+ * FP8-operand mode (fp8_operands = 1; p_scale, ds_scale as in bsp_attn_fp8_t) runs the rounded
+ * backward once per draw: there dQ and dK pass through the nearest rounding of dS, which is not
+ * linear in D, so their rows are marked `informational` and the verdict of the use is the row of D. */
 typedef struct {
   int32_t B, H, S, Dh;
   int32_t causal;
@@ -450,11 +520,23 @@ typedef struct {
   uint64_t seed;
   uint32_t tensor_id;
   uint32_t policy_mask;
+  int32_t fp8_operands;      /* 0: BF16 operands; 1: the FP8-operand mode */
+  float p_scale, ds_scale;   /* FP8-operand mode only */
 } bsp_attn_desc_t;
 
 size_t bsp_mc_check_attn_workspace_bytes(const bsp_attn_desc_t* op, int K);
-int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* results, int* n_results,
-                      void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream);
+int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, const bsp_verdict_rule_t* rule,
+                      bsp_use_result_t* results, int* n_results, void* ws, size_t ws_bytes,
+                      bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait a kernel of
+ * this library performs on a barrier gives up after a time limit, raises BSP_ERR_TIMEOUT in `diag`
+ * and lets the kernel return normally.  This entry launches one small block whose wait is on a
+ * barrier that nothing ever completes, with the limit set to `limit_ns` nanoseconds (1 .. 10^8);
+ * after synchronising, diag.status == BSP_ERR_TIMEOUT and the context is intact.
+ * ------------------------------------------------------------------------------------------ */
+int bsp_selftest_bounded_wait(uint64_t limit_ns, bsp_diag_t* diag, void* stream);
 
 #ifdef __cplusplus
 }

@@ -43,10 +43,21 @@ class UseResult(C.Structure):
                 ("n_elements", C.c_int64), ("rel_l2_mean_err", C.c_double), ("R", C.c_double),
                 ("Qprime", C.c_double), ("mean_z", C.c_double), ("rms_z", C.c_double),
                 ("max_abs_z", C.c_double), ("frac_abs_z_gt3", C.c_double), ("verdict", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("informational", C.c_int32)]
 
     def as_dict(self):
-        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class VerdictRule(C.Structure):
+    _fields_ = [("rel_tol_deterministic", C.c_double), ("qprime_hold", C.c_double), ("r_hold", C.c_double),
+                ("qprime_fail", C.c_double), ("r_fail", C.c_double), ("rel_hold", C.c_double)]
+
+
+class McLayout(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in (
+        "dgamma_ref", "dbeta_ref", "dgamma_forward", "dgamma_S1", "dgamma_S2", "dW_ref", "dW_S1", "dW_S2", "dx",
+        "rstd", "mean", "u_codes", "scale_u", "scale_dy", "du")]
 
 
 class NormLinearDesc(C.Structure):
@@ -54,14 +65,16 @@ class NormLinearDesc(C.Structure):
                 ("O", C.c_int64), ("x", C.c_void_p), ("gamma", C.c_void_p), ("beta", C.c_void_p),
                 ("W", C.c_void_p), ("dY", C.c_void_p), ("eps", C.c_float), ("store_fmt", C.c_int32),
                 ("grad_fmt", C.c_int32), ("forward_mode", C.c_int32), ("seed", C.c_uint64),
-                ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
+                ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32), ("side_stream", C.c_void_p),
+                ("draw_buffer_bytes", C.c_size_t)]
 
 
 class AttnDesc(C.Structure):
     _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("S", C.c_int32), ("Dh", C.c_int32), ("causal", C.c_int32),
                 ("softmax_scale", C.c_float), ("dtype", C.c_int32), ("q", C.c_void_p), ("k", C.c_void_p),
                 ("v", C.c_void_p), ("dO", C.c_void_p), ("store_fmt", C.c_int32), ("forward_mode", C.c_int32),
-                ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
+                ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32),
+                ("fp8_operands", C.c_int32), ("p_scale", C.c_float), ("ds_scale", C.c_float)]
 
 
 class AttnFp8(C.Structure):
@@ -82,6 +95,7 @@ _P, _SZ, _I, _I64, _U64, _F = C.c_void_p, C.c_size_t, C.c_int, C.c_int64, C.c_ui
 _SIGNATURES = {
     "bsp_status_string": (C.c_char_p, [_I]),
     "bsp_launch_count": (C.c_ulonglong, []),
+    "bsp_d2h_byte_count": (C.c_ulonglong, []),
     "bsp_diag_clear": (_I, [_P, _P]),
     "bsp_philox_fill": (_I, [Key, _SZ, _P, _P]),
     "bsp_amax": (_I, [_P, _I, _SZ, _SZ, _P, _P, _P]),
@@ -95,9 +109,9 @@ _SIGNATURES = {
     "bsp_gemm": (_I, [_I64, _I64, _I64, _I, _P, _I64, _I, _I, _P, _I64, _I, _I, _F, _P, _I64, _P, _P]),
     "bsp_linear_wgrad_mc": (_I, [_I64, _I64, _I64, _P, Quant, _P, Quant, _I64, _I, _P, _P, _P, _P, _P]),
     "bsp_norm_bwd_workspace_bytes": (_SZ, [_I64, _I64]),
-    "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
+    "bsp_norm_bwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _I, _P, Quant, Key, _P, _P, _P,
                           _P, _SZ, _P, _P]),
-    "bsp_norm_bwd_noalloc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _P, Quant, Key, _P, _P, _P,
+    "bsp_norm_bwd_noalloc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, _I, _I, _P, Quant, Key, _P, _P, _P,
                                   _P, _P]),
     "bsp_norm_gain_mc_workspace_bytes": (_SZ, [_I64, _I64, _I]),
     "bsp_norm_gain_mc": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _I, Quant, Key, _I, _I, _P, _P, _P,
@@ -106,22 +120,25 @@ _SIGNATURES = {
     "bsp_linear_wgrad": (_I, [_I64, _I64, _I64, _P, Quant, _I, _P, Quant, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
     "bsp_linear_dgrad_workspace_bytes": (_SZ, [_I64, _I64, _I64]),
     "bsp_linear_dgrad": (_I, [_I64, _I64, _I64, _P, Quant, _P, _I, _P, _I, _P, _SZ, _P, _P]),
-    "bsp_attn_fwd_stats": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _I, _P, _P, _P, _P]),
-    "bsp_attn_dterm": (_I, [_I, _I, _I, _I, _P, _I, _P, _P, _P, _I, _I, Key, _I, _I, _P, _P, _P]),
-    "bsp_attn_bwd_dterm": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P]),
-    "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, _P, _P, _P, _P, _I, _I, Key, _P, _P, _P,
-                          _P, _P, _P]),
+    "bsp_attn_fwd_stats": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P]),
+    "bsp_attn_dterm": (_I, [_I, _I, _I, _I, _P, _I, _P, _P, _P, _P, _I, _I, Key, _I, _I, _P, _P, _P]),
+    "bsp_attn_bwd_dterm": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _P,
+                                _P, _P]),
+    "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _I, _I,
+                          Key, _P, _P, _P, _P, _P, _P]),
     "bsp_attn_quantize": (_I, [_P, _I, _SZ, _I, _P, _P, _P, _P, _P]),
-    "bsp_attn_fwd_stats_fp8": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P]),
-    "bsp_attn_bwd_fp8": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _I, _I,
-                              Key, _P, _P, _P, _P, _P, _P]),
     "bsp_mc_accumulate": (_I, [_P, _P, _P, _P, _SZ, _P]),
+    "bsp_mc_moments": (_I, [_P, _P, _P, _SZ, _I, _P, _P, _P, _P]),
     "bsp_mc_check_attn_workspace_bytes": (_SZ, [C.POINTER(AttnDesc), _I]),
-    "bsp_mc_check_attn": (_I, [C.POINTER(AttnDesc), _I, C.POINTER(UseResult), C.POINTER(_I), _P, _SZ, _P, _P]),
+    "bsp_mc_check_attn": (_I, [C.POINTER(AttnDesc), _I, C.POINTER(VerdictRule), C.POINTER(UseResult), C.POINTER(_I),
+                               _P, _SZ, _P, _P]),
     "bsp_mc_stats_workspace_bytes": (_SZ, [_I64]),
-    "bsp_mc_stats": (_I, [_P, _P, _P, _I64, _I, _I, C.POINTER(UseResult), _P, _SZ, _P]),
+    "bsp_mc_stats": (_I, [_P, _P, _P, _I64, _I, _I, C.POINTER(VerdictRule), C.POINTER(UseResult), _P, _SZ, _P]),
     "bsp_mc_check_workspace_bytes": (_SZ, [C.POINTER(NormLinearDesc), _I]),
-    "bsp_mc_check": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(UseResult), C.POINTER(_I), _P, _SZ, _P, _P]),
+    "bsp_mc_check_layout": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(McLayout)]),
+    "bsp_mc_check": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(VerdictRule), C.POINTER(UseResult), C.POINTER(_I),
+                          _P, _SZ, _P, _P]),
+    "bsp_selftest_bounded_wait": (_I, [_U64, _P, _P]),
 }
 
 
@@ -217,6 +234,10 @@ def bsp_launch_count() -> int:
     return int(lib().bsp_launch_count())
 
 
+def bsp_d2h_byte_count() -> int:
+    return int(lib().bsp_d2h_byte_count())
+
+
 def bsp_diag_clear(diag, stream=None):
     check(lib().bsp_diag_clear(ptr(diag), stream if stream is not None else cur_stream()), "bsp_diag_clear")
 
@@ -288,20 +309,20 @@ def bsp_norm_bwd_workspace_bytes(T, Cc):
 
 
 def bsp_norm_bwd(kind, x, T, Cc, gamma, beta, rstd, mean, du, gain_read, u_codes, q: Quant, k: Key,
-                 dgamma, dbeta, dx, ws, diag=None, stream=None):
+                 dgamma, dbeta, dx, ws, diag=None, stream=None, dx_read=READ_ORIGINAL):
     check(lib().bsp_norm_bwd(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
-                             ptr(du), dtype_code(du), gain_read, ptr(u_codes), q, k, ptr(dgamma), ptr(dbeta),
+                             ptr(du), dtype_code(du), gain_read, dx_read, ptr(u_codes), q, k, ptr(dgamma), ptr(dbeta),
                              ptr(dx), ptr(ws), ws.numel() if ws is not None else 0, ptr(diag),
                              stream if stream is not None else cur_stream()), "bsp_norm_bwd")
 
 
 def bsp_norm_bwd_noalloc(kind, x, T, Cc, gamma, beta, rstd, mean, du, gain_read, u_codes, q: Quant, k: Key,
-                         dgamma, dbeta, dx, diag=None, stream=None):
+                         dgamma, dbeta, dx, diag=None, stream=None, dx_read=READ_ORIGINAL):
     """bsp_norm_bwd without a workspace argument: scratch is the library's own fixed device array
     (for callers that may not allocate device memory).  Raises BspError(ERR_TOO_LARGE) when the
     problem does not fit NORM_BWD_NOALLOC_CAPACITY_BYTES.  Calls that overlap on the GPU race."""
     check(lib().bsp_norm_bwd_noalloc(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd),
-                                     ptr(mean), ptr(du), dtype_code(du), gain_read, ptr(u_codes), q, k,
+                                     ptr(mean), ptr(du), dtype_code(du), gain_read, dx_read, ptr(u_codes), q, k,
                                      ptr(dgamma), ptr(dbeta), ptr(dx), ptr(diag),
                                      stream if stream is not None else cur_stream()), "bsp_norm_bwd_noalloc")
 
@@ -343,29 +364,36 @@ def _st(stream):
     return stream if stream is not None else cur_stream()
 
 
-def bsp_attn_fwd_stats(B, H, S, Dh, causal, softmax_scale, q, k, v, o, lse, diag=None, stream=None):
+def _fp8ref(f):
+    return C.byref(f) if f is not None else None
+
+
+def bsp_attn_fwd_stats(B, H, S, Dh, causal, softmax_scale, q, k, v, o, lse, diag=None, stream=None, fp8=None):
     check(lib().bsp_attn_fwd_stats(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), dtype_code(q),
-                                   ptr(o), ptr(lse), ptr(diag), _st(stream)), "bsp_attn_fwd_stats")
+                                   _fp8ref(fp8), ptr(o), ptr(lse), ptr(diag), _st(stream)), "bsp_attn_fwd_stats")
 
 
 def bsp_attn_dterm(B, H, S, Dh, dO, o_orig, o_codes, o_scales, o_fmt, d_read, k: Key, draw0, n_draws, d_out,
-                   diag=None, stream=None):
-    check(lib().bsp_attn_dterm(B, H, S, Dh, ptr(dO), dtype_code(dO), ptr(o_orig), ptr(o_codes), ptr(o_scales), o_fmt,
-                               d_read, k, draw0, n_draws, ptr(d_out), ptr(diag), _st(stream)), "bsp_attn_dterm")
+                   diag=None, stream=None, do_scales=None):
+    check(lib().bsp_attn_dterm(B, H, S, Dh, ptr(dO), dtype_code(dO), ptr(do_scales), ptr(o_orig), ptr(o_codes),
+                               ptr(o_scales), o_fmt, d_read, k, draw0, n_draws, ptr(d_out), ptr(diag), _st(stream)),
+          "bsp_attn_dterm")
 
 
 def bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, lse, dterm, dq, dk, dv, diag=None,
-                       stream=None):
+                       stream=None, fp8=None):
     check(lib().bsp_attn_bwd_dterm(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), ptr(dO),
-                                   dtype_code(q), ptr(lse), ptr(dterm), ptr(dq), ptr(dk), ptr(dv), ptr(diag),
-                                   _st(stream)), "bsp_attn_bwd_dterm")
+                                   dtype_code(q), _fp8ref(fp8), ptr(lse), ptr(dterm), ptr(dq), ptr(dk), ptr(dv),
+                                   ptr(diag), _st(stream)), "bsp_attn_bwd_dterm")
 
 
 def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, lse, o_orig, o_codes, o_scales,
-                 o_fmt, d_read, key_: Key, dq, dk, dv, d_out, diag=None, stream=None):
+                 o_fmt, d_read, key_: Key, dq, dk, dv, d_out, diag=None, stream=None, fp8=None):
+    """fp8_operands = 1 needs `fp8` (an AttnFp8 with the operand scales) and q, k, v, dO as written by
+    bsp_attn_quantize."""
     check(lib().bsp_attn_bwd(B, H, S, Dh, int(causal), softmax_scale, int(fp8_operands), ptr(q), ptr(k), ptr(v),
-                             ptr(dO), dtype_code(q), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales), o_fmt,
-                             d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
+                             ptr(dO), dtype_code(q), _fp8ref(fp8), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales),
+                             o_fmt, d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
           "bsp_attn_bwd")
 
 
@@ -378,34 +406,37 @@ def attn_fp8(q_scale, k_scale, v_scale, do_scale, p_scale=256.0, ds_scale=1.0) -
     return AttnFp8(ptr(q_scale), ptr(k_scale), ptr(v_scale), ptr(do_scale), float(p_scale), float(ds_scale))
 
 
-def bsp_attn_fwd_stats_fp8(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, f: AttnFp8, o, lse, diag=None, stream=None):
-    check(lib().bsp_attn_fwd_stats_fp8(B, H, S, Dh, int(causal), softmax_scale, ptr(q8), ptr(k8), ptr(v8),
-                                       dtype_code(q8), C.byref(f), ptr(o), ptr(lse), ptr(diag), _st(stream)),
-          "bsp_attn_fwd_stats_fp8")
+def rule(rel_tol_deterministic=1e-4, qprime_hold=2.0, r_hold=3.0, qprime_fail=4.0, r_fail=6.0, rel_hold=0.0):
+    return VerdictRule(rel_tol_deterministic, qprime_hold, r_hold, qprime_fail, r_fail, rel_hold)
 
 
-def bsp_attn_bwd_fp8(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dO8, f: AttnFp8, lse, o_orig, o_codes, o_scales,
-                     o_fmt, d_read, key_: Key, dq, dk, dv, d_out, diag=None, stream=None):
-    check(lib().bsp_attn_bwd_fp8(B, H, S, Dh, int(causal), softmax_scale, ptr(q8), ptr(k8), ptr(v8), ptr(dO8),
-                                 dtype_code(q8), C.byref(f), ptr(lse), ptr(o_orig), ptr(o_codes), ptr(o_scales),
-                                 o_fmt, d_read, key_, ptr(dq), ptr(dk), ptr(dv), ptr(d_out), ptr(diag), _st(stream)),
-          "bsp_attn_bwd_fp8")
+def _ruleref(r):
+    return C.byref(r) if r is not None else None
 
 
 def bsp_mc_accumulate(g, g_ref, S1, S2, n, stream=None):
     check(lib().bsp_mc_accumulate(ptr(g), ptr(g_ref), ptr(S1), ptr(S2), n, _st(stream)), "bsp_mc_accumulate")
 
 
+def bsp_mc_moments(g_ref, S1, S2, n, K, mean=None, var=None, z=None, stream=None):
+    check(lib().bsp_mc_moments(ptr(g_ref), ptr(S1), ptr(S2), n, K, ptr(mean), ptr(var), ptr(z), _st(stream)),
+          "bsp_mc_moments")
+
+
+def bsp_selftest_bounded_wait(limit_ns, diag, stream=None):
+    check(lib().bsp_selftest_bounded_wait(int(limit_ns), ptr(diag), _st(stream)), "bsp_selftest_bounded_wait")
+
+
 def bsp_mc_check_attn_workspace_bytes(desc: AttnDesc, K):
     return lib().bsp_mc_check_attn_workspace_bytes(C.byref(desc), K)
 
 
-def bsp_mc_check_attn(desc: AttnDesc, K, ws, diag=None, stream=None):
+def bsp_mc_check_attn(desc: AttnDesc, K, ws, diag=None, stream=None, rule=None):
     """Returns the list of UseResult: per selected policy (U, R, N) the four outputs D, dQ, dK, dV."""
     res = (UseResult * 12)()
     n = C.c_int(0)
-    check(lib().bsp_mc_check_attn(C.byref(desc), K, res, C.byref(n), ptr(ws), ws.numel(), ptr(diag), _st(stream)),
-          "bsp_mc_check_attn")
+    check(lib().bsp_mc_check_attn(C.byref(desc), K, _ruleref(rule), res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
+                                  _st(stream)), "bsp_mc_check_attn")
     return [res[i] for i in range(n.value)]
 
 
@@ -413,10 +444,10 @@ def bsp_mc_stats_workspace_bytes(n):
     return lib().bsp_mc_stats_workspace_bytes(n)
 
 
-def bsp_mc_stats(g_ref, g, S2, n, K, fresh, ws, stream=None) -> UseResult:
+def bsp_mc_stats(g_ref, g, S2, n, K, fresh, ws, stream=None, rule=None) -> UseResult:
     r = UseResult()
-    check(lib().bsp_mc_stats(ptr(g_ref), ptr(g), ptr(S2), n, K, fresh, C.byref(r), ptr(ws), ws.numel(),
-                             stream if stream is not None else cur_stream()), "bsp_mc_stats")
+    check(lib().bsp_mc_stats(ptr(g_ref), ptr(g), ptr(S2), n, K, fresh, _ruleref(rule), C.byref(r), ptr(ws),
+                             ws.numel(), _st(stream)), "bsp_mc_stats")
     return r
 
 
@@ -424,10 +455,24 @@ def bsp_mc_check_workspace_bytes(desc: NormLinearDesc, K):
     return lib().bsp_mc_check_workspace_bytes(C.byref(desc), K)
 
 
-def bsp_mc_check(desc: NormLinearDesc, K, ws, diag=None, stream=None):
-    """Returns the list of UseResult (gain U,R,N then weight U,R,N; selected ones only)."""
-    res = (UseResult * 8)()
+def bsp_mc_check_layout(desc: NormLinearDesc, K) -> McLayout:
+    lay = McLayout()
+    check(lib().bsp_mc_check_layout(C.byref(desc), K, C.byref(lay)), "bsp_mc_check_layout")
+    return lay
+
+
+def bsp_mc_check(desc: NormLinearDesc, K, ws, diag=None, stream=None, rule=None):
+    """Returns the list of UseResult: gain U (dgamma, dbeta), R, N, then weight U, R, N; selected ones only."""
+    res = (UseResult * 12)()
     n = C.c_int(0)
-    check(lib().bsp_mc_check(C.byref(desc), K, res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
-                             stream if stream is not None else cur_stream()), "bsp_mc_check")
+    check(lib().bsp_mc_check(C.byref(desc), K, _ruleref(rule), res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
+                             _st(stream)), "bsp_mc_check")
     return [res[i] for i in range(n.value)]
+
+
+def ws_view(ws, offset, count, dtype=None):
+    """A typed view of `count` elements at byte `offset` of a workspace tensor (float32 by default)."""
+    import torch
+    dtype = dtype or torch.float32
+    nbytes = count * torch.empty((), dtype=dtype).element_size()
+    return ws[offset:offset + nbytes].view(dtype)

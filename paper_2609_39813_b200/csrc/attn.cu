@@ -21,17 +21,14 @@
 // Head dimension 64, bf16 inputs, FP32 outputs.  Every wait is bounded.
 #include <string.h>
 
+#include <atomic>
 
-#include "common.cuh"
+
+#include "attn_common.cuh"
 #include "mc_stats.cuh"
-#include "tc.cuh"
 
 namespace bsp {
 
-enum { AT_DKV = 0, AT_DQ = 1, AT_FWD = 2 };
-
-constexpr int AT_BLK = 128, AT_D = 64;
-constexpr int kAtTile = AT_BLK * AT_D * 2;        // 16 KB: one 128 x 64 bf16 tile
 constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
 constexpr int kAtThreads = 320;
 constexpr int kAtSoftWarp0 = 2;                   // first softmax warp
@@ -41,7 +38,6 @@ constexpr int kAtBiasTile = AT_BLK * 16 * 2;      // 4 KB: one 128 x 16 bf16 til
 constexpr int kAtBias = 7 * kAtBiasTile;          // a tile of ones, then three buffers of (LSE tile, D tile)
 constexpr int kAtSmem = 4 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/ +
                         kAtBias;
-constexpr float kLog2e = 1.4426950408889634f;
 
 struct AttnParams {
   int BH, S, nblk;
@@ -68,24 +64,6 @@ struct AttnParams {
   float p_scale, ds_scale;
 };
 
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-
-// 2^x on the special-function unit (2^-inf = 0): one instruction per probability.
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// Two floats to one packed bf16 pair (round to nearest even): `lo` in bits 0..15, `hi` in 16..31.
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  uint32_t d;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-  return d;
-}
-
 // Two floats rounded to the nearest FP8 grid value (ties to even, saturating: what f8_rn_value
 // gives) and packed as a bf16 pair, through the hardware conversions: f32 pair -> FP8 pair -> f16 pair
 // (every FP8 value is an f16 value) -> f32 -> bf16 pair (every FP8 value is a bf16 value too).
@@ -97,20 +75,6 @@ __device__ __forceinline__ uint32_t f8_grid_bf16x2(float lo, float hi) {
   else asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(h2) : "h"(c));
   const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2));
   return pack_bf16x2(f.x, f.y);
-}
-
-// tcgen05.ld of 32 columns without the wait, so several loads can be in flight before one wait.
-__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
 }
 
 // FP8: the FP8-operand mode (per-head operand scales, P and dS rounded onto the FP8 grids); a
@@ -1000,69 +964,7 @@ attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig,
   }
 }
 
-// S1 += times * (g - ref), S2 += times * (g - ref)^2, elementwise (times = 1: one draw; K: a value
-// that is the same for K draws).
-__global__ void mc_accumulate_kernel(const float* __restrict__ g, const float* __restrict__ ref, float* __restrict__ S1,
-                                     float* __restrict__ S2, size_t n4, float times) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n4) return;
-  const float4 a = __ldg(reinterpret_cast<const float4*>(g) + i), r = __ldg(reinterpret_cast<const float4*>(ref) + i);
-  float4 s1 = reinterpret_cast<float4*>(S1)[i], s2 = reinterpret_cast<float4*>(S2)[i];
-  const float d0 = a.x - r.x, d1 = a.y - r.y, d2 = a.z - r.z, d3 = a.w - r.w;
-  s1.x = fmaf(times, d0, s1.x); s1.y = fmaf(times, d1, s1.y); s1.z = fmaf(times, d2, s1.z); s1.w = fmaf(times, d3, s1.w);
-  s2.x = fmaf(times * d0, d0, s2.x); s2.y = fmaf(times * d1, d1, s2.y);
-  s2.z = fmaf(times * d2, d2, s2.z); s2.w = fmaf(times * d3, d3, s2.w);
-  reinterpret_cast<float4*>(S1)[i] = s1;
-  reinterpret_cast<float4*>(S2)[i] = s2;
-}
-
-// The same over nd draws held back to back (g[d * stride + i]), in draw order: one launch instead of
-// nd for a tensor as small as the correction term.
-__global__ void mc_accumulate_draws_kernel(const float* __restrict__ g, size_t stride, int nd,
-                                           const float* __restrict__ ref, float* __restrict__ S1,
-                                           float* __restrict__ S2, size_t n4) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n4) return;
-  const float4 r = __ldg(reinterpret_cast<const float4*>(ref) + i);
-  float4 s1 = reinterpret_cast<float4*>(S1)[i], s2 = reinterpret_cast<float4*>(S2)[i];
-  for (int d = 0; d < nd; ++d) {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(g + (size_t)d * stride) + i);
-    const float d0 = a.x - r.x, d1 = a.y - r.y, d2 = a.z - r.z, d3 = a.w - r.w;
-    s1.x += d0; s1.y += d1; s1.z += d2; s1.w += d3;
-    s2.x = fmaf(d0, d0, s2.x); s2.y = fmaf(d1, d1, s2.y); s2.z = fmaf(d2, d2, s2.z); s2.w = fmaf(d3, d3, s2.w);
-  }
-  reinterpret_cast<float4*>(S1)[i] = s1;
-  reinterpret_cast<float4*>(S2)[i] = s2;
-}
-
 // ------------------------------------------------------------------------------- host side
-
-// FP32 output [BH][S][64] as two 32-column boxes per 128-row block (128-byte swizzle).
-static int make_out_map(CUtensorMap* map, const void* base, int BH, int S) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return BSP_ERR_CUDA;
-  cuuint64_t gdim[3] = {(cuuint64_t)AT_D, (cuuint64_t)S, (cuuint64_t)BH};
-  cuuint64_t gstr[2] = {(cuuint64_t)AT_D * 4, (cuuint64_t)S * AT_D * 4};
-  cuuint32_t box[3] = {32u, (cuuint32_t)AT_BLK, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), gdim, gstr, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
-}
-
-static int make_head_map(CUtensorMap* map, const void* base, int BH, int S) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return BSP_ERR_CUDA;
-  cuuint64_t gdim[3] = {(cuuint64_t)AT_D, (cuuint64_t)S, (cuuint64_t)BH};
-  cuuint64_t gstr[2] = {(cuuint64_t)AT_D * 2, (cuuint64_t)S * AT_D * 2};
-  cuuint32_t box[3] = {(cuuint32_t)AT_D, (cuuint32_t)AT_BLK, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
-}
 
 template <int MODE, bool FP8, bool DV, bool MC = false, int ND = 1>
 static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
@@ -1074,11 +976,11 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
-  static bool attr_set_dev[kMaxDevices] = {};
-  bool& attr_set = attr_set_dev[device_slot()];
-  if (!attr_set) {
+  static std::atomic<bool> attr_set_dev[kMaxDevices];       // per kernel instantiation and device
+  std::atomic<bool>& attr_set = attr_set_dev[device_slot()];
+  if (!attr_set.load(std::memory_order_acquire)) {
     BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC, ND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
-    attr_set = true;
+    attr_set.store(true, std::memory_order_release);
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
   int nsm = kNumSMs, dev = 0, sm_count = 0;
@@ -1095,7 +997,10 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
 template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   if (MODE != AT_FWD && p.mc_ref != nullptr) {               // Monte-Carlo epilogue: BF16 operands, no dV
-    if (p.fp8) return BSP_ERR_UNSUPPORTED;
+    if (p.fp8) {                                             // FP8-operand mode: one draw per launch
+      if (p.nd != 1) return BSP_ERR_UNSUPPORTED;
+      return launch_attn_mode<MODE, true, MODE != AT_DKV, MODE != AT_FWD>(q, k, v, dO, p, st);
+    }
     if (p.nd == 2) return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD, MODE != AT_FWD ? 2 : 1>(q, k, v, dO, p, st);
     return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD>(q, k, v, dO, p, st);
   }
@@ -1105,13 +1010,6 @@ static int launch_attn(const void* q, const void* k, const void* v, const void* 
 }
 
 static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
-
-static int check_attn_shape(int B, int H, int S, int Dh, int dt) {
-  if (B <= 0 || H <= 0 || S <= 0) return BSP_ERR_ARG;
-  if (Dh != AT_D || dt != BSP_BF16) return BSP_ERR_UNSUPPORTED;
-  if ((int64_t)B * H > 65535 * 16) return BSP_ERR_UNSUPPORTED;
-  return BSP_OK;
-}
 
 static int set_fp8(AttnParams& p, const bsp_attn_fp8_t* f) {
   p.fp8 = f ? 1 : 0;
@@ -1123,7 +1021,7 @@ static int set_fp8(AttnParams& p, const bsp_attn_fp8_t* f) {
   return BSP_OK;
 }
 
-static int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
                          const void* v, int dt, const bsp_attn_fp8_t* f, float* o, float* lse, bsp_diag_t* diag,
                          void* stream) {
   int rc = check_attn_shape(B, H, S, Dh, dt);
@@ -1137,10 +1035,10 @@ static int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_
   return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
 }
 
-static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
+int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
                            const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
                            bsp_key_t key, int draw0, int n_draws, float* d_out, void* stream);
-static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
                                const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* f,
                                const float* lse, const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
                                void* stream);
@@ -1152,15 +1050,16 @@ using namespace bsp;
 extern "C" {
 
 int bsp_attn_fwd_stats(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
-                       const void* v, int dt, float* o, float* lse, bsp_diag_t* diag, void* stream) {
-  return attn_fwd_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dt, nullptr, o, lse, diag, stream);
+                       const void* v, int dt, const bsp_attn_fp8_t* fp8, float* o, float* lse, bsp_diag_t* diag,
+                       void* stream) {
+  return attn_fwd_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dt, fp8, o, lse, diag, stream);
 }
 
-int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* o_orig, const uint8_t* o_codes,
-                   const float* o_scales, int o_fmt, int d_read, bsp_key_t key, int draw0, int n_draws, float* d_out,
-                   bsp_diag_t* diag, void* stream) {
+int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales, const float* o_orig,
+                   const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key, int draw0,
+                   int n_draws, float* d_out, bsp_diag_t* diag, void* stream) {
   (void)diag;
-  return attn_dterm_impl(B, H, S, Dh, dO, dt, nullptr, o_orig, o_codes, o_scales, o_fmt, d_read, key, draw0, n_draws,
+  return attn_dterm_impl(B, H, S, Dh, dO, dt, do_scales, o_orig, o_codes, o_scales, o_fmt, d_read, key, draw0, n_draws,
                          d_out, stream);
 }
 
@@ -1168,7 +1067,7 @@ int bsp_attn_dterm(int B, int H, int S, int Dh, const void* dO, int dt, const fl
 
 namespace bsp {
 
-static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
+int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales,
                            const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
                            bsp_key_t key, int draw0, int n_draws, float* d_out, void* stream) {
   if (B <= 0 || H <= 0 || S <= 0 || !valid_enum(dt, 1) || !valid_enum(o_fmt, 1) || !valid_enum(d_read, 2)) return BSP_ERR_ARG;
@@ -1197,7 +1096,7 @@ static int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, 
   return BSP_OK;
 }
 
-static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
                                const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* f,
                                const float* lse, const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
                                void* stream) {
@@ -1224,25 +1123,25 @@ static int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float so
   return BSP_OK;
 }
 
-// nd (1 or 2) fresh draws of the D use for dQ and dK with the Monte-Carlo epilogue: the kernels add
-// g - ref and its square to the running sums of their gradient and write no gradient (BF16-operand
-// mode; dV is not computed).  dterm holds the draws' correction terms back to back, [nd][B*H*S]; both
-// kernels take the two draws in one launch (S, dP and P are formed once per step).  The sums must not
-// be touched by anything else while this runs.
-static int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
-                             const void* k, const void* v, const void* dO, int dt, const float* lse,
-                             const float* dterm, int nd, const float* ref_dq, float* S1q, float* S2q,
-                             const float* ref_dk, float* S1k, float* S2k, bsp_diag_t* diag, void* stream) {
+// nd (1 or 2) draws of the D use for dQ and dK with the Monte-Carlo epilogue: the kernels add g - ref
+// and its square to the running sums of their gradient and write no gradient (dV is not computed).
+// dterm holds the draws' correction terms back to back, [nd][B*H*S]; with nd = 2 (BF16-operand mode
+// only) both kernels take the two draws in one launch (S, dP and P are formed once per step).  The
+// sums must not be touched by anything else while this runs.
+int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                      const void* v, const void* dO, int dt, const bsp_attn_fp8_t* f, const float* lse,
+                      const float* dterm, int nd, const float* ref_dq, float* S1q, float* S2q, const float* ref_dk,
+                      float* S1k, float* S2k, bsp_diag_t* diag, void* stream) {
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !dO || !lse || !dterm || !ref_dq || !S1q || !S2q || !ref_dk || !S1k || !S2k) return BSP_ERR_ARG;
-  if (nd < 1 || nd > 2) return BSP_ERR_ARG;
+  if (nd < 1 || nd > 2 || (f && nd != 1)) return BSP_ERR_ARG;
   if (!aligned16(ref_dq) || !aligned16(ref_dk) || !aligned16(S1q) || !aligned16(S2q) || !aligned16(S1k) || !aligned16(S2k))
     return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
   p.lse = lse; p.lse_out = nullptr; p.diag = diag;
-  if ((rc = set_fp8(p, nullptr)) != BSP_OK) return rc;
+  if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   p.dterm = dterm; p.nd = nd;
   p.mc_ref = ref_dk; p.out0 = S1k; p.out1 = S2k;
@@ -1278,22 +1177,23 @@ quantize_decode_kernel(const uint16_t* __restrict__ x, size_t group_size, const 
 extern "C" {
 
 int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
-                       const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq,
-                       float* dk, float* dv, bsp_diag_t* diag, void* stream) {
-  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, nullptr, lse, dterm, dq, dk, dv, diag,
+                       const void* v, const void* dO, int dt, const bsp_attn_fp8_t* fp8, const float* lse,
+                       const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag, void* stream) {
+  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, fp8, lse, dterm, dq, dk, dv, diag,
                              stream);
 }
 
 int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands, const void* q,
-                 const void* k, const void* v, const void* dO, int dt, const float* lse, const float* o_orig,
-                 const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key, float* dq,
-                 float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
-  if (fp8_operands) return BSP_ERR_UNSUPPORTED;      // that mode needs the operand scales: bsp_attn_bwd_fp8
-  if (!d_out) return BSP_ERR_ARG;
-  int rc = bsp_attn_dterm(B, H, S, Dh, dO, dt, o_orig, o_codes, o_scales, o_fmt, d_read, key, (int)key.draw, 1, d_out,
-                          diag, stream);
+                 const void* k, const void* v, const void* dO, int dt, const bsp_attn_fp8_t* fp8, const float* lse,
+                 const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
+                 bsp_key_t key, float* dq, float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
+  if ((fp8_operands != 0) != (fp8 != nullptr)) return BSP_ERR_ARG;
+  if (!d_out || (fp8 && !fp8->do_scale)) return BSP_ERR_ARG;
+  int rc = attn_dterm_impl(B, H, S, Dh, dO, dt, fp8 ? fp8->do_scale : nullptr, o_orig, o_codes, o_scales, o_fmt,
+                           d_read, key, (int)key.draw, 1, d_out, stream);
   if (rc != BSP_OK) return rc;
-  return bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, lse, d_out, dq, dk, dv, diag, stream);
+  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, fp8, lse, d_out, dq, dk, dv, diag,
+                             stream);
 }
 
 int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax, float* scales,
@@ -1315,207 +1215,6 @@ int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, v
                                                            reinterpret_cast<uint16_t*>(xq), n8);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
-}
-
-int bsp_attn_fwd_stats_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8, const void* k8,
-                           const void* v8, int dt, const bsp_attn_fp8_t* fp8, float* o, float* lse, bsp_diag_t* diag,
-                           void* stream) {
-  if (!fp8) return BSP_ERR_ARG;
-  return attn_fwd_impl(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dt, fp8, o, lse, diag, stream);
-}
-
-int bsp_attn_bwd_fp8(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q8, const void* k8,
-                     const void* v8, const void* dO8, int dt, const bsp_attn_fp8_t* fp8, const float* lse,
-                     const float* o_orig, const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read,
-                     bsp_key_t key, float* dq, float* dk, float* dv, float* d_out, bsp_diag_t* diag, void* stream) {
-  if (!fp8 || !d_out || !fp8->do_scale) return BSP_ERR_ARG;
-  int rc = attn_dterm_impl(B, H, S, Dh, dO8, dt, fp8->do_scale, o_orig, o_codes, o_scales, o_fmt, d_read, key,
-                           (int)key.draw, 1, d_out, stream);
-  if (rc != BSP_OK) return rc;
-  return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q8, k8, v8, dO8, dt, fp8, lse, d_out, dq, dk, dv, diag,
-                             stream);
-}
-
-int bsp_mc_accumulate(const float* g, const float* g_ref, float* S1, float* S2, size_t n, void* stream) {
-  if (!g || !g_ref || !S1 || !S2) return BSP_ERR_ARG;
-  if (n % 4 != 0) return BSP_ERR_UNSUPPORTED;
-  if (!aligned16(g) || !aligned16(g_ref) || !aligned16(S1) || !aligned16(S2)) return BSP_ERR_ALIGN;
-  if (n == 0) return BSP_OK;
-  const size_t n4 = n / 4;
-  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, (cudaStream_t)stream>>>(g, g_ref, S1, S2, n4, 1.0f);
-  BSP_LAUNCH_CHECK();
-  return BSP_OK;
-}
-
-}  // extern "C"
-
-// ------------------------------------------------------------------------------- per-use check, attention
-
-namespace bsp {
-
-// bsp_mc_accumulate for a value that is the same in `times` draws.
-static int mc_accumulate_times(const float* g, const float* g_ref, float* S1, float* S2, size_t n, float times,
-                               cudaStream_t st) {
-  if (n % 4 != 0) return BSP_ERR_UNSUPPORTED;
-  if (n == 0) return BSP_OK;
-  const size_t n4 = n / 4;
-  mc_accumulate_kernel<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(g, g_ref, S1, S2, n4, times);
-  BSP_LAUNCH_CHECK();
-  return BSP_OK;
-}
-
-struct AttnCheckBuffers {
-  float *o, *lse, *amax, *scales, *d_ref, *d_pol, *d_draws;
-  uint8_t* codes;
-  float *g_ref[3], *g_pol[3], *S1[3], *S2[3], *S1d, *S2d;
-  void* ws_stats;
-  size_t b_stats;
-};
-
-static size_t attn_carve(const bsp_attn_desc_t* op, int K, char* base, AttnCheckBuffers* out) {
-  size_t off = 0;
-  auto take = [&](size_t bytes) -> void* {
-    void* p = base ? base + off : nullptr;
-    off += round_up(bytes ? bytes : 1, 256);
-    return p;
-  };
-  const size_t BH = (size_t)op->B * op->H, rows = BH * op->S, n = rows * op->Dh;
-  AttnCheckBuffers c;
-  c.o = (float*)take(n * 4); c.lse = (float*)take(rows * 4);
-  c.amax = (float*)take(BH * 4); c.scales = (float*)take(BH * 4);
-  c.d_ref = (float*)take(rows * 4); c.d_pol = (float*)take(rows * 4);
-  c.d_draws = (float*)take(rows * 4 * (size_t)(K > 0 ? K : 1));
-  c.codes = (uint8_t*)take(n);
-  for (int t = 0; t < 3; ++t) {
-    c.g_ref[t] = (float*)take(n * 4); c.g_pol[t] = (float*)take(n * 4);
-    c.S1[t] = (float*)take(n * 4); c.S2[t] = (float*)take(n * 4);
-  }
-  c.S1d = (float*)take(rows * 4); c.S2d = (float*)take(rows * 4);
-  c.b_stats = kMaxPendingStats * kStatSlotBytes;
-  c.ws_stats = take(c.b_stats);
-  if (out) *out = c;
-  return off;
-}
-
-}  // namespace bsp
-
-extern "C" {
-
-size_t bsp_mc_check_attn_workspace_bytes(const bsp_attn_desc_t* op, int K) {
-  if (!op || op->B <= 0 || op->H <= 0 || op->S <= 0 || op->Dh <= 0) return 0;
-  return bsp::attn_carve(op, K, nullptr, nullptr);
-}
-
-#define BSP_TRY(expr)              \
-  do {                             \
-    int _rc = (expr);              \
-    if (_rc != BSP_OK) return _rc; \
-  } while (0)
-
-int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, bsp_use_result_t* results, int* n_results, void* ws,
-                      size_t ws_bytes, bsp_diag_t* diag, void* stream) {
-  using namespace bsp;
-  if (!op || !results || !n_results || K < 2) return BSP_ERR_ARG;
-  if (!op->q || !op->k || !op->v || !op->dO) return BSP_ERR_ARG;
-  int rc = check_attn_shape(op->B, op->H, op->S, op->Dh, op->dtype);
-  if (rc != BSP_OK) return rc;
-  if (!ws || ws_bytes < bsp_mc_check_attn_workspace_bytes(op, K) || (reinterpret_cast<uintptr_t>(ws) & 255u))
-    return BSP_ERR_WORKSPACE;
-  cudaStream_t st = (cudaStream_t)stream;
-  AttnCheckBuffers b;
-  attn_carve(op, K, reinterpret_cast<char*>(ws), &b);
-  const int B = op->B, H = op->H, S = op->S, Dh = op->Dh, dt = op->dtype;
-  const size_t BH = (size_t)B * H, rows = BH * S, n = rows * Dh;
-  const float c = op->softmax_scale;
-  *n_results = 0;
-
-  // ---- once: forward output and LSE, the output store (per-(b,h) amax scale, stream 0)
-  BSP_TRY(bsp_attn_fwd_stats(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, dt, b.o, b.lse, diag, st));
-  BSP_TRY(bsp_amax(b.o, BSP_F32, BH, (size_t)S * Dh, b.amax, diag, st));
-  BSP_TRY(bsp_scale_from_amax(b.amax, BH, op->store_fmt, b.scales, st));
-  bsp_key_t key;
-  key.seed = op->seed; key.tensor_id = op->tensor_id; key.stream = BSP_STREAM_FORWARD; key.draw = 0; key.reserved = 0;
-  BSP_TRY(bsp_round_grouped(b.o, BSP_F32, BH, (size_t)S * Dh, op->store_fmt, op->forward_mode, b.scales, key, b.codes,
-                            diag, st));
-  key.stream = BSP_STREAM_ATTN_D;
-
-  // ---- reference: D reads the original output
-  BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_ORIGINAL, key, 0, 1,
-                         b.d_ref, diag, st));
-  BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, b.d_ref, b.g_ref[0],
-                             b.g_ref[1], b.g_ref[2], diag, st));
-  // the twelve statistics passes are read behind one synchronisation at the end
-  PendingStats pend;
-  pend.slots = reinterpret_cast<double*>(b.ws_stats);
-  pend.st = st;
-  int nres = 0;
-  const int out_ids[4] = {BSP_OUT_D, BSP_OUT_DQ, BSP_OUT_DK, BSP_OUT_DV};
-  auto emit = [&](int out, int pol) -> bsp_use_result_t* {
-    bsp_use_result_t* r = &results[nres++];
-    memset(r, 0, sizeof(*r));
-    r->use_id = BSP_STREAM_ATTN_D; r->output_id = out; r->policy = pol;
-    return r;
-  };
-  for (int pol = 0; pol < 2; ++pol) {
-    if (!((op->policy_mask >> pol) & 1u)) continue;
-    const float* dsrc = b.d_ref;
-    float* const* gsrc = b.g_ref;
-    if (pol == BSP_READ_FORWARD) {
-      BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_FORWARD, key, 0,
-                             1, b.d_pol, diag, st));
-      BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, b.d_pol,
-                                 b.g_pol[0], b.g_pol[1], b.g_pol[2], diag, st));
-      dsrc = b.d_pol;
-      gsrc = b.g_pol;
-    }
-    BSP_TRY(pend.add(b.d_ref, dsrc, nullptr, (int64_t)rows, 1, 0, emit(out_ids[0], pol)));
-    for (int t = 0; t < 3; ++t)
-      BSP_TRY(pend.add(b.g_ref[t], gsrc[t], nullptr, (int64_t)n, 1, 0, emit(out_ids[t + 1], pol)));
-  }
-  if ((op->policy_mask >> 2) & 1u) {
-    // fresh read: all K correction terms in one pass, then one backward per draw
-    BSP_TRY(bsp_attn_dterm(B, H, S, Dh, op->dO, dt, b.o, b.codes, b.scales, op->store_fmt, BSP_READ_FRESH, key, 0, K,
-                           b.d_draws, diag, st));
-    BSP_CHECK_CUDA(cudaMemsetAsync(b.S1d, 0, rows * 4, st));
-    BSP_CHECK_CUDA(cudaMemsetAsync(b.S2d, 0, rows * 4, st));
-    for (int t = 0; t < 3; ++t) {
-      BSP_CHECK_CUDA(cudaMemsetAsync(b.S1[t], 0, n * 4, st));
-      BSP_CHECK_CUDA(cudaMemsetAsync(b.S2[t], 0, n * 4, st));
-    }
-    // the sums of D itself over all K draws, in one launch (rows = B*H*S is a multiple of 4 or the
-    // draws go one by one)
-    if (rows % 4 == 0) {
-      mc_accumulate_draws_kernel<<<(unsigned)((rows / 4 + 255) / 256), 256, 0, st>>>(b.d_draws, rows, K, b.d_ref, b.S1d,
-                                                                                   b.S2d, rows / 4);
-      BSP_LAUNCH_CHECK();
-    }
-    for (int k = 0; k < K; ++k) {
-      const float* dk_ = b.d_draws + (size_t)k * rows;
-      if (rows % 4 != 0) BSP_TRY(bsp_mc_accumulate(dk_, b.d_ref, b.S1d, b.S2d, rows, st));
-      if (k > 0) {
-        // the draws after the first, two at a time: dQ and dK go from the accumulators straight into
-        // their sums
-        const int nd = k + 1 < K ? 2 : 1;
-        if (nd == 2 && rows % 4 != 0) BSP_TRY(bsp_mc_accumulate(dk_ + rows, b.d_ref, b.S1d, b.S2d, rows, st));
-        BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, nd,
-                                  b.g_ref[0], b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
-        k += nd - 1;
-        continue;
-      }
-      // the first draw: the whole backward, gradients written.  dV does not read the correction
-      // term, so its value under the fresh read is the same for every draw: it is computed here only
-      // and enters the sums K times
-      BSP_TRY(bsp_attn_bwd_dterm(B, H, S, Dh, op->causal, c, op->q, op->k, op->v, op->dO, dt, b.lse, dk_, b.g_pol[0],
-                                 b.g_pol[1], b.g_pol[2], diag, st));
-      for (int t = 0; t < 2; ++t) BSP_TRY(bsp_mc_accumulate(b.g_pol[t], b.g_ref[t], b.S1[t], b.S2[t], n, st));
-      BSP_TRY(mc_accumulate_times(b.g_pol[2], b.g_ref[2], b.S1[2], b.S2[2], n, (float)K, st));
-    }
-    BSP_TRY(pend.add(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH)));
-    for (int t = 0; t < 3; ++t)
-      BSP_TRY(pend.add(b.g_ref[t], b.S1[t], b.S2[t], (int64_t)n, K, 1, emit(out_ids[t + 1], BSP_READ_FRESH)));
-  }
-  *n_results = nres;
-  return pend.flush();
 }
 
 }  // extern "C"

@@ -25,6 +25,7 @@
 namespace bsp {
 
 void count_launch();          // defined in mc.cu
+void count_d2h(size_t bytes);  // bytes the library itself copies device -> host (mc.cu)
 
 constexpr int kNumSMs = 148;
 

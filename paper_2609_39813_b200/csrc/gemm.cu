@@ -11,6 +11,7 @@
 // in order, so the Monte-Carlo epilogue's read-modify-write of the shifted sums is race-free and
 // bit-reproducible.  Every wait is bounded; on time-out the kernel records BSP_ERR_TIMEOUT in the
 // diagnostics word and unwinds (TMEM is freed on every path).
+#include <atomic>
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -604,11 +605,11 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
     if (rc != BSP_OK) return rc;
     p.idesc = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, MC_BN);
     p.idesc2 = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, 2 * MC_BN);
-    static bool mc_attr_set_dev[kMaxDevices] = {};
-    bool& mc_attr_set = mc_attr_set_dev[device_slot()];
-    if (!mc_attr_set) {
+    static std::atomic<bool> mc_attr_set_dev[kMaxDevices];
+    std::atomic<bool>& mc_attr_set = mc_attr_set_dev[device_slot()];
+    if (!mc_attr_set.load(std::memory_order_acquire)) {
       BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
-      mc_attr_set = true;
+      mc_attr_set.store(true, std::memory_order_release);
     }
     const int ntiles_mc = (int)(((g.M + BM - 1) / BM) * ((g.N + MC_BN - 1) / MC_BN));
     const int grid_mc = ntiles_mc < nsm ? ntiles_mc : nsm;
@@ -619,12 +620,12 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
 
   rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, BN, g.b_mn);
   if (rc != BSP_OK) return rc;
-  static bool attr_set_dev[kMaxDevices][2] = {};
-  bool* attr_set = attr_set_dev[device_slot()];
-  if (!attr_set[g.fp8 ? 1 : 0]) {
+  static std::atomic<bool> attr_set_dev[kMaxDevices][2];
+  std::atomic<bool>* attr_set = attr_set_dev[device_slot()];
+  if (!attr_set[g.fp8 ? 1 : 0].load(std::memory_order_acquire)) {
     if (g.fp8) BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
     else BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem));
-    attr_set[g.fp8 ? 1 : 0] = true;
+    attr_set[g.fp8 ? 1 : 0].store(true, std::memory_order_release);
   }
   const int ntiles = (int)(((g.M + BM - 1) / BM) * ((g.N + BN - 1) / BN));
   const int grid = ntiles < nsm ? ntiles : nsm;

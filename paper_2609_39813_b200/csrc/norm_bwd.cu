@@ -24,9 +24,9 @@ template <int DT, int DU_DT, int FMT, int JMAX, int NT>
 __global__ void __launch_bounds__(NT, 1024 / NT)
 norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                 const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
-                const void* __restrict__ du, int gain_read, const uint8_t* __restrict__ u_codes, float scale_val,
-                const float* __restrict__ scale_dev, PhiloxKey key, float* __restrict__ part_g,
-                float* __restrict__ part_b, float* __restrict__ dx) {
+                const void* __restrict__ du, int gain_read, int dx_read, const uint8_t* __restrict__ u_codes,
+                float scale_val, const float* __restrict__ scale_dev, PhiloxKey key, PhiloxKey key_dx,
+                float* __restrict__ part_g, float* __restrict__ part_b, float* __restrict__ dx) {
   __shared__ float red[2][2][NT / 32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float scale = scale_dev ? __ldg(scale_dev) : scale_val;
@@ -91,21 +91,18 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
                              __fmul_rn(__fsub_rn(xv.z, mu), rs), __fmul_rn(__fsub_rn(xv.w, mu), rs));
         }
         dz[j] = make_float4(g4[j].x * d4[j].x, g4[j].y * d4[j].y, g4[j].z * d4[j].z, g4[j].w * d4[j].w);
-        if (dx) {
-          p1 += (dz[j].x * z[j].x + dz[j].y * z[j].y) + (dz[j].z * z[j].z + dz[j].w * z[j].w);
-          p2 += (dz[j].x + dz[j].y) + (dz[j].z + dz[j].w);
-        }
-
-        // ---- gain use: z_g under the policy
-        float4 zg = z[j];
-        if (gain_read != BSP_READ_ORIGINAL) {
+        // z as a use reads it: the original, or (copy - beta) / gamma from the forward's codes (R)
+        // or from a fresh stochastic rounding under the use's own generator stream (N)
+        const float4 zo = z[j];
+        auto z_read = [&](int policy, const PhiloxKey& kk) -> float4 {
+          if (policy == BSP_READ_ORIGINAL) return zo;
           float dec[4];
-          if (gain_read == BSP_READ_FORWARD) {
+          if (policy == BSP_READ_FORWARD) {
             const uint32_t pk = __ldg(reinterpret_cast<const uint32_t*>(u_codes + i0));
             f8_decode4<FMT>(pk, dec);
           } else {
-            const uint4 w = philox_block(key, (uint64_t)i0 >> 2, key.c2);
-            const float u[4] = {z[j].x, z[j].y, z[j].z, z[j].w};
+            const uint4 w = philox_block(kk, (uint64_t)i0 >> 2, kk.c2);
+            const float u[4] = {zo.x, zo.y, zo.z, zo.w};
             const float gg[4] = {g4[j].x, g4[j].y, g4[j].z, g4[j].w};
             const float bb[4] = {b4[j].x, b4[j].y, b4[j].z, b4[j].w};
             const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
@@ -119,10 +116,14 @@ norm_bwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, cons
           // (copy - beta) / gamma as a multiplication by the per-column reciprocal (one rounding
           // more than a division, far inside the FP32 tolerance; the division would cost ten
           // instructions per element on a pass that has about that many to spend)
-          zg.x = (dec[0] * inv_scale - b4[j].x) * rg4[j].x;
-          zg.y = (dec[1] * inv_scale - b4[j].y) * rg4[j].y;
-          zg.z = (dec[2] * inv_scale - b4[j].z) * rg4[j].z;
-          zg.w = (dec[3] * inv_scale - b4[j].w) * rg4[j].w;
+          return make_float4((dec[0] * inv_scale - b4[j].x) * rg4[j].x, (dec[1] * inv_scale - b4[j].y) * rg4[j].y,
+                             (dec[2] * inv_scale - b4[j].z) * rg4[j].z, (dec[3] * inv_scale - b4[j].w) * rg4[j].w);
+        };
+        const float4 zg = z_read(gain_read, key);
+        if (dx) {
+          if (dx_read != BSP_READ_ORIGINAL) z[j] = z_read(dx_read, key_dx);   // the input gradient's own read
+          p1 += (dz[j].x * z[j].x + dz[j].y * z[j].y) + (dz[j].z * z[j].z + dz[j].w * z[j].w);
+          p2 += (dz[j].x + dz[j].y) + (dz[j].z + dz[j].w);
         }
         accg[j].x = fmaf(zg.x, d4[j].x, accg[j].x); accg[j].y = fmaf(zg.y, d4[j].y, accg[j].y);
         accg[j].z = fmaf(zg.z, d4[j].z, accg[j].z); accg[j].w = fmaf(zg.w, d4[j].w, accg[j].w);
@@ -212,7 +213,8 @@ __global__ void __launch_bounds__(NW * 32, NW == 8 ? 3 : 4)
 gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
-               int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */) {
+               int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */,
+               bsp_diag_t* __restrict__ diag) {
   // A fresh rounding of an element is its round-down value plus, with probability frac, one grid
   // step: value(U) = lo + (U < P) * (hi - lo) with the threshold P of f8_sr_threshold.  So the
   // gain-use sum of draw k is  sum_t (lo/scale - beta)/gamma * du  (the same for every draw, summed
@@ -243,6 +245,7 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
   const uint64_t q0 = (uint64_t)((slab * (NW * ROWS) + warp) * C + (col_ok ? c : 0)) >> 2;
   const uint64_t qstep = (uint64_t)(NW * C) / 4;
   float base[4] = {0.f, 0.f, 0.f, 0.f};                 // the draw-independent part of this thread's sums
+  DiagCounters dc;                                       // non-finite x or du, counted once per element
 #pragma unroll 1
   for (int i = 0; i < ROWS; ++i) {
     const int64_t r = slab * (NW * ROWS) + warp + NW * i;
@@ -265,6 +268,7 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
         else u = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xs[e], mu), rs), gg[e]), bb[e]);
         const float v = __fmul_rn(u, scale);
         const float w = __fdiv_rn(ds[e], gg[e]);
+        if (!isfinite(xs[e]) || !isfinite(ds[e])) dc.nonfinite++;
         const float lo = sr_value<FMT>(v, 0xFFFFFFFFu), hi = sr_value<FMT>(v, 0u);   // never up / up whenever possible
         thr[e] = f8_sr_threshold<FMT>(v);
         base[e] = fmaf(fmaf(lo, inv_scale, -bb[e]), w, base[e]);
@@ -274,6 +278,7 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
     sp[i * NT + tid] = make_uint4(thr[0], thr[1], thr[2], thr[3]);
     sw[i * NT + tid] = make_float4(wgt[0], wgt[1], wgt[2], wgt[3]);
   }
+  diag_flush_warp(diag, dc);                             // (the host hands diag to the first chunk of draws only)
   for (int k = 0; k < ndraws; ++k) {
     const uint32_t draw = (uint32_t)(draw_begin + k);
     float acc[4] = {base[0], base[1], base[2], base[3]};
@@ -345,16 +350,16 @@ static int bwd_grid(int64_t T) {
 template <int DT, int DU_DT, int FMT>
 static int launch_norm_bwd(int jmax, int grid, cudaStream_t st, int kind, const void* x, int64_t T, int64_t C,
                            const float* gamma, const float* beta, const float* rstd, const float* mean,
-                           const void* du, int gain_read, const uint8_t* u_codes, bsp_quant_t q, PhiloxKey key,
-                           float* part_g, float* part_b, float* dx) {
+                           const void* du, int gain_read, int dx_read, const uint8_t* u_codes, bsp_quant_t q,
+                           PhiloxKey key, PhiloxKey key_dx, float* part_g, float* part_b, float* dx) {
   // jmax encodes the launch shape: C/4 column groups over 256, 512 or 1024 threads, two groups per
   // thread only beyond 4096 columns
   (void)jmax;
   const int64_t groups = C / 4;
 #define BSP_NB(J, NT)                                                                                        \
   norm_bwd_kernel<DT, DU_DT, FMT, J, NT><<<grid, NT, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
-                                                               gain_read, u_codes, q.scale, q.scale_dev, key, \
-                                                               part_g, part_b, dx)
+                                                               gain_read, dx_read, u_codes, q.scale,           \
+                                                               q.scale_dev, key, key_dx, part_g, part_b, dx)
   if (groups <= 256) BSP_NB(1, 256);
   else if (groups <= 512) BSP_NB(1, 512);
   else if (groups <= 1024) BSP_NB(1, 1024);
@@ -378,11 +383,11 @@ size_t bsp_norm_bwd_workspace_bytes(int64_t T, int64_t C) {
 }
 
 int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma, const float* beta,
-                 const float* rstd, const float* mean, const void* du, int du_dt, int gain_read,
+                 const float* rstd, const float* mean, const void* du, int du_dt, int gain_read, int dx_read,
                  const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key, float* dgamma, float* dbeta, float* dx,
                  void* ws, size_t ws_bytes, bsp_diag_t* diag, void* stream) {
   if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(gain_read, 2) ||
-      !valid_enum(q.fmt, 1))
+      !valid_enum(dx_read, 2) || !valid_enum(q.fmt, 1))
     return BSP_ERR_ARG;
   if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
   if (T < 0 || C <= 0) return BSP_ERR_ARG;
@@ -394,7 +399,8 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
     return BSP_OK;
   }
   if (!x || !gamma || !rstd || !du || (kind == BSP_LAYERNORM && (!beta || !mean))) return BSP_ERR_ARG;
-  if (gain_read == BSP_READ_FORWARD && !u_codes) return BSP_ERR_ARG;
+  if (!dx) dx_read = BSP_READ_ORIGINAL;                        // no input gradient asked for: nothing reads
+  if ((gain_read == BSP_READ_FORWARD || dx_read == BSP_READ_FORWARD) && !u_codes) return BSP_ERR_ARG;
   if (C % 4 != 0 || C > 8192) return BSP_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(du) || !aligned16(gamma) || !aligned16(beta) || !aligned16(dx) ||
       (reinterpret_cast<uintptr_t>(u_codes) & 3u))
@@ -402,7 +408,9 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
   if (!ws || ws_bytes < bsp_norm_bwd_workspace_bytes(T, C) || (reinterpret_cast<uintptr_t>(ws) & 255u))
     return BSP_ERR_WORKSPACE;
   // whole stages of 256-column multiples take the streamed kernel, every other shape the plain one
-  const StreamPlan plan = plan_stream(T, C, dt, du_dt, gain_read, x, du, u_codes);
+  // (an input gradient that reads a copy is outside the reference and takes the plain kernel too)
+  StreamPlan plan = plan_stream(T, C, dt, du_dt, gain_read, x, du, u_codes);
+  if (dx_read != BSP_READ_ORIGINAL) plan.ok = false;
   const int grid = plan.ok ? plan.grid : bwd_grid(T);
   float* part_g = reinterpret_cast<float*>(ws);
   float* part_b = dbeta ? reinterpret_cast<float*>(reinterpret_cast<char*>(ws) +
@@ -411,12 +419,15 @@ int bsp_norm_bwd(int kind, const void* x, int dt, int64_t T, int64_t C, const fl
   const int64_t groups = (C / 4 + 255) / 256;
   const int jmax = groups <= 1 ? 1 : groups <= 2 ? 2 : groups <= 4 ? 4 : 8;
   const PhiloxKey pk = make_key(key);
+  bsp_key_t key_dx = key;                                      // the input gradient's own generator stream
+  key_dx.stream = BSP_STREAM_DX;
+  const PhiloxKey pk_dx = make_key(key_dx);
   int rc;
 #define BSP_CALL(DT, DU, FMT)                                                                                 \
   rc = plan.ok ? launch_norm_bwd_stream<DT, DU, FMT>(plan, st, kind, x, T, C, gamma, beta, rstd, mean, du,    \
                                                      gain_read, u_codes, q, pk, part_g, part_b, dx, diag)     \
                : launch_norm_bwd<DT, DU, FMT>(jmax, grid, st, kind, x, T, C, gamma, beta, rstd, mean, du,     \
-                                              gain_read, u_codes, q, pk, part_g, part_b, dx)
+                                              gain_read, dx_read, u_codes, q, pk, pk_dx, part_g, part_b, dx)
   if (q.fmt == BSP_E4M3) {
     if (dt == BSP_F32 && du_dt == BSP_F32) BSP_CALL(BSP_F32, BSP_F32, BSP_E4M3);
     else if (dt == BSP_F32) BSP_CALL(BSP_F32, BSP_BF16, BSP_E4M3);
@@ -466,7 +477,6 @@ int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int6
                      const float* beta, const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q,
                      bsp_key_t key, int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
                      bsp_diag_t* diag, void* stream) {
-  (void)diag;
   if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(q.fmt, 1)) return BSP_ERR_ARG;
   if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
   if (T < 0 || C <= 0 || K < 0 || draw0 < 0) return BSP_ERR_ARG;
@@ -493,14 +503,14 @@ int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int6
   do {                                                                                                          \
     if (thin) {                                                                                                 \
       gain_mc_kernel<DT, DU, FMT, kMcThinWarps, kMcThinRows><<<grid, kMcThinWarps * 32, kMcThinSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du, \
-                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd, partial); \
+                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd, partial, kb == 0 ? diag : nullptr); \
       break;                                                                                                    \
     }                                                                                                           \
     BSP_CHECK_CUDA(cudaFuncSetAttribute(gain_mc_kernel<DT, DU, FMT, 8, kMcRows>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                         (int)kMcSmemBytes));                                                    \
     gain_mc_kernel<DT, DU, FMT, 8, kMcRows><<<grid, 256, kMcSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
                                                                  q.scale, q.scale_dev, pk, draw0 + kb, nd,      \
-                                                                 partial);                                      \
+                                                                 partial, kb == 0 ? diag : nullptr);            \
   } while (0)
       if (q.fmt == BSP_E4M3) {
         if (dt == BSP_F32 && du_dt == BSP_F32) BSP_GM(BSP_F32, BSP_F32, BSP_E4M3);
@@ -562,8 +572,8 @@ extern "C" {
 
 int bsp_norm_bwd_noalloc(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                          const float* beta, const float* rstd, const float* mean, const void* du, int du_dt,
-                         int gain_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key, float* dgamma,
-                         float* dbeta, float* dx, bsp_diag_t* diag, void* stream) {
+                         int gain_read, int dx_read, const uint8_t* u_codes, bsp_quant_t q, bsp_key_t key,
+                         float* dgamma, float* dbeta, float* dx, bsp_diag_t* diag, void* stream) {
   // size check first: pure host arithmetic, nothing is touched when the problem does not fit
   if (T < 0 || C <= 0) return BSP_ERR_ARG;
   const size_t need = bsp_norm_bwd_workspace_bytes(T, C);
@@ -573,8 +583,8 @@ int bsp_norm_bwd_noalloc(int kind, const void* x, int dt, int64_t T, int64_t C, 
   if (rc != BSP_OK) return rc;
   // The column partials this pass keeps in scratch are written in full before they are read, so
   // whatever an earlier call left in the array is harmless and nothing has to be cleared.
-  return bsp_norm_bwd(kind, x, dt, T, C, gamma, beta, rstd, mean, du, du_dt, gain_read, u_codes, q, key, dgamma,
-                      dbeta, dx, scratch, bsp::kNoAllocScratchBytes, diag, stream);
+  return bsp_norm_bwd(kind, x, dt, T, C, gamma, beta, rstd, mean, du, du_dt, gain_read, dx_read, u_codes, q, key,
+                      dgamma, dbeta, dx, scratch, bsp::kNoAllocScratchBytes, diag, stream);
 }
 
 }  // extern "C"

@@ -239,7 +239,16 @@ norm_bwd_stream_kernel(const void* __restrict__ x, int64_t T, int64_t C, int64_t
     }
   }
   if (failed) {
+    // a bounded wait ran out: the status says so, and the block's column partials are written as NaN
+    // so that dgamma / dbeta come out recognisably invalid instead of being summed from whatever the
+    // workspace held before
     if (tid == 0 && diag) atomicMax(&diag->status, (int)BSP_ERR_TIMEOUT);
+    const float4 bad = make_float4(NAN, NAN, NAN, NAN);
+#pragma unroll
+    for (int j = 0; j < kNJ; ++j) {
+      *reinterpret_cast<float4*>(part_g + (size_t)blockIdx.x * C + col[j]) = bad;
+      if (part_b) *reinterpret_cast<float4*>(part_b + (size_t)blockIdx.x * C + col[j]) = bad;
+    }
     return;
   }
 #pragma unroll

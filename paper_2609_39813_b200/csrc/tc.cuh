@@ -43,16 +43,20 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legiti
 
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the limit is hit or another
 // role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (global_timer_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs);
 }
 
 // The same bounded wait for barriers that whole blocks wait on: each try suspends the thread in

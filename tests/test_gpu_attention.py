@@ -1,6 +1,13 @@
-"""Attention on the GPU (forward statistics, the D use under the three reads, backward) against
-the float64 oracle.  Tensor-core products: <= 2e-3 relative L2 per tensor; D is CUDA-core FP32:
-<= 1e-5; codes of the output store bit-exact."""
+"""Attention on the GPU (forward statistics, the D use under the three reads, backward, the per-use
+check) against the float64 oracle in its plain form: every product on unrounded operands.
+
+Tolerances (relative L2 per tensor): D is CUDA-core FP32: <= 1e-5; codes of the output store
+bit-exact; products whose operands are the inputs themselves (O, and everything in the FP8-operand
+mode, where the oracle rounds at the same points): <= 2e-3; the BF16-operand backward, whose
+computed operands P and dS are rounded to bf16 before dV, dQ and dK: <= 3e-3 against the plain
+definition (the operand rounding alone is 1.5e-3 .. 1.8e-3 on these inputs: 2^-9 per element,
+uniformly distributed, times the cancellation in the sums); the same outputs against the oracle
+with that operand rounding applied are kept as a diagnostic at 2e-3."""
 import numpy as np
 import pytest
 
@@ -13,6 +20,7 @@ from paper_2609_39813_b200 import workloads
 pytestmark = pytest.mark.gpu
 
 TOL_TC = 2e-3
+TOL_TC_BF16_OPERANDS = 3e-3
 TOL_FP32 = 1e-5
 
 
@@ -128,12 +136,16 @@ def test_backward_against_oracle(b, case, policy):
     for idx, q, k, v, dO in _slices(inp):
         prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, g.causal, o32=o[idx])
         copy = check.attention_d_copy(prep, policy, inp.seed, 0)
-        # P and dS enter their products as bf16 tensor-core operands: the oracle rounds them alike
-        want = attention.backward(q, k, v, dO, inp.softmax_scale, copy, g.causal,
-                                  operand_round=linear.bf16_round)
+        want = attention.backward(q, k, v, dO, inp.softmax_scale, copy, g.causal)
+        # diagnostic: the same with P and dS rounded to bf16 as the tensor-core operands are
+        diag_want = attention.backward(q, k, v, dO, inp.softmax_scale, copy, g.causal,
+                                       operand_round=linear.bf16_round)
         for name in ("dq", "dk", "dv"):
             assert np.isfinite(got[name][idx]).all(), name
-            assert _rel(got[name][idx], want[name]) <= TOL_TC, (name, idx)
+            dist = _rel(got[name][idx], want[name])
+            print("bf16-operand backward vs plain oracle: %s slice %d rel-L2 %.3e" % (name, idx, dist))
+            assert dist <= TOL_TC_BF16_OPERANDS, (name, idx, dist)
+            assert _rel(got[name][idx], diag_want[name]) <= TOL_TC, (name, idx)
 
 
 def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
@@ -165,44 +177,61 @@ def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
     assert not torch.equal(outs[0][0], outs[2][0])                         # dQ does
 
 
-def test_mc_check_attention_verdicts(b):
-    """The whole per-use check of the D use on a small workload: verdicts identical to the oracle's
-    (U holds exactly, R fails, N holds on average; dV is untouched by the read), statistics close."""
-    from oracle import mc
-    inp = workloads.config3(B=1, H=2, S=192, D=64, K=24, seed=77)
-    g = AttnGpu(b, inp, True)
+def _attn_desc(b, g, inp, K, mask, fp8_operands=0, p_scale=256.0, ds_scale=1.0):
     d = b.AttnDesc()
     d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = inp.B, inp.H, inp.S, inp.D, 1, inp.softmax_scale, b.BF16
     d.q, d.k, d.v, d.dO = b.ptr(g.q), b.ptr(g.k), b.ptr(g.v), b.ptr(g.dO)
-    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, 7
+    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, mask
+    d.fp8_operands, d.p_scale, d.ds_scale = fp8_operands, p_scale, ds_scale
+    return d
+
+
+def _pooled(parts, K, fresh):
+    """Oracle statistics of a tensor given slice by slice: pool the per-slice (ref, mean, m2)."""
+    from oracle import mc
+    ref = np.concatenate([p["ref"].ravel() for p in parts])
+    mean = np.concatenate([p["mean"].ravel() for p in parts])
+    m2 = np.concatenate([p["m2"].ravel() for p in parts]) if fresh else None
+    return mc.statistics(mean, m2, K if fresh else 1, ref, fresh)
+
+
+def test_mc_check_attention_verdicts(b):
+    """The whole per-use check of the D use on a small workload against the PLAIN oracle (unrounded
+    operands): U holds exactly on every output; R fails on D, dQ, dK; N holds on average on D, dQ and
+    dK (they are affine in D); dV is untouched by the read."""
+    from oracle import mc
+    inp = workloads.config3(B=1, H=2, S=192, D=64, K=24, seed=77)
+    g = AttnGpu(b, inp, True)
+    d = _attn_desc(b, g, inp, inp.K, 7)
     ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, inp.K))
     diag = b.new_diag()
     res = b.bsp_mc_check_attn(d, inp.K, ws, diag)
     assert len(res) == 12 and b.read_diag(diag)["status"] == 0
     assert [(r.policy, r.output_id) for r in res] == [(p, o) for p in (0, 1, 2) for o in (b.OUT_D, b.OUT_DQ, b.OUT_DK, b.OUT_DV)]
     H_, F_ = mc.HOLDS, mc.FAILS
-    # U: everything exact.  R: D, dQ, dK fail, dV is untouched.  N: the use's own output D holds on
-    # average and dV is untouched.  (dQ and dK under N are compared with the oracle below: their
-    # products round dS to bf16, which is not linear in D, so their fresh-draw means carry a
-    # quantisation bias that is not the D use's fault -- the D-use verdict is the one on D.)
-    got = [r.verdict for r in res]
-    assert got[:8] == [H_, H_, H_, H_, F_, F_, F_, H_] and got[8] == H_ and got[11] == H_
+    assert [r.verdict for r in res] == [H_, H_, H_, H_, F_, F_, F_, H_, H_, H_, H_, H_]
+    assert all(r.informational == 0 for r in res)
     for r in res[:4]:
         assert r.rel_l2_mean_err == 0.0
     assert res[7].rel_l2_mean_err == 0.0 and res[11].rel_l2_mean_err == 0.0 and res[11].R == 0.0     # dV
-    # the oracle on the same stored output (slice by slice; statistics pooled over the slices for D)
+    # the plain oracle on the same stored output, slice by slice, pooled over the slices
     o = g.o.cpu().numpy().reshape(inp.B * inp.H, inp.S, inp.D)
+    per = {pol: [] for pol in (0, 1, 2)}
     for idx, q, k, v, dO in _slices(inp):
         prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, True, o32=o[idx])
         for pol in (0, 1, 2):
-            want = check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, pol, inp.K, inp.seed,
-                                         operand_round=linear.bf16_round)
-            for j, name in enumerate(("D", "dq", "dk", "dv")):
-                assert want[name]["stats"].verdict == res[4 * pol + j].verdict, (pol, name)
-        # with unrounded operands the fresh read holds on average for dQ and dK too (the paper's
-        # statement about the D use); the bias above is the bf16 operand format's, not the read's
-        exact = check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, 2, inp.K, inp.seed)
-        assert [exact[n_]["stats"].verdict for n_ in ("D", "dq", "dk", "dv")] == [H_, H_, H_, H_]
+            per[pol].append(check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, pol, inp.K, inp.seed))
+    for pol in (0, 1, 2):
+        for j, name in enumerate(("D", "dq", "dk", "dv")):
+            want = _pooled([s_[name] for s_ in per[pol]], inp.K, pol == 2)
+            got = res[4 * pol + j]
+            assert want.verdict == got.verdict, (pol, name, want, got.as_dict())
+            if pol == 1 and name != "dv":
+                assert np.isclose(got.rel_l2_mean_err, want.rel_l2_mean_err, rtol=2e-2), (name, got.rel_l2_mean_err)
+            if pol == 2 and name != "dv":
+                # same draws, same differences; the GPU forms them from bf16 operands
+                for f in ("rel_l2_mean_err", "R", "Qprime", "rms_z"):
+                    assert np.isclose(getattr(got, f), getattr(want, f), rtol=1e-2), (name, f, getattr(got, f), getattr(want, f))
     # R's error on D is the size of the store's rounding error, as for the norm store
     assert 0.005 < res[4].rel_l2_mean_err < 0.5
     # determinism
@@ -210,76 +239,49 @@ def test_mc_check_attention_verdicts(b):
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
 
 
-@pytest.mark.parametrize("K", [4, 7, 8])
-def test_mc_check_attention_fused_sums_match_draw_by_draw(b, K):
-    """Inside the check the draws after the first go two at a time through kernels that add g - g*
-    and its square straight into the running sums.  The same statistics taken draw by draw through
-    the single-draw entry points (gradient written, then accumulated) must agree: same draws, same
-    per-draw arithmetic, only the order of a few FP32 additions differs.  K = 4: one plain draw, a
-    pair and a single fused draw; K = 7: three pairs; K = 8: three pairs and a single draw left over.
-    S = 328: three blocks, the last one ragged."""
+@pytest.mark.parametrize("K", [4, 7, 9])
+def test_mc_check_attention_draw_groups(b, K):
+    """The fresh read takes the draws of dK four at a time (K = 4: one full group; 7: a group and a
+    group of three; 9: two groups and a single draw) and collapses the draws of dQ into one pass.
+    Statistics against the plain oracle on S = 328 (three blocks, the last one ragged), six slices."""
     inp = workloads.config3(B=2, H=3, S=328, D=64, K=K, seed=91)
     g = AttnGpu(b, inp, True)
-    B, H, S, D, K = inp.B, inp.H, inp.S, inp.D, inp.K
-    rows, n = B * H * S, B * H * S * D
-    d = b.AttnDesc()
-    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, inp.softmax_scale, b.BF16
-    d.q, d.k, d.v, d.dO = b.ptr(g.q), b.ptr(g.k), b.ptr(g.v), b.ptr(g.dO)
-    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, 4
+    d = _attn_desc(b, g, inp, K, 4)
     ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
     diag = b.new_diag()
     res = b.bsp_mc_check_attn(d, K, ws, diag)
     assert b.read_diag(diag)["status"] == 0
-    assert [(r.policy, r.output_id) for r in res] == [(2, o) for o in (b.OUT_D, b.OUT_DQ, b.OUT_DK, b.OUT_DV)]
-    # draw by draw, through the public single-draw calls
-    key = b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0)
-    d_ref = torch.zeros(rows, device="cuda")
-    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, g.codes, g.scales, fp8.E4M3, b.READ_ORIGINAL, key, 0, 1, d_ref)
-    ref = [torch.zeros(n, device="cuda") for _ in range(3)]
-    b.bsp_attn_bwd_dterm(B, H, S, D, True, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, d_ref, *ref)
-    d_draws = torch.zeros(K * rows, device="cuda")
-    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, g.codes, g.scales, fp8.E4M3, b.READ_FRESH, key, 0, K, d_draws)
-    S1 = [torch.zeros(n, device="cuda") for _ in range(2)]
-    S2 = [torch.zeros(n, device="cuda") for _ in range(2)]
-    gk = [torch.zeros(n, device="cuda") for _ in range(2)]
-    for k in range(K):
-        b.bsp_attn_bwd_dterm(B, H, S, D, True, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse,
-                             d_draws[k * rows:(k + 1) * rows], gk[0], gk[1], None)
-        for t in range(2):
-            b.bsp_mc_accumulate(gk[t], ref[t], S1[t], S2[t], n)
-    wss = b.workspace(b.bsp_mc_stats_workspace_bytes(n))
-    for t in range(2):
-        want = b.bsp_mc_stats(ref[t], S1[t], S2[t], n, K, 1, wss)
-        got = res[1 + t]
-        assert got.verdict == want.verdict and got.K == want.K and got.n_elements == want.n_elements
-        for f in ("rel_l2_mean_err", "R", "Qprime", "mean_z", "rms_z", "max_abs_z", "frac_abs_z_gt3"):
+    assert [(r.policy, r.output_id) for r in res] == [(2, o_) for o_ in (b.OUT_D, b.OUT_DQ, b.OUT_DK, b.OUT_DV)]
+    o = g.o.cpu().numpy().reshape(inp.B * inp.H, inp.S, inp.D)
+    parts = []
+    for idx, q, k, v, dO in _slices(inp):
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, True, o32=o[idx])
+        parts.append(check.attention_d_use(q, k, v, dO, inp.softmax_scale, prep, 2, K, inp.seed))
+    for j, name in enumerate(("D", "dq", "dk")):
+        want = _pooled([p_[name] for p_ in parts], K, True)
+        got = res[j]
+        assert got.K == K and got.n_elements == want.n_elements
+        tol = 1e-4 if name == "D" else 1e-2
+        for f in ("rel_l2_mean_err", "R", "Qprime", "rms_z", "frac_abs_z_gt3"):
             x, y = getattr(got, f), getattr(want, f)
-            # the mean of the signed z-scores is a cancellation of values of size rms_z: that is its scale
-            scale = max(abs(y), want.rms_z if f == "mean_z" else 1e-3)
-            assert x == y or abs(x - y) <= 2e-3 * scale, (t, f, x, y)
+            assert np.isclose(x, y, rtol=tol, atol=2e-3 if f == "frac_abs_z_gt3" else 0), (name, f, x, y)
+        assert got.verdict == want.verdict
 
 
-@pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks", "many_items_ragged"])
-def test_fp8_operand_mode(b, name):
-    """The emulated FP8 attention backward: Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice, P rounded
-    to E4M3 at scale 256 before dV, dS rounded to E5M2 at a supplied scale before dQ and dK."""
+def _quantised_operands(b, inp):
+    """Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice on the GPU, and the oracle's values of the same."""
     from paper_2609_39813_b200.harness import up
-    cfg = CASES[name]
-    inp = workloads.config3(B=cfg["B"], H=cfg["H"], S=cfg["S"], D=64, K=4, seed=2000 + cfg["S"])
     B, H, S, D = inp.B, inp.H, inp.S, inp.D
     BH, n = B * H, B * H * S * D
-    dev = {}
+    dev, hat = {}, {}
     for nm, arr, fmt in (("q", inp.q, fp8.E4M3), ("k", inp.k, fp8.E4M3), ("v", inp.v, fp8.E4M3), ("dO", inp.dO, fp8.E5M2)):
         x = up(arr, "bf16")
         xq = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
         amax, sc = torch.zeros(BH, device="cuda"), torch.zeros(BH, device="cuda")
         b.bsp_attn_quantize(x, BH, S * D, fmt, xq, amax, sc)
         dev[nm] = (xq, sc)
-    # quantised operands: bit-exact against the oracle's nearest rounding at the slice's amax scale
-    hat = {}
-    for nm, arr, fmt in (("q", inp.q, fp8.E4M3), ("k", inp.k, fp8.E4M3), ("v", inp.v, fp8.E4M3), ("dO", inp.dO, fp8.E5M2)):
-        got = dev[nm][0].float().cpu().numpy().reshape(BH, S, D)
-        scs = dev[nm][1].cpu().numpy()
+        got = xq.float().cpu().numpy().reshape(BH, S, D)
+        scs = sc.cpu().numpy()
         vals = np.zeros((BH, S, D))
         for idx in range(BH):
             value, codes, s32, _ = attention.quantise_rn(arr.reshape(BH, S, D)[idx], fmt)
@@ -287,6 +289,64 @@ def test_fp8_operand_mode(b, name):
             assert np.array_equal(got[idx], fp8.decode(codes, fmt).astype(np.float32))
             vals[idx] = value
         hat[nm] = vals
+    return dev, hat
+
+
+def test_mc_check_attention_fp8_operand_mode(b):
+    """The check in the FP8-operand mode: the rounded backward runs once per draw.  The use's own
+    output D carries the verdict (N holds); dQ and dK pass through the nearest rounding of dS and are
+    reported as information.  Against the oracle's emulated backward with the same quantisation
+    points, slice by slice."""
+    from oracle import mc
+    K = 12
+    inp = workloads.config3(B=1, H=2, S=200, D=64, K=K, seed=314)
+    g = AttnGpu(b, inp, True)
+    dev, hat = _quantised_operands(b, inp)
+    o0, _ = attention.forward_output(hat["q"][0], hat["k"][0], hat["v"][0], inp.softmax_scale, True)
+    ds0 = attention.backward(hat["q"][0], hat["k"][0], hat["v"][0], hat["dO"][0], inp.softmax_scale, o0, True)["dS"]
+    ds_scale = float(np.float32(2.0 ** np.floor(np.log2(57344.0 / (2.0 * np.max(np.abs(ds0)))))))
+    d = _attn_desc(b, g, inp, K, 7, fp8_operands=1, p_scale=256.0, ds_scale=ds_scale)
+    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+    diag = b.new_diag()
+    res = b.bsp_mc_check_attn(d, K, ws, diag)
+    assert len(res) == 12 and b.read_diag(diag)["status"] == 0
+    assert [r.informational for r in res] == [0] * 8 + [0, 1, 1, 0]
+    H_, F_ = mc.HOLDS, mc.FAILS
+    got = [r.verdict for r in res]
+    assert got[:8] == [H_, H_, H_, H_, F_, F_, F_, H_] and got[8] == H_ and got[11] == H_
+    # the forward output the check stored: recomputed through the same entry point
+    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale)
+    n = inp.B * inp.H * inp.S * inp.D
+    o, lse = torch.zeros(n, device="cuda"), torch.zeros(inp.B * inp.H * inp.S, device="cuda")
+    b.bsp_attn_fwd_stats(inp.B, inp.H, inp.S, inp.D, True, inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], o, lse, fp8=f)
+    oh = o.cpu().numpy().reshape(inp.B * inp.H, inp.S, inp.D)
+    per = {pol: [] for pol in (1, 2)}
+    for idx in range(inp.B * inp.H):
+        qh, kh, vh, dOh = hat["q"][idx], hat["k"][idx], hat["v"][idx], hat["dO"][idx]
+        prep = check.prepare_attention_slice(qh, kh, vh, dOh, inp.softmax_scale, inp.seed, idx, True, o32=oh[idx])
+        for pol in (1, 2):
+            per[pol].append(check.attention_d_use(qh, kh, vh, dOh, inp.softmax_scale, prep, pol, K, inp.seed,
+                                                  fp8_operands=True, scale_p=256.0, scale_ds=ds_scale))
+    for pol in (1, 2):
+        for j, name in enumerate(("D", "dq", "dk")):
+            want = _pooled([s_[name] for s_ in per[pol]], K, pol == 2)
+            r = res[4 * pol + j]
+            assert np.isclose(r.rel_l2_mean_err, want.rel_l2_mean_err, rtol=5e-2), (pol, name, r.rel_l2_mean_err, want.rel_l2_mean_err)
+            if name == "D":
+                assert r.verdict == want.verdict
+                if pol == 2:
+                    assert np.isclose(r.R, want.R, rtol=1e-3) and np.isclose(r.Qprime, want.Qprime, rtol=1e-3)
+
+
+@pytest.mark.parametrize("name", ["two_blocks_ragged", "three_blocks", "many_items_ragged"])
+def test_fp8_operand_mode(b, name):
+    """The emulated FP8 attention backward: Q, K, V -> E4M3 and dO -> E5M2 per (b,h) slice, P rounded
+    to E4M3 at scale 256 before dV, dS rounded to E5M2 at a supplied scale before dQ and dK."""
+    cfg = CASES[name]
+    inp = workloads.config3(B=cfg["B"], H=cfg["H"], S=cfg["S"], D=64, K=4, seed=2000 + cfg["S"])
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    BH, n = B * H, B * H * S * D
+    dev, hat = _quantised_operands(b, inp)
     # one dS scale for the whole tensor, from the exact dS of the first slice (a "previous amax")
     o0, _ = attention.forward_output(hat["q"][0], hat["k"][0], hat["v"][0], inp.softmax_scale, cfg["causal"])
     ds0 = attention.backward(hat["q"][0], hat["k"][0], hat["v"][0], hat["dO"][0], inp.softmax_scale, o0, cfg["causal"])["dS"]
@@ -294,12 +354,16 @@ def test_fp8_operand_mode(b, name):
     f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale)
     o, lse = torch.zeros(n, device="cuda"), torch.zeros(BH * S, device="cuda")
     diag = b.new_diag()
-    b.bsp_attn_fwd_stats_fp8(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], f, o, lse, diag)
+    b.bsp_attn_fwd_stats(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], o, lse, diag, fp8=f)
     dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
     d_out = torch.zeros(BH * S, device="cuda")
-    b.bsp_attn_bwd_fp8(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], dev["dO"][0],
-                       f, lse, o, None, None, fp8.E4M3, 0, b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0),
-                       dq, dk, dv, d_out, diag)
+    key = b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0)
+    # the flag and the scales must agree
+    with pytest.raises(b.BspError):
+        b.bsp_attn_bwd(B, H, S, D, cfg["causal"], inp.softmax_scale, 1, dev["q"][0], dev["k"][0], dev["v"][0], dev["dO"][0],
+                       lse, o, None, None, fp8.E4M3, 0, key, dq, dk, dv, d_out, diag)
+    b.bsp_attn_bwd(B, H, S, D, cfg["causal"], inp.softmax_scale, 1, dev["q"][0], dev["k"][0], dev["v"][0], dev["dO"][0],
+                   lse, o, None, None, fp8.E4M3, 0, key, dq, dk, dv, d_out, diag, fp8=f)
     assert b.read_diag(diag)["status"] == 0
     oh = o.cpu().numpy().reshape(BH, S, D)
     for idx in range(BH):
@@ -341,3 +405,37 @@ def test_attention_row_case_of_the_paper(b):
         for h, want in ((sig * a, float(t_dev)), (a, float(t_fixed))):
             T = (dq_at(s + tau * a, h) - dq_at(s + sig * a, h)) / c
             assert abs(T - want) <= 1e-6, (sig, tau, h, T, want)
+
+
+def test_attention_row_case_fp8_operands_exact(b):
+    """The same eight cells in the FP8-operand mode, the setting of the paper's operator test: every
+    deciding value is representable (unit operand scales, P = 1/64 -> 4 at scale 256, dS = +-2^-9 or 0
+    at unit scale), so the deviation is exactly zero."""
+    from paper_2609_39813_b200.harness import up
+    S, D, a, s, c = 64, 64, 0.25, 1.25, 0.125
+    q = np.zeros((1, 1, S, D), np.float32); q[..., 1] = 1.0
+    k = np.zeros((1, 1, S, D), np.float32); k[..., 0] = 1.0
+    v = np.zeros((1, 1, S, D), np.float32); v[0, 0, :, 0] = np.where(np.arange(S) % 2 == 0, 1.0, 1.5)
+    qd, kd, vd = up(q, "bf16"), up(k, "bf16"), up(v, "bf16")
+    one = torch.ones(1, device="cuda")
+    f = b.attn_fp8(one, one, one, one, 256.0, 1.0)
+    o = torch.zeros(S * D, device="cuda"); lse = torch.zeros(S, device="cuda")
+    b.bsp_attn_fwd_stats(1, 1, S, D, True, c, qd, kd, vd, o, lse, fp8=f)
+    cells = [l.split() for l in open(golden_path("attention_row_cells.txt")) if l[0] in "+-"]
+
+    def dq_at(x, h):
+        dO = np.zeros((1, 1, S, D), np.float32); dO[0, 0, 63, 0] = h
+        saved = o.clone(); saved[63 * D] = x
+        dq = torch.zeros(S * D, device="cuda"); d_out = torch.zeros(S, device="cuda")
+        b.bsp_attn_bwd(1, 1, S, D, True, c, 1, qd, kd, vd, up(dO, "bf16"), lse, saved, None, None, fp8.E4M3, 0,
+                       b.key(0, 2, 4, 0), dq, None, None, d_out, fp8=f)
+        return float(dq.cpu().numpy().reshape(S, D)[63, 0])
+
+    for sig, tau, t_dev, t_fixed in cells:
+        sig, tau = float(sig), float(tau)
+        for h, want in ((sig * a, float(t_dev)), (a, float(t_fixed))):
+            # the closed form itself: dQ[63, 0] = c h (s - x), with no deviation
+            assert dq_at(s + tau * a, h) == c * h * (s - (s + tau * a))
+            T = (dq_at(s + tau * a, h) - dq_at(s + sig * a, h)) / c
+            assert T == want, (sig, tau, h, T, want)
+

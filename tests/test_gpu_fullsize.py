@@ -31,7 +31,7 @@ def _rel(a, ref):
 
 FULL = {
     "cfg2": (workloads.config2, 64),
-    "cfg4": (workloads.config4, 32),      # K = 1024 in the config; 32 draws here keep the test short
+    "cfg4": (workloads.config4, 1024),
     "cfg5": (workloads.config5, 16),
 }
 
@@ -158,20 +158,67 @@ def test_full_weight_use(b, full):
     assert _rel(down(S2).reshape(O, C)[pick], s2) <= 2e-2
 
 
-def test_full_mc_check_verdicts(b, full):
-    inp, g, K = full["inp"], full["g"], full["K"]
+def test_full_mc_check_verdicts_and_sampled_statistics(b, full):
+    """The whole check at the configuration's own K (config 4: 1024 draws in 16 chunks), then the
+    per-element sums it leaves in the workspace against the oracle on seeded sub-blocks: eight columns
+    of dgamma (all tokens, all draws) and a 48 x 8 block of dW."""
+    from paper_2609_39813_b200.harness import down
+    inp, g, K, kind, prep = full["inp"], full["g"], full["K"], full["kind"], dict(full["prep"])
+    T, C, O = inp.T, inp.C, inp.O
     desc = g.desc()
     ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
     diag = b.new_diag()
     res = b.bsp_mc_check(desc, K, ws, diag)
     assert b.read_diag(diag)["status"] == 0
-    # gain use: U holds exactly, R fails, N holds on average; weight use: U fails, R holds exactly,
-    # N fails (its mean tends to the original's value)
-    assert [r.verdict for r in res] == [mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS]
-    assert res[0].rel_l2_mean_err == 0.0 and res[4].rel_l2_mean_err == 0.0
-    assert 0.005 < res[1].rel_l2_mean_err < 0.5 and 0.005 < res[3].rel_l2_mean_err < 0.5
-    assert res[2].Qprime < 1.6 and res[2].R < 2.0 and res[5].R > 6.0
-    assert [r.n_elements for r in res] == [inp.C] * 3 + [inp.O * inp.C] * 3
+    # gain use: U holds exactly, R fails, N holds on average (dbeta holds under every read); weight use:
+    # U fails, R holds exactly, N fails (its mean tends to the original's value)
+    H_, F_ = mc.HOLDS, mc.FAILS
+    assert [r.verdict for r in res] == [H_, H_, F_, H_, H_, H_, F_, H_, F_]
+    assert res[0].rel_l2_mean_err == 0.0 and res[7].rel_l2_mean_err == 0.0
+    assert 0.005 < res[2].rel_l2_mean_err < 0.5 and 0.005 < res[6].rel_l2_mean_err < 0.5
+    assert res[4].Qprime < 1.6 and res[4].R < 2.0 and res[8].R > 6.0
+    assert [r.n_elements for r in res] == [C] * 6 + [O * C] * 3
+    # ---- sampled statistics
+    lay = b.bsp_mc_check_layout(desc, K)
+    dt = torch.bfloat16 if inp.dtype == "bf16" else torch.float32
+    rng = np.random.default_rng(21)
+    cols = np.sort(rng.choice(C, 8, replace=False))
+    rows = np.sort(rng.choice(O, 48, replace=False))
+    du = down(b.ws_view(ws, lay.du, T * C, dt)).reshape(T, C)[:, cols].astype(np.float64)
+    gam, bet = inp.gamma[cols], (inp.beta[cols] if inp.beta is not None else None)
+    z = prep["fw"]["z"][:, cols]
+    g_ref = np.sum(z * du, axis=0)
+    assert _rel(down(b.ws_view(ws, lay.dgamma_ref, C))[cols], g_ref) <= TOL_FP32
+    amax_dy = np.float32(np.max(np.abs(inp.dY)))
+    s_dy, inv_dy = fp8.scale_from_amax(amax_dy, inp.grad_fmt)
+    dyc, _, _ = fp8.encode((inp.dY[:, rows] * np.float32(s_dy)).astype(np.float32), inp.grad_fmt, fp8.RN)
+    dy = fp8.decode(dyc, inp.grad_fmt) * float(inv_dy)
+    w_ref = dy.T @ norm.read_value(prep["codes"][:, cols], inp.store_fmt, prep["inv_scale"])
+    accg, accw = mc.Welford(g_ref.shape), mc.Welford(w_ref.shape)
+    for k in range(K):
+        cg, _ = check.fresh_copy(prep, inp.seed, philox.STREAM_GAIN, k, cols)
+        accg.add(norm.dgamma_from_copy(cg, gam, bet, du))
+        cw, _ = check.fresh_copy(prep, inp.seed, philox.STREAM_WGRAD, k, cols)
+        accw.add(dy.T @ cw)
+    ref32 = down(b.ws_view(ws, lay.dgamma_ref, C))[cols]
+    mean_g, m2_g = mc.shifted_sums_to_moments(down(b.ws_view(ws, lay.dgamma_S1, C))[cols],
+                                              down(b.ws_view(ws, lay.dgamma_S2, C))[cols], K, ref32)
+    assert _rel(mean_g, accg.mean) <= TOL_FP32
+    assert _rel(m2_g, accg.m2) <= 2e-3
+    pick = np.ix_(rows, cols)
+    wref32 = down(b.ws_view(ws, lay.dW_ref, O * C)).reshape(O, C)[pick]
+    assert _rel(wref32, w_ref) <= TOL_TC
+    mean_w, m2_w = mc.shifted_sums_to_moments(down(b.ws_view(ws, lay.dW_S1, O * C)).reshape(O, C)[pick],
+                                              down(b.ws_view(ws, lay.dW_S2, O * C)).reshape(O, C)[pick], K, wref32)
+    assert _rel(mean_w, accw.mean) <= TOL_TC
+    assert _rel(m2_w, accw.m2) <= 1e-2
+    # per-element z-scores of the sampled dW block, as config 4 asks for them
+    n = O * C
+    zz = torch.zeros(n, device="cuda")
+    b.bsp_mc_moments(b.ws_view(ws, lay.dW_ref, n), b.ws_view(ws, lay.dW_S1, n), b.ws_view(ws, lay.dW_S2, n), n, K, None, None, zz)
+    z_or = (accw.mean - w_ref) / np.sqrt(accw.m2 / (K - 1) / K)
+    z_gpu = down(zz).reshape(O, C)[pick]
+    assert np.max(np.abs(z_gpu - z_or)) <= 0.05 + 2e-2 * np.max(np.abs(z_or))
 
 
 def test_full_attention_sampled_heads(b):
@@ -206,7 +253,64 @@ def test_full_attention_sampled_heads(b):
         prep = check.prepare_attention_slice(qs, ks, vs, dOs, inp.softmax_scale, inp.seed, idx, True, o32=oh[idx])
         assert np.array_equal(ch[idx], prep["codes"])
         copy = check.attention_d_copy(prep, pol, inp.seed, draw)
-        want = attention.backward(qs, ks, vs, dOs, inp.softmax_scale, copy, True, operand_round=linear.bf16_round)
+        want = attention.backward(qs, ks, vs, dOs, inp.softmax_scale, copy, True)
         assert _rel(d_out.cpu().numpy().reshape(B * H, S)[idx], want["D"]) <= TOL_FP32
         for name, t in (("dq", dq), ("dk", dk), ("dv", dv)):
-            assert _rel(t.cpu().numpy().reshape(B * H, S, D)[idx], want[name]) <= TOL_TC, (name, idx)
+            # P and dS enter their products rounded to bf16: 3e-3 against the plain definition
+            dist = _rel(t.cpu().numpy().reshape(B * H, S, D)[idx], want[name])
+            print("config 3, slice %d, %s vs plain oracle: rel-L2 %.3e" % (idx, name, dist))
+            assert dist <= 3e-3, (name, idx, dist)
+
+
+@pytest.mark.parametrize("fp8_operands", [0, 1])
+def test_full_attention_check(b, fp8_operands):
+    """bsp_mc_check_attn on config 3 as defined (K = 32), all three policies, in both operand modes.
+    Verdicts: the paper's table for the D use.  Statistics of the fresh read on D itself against the
+    oracle on two (batch, head) slices (rows of those slices pooled): D is CUDA-core FP32, so the
+    per-row sums agree closely; in BF16-operand mode also the mean error of dQ and dK under R."""
+    from paper_2609_39813_b200.harness import up
+    inp = workloads.config3()
+    B, H, S, D, K = inp.B, inp.H, inp.S, inp.D, inp.K
+    q, k, v, dO = (up(a, "bf16") for a in (inp.q, inp.k, inp.v, inp.dO))
+    d = b.AttnDesc()
+    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, inp.softmax_scale, b.BF16
+    d.q, d.k, d.v, d.dO = b.ptr(q), b.ptr(k), b.ptr(v), b.ptr(dO)
+    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = fp8.E4M3, fp8.SR, inp.seed, check.TENSOR_O, 7
+    d.fp8_operands, d.p_scale, d.ds_scale = fp8_operands, 256.0, 1024.0
+    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+    diag = b.new_diag()
+    res = b.bsp_mc_check_attn(d, K, ws, diag)
+    assert len(res) == 12 and b.read_diag(diag)["status"] == 0
+    H_, F_ = mc.HOLDS, mc.FAILS
+    got = [r.verdict for r in res]
+    assert got[:8] == [H_, H_, H_, H_, F_, F_, F_, H_] and got[8] == H_ and got[11] == H_
+    if not fp8_operands:
+        assert got[9] == H_ and got[10] == H_          # dQ and dK are affine in D
+        assert all(r.informational == 0 for r in res)
+    else:
+        assert [r.informational for r in res[8:]] == [0, 1, 1, 0]
+    if fp8_operands:
+        return
+    # the oracle on two slices, against the per-slice part of what the check left: D sums are not
+    # exported, so compare through the public single entry points on the same stored output
+    n = B * H * S * D
+    o, lse = torch.zeros(n, device="cuda"), torch.zeros(B * H * S, device="cuda")
+    b.bsp_attn_fwd_stats(B, H, S, D, True, inp.softmax_scale, q, k, v, o, lse)
+    oh = o.cpu().numpy().reshape(B * H, S, D)
+    parts = {1: [], 2: []}
+    for idx in (17, 100):
+        bi, hi = divmod(idx, H)
+        qs, ks, vs, dOs = inp.q[bi, hi], inp.k[bi, hi], inp.v[bi, hi], inp.dO[bi, hi]
+        prep = check.prepare_attention_slice(qs, ks, vs, dOs, inp.softmax_scale, inp.seed, idx, True, o32=oh[idx])
+        parts[1].append(check.attention_d_use(qs, ks, vs, dOs, inp.softmax_scale, prep, 1, K, inp.seed))
+        parts[2].append(check.attention_d_use(qs, ks, vs, dOs, inp.softmax_scale, prep, 2, 8, inp.seed))
+    # R: the mean error of every output is the size the oracle finds on the sampled slices (pooled
+    # over 2 of 128 slices: a sample, so the comparison is loose); N: the oracle's sampled slices hold
+    for j, name in enumerate(("D", "dq", "dk")):
+        ref = np.concatenate([p_[name]["ref"].ravel() for p_ in parts[1]])
+        mean = np.concatenate([p_[name]["mean"].ravel() for p_ in parts[1]])
+        want_rel = np.linalg.norm(mean - ref) / np.linalg.norm(ref)
+        assert 0.5 * want_rel < res[4 + j].rel_l2_mean_err < 2.0 * want_rel, (name, want_rel, res[4 + j].rel_l2_mean_err)
+        assert all(p_[name]["stats"].verdict == mc.HOLDS for p_ in parts[2])
+        assert 0.5 < res[8 + j].Qprime < 1.5 and res[8 + j].R < 2.0
+

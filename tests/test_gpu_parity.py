@@ -338,14 +338,52 @@ def test_mc_statistics_match_oracle(b):
     assert np.isclose(r1.rel_l2_mean_err, 0.01, rtol=1e-4) and r1.verdict == mc.FAILS
 
 
+@pytest.mark.parametrize("dx_read", [1, 2])
+def test_input_gradient_reading_a_copy(b, case, dx_read):
+    """dx with z read from the forward's codes (R) or from a fresh rounding under the input
+    gradient's own generator stream (N); the gain use keeps reading the original."""
+    inp, g, kind, prep = case
+    T, C = inp.T, inp.C
+    du = up(prep["du"].astype(np.float32), inp.dtype)
+    dg, db, dx = torch.zeros(C, device="cuda"), torch.zeros(C, device="cuda"), torch.zeros(T * C, device="cuda")
+    ws = b.workspace(b.bsp_norm_bwd_workspace_bytes(T, C))
+    draw = 2
+    b.bsp_norm_bwd(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, du, 0, g.u_codes, g.q,
+                   b.key(inp.seed, g.tensor_id, b.STREAM_GAIN, draw), dg, db, dx, ws, dx_read=dx_read)
+    if dx_read == 1:
+        copy = norm.read_value(prep["codes"], inp.store_fmt, prep["inv_scale"])
+    else:
+        copy, _ = check.fresh_copy(prep, inp.seed, philox.STREAM_DX, draw)
+    want = norm.backward(inp.x, inp.gamma, inp.beta, kind, inp.eps, prep["du"], dx_copy=copy)
+    assert rel_l2(down(dg), want["dgamma"]) <= TOL_FP32
+    assert rel_l2(down(dx), want["dx"]) <= TOL_FP32
+    # and it is a different tensor from the reference's input gradient
+    ref = norm.backward(inp.x, inp.gamma, inp.beta, kind, inp.eps, prep["du"])
+    assert rel_l2(down(dx), ref["dx"]) > 1e-4
+
+
 def _oracle_table(inp, kind, prep, K):
+    """Oracle statistics in the order the check returns them: gain U (dgamma, dbeta), R, N, weight U, R, N."""
     args = (inp.x, inp.gamma, inp.beta, kind, inp.eps, prep)
     out = []
     for p in (check.U, check.R, check.N):
-        out.append(check.gain_use(*args, p, K, inp.seed)["stats"])
+        r = check.gain_use(*args, p, K, inp.seed)
+        out.append(r["stats"])
+        # dbeta reads no saved tensor: its value under every read is the reference's
+        zero = np.zeros_like(r["dbeta"])
+        out.append(mc.statistics(r["dbeta"], zero if p == check.N else None, K, r["dbeta"], p == check.N))
     for p in (check.U, check.R, check.N):
         out.append(check.wgrad_use(prep, p, K, inp.seed)["stats"])
     return out
+
+
+def _gpu_du(b, g, desc, K, ws):
+    lay = b.bsp_mc_check_layout(desc, K)
+    dt = torch.bfloat16 if g.inp.dtype == "bf16" else torch.float32
+    return lay, down(b.ws_view(ws, lay.du, g.T * g.C, dt)).reshape(g.T, g.C)
+
+
+EXPECTED_NORM_LINEAR = [mc.HOLDS, mc.HOLDS, mc.FAILS, mc.HOLDS, mc.HOLDS, mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS]
 
 
 def test_mc_check_small_configs_verdicts_and_statistics(b, case):
@@ -355,22 +393,133 @@ def test_mc_check_small_configs_verdicts_and_statistics(b, case):
     ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
     diag = b.new_diag()
     res = b.bsp_mc_check(desc, K, ws, diag)
-    assert len(res) == 6 and b.read_diag(diag)["status"] == 0
-    # the oracle takes the GPU's saved statistics; du is each side's own (the GPU's helper vs float64)
+    assert len(res) == 9 and b.read_diag(diag)["status"] == 0
+    assert [(r.use_id, r.output_id, r.policy) for r in res] == \
+        [(b.STREAM_GAIN, o, p) for p in (0, 1, 2) for o in (b.OUT_DGAMMA, b.OUT_DBETA)] + \
+        [(b.STREAM_WGRAD, b.OUT_DW, p) for p in (0, 1, 2)]
+    # the oracle takes the GPU's saved statistics and the incoming gradient du the GPU's helper made
+    # (read back from the workspace), so both sides evaluate the uses on the same received gradient
+    lay, du_gpu = _gpu_du(b, g, desc, K, ws)
     prep = check.prepare_norm_linear(inp.x, inp.gamma, inp.beta, inp.W, inp.dY, kind, inp.eps, inp.seed,
-                                     inp.dtype, rstd32=down(g.rstd), mean32=down(g.mean) if kind == norm.LAYER else None)
+                                     inp.dtype, rstd32=down(g.rstd), mean32=down(g.mean) if kind == norm.LAYER else None,
+                                     du=du_gpu)
     want = _oracle_table(inp, kind, prep, K)
-    expected = [mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS, mc.HOLDS, mc.FAILS]
-    for r, w, e in zip(res, want, expected):
+    for r, w, e in zip(res, want, EXPECTED_NORM_LINEAR):
         assert r.verdict == w.verdict == e, (r.as_dict(), w)
+        assert r.K == w.K and r.n_elements == w.n_elements
         if r.policy != b.READ_FRESH:
-            assert np.isclose(r.rel_l2_mean_err, w.rel_l2_mean_err, rtol=0.02, atol=1e-9)
+            assert np.isclose(r.rel_l2_mean_err, w.rel_l2_mean_err, rtol=2e-3, atol=1e-9)
         else:
-            assert np.isclose(r.R, w.R, rtol=0.25, atol=0.3) and np.isclose(r.Qprime, w.Qprime, rtol=0.25, atol=0.3)
-    assert res[0].rel_l2_mean_err == 0.0 and res[4].rel_l2_mean_err == 0.0
+            for f in ("rel_l2_mean_err", "R", "Qprime", "rms_z"):
+                assert np.isclose(getattr(r, f), getattr(w, f), rtol=2e-3, atol=1e-9), (r.as_dict(), w, f)
+    assert res[0].rel_l2_mean_err == 0.0 and res[7].rel_l2_mean_err == 0.0
+    for i in (1, 3, 5):          # dbeta: exactly the reference under every read
+        assert res[i].rel_l2_mean_err == 0.0 and res[i].R == 0.0 and res[i].max_abs_z == 0.0
+    # per-element moments from the workspace: mean, variance and z of dgamma under the fresh read
+    C = inp.C
+    ref = b.ws_view(ws, lay.dgamma_ref, C)
+    S1, S2 = b.ws_view(ws, lay.dgamma_S1, C), b.ws_view(ws, lay.dgamma_S2, C)
+    mean, var, z = (torch.zeros(C, device="cuda") for _ in range(3))
+    b.bsp_mc_moments(ref, S1, S2, C, K, mean, var, z)
+    gain_n = check.gain_use(inp.x, inp.gamma, inp.beta, kind, inp.eps, prep, check.N, K, inp.seed)
+    assert rel_l2(down(mean), gain_n["mean"]) <= TOL_FP32
+    assert rel_l2(down(var), gain_n["m2"] / (K - 1)) <= 2e-3
+    se = np.sqrt(gain_n["m2"] / (K - 1) / K)
+    assert rel_l2(down(z), (gain_n["mean"] - gain_n["ref"]) / se) <= 2e-3
+    # dbeta and dx of the reference are there too
+    assert rel_l2(down(b.ws_view(ws, lay.dbeta_ref, C)), np.sum(du_gpu.astype(np.float64), axis=0)) <= TOL_FP32
     # determinism: a second call returns byte-identical results
     res2 = b.bsp_mc_check(desc, K, ws, diag)
     assert [bytes(r) for r in res] == [bytes(r) for r in res2]
+
+
+def test_mc_check_draws_in_chunks(b, case):
+    """A small code buffer makes the weight use take its K draws in several chunks (re-round launch +
+    contraction launch per chunk, sums chained through memory, an odd tail): same per-element sums as
+    the one-chunk run to FP32 accumulation order, same verdicts, and the oracle's statistics."""
+    inp, g, kind, _ = case
+    K = 11
+    desc = g.desc(policy_mask=0x24)          # the two fresh reads
+    ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
+    diag = b.new_diag()
+    one = b.bsp_mc_check(desc, K, ws, diag)
+    lay = b.bsp_mc_check_layout(desc, K)
+    n = inp.O * inp.C
+    s1_one, s2_one = down(b.ws_view(ws, lay.dW_S1, n)).copy(), down(b.ws_view(ws, lay.dW_S2, n)).copy()
+    desc.draw_buffer_bytes = 3 * inp.C * g.ld_t + 7          # room for three draws: chunks 3, 3, 3, 2
+    ws2 = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
+    assert ws2.numel() < ws.numel()
+    side = torch.cuda.Stream()
+    desc.side_stream = side.cuda_stream          # and the gain kernel beside the first contraction
+    many = b.bsp_mc_check(desc, K, ws2, diag)
+    assert b.read_diag(diag)["status"] == 0
+    lay2 = b.bsp_mc_check_layout(desc, K)
+    s1, s2 = down(b.ws_view(ws2, lay2.dW_S1, n)), down(b.ws_view(ws2, lay2.dW_S2, n))
+    ref = down(b.ws_view(ws2, lay2.dW_ref, n))
+    assert np.linalg.norm(s1 - s1_one) <= 1e-5 * K * np.linalg.norm(ref)
+    assert rel_l2(s2, s2_one) <= 1e-4
+    assert [r.verdict for r in many] == [r.verdict for r in one] == [mc.HOLDS, mc.HOLDS, mc.FAILS]
+    for x, y in zip(many, one):
+        assert np.isclose(x.R, y.R, rtol=1e-3, atol=1e-9) and np.isclose(x.Qprime, y.Qprime, rtol=1e-3, atol=1e-9)
+    # against the oracle, element by element on the sums
+    _, du_gpu = _gpu_du(b, g, desc, K, ws2)
+    prep = check.prepare_norm_linear(inp.x, inp.gamma, inp.beta, inp.W, inp.dY, kind, inp.eps, inp.seed,
+                                     inp.dtype, rstd32=down(g.rstd), mean32=down(g.mean) if kind == norm.LAYER else None,
+                                     du=du_gpu)
+    w = check.wgrad_use(prep, check.N, K, inp.seed)
+    mean_gpu, m2_gpu = mc.shifted_sums_to_moments(s1.reshape(inp.O, inp.C), s2.reshape(inp.O, inp.C), K, ref.reshape(inp.O, inp.C))
+    assert rel_l2(mean_gpu, w["mean"]) <= TOL_TC and rel_l2(m2_gpu, w["m2"]) <= 1e-2
+    assert many[2].verdict == w["stats"].verdict and np.isclose(many[2].R, w["stats"].R, rtol=5e-3)
+
+
+def test_verdict_rule_is_an_argument(b):
+    """The thresholds are the caller's: the same sums read under a stricter and a looser rule."""
+    rng = np.random.default_rng(5)
+    n, K = 4096, 16
+    ref = rng.standard_normal(n).astype(np.float32)
+    d = rng.standard_normal((K, n)) * 0.1 + 0.05           # a bias of two standard errors per element
+    S1, S2 = d.sum(0).astype(np.float32), (d * d).sum(0).astype(np.float32)
+    ws = b.workspace(b.bsp_mc_stats_workspace_bytes(n))
+    args = (up(ref), up(S1), up(S2), n, K, 1, ws)
+    default = b.bsp_mc_stats(*args)
+    assert default.verdict == mc.FAILS and 4.0 < default.Qprime < 8.0
+    loose = b.bsp_mc_stats(*args, rule=b.rule(qprime_hold=10.0, r_hold=10.0, qprime_fail=20.0, r_fail=20.0))
+    assert loose.verdict == mc.HOLDS and loose.Qprime == default.Qprime
+    # "z < 2 and under x %": a magnitude bound on top of the statistics
+    bounded = b.bsp_mc_stats(*args, rule=b.rule(qprime_hold=10.0, r_hold=10.0, qprime_fail=20.0, r_fail=20.0, rel_hold=1e-3))
+    assert bounded.verdict == mc.UNDECIDED
+    det = b.bsp_mc_stats(up(ref), up(ref * np.float32(1.001)), None, n, 1, 0, ws, rule=b.rule(rel_tol_deterministic=1e-2))
+    assert det.verdict == mc.HOLDS
+    with pytest.raises(b.BspError):
+        b.bsp_mc_stats(*args, rule=b.rule(qprime_hold=5.0, qprime_fail=4.0))
+    with pytest.raises(b.BspError):          # fresh statistics need K >= 4
+        b.bsp_mc_stats(up(ref), up(S1), up(S2), n, 3, 1, ws)
+
+
+def test_a_bounded_wait_that_runs_out(b):
+    """A wait on a barrier that nothing completes gives up after its limit: the kernel returns, the
+    status word says BSP_ERR_TIMEOUT, and the device goes on working (a contraction right after)."""
+    diag = b.new_diag()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    b.bsp_selftest_bounded_wait(1_000_000, diag)          # 1 ms
+    t1.record()
+    d = b.read_diag(diag)
+    assert d["status"] == b.ERR_TIMEOUT
+    assert 0.5 <= t0.elapsed_time(t1) < 200.0
+    with pytest.raises(b.BspError):
+        b.bsp_selftest_bounded_wait(0, diag)
+    with pytest.raises(b.BspError):
+        b.bsp_selftest_bounded_wait(10**9, diag)
+    # the context is intact: a tensor-core product on the same device, against numpy
+    rng = np.random.default_rng(0)
+    A = workloads.to_bf16_grid(rng.standard_normal((128, 64)).astype(np.float32))
+    Bm = workloads.to_bf16_grid(rng.standard_normal((128, 64)).astype(np.float32))
+    Cd = torch.zeros(128 * 128, device="cuda")
+    diag2 = b.new_diag()
+    b.bsp_gemm(128, 128, 64, 2, up(A, "bf16"), 64, False, 0, up(Bm, "bf16"), 64, False, 0, 1.0, Cd, 128, diag2)
+    assert b.read_diag(diag2)["status"] == 0
+    assert rel_l2(down(Cd).reshape(128, 128), A.astype(np.float64) @ Bm.astype(np.float64).T) <= 1e-5
 
 
 def test_edge_cases(b):

@@ -62,6 +62,14 @@ def _run_both(b, inp, gain_read, draw):
     for a, r in ((dg1, dg0), (db1, db0), (dx1, dx0)):
         assert torch.isfinite(a).all() and torch.isfinite(r).all()
         assert _rel(a, r) <= TOL_FP32
+    if gain_read == b.READ_ORIGINAL:
+        # and against the float64 checker, not only against the sibling entry point
+        from oracle import norm
+        kind = norm.RMS if inp.norm == "rms" else norm.LAYER
+        du64 = du.float().cpu().numpy().astype(np.float64)
+        want = norm.backward(inp.x, inp.gamma, inp.beta, kind, inp.eps, du64)
+        for a, r in ((dg1, want["dgamma"]), (db1, want["dbeta"]), (dx1, want["dx"])):
+            assert _rel(a, torch.from_numpy(np.ascontiguousarray(r))) <= TOL_FP32
 
 
 def test_noalloc_matches_workspace_entry_two_calls_in_a_row(b):
