@@ -3,18 +3,24 @@
 
 A step is one pass of the whole hot path over one batch of synthetic input: statistics and
 current-amax scale, forward store, incoming gradient to E5M2, du = dY W, then the six
-(use, policy) evaluations of the check -- gain use {U, R, N x K}, weight use {U, R, N x K}.
-Workload at every N: config 2, RMSNorm -> Linear at 390M-model shapes, replicated per GPU
-(the path has no exchange step, so N GPUs run N independent replicas: weak scaling).
+(use, policy) evaluations of the check -- gain use {U, R, N x K}, weight use {U, R, N x K} --
+i.e. one call of bsp_mc_check.  Workload at every N: config 5, RMSNorm -> Linear at the large-MLP
+shape (T = 16384, C = 4096, O = 11008, bf16, K = 16 draws), the largest single-GPU configuration,
+from the seeded host recipe; N GPUs run N independent replicas (the path has no exchange step:
+weak scaling).  Configs 2, 3 (both operand modes) and 4 (K = 1024) ride along as sub-objects.
 
 metric = per-use check elements/s: sum over use-evaluations of (saved-tensor elements x draws
 consumed) divided by the time of the step.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With --gpus N > 1 and no launcher environment, bench.py starts its N ranks itself (one process per
+GPU, rendezvous on 127.0.0.1); under torchrun it is one of the ranks.
 """
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -26,7 +32,10 @@ if ROOT not in sys.path:
 
 METRIC = "per_use_check_elements_per_s"
 UNIT = "elements/s"
-WORKLOAD = "cfg2_rmsnorm_linear_390m"
+WORKLOAD = "cfg5_rmsnorm_linear_large_mlp"
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_FP8_TFLOPS = 4500.0
 
 
 def check_elements(T, C, K):
@@ -96,6 +105,46 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+# ----------------------------------------------------------------------------------- replicas
+
+
+def free_port():
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_replicas(n, argv):
+    """Starts n copies of this script, one per GPU, with the launcher environment a rank expects
+    (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT); rank 0 prints the line.  Returns the
+    largest exit code."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + argv, env=env))
+    return max(p.wait() for p in procs)
+
+
+def replica_selftest(args):
+    """The timing protocol of the replicas alone, on CPU with gloo (no CUDA): every rank reports a
+    made-up step time, rank 0 prints the line built from the maximum.  Used by the CPU tests to cover
+    the launch path of --gpus N."""
+    import torch.distributed as dist
+    from paper_2609_39813_b200.harness import max_over_ranks, replica_throughput
+    world, rank = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo", init_method="env://")
+    ms = 10.0 * (rank + 1)
+    ms_max = max_over_ranks(ms, device="cpu")
+    if rank == 0:
+        print(json.dumps(dict(selftest="replicas", n_gpus=world, ms_max=ms_max,
+                              value=replica_throughput(1000, 1, world, ms_max))), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------------- oracle arm
 
 
@@ -147,25 +196,29 @@ def blas_threads():
 
 
 def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step is the check on a token slice of
+    config 5 (every column, every output row, all K = 16 draws of both uses)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2609_39813_b200 import workloads
-    inp = workloads.config2()
+    inp = workloads.config5()
+    K = inp.K
     # calibrate on a small slice, then size each step so the whole run stays within ~2.5 minutes
-    dt0, el0 = oracle_sample(inp, 64, 2, 2)
+    dt0, el0 = oracle_sample(inp, 32, K, K)
     budget = 150.0 / max(1, args.steps + args.warmup)
-    rows = int(max(64, min(inp.T, 64 * budget / max(dt0, 1e-3))))
-    rows = max(64, rows // 64 * 64)
+    rows = int(max(32, min(inp.T, 32 * budget / max(dt0, 1e-3))))
+    rows = max(32, rows // 32 * 32)
     for _ in range(args.warmup):
-        oracle_sample(inp, rows, 2, 2)
+        oracle_sample(inp, rows, K, K)
     total_t, total_el = 0.0, 0
     for _ in range(args.steps):
-        dt, el = oracle_sample(inp, rows, 2, 2)
+        dt, el = oracle_sample(inp, rows, K, K)
         total_t += dt
         total_el += el
     value = total_el / total_t
-    sample = "first %d of %d tokens, gain {U,R,N x2} + weight {U,R,N x2}, numpy float64" % (rows, inp.T)
+    sample = ("first %d of %d tokens, all %d columns and %d output rows, gain {U,R,N x%d} + weight {U,R,N x%d}, "
+              "numpy float64" % (rows, inp.T, inp.C, inp.O, K, K))
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * total_t / max(1, args.steps), higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
@@ -178,76 +231,100 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------- CUDA arm
 
 
-def attention_section(b, peaks, steps=3):
-    """Config 3 (causal attention backward, B=8 H=16 S=2048 d=64, K=32): the per-use check of the D
-    use, timed as a whole, and the two backward kernels timed alone.  Extra information beside the
-    headline number; inputs are drawn on the device (same distributions as the seeded recipe)."""
-    import torch
-    B, H, S, D, K = 8, 16, 2048, 64, 32
-    tensor_o = 2                                              # generator tensor id of the attention output store
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(1003)
-    n = B * H * S * D
-    q, k, v = (torch.randn(n, device="cuda", generator=gen).mul_(0.125).bfloat16() for _ in range(3))
-    dO = torch.randn(n, device="cuda", generator=gen).bfloat16()
-    d = b.AttnDesc()
-    d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, 0.125, b.BF16
-    d.q, d.k, d.v, d.dO = b.ptr(q), b.ptr(k), b.ptr(v), b.ptr(dO)
-    d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = b.E4M3, b.ROUND_STOCHASTIC, 1003, tensor_o, 7
-    ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+def timed(torch, stream, fn, reps=5, warm=2):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(reps):
+        fn()
+    c.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(c) / reps
+
+
+def norm_linear_check(b, torch, inp, steps=3, side=None):
+    """One normalisation -> linear configuration from the seeded host recipe: the whole check, timed."""
+    from paper_2609_39813_b200.harness import NormLinearGpu
+    g = NormLinearGpu(inp)
+    d = g.desc()
+    if side is not None:
+        d.side_stream = side.cuda_stream
+    ws = b.workspace(b.bsp_mc_check_workspace_bytes(d, inp.K))
     diag = b.new_diag()
     stream = torch.cuda.current_stream()
-    res = b.bsp_mc_check_attn(d, K, ws, diag)                 # warm-up
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(steps):
-        res = b.bsp_mc_check_attn(d, K, ws, diag)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
+    res = b.bsp_mc_check(d, inp.K, ws, diag)
+    ms = timed(torch, stream, lambda: b.bsp_mc_check(d, inp.K, ws, diag), reps=steps, warm=1)
+    return dict(workload=inp.name, T=inp.T, C=inp.C, O=inp.O, K=inp.K, ms_per_check=ms,
+                check_elements_per_s=check_elements(inp.T, inp.C, inp.K) / (ms * 1e-3),
+                verdicts=[int(r.verdict) for r in res if r.output_id != b.OUT_DBETA],
+                dbeta_verdicts=[int(r.verdict) for r in res if r.output_id == b.OUT_DBETA],
+                data="seeded host recipe", diag_status=b.read_diag(diag)["status"])
+
+
+def attention_section(b, peaks, steps=3):
+    """Config 3 (causal attention backward, B=8 H=16 S=2048 d=64, K=32) from the seeded host recipe:
+    the per-use check of the D use in both operand modes, timed as a whole, and its kernels alone."""
+    import torch
+    from paper_2609_39813_b200 import workloads
+    from paper_2609_39813_b200.harness import up
+    inp = workloads.config3()
+    B, H, S, D, K = inp.B, inp.H, inp.S, inp.D, inp.K
+    tensor_o = 2                                              # generator tensor id of the attention output store
+    n = B * H * S * D
+    q, k, v, dO = (up(a, "bf16").reshape(-1) for a in (inp.q, inp.k, inp.v, inp.dO))
+    stream = torch.cuda.current_stream()
+    diag = b.new_diag()
     elements = n * (1 + 1 + K)
-    # the backward kernels alone
+
+    def check(fp8_operands):
+        d = b.AttnDesc()
+        d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = B, H, S, D, 1, inp.softmax_scale, b.BF16
+        d.q, d.k, d.v, d.dO = b.ptr(q), b.ptr(k), b.ptr(v), b.ptr(dO)
+        d.store_fmt, d.forward_mode, d.seed, d.tensor_id, d.policy_mask = b.E4M3, b.ROUND_STOCHASTIC, inp.seed, tensor_o, 7
+        d.fp8_operands, d.p_scale, d.ds_scale = fp8_operands, 256.0, 1024.0
+        ws = b.workspace(b.bsp_mc_check_attn_workspace_bytes(d, K))
+        res = b.bsp_mc_check_attn(d, K, ws, diag)
+        ms = timed(torch, stream, lambda: b.bsp_mc_check_attn(d, K, ws, diag), reps=steps, warm=0)
+        return dict(ms_per_check=ms, check_elements_per_s=elements / (ms * 1e-3), verdicts=[int(r.verdict) for r in res],
+                    informational=[int(r.informational) for r in res])
+
+    mode_b = check(0)
+    mode_a = check(1)
+    torch.cuda.empty_cache()
+    # ---- the kernels alone
+    c = inp.softmax_scale
     o = torch.zeros(n, device="cuda"); lse = torch.zeros(B * H * S, device="cuda")
     dq, dk, dv = (torch.zeros(n, device="cuda") for _ in range(3))
     dterm = torch.zeros(B * H * S, device="cuda")
-    b.bsp_attn_fwd_stats(B, H, S, D, True, 0.125, q, k, v, o, lse, diag)
+    b.bsp_attn_fwd_stats(B, H, S, D, True, c, q, k, v, o, lse, diag)
     b.bsp_attn_dterm(B, H, S, D, dO, o, None, None, b.E4M3, b.READ_ORIGINAL, b.key(0, 2, 4), 0, 1, dterm)
-
-    def timed(fn, reps=5):
-        fn(); fn()
-        torch.cuda.synchronize()
-        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(reps):
-            fn()
-        c.record(stream)
-        torch.cuda.synchronize()
-        return a.elapsed_time(c) / reps
-
-    ms_dkv = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, None, dk, dv, diag))
-    ms_dq = timed(lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, 0.125, q, k, v, dO, lse, dterm, dq, None, None, diag))
+    ms_dkv = timed(torch, stream, lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, c, q, k, v, dO, lse, dterm, None, dk, dv, diag))
+    ms_dq = timed(torch, stream, lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, c, q, k, v, dO, lse, dterm, dq, None, None, diag))
     # the D pre-pass alone under its three reads (HBM-bound for U and R: dO read once, the copy of O
     # read once; the fresh read is bound by the generator: one word per element and draw)
     amax_o, scales_o = torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
     codes_o = torch.zeros(n, dtype=torch.uint8, device="cuda")
     b.bsp_amax(o, B * H, S * D, amax_o)
     b.bsp_scale_from_amax(amax_o, B * H, b.E4M3, scales_o)
-    b.bsp_round_grouped(o, B * H, S * D, b.E4M3, b.ROUND_STOCHASTIC, scales_o, b.key(1003, tensor_o, 0, 0), codes_o)
+    b.bsp_round_grouped(o, B * H, S * D, b.E4M3, b.ROUND_STOCHASTIC, scales_o, b.key(inp.seed, tensor_o, 0, 0), codes_o)
     d_draws = torch.zeros(K * B * H * S, device="cuda")
-    kd = b.key(1003, tensor_o, b.STREAM_ATTN_D, 0)
-    ms_du = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_ORIGINAL, kd, 0, 1, dterm))
-    ms_dr = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FORWARD, kd, 0, 1, dterm))
-    ms_dn = timed(lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FRESH, kd, 0, K, d_draws))
+    kd = b.key(inp.seed, tensor_o, b.STREAM_ATTN_D, 0)
+    ms_du = timed(torch, stream, lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_ORIGINAL, kd, 0, 1, dterm))
+    ms_dr = timed(torch, stream, lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FORWARD, kd, 0, 1, dterm))
+    ms_dn = timed(torch, stream, lambda: b.bsp_attn_dterm(B, H, S, D, dO, o, codes_o, scales_o, b.E4M3, b.READ_FRESH, kd, 0, K, d_draws))
     hbm = peaks["hbm_gbs"]
     dterm_rows = dict(
-        read_U=dict(us=ms_du * 1e3, algorithmic_mb=n * 6 / 1e6, gb_per_s=n * 6 / ms_du / 1e6, frac_of_hbm=n * 6 / ms_du / 1e6 / hbm),
-        read_R=dict(us=ms_dr * 1e3, algorithmic_mb=n * 3 / 1e6, gb_per_s=n * 3 / ms_dr / 1e6, frac_of_hbm=n * 3 / ms_dr / 1e6 / hbm),
+        read_U=dict(us=ms_du * 1e3, algorithmic_mb=n * 6 / 1e6, gb_per_s=n * 6 / ms_du / 1e6, frac_of_hbm=n * 6 / ms_du / 1e6 / hbm,
+                    frac_of_nominal_hbm=n * 6 / ms_du / 1e6 / NOMINAL_HBM_GBS),
+        read_R=dict(us=ms_dr * 1e3, algorithmic_mb=n * 3 / 1e6, gb_per_s=n * 3 / ms_dr / 1e6, frac_of_hbm=n * 3 / ms_dr / 1e6 / hbm,
+                    frac_of_nominal_hbm=n * 3 / ms_dr / 1e6 / NOMINAL_HBM_GBS),
         read_N=dict(us=ms_dn * 1e3, draws=K, g_element_draws_per_s=n * K / ms_dn / 1e6))
-    # the forward helper, and mode A of the config (FP8 operands: quantise Q, K, V, dO per (b,h) slice,
-    # then the whole backward with P and dS rounded onto the FP8 grids inside the kernels)
-    ms_fwd = timed(lambda: b.bsp_attn_fwd_stats(B, H, S, D, True, 0.125, q, k, v, o, lse, diag))
+    # the forward helper, and the FP8-operand mode of the backward
+    ms_fwd = timed(torch, stream, lambda: b.bsp_attn_fwd_stats(B, H, S, D, True, c, q, k, v, o, lse, diag))
     hatq, amq, scq = torch.zeros(n, dtype=torch.bfloat16, device="cuda"), torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
-    ms_quant = timed(lambda: b.bsp_attn_quantize(q, B * H, S * D, b.E4M3, hatq, amq, scq))
+    ms_quant = timed(torch, stream, lambda: b.bsp_attn_quantize(q, B * H, S * D, b.E4M3, hatq, amq, scq))
     ops = {}
     for nm, src, fmt in (("q", q, b.E4M3), ("k", k, b.E4M3), ("v", v, b.E4M3), ("dO", dO, b.E5M2)):
         xq, am, sc = torch.zeros(n, dtype=torch.bfloat16, device="cuda"), torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
@@ -255,43 +332,40 @@ def attention_section(b, peaks, steps=3):
         ops[nm] = (xq, sc)
     f8 = b.attn_fp8(ops["q"][1], ops["k"][1], ops["v"][1], ops["dO"][1], 256.0, 1024.0)
     o8, lse8 = torch.zeros(n, device="cuda"), torch.zeros(B * H * S, device="cuda")
-    b.bsp_attn_fwd_stats_fp8(B, H, S, D, True, 0.125, ops["q"][0], ops["k"][0], ops["v"][0], f8, o8, lse8, diag)
+    b.bsp_attn_fwd_stats(B, H, S, D, True, c, ops["q"][0], ops["k"][0], ops["v"][0], o8, lse8, diag, fp8=f8)
     d8 = torch.zeros(B * H * S, device="cuda")
-    ms_fp8 = timed(lambda: b.bsp_attn_bwd_fp8(B, H, S, D, True, 0.125, ops["q"][0], ops["k"][0], ops["v"][0], ops["dO"][0],
-                                              f8, lse8, o8, None, None, b.E4M3, b.READ_ORIGINAL, kd, dq, dk, dv, d8, diag))
+    ms_fp8 = timed(torch, stream, lambda: b.bsp_attn_bwd(B, H, S, D, True, c, 1, ops["q"][0], ops["k"][0], ops["v"][0], ops["dO"][0],
+                                                          lse8, o8, None, None, b.E4M3, b.READ_ORIGINAL, kd, dq, dk, dv, d8, diag, fp8=f8))
     prod = 2.0 * B * H * S * S * D / 2                         # one causal S x S x d product over all heads
     tf_dkv, tf_dq = 4 * prod / (ms_dkv * 1e-3) / 1e12, 3 * prod / (ms_dq * 1e-3) / 1e12
     peak = peaks["bf16_tflops"]
-    return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, ms_per_check=ms,
-                check_elements_per_s=elements / (ms * 1e-3), verdicts=[r.verdict for r in res],
+    bwd = (ms_dkv + ms_dq) * 1e-3
+    return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, data="seeded host recipe",
+                ms_per_check=mode_b["ms_per_check"], check_elements_per_s=mode_b["check_elements_per_s"],
+                verdicts=mode_b["verdicts"], bf16_operands=mode_b, fp8_operands=mode_a,
                 bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3, dterm=dterm_rows,
                 fwd_stats_us=ms_fwd * 1e3, quantize_one_tensor_us=ms_quant * 1e3,
                 bwd_fp8_operands_us=ms_fp8 * 1e3,   # D pre-pass + dK/dV + dQ kernels, FP8-operand mode
                 roofline=dict(bound="tensor", kernel="attn_kernel<dK/dV> + attn_kernel<dQ> (bf16 operands)",
-                              achieved=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12, peak=peak, unit="TFLOP/s",
-                              frac=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
-                              dkv_tflops=tf_dkv, dq_tflops=tf_dq,
+                              achieved=(4 + 3) * prod / bwd / 1e12, peak=peak, unit="TFLOP/s",
+                              frac=(4 + 3) * prod / bwd / 1e12 / peak, dkv_tflops=tf_dkv, dq_tflops=tf_dq,
                               # a backward needs 5 of those products; the two kernels form S and dP once each
-                              algorithmic_tflops=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12,
-                              algorithmic_frac=5 * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / peak,
-                              peak_nominal=2250.0, frac_of_nominal=(4 + 3) * prod / ((ms_dkv + ms_dq) * 1e-3) / 1e12 / 2250.0,
+                              algorithmic_tflops=5 * prod / bwd / 1e12, algorithmic_frac=5 * prod / bwd / 1e12 / peak,
+                              peak_nominal=NOMINAL_BF16_TFLOPS, frac_of_nominal=(4 + 3) * prod / bwd / 1e12 / NOMINAL_BF16_TFLOPS,
                               note="achieved counts the 7 causal products of 2*S*S*d/2 flop per head that the two "
                                    "kernels compute, algorithmic_* the 5 a backward needs; exp on the SFU co-bounds it"),
                 diag_status=b.read_diag(diag)["status"])
 
 
-def kernel_table(b, peaks):
-    """The streaming kernels one by one at the large-MLP shape (T=16384, C=4096, O=11008, bf16):
+def kernel_table(b, peaks, g):
+    """The streaming kernels one by one on config 5's own tensors (T=16384, C=4096, O=11008, bf16):
     microseconds per launch and algorithmic GB/s (bytes the method must move / time) against the
-    measured copy bandwidth.  Inputs are drawn on the device."""
+    measured copy bandwidth and the nominal 8 TB/s; then the K-draw kernels and the contractions."""
     import torch
-    T, C, O = 16384, 4096, 11008
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(5)
-    x = torch.randn(T * C, device="cuda", generator=gen).bfloat16()
-    dY = (torch.randn(T * O, device="cuda", generator=gen) * 0.1).bfloat16()
-    du = torch.randn(T * C, device="cuda", generator=gen).bfloat16()
-    gamma = torch.ones(C, device="cuda")
+    inp = g.inp
+    T, C, O = inp.T, inp.C, inp.O
+    x, dY, gamma = g.x, g.dY, g.gamma
+    du = torch.randn(T * C, device="cuda").bfloat16()       # any incoming gradient: only its bytes matter here
     rstd, mean = torch.zeros(T, device="cuda"), torch.zeros(T, device="cuda")
     amax, scale = torch.zeros(1, device="cuda"), torch.ones(1, device="cuda")
     codes = torch.zeros(T * C, dtype=torch.uint8, device="cuda")
@@ -304,26 +378,17 @@ def kernel_table(b, peaks):
     wss = b.workspace(b.bsp_mc_stats_workspace_bytes(O * C))
     stream = torch.cuda.current_stream()
     q = b.quant(b.E4M3, b.ROUND_STOCHASTIC, 1.0, scale)
-    qrn = b.quant(b.E5M2, b.ROUND_NEAREST, 100.0)
+    qrn = b.quant(b.E5M2, b.ROUND_NEAREST, 1.0, g.scale_dy)
     k = b.key(1, 1, 0)
     b.bsp_norm_stats(b.RMSNORM, x, T, C, gamma, None, 1e-6, rstd, mean, amax)
     b.bsp_scale_from_amax(amax, 1, b.E4M3, scale)
     rows = []
 
     def t(name, bound, fn, nbytes, reps=10):
-        for _ in range(3):
-            fn()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(reps):
-            fn()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) / reps * 1e3
+        us = timed(torch, stream, fn, reps=reps, warm=3) * 1e3
         gbs = nbytes / us / 1e3
         rows.append(dict(kernel=name, bound=bound, us=us, algorithmic_mb=nbytes / 1e6, gb_per_s=gbs,
-                         frac_of_hbm=gbs / peaks["hbm_gbs"], frac_of_nominal_hbm=gbs / 8000.0))
+                         frac_of_hbm=gbs / peaks["hbm_gbs"], frac_of_nominal_hbm=gbs / NOMINAL_HBM_GBS))
 
     t("amax(dY)", "hbm", lambda: b.bsp_amax(dY, 1, T * O, amax), T * O * 2)
     t("round dY -> E5M2 nearest", "hbm", lambda: b.bsp_round(dY, T * O, qrn, k, 0, dyc), T * O * 3)
@@ -336,9 +401,8 @@ def kernel_table(b, peaks):
     t("norm_bwd read N: dgamma, one fresh draw", "alu", lambda: b.bsp_norm_bwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, 2, codes, q, k, dg, None, None, ws), T * C * 4)
     t("mc_stats (45 M elements, fresh)", "hbm", lambda: b.bsp_mc_stats(ref, ref, S2, O * C, 16, 1, wss), O * C * 12)
     # ---- the K-draw kernels and the contractions at the same shape (K = 16 draws, as config 5)
-    Kd = 16
+    Kd = inp.K
     qf = b.quant(b.E4M3, b.ROUND_STOCHASTIC, 1.0, scale)
-    qdy = b.quant(b.E5M2, b.ROUND_NEAREST, 100.0)
     fresh_t = torch.zeros(Kd * C * T, dtype=torch.uint8, device="cuda")
     S1 = torch.zeros(O * C, device="cuda")
     diag = b.new_diag()
@@ -350,20 +414,13 @@ def kernel_table(b, peaks):
     wsw = b.workspace(max(b.bsp_linear_wgrad_workspace_bytes(T, O, C, b.READ_FORWARD), 256))
     compute = []
 
-    def tc(name, bound, fn, work, unit, peak, reps=5):
-        for _ in range(2):
-            fn()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(reps):
-            fn()
-        e1.record(stream)
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) / reps * 1e3
-        rate = work / (us * 1e-6)
-        compute.append(dict(kernel=name, bound=bound, us=us, achieved=rate / (1e9 if unit == "G element-draws/s" else 1e12),
-                            unit=unit, peak=peak, frac=(rate / (1e9 if unit == "G element-draws/s" else 1e12)) / peak))
+    def tc(name, bound, fn, work, unit, peak, nominal=None, reps=5):
+        us = timed(torch, stream, fn, reps=reps, warm=2) * 1e3
+        rate = work / (us * 1e-6) / (1e9 if unit == "G element-draws/s" else 1e12)
+        row = dict(kernel=name, bound=bound, us=us, achieved=rate, unit=unit, peak=peak, frac=rate / peak)
+        if nominal:
+            row["peak_nominal"], row["frac_of_nominal"] = nominal, rate / nominal
+        compute.append(row)
 
     # The ceiling of the generator-bound kernels is measured, not assumed: the rate at which the
     # generator alone produces its words (bsp_philox_fill: one Philox4x32-10 block per four words,
@@ -383,71 +440,28 @@ def kernel_table(b, peaks):
        lambda: b.bsp_norm_gain_mc(b.RMSNORM, x, T, C, gamma, None, rstd, mean, du, qf, b.key(1, 1, 1), 0, Kd, dg, g1, g2, wsg, diag),
        float(T) * C * Kd, "G element-draws/s", alu_peak)
     tc("weight gradient, read R (gemm_tc fp8)", "tensor",
-       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qdy, b.READ_FORWARD, codes_t, qf, T, dW, ws=wsw, diag=diag),
-       2.0 * T * O * C, "TFLOP/s", 2.0 * peaks["bf16_tflops"])
+       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qrn, b.READ_FORWARD, codes_t, qf, T, dW, ws=wsw, diag=diag),
+       2.0 * T * O * C, "TFLOP/s", 2.0 * peaks["bf16_tflops"], NOMINAL_FP8_TFLOPS)
     # the two BF16 contractions of the path: the weight gradient reading the original u, and the
     # incoming-gradient helper du = dY W (decoded dY codes; a bf16 W is read in place)
     u_bf16_t = torch.zeros(C * T, dtype=torch.bfloat16, device="cuda")
     b.bsp_norm_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, q, k, codes, codes_t, T, None, u_bf16_t)
     wsu = b.workspace(max(b.bsp_linear_wgrad_workspace_bytes(T, O, C, b.READ_ORIGINAL), 256))
     tc("weight gradient, read U (decode + gemm_tc bf16)", "tensor",
-       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qdy, b.READ_ORIGINAL, u_bf16_t, qf, T, dW, ws=wsu, diag=diag),
-       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"])
-    Wb = (torch.randn(O * C, device="cuda") / 64).to(torch.bfloat16)
+       lambda: b.bsp_linear_wgrad(T, O, C, dyc_t, qrn, b.READ_ORIGINAL, u_bf16_t, qf, T, dW, ws=wsu, diag=diag),
+       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"], NOMINAL_BF16_TFLOPS)
     du_out = torch.zeros(T * C, dtype=torch.bfloat16, device="cuda")
     wsd = b.workspace(b.bsp_linear_dgrad_workspace_bytes(T, O, C))
     tc("incoming gradient du = dY W (decode + gemm_tc bf16)", "tensor",
-       lambda: b.bsp_linear_dgrad(T, O, C, dyc, qdy, Wb, du_out, wsd, diag),
-       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"])
-    del u_bf16_t, Wb, du_out, wsu, wsd
+       lambda: b.bsp_linear_dgrad(T, O, C, dyc, qrn, g.W, du_out, wsd, diag),
+       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"], NOMINAL_BF16_TFLOPS)
+    del u_bf16_t, du_out, wsu, wsd
     tc("weight gradient, 16 fresh draws with sums (gemm_mc)", "tensor",
-       lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qdy, fresh_t, qf, T, Kd, ref, S1, S2, diag),
-       2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], reps=3)
-    # ---- the whole per-use check at this shape (K = 16, all six evaluations), as one call
-    del fresh_t, dyc, dyc_t, codes, codes_t, dx, du, dW, S1, S2, ref
-    torch.cuda.empty_cache()
-    Wc = (torch.randn(O * C, device="cuda", generator=gen) / 64).to(torch.bfloat16)
-    d = b.NormLinearDesc()
-    d.norm_kind, d.dtype = b.RMSNORM, b.BF16
-    d.T, d.C, d.O = T, C, O
-    d.x, d.gamma, d.beta, d.W, d.dY = b.ptr(x), b.ptr(gamma), None, b.ptr(Wc), b.ptr(dY)
-    d.eps = 1e-6
-    d.store_fmt, d.grad_fmt, d.forward_mode = b.E4M3, b.E5M2, b.ROUND_STOCHASTIC
-    d.seed, d.tensor_id, d.policy_mask = 1005, 1, 0x3F
-    wsc = b.workspace(b.bsp_mc_check_workspace_bytes(d, Kd))
-    for _ in range(2):
-        res = b.bsp_mc_check(d, Kd, wsc, diag)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(3):
-        res = b.bsp_mc_check(d, Kd, wsc, diag)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / 3
-    whole = dict(K=Kd, ms_per_check=ms, check_elements_per_s=check_elements(T, C, Kd) / (ms * 1e-3),
-                 verdicts=[int(r.verdict) for r in res])
-    # ---- config 4 as it is defined (LayerNorm, FP32 inputs, Student-t values, K = 1024): the whole check
-    del wsc, Wc, x, dY
-    torch.cuda.empty_cache()
-    from paper_2609_39813_b200 import workloads
-    from paper_2609_39813_b200.harness import NormLinearGpu
-    inp4 = workloads.config4()
-    g4 = NormLinearGpu(inp4)
-    d4 = g4.desc()
-    ws4 = b.workspace(b.bsp_mc_check_workspace_bytes(d4, inp4.K))
-    res4 = b.bsp_mc_check(d4, inp4.K, ws4, diag)
-    e0.record(stream)
-    for _ in range(2):
-        res4 = b.bsp_mc_check(d4, inp4.K, ws4, diag)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    ms4 = e0.elapsed_time(e1) / 2
-    cfg4 = dict(T=inp4.T, C=inp4.C, O=inp4.O, K=inp4.K, ms_per_check=ms4,
-                check_elements_per_s=check_elements(inp4.T, inp4.C, inp4.K) / (ms4 * 1e-3),
-                verdicts=[int(r.verdict) for r in res4])
-    return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), hbm_peak_gbs=peaks["hbm_gbs"], peak_source=peaks["source"],
-                kernels=rows, compute_kernels=compute, whole_check=whole, config4_check=cfg4,
-                diag_status=b.read_diag(diag)["status"])
+       lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qrn, fresh_t, qf, T, Kd, ref, S1, S2, diag),
+       2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], NOMINAL_FP8_TFLOPS, reps=3)
+    return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), data="seeded host recipe (config 5)",
+                hbm_peak_gbs=peaks["hbm_gbs"], hbm_nominal_gbs=NOMINAL_HBM_GBS, peak_source=peaks["source"],
+                kernels=rows, compute_kernels=compute, diag_status=b.read_diag(diag)["status"])
 
 
 def run_ours(args):
@@ -467,20 +481,25 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     b.lib()
+    peaks = read_peaks()
 
-    if args.kernel_table:
-        if rank == 0:
-            print(json.dumps(dict(kernel_table=kernel_table(b, read_peaks()))), flush=True)
-        return
     if args.attention_only:
         if rank == 0:
-            print(json.dumps(dict(attention=attention_section(b, read_peaks(), steps=args.attention_steps))), flush=True)
+            print(json.dumps(dict(attention=attention_section(b, peaks, steps=args.attention_steps))), flush=True)
         return
 
-    inp = workloads.config2()
+    inp = workloads.config5()
     T, C, O, K = inp.T, inp.C, inp.O, inp.K
     g = NormLinearGpu(inp)
+    if args.kernel_table:
+        if rank == 0:
+            print(json.dumps(dict(kernel_table=kernel_table(b, peaks, g))), flush=True)
+        return
+    # the preparation NormLinearGpu did (codes, statistics) is for the isolated kernel timing further
+    # down; the step itself starts from x, gamma, W, dY
+    side = torch.cuda.Stream()
     desc = g.desc()
+    desc.side_stream = side.cuda_stream
     ws = b.workspace(b.bsp_mc_check_workspace_bytes(desc, K))
     diag = b.new_diag()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB of L2
@@ -494,16 +513,17 @@ def run_ours(args):
     def step():
         return b.bsp_mc_check(desc, K, ws, diag)
 
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         res = step()
-    verdicts = [r.verdict for r in res]
+    verdicts = [int(r.verdict) for r in res if r.output_id != b.OUT_DBETA]
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
     barrier()
-    n0 = b.bsp_launch_count()
+    n0, d0 = b.bsp_launch_count(), b.bsp_d2h_byte_count()
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     for i in range(args.steps):
@@ -513,6 +533,7 @@ def run_ours(args):
         ends[i].record(stream)
     barrier()
     launches = b.bsp_launch_count() - n0
+    d2h = (b.bsp_d2h_byte_count() - d0) // max(1, args.steps)
     clocks = sampler.stop() if rank == 0 else None
     ms = sum(s.elapsed_time(e) for s, e in zip(starts, ends))
     ms_total = max_over_ranks(ms, device="cuda")
@@ -523,21 +544,21 @@ def run_ours(args):
     host = dict(x=g.x.cpu().pin_memory(), gamma=g.gamma.cpu().pin_memory(), W=g.W.cpu().pin_memory(),
                 dY=g.dY.cpu().pin_memory())
     h2d = sum(v.numel() * v.element_size() for v in host.values())
-    d2h = sum(min(592, (n + 255) // 256) * 64 for n in (C, C, C, O * C, O * C, O * C))
-    e2e_steps = max(3, min(args.steps, 20))
-    # two sets of device buffers: the inputs of step i + 1 cross PCIe on a copy stream while step i
-    # computes (every step's copy is inside the timed region; a step starts only when its own inputs
-    # have landed, and bsp_mc_check returns with the results on the host)
-    g2 = NormLinearGpu(inp)
-    sets = [(g, desc), (g2, g2.desc())]
+    e2e_steps = max(3, min(args.steps, 10))
+    # two sets of device input buffers: the inputs of step i + 1 cross PCIe on a copy stream while
+    # step i computes (every step's copy is inside the timed region; a step starts only when its own
+    # inputs have landed, and bsp_mc_check returns with the results on the host)
+    alt = dict(x=torch.empty_like(g.x), gamma=torch.empty_like(g.gamma), W=torch.empty_like(g.W), dY=torch.empty_like(g.dY))
+    desc2 = g.desc()
+    desc2.side_stream = side.cuda_stream
+    desc2.x, desc2.gamma, desc2.W, desc2.dY = b.ptr(alt["x"]), b.ptr(alt["gamma"]), b.ptr(alt["W"]), b.ptr(alt["dY"])
+    sets = [(dict(x=g.x, gamma=g.gamma, W=g.W, dY=g.dY), desc), (alt, desc2)]
     copy_stream = torch.cuda.Stream()
 
-    def upload(gs):
+    def upload(bufs):
         with torch.cuda.stream(copy_stream):
-            gs.x.copy_(host["x"], non_blocking=True)
-            gs.gamma.copy_(host["gamma"], non_blocking=True)
-            gs.W.copy_(host["W"], non_blocking=True)
-            gs.dY.copy_(host["dY"], non_blocking=True)
+            for name in ("x", "gamma", "W", "dY"):
+                bufs[name].copy_(host[name], non_blocking=True)
             ev = torch.cuda.Event()
             ev.record(copy_stream)
         return ev
@@ -548,7 +569,7 @@ def run_ours(args):
     copy_stream.wait_event(e0)
     landed = upload(sets[0][0])
     for i in range(e2e_steps):
-        gs, ds = sets[i & 1]
+        bufs, ds = sets[i & 1]
         stream.wait_event(landed)
         if i + 1 < e2e_steps:
             landed = upload(sets[(i + 1) & 1][0])
@@ -556,19 +577,20 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_value = replica_throughput(elements, e2e_steps, world, max_over_ranks(e0.elapsed_time(e1), device="cuda"))
+    del alt, host
 
     # ---- roofline of the dominant kernel: the FP8 weight-gradient contraction with the fused
     # shifted-sum epilogue, timed alone with CUDA events on the launching stream
-    peaks = read_peaks()
-    fresh_t = torch.zeros(K * C * g.ld_t, dtype=torch.uint8, device="cuda")
+    lay = b.bsp_mc_check_layout(desc, K)
     qf = b.quant(inp.store_fmt, b.ROUND_STOCHASTIC, 1.0, g.scale)
+    fresh_t = torch.zeros(K * C * g.ld_t, dtype=torch.uint8, device="cuda")
     b.bsp_norm_fwd_draws(g.kind, g.x, T, C, g.gamma, g.beta, g.rstd, g.mean, qf,
                          b.key(inp.seed, g.tensor_id, b.STREAM_WGRAD, 0), 0, K, fresh_t, g.ld_t)
-    ref = torch.zeros(O * C, device="cuda")
+    ref = b.ws_view(ws, lay.dW_ref, O * C)
     S1 = torch.zeros(O * C, device="cuda")
     S2 = torch.zeros(O * C, device="cuda")
-    reps = 8
-    for _ in range(3):
+    reps = 5
+    for _ in range(2):
         b.bsp_linear_wgrad_mc(T, O, C, g.dy_codes_t, g.q_dy, fresh_t, qf, g.ld_t, K, ref, S1, S2, diag)
     torch.cuda.synchronize()
     r0 = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]
@@ -583,17 +605,19 @@ def run_ours(args):
     flops = 2.0 * T * O * C * K               # one launch contracts all K draws
     achieved = flops / (gemm_ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16_tflops"]        # FP8 dense = 2 x the measured BF16 burst figure
-    # DRAM bytes of one launch of this kernel at this shape, from one ncu capture of this command
-    # (dram__bytes_read.sum 604.7 MB + dram__bytes_write.sum 23.1 MB; profiles/gemm_mc_kernel_cfg2.md).
-    # The launch's operands are K x T x C = 268 MB of fresh codes, read once per column of output
-    # tiles that does not find them in L2, plus 16.8 MB of dY codes and 3 x 16.8 MB of sums.
-    traffic = 627.8e6 if (T, C, O, K) == (4096, 1024, 4096, 64) else None
+    # DRAM bytes of one launch of this kernel at this shape: dram__bytes_read.sum + dram__bytes_write.sum
+    # of one ncu capture of this command (profiles/gemm_mc_kernel_cfg5.md); null for any other shape
+    traffic = GEMM_MC_TRAFFIC.get((T, C, O, K))
     roofline = dict(bound="tensor", kernel="gemm_mc_kernel (FP8 weight gradient over K draws, TMEM-resident sums)",
                     achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=traffic,
                     traffic_unit="bytes per launch (ncu dram read + write, one capture)",
+                    algorithmic_bytes=float(K * C * g.ld_t + O * g.ld_t + 5 * 4 * O * C),
                     us_per_launch=gemm_ms * 1e3, draws_per_launch=K,
+                    share_of_step=gemm_ms / (ms_total / args.steps),
                     peak_source="2 x bf16_tflops (%s)" % peaks["source"],
-                    peak_nominal=4500.0, frac_of_nominal=achieved / 4500.0)
+                    peak_sustained=2.0 * peaks["bf16_tflops_sustained"],
+                    frac_of_sustained=achieved / (2.0 * peaks["bf16_tflops_sustained"]),
+                    peak_nominal=NOMINAL_FP8_TFLOPS, frac_of_nominal=achieved / NOMINAL_FP8_TFLOPS)
     # Context beside that denominator: what the vendor library's own FP8 contraction reaches on this
     # GPU in this run (8192^3, E4M3 x E4M3, a short burst), measured the way the BF16 figure was.
     lib_fp8 = library_fp8_tflops() if rank == 0 else None
@@ -609,24 +633,30 @@ def run_ours(args):
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
-        # a bounded sample of the same workload (all tokens, eight fresh draws per use instead of K):
-        # ten to twenty seconds of host work
-        dt, el = oracle_sample(inp, T, 8, 8)
+        # a bounded sample of the same workload: a token slice (every column, every output row, all K
+        # draws of both uses), ten to thirty seconds of host work
+        rows = 384
+        dt, el = oracle_sample(inp, rows, K, K)
         cpu_baseline = dict(value=el / dt, unit=UNIT, cores=blas_threads(), kind="oracle",
-                            sample="all %d tokens, gain {U,R,N x8} + weight {U,R,N x8}, %.1f s" % (T, dt))
+                            sample="first %d of %d tokens, all columns and output rows, gain {U,R,N x%d} + weight "
+                                   "{U,R,N x%d}, %.1f s" % (rows, T, K, K, dt))
 
-    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=warmup,
                 ms_per_step=ms_total / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f8e4m3/f8e5m2 operands, f32 accumulate", data="synthetic",
                 config=dict(workload=WORKLOAD, T=T, C=C, O=O, K=K, policies="gain{U,R,N} x weight{U,R,N}",
-                            l2="flushed between timed steps (256 MiB write, outside the timed spans)",
-                            replicas=world),
+                            inputs="seeded host recipe (numpy PCG64, data seed 1005)",
+                            l2="inputs larger than L2, and L2 flushed between timed steps (256 MiB write, outside "
+                               "the timed spans)", replicas=world),
                 clocks=clocks,
-                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
+                e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=int(d2h), steps=e2e_steps),
                 gpu_launches=int(launches), roofline=roofline, cpu_baseline=cpu_baseline,
                 verdicts=verdicts, diag_status=dstat["status"])
-    if not args.no_attention and world == 1:
-        del ws, flush, fresh_t
+    if not args.no_extras and world == 1:
+        del ws, flush, fresh_t, S1, S2, g
+        torch.cuda.empty_cache()
+        line["config2"] = norm_linear_check(b, torch, workloads.config2(), steps=10, side=side)
+        line["config4"] = norm_linear_check(b, torch, workloads.config4(), steps=2, side=side)
         torch.cuda.empty_cache()
         line["attention"] = attention_section(b, peaks, steps=args.attention_steps)
     print(json.dumps(line), flush=True)
@@ -634,22 +664,32 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# DRAM traffic of one gemm_mc_kernel launch by (T, C, O, K), bytes, from ncu (see profiles/)
+GEMM_MC_TRAFFIC = {}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-attention", action="store_true", help="skip the config-3 attention section")
+    ap.add_argument("--no-extras", action="store_true", help="skip the sub-objects for configs 2, 3 and 4")
     ap.add_argument("--attention-only", action="store_true", help="run only the config-3 attention section")
     ap.add_argument("--attention-steps", type=int, default=3)
     ap.add_argument("--kernel-table", action="store_true",
-                    help="time the streaming kernels one by one at the large-MLP shape and print their GB/s")
+                    help="time the kernels one by one on config 5's tensors and print their GB/s and TFLOP/s")
+    ap.add_argument("--selftest-replicas", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
-        if args.steps == 100 and args.warmup == 5:
-            args.steps, args.warmup = 5, 1
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # not under a launcher: start the ranks here
+        sys.exit(spawn_replicas(args.gpus, sys.argv[1:]))
+    if args.selftest_replicas:
+        replica_selftest(args)
+    elif args.impl == "reference":
+        if args.steps == 30 and args.warmup == 3:
+            args.steps, args.warmup = 3, 1
         run_reference(args)
     else:
         run_ours(args)

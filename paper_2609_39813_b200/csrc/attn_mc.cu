@@ -320,7 +320,8 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
         // ---- the B operand: row r of the streamed Q tile times this row's factor of each draw, written
         // at the same (swizzled) place of the draw's tile.  Thread (r, h) takes the four 16-byte chunks
-        // 4h .. 4h+3 of its row.
+        // whose logical index is 4h .. 4h+3; chunk c of row r sits at position c ^ (r & 7), so the lanes
+        // of a warp (consecutive rows) spread over all banks.
         if (store_pending) {
           if (warp == 2 && lane == 0) tma_store_wait_read();
           named_bar_sync(2, 256);
@@ -333,11 +334,11 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           uint32_t f2[kDkND];
 #pragma unroll
           for (int d = 0; d < kDkND; ++d) f2[d] = pack_bf16x2(fk[d], fk[d]);
-          const uint32_t row_off = (uint32_t)r * 128u + (uint32_t)h * 64u;
+          const uint32_t row_off = (uint32_t)r * 128u;
 #pragma unroll
           for (int cch = 0; cch < 4; ++cch) {
             uint32_t a0, a1, a2, a3;
-            const uint32_t off = row_off + (uint32_t)cch * 16u;
+            const uint32_t off = row_off + ((uint32_t)((4 * h + cch) ^ (r & 7)) << 4);
             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(q0 + s * kAtTile + off));
 #pragma unroll
             for (int d = 0; d < kDkND; ++d)

@@ -39,12 +39,14 @@ FMT_E5M2 = 1
 
 
 def to_bf16_grid(a: np.ndarray) -> np.ndarray:
-    """Round float32 values to the nearest bf16 value (ties to even); result stays float32."""
-    a = np.ascontiguousarray(a, dtype=np.float32)
-    b = a.view(np.uint32).astype(np.uint64)
-    lsb = (b >> np.uint64(16)) & np.uint64(1)
-    b = (b + np.uint64(0x7FFF) + lsb) & np.uint64(0xFFFF0000)
-    return b.astype(np.uint32).view(np.float32).reshape(a.shape)
+    """Round finite float32 values to the nearest bf16 value (ties to even); result stays float32."""
+    out = np.array(a, dtype=np.float32, order="C", copy=True)
+    b = out.view(np.uint32)
+    lsb = (b >> np.uint32(16)) & np.uint32(1)
+    lsb += np.uint32(0x7FFF)
+    b += lsb                               # finite values: no carry out of the exponent field's top
+    b &= np.uint32(0xFFFF0000)
+    return out
 
 
 def bf16_bits(a_on_grid: np.ndarray) -> np.ndarray:

@@ -39,3 +39,21 @@ def test_single_process_is_identity():
     from paper_2609_39813_b200 import harness
     assert harness.max_over_ranks(3.5) == 3.5
     assert harness.replica_throughput(10, 2, 1, 1000.0) == 20.0
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher environment starts two ranks itself (one process
+    per GPU on a GPU machine; here the timing protocol alone, on gloo) and rank 0 prints one line."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--selftest-replicas"],
+                         env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms_max"] == 20.0           # the slower of the two ranks
+    assert line["value"] == pytest.approx(2 * 1000 / 0.020)
