@@ -324,3 +324,75 @@ def test_attention_operand_rounding_option():
         rel = np.linalg.norm(rounded[n] - exact[n]) / np.linalg.norm(exact[n])
         assert 1e-5 < rel < 4e-3, (n, rel)
     assert np.array_equal(rounded["D"], exact["D"])
+
+
+def test_bf16_round_against_an_independent_cast():
+    """linear.bf16_round (the operand rounding of the U read) against ml_dtypes' bfloat16 cast:
+    random values over many binades, every tie between neighbouring bf16 values in a binade, zeros,
+    subnormals of float32, and values that round up into the next binade."""
+    ml_dtypes = pytest.importorskip("ml_dtypes")
+    rng = np.random.default_rng(12)
+    a = (rng.standard_normal(200000) * np.exp(rng.uniform(-60, 60, 200000))).astype(np.float32)
+    # exact ties: a bf16 value plus half its spacing (representable in float32), both parities
+    base = np.arange(0x3F80, 0x4000, dtype=np.uint32) << np.uint32(16)
+    ties = (base | np.uint32(0x8000)).view(np.float32)
+    special = np.array([0.0, -0.0, 1e-40, -1e-45, 1.0, -1.0, np.float32(1.99609375), np.float32(1.998046875),
+                        3.3e38, -3.3e38], dtype=np.float32)
+    for v in (a, ties, -ties, special):
+        want = v.astype(ml_dtypes.bfloat16).astype(np.float32)
+        got = linear.bf16_round(v.astype(np.float64)).astype(np.float32)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # float64 inputs are first brought to float32 (the operands are float32 tensors)
+    assert linear.bf16_round(np.float64(1.0) + 2.0 ** -30) == 1.0
+
+
+def test_fresh_read_variance_closed_form_weight_use_and_d(cfg1):
+    """The closed-form variances of the other two uses under a fresh read: weight use
+    Var dW[o, c] = sum_t dY[t, o]^2 sigma^2[t, c]; attention's D: Var D[i] = sum_d dO[i, d]^2 sigma^2[i, d],
+    with sigma^2 = (v - lo)(hi - v) / scale^2 the variance of one stochastic rounding.  Sample variances
+    over K draws match within sampling error, and the means are the values read from the unrounded
+    tensor."""
+    inp, prep = cfg1
+    K = 192
+    res = check.wgrad_use(prep, check.N, K, inp.seed)
+    lo, hi, _ = fp8.neighbours(prep["v32"], fp8.E4M3)
+    a = np.abs(prep["v32"].astype(np.float64))
+    var_el = (a - lo) * (hi - a) * float(prep["inv_scale"]) ** 2
+    dy = prep["dy"]["value"]
+    var_cf = (dy * dy).T @ var_el
+    ratio = (res["m2"] / (K - 1)) / var_cf
+    assert abs(np.mean(ratio) - 1) < 4 * np.sqrt(2.0 / (K - 1)) / np.sqrt(ratio.size)
+    assert np.all(np.abs(ratio - 1) < 7 * np.sqrt(2.0 / (K - 1)))
+    # the mean tends to the value of the chain's own FP32 u (the original), not to the reference
+    g_u = linear.wgrad(dy, prep["u32"].astype(np.float64))
+    z = (res["mean"] - g_u) / np.sqrt(var_cf / K)
+    assert np.max(np.abs(z)) < 5.5 and abs(np.mean(z * z) - 1) < 0.1
+    # ---- attention's D use
+    ai = workloads.config3(B=1, H=1, S=96, D=64, K=K, seed=5)
+    q, k, v, dO = ai.q[0, 0], ai.k[0, 0], ai.v[0, 0], ai.dO[0, 0]
+    ap = check.prepare_attention_slice(q, k, v, dO, ai.softmax_scale, ai.seed, 0, True)
+    rd = check.attention_d_use(q, k, v, dO, ai.softmax_scale, ap, check.N, K, ai.seed, outputs=("D",))["D"]
+    lo, hi, _ = fp8.neighbours(ap["v32"], fp8.E4M3)
+    a = np.abs(ap["v32"].astype(np.float64))
+    var_o = (a - lo) * (hi - a) * float(ap["inv_scale"]) ** 2
+    var_d = np.sum(dO.astype(np.float64) ** 2 * var_o, axis=1)
+    ratio = (rd["m2"] / (K - 1)) / var_d
+    assert abs(np.mean(ratio) - 1) < 4 * np.sqrt(2.0 / (K - 1)) / np.sqrt(ratio.size)
+    assert np.all(np.abs(ratio - 1) < 6 * np.sqrt(2.0 / (K - 1)))
+    z = (rd["mean"] - rd["ref"]) / np.sqrt(var_d / K)
+    assert np.max(np.abs(z)) < 5 and abs(np.mean(z * z) - 1) < 0.5
+
+
+def test_elements_without_variance_are_judged_as_deterministic_reads():
+    """Where every draw of an element gave the same value, z is 0 if the error is within the
+    deterministic tolerance of the reference and infinite otherwise; the other elements keep z = err/se."""
+    K = 8
+    ref = np.array([1.0, 1.0, 1.0, 0.0, 2.0])
+    mean = np.array([1.0 + 5e-8, 1.0 + 1e-3, 1.2, 0.0, 2.0])
+    m2 = np.array([0.0, 0.0, 0.7, 0.0, 0.0])
+    st = mc.statistics(mean, m2, K, ref, True)
+    assert np.isinf(st.max_abs_z) and np.isinf(st.Qprime) and st.verdict == mc.FAILS
+    st = mc.statistics(np.array([1.0 + 5e-8, 1.2, 0.0]), np.array([0.0, 0.7, 0.0]), K, np.array([1.0, 1.0, 0.0]), True)
+    se = np.sqrt(0.7 / (K - 1) / K)
+    assert st.max_abs_z == pytest.approx(0.2 / se) and st.mean_z == pytest.approx(0.2 / se / 3)
+    assert st.frac_abs_z_gt3 == 0.0 if 0.2 / se <= 3 else st.frac_abs_z_gt3 == pytest.approx(1 / 3)
