@@ -61,7 +61,10 @@ typedef enum {
 typedef enum { BSP_E4M3 = 0, BSP_E5M2 = 1 } bsp_format_t;
 typedef enum { BSP_ROUND_NEAREST = 0, BSP_ROUND_STOCHASTIC = 1 } bsp_round_mode_t;
 /* What a backward use reads (Section "One tensor, two uses"; Appendix table "Store policies"). */
-typedef enum { BSP_READ_ORIGINAL = 0 /* U */, BSP_READ_FORWARD = 1 /* R */, BSP_READ_FRESH = 2 /* N */ } bsp_policy_t;
+typedef enum { BSP_READ_ORIGINAL = 0 /* U */, BSP_READ_FORWARD = 1 /* R */, BSP_READ_FRESH = 2 /* N */,
+               /* the forward's rounding plus the error of a new one, u_q + (u_f - u): the weight-use
+                  read of the table's last policy, U/R+eps (b-bit store only) */
+               BSP_READ_FORWARD_PLUS_FRESH_ERROR = 3 } bsp_policy_t;
 typedef enum { BSP_F32 = 0, BSP_BF16 = 1 } bsp_dtype_t;
 typedef enum { BSP_RMSNORM = 0, BSP_LAYERNORM = 1 } bsp_norm_t;
 typedef enum { BSP_HOLDS = 0, BSP_FAILS = 1, BSP_UNDECIDED = 2 } bsp_verdict_t;
@@ -528,6 +531,67 @@ size_t bsp_mc_check_attn_workspace_bytes(const bsp_attn_desc_t* op, int K);
 int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, const bsp_verdict_rule_t* rule,
                       bsp_use_result_t* results, int* n_results, void* ws, size_t ws_bytes,
                       bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * The paper's own store (Appendix "The normalization store"; table "Store policies"): for each
+ * token a b-bit uniform grid of step s = max_j |u_j| / (2^(b-1) - 1), u_q = s floor(u / s + xi)
+ * with an independent uniform xi per entry, so that u_q averages to u without clipping; the new
+ * rounding u_f uses a separate generator stream.  Reads: gain use z | u_q / gamma | u_f / gamma;
+ * weight use u | u_q | u_f | u_q + (u_f - u).  Reference: gain use z, weight use u_q.
+ * Arithmetic: u is the FP32 chain value of the normalisation; s = fl32(amax / M), M = 2^(b-1) - 1
+ * (1 for an all-zero token); t = fl32(u / s); n = floor(t) + [W < P] with W the element's generator
+ * word and P = min(floor(fl32(t - floor(t)) 2^32), 2^32 - 1) -- the same law as floor(t + xi).
+ * Codes are int8 (b = 2 .. 7; the paper ran 6 and 5), a code stands for s * code.
+ * ------------------------------------------------------------------------------------------ */
+
+/* codes[T*C], steps[T] from the saved statistics (rstd, mean as for bsp_norm_fwd) under `key`
+ * (stream BSP_STREAM_FORWARD: the forward's store). */
+int bsp_store_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                  const float* beta, const float* rstd, const float* mean, int bits, bsp_key_t key,
+                  int8_t* codes, float* steps, void* stream);
+
+/* The copy of u a use reads: read = BSP_READ_ORIGINAL (u), BSP_READ_FORWARD (s * code),
+ * BSP_READ_FRESH (a new rounding under `key`) or BSP_READ_FORWARD_PLUS_FRESH_ERROR.  Outputs, each
+ * may be NULL: copy_f32[T*C], and copy_split_t[C][2*ld_t] bf16, the operand of bsp_store_wgrad:
+ * the copy split into two bf16 terms hi + lo (16 significant bits), token-minor, hi in columns
+ * [0, ld_t), lo in [ld_t, 2 ld_t); ld_t >= T, a multiple of 16, padding zeroed. */
+int bsp_store_read(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
+                   const float* beta, const float* rstd, const float* mean, const int8_t* codes,
+                   const float* steps, int read, bsp_key_t key, float* copy_f32, void* copy_split_t,
+                   int64_t ld_t, void* stream);
+
+/* dW[O, C] = dY^T X for a copy X given as the split operand of bsp_store_read: BF16 tensor cores,
+ * dW = [dY | dY] [X_hi | X_lo]^T with dY's codes decoded to bf16 (exact), FP32 accumulation.  The
+ * per-token step is part of X, so no operand is rounded below 16 bits. */
+size_t bsp_store_wgrad_workspace_bytes(int64_t T, int64_t O);
+int bsp_store_wgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes_t, bsp_quant_t q_dy,
+                    const void* copy_split_t, int64_t ld_t, float* dW, void* ws, size_t ws_bytes,
+                    bsp_diag_t* diag, void* stream);
+
+/* The per-use check with the b-bit store in place of the FP8 store: as bsp_mc_check, with
+ * policy_mask bits 0..2 = gain use U, R, N and bits 3..6 = weight use U, R, N, U/R+eps (K >= 4 draws
+ * for each fresh read).  results: HOST array of at least 7 entries in that order (dgamma, dW). */
+typedef struct {
+  int32_t norm_kind;         /* bsp_norm_t  */
+  int32_t dtype;             /* bsp_dtype_t of x, W, dY (and of du) */
+  int64_t T, C, O;
+  const void* x;             /* [T, C] */
+  const float* gamma;        /* [C]    */
+  const float* beta;         /* [C] or NULL */
+  const void* W;             /* [O, C] */
+  const void* dY;            /* [T, O] */
+  float eps;
+  int32_t bits;              /* width of the store: 2 .. 7 */
+  int32_t grad_fmt;          /* bsp_format_t of dY (E5M2) */
+  uint64_t seed;
+  uint32_t tensor_id;
+  uint32_t policy_mask;
+} bsp_store_desc_t;
+
+size_t bsp_mc_check_store_workspace_bytes(const bsp_store_desc_t* op, int K);
+int bsp_mc_check_store(const bsp_store_desc_t* op, int K, const bsp_verdict_rule_t* rule,
+                       bsp_use_result_t* results, int* n_results, void* ws, size_t ws_bytes,
+                       bsp_diag_t* diag, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait a kernel of

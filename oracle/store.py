@@ -32,8 +32,8 @@ READ_U, READ_R, READ_N, READ_R_EPS = 0, 1, 2, 3
 
 def levels(bits: int) -> int:
     """M = 2^(b-1) - 1: the grid has the codes -M .. M."""
-    if not 2 <= bits <= 8:
-        raise ValueError("store width must be 2..8 bits")
+    if not 2 <= bits <= 7:
+        raise ValueError("store width must be 2..7 bits")
     return (1 << (bits - 1)) - 1
 
 
@@ -46,12 +46,13 @@ def steps(u32, bits: int) -> np.ndarray:
 
 
 def position(u32, s32):
-    """t = fl32(u / s), n0 = floor(t), f = fl32(t - n0), P = floor(f 2^32) (uint64 < 2^32)."""
+    """t = fl32(u / s), n0 = floor(t), f = fl32(t - n0), P = min(floor(f 2^32), 2^32 - 1): a 32-bit
+    threshold (f can round to 1 when t is a hair below an integer; P then saturates)."""
     u32 = np.asarray(u32, dtype=np.float32)
     t = (u32 / np.asarray(s32, dtype=np.float32)[:, None]).astype(np.float32)
     n0 = np.floor(t).astype(np.float32)
     f = (t - n0).astype(np.float32)
-    P = np.floor(f.astype(np.float64) * 4294967296.0).astype(np.uint64)
+    P = np.minimum(np.floor(f.astype(np.float64) * 4294967296.0), 4294967295.0).astype(np.uint64)
     return t, n0.astype(np.int64), f, P
 
 

@@ -16,7 +16,7 @@ OK, ERR_ARG, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_NONFINITE, ERR_TIMEO
 NORM_BWD_NOALLOC_CAPACITY_BYTES = 20 << 20
 E4M3, E5M2 = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
-READ_ORIGINAL, READ_FORWARD, READ_FRESH = 0, 1, 2
+READ_ORIGINAL, READ_FORWARD, READ_FRESH, READ_FORWARD_PLUS_FRESH_ERROR = 0, 1, 2, 3
 F32, BF16 = 0, 1
 RMSNORM, LAYERNORM = 0, 1
 HOLDS, FAILS, UNDECIDED = 0, 1, 2
@@ -75,6 +75,13 @@ class AttnDesc(C.Structure):
                 ("v", C.c_void_p), ("dO", C.c_void_p), ("store_fmt", C.c_int32), ("forward_mode", C.c_int32),
                 ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32),
                 ("fp8_operands", C.c_int32), ("p_scale", C.c_float), ("ds_scale", C.c_float)]
+
+
+class StoreDesc(C.Structure):
+    _fields_ = [("norm_kind", C.c_int32), ("dtype", C.c_int32), ("T", C.c_int64), ("C", C.c_int64),
+                ("O", C.c_int64), ("x", C.c_void_p), ("gamma", C.c_void_p), ("beta", C.c_void_p),
+                ("W", C.c_void_p), ("dY", C.c_void_p), ("eps", C.c_float), ("bits", C.c_int32),
+                ("grad_fmt", C.c_int32), ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
 
 
 class AttnFp8(C.Structure):
@@ -139,6 +146,13 @@ _SIGNATURES = {
     "bsp_mc_check": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(VerdictRule), C.POINTER(UseResult), C.POINTER(_I),
                           _P, _SZ, _P, _P]),
     "bsp_selftest_bounded_wait": (_I, [_U64, _P, _P]),
+    "bsp_store_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _I, Key, _P, _P, _P]),
+    "bsp_store_read": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _P, _I, Key, _P, _P, _I64, _P]),
+    "bsp_store_wgrad_workspace_bytes": (_SZ, [_I64, _I64]),
+    "bsp_store_wgrad": (_I, [_I64, _I64, _I64, _P, Quant, _P, _I64, _P, _P, _SZ, _P, _P]),
+    "bsp_mc_check_store_workspace_bytes": (_SZ, [C.POINTER(StoreDesc), _I]),
+    "bsp_mc_check_store": (_I, [C.POINTER(StoreDesc), _I, C.POINTER(VerdictRule), C.POINTER(UseResult), C.POINTER(_I),
+                                _P, _SZ, _P, _P]),
 }
 
 
@@ -467,6 +481,40 @@ def bsp_mc_check(desc: NormLinearDesc, K, ws, diag=None, stream=None, rule=None)
     n = C.c_int(0)
     check(lib().bsp_mc_check(C.byref(desc), K, _ruleref(rule), res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
                              _st(stream)), "bsp_mc_check")
+    return [res[i] for i in range(n.value)]
+
+
+def bsp_store_fwd(kind, x, T, Cc, gamma, beta, rstd, mean, bits, k: Key, codes, steps, stream=None):
+    check(lib().bsp_store_fwd(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean), bits, k,
+                              ptr(codes), ptr(steps), _st(stream)), "bsp_store_fwd")
+
+
+def bsp_store_read(kind, x, T, Cc, gamma, beta, rstd, mean, codes, steps, read, k: Key, copy_f32, copy_split_t, ld_t,
+                   stream=None):
+    check(lib().bsp_store_read(kind, ptr(x), dtype_code(x), T, Cc, ptr(gamma), ptr(beta), ptr(rstd), ptr(mean),
+                               ptr(codes), ptr(steps), read, k, ptr(copy_f32), ptr(copy_split_t), ld_t, _st(stream)),
+          "bsp_store_read")
+
+
+def bsp_store_wgrad_workspace_bytes(T, O):
+    return lib().bsp_store_wgrad_workspace_bytes(T, O)
+
+
+def bsp_store_wgrad(T, O, Cc, dy_codes_t, q_dy: Quant, copy_split_t, ld_t, dW, ws, diag=None, stream=None):
+    check(lib().bsp_store_wgrad(T, O, Cc, ptr(dy_codes_t), q_dy, ptr(copy_split_t), ld_t, ptr(dW), ptr(ws), ws.numel(),
+                                ptr(diag), _st(stream)), "bsp_store_wgrad")
+
+
+def bsp_mc_check_store_workspace_bytes(desc: StoreDesc, K):
+    return lib().bsp_mc_check_store_workspace_bytes(C.byref(desc), K)
+
+
+def bsp_mc_check_store(desc: StoreDesc, K, ws, diag=None, stream=None, rule=None):
+    """Returns the list of UseResult: gain U, R, N then weight U, R, N, U/R+eps; selected ones only."""
+    res = (UseResult * 8)()
+    n = C.c_int(0)
+    check(lib().bsp_mc_check_store(C.byref(desc), K, _ruleref(rule), res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
+                                   _st(stream)), "bsp_mc_check_store")
     return [res[i] for i in range(n.value)]
 
 

@@ -31,11 +31,13 @@ constexpr int kNumSMs = 148;
 
 // The K-draw gain use behind bsp_norm_gain_mc; `thin` selects the kernel variant made to run beside
 // a kernel that already fills the SMs (its slabs are shorter, so its workspace is larger).
+// `grid_steps` (per-token steps [T]) switches the rounding law from the FP8 store to the b-bit
+// per-token grid (q is then ignored apart from its format, which must still be valid).
 size_t norm_gain_mc_workspace(int64_t T, int64_t C, int K, bool thin);
 int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                      const float* beta, const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q,
                      bsp_key_t key, int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
-                     bsp_diag_t* diag, void* stream);
+                     bsp_diag_t* diag, void* stream, const float* grid_steps = nullptr);
 
 // Index of the current device into a per-device flag array of kMaxDevices entries (a function
 // attribute such as the dynamic shared-memory limit is set once per device, not once per process).

@@ -212,9 +212,9 @@ template <int DT, int DU_DT, int FMT, int NW, int ROWS>
 __global__ void __launch_bounds__(NW * 32, NW == 8 ? 3 : 4)
 gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
-               const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev, PhiloxKey key,
-               int draw_begin, int ndraws, float* __restrict__ partial /* [ndraws][nslabs][C] */,
-               bsp_diag_t* __restrict__ diag) {
+               const void* __restrict__ du, float scale_val, const float* __restrict__ scale_dev,
+               const float* __restrict__ grid_steps, PhiloxKey key, int draw_begin, int ndraws,
+               float* __restrict__ partial /* [ndraws][nslabs][C] */, bsp_diag_t* __restrict__ diag) {
   // A fresh rounding of an element is its round-down value plus, with probability frac, one grid
   // step: value(U) = lo + (U < P) * (hi - lo) with the threshold P of f8_sr_threshold.  So the
   // gain-use sum of draw k is  sum_t (lo/scale - beta)/gamma * du  (the same for every draw, summed
@@ -223,6 +223,9 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
   // shared memory (each thread reads back only what it wrote), which keeps the register count low
   // enough for three blocks per SM: the draw loop is a chain of dependent integer multiplies, and it
   // is occupancy that hides their latency.
+  // grid_steps != NULL selects the b-bit per-token store instead of the FP8 store: the element sits at
+  // t = u / s on the uniform grid of its token's step s, lo = s floor(t), the step weight is s and the
+  // threshold floor(frac(t) 2^32).  Everything after the prologue is the same.
   extern __shared__ __align__(16) float4 mc_smem[];
   uint4* sp = reinterpret_cast<uint4*>(mc_smem);   // [kMcRows][256] thresholds
   constexpr int NT = NW * 32;
@@ -231,7 +234,7 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t c = (int64_t)blockIdx.x * kMcCols + lane * 4;
   const int64_t slab = blockIdx.y, nslabs = gridDim.y;
-  const float scale = scale_dev ? __ldg(scale_dev) : scale_val;
+  const float scale = grid_steps ? 1.0f : (scale_dev ? __ldg(scale_dev) : scale_val);
   const float inv_scale = __fdiv_rn(1.0f, scale);
   const bool col_ok = c < C;
 
@@ -266,9 +269,18 @@ gain_mc_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const
         float u;
         if (kind == BSP_RMSNORM) u = __fmul_rn(__fmul_rn(xs[e], rs), gg[e]);
         else u = __fadd_rn(__fmul_rn(__fmul_rn(__fsub_rn(xs[e], mu), rs), gg[e]), bb[e]);
-        const float v = __fmul_rn(u, scale);
         const float w = __fdiv_rn(ds[e], gg[e]);
         if (!isfinite(xs[e]) || !isfinite(ds[e])) dc.nonfinite++;
+        if (grid_steps) {
+          const float st = __ldg(grid_steps + r);
+          const float t = __fdiv_rn(u, st);
+          const float n0 = floorf(t);
+          thr[e] = __float2uint_rd(__fsub_rn(t, n0) * 4294967296.0f);
+          base[e] = fmaf(fmaf(st, n0, -bb[e]), w, base[e]);
+          wgt[e] = thr[e] ? st * w : 0.f;
+          continue;
+        }
+        const float v = __fmul_rn(u, scale);
         const float lo = sr_value<FMT>(v, 0xFFFFFFFFu), hi = sr_value<FMT>(v, 0u);   // never up / up whenever possible
         thr[e] = f8_sr_threshold<FMT>(v);
         base[e] = fmaf(fmaf(lo, inv_scale, -bb[e]), w, base[e]);
@@ -476,7 +488,7 @@ size_t norm_gain_mc_workspace(int64_t T, int64_t C, int K, bool thin) {
 int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                      const float* beta, const float* rstd, const float* mean, const void* du, int du_dt, bsp_quant_t q,
                      bsp_key_t key, int draw0, int K, const float* g_ref, float* S1, float* S2, void* ws, size_t ws_bytes,
-                     bsp_diag_t* diag, void* stream) {
+                     bsp_diag_t* diag, void* stream, const float* grid_steps) {
   if (!valid_enum(kind, 1) || !valid_enum(dt, 1) || !valid_enum(du_dt, 1) || !valid_enum(q.fmt, 1)) return BSP_ERR_ARG;
   if (key.tensor_id >= (1u << 24) || key.stream > 255u || key.reserved != 0) return BSP_ERR_ARG;
   if (T < 0 || C <= 0 || K < 0 || draw0 < 0) return BSP_ERR_ARG;
@@ -503,14 +515,14 @@ int norm_gain_mc_run(bool thin, int kind, const void* x, int dt, int64_t T, int6
   do {                                                                                                          \
     if (thin) {                                                                                                 \
       gain_mc_kernel<DT, DU, FMT, kMcThinWarps, kMcThinRows><<<grid, kMcThinWarps * 32, kMcThinSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du, \
-                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd, partial, kb == 0 ? diag : nullptr); \
+                                                                 q.scale, q.scale_dev, grid_steps, pk, draw0 + kb, nd, partial, kb == 0 ? diag : nullptr); \
       break;                                                                                                    \
     }                                                                                                           \
     BSP_CHECK_CUDA(cudaFuncSetAttribute(gain_mc_kernel<DT, DU, FMT, 8, kMcRows>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                         (int)kMcSmemBytes));                                                    \
     gain_mc_kernel<DT, DU, FMT, 8, kMcRows><<<grid, 256, kMcSmemBytes, st>>>(kind, x, T, C, gamma, beta, rstd, mean, du,    \
-                                                                 q.scale, q.scale_dev, pk, draw0 + kb, nd,      \
-                                                                 partial, kb == 0 ? diag : nullptr);            \
+                                                                 q.scale, q.scale_dev, grid_steps, pk,           \
+                                                                 draw0 + kb, nd, partial, kb == 0 ? diag : nullptr); \
   } while (0)
       if (q.fmt == BSP_E4M3) {
         if (dt == BSP_F32 && du_dt == BSP_F32) BSP_GM(BSP_F32, BSP_F32, BSP_E4M3);
