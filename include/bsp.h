@@ -594,6 +594,31 @@ int bsp_mc_check_store(const bsp_store_desc_t* op, int K, const bsp_verdict_rule
                        bsp_diag_t* diag, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Log-softmax backward with a +-eps error in its saved output (Appendix "Log-softmax").  The
+ * operator's backward returns h - exp(S) (1^T h) from the incoming gradient h and the saved output
+ * S = l + r, r_j = +-eps independently with equal probability (+eps when the top bit of the
+ * element's generator word is set; element = row * classes + class; draw = trial; the consumed
+ * error on stream 0 of (seed, tensor_id), the independent copy r' on stream 1).  With p = exp(l), g
+ * the returned gradient and g* the one from l itself with the same h, a trial's statistic is the
+ * mean over rows and classes of (g_j - g*_j) / p_j.  Statistics, in order:
+ *   0 likelihood (h = -e_target), S read under reuse (l + r)        -> mean cosh(eps) - 1
+ *   1 likelihood, independent copy (l + r')                         -> mean cosh(eps) - 1
+ *   2 constructed loss (h = r), reuse                               -> mean -eps sinh(eps)
+ *   3 constructed loss, independent copy                            -> mean 0
+ *   4 as 0 with the reconstruction exp(S) divided by cosh(eps)      -> mean 0
+ *   5 as 2 with that division                                       -> mean -eps sinh(eps) / cosh(eps)
+ *   6, 7 the paired contrasts 0 - 1 and 2 - 3 (reuse minus independent copy), trial by trial
+ * stats: HOST array of 8 {mean over trials, standard error over trials, z = |mean| / se}.
+ * per_trial: device [trials * 6] (the six statistics of every trial) or NULL.  logits FP32
+ * [rows * classes], classes a multiple of 4 and at most 8192; trials >= 2.  Synchronises.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct { double mean, se, z; } bsp_lsm_stat_t;
+size_t bsp_lsm_check_workspace_bytes(int rows, int classes, int trials);
+int bsp_lsm_check(const float* logits, const int32_t* target, int rows, int classes, float eps, int trials,
+                  uint64_t seed, uint32_t tensor_id, float* per_trial, bsp_lsm_stat_t* stats, void* ws,
+                  size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait a kernel of
  * this library performs on a barrier gives up after a time limit, raises BSP_ERR_TIMEOUT in `diag`
  * and lets the kernel return normally.  This entry launches one small block whose wait is on a

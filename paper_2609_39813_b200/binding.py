@@ -84,6 +84,10 @@ class StoreDesc(C.Structure):
                 ("grad_fmt", C.c_int32), ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
 
 
+class LsmStat(C.Structure):
+    _fields_ = [("mean", C.c_double), ("se", C.c_double), ("z", C.c_double)]
+
+
 class AttnFp8(C.Structure):
     _fields_ = [("q_scale", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
                 ("do_scale", C.c_void_p), ("p_scale", C.c_float), ("ds_scale", C.c_float)]
@@ -146,6 +150,8 @@ _SIGNATURES = {
     "bsp_mc_check": (_I, [C.POINTER(NormLinearDesc), _I, C.POINTER(VerdictRule), C.POINTER(UseResult), C.POINTER(_I),
                           _P, _SZ, _P, _P]),
     "bsp_selftest_bounded_wait": (_I, [_U64, _P, _P]),
+    "bsp_lsm_check_workspace_bytes": (_SZ, [_I, _I, _I]),
+    "bsp_lsm_check": (_I, [_P, _P, _I, _I, _F, _I, _U64, C.c_uint32, _P, C.POINTER(LsmStat), _P, _SZ, _P]),
     "bsp_store_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _I, Key, _P, _P, _P]),
     "bsp_store_read": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _P, _I, Key, _P, _P, _I64, _P]),
     "bsp_store_wgrad_workspace_bytes": (_SZ, [_I64, _I64]),
@@ -516,6 +522,18 @@ def bsp_mc_check_store(desc: StoreDesc, K, ws, diag=None, stream=None, rule=None
     check(lib().bsp_mc_check_store(C.byref(desc), K, _ruleref(rule), res, C.byref(n), ptr(ws), ws.numel(), ptr(diag),
                                    _st(stream)), "bsp_mc_check_store")
     return [res[i] for i in range(n.value)]
+
+
+def bsp_lsm_check_workspace_bytes(rows, classes, trials):
+    return lib().bsp_lsm_check_workspace_bytes(rows, classes, trials)
+
+
+def bsp_lsm_check(logits, target, rows, classes, eps, trials, seed, tensor_id, per_trial, ws, stream=None):
+    """Returns the eight LsmStat (mean, se, z) of the log-softmax test."""
+    out = (LsmStat * 8)()
+    check(lib().bsp_lsm_check(ptr(logits), ptr(target), rows, classes, eps, trials, int(seed), tensor_id, ptr(per_trial),
+                              out, ptr(ws), ws.numel(), _st(stream)), "bsp_lsm_check")
+    return [out[i] for i in range(8)]
 
 
 def ws_view(ws, offset, count, dtype=None):
