@@ -37,9 +37,10 @@ constexpr int kDkThreads = 320;
 constexpr int kDkND = 4;                           // draws per launch
 constexpr uint32_t kDkStages = 3;                  // ring of streamed Q tiles
 constexpr int kDkBiasTile = AT_BLK * 16 * 2;       // 4 KB: one 128 x 16 bf16 tile of the extra K = 16 step
-// shared memory: K tiles [2], Q ring [3], scaled Q tiles [4] (= the epilogue's 64 KB of staging),
-// barriers, then the ones tile and three buffers of the -LSE tile
-constexpr int kDkSmem = 1024 + (2 + (int)kDkStages + kDkND) * kAtTile + 1024 + 4 * kDkBiasTile;
+// shared memory: K tiles [2], Q ring [3], two buffers of the scaled Q tiles [2][4] (the first one is
+// also the epilogue's 64 KB of staging), barriers, then the ones tile and three buffers of the -LSE tile
+constexpr int kDkSmem = 1024 + (2 + (int)kDkStages + 2 * kDkND) * kAtTile + 1024 + 4 * kDkBiasTile;
+static_assert(kDkSmem <= 232448, "dynamic shared memory of attn_dk_diff_kernel exceeds the SM's");
 
 struct DkDiffParams {
   int BH, S, nblk, causal;
@@ -66,15 +67,17 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   const uint32_t base = (raw + 1023u) & ~1023u;
   const uint32_t res_base = base;                                   // K tile of the item, two buffers
   const uint32_t q0 = base + 2 * kAtTile;                           // stage s: q0 + s * kAtTile
-  const uint32_t bs0 = q0 + kDkStages * kAtTile;                    // draw d: bs0 + d * kAtTile
-  const uint32_t bars = bs0 + kDkND * kAtTile;
+  const uint32_t bs0 = q0 + kDkStages * kAtTile;                    // buffer pb, draw d: bs0 + (4 pb + d) * kAtTile
+  const uint32_t bars = bs0 + 2 * kDkND * kAtTile;
+  // P^T and the scaled tiles are double-buffered (buffer = step & 1), so the probabilities of step
+  // j + 1 are formed while the accumulating product of step j runs
   const uint32_t b_res = bars, b_res_empty = bars + 16, b_sfull = bars + 32, b_sempty = bars + 56,
-                 b_sdp_full = bars + 80, b_sdp_free = bars + 88, b_pds_ready = bars + 96, b_pds_free = bars + 104,
-                 b_acc = bars + 112, b_acc_free = bars + 120, b_bias = bars + 128;
+                 b_sdp_full = bars + 80, b_sdp_free = bars + 88, b_pds_ready = bars + 96 /* [2] */,
+                 b_pds_free = bars + 112 /* [2] */, b_acc = bars + 128, b_acc_free = bars + 136, b_bias = bars + 144;
   const uint32_t bias0 = bars + 1024;                               // ones tile; buffer b: the -LSE tile at 1 + b
   uint8_t* bars_gen = smem_raw + (bars - raw);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 160);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 176);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 180);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nitems = p.nblk * p.BH;
@@ -94,7 +97,8 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     for (int s = 0; s < 2; ++s) { mbar_init(b_res + 8 * s, 1); mbar_init(b_res_empty + 8 * s, 1); }
     for (uint32_t s = 0; s < kDkStages; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
     for (uint32_t s = 0; s < 3; ++s) mbar_init(b_bias + 8 * s, 8);
-    mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
+    mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8);
+    for (int s = 0; s < 2; ++s) { mbar_init(b_pds_ready + 8 * s, 8); mbar_init(b_pds_free + 8 * s, 1); }
     mbar_init(b_acc, 1); mbar_init(b_acc_free, 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -105,7 +109,8 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t t_s = tmem, t_p = tmem + 128, t_acc = tmem + 256;  // accumulator of draw d at t_acc + 64 d
+  // S^T 128 columns, two P^T operands of 64, the accumulator of draw d at t_acc + 64 d
+  const uint32_t t_s = tmem, t_p = tmem + 128, t_acc = tmem + 256;
 
   const uint32_t id_s = make_idesc(1u, 1u, 128, 128);                          // A, B K-major
   const uint32_t id_acc = make_idesc(1u, 1u, 128, 64 * kDkND) | (1u << 16);    // A from tensor memory, B MN-major
@@ -165,18 +170,18 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (nsteps > 0) ok = issue_s(itg);
         for (int it = 0; it < nsteps && ok; ++it) {
           const uint32_t jg = itg + (uint32_t)it;
-          const uint32_t s = jg % kDkStages, ip = jg & 1u;
+          const uint32_t s = jg % kDkStages, pb = jg & 1u, pph = (jg >> 1) & 1u;
           if (it + 1 < nsteps && !issue_s(jg + 1)) { ok = false; break; }
-          if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(b_pds_ready + 8 * pb, pph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           // the accumulators are free once the epilogue of the item before has read them
           if (it == 0 && !mbar_wait(b_acc_free, aph ^ 1u, abort_flag)) { ok = false; break; }
           // all four draws at once: P^T (tensor memory, eight columns per 16 queries) against the four
           // scaled Q tiles side by side (MN-major, one 128-byte atom of 64 columns per draw)
-          const uint64_t bq = make_smem_desc_mn(bs0, (uint32_t)kAtTile);
+          const uint64_t bq = make_smem_desc_mn(bs0 + pb * kDkND * kAtTile, (uint32_t)kAtTile);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc, t_p + 8u * k, bq + 128u * k, id_acc, (it != 0) | (k != 0));
-          tc_commit(b_pds_free);
+          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc, t_p + 64u * pb + 8u * k, bq + 128u * k, id_acc, (it != 0) | (k != 0));
+          tc_commit(b_pds_free + 8 * pb);
           tc_commit(b_sempty + 8 * s);
         }
         itg += (uint32_t)nsteps;
@@ -255,19 +260,18 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int key = blk * AT_BLK + r;                             // this thread's row of S^T
       for (int it = 0; it < nsteps && ok; ++it) {
         const int step = it_begin + it;
-        const uint32_t jt = itg + (uint32_t)it, ip = jt & 1u;
-        // this step's row factors -c (D_k - D*) of query step*128 + r (used after the exponentials)
-        float fk[kDkND];
+        const uint32_t jt = itg + (uint32_t)it, ip = jt & 1u, pb = jt & 1u, pph = (jt >> 1) & 1u;
+        const uint32_t t_pb = t_p + 64u * pb, bsb = bs0 + pb * kDkND * kAtTile;
+        // this step's correction terms of query step*128 + r: requested here, first used after the
+        // exponentials (nothing may depend on these loads before then, or the in-order warp sits out
+        // their latency)
+        float draw_raw[kDkND], dref_raw;
+        const bool q_in = step * AT_BLK + r < p.S;
         {
-          const int q = step * AT_BLK + r;
-          const bool in = q < p.S;
-          const size_t qi = (size_t)bh * p.S + (in ? q : 0);
-          const float dref = __ldg(p.d_ref + qi);
+          const size_t qi = (size_t)bh * p.S + (q_in ? step * AT_BLK + r : 0);
+          dref_raw = __ldg(p.d_ref + qi);
 #pragma unroll
-          for (int d = 0; d < kDkND; ++d) {
-            const float dd = d < p.nd ? __ldg(p.d_draws + (size_t)d * rows_total + qi) : dref;
-            fk[d] = in ? -p.c * (dd - dref) : 0.f;
-          }
+          for (int d = 0; d < kDkND; ++d) draw_raw[d] = d < p.nd ? __ldg(p.d_draws + (size_t)d * rows_total + qi) : 0.f;
         }
         int bias_bh = 0, bias_step = 0;
         const bool bias_due = bias_written == jt + 2u && bias_target(it, bias_bh, bias_step);
@@ -306,10 +310,11 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int j = 0; j < 32; j += 2) pair_at(j, true);
         }
-        // the P^T operand and the scaled tiles are free once the product of the step before has read them
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+        // this buffer of the P^T operand and of the scaled tiles is free once the product of two steps
+        // ago has read it
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free + 8 * pb, pph ^ 1u, abort_flag));
         if (!ok) break;
-        tmem_st16(t_p + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+        tmem_st16(t_pb + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
         if (!edge) {
 #pragma unroll
           for (int j = 32; j < 64; j += 2) pair_at(j, false);
@@ -317,7 +322,7 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
           for (int j = 32; j < 64; j += 2) pair_at(j, true);
         }
-        tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+        tmem_st16(t_pb + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
         // ---- the B operand: row r of the streamed Q tile times this row's factor of each draw, written
         // at the same (swizzled) place of the draw's tile.  Thread (r, h) takes the four 16-byte chunks
         // whose logical index is 4h .. 4h+3; chunk c of row r sits at position c ^ (r & 7), so the lanes
@@ -331,9 +336,15 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
           const uint32_t s = jt % kDkStages, ph = (jt / kDkStages) & 1u;
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sfull + 8 * s, ph, abort_flag));   // (long complete: S^T read the tile)
           if (!ok) break;
+          // the row factors -c (D_k - D*) of the draws (zero for a draw this launch does not have)
           uint32_t f2[kDkND];
+          asm volatile("" : "+f"(dref_raw));
 #pragma unroll
-          for (int d = 0; d < kDkND; ++d) f2[d] = pack_bf16x2(fk[d], fk[d]);
+          for (int d = 0; d < kDkND; ++d) {
+            asm volatile("" : "+f"(draw_raw[d]));
+            const float fk = (q_in && d < p.nd) ? -p.c * (draw_raw[d] - dref_raw) : 0.f;
+            f2[d] = pack_bf16x2(fk, fk);
+          }
           const uint32_t row_off = (uint32_t)r * 128u;
 #pragma unroll
           for (int cch = 0; cch < 4; ++cch) {
@@ -342,7 +353,7 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(q0 + s * kAtTile + off));
 #pragma unroll
             for (int d = 0; d < kDkND; ++d)
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(bs0 + (uint32_t)d * kAtTile + off),
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(bsb + (uint32_t)d * kAtTile + off),
                            "r"(mul_bf16x2(a0, f2[d])), "r"(mul_bf16x2(a1, f2[d])), "r"(mul_bf16x2(a2, f2[d])),
                            "r"(mul_bf16x2(a3, f2[d])) : "memory");
           }
@@ -351,7 +362,7 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         tc_fence_before();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(b_pds_ready);
+        if (lane == 0) mbar_arrive(b_pds_ready + 8 * pb);
         if (bias_due) {
           asm volatile("" : "+f"(bias_next));                       // keeps the first use of the load here
           bias_put(bias_written, bias_next);
