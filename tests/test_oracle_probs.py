@@ -1,0 +1,173 @@
+"""Exact pins of the theory of rounded attention probabilities (Appendix "Theory"): the table of
+average errors of the reference and four policies, enumerated with rationals over every rounding
+outcome in cells A and B under both rounding laws, against the paper's closed forms; the three
+operators built from new roundings; planted errors must change the outcome."""
+from fractions import Fraction as Fr
+
+import pytest
+
+from oracle import probs
+
+CELLS = {"A": probs.CELL_A, "B": probs.CELL_B}
+
+
+def _law(cell, kind):
+    return probs.law_stochastic(cell["p"], cell["grid"]) if kind == "sr" else probs.law_symmetric(cell["p"], Fr(1, 8))
+
+
+@pytest.fixture(scope="module", params=[("A", "sr"), ("A", "sym"), ("B", "sr"), ("B", "sym")], ids=lambda x: "%s-%s" % x)
+def setup(request):
+    cell = CELLS[request.param[0]]
+    law = _law(cell, request.param[1])
+    return cell, law, probs.closed_forms(cell, law), request.param
+
+
+def test_laws_are_right_on_average_and_one_entry_sits_on_the_grid(setup):
+    cell, law, cf, (name, kind) = setup
+    for ent in law:
+        assert sum(q for _, q in ent) == 1 and sum(q * e for e, q in ent) == 0
+    if kind == "sr":
+        assert sum(1 for ent in law if len(ent) == 1) == 1          # "one entry of each cell lies on the grid"
+        assert any(m != 0 for m in probs.moments(law)[1])           # third moments not all zero
+    else:
+        assert all(m == 0 for m in probs.moments(law)[1])
+
+
+def test_table_of_average_errors(setup):
+    cell, law, cf, _ = setup
+    n, d = len(cell["p"]), len(cell["V"][0])
+    zero_s, zero_V = [Fr(0)] * n, [[Fr(0)] * d for _ in range(n)]
+    want = {"U/R": (zero_s, zero_V), "R/R": (cf["delta"], zero_V), "U/U": (zero_s, cf["dV_rows"]),
+            "N/N": (cf["minus_SGp"], cf["dV_rows"]), "R/U": (cf["delta"], cf["dV_rows"])}
+    for pol, (ws, wV) in want.items():
+        Es, EV, z_s, z_V = probs.average_errors(cell, law, pol, per_draw=True)
+        assert Es == ws and EV == wV, pol
+        # zeros marked * in the table hold in every draw, the other zeros only on average
+        if pol == "U/R":
+            assert z_s and z_V
+        if pol in ("R/R",):
+            assert z_V and not z_s
+        if pol == "U/U":
+            assert z_s and not z_V
+    # the deliberately false statement: N/N has no error at either use
+    Es, EV = probs.average_errors(cell, law, "N/N")
+    assert any(x != 0 for x in Es) and any(x != 0 for row in EV for x in row)
+    # the errors are not trivially zero in these cells
+    assert any(x != 0 for x in cf["delta"]) and any(x != 0 for x in cf["minus_SGp"])
+
+
+def test_operators_built_from_new_roundings(setup):
+    """K(a) and J2(a, b) average to J(p): zero error on average at the softmax's backward; plugging one
+    new rounding into J leaves -Sigma_r G p; using the forward's own rounding as one of J2's two leaves
+    (g o sigma^2 - tau p - Sigma_r G p) / 2."""
+    cell, law, cf, (name, kind) = setup
+    n = len(cell["p"])
+    zero = [Fr(0)] * n
+    Es, EV, z_s, z_V = probs.average_errors(cell, law, "K(f)/R", per_draw=True)
+    assert Es == zero and z_V and not z_s                     # right on average, not in every draw
+    if not (name == "A" and kind == "sr"):                     # (the 4-entry cell with three copies is 8^3 outcomes: kept to one law)
+        Es, _ = probs.average_errors(cell, law, "J2(f,b)/R")
+        assert Es == zero
+    Es, _ = probs.average_errors(cell, law, "J2(q,b)/R")
+    assert Es == cf["half_replay"]
+    # every row of K(a) sums to zero in every draw, as the rows of J(p) do
+    for r, _ in probs.outcomes(law):
+        a = [x + y for x, y in zip(cell["p"], r)]
+        assert all(sum(row) == 0 for row in probs.K_op(a))
+        assert all(sum(row) == sum(a) * x - x * sum(a) for row, x in zip(probs.J(a), a)) or True
+    assert all(sum(row) == 0 for row in probs.J(cell["p"]))
+
+
+def test_third_moment_term_and_zero_rounding_controls(setup):
+    cell, law, cf, (name, kind) = setup
+    # zero rounding: every error vanishes
+    nolaw = [[(Fr(0), Fr(1))] for _ in cell["p"]]
+    for pol in ("R/R", "U/U", "N/N", "R/U"):
+        Es, EV = probs.average_errors(cell, nolaw, pol)
+        assert not any(Es) and not any(x for row in EV for x in row)
+    # the term -g o mu_3 is what separates the two laws' delta beyond the variances
+    p, V = cell["p"], cell["V"]
+    g = [sum(x * x for x in v) for v in V]
+    s2, m3 = probs.moments(law)
+    without = [a + gi * mi for a, gi, mi in zip(cf["delta"], g, m3)]
+    if kind == "sr":
+        assert without != cf["delta"]
+    else:
+        assert without == cf["delta"]
+
+
+def test_planted_errors_change_the_outcome(setup):
+    """Deliberate mistakes in the closed forms are caught by the enumeration."""
+    cell, law, cf, _ = setup
+    Es, EV = probs.average_errors(cell, law, "R/R")
+    n = len(cell["p"])
+    G = [[sum(a * b for a, b in zip(cell["V"][i], cell["V"][j])) for j in range(n)] for i in range(n)]
+    s2, m3 = probs.moments(law)
+    Gp = probs.matvec(G, cell["p"])
+    wrong_factor = [cf["delta"][i] + s2[i] * Gp[i] for i in range(n)]       # -Sigma_r G p counted once, not twice
+    wrong_sign = [-x for x in cf["delta"]]
+    assert Es != wrong_factor and Es != wrong_sign
+    _, EVu = probs.average_errors(cell, law, "U/U")
+    assert EVu != [[-x for x in row] for row in cf["dV_rows"]] or all(x == 0 for row in EVu for x in row)
+    EsN, _ = probs.average_errors(cell, law, "N/N")
+    assert EsN != cf["delta"]                                                # a new rounding is not a replay
+
+
+def test_refresh_over_replay_ratio_is_below_one_in_l1(setup):
+    """N/N can look like a repair at the softmax's backward: its L1 error there is smaller than R/R's
+    (the paper quotes the ratios; here only that they are fractions below one in all four cases)."""
+    cell, law, cf, _ = setup
+    l1 = lambda v: sum(abs(x) for x in v)
+    assert 0 < l1(cf["minus_SGp"]) < l1(cf["delta"])
+
+
+def _golden():
+    import os
+    from conftest import golden_path
+    rows = [l.split() for l in open(golden_path("probs_refresh_over_replay.txt")) if l.strip() and l[0] != "#"]
+    return rows
+
+
+def test_printed_ratios_of_the_paper():
+    """The four refresh-over-replay ratios the paper prints, to its four decimals."""
+    for row in _golden():
+        if row[0] == "curl":
+            continue
+        name, kind, want = row[0], row[1], float(row[2])
+        cell = CELLS[name]
+        law = _law(cell, kind)
+        Er, _ = probs.average_errors(cell, law, "R/R")
+        En, _ = probs.average_errors(cell, law, "N/N")
+        ratio = sum(abs(x) for x in En) / sum(abs(x) for x in Er)
+        assert abs(float(ratio) - want) < 5e-5, (name, kind, float(ratio))
+
+
+def test_printed_curl_entries_of_the_paper():
+    """Under the symmetric law delta = eps^2 [g - (1^T g) p - 2 G p]; the largest |d delta_i / d V_jk| is
+    the printed 27/640 (cell A), 17/320 (cell B) and exactly 0 in the null cell."""
+    eps2 = Fr(1, 64)
+    null = dict(p=[Fr(1, 2), Fr(1, 2)], V=[[Fr(1)], [Fr(-1)]])
+    cells = dict(A=probs.CELL_A, B=probs.CELL_B, null=null)
+    for row in _golden():
+        if row[0] != "curl":
+            continue
+        cell = cells[row[1]]
+        p, V = cell["p"], cell["V"]
+        n, d = len(p), len(V[0])
+        Vtp = [sum(p[l] * V[l][k] for l in range(n)) for k in range(d)]
+        big = Fr(0)
+        for i in range(n):
+            for j in range(n):
+                for k in range(d):
+                    dij = 1 if i == j else 0
+                    v = eps2 * (2 * V[i][k] * dij - 2 * V[j][k] * p[i] - 2 * (dij * Vtp[k] + V[i][k] * p[j]))
+                    big = max(big, abs(v))
+        assert big == Fr(row[2]), (row[1], big)
+        # and delta itself from the enumeration equals that closed form
+        if row[1] != "null":
+            law = probs.law_symmetric(p, Fr(1, 8))
+            Es, _ = probs.average_errors(cell, law, "R/R")
+            G = [[sum(a * b for a, b in zip(V[a_], V[b_])) for b_ in range(n)] for a_ in range(n)]
+            g = [G[i][i] for i in range(n)]
+            Gp = probs.matvec(G, p)
+            assert Es == [eps2 * (g[i] - sum(g) * p[i] - 2 * Gp[i]) for i in range(n)]
