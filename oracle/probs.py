@@ -168,3 +168,102 @@ def closed_forms(cell, law):
     half = [(g[i] * s2[i] - tau * p[i] - SGp[i]) / 2 for i in range(n)]
     dV = [[-s2[j] * x for x in V[j]] for j in range(n)]
     return dict(delta=delta, minus_SGp=[-x for x in SGp], half_replay=half, dV_rows=dV)
+
+
+# ----------------------------------------------------------------------------- Monte-Carlo form (float64)
+#
+# The same quantities for many rows at once, over seeded draws instead of every outcome: the form
+# the GPU path evaluates.  p[R, n] rows of probabilities, V[n, d] shared values.  Per draw k the
+# forward's rounding comes from generator stream 0, the new roundings a and b from streams 1 and 2
+# (tensor id TENSOR_P, element = row * n + entry, draw = k).  Laws: LAW_GRID, stochastic rounding to
+# a uniform grid of spacing `param` in threshold form (t = fl32(p / param), up iff W < floor(frac(t)
+# 2^32)); LAW_SIGN, r = +param when the top bit of W is set, else -param.
+
+import numpy as np  # noqa: E402
+
+from . import philox  # noqa: E402
+
+TENSOR_P = 4
+LAW_GRID, LAW_SIGN = 0, 1
+OPERATORS = ("J(q)", "J(f)", "K(f)", "J2(f,b)", "J2(q,b)")        # read at the softmax's backward
+V_READS = ("u", "f")                                               # read at the gradient of V (p_q is exact)
+
+
+def rounded(p32, law: int, param: float, seed: int, stream: int, draw: int) -> np.ndarray:
+    """One rounding of every entry of p32[R, n] (float64 result)."""
+    p32 = np.asarray(p32, dtype=np.float32)
+    w = philox.tensor_words(seed, TENSOR_P, stream, draw, p32.size).reshape(p32.shape)
+    if law == LAW_SIGN:
+        return p32.astype(np.float64) + np.where((w >> np.uint64(31)) & np.uint64(1), param, -param)
+    g = np.float32(param)
+    t = (p32 / g).astype(np.float32)
+    n0 = np.floor(t).astype(np.float32)
+    f = (t - n0).astype(np.float32)
+    P = np.minimum(np.floor(f.astype(np.float64) * 4294967296.0), 4294967295.0).astype(np.uint64)
+    return (n0.astype(np.float64) + (w < P)) * float(g)
+
+
+def apply_J(x, dp):
+    return x * dp - x * np.sum(x * dp, axis=1, keepdims=True)
+
+
+def apply_K(a, dp):
+    return a * np.sum(a, axis=1, keepdims=True) * dp - a * np.sum(a * dp, axis=1, keepdims=True)
+
+
+def apply_J2(a, b, dp):
+    return 0.5 * (a + b) * dp - 0.5 * (a * np.sum(b * dp, axis=1, keepdims=True) + b * np.sum(a * dp, axis=1, keepdims=True))
+
+
+def mc_sums(p32, V, law: int, param: float, seed: int, K: int, draw0: int = 0):
+    """Sums over draws draw0 .. draw0 + K - 1 of the errors Delta_s (per operator of OPERATORS,
+    [5, R, n]) and Delta_V (per read of V_READS, [2, R, n, d]), and of the squares of Delta_s."""
+    p = np.asarray(p32, dtype=np.float32).astype(np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    R, n = p.shape
+    ds = np.zeros((len(OPERATORS), R, n))
+    ds2 = np.zeros_like(ds)
+    dV = np.zeros((len(V_READS), R, n, V.shape[1]))
+    for k in range(draw0, draw0 + K):
+        pq = rounded(p32, law, param, seed, 0, k)
+        pf = rounded(p32, law, param, seed, 1, k)
+        pb = rounded(p32, law, param, seed, 2, k)
+        h = pq @ V                                  # o = V^T p_q row by row; h = o
+        dp = h @ V.T
+        ref = apply_J(p, dp)
+        errs = (apply_J(pq, dp), apply_J(pf, dp), apply_K(pf, dp), apply_J2(pf, pb, dp), apply_J2(pq, pb, dp))
+        for i, e in enumerate(errs):
+            ds[i] += e - ref
+            ds2[i] += (e - ref) ** 2
+        dV[0] += (p - pq)[:, :, None] * h[:, None, :]
+        dV[1] += (pf - pq)[:, :, None] * h[:, None, :]
+    return ds, ds2, dV
+
+
+def closed_forms_rows(p32, V, law: int, param: float):
+    """The paper's closed forms row by row (float64): delta, -Sigma_r G p, the half-replayed J2 error
+    and the rows -sigma_j^2 v_j^T, from the law's exact per-entry variance and third moment."""
+    p32 = np.asarray(p32, dtype=np.float32)
+    p = p32.astype(np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    if law == LAW_SIGN:
+        s2, m3 = np.full_like(p, param * param), np.zeros_like(p)
+    else:
+        g = np.float32(param)
+        t = (p32 / g).astype(np.float32)
+        n0 = np.floor(t).astype(np.float32)
+        f = (t - n0).astype(np.float32)
+        pu = np.minimum(np.floor(f.astype(np.float64) * 4294967296.0), 4294967295.0) / 4294967296.0
+        lo = n0.astype(np.float64) * float(g)
+        mean = lo + pu * float(g)                   # the law's own mean (p up to the FP32 quotient's rounding)
+        e_lo, e_hi = lo - mean, lo + float(g) - mean
+        s2 = (1 - pu) * e_lo ** 2 + pu * e_hi ** 2
+        m3 = (1 - pu) * e_lo ** 3 + pu * e_hi ** 3
+    G = V @ V.T
+    gd = np.diag(G)[None, :]
+    Gp = p @ G
+    tau = np.sum(gd * s2, axis=1, keepdims=True)
+    delta = gd * s2 - tau * p - 2 * s2 * Gp - gd * m3
+    half = 0.5 * (gd * s2 - tau * p - s2 * Gp)
+    dV_rows = -s2[:, :, None] * V[None, :, :]
+    return dict(delta=delta, minus_SGp=-s2 * Gp, half_replay=half, dV_rows=dV_rows, s2=s2)

@@ -171,3 +171,43 @@ def test_printed_curl_entries_of_the_paper():
             g = [G[i][i] for i in range(n)]
             Gp = probs.matvec(G, p)
             assert Es == [eps2 * (g[i] - sum(g) * p[i] - 2 * Gp[i]) for i in range(n)]
+
+
+def test_monte_carlo_form_agrees_with_the_enumeration():
+    """The float64 Monte-Carlo form (the one the GPU path evaluates) on cells A and B: its averages
+    over many seeded draws sit within sampling error of the exact enumeration, for every operator and
+    both reads at the gradient of V (standard errors from the spread of 24 chunks of 400 draws)."""
+    import numpy as np
+    chunks, per = 24, 400
+    for name, cell in CELLS.items():
+        for law_id, kind, param in ((probs.LAW_GRID, "sr", float(cell["grid"])), (probs.LAW_SIGN, "sym", 0.125)):
+            p32 = np.array([[float(x) for x in cell["p"]]], np.float32)
+            V = np.array([[float(x) for x in row] for row in cell["V"]])
+            parts = [probs.mc_sums(p32, V, law_id, param, 17, per, draw0=c * per) for c in range(chunks)]
+            ds = np.stack([q[0][:, 0] / per for q in parts])            # [chunks, 5, n]
+            dV = np.stack([q[2][:, 0] / per for q in parts])            # [chunks, 2, n, d]
+            law = _law(cell, kind)
+            zs = []
+            for i, pol in enumerate(("R/R", "N/N", "K(f)/R", "J2(f,b)/R", "J2(q,b)/R")):
+                if pol == "J2(f,b)/R" and name == "A" and kind == "sr":
+                    want = np.zeros(len(cell["p"]))
+                else:
+                    want = np.array([float(x) for x in probs.average_errors(cell, law, pol)[0]])
+                mean, se = ds[:, i].mean(0), ds[:, i].std(0, ddof=1) / np.sqrt(chunks)
+                zs.append((mean - want)[se > 1e-9] / se[se > 1e-9])
+                assert np.all(np.abs(mean - want) <= 5 * se + 1e-6), (name, kind, pol, mean, want)
+            for i, pol in enumerate(("U/U", "N/N")):
+                want = np.array([[float(x) for x in row] for row in probs.average_errors(cell, law, pol)[1]])
+                mean, se = dV[:, i].mean(0), dV[:, i].std(0, ddof=1) / np.sqrt(chunks)
+                zs.append((mean - want)[se > 1e-9] / se[se > 1e-9])
+                assert np.all(np.abs(mean - want) <= 5 * se + 1e-6), (name, kind, pol)
+            z = np.concatenate(zs)
+            assert np.mean(z * z) < 4.0          # the spread is the sampling error's (entries of a row share a factor)
+            # the closed forms row by row are the enumeration's
+            cf = probs.closed_forms_rows(p32, V, law_id, param)
+            ex = probs.closed_forms(cell, law)
+            # (p is float32 in the Monte-Carlo form: 2/5, 1/5, 3/20, 3/10 are not exact there)
+            assert np.allclose(cf["delta"][0], [float(x) for x in ex["delta"]], rtol=1e-5, atol=1e-7)
+            assert np.allclose(cf["minus_SGp"][0], [float(x) for x in ex["minus_SGp"]], rtol=1e-5, atol=1e-7)
+            assert np.allclose(cf["half_replay"][0], [float(x) for x in ex["half_replay"]], rtol=1e-5, atol=1e-7)
+            assert np.allclose(cf["dV_rows"][0], [[float(x) for x in row] for row in ex["dV_rows"]], rtol=1e-5, atol=1e-7)
