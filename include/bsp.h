@@ -619,6 +619,29 @@ int bsp_lsm_check(const float* logits, const int32_t* target, int rows, int clas
                   size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Rounded attention probabilities as the saved tensor (Appendix "Theory": the theorem "No shared
+ * substitute serves both uses of attention probabilities", the table of average errors, and "One
+ * new rounding suffices at the softmax's backward").  A row has probabilities p[n] and values
+ * V[n, d] (shared by all rows); the forward rounds p to p_q and outputs o = V^T p_q; with the loss
+ * ||o||^2 / 2 the incoming gradient is h = o and dp = V h.  Reference: dV = p_q h^T, ds = J(p) dp,
+ * J(x) = diag(x) - x x^T.  For draws draw0 .. draw0 + K - 1 (the forward's rounding on generator
+ * stream 0, new roundings a and b on streams 1 and 2 of (seed, tensor_id); element = row * n +
+ * entry) the kernel sums the errors of
+ *   ds_sum[5][rows][n]:  (J_hat - J(p)) dp for J_hat = J(p_q) | J(a) | K(a) | J2(a, b) | J2(p_q, b),
+ *     K(a) = diag(a 1^T a) - a a^T,  J2(a, b) = diag((a + b)/2) - (a b^T + b a^T)/2;
+ *   ds_sq (same shape, may be NULL): the sums of their squares;
+ *   dV_sum[2][rows][n][d]:  (p_hat - p_q) h^T for p_hat = p | a.
+ * Averages over the draws estimate the table's entries: delta, -Sigma_r G p, 0, 0,
+ * (g o sigma^2 - tau p - Sigma_r G p)/2, and rows -sigma_j^2 v_j^T for both reads.
+ * law 0: stochastic rounding to a uniform grid of spacing `param` (t = fl32(p / param), up iff
+ * W < floor(frac(t) 2^32)); law 1: r = +param when the top bit of W is set, else -param.
+ * n <= 256, d <= 64, d <= n.  Outputs are overwritten.
+ * ------------------------------------------------------------------------------------------ */
+int bsp_probs_mc(const float* p, const float* V, int64_t rows, int n, int d, int law, float param,
+                 uint64_t seed, uint32_t tensor_id, int draw0, int K, float* ds_sum, float* ds_sq,
+                 float* dV_sum, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait a kernel of
  * this library performs on a barrier gives up after a time limit, raises BSP_ERR_TIMEOUT in `diag`
  * and lets the kernel return normally.  This entry launches one small block whose wait is on a

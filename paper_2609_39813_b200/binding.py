@@ -152,6 +152,7 @@ _SIGNATURES = {
     "bsp_selftest_bounded_wait": (_I, [_U64, _P, _P]),
     "bsp_lsm_check_workspace_bytes": (_SZ, [_I, _I, _I]),
     "bsp_lsm_check": (_I, [_P, _P, _I, _I, _F, _I, _U64, C.c_uint32, _P, C.POINTER(LsmStat), _P, _SZ, _P]),
+    "bsp_probs_mc": (_I, [_P, _P, _I64, _I, _I, _I, _F, _U64, C.c_uint32, _I, _I, _P, _P, _P, _P]),
     "bsp_store_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _I, Key, _P, _P, _P]),
     "bsp_store_read": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _P, _I, Key, _P, _P, _I64, _P]),
     "bsp_store_wgrad_workspace_bytes": (_SZ, [_I64, _I64]),
@@ -534,6 +535,11 @@ def bsp_lsm_check(logits, target, rows, classes, eps, trials, seed, tensor_id, p
     check(lib().bsp_lsm_check(ptr(logits), ptr(target), rows, classes, eps, trials, int(seed), tensor_id, ptr(per_trial),
                               out, ptr(ws), ws.numel(), _st(stream)), "bsp_lsm_check")
     return [out[i] for i in range(8)]
+
+
+def bsp_probs_mc(p, V, rows, n, d, law, param, seed, tensor_id, draw0, K, ds_sum, ds_sq, dV_sum, stream=None):
+    check(lib().bsp_probs_mc(ptr(p), ptr(V), rows, n, d, law, param, int(seed), tensor_id, draw0, K, ptr(ds_sum),
+                             ptr(ds_sq), ptr(dV_sum), _st(stream)), "bsp_probs_mc")
 
 
 def ws_view(ws, offset, count, dtype=None):
