@@ -664,8 +664,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-# DRAM traffic of one gemm_mc_kernel launch by (T, C, O, K), bytes, from ncu (see profiles/)
-GEMM_MC_TRAFFIC = {}
+# DRAM traffic of one gemm_mc_kernel launch by (T, C, O, K), bytes: dram__bytes_read.sum +
+# dram__bytes_write.sum of one ncu capture of `python bench.py --steps 1 --warmup 3 --no-extras
+# --no-cpu-baseline` (profiles/gemm_mc_kernel_cfg5.md)
+GEMM_MC_TRAFFIC = {(16384, 4096, 11008, 16): 8934639360.0 + 362149120.0}
 
 
 def main():

@@ -308,6 +308,9 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (lane == 0) {
       tma_prefetch_desc(&tmap_a);
       tma_prefetch_desc(&tmap_b);
+      // the dY panel of a tile row is read again by every pass over a pair of draws (and by the
+      // other tiles of the row): it should outlive the fresh-code panels, which a wave reads once
+      const uint64_t keep = l2_policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
@@ -320,7 +323,7 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
             mbar_expect_tx(full0 + 8 * s, kMcABytes + (two ? 2 : 1) * kMcBBytes);
-            tma_load_2d(sa, &tmap_a, full0 + 8 * s, kb * BKB, tm * BM);
+            tma_load_2d_hint(sa, &tmap_a, full0 + 8 * s, kb * BKB, tm * BM, keep);
             tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b);
             if (two) tma_load_3d(sb + kMcBBytes, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b + 1);
           }
