@@ -642,6 +642,48 @@ int bsp_probs_mc(const float* p, const float* V, int64_t rows, int n, int d, int
                  float* dV_sum, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Averages over the forward's rounding (Appendix "What the checker reads and reports": the split
+ * E[Delta h] = E[Delta] E[h] + E[(Delta - E Delta)(h - E h)]; Appendix "The same dependence in a
+ * normalization backward": the paired statistic T and its control; Appendix "The normalization
+ * store", continuation probes: the estimator X).  Setting: normalisation -> FP8 store u_q = u + r
+ * (per-tensor amax scale, `forward_mode`) -> y = u_q W^T under the loss ||y||^2 / 2, so dy = y and
+ * du = dy W depend on the rounding the forward consumed.  2 * pairs forwards are drawn (generator
+ * stream 0 of (seed, tensor_id), draws 0, 1, ...; pair k = draws 2k and 2k + 1) and the call leaves
+ * in `ws`, at the offsets bsp_coupling_layout gives, the FP32 averages
+ *   gain_total[C]      the gain-use error under read R, sum_t (r / gamma) o du
+ *   gain_mean_part[C]  sum_t (E r / gamma) o E du; the coupling is gain_total - gain_mean_part
+ *   gain_fresh[C]      the same error under a fresh read (stream 1, the draw of its forward)
+ *   X[C*O], X_sq[C*O]  the mean over pairs of X_k = -(r_a - r_b)^T (dy_a - dy_b) / 2 and of X_k^2;
+ *                      X averages to the weight-use error -r^T dy
+ * and returns in HOST arrays of `pairs` doubles T_k = <r_a - r_b, du_a - du_b> / 2 and the control
+ * <du_a, r_b>.  Under stochastic rounding with per-entry variance sigma^2 and A = W^T W the averages
+ * tend to: gain_total_c -> sum_t sigma^2[t, c] A[c, c] / gamma_c (all of it coupling), T -> sum_{t, c}
+ * sigma^2 A[c, c], control -> 0, X -> -diag(sum_t sigma^2) W^T; with round-to-nearest the forwards
+ * coincide and T and X are exactly zero.  W is rounded to bf16 for the tensor cores (exact for
+ * bf16 workloads); r = u_q - u with u the FP32 chain value.  C, O multiples of 16.  Synchronises.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+  int32_t norm_kind;         /* bsp_norm_t  */
+  int32_t dtype;             /* bsp_dtype_t of x and W */
+  int64_t T, C, O;
+  const void* x;             /* [T, C] */
+  const float* gamma;        /* [C]    */
+  const float* beta;         /* [C] or NULL */
+  const void* W;             /* [O, C] */
+  float eps;
+  int32_t store_fmt;         /* bsp_format_t of the store */
+  int32_t forward_mode;      /* bsp_round_mode_t of the store */
+  uint64_t seed;
+  uint32_t tensor_id;
+  uint32_t reserved;
+} bsp_coupling_desc_t;
+typedef struct { size_t gain_total, gain_mean_part, gain_fresh, X, X_sq; } bsp_coupling_layout_t;
+size_t bsp_coupling_check_workspace_bytes(const bsp_coupling_desc_t* op, int pairs);
+int bsp_coupling_layout(const bsp_coupling_desc_t* op, int pairs, bsp_coupling_layout_t* layout);
+int bsp_coupling_check(const bsp_coupling_desc_t* op, int pairs, double* T, double* control, void* ws,
+                       size_t ws_bytes, bsp_diag_t* diag, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Self-test of the bounded device-side wait (no counterpart in the paper).  Every wait a kernel of
  * this library performs on a barrier gives up after a time limit, raises BSP_ERR_TIMEOUT in `diag`
  * and lets the kernel return normally.  This entry launches one small block whose wait is on a

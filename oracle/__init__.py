@@ -15,6 +15,7 @@ Modules (each function cites the passage of the paper it follows):
   mc         Monte-Carlo reduction, statistics z, R, Q', verdict
   store      the paper's own b-bit per-token store and its reads (incl. the U/R+eps read)
   logsoftmax log-softmax backward with a +-eps error in its saved output, two losses
+  coupling   averages over the forward's rounding: mean-error / coupling split, statistics T and X
   probs      rounded attention probabilities as the saved tensor: exact enumeration and Monte-Carlo form
 
 Parity unpinned (no value of the paper fixes them; only GPU == oracle): the verdict

@@ -84,6 +84,17 @@ class StoreDesc(C.Structure):
                 ("grad_fmt", C.c_int32), ("seed", C.c_uint64), ("tensor_id", C.c_uint32), ("policy_mask", C.c_uint32)]
 
 
+class CouplingDesc(C.Structure):
+    _fields_ = [("norm_kind", C.c_int32), ("dtype", C.c_int32), ("T", C.c_int64), ("C", C.c_int64), ("O", C.c_int64),
+                ("x", C.c_void_p), ("gamma", C.c_void_p), ("beta", C.c_void_p), ("W", C.c_void_p), ("eps", C.c_float),
+                ("store_fmt", C.c_int32), ("forward_mode", C.c_int32), ("seed", C.c_uint64), ("tensor_id", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+
+class CouplingLayout(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("gain_total", "gain_mean_part", "gain_fresh", "X", "X_sq")]
+
+
 class LsmStat(C.Structure):
     _fields_ = [("mean", C.c_double), ("se", C.c_double), ("z", C.c_double)]
 
@@ -153,6 +164,9 @@ _SIGNATURES = {
     "bsp_lsm_check_workspace_bytes": (_SZ, [_I, _I, _I]),
     "bsp_lsm_check": (_I, [_P, _P, _I, _I, _F, _I, _U64, C.c_uint32, _P, C.POINTER(LsmStat), _P, _SZ, _P]),
     "bsp_probs_mc": (_I, [_P, _P, _I64, _I, _I, _I, _F, _U64, C.c_uint32, _I, _I, _P, _P, _P, _P]),
+    "bsp_coupling_check_workspace_bytes": (_SZ, [C.POINTER(CouplingDesc), _I]),
+    "bsp_coupling_layout": (_I, [C.POINTER(CouplingDesc), _I, C.POINTER(CouplingLayout)]),
+    "bsp_coupling_check": (_I, [C.POINTER(CouplingDesc), _I, C.POINTER(C.c_double), C.POINTER(C.c_double), _P, _SZ, _P, _P]),
     "bsp_store_fwd": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _I, Key, _P, _P, _P]),
     "bsp_store_read": (_I, [_I, _P, _I, _I64, _I64, _P, _P, _P, _P, _P, _P, _I, Key, _P, _P, _I64, _P]),
     "bsp_store_wgrad_workspace_bytes": (_SZ, [_I64, _I64]),
@@ -540,6 +554,25 @@ def bsp_lsm_check(logits, target, rows, classes, eps, trials, seed, tensor_id, p
 def bsp_probs_mc(p, V, rows, n, d, law, param, seed, tensor_id, draw0, K, ds_sum, ds_sq, dV_sum, stream=None):
     check(lib().bsp_probs_mc(ptr(p), ptr(V), rows, n, d, law, param, int(seed), tensor_id, draw0, K, ptr(ds_sum),
                              ptr(ds_sq), ptr(dV_sum), _st(stream)), "bsp_probs_mc")
+
+
+def bsp_coupling_check_workspace_bytes(desc: CouplingDesc, pairs):
+    return lib().bsp_coupling_check_workspace_bytes(C.byref(desc), pairs)
+
+
+def bsp_coupling_layout(desc: CouplingDesc, pairs) -> CouplingLayout:
+    lay = CouplingLayout()
+    check(lib().bsp_coupling_layout(C.byref(desc), pairs, C.byref(lay)), "bsp_coupling_layout")
+    return lay
+
+
+def bsp_coupling_check(desc: CouplingDesc, pairs, ws, diag=None, stream=None):
+    """Returns (T[pairs], control[pairs]) as lists of floats; the averaged tensors stay in `ws`."""
+    T = (C.c_double * pairs)()
+    ctl = (C.c_double * pairs)()
+    check(lib().bsp_coupling_check(C.byref(desc), pairs, T, ctl, ptr(ws), ws.numel(), ptr(diag), _st(stream)),
+          "bsp_coupling_check")
+    return list(T), list(ctl)
 
 
 def ws_view(ws, offset, count, dtype=None):
