@@ -357,6 +357,86 @@ def attention_section(b, peaks, steps=3):
                 diag_status=b.read_diag(diag)["status"])
 
 
+def widened_section(b, torch):
+    """The rows built after the core path, each timed as a whole through its own entry point on seeded
+    inputs: the b-bit per-token store's check (config 2's shape, 6 bits, K = 16), the averages over the
+    forward's rounding (config 2's shape, 8 pairs of forwards), rounded attention probabilities
+    (16384 rows of 128 keys, d = 64, 256 draws) and the log-softmax case (64 x 128, 4096 trials)."""
+    import numpy as np
+    from paper_2609_39813_b200 import workloads
+    from paper_2609_39813_b200.harness import NormLinearGpu, up
+    stream = torch.cuda.current_stream()
+    out = {}
+    inp = workloads.config2()
+    g = NormLinearGpu(inp)
+    diag = b.new_diag()
+
+    # f1: the paper's own store
+    K, bits = 16, 6
+    d = b.StoreDesc()
+    d.norm_kind, d.dtype = g.kind, b.BF16
+    d.T, d.C, d.O = inp.T, inp.C, inp.O
+    d.x, d.gamma, d.beta, d.W, d.dY = b.ptr(g.x), b.ptr(g.gamma), b.ptr(g.beta), b.ptr(g.W), b.ptr(g.dY)
+    d.eps, d.bits, d.grad_fmt = inp.eps, bits, inp.grad_fmt
+    d.seed, d.tensor_id, d.policy_mask = inp.seed, 1, 0x7F
+    ws = b.workspace(b.bsp_mc_check_store_workspace_bytes(d, K))
+    res = b.bsp_mc_check_store(d, K, ws, diag)
+    ms = timed(torch, stream, lambda: b.bsp_mc_check_store(d, K, ws, diag), reps=5, warm=1)
+    el = inp.T * inp.C * ((1 + 1 + K) + (1 + 1 + K + K))
+    out["store"] = dict(workload="cfg2 shape, %d-bit per-token store, K=%d" % (bits, K), ms_per_check=ms,
+                        check_elements_per_s=el / (ms * 1e-3), verdicts=[int(r.verdict) for r in res],
+                        rows="gain U,R,N then weight U,R,N,R+eps")
+    del ws
+
+    # f2: averages over the forward's rounding
+    pairs = 8
+    c = b.CouplingDesc()
+    c.norm_kind, c.dtype = g.kind, b.BF16
+    c.T, c.C, c.O = inp.T, inp.C, inp.O
+    c.x, c.gamma, c.beta, c.W = b.ptr(g.x), b.ptr(g.gamma), b.ptr(g.beta), b.ptr(g.W)
+    c.eps, c.store_fmt, c.forward_mode, c.seed, c.tensor_id = inp.eps, 0, 1, inp.seed, 1
+    ws = b.workspace(b.bsp_coupling_check_workspace_bytes(c, pairs))
+    Tst, ctl = b.bsp_coupling_check(c, pairs, ws, diag)
+    ms = timed(torch, stream, lambda: b.bsp_coupling_check(c, pairs, ws, diag), reps=3, warm=1)
+    out["coupling"] = dict(workload="cfg2 shape, E4M3 store, loss |y|^2/2, %d pairs of forwards" % pairs,
+                           ms_per_check=ms, forwards_per_s=2 * pairs / (ms * 1e-3),
+                           T_mean=float(np.mean(Tst)), control_mean=float(np.mean(ctl)))
+    del ws
+
+    # f3: rounded probabilities
+    R, n, dd, draws = 16384, 128, 64, 256
+    rng = np.random.default_rng(3003)
+    sc = rng.standard_normal((R, n)) * 1.5
+    p = np.exp(sc - sc.max(1, keepdims=True))
+    p = (p / p.sum(1, keepdims=True)).astype(np.float32)
+    V = (rng.standard_normal((n, dd)) / np.sqrt(dd)).astype(np.float32)
+    pg, Vg = torch.from_numpy(p).cuda(), torch.from_numpy(V).cuda()
+    ds = torch.zeros(5 * R * n, device="cuda")
+    sq = torch.zeros(5 * R * n, device="cuda")
+    dV = torch.zeros(2 * R * n * dd, device="cuda")
+    fn = lambda: b.bsp_probs_mc(pg, Vg, R, n, dd, 0, 1.0 / 64, 3003, 4, 0, draws, ds, sq, dV)
+    ms = timed(torch, stream, fn, reps=3, warm=1)
+    out["probs"] = dict(workload="%d rows x %d keys, d=%d, grid 1/64, %d draws" % (R, n, dd, draws), ms=ms,
+                        entry_draws_per_s=R * n * draws / (ms * 1e-3))
+    del ds, sq, dV
+
+    # f4: log-softmax
+    rows, classes, trials, eps = 64, 128, 4096, 0.1
+    rng = np.random.default_rng(1926)
+    logits = torch.from_numpy(rng.standard_normal((rows, classes)).astype(np.float32)).cuda()
+    target = torch.from_numpy(rng.integers(0, classes, rows).astype(np.int32)).cuda()
+    ws = b.workspace(b.bsp_lsm_check_workspace_bytes(rows, classes, trials))
+    st = b.bsp_lsm_check(logits, target, rows, classes, eps, trials, 1926, 3, None, ws)
+    ms = timed(torch, stream, lambda: b.bsp_lsm_check(logits, target, rows, classes, eps, trials, 1926, 3, None, ws),
+               reps=3, warm=1)
+    out["logsoftmax"] = dict(workload="%d x %d, eps %.2f, %d trials" % (rows, classes, eps, trials), ms=ms,
+                             entry_trials_per_s=rows * classes * trials / (ms * 1e-3),
+                             mean_error_reuse=st[0].mean, predicted=float(np.cosh(eps) - 1),
+                             coupling=st[2].mean, predicted_coupling=float(-eps * np.sinh(eps)))
+    out["diag_status"] = b.read_diag(diag)["status"]
+    return out
+
+
 def kernel_table(b, peaks, g):
     """The streaming kernels one by one on config 5's own tensors (T=16384, C=4096, O=11008, bf16):
     microseconds per launch and algorithmic GB/s (bytes the method must move / time) against the
@@ -659,6 +739,8 @@ def run_ours(args):
         line["config4"] = norm_linear_check(b, torch, workloads.config4(), steps=2, side=side)
         torch.cuda.empty_cache()
         line["attention"] = attention_section(b, peaks, steps=args.attention_steps)
+        torch.cuda.empty_cache()
+        line["widened"] = widened_section(b, torch)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
