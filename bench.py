@@ -539,6 +539,29 @@ def kernel_table(b, peaks, g):
     tc("weight gradient, 16 fresh draws with sums (gemm_mc)", "tensor",
        lambda: b.bsp_linear_wgrad_mc(T, O, C, dyc_t, qrn, fresh_t, qf, T, Kd, ref, S1, S2, diag),
        2.0 * T * O * C * Kd, "TFLOP/s", 2.0 * peaks["bf16_tflops"], NOMINAL_FP8_TFLOPS, reps=3)
+    # ---- the b-bit per-token store (6 bits) on the same tensors
+    del fresh_t
+    torch.cuda.empty_cache()
+    bits = 6
+    scodes = torch.zeros(T * C, dtype=torch.int8, device="cuda")
+    ssteps = torch.zeros(T, device="cuda")
+    split = torch.zeros(C * 2 * T, dtype=torch.bfloat16, device="cuda")
+    tc("b-bit store forward, stochastic (store_fwd_kernel)", "alu",
+       lambda: b.bsp_store_fwd(b.RMSNORM, x, T, C, gamma, None, rstd, mean, bits, b.key(1, 1, 0), scodes, ssteps),
+       float(T) * C, "G element-draws/s", alu_peak, reps=10)
+    compute[-1]["gb_per_s"] = T * C * 3 / compute[-1]["us"] / 1e3
+    tc("b-bit store, copy for the weight use, read U/R+eps (store_operand_kernel)", "alu",
+       lambda: b.bsp_store_read(b.RMSNORM, x, T, C, gamma, None, rstd, mean, scodes, ssteps, 3, b.key(1, 1, 2, 1), None, split, T),
+       float(T) * C, "G element-draws/s", alu_peak, reps=10)
+    compute[-1]["gb_per_s"] = T * C * 7 / compute[-1]["us"] / 1e3
+    t("b-bit store, copy for the weight use, read R (store_operand_kernel)", "hbm",
+      lambda: b.bsp_store_read(b.RMSNORM, x, T, C, gamma, None, rstd, mean, scodes, ssteps, 1, b.key(1, 1, 2, 1), None, split, T),
+      T * C * 7)
+    wst = b.workspace(max(b.bsp_store_wgrad_workspace_bytes(T, O), 256))
+    tc("b-bit store weight gradient, hi+lo split operand (decode + gemm_tc bf16, contraction over 2T)", "tensor",
+       lambda: b.bsp_store_wgrad(T, O, C, dyc_t, qrn, split, T, dW, wst, diag),
+       2.0 * T * O * C, "TFLOP/s", peaks["bf16_tflops"], NOMINAL_BF16_TFLOPS)
+    compute[-1]["note"] = "algorithmic flop 2 T O C; the kernel computes twice that (two bf16 terms per operand value)"
     return dict(shape=dict(T=T, C=C, O=O, dtype="bf16"), data="seeded host recipe (config 5)",
                 hbm_peak_gbs=peaks["hbm_gbs"], hbm_nominal_gbs=NOMINAL_HBM_GBS, peak_source=peaks["source"],
                 kernels=rows, compute_kernels=compute, diag_status=b.read_diag(diag)["status"])

@@ -7,9 +7,12 @@
 //   Delta_s for J_hat in { J(p_q), J(a), K(a), J2(a, b), J2(p_q, b) }  (a, b: new roundings;
 //     K(a) = diag(a 1^T a) - a a^T, J2(a, b) = diag((a + b) / 2) - (a b^T + b a^T) / 2);
 //   Delta_V for p_hat in { p, a }.
-// One block per row, one thread per entry (n <= 256), V (n x d, d <= 64) in shared memory; per draw
-// three generator words per entry, two small dense products (h = V^T p_q, dp = V h) and five
-// block-wide dot products.  CUDA cores only: the rows are far too small for tensor tiles.
+// One block per row, one thread per entry (n <= 256).  V (n x d, d <= 64) lies in shared memory for
+// h = V^T p_q (every thread sums a slice of one column) and, row by row, in the threads' registers
+// for dp = V h; a thread keeps its 2 x d sums of the gradient-of-V errors in registers for all draws.
+// Per draw: three generator words per entry (the four threads of a generator block share its
+// streams), 4 n d multiply-adds, five block-wide dot products, three block barriers.  CUDA cores
+// only: bound by the FP32 multiply-add rate (4 n d per row and draw).
 #include "common.cuh"
 
 namespace bsp {
@@ -24,80 +27,156 @@ __device__ __forceinline__ float probs_round(float p, int law, float param, uint
   return (n0 + (w < P ? 1.f : 0.f)) * param;
 }
 
-// Sum over the block of up to five values per thread (warp shuffles, then one shared-memory pass).
-template <int NV>
-__device__ __forceinline__ void block_sums(float (&v)[NV], float (*red)[NV], int nwarps) {
-#pragma unroll
-  for (int i = 0; i < NV; ++i) v[i] = warp_sum(v[i]);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0)
-    for (int i = 0; i < NV; ++i) red[threadIdx.x >> 5][i] = v[i];
-  __syncthreads();
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    float t = 0.f;
-    for (int w = 0; w < nwarps; ++w) t += red[w][i];
-    v[i] = t;
+// Shared memory of a block: V as [npad][d] (rows beyond n are zero), the forward's rounding of the
+// row pq[npad], and the partial sums of h = V^T p_q as [parts][64] (columns beyond d are zero).
+struct ProbsSmem {
+  int parts, per, npad;
+  __host__ __device__ ProbsSmem(int n, int d, int threads) {
+    parts = threads / d;
+    if (parts > 4) parts = 4;
+    if (parts < 1) parts = 1;
+    per = ((n + parts - 1) / parts + 3) & ~3;
+    npad = parts * per;
   }
-}
+  __host__ __device__ size_t floats(int d) const { return (size_t)npad * d + npad + (size_t)parts * kPrMaxD; }
+};
 
-__global__ void __launch_bounds__(kPrMaxN)
+// SHARE: n is a multiple of 4, so the four threads of entries 4q .. 4q+3 need words of the same
+// generator blocks: each computes the block of one stream and they exchange words by shuffles.
+template <bool SHARE>
+__global__ void __launch_bounds__(kPrMaxN, 1)
 probs_mc_kernel(const float* __restrict__ p_all, const float* __restrict__ V, int n, int d, int law, float param,
                 PhiloxKey kq, PhiloxKey ka, PhiloxKey kb, int draw0, int K, float* __restrict__ ds_sum,
                 float* __restrict__ ds_sq, float* __restrict__ dV_sum, size_t rows) {
-  extern __shared__ float sm[];
-  float* Vs = sm;                                  // [n][d]
-  float* pq_s = Vs + (size_t)n * d;                // [n]
-  float* h_s = pq_s + n;                           // [d]
-  __shared__ float red[kPrMaxN / 32][6];
+  extern __shared__ __align__(16) float sm[];
+  const ProbsSmem lay(n, d, blockDim.x);
+  float* Vs = sm;                                  // [npad][d]
+  float* pq_s = Vs + (size_t)lay.npad * d;         // [npad]
+  float* hp_s = pq_s + lay.npad;                   // [parts][64]
+  __shared__ float red[kPrMaxN / 32][5];
   const size_t row = blockIdx.x;
-  const int j = threadIdx.x, nwarps = (blockDim.x + 31) / 32;
+  const int j = threadIdx.x, lane = j & 31, nwarps = (blockDim.x + 31) / 32;
   const bool on = j < n;
-  for (int i = threadIdx.x; i < n * d; i += blockDim.x) Vs[i] = V[i];
+  for (int i = threadIdx.x; i < lay.npad * d; i += blockDim.x) Vs[i] = i < n * d ? V[i] : 0.f;
+  for (int i = threadIdx.x; i < lay.npad; i += blockDim.x) pq_s[i] = 0.f;
+  for (int i = threadIdx.x; i < lay.parts * kPrMaxD; i += blockDim.x) hp_s[i] = 0.f;
+  // this thread's row of V stays in registers: dp_j = sum_c V[j][c] h[c]
+  float Vr[kPrMaxD];
+#pragma unroll
+  for (int c = 0; c < kPrMaxD; ++c) Vr[c] = (on && c < d) ? V[(size_t)j * d + c] : 0.f;
   const float p = on ? p_all[row * n + j] : 0.f;
   const size_t e = row * n + (on ? j : 0);
   float acc_s[kPrOps] = {0.f, 0.f, 0.f, 0.f, 0.f}, acc_q[kPrOps] = {0.f, 0.f, 0.f, 0.f, 0.f};
   float acc_vu[kPrMaxD], acc_va[kPrMaxD];
 #pragma unroll
   for (int c = 0; c < kPrMaxD; ++c) acc_vu[c] = acc_va[c] = 0.f;
+  // the partial sum of h this thread forms: column hc over the entries [i0, i0 + per)
+  const bool h_worker = j < lay.parts * d;
+  const int hc = j % d, hpart = j / d, i0 = hpart * lay.per;
+  // sum_j p_j - 1 in double, once per row (K(a) needs 1^T a - 1 = sum (a - p) + (sum p - 1))
+  __shared__ double red_d[kPrMaxN / 32];
+  {
+    double t = (double)p;
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if (lane == 0) red_d[j >> 5] = t;
+  }
   __syncthreads();
+  float sum_p_m1;
+  {
+    double t = 0.0;
+    for (int w = 0; w < nwarps; ++w) t += red_d[w];
+    sum_p_m1 = (float)(t - 1.0);
+  }
   for (int k = draw0; k < draw0 + K; ++k) {
+    uint32_t wq, wa, wb;
+    if (SHARE) {
+      const int pos = j & 3;
+      const uint64_t q = (row * (size_t)n + (size_t)j) >> 2;             // the same for the four threads of a group
+      const uint32_t c3 = (kq.c3 & ~0xFFu) | (uint32_t)pos;               // streams 0, 1, 2 (3: unused)
+      const uint4 w = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)k, c3, kq.k0, kq.k1);
+      wq = wa = wb = 0u;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        // round r: every thread sends word (pos + r) & 3 and reads from the group's thread (pos - r) & 3,
+        // which is that thread's word `pos`
+        const int src = (pos - r) & 3;
+        const uint32_t got = __shfl_sync(0xFFFFFFFFu, word_of(w, (uint32_t)((pos + r) & 3)), (lane & ~3) | src);
+        if (src == 0) wq = got; else if (src == 1) wa = got; else if (src == 2) wb = got;
+      }
+    } else {
+      wq = word_of(philox_block(kq, e >> 2, (uint32_t)k), (uint32_t)(e & 3));
+      wa = word_of(philox_block(ka, e >> 2, (uint32_t)k), (uint32_t)(e & 3));
+      wb = word_of(philox_block(kb, e >> 2, (uint32_t)k), (uint32_t)(e & 3));
+    }
     float pq = 0.f, a = 0.f, b = 0.f;
     if (on) {
-      pq = probs_round(p, law, param, word_of(philox_block(kq, e >> 2, (uint32_t)k), (uint32_t)(e & 3)));
-      a = probs_round(p, law, param, word_of(philox_block(ka, e >> 2, (uint32_t)k), (uint32_t)(e & 3)));
-      b = probs_round(p, law, param, word_of(philox_block(kb, e >> 2, (uint32_t)k), (uint32_t)(e & 3)));
+      pq = probs_round(p, law, param, wq);
+      a = probs_round(p, law, param, wa);
+      b = probs_round(p, law, param, wb);
+      pq_s[j] = pq;
     }
-    __syncthreads();                               // the previous draw's readers of pq_s / h_s are done
-    if (on) pq_s[j] = pq;
     __syncthreads();
-    if (j < d) {                                   // h = V^T p_q
+    if (h_worker) {                                // h = V^T p_q, in `parts` partial sums per column
+      float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+      const float* vcol = Vs + (size_t)i0 * d + hc;
+      for (int i = 0; i < lay.per; i += 4) {
+        const float4 q4 = *reinterpret_cast<const float4*>(pq_s + i0 + i);
+        t0 = fmaf(vcol[(size_t)(i + 0) * d], q4.x, t0);
+        t1 = fmaf(vcol[(size_t)(i + 1) * d], q4.y, t1);
+        t2 = fmaf(vcol[(size_t)(i + 2) * d], q4.z, t2);
+        t3 = fmaf(vcol[(size_t)(i + 3) * d], q4.w, t3);
+      }
+      hp_s[hpart * kPrMaxD + hc] = (t0 + t1) + (t2 + t3);
+    }
+    __syncthreads();
+    // dp = V h and the two gradient-of-V errors (p_hat - p_q) h^T in one walk over the columns
+    const float eu = p - pq, ea = a - pq;
+    float dp = 0.f;
+#pragma unroll
+    for (int c0 = 0; c0 < kPrMaxD; c0 += 4) {
+      if (c0 < d) {
+        float4 h4 = *reinterpret_cast<const float4*>(hp_s + c0);
+        for (int pp = 1; pp < lay.parts; ++pp) {
+          const float4 g4 = *reinterpret_cast<const float4*>(hp_s + pp * kPrMaxD + c0);
+          h4.x += g4.x; h4.y += g4.y; h4.z += g4.z; h4.w += g4.w;
+        }
+        dp = fmaf(Vr[c0], h4.x, dp); dp = fmaf(Vr[c0 + 1], h4.y, dp);
+        dp = fmaf(Vr[c0 + 2], h4.z, dp); dp = fmaf(Vr[c0 + 3], h4.w, dp);
+        acc_vu[c0] = fmaf(eu, h4.x, acc_vu[c0]); acc_vu[c0 + 1] = fmaf(eu, h4.y, acc_vu[c0 + 1]);
+        acc_vu[c0 + 2] = fmaf(eu, h4.z, acc_vu[c0 + 2]); acc_vu[c0 + 3] = fmaf(eu, h4.w, acc_vu[c0 + 3]);
+        acc_va[c0] = fmaf(ea, h4.x, acc_va[c0]); acc_va[c0 + 1] = fmaf(ea, h4.y, acc_va[c0 + 1]);
+        acc_va[c0 + 2] = fmaf(ea, h4.z, acc_va[c0 + 2]); acc_va[c0 + 3] = fmaf(ea, h4.w, acc_va[c0 + 3]);
+      }
+    }
+    // the block-wide sums the operators need, taken on the differences to p so that no operator's
+    // error is formed as a small difference of large terms:
+    //   s0 = p.dp, Dq = (pq - p).dp, Da = (a - p).dp, Db = (b - p).dp, Sa = sum (a - p)
+    const float dq = pq - p, da = a - p, db = b - p;
+    float dots[5] = {p * dp, dq * dp, da * dp, db * dp, da};
+#pragma unroll
+    for (int i = 0; i < 5; ++i) dots[i] = warp_sum(dots[i]);
+    if (lane == 0)
+      for (int i = 0; i < 5; ++i) red[j >> 5][i] = dots[i];
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 5; ++i) {
       float t = 0.f;
-      for (int i = 0; i < n; ++i) t = fmaf(Vs[i * d + j], pq_s[i], t);
-      h_s[j] = t;
+      for (int w = 0; w < nwarps; ++w) t += red[w][i];
+      dots[i] = t;
     }
-    __syncthreads();
-    float dp = 0.f;                                // dp = V h
-    if (on)
-      for (int c = 0; c < d; ++c) dp = fmaf(Vs[j * d + c], h_s[c], dp);
-    // the dot products the operators need: p.dp, pq.dp, a.dp, b.dp, sum a
-    float dots[5] = {p * dp, pq * dp, a * dp, b * dp, a};
-    block_sums<5>(dots, reinterpret_cast<float(*)[5]>(&red[0][0]), nwarps);
     if (on) {
-      const float ref = p * dp - p * dots[0];                                   // J(p) dp
+      // with J(x) dp = x o dp - x (x.dp) and x = p + dx:  (J(x) - J(p)) dp = dx (dp - s0) - x (dx.dp)
+      const float c = dp - dots[0];
       float err[kPrOps];
-      err[0] = (pq * dp - pq * dots[1]) - ref;                                   // J(p_q)
-      err[1] = (a * dp - a * dots[2]) - ref;                                     // J(a)
-      err[2] = (a * dots[4] * dp - a * dots[2]) - ref;                           // K(a)
-      err[3] = (0.5f * (a + b) * dp - 0.5f * (a * dots[3] + b * dots[2])) - ref; // J2(a, b)
-      err[4] = (0.5f * (pq + b) * dp - 0.5f * (pq * dots[3] + b * dots[1])) - ref;   // J2(p_q, b)
+      err[0] = dq * c - pq * dots[1];                                            // J(p_q)
+      err[1] = da * c - a * dots[2];                                             // J(a)
+      err[2] = a * (dots[4] + sum_p_m1) * dp + err[1];                           // K(a): + a (1^T a - 1) dp
+      err[3] = 0.5f * ((da + db) * c - (a * dots[3] + b * dots[2]));             // J2(a, b)
+      err[4] = 0.5f * ((dq + db) * c - (pq * dots[3] + b * dots[1]));            // J2(p_q, b)
 #pragma unroll
       for (int i = 0; i < kPrOps; ++i) { acc_s[i] += err[i]; acc_q[i] = fmaf(err[i], err[i], acc_q[i]); }
-      const float eu = p - pq, ea = a - pq;
-#pragma unroll
-      for (int c = 0; c < kPrMaxD; ++c)
-        if (c < d) { acc_vu[c] = fmaf(eu, h_s[c], acc_vu[c]); acc_va[c] = fmaf(ea, h_s[c], acc_va[c]); }
     }
+    // red[] and pq_s are written again only after the next draw's first barrier, hp_s after its second
   }
   if (!on) return;
 #pragma unroll
@@ -105,12 +184,20 @@ probs_mc_kernel(const float* __restrict__ p_all, const float* __restrict__ V, in
     ds_sum[((size_t)i * rows + row) * n + j] = acc_s[i];
     if (ds_sq) ds_sq[((size_t)i * rows + row) * n + j] = acc_q[i];
   }
+  float* o_u = dV_sum + (((size_t)0 * rows + row) * n + j) * d;
+  float* o_a = dV_sum + (((size_t)1 * rows + row) * n + j) * d;
+  if ((d & 3) == 0) {
 #pragma unroll
-  for (int c = 0; c < kPrMaxD; ++c)
-    if (c < d) {
-      dV_sum[(((size_t)0 * rows + row) * n + j) * d + c] = acc_vu[c];
-      dV_sum[(((size_t)1 * rows + row) * n + j) * d + c] = acc_va[c];
-    }
+    for (int c = 0; c < kPrMaxD; c += 4)
+      if (c < d) {
+        *reinterpret_cast<float4*>(o_u + c) = make_float4(acc_vu[c], acc_vu[c + 1], acc_vu[c + 2], acc_vu[c + 3]);
+        *reinterpret_cast<float4*>(o_a + c) = make_float4(acc_va[c], acc_va[c + 1], acc_va[c + 2], acc_va[c + 3]);
+      }
+  } else {
+#pragma unroll
+    for (int c = 0; c < kPrMaxD; ++c)
+      if (c < d) { o_u[c] = acc_vu[c]; o_a[c] = acc_va[c]; }
+  }
 }
 
 }  // namespace bsp
@@ -132,11 +219,14 @@ int bsp_probs_mc(const float* p, const float* V, int64_t rows, int n, int d, int
   k.stream = 1; const PhiloxKey ka = make_key(k);
   k.stream = 2; const PhiloxKey kb = make_key(k);
   const int threads = (n + 31) / 32 * 32;
-  const size_t smem = ((size_t)n * d + n + d) * sizeof(float);
+  const ProbsSmem lay(n, d, threads);
+  const size_t smem = lay.floats(d) * sizeof(float);
+  const bool share = (n & 3) == 0;
+  auto kern = share ? probs_mc_kernel<true> : probs_mc_kernel<false>;
   if (smem > 48 * 1024)
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(probs_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  probs_mc_kernel<<<(unsigned)rows, threads, smem, (cudaStream_t)stream>>>(p, V, n, d, law, param, kq, ka, kb, draw0, K, ds_sum,
-                                                                          ds_sq, dV_sum, (size_t)rows);
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  kern<<<(unsigned)rows, threads, smem, (cudaStream_t)stream>>>(p, V, n, d, law, param, kq, ka, kb, draw0, K, ds_sum, ds_sq,
+                                                               dV_sum, (size_t)rows);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
