@@ -275,6 +275,7 @@ constexpr int kMcThreads = 320;
 constexpr size_t kMcSmem = (size_t)kMcStages * kMcStageBytes + 1024 + 256;
 
 
+template <bool FP8>
 __global__ void __launch_bounds__(kMcThreads, 1)
 gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -289,7 +290,8 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + MC_BN - 1) / MC_BN;
   const int ntiles = tiles_m * tiles_n;
-  const int kblocks = (p.K + BKB - 1) / BKB;          // FP8: one byte per element
+  constexpr int kElemsPerStage = FP8 ? BKB : BKB / 2;   // K extent of one 128-byte stage in elements
+  const int kblocks = (p.K + kElemsPerStage - 1) / kElemsPerStage;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kMcStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -323,9 +325,9 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t sa = tiles + s * kMcStageBytes, sb = sa + kMcABytes;
             mbar_expect_tx(full0 + 8 * s, kMcABytes + (two ? 2 : 1) * kMcBBytes);
-            tma_load_2d_hint(sa, &tmap_a, full0 + 8 * s, kb * BKB, tm * BM, keep);
-            tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b);
-            if (two) tma_load_3d(sb + kMcBBytes, &tmap_b, full0 + 8 * s, kb * BKB, tn * MC_BN, b + 1);
+            tma_load_2d_hint(sa, &tmap_a, full0 + 8 * s, kb * kElemsPerStage, tm * BM, keep);
+            tma_load_3d(sb, &tmap_b, full0 + 8 * s, kb * kElemsPerStage, tn * MC_BN, b);
+            if (two) tma_load_3d(sb + kMcBBytes, &tmap_b, full0 + 8 * s, kb * kElemsPerStage, tn * MC_BN, b + 1);
           }
         }
       }
@@ -353,7 +355,7 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);   // B: 128 or 256 rows
 #pragma unroll
             for (int k = 0; k < BKB / 32; ++k)
-              tc_mma<true>(tmem_base, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+              tc_mma<FP8>(tmem_base, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
             tc_commit(empty0 + 8 * s);
           }
           if (ok) tc_commit(tfull0);
@@ -386,7 +388,8 @@ gemm_mc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           const size_t off = (size_t)row * p.ldc + col;
 #pragma unroll
           for (int j = 0; j < 16; j += 4) {
-            const float4 g0 = *reinterpret_cast<const float4*>(p.ref + off + j);
+            // no reference: the products are differences to the reference already
+            const float4 g0 = p.ref ? *reinterpret_cast<const float4*>(p.ref + off + j) : make_float4(0.f, 0.f, 0.f, 0.f);
             const uint4 v1 = *reinterpret_cast<const uint4*>(p.S1 + off + j);
             const uint4 v2 = *reinterpret_cast<const uint4*>(p.S2 + off + j);
             refv[c * 16 + j] = g0.x; refv[c * 16 + j + 1] = g0.y; refv[c * 16 + j + 2] = g0.z; refv[c * 16 + j + 3] = g0.w;
@@ -516,7 +519,7 @@ gemm_simt_kernel(const void* __restrict__ A, const void* __restrict__ B, int a_f
     } else if (p.mode == EPI_STORE_BF16) {
       reinterpret_cast<uint16_t*>(p.C)[(size_t)b * p.M * p.ldc + off] = (uint16_t)float_to_bf16_bits(v);
     } else {
-      const float d = v - p.ref[off];
+      const float d = v - (p.ref ? p.ref[off] : 0.f);
       p.S1[off] += d;
       p.S2[off] = fmaf(d, d, p.S2[off]);
     }
@@ -602,21 +605,23 @@ int gemm_run(const GemmArgs& g, cudaStream_t st) {
 
   if (g.mode == EPI_MC) {
     // shifted sums resident in tensor memory over all draws of a tile
-    if (!g.fp8) return BSP_ERR_UNSUPPORTED;
-    if (g.N % 16 != 0 || !g.ref || !g.S1 || !g.S2) return BSP_ERR_ARG;
+    if (g.N % 16 != 0 || !g.S1 || !g.S2) return BSP_ERR_ARG;
     rc = make_operand_map(&mb, g.B, eb, g.K, g.N, g.ldb, g.nb, g.b_batch_stride, MC_BN);
     if (rc != BSP_OK) return rc;
-    p.idesc = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, MC_BN);
-    p.idesc2 = make_idesc(g.a_fmt == BSP_E5M2 ? 1u : 0u, g.b_fmt == BSP_E5M2 ? 1u : 0u, BM, 2 * MC_BN);
-    static std::atomic<bool> mc_attr_set_dev[kMaxDevices];
-    std::atomic<bool>& mc_attr_set = mc_attr_set_dev[device_slot()];
+    const uint32_t fa = g.fp8 ? (g.a_fmt == BSP_E5M2 ? 1u : 0u) : 1u, fb = g.fp8 ? (g.b_fmt == BSP_E5M2 ? 1u : 0u) : 1u;
+    p.idesc = make_idesc(fa, fb, BM, MC_BN);
+    p.idesc2 = make_idesc(fa, fb, BM, 2 * MC_BN);
+    static std::atomic<bool> mc_attr_set_dev[kMaxDevices][2];
+    std::atomic<bool>& mc_attr_set = mc_attr_set_dev[device_slot()][g.fp8 ? 1 : 0];
     if (!mc_attr_set.load(std::memory_order_acquire)) {
-      BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
+      if (g.fp8) BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
+      else BSP_CHECK_CUDA(cudaFuncSetAttribute(gemm_mc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMcSmem));
       mc_attr_set.store(true, std::memory_order_release);
     }
     const int ntiles_mc = (int)(((g.M + BM - 1) / BM) * ((g.N + MC_BN - 1) / MC_BN));
     const int grid_mc = ntiles_mc < nsm ? ntiles_mc : nsm;
-    gemm_mc_kernel<<<grid_mc, kMcThreads, kMcSmem, st>>>(ma, mb, p);
+    if (g.fp8) gemm_mc_kernel<true><<<grid_mc, kMcThreads, kMcSmem, st>>>(ma, mb, p);
+    else gemm_mc_kernel<false><<<grid_mc, kMcThreads, kMcSmem, st>>>(ma, mb, p);
     BSP_LAUNCH_CHECK();
     return BSP_OK;
   }

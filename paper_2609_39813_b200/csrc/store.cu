@@ -166,6 +166,109 @@ __global__ void decode_twice_kernel(const uint8_t* __restrict__ codes, int64_t l
   out[o * 2 * ld_t + ld_t + t] = v;
 }
 
+// The A operand of the K-draw weight-use contraction: dY's codes (token-minor [O][ld_t]) decoded and
+// multiplied by the token's step, rounded to bf16: out[o][t] = bf16(decode(code[o][t]) * s_t).  The
+// contraction it feeds forms *differences* to the reference gradient, so this rounding costs 2^-9 of
+// the difference, not of the gradient.
+template <int FMT>
+__global__ void __launch_bounds__(256)
+store_dys_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ steps, int64_t T, int64_t ld_t, size_t n8,
+                 uint16_t* __restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n8) return;
+  const size_t e0 = i * 8;
+  const int64_t t0 = (int64_t)(e0 % (size_t)ld_t);
+  const uint2 c8 = __ldg(reinterpret_cast<const uint2*>(codes + e0));
+  float d[8];
+  f8_decode4<FMT>(c8.x, *reinterpret_cast<float(*)[4]>(&d[0]));
+  f8_decode4<FMT>(c8.y, *reinterpret_cast<float(*)[4]>(&d[4]));
+  uint32_t pk[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int64_t ta = t0 + 2 * j, tb = ta + 1;
+    const uint32_t lo = ta < T ? float_to_bf16_bits(d[2 * j] * __ldg(steps + ta)) : 0u;
+    const uint32_t hi = tb < T ? float_to_bf16_bits(d[2 * j + 1] * __ldg(steps + tb)) : 0u;
+    pk[j] = lo | (hi << 16);
+  }
+  *reinterpret_cast<uint4*>(out + e0) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+
+// K fresh roundings of the store as differences to the reference's operand, in grid steps, token-minor
+// bf16: out[d][c][t] = n_f - n_q (read N: the new code minus the forward's, a small integer) or
+// n_f - u / s (read U/R+eps: u_q + (u_f - u) - u_q = s (n_f - t), |.| < 1).  An element's grid position
+// is found once; a draw is one generator word and one comparison.  64 x 64 tiles, 256 threads: a thread
+// forms 16 consecutive columns of one token and writes 16 consecutive tokens of one column.
+template <int DT>
+__global__ void __launch_bounds__(256)
+store_diff_draws_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
+                        const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
+                        const int8_t* __restrict__ codes, const float* __restrict__ steps, int read, PhiloxKey key,
+                        int draw0, int ndraws, uint16_t* __restrict__ out_t, int64_t ld_t) {
+  constexpr int TS = 64, PITCH = TS + 2;
+  __shared__ __align__(16) uint16_t s_tile[2][TS][PITCH];
+  const int64_t r0 = (int64_t)blockIdx.y * TS, c0 = (int64_t)blockIdx.x * TS;
+  const int tr = threadIdx.x >> 2, tc = (threadIdx.x & 3) * 16;
+  const int64_t r = r0 + tr, c = c0 + tc;
+  const bool active = r < T && c < C;
+  const size_t i0 = (size_t)r * C + c;
+  float base[16];
+  uint32_t thr[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) { base[j] = 0.f; thr[j] = 0u; }
+  if (active) {
+    const float rs = __ldg(rstd + r), mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+    const float s = __ldg(steps + r);
+    float xv[16];
+    load16<DT>(x, i0, xv);
+    const uint4 cq = read == STORE_READ_N ? __ldg(reinterpret_cast<const uint4*>(codes + i0)) : make_uint4(0, 0, 0, 0);
+    const uint32_t cw[4] = {cq.x, cq.y, cq.z, cq.w};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float u = store_chain(kind, xv[j], rs, mu, __ldg(gamma + c + j), kind == BSP_LAYERNORM ? __ldg(beta + c + j) : 0.f);
+      const float t = __fdiv_rn(u, s);
+      const float n0 = floorf(t);
+      const float f = __fsub_rn(t, n0);
+      thr[j] = __float2uint_rd(f * 4294967296.0f);
+      if (read == STORE_READ_N) base[j] = n0 - (float)(int8_t)((cw[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+      else base[j] = -f;
+    }
+  }
+  const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
+  const int64_t cc = c0 + tcol, rr = r0 + trow;
+  const bool wr = cc < C && rr < ld_t;
+  for (int d = 0; d < ndraws; ++d) {
+    const int buf = d & 1;
+    uint32_t pk[8];
+#pragma unroll
+    for (int b4 = 0; b4 < 4; ++b4) {
+      uint4 w = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+      if (active) w = philox_block(key, ((uint64_t)i0 >> 2) + b4, (uint32_t)(draw0 + d));
+      const float v0 = active ? base[4 * b4 + 0] + (w.x < thr[4 * b4 + 0] ? 1.f : 0.f) : 0.f;
+      const float v1 = active ? base[4 * b4 + 1] + (w.y < thr[4 * b4 + 1] ? 1.f : 0.f) : 0.f;
+      const float v2 = active ? base[4 * b4 + 2] + (w.z < thr[4 * b4 + 2] ? 1.f : 0.f) : 0.f;
+      const float v3 = active ? base[4 * b4 + 3] + (w.w < thr[4 * b4 + 3] ? 1.f : 0.f) : 0.f;
+      pk[2 * b4] = float_to_bf16_bits(v0) | (float_to_bf16_bits(v1) << 16);
+      pk[2 * b4 + 1] = float_to_bf16_bits(v2) | (float_to_bf16_bits(v3) << 16);
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(&s_tile[buf][tr][tc]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) dst[j] = pk[j];
+    __syncthreads();
+    if (wr) {
+      uint32_t o[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t lo = rr + 2 * j < T ? s_tile[buf][trow + 2 * j][tcol] : 0u;
+        const uint32_t hi = rr + 2 * j + 1 < T ? s_tile[buf][trow + 2 * j + 1][tcol] : 0u;
+        o[j] = lo | (hi << 16);
+      }
+      uint4* dstg = reinterpret_cast<uint4*>(out_t + ((size_t)d * C + cc) * ld_t + rr);
+      dstg[0] = make_uint4(o[0], o[1], o[2], o[3]);
+      dstg[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+  }
+}
+
 static bool valid_enum(int v, int hi) { return v >= 0 && v <= hi; }
 
 static int store_levels(int bits) { return (1 << (bits - 1)) - 1; }
@@ -174,7 +277,8 @@ struct StoreBuffers {
   float *rstd, *mean, *amax_u, *steps, *amax_dy, *scale_dy;
   int8_t* codes;
   uint8_t *dy_codes, *dy_codes_t;
-  uint16_t *dy_twice, *x_split;
+  uint16_t *dy_twice, *x_split, *dys_t, *diff_t;
+  int chunk;
   void* du;
   float *dg_ref, *db_ref, *dg_pol, *S1g, *S2g, *dx, *zero_c;
   float *dW_ref, *dW_pol, *S1w, *S2w;
@@ -200,6 +304,17 @@ static size_t store_carve(const bsp_store_desc_t* op, int K, char* base, StoreBu
   c.codes = (int8_t*)take(T * C);
   c.dy_codes = (uint8_t*)take(T * O); c.dy_codes_t = (uint8_t*)take(O * ld_t);
   c.dy_twice = (uint16_t*)take(O * 2 * ld_t * 2); c.x_split = (uint16_t*)take(C * 2 * ld_t * 2);
+  // the K-draw contraction: dY o s once, and the difference operands of as many draws as fit 1 GiB
+  {
+    const size_t per = C * ld_t * 2;
+    size_t fit = ((size_t)1 << 30) / (per ? per : 1);
+    if (fit < 1) fit = 1;
+    const size_t k = K > 0 ? (size_t)K : 1;
+    if (fit >= k) c.chunk = (int)k;
+    else { const size_t nch = (k + fit - 1) / fit; c.chunk = (int)((k + nch - 1) / nch); }
+    c.dys_t = (uint16_t*)take(O * ld_t * 2);
+    c.diff_t = (uint16_t*)take((size_t)c.chunk * per);
+  }
   c.du = take(T * C * eb);
   c.dg_ref = (float*)take(C * 4); c.db_ref = (float*)take(C * 4); c.dg_pol = (float*)take(C * 4);
   c.S1g = (float*)take(C * 4); c.S2g = (float*)take(C * 4); c.zero_c = (float*)take(C * 4);
@@ -388,14 +503,43 @@ int bsp_mc_check_store(const bsp_store_desc_t* op, int K, const bsp_verdict_rule
       // (the statistics pass above reads dW_pol before the draws below overwrite it: same stream)
     }
     if (w_mask & 2u) BSP_TRY(pend.add(b.dW_ref, b.dW_ref, nullptr, O * C, 1, 0, emit(BSP_STREAM_WGRAD, BSP_OUT_DW, BSP_READ_FORWARD)));
+    if (w_mask & 12u) {
+      const size_t n8 = (size_t)O * b.ld_t / 8;
+      if (op->grad_fmt == BSP_E5M2)
+        store_dys_kernel<BSP_E5M2><<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(b.dy_codes_t, b.steps, T, b.ld_t, n8, b.dys_t);
+      else
+        store_dys_kernel<BSP_E4M3><<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>(b.dy_codes_t, b.steps, T, b.ld_t, n8, b.dys_t);
+      BSP_LAUNCH_CHECK();
+    }
     for (int which = 0; which < 2; ++which) {
       if (!((w_mask >> (2 + which)) & 1u)) continue;
+      // Both fresh reads differ from the reference's operand u_q = s n_q by a multiple of the token's
+      // step: s (n_f - n_q) under N, s (n_f - u / s) under U/R+eps.  So the K draws are one contraction
+      // of (dY o s) with the K difference matrices, whose products are g_k - g* themselves: the shifted
+      // sums take them as they come, no per-draw gradient is written, and the bf16 rounding of an
+      // operand costs 2^-9 of the difference.
       const int read = which == 0 ? STORE_READ_N : STORE_READ_R_EPS;
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S1w, 0, (size_t)O * C * sizeof(float), st));
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S2w, 0, (size_t)O * C * sizeof(float), st));
-      for (int k = 0; k < K; ++k) {
-        BSP_TRY(wgrad(read, k, b.dW_pol));
-        BSP_TRY(bsp_mc_accumulate(b.dW_pol, b.dW_ref, b.S1w, b.S2w, (size_t)O * C, st));
+      bsp_key_t wk = key;
+      wk.stream = BSP_STREAM_WGRAD; wk.draw = 0;
+      const PhiloxKey pk = make_key(wk);
+      for (int k0 = 0; k0 < K; k0 += b.chunk) {
+        const int nd = (K - k0) < b.chunk ? (K - k0) : b.chunk;
+        dim3 grid((unsigned)((C + 63) / 64), (unsigned)((b.ld_t + 63) / 64));
+        if (dt == BSP_F32)
+          store_diff_draws_kernel<BSP_F32><<<grid, 256, 0, st>>>(kind, op->x, T, C, op->gamma, op->beta, b.rstd, b.mean, b.codes,
+                                                                 b.steps, read, pk, k0, nd, b.diff_t, b.ld_t);
+        else
+          store_diff_draws_kernel<BSP_BF16><<<grid, 256, 0, st>>>(kind, op->x, T, C, op->gamma, op->beta, b.rstd, b.mean, b.codes,
+                                                                  b.steps, read, pk, k0, nd, b.diff_t, b.ld_t);
+        BSP_LAUNCH_CHECK();
+        GemmArgs g;
+        g.M = O; g.N = C; g.K = T; g.nb = nd; g.fp8 = false;
+        g.A = b.dys_t; g.B = b.diff_t; g.lda = b.ld_t; g.ldb = b.ld_t; g.b_batch_stride = (int64_t)C * b.ld_t;
+        g.sa = 1.f; g.sa_dev = b.scale_dy; g.sb = 1.f; g.sb_dev = nullptr;
+        g.mode = EPI_MC; g.ldc = C; g.ref = nullptr; g.S1 = b.S1w; g.S2 = b.S2w; g.diag = diag;
+        BSP_TRY(gemm_run(g, st));
       }
       BSP_TRY(pend.add(b.dW_ref, b.S1w, b.S2w, O * C, K, 1,
                        emit(BSP_STREAM_WGRAD, BSP_OUT_DW, which == 0 ? BSP_READ_FRESH : BSP_READ_FORWARD_PLUS_FRESH_ERROR)));
