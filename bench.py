@@ -433,6 +433,15 @@ def widened_section(b, torch):
                              entry_trials_per_s=rows * classes * trials / (ms * 1e-3),
                              mean_error_reuse=st[0].mean, predicted=float(np.cosh(eps) - 1),
                              coupling=st[2].mean, predicted_coupling=float(-eps * np.sinh(eps)))
+    # the same operator at a vocabulary-sized row (the generator's rate shows only on a large case)
+    rows, classes, trials = 256, 8192, 256
+    logits = torch.from_numpy(rng.standard_normal((rows, classes)).astype(np.float32)).cuda()
+    target = torch.from_numpy(rng.integers(0, classes, rows).astype(np.int32)).cuda()
+    ws = b.workspace(b.bsp_lsm_check_workspace_bytes(rows, classes, trials))
+    ms = timed(torch, stream, lambda: b.bsp_lsm_check(logits, target, rows, classes, eps, trials, 1926, 3, None, ws),
+               reps=3, warm=1)
+    out["logsoftmax_large"] = dict(workload="%d x %d, eps %.2f, %d trials" % (rows, classes, eps, trials), ms=ms,
+                                   entry_trials_per_s=rows * classes * trials / (ms * 1e-3))
     out["diag_status"] = b.read_diag(diag)["status"]
     return out
 

@@ -73,20 +73,24 @@ __global__ void cp_weight_kernel(const void* __restrict__ W, int64_t O, int64_t 
 }
 
 // out[c] += sum_t w[t][c] * du[t][c] / gamma[c], w = r (given) or the residual of `codes` (a fresh
-// rounding, formed on the fly); and sum_du += du when given.  One block per 32 columns walks all
-// rows (eight rows at a time), so every output has one writer and a fixed order of additions.
+// rounding, formed on the fly); and sum_du += du when given.  Block (x, y) walks the y-th slab of rows
+// for 32 columns (eight rows at a time) and writes one partial per column; cp_gain_final_kernel adds
+// the slabs in order, so every output has one writer and a fixed order of additions.
+constexpr int kCpSlabs = 64;
 template <int FMT>
 __global__ void __launch_bounds__(256)
 cp_gain_kernel(const float* __restrict__ r, const uint8_t* __restrict__ codes, const float* __restrict__ scale_dev,
-               const float* __restrict__ u, const float* __restrict__ du, const float* __restrict__ gamma, int64_t T,
-               int64_t C, float* __restrict__ out, float* __restrict__ sum_du) {
+               const float* __restrict__ u, const float* __restrict__ du, int64_t T, int64_t C, int64_t slab_rows,
+               float* __restrict__ partial /* [gridDim.y][C] */, float* __restrict__ sum_du) {
   __shared__ float sm[8][33];
   const int cl = threadIdx.x & 31, rl = threadIdx.x >> 5;
   const int64_t c = (int64_t)blockIdx.x * 32 + cl;
   const float inv = codes ? __fdiv_rn(1.0f, __ldg(scale_dev)) : 0.f;
+  const int64_t t_begin = (int64_t)blockIdx.y * slab_rows;
+  const int64_t t_end = t_begin + slab_rows < T ? t_begin + slab_rows : T;
   float s = 0.f;
   if (c < C) {
-    for (int64_t t = rl; t < T; t += 8) {
+    for (int64_t t = t_begin + rl; t < t_end; t += 8) {
       const size_t i = (size_t)t * C + c;
       const float d = du[i];
       const float w = codes ? f8_decode<FMT>(codes[i]) * inv - u[i] : r[i];
@@ -100,8 +104,18 @@ cp_gain_kernel(const float* __restrict__ r, const uint8_t* __restrict__ codes, c
     float t = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) t += sm[w][cl];
-    out[c] += t / gamma[c];
+    partial[(size_t)blockIdx.y * C + c] = t;
   }
+}
+
+__global__ void __launch_bounds__(256)
+cp_gain_final_kernel(const float* __restrict__ partial, int nslabs, const float* __restrict__ gamma, int64_t C,
+                     float* __restrict__ out) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  float t = 0.f;
+  for (int y = 0; y < nslabs; ++y) t += partial[(size_t)y * C + c];
+  out[c] += t / gamma[c];
 }
 
 // partial[b] = { sum (ra - rb)(dua - dub), sum dua * rb } over the block's grid-stride share, in double.
@@ -203,7 +217,7 @@ struct CouplingBuffers {
   uint8_t* codes_f;
   uint16_t *uq, *Wb, *Wt2, *ysplit, *dr_t, *dy_t;
   float *r[2], *y[2], *du[2], *sum_r, *sum_du, *xk;
-  float *gain_total, *gain_mean_part, *gain_fresh, *X, *X_sq;
+  float *gain_total, *gain_mean_part, *gain_fresh, *X, *X_sq, *gain_partial;
   double *dot_partial, *dots;
   int64_t ld_t;
 };
@@ -230,6 +244,7 @@ static size_t coupling_carve(const bsp_coupling_desc_t* op, int pairs, char* bas
   c.X = (float*)take(C * O * 4); c.X_sq = (float*)take(C * O * 4);
   c.dot_partial = (double*)take(kCpDotBlocks * 2 * sizeof(double));
   c.dots = (double*)take((size_t)(pairs > 0 ? pairs : 1) * 2 * sizeof(double));
+  c.gain_partial = (float*)take((size_t)kCpSlabs * C * 4);
   if (out) *out = c;
   return off;
 }
@@ -296,6 +311,9 @@ int bsp_coupling_check(const bsp_coupling_desc_t* op, int pairs, double* T_out, 
   bsp_key_t key;
   key.seed = op->seed; key.tensor_id = op->tensor_id; key.reserved = 0;
   const unsigned g4 = (unsigned)((n / 4 + 255) / 256), gcol = (unsigned)((C + 31) / 32);
+  const int64_t slab_rows = ((T + kCpSlabs - 1) / kCpSlabs + 7) & ~(int64_t)7;
+  const int nslabs = (int)((T + slab_rows - 1) / slab_rows);
+  const dim3 ggain(gcol, (unsigned)nslabs);
 
   auto forward = [&](int draw, int slot) -> int {
     key.stream = BSP_STREAM_FORWARD; key.draw = (uint32_t)draw;
@@ -319,14 +337,16 @@ int bsp_coupling_check(const bsp_coupling_desc_t* op, int pairs, double* T_out, 
     h.sa = 1.f; h.sb = 1.f; h.mode = EPI_STORE_F32; h.C = b.du[slot]; h.ldc = C; h.diag = diag;
     BSP_TRY(gemm_run(h, st));
     // gain-use errors: read R (this forward's own error) and a fresh read (stream 1, same draw)
-    if (fmt == BSP_E4M3) cp_gain_kernel<BSP_E4M3><<<gcol, 256, 0, st>>>(b.r[slot], nullptr, b.scale, b.u, b.du[slot], op->gamma, T, C, b.gain_total, b.sum_du);
-    else cp_gain_kernel<BSP_E5M2><<<gcol, 256, 0, st>>>(b.r[slot], nullptr, b.scale, b.u, b.du[slot], op->gamma, T, C, b.gain_total, b.sum_du);
+    if (fmt == BSP_E4M3) cp_gain_kernel<BSP_E4M3><<<ggain, 256, 0, st>>>(b.r[slot], nullptr, b.scale, b.u, b.du[slot], T, C, slab_rows, b.gain_partial, b.sum_du);
+    else cp_gain_kernel<BSP_E5M2><<<ggain, 256, 0, st>>>(b.r[slot], nullptr, b.scale, b.u, b.du[slot], T, C, slab_rows, b.gain_partial, b.sum_du);
+    cp_gain_final_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(b.gain_partial, nslabs, op->gamma, C, b.gain_total);
     BSP_LAUNCH_CHECK();
     key.stream = BSP_STREAM_GAIN;
     BSP_TRY(bsp_norm_fwd(kind, op->x, dt, T, C, op->gamma, op->beta, b.rstd, b.mean, qf, key, b.codes_f, nullptr, 0, nullptr,
                          nullptr, diag, st));
-    if (fmt == BSP_E4M3) cp_gain_kernel<BSP_E4M3><<<gcol, 256, 0, st>>>(nullptr, b.codes_f, b.scale, b.u, b.du[slot], op->gamma, T, C, b.gain_fresh, nullptr);
-    else cp_gain_kernel<BSP_E5M2><<<gcol, 256, 0, st>>>(nullptr, b.codes_f, b.scale, b.u, b.du[slot], op->gamma, T, C, b.gain_fresh, nullptr);
+    if (fmt == BSP_E4M3) cp_gain_kernel<BSP_E4M3><<<ggain, 256, 0, st>>>(nullptr, b.codes_f, b.scale, b.u, b.du[slot], T, C, slab_rows, b.gain_partial, nullptr);
+    else cp_gain_kernel<BSP_E5M2><<<ggain, 256, 0, st>>>(nullptr, b.codes_f, b.scale, b.u, b.du[slot], T, C, slab_rows, b.gain_partial, nullptr);
+    cp_gain_final_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(b.gain_partial, nslabs, op->gamma, C, b.gain_fresh);
     BSP_LAUNCH_CHECK();
     return BSP_OK;
   };

@@ -122,19 +122,34 @@ lsm_trial_kernel(const float* __restrict__ l, const float* __restrict__ p, const
 }
 
 // Column c < 6: the statistic itself; 6 and 7: the paired contrasts reuse - independent (likelihood,
-// constructed).  out[c] = {sum, sum of squares} over trials, in double, in trial order.
-__global__ void lsm_reduce_kernel(const float* __restrict__ per_trial, int trials, double* __restrict__ out) {
-  const int c = threadIdx.x;
-  if (c >= kLsmCols) return;
-  double s1 = 0.0, s2 = 0.0;
-  for (int t = 0; t < trials; ++t) {
+// constructed).  out[2c], out[2c + 1] = sum and sum of squares over trials, in double.
+__global__ void __launch_bounds__(256)
+lsm_reduce_kernel(const float* __restrict__ per_trial, int trials, double* __restrict__ out) {
+  // thread t sums the trials t, t + 256, ... of every column; the 256 partial sums are then added
+  // pairwise in a fixed tree, so the result does not depend on scheduling
+  __shared__ double sh[2 * kLsmCols][256];
+  double s1[kLsmCols], s2[kLsmCols];
+#pragma unroll
+  for (int c = 0; c < kLsmCols; ++c) s1[c] = s2[c] = 0.0;
+  for (int t = threadIdx.x; t < trials; t += 256) {
     const float* v = per_trial + (size_t)t * kLsmStats;
-    const double x = c < kLsmStats ? (double)v[c] : (c == 6 ? (double)v[0] - (double)v[1] : (double)v[2] - (double)v[3]);
-    s1 += x;
-    s2 += x * x;
+    double x[kLsmCols];
+#pragma unroll
+    for (int c = 0; c < kLsmStats; ++c) x[c] = (double)v[c];
+    x[6] = x[0] - x[1];
+    x[7] = x[2] - x[3];
+#pragma unroll
+    for (int c = 0; c < kLsmCols; ++c) { s1[c] += x[c]; s2[c] += x[c] * x[c]; }
   }
-  out[2 * c] = s1;
-  out[2 * c + 1] = s2;
+#pragma unroll
+  for (int c = 0; c < kLsmCols; ++c) { sh[2 * c][threadIdx.x] = s1[c]; sh[2 * c + 1][threadIdx.x] = s2[c]; }
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if ((int)threadIdx.x < o)
+      for (int c = 0; c < 2 * kLsmCols; ++c) sh[c][threadIdx.x] += sh[c][threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x < 2 * kLsmCols) out[threadIdx.x] = sh[threadIdx.x][0];
 }
 
 }  // namespace bsp
@@ -174,7 +189,7 @@ int bsp_lsm_check(const float* logits, const int32_t* target, int rows, int clas
   BSP_LAUNCH_CHECK();
   lsm_trial_kernel<<<(unsigned)trials, kLsmThreads, 0, st>>>(l, p, target, rows, classes, eps, kr, kc, pt);
   BSP_LAUNCH_CHECK();
-  lsm_reduce_kernel<<<1, 32, 0, st>>>(pt, trials, sums);
+  lsm_reduce_kernel<<<1, 256, 0, st>>>(pt, trials, sums);
   BSP_LAUNCH_CHECK();
   double host[2 * kLsmCols];
   BSP_CHECK_CUDA(cudaMemcpyAsync(host, sums, sizeof(host), cudaMemcpyDeviceToHost, st));
