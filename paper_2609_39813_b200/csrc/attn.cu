@@ -155,7 +155,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     nsteps = it_end - it_begin;
   };
-  constexpr int npass = MODE == AT_FWD ? 2 : 1;
+  // FWD with the rows' log-sum-exp already known (p.lse): one pass, P = exp(s - LSE) directly
+  const bool one_pass = MODE == AT_FWD && p.lse != nullptr;
+  const int npass = (MODE == AT_FWD && !one_pass) ? 2 : 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -284,14 +286,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       };
       if (ok && total > 0) ok = issue_sdp(itg);
       for (int it = 0; it < total && ok; ++it) {
-        const bool pass2 = it >= nsteps;                      // FWD only
+        const bool pass2 = one_pass || it >= nsteps;          // FWD only
         const uint32_t jg = itg + (uint32_t)it;
         const uint32_t s = jg % kStg, ip = jg & 1u;
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
         if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t first = (MODE == AT_FWD ? it == nsteps : it == 0) ? 0u : 1u;   // overwrite on the first product
+        const uint32_t first = (MODE == AT_FWD ? it == (one_pass ? 0 : nsteps) : it == 0) ? 0u : 1u;   // overwrite on the first product
         if (!kAccDouble && it == 0 && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
         if (MODE == AT_DKV) {
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
@@ -452,10 +454,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
         if (ND == 2) dq2 = __ldg(p.dterm + (size_t)p.BH * p.S + (size_t)bh * p.S + qrow);
       }
+      if (MODE == AT_FWD && one_pass && qrow < p.S) lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
     }
     float run_m = -INFINITY, run_l = 0.f;                     // FWD pass 1: running max and sum (this half)
     for (int it = 0; it < total && ok; ++it) {
-      const bool pass2 = it >= nsteps;
+      const bool pass2 = one_pass || it >= nsteps;
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
@@ -723,7 +726,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       named_bar_sync(1, 256);
       const float l = xm[256 + r] + xm[384 + r];
       fwd_inv_l = __fdividef(1.0f, l);
-      if (h == 0 && qrow < p.S) p.lse_out[(size_t)bh * p.S + qrow] = (lse2 + log2f(l)) / kLog2e;
+      if (h == 0 && qrow < p.S && p.lse_out) p.lse_out[(size_t)bh * p.S + qrow] = (lse2 + log2f(l)) / kLog2e;
     }
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise), 32 KB at a
     // time through the item's resident-tile buffer (no product reads it any more): every thread puts
@@ -1023,14 +1026,14 @@ static int set_fp8(AttnParams& p, const bsp_attn_fp8_t* f) {
 
 int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
                          const void* v, int dt, const bsp_attn_fp8_t* f, float* o, float* lse, bsp_diag_t* diag,
-                         void* stream) {
+                         void* stream, const float* lse_known) {
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
-  if (!q || !k || !v || !o || !lse) return BSP_ERR_ARG;
+  if (!q || !k || !v || !o || (!lse && !lse_known)) return BSP_ERR_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
   AttnParams p;
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
-  p.lse = nullptr; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
+  p.lse = lse_known; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
   return launch_attn<AT_FWD>(q, k, v, nullptr, p, (cudaStream_t)stream);
 }

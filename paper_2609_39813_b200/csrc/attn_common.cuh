@@ -92,7 +92,8 @@ inline int sm_count_or_default() {
 // Internal entry points of attn.cu used by the per-use check (attn_mc.cu).  `f` = NULL: BF16-operand
 // mode; otherwise the FP8-operand mode with the operands holding decoded codes.
 int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
-                  const void* v, int dt, const bsp_attn_fp8_t* f, float* o, float* lse, bsp_diag_t* diag, void* stream);
+                  const void* v, int dt, const bsp_attn_fp8_t* f, float* o, float* lse, bsp_diag_t* diag, void* stream,
+                  const float* lse_known = nullptr);   // rows' LSE given: one pass over the keys, `lse` may be NULL
 int attn_dterm_impl(int B, int H, int S, int Dh, const void* dO, int dt, const float* do_scales, const float* o_orig,
                     const uint8_t* o_codes, const float* o_scales, int o_fmt, int d_read, bsp_key_t key, int draw0,
                     int n_draws, float* d_out, void* stream);

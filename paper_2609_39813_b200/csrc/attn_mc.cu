@@ -663,9 +663,9 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, const bsp_verdict_rule_t
       BSP_CHECK_CUDA(cudaMemsetAsync(b.S2[t], 0, n * 4, st));
     }
     if (!fp8) {
-      // dQ: P K once (the forward kernel with K in place of V; g_pol[0] is free by now, the LSE it
-      // recomputes goes to d_pol), then the K draws collapse to one elementwise pass
-      BSP_TRY(attn_fwd_impl(B, H, S, Dh, op->causal, c, q, k, k, dt, nullptr, b.g_pol[0], b.d_pol, diag, st));
+      // dQ: P K once (the forward kernel with K in place of V and the rows' LSE given, so it takes one
+      // pass over the keys; g_pol[0] is free by now), then the K draws collapse to one elementwise pass
+      BSP_TRY(attn_fwd_impl(B, H, S, Dh, op->causal, c, q, k, k, dt, nullptr, b.g_pol[0], nullptr, diag, st, b.lse));
       attn_dq_sums_kernel<<<(unsigned)((n / 4 + 255) / 256), 256, 0, st>>>(b.g_pol[0], b.S1d, b.S2d, c, b.S1[0], b.S2[0],
                                                                           n / 4);
       BSP_LAUNCH_CHECK();
