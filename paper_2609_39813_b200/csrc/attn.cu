@@ -522,6 +522,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
         // first rounds P onto the E4M3 grid at p_scale and dS onto the E5M2 grid at ds_scale (the
         // grid values are exact in bf16; the scales come back in the epilogue).
+        // a pair of dS values as a packed bf16 operand (FP8-operand mode: on the E5M2 grid at ds_scale)
+        auto pack_ds = [&](float s0, float s1) -> uint32_t {
+          if (FP8) return f8_grid_bf16x2<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);
+          return pack_bf16x2(s0, s1);
+        };
         auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, float d0, float d1, uint32_t& po,
                              uint32_t& dso) {
           float s0 = 0.f, s1 = 0.f;
@@ -590,8 +595,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             }
             const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
             const float x0 = __uint_as_float(dv[j]) * dp_mul, x1 = __uint_as_float(dv[j + 1]) * dp_mul;
-            da[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 - dq), p1 * (x1 - dq));
-            db[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 - dq2), p1 * (x1 - dq2));
+            da[(j & 31) >> 1] = pack_ds(p0 * (x0 - dq), p1 * (x1 - dq));
+            db[(j & 31) >> 1] = pack_ds(p0 * (x0 - dq2), p1 * (x1 - dq2));
           };
           if (!edge) {
 #pragma unroll
@@ -645,8 +650,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             float e0, e1;
             asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(e0), "=f"(e1) : "r"(dbase + (uint32_t)j * 4u));
             const float x0 = __uint_as_float(dv[j]) * dp_mul, x1 = __uint_as_float(dv[j + 1]) * dp_mul;
-            da[(j & 31) >> 1] = pack_bf16x2(p0 * x0, p1 * x1);
-            db[(j & 31) >> 1] = pack_bf16x2(p0 * (x0 + e0), p1 * (x1 + e1));
+            da[(j & 31) >> 1] = pack_ds(p0 * x0, p1 * x1);
+            db[(j & 31) >> 1] = pack_ds(p0 * (x0 + e0), p1 * (x1 + e1));
           };
           if (!edge) {
 #pragma unroll
@@ -1000,8 +1005,8 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
 template <int MODE>
 static int launch_attn(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
   if (MODE != AT_FWD && p.mc_ref != nullptr) {               // Monte-Carlo epilogue: BF16 operands, no dV
-    if (p.fp8) {                                             // FP8-operand mode: one draw per launch
-      if (p.nd != 1) return BSP_ERR_UNSUPPORTED;
+    if (p.fp8) {
+      if (p.nd == 2) return launch_attn_mode<MODE, true, MODE != AT_DKV, MODE != AT_FWD, MODE != AT_FWD ? 2 : 1>(q, k, v, dO, p, st);
       return launch_attn_mode<MODE, true, MODE != AT_DKV, MODE != AT_FWD>(q, k, v, dO, p, st);
     }
     if (p.nd == 2) return launch_attn_mode<MODE, false, MODE != AT_DKV, MODE != AT_FWD, MODE != AT_FWD ? 2 : 1>(q, k, v, dO, p, st);
@@ -1138,7 +1143,7 @@ int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_sca
   int rc = check_attn_shape(B, H, S, Dh, dt);
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !dO || !lse || !dterm || !ref_dq || !S1q || !S2q || !ref_dk || !S1k || !S2k) return BSP_ERR_ARG;
-  if (nd < 1 || nd > 2 || (f && nd != 1)) return BSP_ERR_ARG;
+  if (nd < 1 || nd > 2) return BSP_ERR_ARG;
   if (!aligned16(ref_dq) || !aligned16(ref_dk) || !aligned16(S1q) || !aligned16(S2q) || !aligned16(S1k) || !aligned16(S2k))
     return BSP_ERR_ALIGN;
   AttnParams p;

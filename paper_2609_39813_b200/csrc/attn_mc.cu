@@ -677,9 +677,10 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, const bsp_verdict_rule_t
       }
     } else {
       // the rounded backward once per draw; dQ and dK go from the accumulators straight into their sums
-      for (int k0 = 0; k0 < K; ++k0)
+      // (two draws per launch: the scores, dP and the exponentials are formed once for both)
+      for (int k0 = 0; k0 < K; k0 += 2)
         BSP_TRY(attn_bwd_dterm_mc(B, H, S, Dh, op->causal, c, q, k, v, dO, dt, f, b.lse, b.d_draws + (size_t)k0 * rows,
-                                  1, b.g_ref[0], b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
+                                  K - k0 >= 2 ? 2 : 1, b.g_ref[0], b.S1[0], b.S2[0], b.g_ref[1], b.S1[1], b.S2[1], diag, st));
     }
     BSP_TRY(pend.add(b.d_ref, b.S1d, b.S2d, (int64_t)rows, K, 1, emit(out_ids[0], BSP_READ_FRESH)));
     for (int t = 0; t < 2; ++t)
