@@ -554,7 +554,8 @@ int bsp_store_fwd(int kind, const void* x, int dt, int64_t T, int64_t C, const f
  * BSP_READ_FRESH (a new rounding under `key`) or BSP_READ_FORWARD_PLUS_FRESH_ERROR.  Outputs, each
  * may be NULL: copy_f32[T*C], and copy_split_t[C][2*ld_t] bf16, the operand of bsp_store_wgrad:
  * the copy split into two bf16 terms hi + lo (16 significant bits), token-minor, hi in columns
- * [0, ld_t), lo in [ld_t, 2 ld_t); ld_t >= T, a multiple of 16, padding zeroed. */
+ * [0, ld_t), lo in [ld_t, 2 ld_t); ld_t >= T, a multiple of 16, padding zeroed.
+ * C a multiple of 16 (BSP_ERR_UNSUPPORTED otherwise); x, codes and the outputs 16-byte aligned. */
 int bsp_store_read(int kind, const void* x, int dt, int64_t T, int64_t C, const float* gamma,
                    const float* beta, const float* rstd, const float* mean, const int8_t* codes,
                    const float* steps, int read, bsp_key_t key, float* copy_f32, void* copy_split_t,

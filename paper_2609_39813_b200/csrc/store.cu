@@ -103,54 +103,88 @@ store_fwd_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, con
   }
 }
 
-// The copy X a weight use reads, for a 32 x 32 tile of (tokens x columns): FP32 out (row-major, may be
+// The copy X a weight use reads, for a 64 x 64 tile of (tokens x columns): FP32 out (row-major, may be
 // NULL) and the split bf16 operand out_t[c][t] = hi, out_t[c][ld_t + t] = lo (may be NULL), padding
-// columns t in [T, ld_t) zeroed.
+// columns t in [T, ld_t) zeroed.  A thread forms 16 consecutive columns of one token (four generator
+// blocks, no word wasted) and writes 16 consecutive tokens of one column of each half.
 template <int DT>
 __global__ void __launch_bounds__(256)
 store_operand_kernel(int kind, const void* __restrict__ x, int64_t T, int64_t C, const float* __restrict__ gamma,
                      const float* __restrict__ beta, const float* __restrict__ rstd, const float* __restrict__ mean,
                      const int8_t* __restrict__ codes, const float* __restrict__ steps, int read, PhiloxKey key,
                      float* __restrict__ out_f32, uint16_t* __restrict__ out_t, int64_t ld_t) {
-  __shared__ float tile[32][33];
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;
-  for (int i = ty; i < 32; i += 8) {
-    const int64_t r = r0 + i, c = c0 + tx;
-    float v = 0.f;
-    if (r < T && c < C) {
-      const size_t i0 = (size_t)r * C + c;
-      const float rs = __ldg(rstd + r), mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
-      const float u = store_chain(kind, load1<DT>(x, i0), rs, mu, __ldg(gamma + c), kind == BSP_LAYERNORM ? __ldg(beta + c) : 0.f);
-      const float s = __ldg(steps + r);
-      float nf = 0.f;
-      if (read == STORE_READ_N || read == STORE_READ_R_EPS) {
-        const uint4 w = philox_block(key, (uint64_t)i0 >> 2, key.c2);
-        float n0;
-        uint32_t P;
-        grid_position(u, s, n0, P);
-        nf = n0 + (word_of(w, (uint32_t)(i0 & 3)) < P ? 1.f : 0.f);
+  constexpr int TS = 64, PITCH = TS + 2;
+  __shared__ __align__(16) uint16_t s_hi[TS][PITCH], s_lo[TS][PITCH];
+  const int64_t r0 = (int64_t)blockIdx.y * TS, c0 = (int64_t)blockIdx.x * TS;
+  const int tr = threadIdx.x >> 2, tc = (threadIdx.x & 3) * 16;
+  const int64_t r = r0 + tr, c = c0 + tc;
+  float v[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] = 0.f;
+  if (r < T && c < C) {
+    const size_t i0 = (size_t)r * C + c;
+    const float rs = __ldg(rstd + r), mu = kind == BSP_LAYERNORM ? __ldg(mean + r) : 0.f;
+    const float s = __ldg(steps + r);
+    float xv[16];
+    load16<DT>(x, i0, xv);
+    const bool fresh = read == STORE_READ_N || read == STORE_READ_R_EPS;
+    const bool fwd = read == STORE_READ_R || read == STORE_READ_R_EPS;
+    const uint4 cq = fwd ? __ldg(reinterpret_cast<const uint4*>(codes + i0)) : make_uint4(0, 0, 0, 0);
+    const uint32_t cw[4] = {cq.x, cq.y, cq.z, cq.w};
+#pragma unroll
+    for (int b4 = 0; b4 < 4; ++b4) {
+      uint4 w = make_uint4(0, 0, 0, 0);
+      if (fresh) w = philox_block(key, ((uint64_t)i0 >> 2) + b4, key.c2);
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int j = 4 * b4 + e;
+        const float u = store_chain(kind, xv[j], rs, mu, __ldg(gamma + c + j), kind == BSP_LAYERNORM ? __ldg(beta + c + j) : 0.f);
+        float nf = 0.f;
+        if (fresh) {
+          float n0;
+          uint32_t P;
+          grid_position(u, s, n0, P);
+          nf = n0 + (ww[e] < P ? 1.f : 0.f);
+        }
+        const float nq = fwd ? (float)(int8_t)((cw[b4] >> (8 * e)) & 0xFFu) : 0.f;
+        if (read == STORE_READ_U) v[j] = u;
+        else if (read == STORE_READ_R) v[j] = __fmul_rn(s, nq);
+        else if (read == STORE_READ_N) v[j] = __fmul_rn(s, nf);
+        else v[j] = __fsub_rn(__fmul_rn(s, nq + nf), u);            // u_q + (u_f - u) = s (n + n_f) - u
       }
-      const float nq = (read == STORE_READ_R || read == STORE_READ_R_EPS) ? (float)codes[i0] : 0.f;
-      if (read == STORE_READ_U) v = u;
-      else if (read == STORE_READ_R) v = __fmul_rn(s, nq);
-      else if (read == STORE_READ_N) v = __fmul_rn(s, nf);
-      else v = __fsub_rn(__fmul_rn(s, nq + nf), u);              // u_q + (u_f - u) = s (n + n_f) - u
-      if (out_f32) out_f32[i0] = v;
     }
-    tile[i][tx] = v;
+    if (out_f32) {
+#pragma unroll
+      for (int j = 0; j < 16; j += 4)
+        *reinterpret_cast<float4*>(out_f32 + i0 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+    }
   }
   if (!out_t) return;
+  uint32_t* dh = reinterpret_cast<uint32_t*>(&s_hi[tr][tc]);
+  uint32_t* dl = reinterpret_cast<uint32_t*>(&s_lo[tr][tc]);
+#pragma unroll
+  for (int j = 0; j < 16; j += 2) {
+    const uint32_t h0 = float_to_bf16_bits(v[j]), h1 = float_to_bf16_bits(v[j + 1]);
+    const uint32_t l0 = float_to_bf16_bits(v[j] - bf16_bits_to_float(h0)), l1 = float_to_bf16_bits(v[j + 1] - bf16_bits_to_float(h1));
+    dh[j >> 1] = h0 | (h1 << 16);
+    dl[j >> 1] = l0 | (l1 << 16);
+  }
   __syncthreads();
-  for (int i = ty; i < 32; i += 8) {
-    const int64_t c = c0 + i, r = r0 + tx;
-    if (c < C && r < ld_t) {
-      const float v = r < T ? tile[tx][i] : 0.f;
-      const uint32_t hi = float_to_bf16_bits(v);
-      const uint32_t lo = float_to_bf16_bits(v - bf16_bits_to_float(hi));
-      out_t[(size_t)c * (2 * ld_t) + r] = (uint16_t)hi;
-      out_t[(size_t)c * (2 * ld_t) + ld_t + r] = (uint16_t)lo;
+  const int tcol = threadIdx.x >> 2, trow = (threadIdx.x & 3) * 16;
+  const int64_t cc = c0 + tcol, rr = r0 + trow;
+  if (cc < C && rr < ld_t) {
+    uint32_t oh[8], ol[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const bool a = rr + 2 * j < T, b = rr + 2 * j + 1 < T;
+      oh[j] = (a ? (uint32_t)s_hi[trow + 2 * j][tcol] : 0u) | ((b ? (uint32_t)s_hi[trow + 2 * j + 1][tcol] : 0u) << 16);
+      ol[j] = (a ? (uint32_t)s_lo[trow + 2 * j][tcol] : 0u) | ((b ? (uint32_t)s_lo[trow + 2 * j + 1][tcol] : 0u) << 16);
     }
+    uint4* ph = reinterpret_cast<uint4*>(out_t + (size_t)cc * (2 * ld_t) + rr);
+    uint4* pl = reinterpret_cast<uint4*>(out_t + (size_t)cc * (2 * ld_t) + ld_t + rr);
+    ph[0] = make_uint4(oh[0], oh[1], oh[2], oh[3]); ph[1] = make_uint4(oh[4], oh[5], oh[6], oh[7]);
+    pl[0] = make_uint4(ol[0], ol[1], ol[2], ol[3]); pl[1] = make_uint4(ol[4], ol[5], ol[6], ol[7]);
   }
 }
 
@@ -364,10 +398,12 @@ int bsp_store_read(int kind, const void* x, int dt, int64_t T, int64_t C, const 
   if (!x || !gamma || !rstd || !steps || (kind == BSP_LAYERNORM && (!beta || !mean))) return BSP_ERR_ARG;
   if ((read == STORE_READ_R || read == STORE_READ_R_EPS) && !codes) return BSP_ERR_ARG;
   if (copy_split_t && (ld_t < T || ld_t % 16 != 0)) return BSP_ERR_ALIGN;
+  if (C % 16 != 0) return BSP_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(copy_f32) || !aligned16(copy_split_t)) return BSP_ERR_ALIGN;
   const PhiloxKey pk = make_key(key);
   cudaStream_t st = (cudaStream_t)stream;
   const int64_t rows = copy_split_t ? ld_t : T;                 // the padding columns are written too
-  dim3 grid((unsigned)((C + 31) / 32), (unsigned)((rows + 31) / 32));
+  dim3 grid((unsigned)((C + 63) / 64), (unsigned)((rows + 63) / 64));
   if (dt == BSP_F32)
     store_operand_kernel<BSP_F32><<<grid, 256, 0, st>>>(kind, x, T, C, gamma, beta, rstd, mean, codes, steps, read, pk, copy_f32,
                                                         reinterpret_cast<uint16_t*>(copy_split_t), ld_t);
