@@ -509,14 +509,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                         qb0 + AT_BLK > p.S;
       if (MODE == AT_FWD && !pass2) {
         // running max of c2 * s over the valid keys of this half
-        float mloc = run_m;
+        // (four independent chains; the validity test only where a block needs it, and as a select)
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+        if (!edge && c2 > 0.f) {
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
-          const int key = key0 + j;
-          const bool valid = !edge || (key < p.S && qrow < p.S && (!p.causal || key <= qrow));
-          if (valid) mloc = fmaxf(mloc, __uint_as_float(sv[j]) * c2);
+          for (int j = 0; j < 64; j += 4) {
+            m0 = fmaxf(m0, __uint_as_float(sv[j]));
+            m1 = fmaxf(m1, __uint_as_float(sv[j + 1]));
+            m2 = fmaxf(m2, __uint_as_float(sv[j + 2]));
+            m3 = fmaxf(m3, __uint_as_float(sv[j + 3]));
+          }
+          run_m = fmaxf(run_m, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2);   // c2 > 0: the maximum commutes with the scaling
+        } else {
+          const bool row_ok = qrow < p.S;
+          const int last = p.causal ? (qrow < p.S - 1 ? qrow : p.S - 1) : p.S - 1;   // last valid key of this row
+          float mloc = run_m;
+#pragma unroll
+          for (int j = 0; j < 64; ++j) {
+            const float x = (row_ok && key0 + j <= last) ? __uint_as_float(sv[j]) * c2 : -INFINITY;
+            mloc = fmaxf(mloc, x);
+          }
+          run_m = mloc;
         }
-        run_m = mloc;
       } else {
         uint32_t pk[32], dk[32];
         // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
