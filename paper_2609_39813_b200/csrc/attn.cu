@@ -9,8 +9,10 @@
 //           accumulates dV_j and dK_j in tensor memory;
 //   AT_DQ   the CTA owns query block i: Q_i, dO_i resident, streams (K_j, V_j) for j <= i,
 //           accumulates dQ_i;
-//   AT_FWD  the CTA owns query block i: pass 1 over j gives the row log-sum-exp, pass 2 forms
-//           O_i = sum_j exp(S - LSE) V_j.
+//   AT_FWD  the CTA owns query block i and takes one pass over j: per row and half of 64 keys a
+//           running maximum m_h (moved lazily, only past 2^8) and O_h += exp(S - m_h) V in an
+//           accumulator of its own, rescaled when m_h moves; the halves meet in the epilogue,
+//           O_i = (w_0 O_0 + w_1 O_1), which also gives the row's log-sum-exp.
 // No cross-CTA reduction exists in any mode, so results are bit-reproducible.
 //
 // Per inner step: S = Q K^T and dP = dO V^T (128x128x64 each) land in TMEM columns [0,128) and
@@ -155,9 +157,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     nsteps = it_end - it_begin;
   };
-  // FWD with the rows' log-sum-exp already known (p.lse): one pass, P = exp(s - LSE) directly
-  const bool one_pass = MODE == AT_FWD && p.lse != nullptr;
-  const int npass = (MODE == AT_FWD && !one_pass) ? 2 : 1;
+  // FWD takes one pass over the keys with a running maximum per row and column half (the two halves
+  // of a row keep separate accumulators, so no maximum crosses warps); with the rows' log-sum-exp
+  // already known (p.lse) the shift is fixed: P = exp(s - LSE) directly
+  const bool lse_known = MODE == AT_FWD && p.lse != nullptr;
+  constexpr int npass = 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -286,14 +290,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       };
       if (ok && total > 0) ok = issue_sdp(itg);
       for (int it = 0; it < total && ok; ++it) {
-        const bool pass2 = one_pass || it >= nsteps;          // FWD only
         const uint32_t jg = itg + (uint32_t)it;
         const uint32_t s = jg % kStg, ip = jg & 1u;
         const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
         if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t first = (MODE == AT_FWD ? it == (one_pass ? 0 : nsteps) : it == 0) ? 0u : 1u;   // overwrite on the first product
+        const uint32_t first = it == 0 ? 0u : 1u;             // overwrite on the first product
         if (!kAccDouble && it == 0 && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
         if (MODE == AT_DKV) {
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
@@ -319,13 +322,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
           }
-        } else if (pass2) {
-          // O += P V : A K-major from the P buffer in shared memory, B MN-major = streamed V
+        } else {
+          // O_h += P_h V_h for the two halves of 64 keys, each into its own accumulator (its own running
+          // maximum): A K-major from the P buffer in shared memory, B MN-major = streamed V
           const uint64_t bk = make_smem_desc_mn(st1, 16384u);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint64_t a = make_smem_desc(pbuf + (k >> 2) * 16384u + (k & 3) * 32u);
-            tc_mma<false>(t_acc0, a, bk + 128u * k, id_kmn, first | (k != 0));
+            tc_mma<false>(k < 4 ? t_acc0 : t_acc1, a, bk + 128u * k, id_kmn, first | ((k & 3) != 0));
           }
         }
         tc_commit(b_pds_free);
@@ -454,11 +458,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         dq = __ldg(p.dterm + (size_t)bh * p.S + qrow);
         if (ND == 2) dq2 = __ldg(p.dterm + (size_t)p.BH * p.S + (size_t)bh * p.S + qrow);
       }
-      if (MODE == AT_FWD && one_pass && qrow < p.S) lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
+      if (lse_known && qrow < p.S) lse2 = __ldg(p.lse + (size_t)bh * p.S + qrow) * kLog2e;
     }
-    float run_m = -INFINITY, run_l = 0.f;                     // FWD pass 1: running max and sum (this half)
+    // FWD: the shift in use (log2 units) and the sum of exp2(c2 s - shift) of this row and column half
+    float run_m = lse_known ? lse2 : -INFINITY, run_l = 0.f;
     for (int it = 0; it < total && ok; ++it) {
-      const bool pass2 = one_pass || it >= nsteps;
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
       int kblk;                                               // key block of this step
@@ -471,17 +475,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         kblk = step;
       }
       const int qb0 = (MODE == AT_DKV ? step : blk) * AT_BLK;  // first query of this step's score tile
-      if (MODE == AT_FWD && it == nsteps) {
-        // between the passes: the row's maximum over both column halves.  The second pass forms
-        // exp2(c2 s - max) (no exponential is spent in the first pass), sums it per row and divides
-        // the output by that sum at the end, where the LSE is written too.
-        float* xm = xchg;                                     // [2][128] max, then [2][128] sum
-        xm[h * 128 + r] = run_m;
-        named_bar_sync(1, 256);
-        lse2 = fmaxf(xm[r], xm[128 + r]);                     // the shift of the second pass, in units of log2
-        run_l = 0.f;
-        named_bar_sync(1, 256);
-      }
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sdp_full, ip, abort_flag));
       if (!ok) break;
       tc_fence_after();
@@ -507,11 +500,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       // masking is needed only on the diagonal block and where the sequence ends inside the block
       const bool edge = (p.causal && kblk * AT_BLK + AT_BLK - 1 > qb0) || (kblk + 1) * AT_BLK > p.S ||
                         qb0 + AT_BLK > p.S;
-      if (MODE == AT_FWD && !pass2) {
-        // running max of c2 * s over the valid keys of this half
-        // (four independent chains; the validity test only where a block needs it, and as a select)
-        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+      float resc = 1.f;                                       // FWD: factor for this half's sums when the shift moves
+      if (MODE == AT_FWD && !lse_known) {
+        // largest c2 * s over the valid keys of this half (four independent chains; the validity
+        // test only where a block needs it, and as a select)
+        float mx;
         if (!edge && c2 > 0.f) {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
           for (int j = 0; j < 64; j += 4) {
             m0 = fmaxf(m0, __uint_as_float(sv[j]));
@@ -519,19 +514,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             m2 = fmaxf(m2, __uint_as_float(sv[j + 2]));
             m3 = fmaxf(m3, __uint_as_float(sv[j + 3]));
           }
-          run_m = fmaxf(run_m, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2);   // c2 > 0: the maximum commutes with the scaling
+          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * c2;      // c2 > 0: the maximum commutes with the scaling
         } else {
           const bool row_ok = qrow < p.S;
           const int last = p.causal ? (qrow < p.S - 1 ? qrow : p.S - 1) : p.S - 1;   // last valid key of this row
-          float mloc = run_m;
+          mx = -INFINITY;
 #pragma unroll
           for (int j = 0; j < 64; ++j) {
             const float x = (row_ok && key0 + j <= last) ? __uint_as_float(sv[j]) * c2 : -INFINITY;
-            mloc = fmaxf(mloc, x);
+            mx = fmaxf(mx, x);
           }
-          run_m = mloc;
         }
-      } else {
+        // The shift follows the maximum lazily: it moves only when the maximum has grown by more than
+        // 2^8 (the probabilities of a step then stay below 2^8, harmless in FP32 sums and bf16
+        // operands), so the accumulator is rescaled on few steps.  While nothing finite has been seen
+        // (a fully masked half) the sums are zero and the shift is simply taken.
+        if (run_m == -INFINITY) {
+          run_m = mx;
+        } else if (mx > run_m + 8.0f) {
+          resc = ex2_approx(run_m - mx);
+          run_l *= resc;
+          run_m = mx;
+        }
+        lse2 = run_m == -INFINITY ? 0.f : run_m;
+      }
+      {
         uint32_t pk[32], dk[32];
         // two neighbouring keys: P and dS = P (dP - D) as packed bf16 operands.  FP8-operand mode
         // first rounds P onto the E4M3 grid at p_scale and dS onto the E5M2 grid at ds_scale (the
@@ -590,6 +597,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // the P buffer is free once the product of the previous step has read it
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
+          if (__any_sync(0xFFFFFFFFu, resc != 1.f)) {
+            // that product was also the last one to add to this half's accumulator: rescale the row
+            // (the whole warp takes part in the tensor-memory accesses; rows that keep their shift
+            // multiply by one).  Never on an item's first step: resc is 1 until a shift exists.
+            tc_fence_after();
+            const uint32_t t_mine = (h == 0 ? t_acc0 : t_acc1) + lane_off;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              uint32_t a[32];
+              tmem_ld32(t_mine + c * 32, a);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) a[j] = __float_as_uint(__uint_as_float(a[j]) * resc);
+              tmem_st32(t_mine + c * 32, a);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+          }
           // 64 keys = 8 chunks of 16 bytes in row r of half h of the shared P buffer: chunk index t ^ (r & 7)
 #pragma unroll
           for (int t = 0; t < 8; ++t) {
@@ -737,15 +761,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
     }
     itg += (uint32_t)total;
-    float fwd_inv_l = 1.f;
+    float fwd_w0 = 1.f, fwd_w1 = 1.f;                         // FWD: weights of the two halves' accumulators
     if (MODE == AT_FWD) {
-      // the row's normaliser over both column halves; the LSE in natural-log units
-      float* xm = xchg;
+      // the two column halves of the row meet: common shift m, normaliser l, and the LSE in
+      // natural-log units.  A half that saw no valid key has shift -inf, sum 0 and weight 0.
+      float* xm = xchg;                                       // [2][128] shifts, then [2][128] sums
+      xm[h * 128 + r] = run_m;
       xm[256 + h * 128 + r] = run_l;
       named_bar_sync(1, 256);
-      const float l = xm[256 + r] + xm[384 + r];
-      fwd_inv_l = __fdividef(1.0f, l);
-      if (h == 0 && qrow < p.S && p.lse_out) p.lse_out[(size_t)bh * p.S + qrow] = (lse2 + log2f(l)) / kLog2e;
+      const float m0 = xm[r], m1 = xm[128 + r], l0 = xm[256 + r], l1 = xm[384 + r];
+      const float m = fmaxf(m0, m1);
+      const float e0 = m0 == -INFINITY ? 0.f : ex2_approx(m0 - m), e1 = m1 == -INFINITY ? 0.f : ex2_approx(m1 - m);
+      const float l = l0 * e0 + l1 * e1;
+      const float inv_l = __fdividef(1.0f, l);
+      fwd_w0 = e0 * inv_l;
+      fwd_w1 = e1 * inv_l;
+      if (h == 0 && qrow < p.S && p.lse_out) p.lse_out[(size_t)bh * p.S + qrow] = (m + log2f(l)) / kLog2e;
+      named_bar_sync(1, 256);                                 // the exchange buffer is written again by the next item
     }
     // ---- epilogue: accumulators to global memory (rows = keys for DKV, queries otherwise), 32 KB at a
     // time through the item's resident-tile buffer (no product reads it any more): every thread puts
@@ -802,10 +834,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         float mul;
         if (MODE == AT_DKV) mul = o == 0 ? (FP8 ? inv_do / p.p_scale : 1.f) : p.c * (FP8 ? inv_q / p.ds_scale : 1.f);
         else if (MODE == AT_DQ) mul = p.c * (FP8 ? inv_k / p.ds_scale : 1.f);
-        else mul = inv_v * fwd_inv_l;
+        else mul = inv_v * fwd_w0;
         uint32_t a[32], a2[ND == 2 ? 32 : 1];
         tmem_ld32((o == 0 ? t_acc0 : t_acc1) + lane_off + h * 32, a);
         if (ND == 2) tmem_ld32((o == 0 ? t_acc1 : t_acc0) + lane_off + h * 32, *reinterpret_cast<uint32_t(*)[32]>(&a2[0]));
+        if (MODE == AT_FWD) {
+          // O = w0 O_0 + w1 O_1: fold the second half's accumulator in here
+          uint32_t a1[32];
+          tmem_ld32(t_acc1 + lane_off + h * 32, a1);
+          const float mul1 = inv_v * fwd_w1;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) a[j] = __float_as_uint(fmaf(__uint_as_float(a1[j]), mul1, __uint_as_float(a[j]) * mul));
+          mul = 1.f;
+        }
         if (o == nout - 1) {
           // the accumulators may be overwritten by the next item (FWD: the item after next)
           tc_fence_before();

@@ -102,6 +102,59 @@ def test_forward_statistics_and_store(b, case):
         assert np.array_equal(codes[idx], prep["codes"])
 
 
+@pytest.mark.parametrize("causal", [1, 0])
+@pytest.mark.parametrize("kind", ["growing", "wild", "flat_then_spike"])
+def test_forward_running_maximum(b, kind, causal):
+    """The forward helper takes one pass over the keys with a running maximum per row and column
+    half that moves lazily (only past 2^8): scores that grow from block to block, scores of wild
+    size, and a late spike all make the shift move and the accumulators be rescaled.  Output and
+    log-sum-exp against the plain float64 softmax."""
+    from paper_2609_39813_b200.harness import up
+    B, H, S, D = 1, 2, 700, 64                                   # 6 key blocks, ragged tail
+    rng = np.random.default_rng(77)
+    q = rng.standard_normal((B, H, S, D))
+    k = rng.standard_normal((B, H, S, D))
+    v = rng.standard_normal((B, H, S, D))
+    if kind == "growing":
+        k *= np.linspace(0.2, 6.0, S)[None, None, :, None]       # later keys score higher and higher
+        q *= 2.0
+    elif kind == "wild":
+        q *= 4.0
+        k *= 4.0
+    else:
+        k *= 0.05
+        k[:, :, 650] = 9.0 * q[:, :, 650] / np.linalg.norm(q[:, :, 650], axis=-1, keepdims=True)   # one late, huge score
+    q, k, v = (workloads.to_bf16_grid(a.astype(np.float32)) for a in (q, k, v))
+    scale = 0.125
+    o = torch.full((B * H * S * D,), float("nan"), device="cuda")
+    lse = torch.full((B * H * S,), float("nan"), device="cuda")
+    diag = b.new_diag()
+    b.bsp_attn_fwd_stats(B, H, S, D, causal, scale, up(q, "bf16").reshape(-1), up(k, "bf16").reshape(-1),
+                         up(v, "bf16").reshape(-1), o, lse, diag)
+    assert b.read_diag(diag)["status"] == 0
+    got_o = o.cpu().numpy().reshape(B * H, S, D)
+    got_l = lse.cpu().numpy().reshape(B * H, S)
+    spread = 0.0
+    for idx in range(B * H):
+        bi, hi = divmod(idx, H)
+        want_o, want_lse = attention.forward_output(q[bi, hi], k[bi, hi], v[bi, hi], scale, bool(causal))
+        assert np.isfinite(got_o[idx]).all() and np.isfinite(got_l[idx]).all()
+        assert _rel(got_o[idx], want_o) <= TOL_TC_BF16_OPERANDS, _rel(got_o[idx], want_o)
+        assert np.max(np.abs(got_l[idx] - want_lse)) <= 1e-4 * max(1.0, np.max(np.abs(want_lse)))
+        # how far a later block of 64 keys tops everything before it, in a row (log2 units)
+        sc = scale * q[bi, hi].astype(np.float64) @ k[bi, hi].astype(np.float64).T * 1.4427
+        if causal:
+            sc = np.where(np.tril(np.ones((S, S), dtype=bool)), sc, -np.inf)
+        run = np.full(S, -np.inf)
+        for j0 in range(0, S, 64):
+            blk = np.max(sc[:, j0:j0 + 64], axis=1)
+            ok = np.isfinite(run) & np.isfinite(blk)
+            if ok.any():
+                spread = max(spread, float(np.max((blk - run)[ok])))
+            run = np.maximum(run, blk)
+    assert spread > 8.0                                           # the case does make the shift move
+
+
 @pytest.mark.parametrize("policy", [0, 1, 2])
 def test_dterm_three_reads(b, case, policy):
     inp, g = case
