@@ -219,7 +219,8 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const int q = step * AT_BLK + ts;
       return q < p.S ? __ldg(p.lse + (size_t)tbh * p.S + q) : 0.f;
     };
-    auto bias_put = [&](uint32_t jt, float rawv) {
+    // (fenced = false: the caller issues the proxy fence itself, after other stores that need one too)
+    auto bias_put = [&](uint32_t jt, float rawv, bool fenced = true) {
       if (ts < 128) {
         const float x = rawv * bias_mul;
         const __nv_bfloat16 h1 = __float2bfloat16_rn(x);
@@ -231,8 +232,9 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const uint32_t tile = bias0 + (1u + jt % 3u) * kDkBiasTile;
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %3};" ::"r"(tile + (uint32_t)(ts >> 3) * 256u + (uint32_t)(ts & 7) * 16u),
                      "r"(w0), "r"(w1), "r"(0u) : "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (fenced) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       }
+      if (!fenced) return;
       __syncwarp();
       if (lane == 0) mbar_arrive(b_bias + 8 * (jt % 3u));
     };
@@ -360,14 +362,19 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         tmem_wait_st();
         tc_fence_before();
+        if (bias_due) {
+          // the -LSE row two steps ahead goes out under the same proxy fence as the scaled tiles (a
+          // fence waits for the thread's shared-memory stores to drain: one per step, not two)
+          asm volatile("" : "+f"(bias_next));                       // keeps the first use of the load here
+          bias_put(bias_written, bias_next, false);
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(b_pds_ready + 8 * pb);
-        if (bias_due) {
-          asm volatile("" : "+f"(bias_next));                       // keeps the first use of the load here
-          bias_put(bias_written, bias_next);
-          ++bias_written;
+        if (lane == 0) {
+          mbar_arrive(b_pds_ready + 8 * pb);
+          if (bias_due) mbar_arrive(b_bias + 8 * (bias_written % 3u));
         }
+        if (bias_due) ++bias_written;
       }
       itg += (uint32_t)nsteps;
       // ---- epilogue: the four accumulators hold the draws' differences; their sum and sum of squares
