@@ -599,6 +599,10 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps(dict(attention=attention_section(b, peaks, steps=args.attention_steps))), flush=True)
         return
+    if args.widened_only:
+        if rank == 0:
+            print(json.dumps(dict(widened=widened_section(b, torch))), flush=True)
+        return
 
     inp = workloads.config5()
     T, C, O, K = inp.T, inp.C, inp.O, inp.K
@@ -794,6 +798,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the sub-objects for configs 2, 3 and 4")
     ap.add_argument("--attention-only", action="store_true", help="run only the config-3 attention section")
     ap.add_argument("--attention-steps", type=int, default=3)
+    ap.add_argument("--widened-only", action="store_true",
+                    help="run only the b-bit store, coupling, rounded-probabilities and log-softmax checks")
     ap.add_argument("--kernel-table", action="store_true",
                     help="time the kernels one by one on config 5's tensors and print their GB/s and TFLOP/s")
     ap.add_argument("--selftest-replicas", action="store_true", help=argparse.SUPPRESS)
