@@ -200,6 +200,201 @@ probs_mc_kernel(const float* __restrict__ p_all, const float* __restrict__ V, in
   }
 }
 
+// The same sums for rows of 128 entries and 64 value columns (an attention key block at head width 64),
+// eight draws at a time: 256 threads, one warp per draw.
+//   Phase 1 (a warp, its draw): a lane owns four consecutive entries, i.e. exactly one generator block
+//   per stream (no word wasted).  An entry's grid position is found once per row; a draw is a
+//   comparison.  h = V^T p_q with the lane owning two columns (V row-major in shared memory, p_q
+//   broadcast), dp = V h with the lane's four entries read from a transposed copy of V (one 16-byte
+//   load per column).  The five dot products are warp sums.  Errors, p - p_q, a - p_q and h go to
+//   shared memory.
+//   Phase 2 (the block): thread (entry j, column half) owns 2 x 32 sums of the gradient-of-V errors and
+//   the sums of two or three operators' errors of its entry, and adds the eight draws to them.
+constexpr int kPfN = 128, kPfD = 64, kPfDraws = 8, kPfThreads = 256;
+constexpr size_t kPfSmemFloats = (size_t)2 * kPfN * kPfD + kPfDraws * kPfN /*pq*/ + kPfDraws * kPfD /*h*/ +
+                                 2 * kPfDraws * kPfN /*eu, ea*/ + (size_t)kPfDraws * kPrOps * kPfN /*err*/;
+
+__global__ void __launch_bounds__(kPfThreads, 2)
+probs_mc_128x64_kernel(const float* __restrict__ p_all, const float* __restrict__ V, int law, float param,
+                       PhiloxKey kq, int draw0, int K, float* __restrict__ ds_sum, float* __restrict__ ds_sq,
+                       float* __restrict__ dV_sum, size_t rows) {
+  extern __shared__ __align__(16) float sm[];
+  float* Vs = sm;                                   // [128][64]
+  float* Vt = Vs + kPfN * kPfD;                     // [64][128]: Vt[c][j] = V[j][c]
+  float* pq_s = Vt + kPfN * kPfD;                   // [8][128]
+  float* h_s = pq_s + kPfDraws * kPfN;              // [8][64]
+  float* eu_s = h_s + kPfDraws * kPfD;              // [8][128]
+  float* ea_s = eu_s + kPfDraws * kPfN;             // [8][128]
+  float* err_s = ea_s + kPfDraws * kPfN;            // [8][5][128]
+  __shared__ double red_d[kPfThreads / 32];
+  const size_t row = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  for (int i = tid; i < kPfN * kPfD; i += kPfThreads) {
+    const float v = V[i];
+    Vs[i] = v;
+    Vt[(i % kPfD) * kPfN + i / kPfD] = v;
+  }
+  // this lane's four entries (the same for every warp): values, and where they sit on the grid
+  const float4 p4 = *reinterpret_cast<const float4*>(p_all + row * kPfN + 4 * lane);
+  const float pv[4] = {p4.x, p4.y, p4.z, p4.w};
+  float lo[4], hi[4];
+  uint32_t thr[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (law == 1) {
+      lo[e] = pv[e] - param; hi[e] = pv[e] + param; thr[e] = 0x80000000u;     // up iff the word's top bit is set
+    } else {
+      const float t = __fdiv_rn(pv[e], param);
+      const float n0 = floorf(t);
+      thr[e] = __float2uint_rd(__fsub_rn(t, n0) * 4294967296.0f);
+      lo[e] = n0 * param;
+      hi[e] = (n0 + 1.f) * param;
+    }
+  }
+  // sum_j p_j - 1 in double, once per row (threads of warp 0 cover the row)
+  {
+    double t = w == 0 ? ((double)pv[0] + (double)pv[1]) + ((double)pv[2] + (double)pv[3]) : 0.0;
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if (tid == 0) red_d[0] = t;
+  }
+  __syncthreads();
+  const float sum_p_m1 = (float)(red_d[0] - 1.0);
+  // phase-2 ownership
+  const int j2 = tid & (kPfN - 1), hh = tid >> 7;
+  float acc_u[32], acc_a[32], acc_s[3] = {0.f, 0.f, 0.f}, acc_q[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+  for (int c = 0; c < 32; ++c) acc_u[c] = acc_a[c] = 0.f;
+  const uint64_t q = (uint64_t)row * (kPfN / 4) + (uint64_t)lane;       // generator block of this lane's entries
+  const uint32_t c3 = kq.c3 & ~0xFFu;
+
+  for (int k0 = 0; k0 < K; k0 += kPfDraws) {
+    const int nd = K - k0 < kPfDraws ? K - k0 : kPfDraws;
+    if (w < nd) {
+      const uint32_t k = (uint32_t)(draw0 + k0 + w);
+      const uint4 wq = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, c3 | 0u, kq.k0, kq.k1);
+      const uint4 wa = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, c3 | 1u, kq.k0, kq.k1);
+      const uint4 wb = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), k, c3 | 2u, kq.k0, kq.k1);
+      const uint32_t uq[4] = {wq.x, wq.y, wq.z, wq.w}, ua[4] = {wa.x, wa.y, wa.z, wa.w}, ub[4] = {wb.x, wb.y, wb.z, wb.w};
+      float pq[4], a[4], b[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        // law 0: up iff word < threshold; law 1: up iff the top bit is set, i.e. word >= 2^31
+        const bool u0 = law == 1 ? uq[e] >= thr[e] : uq[e] < thr[e];
+        const bool u1 = law == 1 ? ua[e] >= thr[e] : ua[e] < thr[e];
+        const bool u2 = law == 1 ? ub[e] >= thr[e] : ub[e] < thr[e];
+        pq[e] = u0 ? hi[e] : lo[e];
+        a[e] = u1 ? hi[e] : lo[e];
+        b[e] = u2 ? hi[e] : lo[e];
+      }
+      float* pqw = pq_s + w * kPfN;
+      *reinterpret_cast<float4*>(pqw + 4 * lane) = make_float4(pq[0], pq[1], pq[2], pq[3]);
+      __syncwarp();
+      // h = V^T p_q: columns 2 lane, 2 lane + 1
+      float h0 = 0.f, h1 = 0.f, g0 = 0.f, g1 = 0.f;
+#pragma unroll 4
+      for (int j = 0; j < kPfN; j += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(pqw + j);
+        const float2 v0 = *reinterpret_cast<const float2*>(Vs + (j + 0) * kPfD + 2 * lane);
+        const float2 v1 = *reinterpret_cast<const float2*>(Vs + (j + 1) * kPfD + 2 * lane);
+        const float2 v2 = *reinterpret_cast<const float2*>(Vs + (j + 2) * kPfD + 2 * lane);
+        const float2 v3 = *reinterpret_cast<const float2*>(Vs + (j + 3) * kPfD + 2 * lane);
+        h0 = fmaf(v0.x, x.x, h0); h1 = fmaf(v0.y, x.x, h1);
+        g0 = fmaf(v1.x, x.y, g0); g1 = fmaf(v1.y, x.y, g1);
+        h0 = fmaf(v2.x, x.z, h0); h1 = fmaf(v2.y, x.z, h1);
+        g0 = fmaf(v3.x, x.w, g0); g1 = fmaf(v3.y, x.w, g1);
+      }
+      float* hw = h_s + w * kPfD;
+      *reinterpret_cast<float2*>(hw + 2 * lane) = make_float2(h0 + g0, h1 + g1);
+      __syncwarp();
+      // dp = V h for the lane's four entries
+      float dp[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+      for (int c = 0; c < kPfD; c += 4) {
+        const float4 hv = *reinterpret_cast<const float4*>(hw + c);
+        const float4 t0 = *reinterpret_cast<const float4*>(Vt + (c + 0) * kPfN + 4 * lane);
+        const float4 t1 = *reinterpret_cast<const float4*>(Vt + (c + 1) * kPfN + 4 * lane);
+        const float4 t2 = *reinterpret_cast<const float4*>(Vt + (c + 2) * kPfN + 4 * lane);
+        const float4 t3 = *reinterpret_cast<const float4*>(Vt + (c + 3) * kPfN + 4 * lane);
+        dp[0] = fmaf(t0.x, hv.x, dp[0]); dp[1] = fmaf(t0.y, hv.x, dp[1]); dp[2] = fmaf(t0.z, hv.x, dp[2]); dp[3] = fmaf(t0.w, hv.x, dp[3]);
+        dp[0] = fmaf(t1.x, hv.y, dp[0]); dp[1] = fmaf(t1.y, hv.y, dp[1]); dp[2] = fmaf(t1.z, hv.y, dp[2]); dp[3] = fmaf(t1.w, hv.y, dp[3]);
+        dp[0] = fmaf(t2.x, hv.z, dp[0]); dp[1] = fmaf(t2.y, hv.z, dp[1]); dp[2] = fmaf(t2.z, hv.z, dp[2]); dp[3] = fmaf(t2.w, hv.z, dp[3]);
+        dp[0] = fmaf(t3.x, hv.w, dp[0]); dp[1] = fmaf(t3.y, hv.w, dp[1]); dp[2] = fmaf(t3.z, hv.w, dp[2]); dp[3] = fmaf(t3.w, hv.w, dp[3]);
+      }
+      // the sums over the row the operators need (on the differences to p: see probs_mc_kernel)
+      float dots[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+      float dq[4], da[4], db[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        dq[e] = pq[e] - pv[e]; da[e] = a[e] - pv[e]; db[e] = b[e] - pv[e];
+        dots[0] = fmaf(pv[e], dp[e], dots[0]);
+        dots[1] = fmaf(dq[e], dp[e], dots[1]);
+        dots[2] = fmaf(da[e], dp[e], dots[2]);
+        dots[3] = fmaf(db[e], dp[e], dots[3]);
+        dots[4] += da[e];
+      }
+#pragma unroll
+      for (int i = 0; i < 5; ++i) dots[i] = warp_sum(dots[i]);
+      float er[kPrOps][4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float c = dp[e] - dots[0];
+        er[0][e] = dq[e] * c - pq[e] * dots[1];
+        er[1][e] = da[e] * c - a[e] * dots[2];
+        er[2][e] = a[e] * (dots[4] + sum_p_m1) * dp[e] + er[1][e];
+        er[3][e] = 0.5f * ((da[e] + db[e]) * c - (a[e] * dots[3] + b[e] * dots[2]));
+        er[4][e] = 0.5f * ((dq[e] + db[e]) * c - (pq[e] * dots[3] + b[e] * dots[1]));
+      }
+      *reinterpret_cast<float4*>(eu_s + w * kPfN + 4 * lane) = make_float4(-dq[0], -dq[1], -dq[2], -dq[3]);   // p - p_q
+      *reinterpret_cast<float4*>(ea_s + w * kPfN + 4 * lane) =
+          make_float4(a[0] - pq[0], a[1] - pq[1], a[2] - pq[2], a[3] - pq[3]);
+#pragma unroll
+      for (int op = 0; op < kPrOps; ++op)
+        *reinterpret_cast<float4*>(err_s + ((size_t)w * kPrOps + op) * kPfN + 4 * lane) =
+            make_float4(er[op][0], er[op][1], er[op][2], er[op][3]);
+    }
+    __syncthreads();
+    // phase 2
+    for (int d8 = 0; d8 < nd; ++d8) {
+      const float eu = eu_s[d8 * kPfN + j2], ea = ea_s[d8 * kPfN + j2];
+      const float* hd = h_s + d8 * kPfD + 32 * hh;
+#pragma unroll
+      for (int c = 0; c < 32; c += 4) {
+        const float4 hv = *reinterpret_cast<const float4*>(hd + c);
+        acc_u[c] = fmaf(eu, hv.x, acc_u[c]); acc_u[c + 1] = fmaf(eu, hv.y, acc_u[c + 1]);
+        acc_u[c + 2] = fmaf(eu, hv.z, acc_u[c + 2]); acc_u[c + 3] = fmaf(eu, hv.w, acc_u[c + 3]);
+        acc_a[c] = fmaf(ea, hv.x, acc_a[c]); acc_a[c + 1] = fmaf(ea, hv.y, acc_a[c + 1]);
+        acc_a[c + 2] = fmaf(ea, hv.z, acc_a[c + 2]); acc_a[c + 3] = fmaf(ea, hv.w, acc_a[c + 3]);
+      }
+      // operators 0, 1, 2 in the first column half's threads, 3 and 4 in the second's
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {
+        const int op = hh == 0 ? i : 3 + i;
+        if (op < kPrOps) {
+          const float v = err_s[((size_t)d8 * kPrOps + op) * kPfN + j2];
+          acc_s[i] += v;
+          acc_q[i] = fmaf(v, v, acc_q[i]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+    const int op = hh == 0 ? i : 3 + i;
+    if (op < kPrOps) {
+      ds_sum[((size_t)op * rows + row) * kPfN + j2] = acc_s[i];
+      if (ds_sq) ds_sq[((size_t)op * rows + row) * kPfN + j2] = acc_q[i];
+    }
+  }
+  float* o_u = dV_sum + (((size_t)0 * rows + row) * kPfN + j2) * kPfD + 32 * hh;
+  float* o_a = dV_sum + (((size_t)1 * rows + row) * kPfN + j2) * kPfD + 32 * hh;
+#pragma unroll
+  for (int c = 0; c < 32; c += 4) {
+    *reinterpret_cast<float4*>(o_u + c) = make_float4(acc_u[c], acc_u[c + 1], acc_u[c + 2], acc_u[c + 3]);
+    *reinterpret_cast<float4*>(o_a + c) = make_float4(acc_a[c], acc_a[c + 1], acc_a[c + 2], acc_a[c + 3]);
+  }
+}
+
 }  // namespace bsp
 
 using namespace bsp;
@@ -218,6 +413,14 @@ int bsp_probs_mc(const float* p, const float* V, int64_t rows, int n, int d, int
   k.stream = 0; const PhiloxKey kq = make_key(k);
   k.stream = 1; const PhiloxKey ka = make_key(k);
   k.stream = 2; const PhiloxKey kb = make_key(k);
+  if (n == kPfN && d == kPfD && (reinterpret_cast<uintptr_t>(p) & 15u) == 0 && (reinterpret_cast<uintptr_t>(dV_sum) & 15u) == 0) {
+    const size_t smem_f = kPfSmemFloats * sizeof(float);
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(probs_mc_128x64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_f));
+    probs_mc_128x64_kernel<<<(unsigned)rows, kPfThreads, smem_f, (cudaStream_t)stream>>>(p, V, law, param, kq, draw0, K, ds_sum,
+                                                                                      ds_sq, dV_sum, (size_t)rows);
+    BSP_LAUNCH_CHECK();
+    return BSP_OK;
+  }
   const int threads = (n + 31) / 32 * 32;
   const ProbsSmem lay(n, d, threads);
   const size_t smem = lay.floats(d) * sizeof(float);
