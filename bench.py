@@ -328,9 +328,11 @@ def attention_section(b, peaks, steps=3):
     ops = {}
     for nm, src, fmt in (("q", q, b.E4M3), ("k", k, b.E4M3), ("v", v, b.E4M3), ("dO", dO, b.E5M2)):
         xq, am, sc = torch.zeros(n, dtype=torch.bfloat16, device="cuda"), torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
-        b.bsp_attn_quantize(src, B * H, S * D, fmt, xq, am, sc)
-        ops[nm] = (xq, sc)
-    f8 = b.attn_fp8(ops["q"][1], ops["k"][1], ops["v"][1], ops["dO"][1], 256.0, 1024.0)
+        cd = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        b.bsp_attn_quantize(src, B * H, S * D, fmt, xq, am, sc, codes=cd)
+        ops[nm] = (xq, sc, cd)
+    f8 = b.attn_fp8(ops["q"][1], ops["k"][1], ops["v"][1], ops["dO"][1], 256.0, 1024.0,
+                    ops["q"][2], ops["k"][2], ops["v"][2], ops["dO"][2])
     o8, lse8 = torch.zeros(n, device="cuda"), torch.zeros(B * H * S, device="cuda")
     b.bsp_attn_fwd_stats(B, H, S, D, True, c, ops["q"][0], ops["k"][0], ops["v"][0], o8, lse8, diag, fp8=f8)
     d8 = torch.zeros(B * H * S, device="cuda")

@@ -354,10 +354,12 @@ int bsp_linear_dgrad(int64_t T, int64_t O, int64_t C, const uint8_t* dy_codes, b
  * / p_scale; dP = dO V^T; D from the assigned output copy; dS = P o (dP - D); dS_q = RN_E5M2(dS
  * ds_scale) / ds_scale feeds dQ and dK (ds_scale supplied by the caller, like a delayed scale).
  * In that mode q, k, v, dO are bf16 tensors holding the DECODED codes as written by
- * bsp_attn_quantize (every FP8 value is a bf16 value, so the tensor-core products are those of the
- * FP8 operands exactly); their scales are folded back in the kernel.  The final E5M2 cast of the
- * returned gradients is not applied (outputs FP32).  Quantisation points and the two scales are
- * this library's reading of that appendix.
+ * bsp_attn_quantize (every FP8 value is a bf16 value): the forward helper reads those (its P V
+ * product has an unrounded P).  The backward reads the codes themselves (bsp_attn_fp8_t: q_codes,
+ * k_codes, v_codes E4M3, do_codes E5M2, uint8 [B, H, S, Dh], all four required) and issues its
+ * seven products as FP8 tensor-core products, P and dS entering as E4M3 / E5M2 codes; the scales are
+ * folded back in the kernel.  The final E5M2 cast of the returned gradients is not applied (outputs
+ * FP32).  Quantisation points and the two scales are this library's reading of that appendix.
  * ------------------------------------------------------------------------------------------ */
 
 typedef struct {
@@ -367,13 +369,18 @@ typedef struct {
   const float* do_scale;
   float p_scale;             /* power of two; 256 keeps P * p_scale <= 256 < 448 */
   float ds_scale;
+  const uint8_t* q_codes;    /* the codes themselves, [B, H, S, Dh]: read by the backward (NULL for the forward helper) */
+  const uint8_t* k_codes;
+  const uint8_t* v_codes;
+  const uint8_t* do_codes;
 } bsp_attn_fp8_t;
 
-/* xq (bf16, same shape) = decode(RN_fmt(x * scale_g)) for each of n_groups contiguous groups of
- * group_size bf16 elements, scale_g = fmax / amax_g; amax[n_groups] and scales[n_groups] are
- * written too.  group_size a multiple of 8. */
-int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax,
-                      float* scales, bsp_diag_t* diag, void* stream);
+/* For each of n_groups contiguous groups of group_size bf16 elements, scale_g = fmax / amax_g:
+ * xq (bf16, same shape, may be NULL) = decode(RN_fmt(x * scale_g)), codes (uint8, same shape, may be
+ * NULL) = RN_fmt(x * scale_g); amax[n_groups] and scales[n_groups] are written too.  group_size a
+ * multiple of 8; x, xq 16-byte and codes 8-byte aligned. */
+int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, uint8_t* codes,
+                      float* amax, float* scales, bsp_diag_t* diag, void* stream);
 
 /* Forward statistics from the operands exactly as the backward will see them: o = P V (FP32, the
  * "original" output the store rounds; P unrounded) and lse = log sum_j exp(c q.k_j). */

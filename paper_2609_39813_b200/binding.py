@@ -101,7 +101,8 @@ class LsmStat(C.Structure):
 
 class AttnFp8(C.Structure):
     _fields_ = [("q_scale", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
-                ("do_scale", C.c_void_p), ("p_scale", C.c_float), ("ds_scale", C.c_float)]
+                ("do_scale", C.c_void_p), ("p_scale", C.c_float), ("ds_scale", C.c_float),
+                ("q_codes", C.c_void_p), ("k_codes", C.c_void_p), ("v_codes", C.c_void_p), ("do_codes", C.c_void_p)]
 
 
 class BspError(RuntimeError):
@@ -148,7 +149,7 @@ _SIGNATURES = {
                                 _P, _P]),
     "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _I, _I,
                           Key, _P, _P, _P, _P, _P, _P]),
-    "bsp_attn_quantize": (_I, [_P, _I, _SZ, _I, _P, _P, _P, _P, _P]),
+    "bsp_attn_quantize": (_I, [_P, _I, _SZ, _I, _P, _P, _P, _P, _P, _P]),
     "bsp_mc_accumulate": (_I, [_P, _P, _P, _P, _SZ, _P]),
     "bsp_mc_moments": (_I, [_P, _P, _P, _SZ, _I, _P, _P, _P, _P]),
     "bsp_mc_check_attn_workspace_bytes": (_SZ, [C.POINTER(AttnDesc), _I]),
@@ -432,13 +433,15 @@ def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, 
           "bsp_attn_bwd")
 
 
-def bsp_attn_quantize(x, n_groups, group_size, fmt, xq, amax, scales, diag=None, stream=None):
-    check(lib().bsp_attn_quantize(ptr(x), n_groups, group_size, fmt, ptr(xq), ptr(amax), ptr(scales), ptr(diag),
-                                  _st(stream)), "bsp_attn_quantize")
+def bsp_attn_quantize(x, n_groups, group_size, fmt, xq, amax, scales, diag=None, stream=None, codes=None):
+    check(lib().bsp_attn_quantize(ptr(x), n_groups, group_size, fmt, ptr(xq), ptr(codes), ptr(amax), ptr(scales),
+                                  ptr(diag), _st(stream)), "bsp_attn_quantize")
 
 
-def attn_fp8(q_scale, k_scale, v_scale, do_scale, p_scale=256.0, ds_scale=1.0) -> AttnFp8:
-    return AttnFp8(ptr(q_scale), ptr(k_scale), ptr(v_scale), ptr(do_scale), float(p_scale), float(ds_scale))
+def attn_fp8(q_scale, k_scale, v_scale, do_scale, p_scale=256.0, ds_scale=1.0, q_codes=None, k_codes=None,
+             v_codes=None, do_codes=None) -> AttnFp8:
+    return AttnFp8(ptr(q_scale), ptr(k_scale), ptr(v_scale), ptr(do_scale), float(p_scale), float(ds_scale),
+                   ptr(q_codes), ptr(k_codes), ptr(v_codes), ptr(do_codes))
 
 
 def rule(rel_tol_deterministic=1e-4, qprime_hold=2.0, r_hold=3.0, qprime_fail=4.0, r_fail=6.0, rel_hold=0.0):

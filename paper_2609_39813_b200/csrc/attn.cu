@@ -64,6 +64,7 @@ struct AttnParams {
   const float* sc_v;
   const float* sc_do;
   float p_scale, ds_scale;
+  const uint8_t *cq, *ck, *cv, *cdo;   // the operands' codes: what the backward modes load in FP8-operand mode
 };
 
 // Two floats rounded to the nearest FP8 grid value (ties to even, saturating: what f8_rn_value
@@ -193,6 +194,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // instruction descriptors (bf16 operands, FP32 accumulation)
   const uint32_t id_sdp = make_idesc(1u, 1u, 128, 128);                                   // A, B K-major
   const uint32_t id_kmn = make_idesc(1u, 1u, 128, 64) | (1u << 16);                       // A K-major, B MN-major
+  // FP8-operand mode of the backward: every product is an FP8 tensor-core product (kind::f8f6f4) on the
+  // codes themselves.  The streamed and resident tiles are 128 rows of 64 bytes (64-byte swizzle), a
+  // K step is 32 elements, and P (E4M3) and dS (E5M2) go back into tensor memory four codes per column.
+  constexpr bool F8K = FP8 && MODE != AT_FWD;
+  constexpr uint32_t kTileB = F8K ? (uint32_t)(AT_BLK * AT_D) : (uint32_t)kAtTile;        // bytes a tile load brings
+  // operand formats (E4M3 = 0, E5M2 = 1): S from Q and K; dP from dO (E5M2) and V
+  const uint32_t id8_s = make_idesc(0u, 0u, 128, 128);
+  const uint32_t id8_dp = MODE == AT_DKV ? make_idesc(0u, 1u, 128, 128) : make_idesc(1u, 0u, 128, 128);
+  const uint32_t id8_pdo = make_idesc(0u, 1u, 128, 64) | (1u << 16);                      // P^T (E4M3) x dO (E5M2, MN-major)
+  const uint32_t id8_ds = make_idesc(1u, 0u, 128, 64) | (1u << 16);                       // dS (E5M2) x Q or K (E4M3, MN-major)
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer
@@ -208,7 +219,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const uint32_t rb = item & 1u, rph = (item >> 1) & 1u;
         if (!mbar_wait(b_res_empty + 8 * rb, rph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t r0 = res_base + rb * 2 * kAtTile, r1 = r0 + kAtTile;
-        mbar_expect_tx(b_res + 8 * rb, (MODE == AT_FWD ? 1 : 2) * kAtTile);
+        mbar_expect_tx(b_res + 8 * rb, (MODE == AT_FWD ? 1 : 2) * kTileB);
         if (MODE == AT_DKV) {
           tma_load_3d(r0, &tm_k, b_res + 8 * rb, 0, blk * AT_BLK, bh);
           tma_load_3d(r1, &tm_v, b_res + 8 * rb, 0, blk * AT_BLK, bh);
@@ -222,7 +233,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const uint32_t s = itg % kStg, ph = (itg / kStg) & 1u;
           if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
-          mbar_expect_tx(b_sfull + 8 * s, 2 * kAtTile);
+          mbar_expect_tx(b_sfull + 8 * s, 2 * kTileB);
           if (MODE == AT_DKV) {
             tma_load_3d(d0, &tm_q, b_sfull + 8 * s, 0, step * AT_BLK, bh);
             tma_load_3d(d1, &tm_do, b_sfull + 8 * s, 0, step * AT_BLK, bh);
@@ -267,15 +278,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const uint32_t do_t = MODE == AT_DKV ? st1 : res1, v_t = MODE == AT_DKV ? res1 : st1;
         // DKV forms the transposes, S^T = K Q^T and dP^T = V dO^T (rows = keys), so that P^T and dS^T
         // come out of the softmax warps as the row-per-lane A operands of dV = P^T dO, dK = dS^T Q
-        {
-          const uint64_t a = make_smem_desc(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc(MODE == AT_DKV ? q_t : k_t);
+        if (F8K) {
+          // 64 bytes of K per row: two steps of 32 elements
+          const uint64_t a = make_smem_desc_sw64(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc_sw64(MODE == AT_DKV ? q_t : k_t);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) tc_mma<false>(t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
-        }
-        if (MODE != AT_FWD) {
-          const uint64_t a = make_smem_desc(MODE == AT_DKV ? v_t : do_t), b = make_smem_desc(MODE == AT_DKV ? do_t : v_t);
+          for (int k = 0; k < 2; ++k) tc_mma<true>(t_s, a + 2u * k, b + 2u * k, id8_s, k != 0);
+          const uint64_t a2 = make_smem_desc_sw64(MODE == AT_DKV ? v_t : do_t), b2 = make_smem_desc_sw64(MODE == AT_DKV ? do_t : v_t);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+          for (int k = 0; k < 2; ++k) tc_mma<true>(t_dp, a2 + 2u * k, b2 + 2u * k, id8_dp, k != 0);
+        } else {
+          {
+            const uint64_t a = make_smem_desc(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc(MODE == AT_DKV ? q_t : k_t);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma<false>(t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+          }
+          if (MODE != AT_FWD) {
+            const uint64_t a = make_smem_desc(MODE == AT_DKV ? v_t : do_t), b = make_smem_desc(MODE == AT_DKV ? do_t : v_t);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+          }
         }
         if (MODE == AT_DKV) {
           // the extra K = 16 step: minus LSE/c into S^T, minus D into dP^T (see the X tiles)
@@ -298,7 +319,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_fence_after();
         const uint32_t first = it == 0 ? 0u : 1u;             // overwrite on the first product
         if (!kAccDouble && it == 0 && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
-        if (MODE == AT_DKV) {
+        if (F8K && MODE == AT_DKV) {
+          // the same products on the codes: eight columns per 32 queries, 128 queries = 4 x 32 along K
+          const uint64_t bdo = make_smem_desc_mn_sw64(st1), bq = make_smem_desc_mn_sw64(st0);
+          if (DV) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_p + 8u * k, bdo + 128u * k, id8_pdo, first | (k != 0));
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc1, t_ds + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
+          if (ND == 2 && !DV) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_ds2 + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
+          }
+        } else if (F8K && MODE == AT_DQ) {
+          const uint64_t bk = make_smem_desc_mn_sw64(st0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_ds + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
+          if (ND == 2) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
+          }
+        } else if (MODE == AT_DKV) {
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
           // queries), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
           const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
@@ -545,8 +587,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         // grid values are exact in bf16; the scales come back in the epilogue).
         // a pair of dS values as a packed bf16 operand (FP8-operand mode: on the E5M2 grid at ds_scale)
         auto pack_ds = [&](float s0, float s1) -> uint32_t {
+          if (F8K) return f8_encode_rn_pair_inrange<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);   // two codes, 16 bits
           if (FP8) return f8_grid_bf16x2<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);
           return pack_bf16x2(s0, s1);
+        };
+        // 32 of this thread's 64 columns of an operand (16 packed pairs) back into tensor memory: two
+        // 16-bit elements per column, or (codes) four per column
+        auto st_half = [&](uint32_t t_base, int half, const uint32_t (&wv)[16]) {
+          if (F8K) {
+            uint32_t c8[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) c8[i] = (wv[2 * i] & 0xFFFFu) | (wv[2 * i + 1] << 16);
+            tmem_st8(t_base + lane_off + h * 16 + half * 8, c8);
+          } else {
+            tmem_st16(t_base + lane_off + h * 32 + half * 16, wv);
+          }
         };
         auto pack_pair = [&](float p0, float p1, uint32_t dp0, uint32_t dp1, float d0, float d1, uint32_t& po,
                              uint32_t& dso) {
@@ -557,6 +612,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
           }
           if (FP8 && MODE != AT_FWD) {                      // the forward keeps P unrounded
+            if (F8K) {                                      // the codes themselves (two per word for now)
+              po = f8_encode_rn_pair_inrange<BSP_E4M3>(p0 * p.p_scale, p1 * p.p_scale);
+              dso = f8_encode_rn_pair_inrange<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);
+              return;
+            }
             po = f8_grid_bf16x2<BSP_E4M3>(p0 * p.p_scale, p1 * p.p_scale);
             dso = f8_grid_bf16x2<BSP_E5M2>(s0 * p.ds_scale, s1 * p.ds_scale);
             return;
@@ -645,8 +705,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
-          tmem_st16(t_ds + lane_off + h * 32, da);
-          tmem_st16(t_ds2 + lane_off + h * 32, db);
+          st_half(t_ds, 0, da);
+          st_half(t_ds2, 0, db);
           if (!edge) {
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair2_at(j, false);
@@ -654,8 +714,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair2_at(j, true);
           }
-          tmem_st16(t_ds + lane_off + h * 32 + 16, da);
-          tmem_st16(t_ds2 + lane_off + h * 32 + 16, db);
+          st_half(t_ds, 1, da);
+          st_half(t_ds2, 1, db);
           tmem_wait_st();
           tc_fence_before();
         } else if (MODE == AT_DQ) {
@@ -670,7 +730,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // 64 columns go back into tensor memory as 32 packed pairs (columns h*32 .. h*32+31)
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
-          tmem_st32(t_ds + lane_off + h * 32, dk);
+          st_half(t_ds, 0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
+          st_half(t_ds, 1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
           tmem_wait_st();
           tc_fence_before();
         } else if (MODE == AT_DKV && ND == 2) {
@@ -700,8 +761,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
-          tmem_st16(t_ds + lane_off + h * 32, da);
-          tmem_st16(t_ds2 + lane_off + h * 32, db);
+          st_half(t_ds, 0, da);
+          st_half(t_ds2, 0, db);
           if (!edge) {
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair2_at(j, false);
@@ -709,8 +770,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair2_at(j, true);
           }
-          tmem_st16(t_ds + lane_off + h * 32 + 16, da);
-          tmem_st16(t_ds2 + lane_off + h * 32 + 16, db);
+          st_half(t_ds, 1, da);
+          st_half(t_ds2, 1, db);
           tmem_wait_st();
           tc_fence_before();
         } else {
@@ -728,8 +789,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
-          if (DV) tmem_st16(t_p + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
-          tmem_st16(t_ds + lane_off + h * 32, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
+          if (DV) st_half(t_p, 0, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+          st_half(t_ds, 0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
           if (!edge) {
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair_at(j, false);
@@ -737,8 +798,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair_at(j, true);
           }
-          if (DV) tmem_st16(t_p + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
-          tmem_st16(t_ds + lane_off + h * 32 + 16, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
+          if (DV) st_half(t_p, 1, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+          st_half(t_ds, 1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
           tmem_wait_st();
           tc_fence_before();
         }
@@ -1035,10 +1096,20 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   int rc;
   if ((rc = make_out_map(&mo0, p.out0 ? p.out0 : p.out1, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_out_map(&mo1, p.out1 ? p.out1 : p.out0, p.BH, p.S)) != BSP_OK) return rc;
-  if ((rc = make_head_map(&mq, q, p.BH, p.S)) != BSP_OK) return rc;
-  if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
-  if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
-  if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
+  if (FP8 && MODE != AT_FWD) {
+    // the backward of the FP8-operand mode loads the codes
+    if (!p.cq || !p.ck || !p.cv || !p.cdo) return BSP_ERR_ARG;
+    if (!aligned16(p.cq) || !aligned16(p.ck) || !aligned16(p.cv) || !aligned16(p.cdo)) return BSP_ERR_ALIGN;
+    if ((rc = make_head_map_u8(&mq, p.cq, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map_u8(&mk, p.ck, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map_u8(&mv, p.cv, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map_u8(&mdo, p.cdo, p.BH, p.S)) != BSP_OK) return rc;
+  } else {
+    if ((rc = make_head_map(&mq, q, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map(&mk, k, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map(&mv, v, p.BH, p.S)) != BSP_OK) return rc;
+    if ((rc = make_head_map(&mdo, dO ? dO : q, p.BH, p.S)) != BSP_OK) return rc;
+  }
   static std::atomic<bool> attr_set_dev[kMaxDevices];       // per kernel instantiation and device
   std::atomic<bool>& attr_set = attr_set_dev[device_slot()];
   if (!attr_set.load(std::memory_order_acquire)) {
@@ -1079,6 +1150,7 @@ static int set_fp8(AttnParams& p, const bsp_attn_fp8_t* f) {
   p.sc_q = f ? f->q_scale : nullptr; p.sc_k = f ? f->k_scale : nullptr;
   p.sc_v = f ? f->v_scale : nullptr; p.sc_do = f ? f->do_scale : nullptr;
   p.p_scale = f ? f->p_scale : 1.f; p.ds_scale = f ? f->ds_scale : 1.f;
+  p.cq = f ? f->q_codes : nullptr; p.ck = f ? f->k_codes : nullptr; p.cv = f ? f->v_codes : nullptr; p.cdo = f ? f->do_codes : nullptr;
   if (f && (!f->q_scale || !f->k_scale || !f->v_scale || !f->do_scale || !(f->p_scale > 0.f) || !(f->ds_scale > 0.f)))
     return BSP_ERR_ARG;
   return BSP_OK;
@@ -1218,21 +1290,25 @@ int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_sca
 template <int FMT>
 __global__ void __launch_bounds__(256)
 quantize_decode_kernel(const uint16_t* __restrict__ x, size_t group_size, const float* __restrict__ scales,
-                       uint16_t* __restrict__ out, size_t n8) {
+                       uint16_t* __restrict__ out, uint8_t* __restrict__ codes, size_t n8) {
   const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= n8) return;
   const size_t i0 = t * 8;
   const float s = __ldg(scales + i0 / group_size);
   const uint4 raw = __ldg(reinterpret_cast<const uint4*>(x) + t);
   const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-  uint32_t o[4];
+  uint32_t o[4], c[4];
+  DiagCounters dc;                                          // (non-finite inputs were counted by the amax pass)
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float a = f8_rn_value<FMT>(__fmul_rn(bf16_bits_to_float(w[i] & 0xFFFFu), s));
-    const float b = f8_rn_value<FMT>(__fmul_rn(bf16_bits_to_float(w[i] >> 16), s));
+    const float va = __fmul_rn(bf16_bits_to_float(w[i] & 0xFFFFu), s), vb = __fmul_rn(bf16_bits_to_float(w[i] >> 16), s);
+    const float a = f8_rn_value<FMT>(va);
+    const float b = f8_rn_value<FMT>(vb);
     o[i] = (__float_as_uint(a) >> 16) | (__float_as_uint(b) & 0xFFFF0000u);     // FP8 values are exact in bf16
+    c[i] = f8_encode<FMT, false>(va, 0u, dc) | (f8_encode<FMT, false>(vb, 0u, dc) << 8);
   }
-  reinterpret_cast<uint4*>(out)[t] = make_uint4(o[0], o[1], o[2], o[3]);
+  if (out) reinterpret_cast<uint4*>(out)[t] = make_uint4(o[0], o[1], o[2], o[3]);
+  if (codes) reinterpret_cast<uint2*>(codes)[t] = make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16));
 }
 
 }  // namespace bsp
@@ -1259,11 +1335,11 @@ int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, i
                              stream);
 }
 
-int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, float* amax, float* scales,
-                      bsp_diag_t* diag, void* stream) {
-  if (!x || !xq || !amax || !scales || n_groups <= 0 || !valid_enum(fmt, 1)) return BSP_ERR_ARG;
+int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, void* xq, uint8_t* codes, float* amax,
+                      float* scales, bsp_diag_t* diag, void* stream) {
+  if (!x || (!xq && !codes) || !amax || !scales || n_groups <= 0 || !valid_enum(fmt, 1)) return BSP_ERR_ARG;
   if (group_size == 0 || group_size % 8 != 0) return BSP_ERR_UNSUPPORTED;
-  if (!aligned16(x) || !aligned16(xq)) return BSP_ERR_ALIGN;
+  if (!aligned16(x) || !aligned16(xq) || (reinterpret_cast<uintptr_t>(codes) & 7u)) return BSP_ERR_ALIGN;
   int rc = bsp_amax(x, BSP_BF16, (size_t)n_groups, group_size, amax, diag, stream);
   if (rc != BSP_OK) return rc;
   if ((rc = bsp_scale_from_amax(amax, (size_t)n_groups, fmt, scales, stream)) != BSP_OK) return rc;
@@ -1272,10 +1348,10 @@ int bsp_attn_quantize(const void* x, int n_groups, size_t group_size, int fmt, v
   cudaStream_t st = (cudaStream_t)stream;
   if (fmt == BSP_E4M3)
     quantize_decode_kernel<BSP_E4M3><<<grid, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), group_size, scales,
-                                                           reinterpret_cast<uint16_t*>(xq), n8);
+                                                           reinterpret_cast<uint16_t*>(xq), codes, n8);
   else
     quantize_decode_kernel<BSP_E5M2><<<grid, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(x), group_size, scales,
-                                                           reinterpret_cast<uint16_t*>(xq), n8);
+                                                           reinterpret_cast<uint16_t*>(xq), codes, n8);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }

@@ -73,6 +73,20 @@ static inline int make_head_map(CUtensorMap* map, const void* base, int BH, int 
   return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
 }
 
+// The operands' FP8 codes, uint8 [BH][S][64]: tiles of 128 rows of 64 bytes, 64-byte swizzle.
+static inline int make_head_map_u8(CUtensorMap* map, const void* base, int BH, int S) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return BSP_ERR_CUDA;
+  cuuint64_t gdim[3] = {(cuuint64_t)AT_D, (cuuint64_t)S, (cuuint64_t)BH};
+  cuuint64_t gstr[2] = {(cuuint64_t)AT_D, (cuuint64_t)S * AT_D};
+  cuuint32_t box[3] = {(cuuint32_t)AT_D, (cuuint32_t)AT_BLK, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? BSP_OK : BSP_ERR_CUDA;
+}
+
 inline int check_attn_shape(int B, int H, int S, int Dh, int dt) {
   if (B <= 0 || H <= 0 || S <= 0) return BSP_ERR_ARG;
   if (Dh != AT_D || dt != BSP_BF16) return BSP_ERR_UNSUPPORTED;

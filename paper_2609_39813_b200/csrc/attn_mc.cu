@@ -514,6 +514,7 @@ struct AttnCheckBuffers {
   float *g_ref[3], *g_pol[3], *S1[2], *S2[2], *S1d, *S2d;
   // FP8-operand mode: the rounded operands (decoded codes as bf16) and their per-slice scales
   void* op8[4];
+  uint8_t* opc[4];                                // the operands' codes (FP8-operand mode)
   float *op_amax[4], *op_scale[4];
   void* ws_stats;
   size_t b_stats;
@@ -539,7 +540,7 @@ static size_t attn_carve(const bsp_attn_desc_t* op, int K, char* base, AttnCheck
   c.S1d = (float*)take(rows * 4); c.S2d = (float*)take(rows * 4);
   if (op->fp8_operands) {
     for (int t = 0; t < 4; ++t) {
-      c.op8[t] = take(n * 2); c.op_amax[t] = (float*)take(BH * 4); c.op_scale[t] = (float*)take(BH * 4);
+      c.op8[t] = take(n * 2); c.opc[t] = (uint8_t*)take(n); c.op_amax[t] = (float*)take(BH * 4); c.op_scale[t] = (float*)take(BH * 4);
     }
   }
   c.b_stats = kMaxPendingStats * kStatSlotBytes;
@@ -601,11 +602,12 @@ int bsp_mc_check_attn(const bsp_attn_desc_t* op, int K, const bsp_verdict_rule_t
   if (fp8) {
     const void* src[4] = {op->q, op->k, op->v, op->dO};
     for (int t = 0; t < 4; ++t)
-      BSP_TRY(bsp_attn_quantize(src[t], (int)BH, (size_t)S * Dh, t == 3 ? BSP_E5M2 : BSP_E4M3, b.op8[t], b.op_amax[t],
-                                b.op_scale[t], diag, st));
+      BSP_TRY(bsp_attn_quantize(src[t], (int)BH, (size_t)S * Dh, t == 3 ? BSP_E5M2 : BSP_E4M3, b.op8[t], b.opc[t],
+                                b.op_amax[t], b.op_scale[t], diag, st));
     q = b.op8[0]; k = b.op8[1]; v = b.op8[2]; dO = b.op8[3];
     f8.q_scale = b.op_scale[0]; f8.k_scale = b.op_scale[1]; f8.v_scale = b.op_scale[2]; f8.do_scale = b.op_scale[3];
     f8.p_scale = op->p_scale; f8.ds_scale = op->ds_scale;
+    f8.q_codes = b.opc[0]; f8.k_codes = b.opc[1]; f8.v_codes = b.opc[2]; f8.do_codes = b.opc[3];
     f = &f8;
   }
   const float* do_scales = fp8 ? f8.do_scale : nullptr;

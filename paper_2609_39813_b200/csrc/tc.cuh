@@ -192,6 +192,17 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint
       : "memory");
 }
 
+// The same with 8-bit operands (kind::f8f6f4): four elements per 32-bit column of `tmem_a` (element k
+// in byte k % 4 of column k / 4), so one K = 32 step spans eight columns.
+__device__ __forceinline__ void tc_mma_ts_f8(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t).
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
@@ -232,6 +243,29 @@ __device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t smem_addr, uint32
   return d;
 }
 
+// Tiles with rows of 64 bytes (8-bit elements at head width 64) in the 64-byte-swizzle layout that TMA
+// writes: rows at a 64-byte pitch, 16-byte chunks XOR-ed with (row / 2) % 4, 8-row groups 512 bytes
+// apart.  K-major: a K = 32 step is 32 bytes of a row.  MN-major (a tile of a matrix stored
+// [K rows][64 bytes of MN]): one atom of 64 bytes of MN by eight k rows every 512 bytes.
+__device__ __forceinline__ uint64_t make_smem_desc_sw64(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(512u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)4 << 61;                                // layout: 64-byte swizzle
+  return d;
+}
+__device__ __forceinline__ uint64_t make_smem_desc_mn_sw64(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(512u >> 4) << 16;                      // leading byte offset (a single atom along MN: unused)
+  d |= (uint64_t)(512u >> 4) << 32;                      // stride byte offset: next eight k rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)4 << 61;
+  return d;
+}
+
 // A K-major operand of one K = 16 step (16-bit elements) without swizzle: rows of 16 bytes, eight
 // rows per 128-byte core matrix, the two 8-element halves of a row 128 bytes apart (leading byte
 // offset), 8-row groups 256 bytes apart (stride byte offset).
@@ -265,6 +299,12 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
       ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {

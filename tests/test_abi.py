@@ -44,7 +44,7 @@ def test_struct_layouts_match_header(built):
     from paper_2609_39813_b200 import binding as b
     assert ctypes.sizeof(b.Key) == 24 and ctypes.sizeof(b.Quant) == 24
     assert ctypes.sizeof(b.Diag) == 24 and ctypes.sizeof(b.UseResult) == 88
-    assert ctypes.sizeof(b.VerdictRule) == 48 and ctypes.sizeof(b.AttnFp8) == 40
+    assert ctypes.sizeof(b.VerdictRule) == 48 and ctypes.sizeof(b.AttnFp8) == 72
     assert ctypes.sizeof(b.NormLinearDesc) == 120 and ctypes.sizeof(b.AttnDesc) == 104
     assert ctypes.sizeof(b.McLayout) == 15 * ctypes.sizeof(ctypes.c_size_t)
     d = b.NormLinearDesc()

@@ -331,15 +331,19 @@ def _quantised_operands(b, inp):
         x = up(arr, "bf16")
         xq = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
         amax, sc = torch.zeros(BH, device="cuda"), torch.zeros(BH, device="cuda")
-        b.bsp_attn_quantize(x, BH, S * D, fmt, xq, amax, sc)
-        dev[nm] = (xq, sc)
+        cd = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        b.bsp_attn_quantize(x, BH, S * D, fmt, xq, amax, sc, codes=cd)
+        dev[nm] = (xq, sc, cd)
         got = xq.float().cpu().numpy().reshape(BH, S, D)
+        got_codes = cd.cpu().numpy().reshape(BH, S, D)
         scs = sc.cpu().numpy()
         vals = np.zeros((BH, S, D))
         for idx in range(BH):
             value, codes, s32, _ = attention.quantise_rn(arr.reshape(BH, S, D)[idx], fmt)
             assert scs[idx] == s32
             assert np.array_equal(got[idx], fp8.decode(codes, fmt).astype(np.float32))
+            # the codes themselves (what the backward's products read): -0 and +0 both decode to zero
+            assert np.array_equal(fp8.decode(got_codes[idx], fmt), fp8.decode(codes, fmt))
             vals[idx] = value
         hat[nm] = vals
     return dev, hat
@@ -368,7 +372,8 @@ def test_mc_check_attention_fp8_operand_mode(b):
     got = [r.verdict for r in res]
     assert got[:8] == [H_, H_, H_, H_, F_, F_, F_, H_] and got[8] == H_ and got[11] == H_
     # the forward output the check stored: recomputed through the same entry point
-    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale)
+    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale,
+                   dev["q"][2], dev["k"][2], dev["v"][2], dev["dO"][2])
     n = inp.B * inp.H * inp.S * inp.D
     o, lse = torch.zeros(n, device="cuda"), torch.zeros(inp.B * inp.H * inp.S, device="cuda")
     b.bsp_attn_fwd_stats(inp.B, inp.H, inp.S, inp.D, True, inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], o, lse, fp8=f)
@@ -404,7 +409,8 @@ def test_fp8_operand_mode(b, name):
     o0, _ = attention.forward_output(hat["q"][0], hat["k"][0], hat["v"][0], inp.softmax_scale, cfg["causal"])
     ds0 = attention.backward(hat["q"][0], hat["k"][0], hat["v"][0], hat["dO"][0], inp.softmax_scale, o0, cfg["causal"])["dS"]
     ds_scale = float(np.float32(2.0 ** np.floor(np.log2(57344.0 / (2.0 * np.max(np.abs(ds0)))))))
-    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale)
+    f = b.attn_fp8(dev["q"][1], dev["k"][1], dev["v"][1], dev["dO"][1], 256.0, ds_scale,
+                   dev["q"][2], dev["k"][2], dev["v"][2], dev["dO"][2])
     o, lse = torch.zeros(n, device="cuda"), torch.zeros(BH * S, device="cuda")
     diag = b.new_diag()
     b.bsp_attn_fwd_stats(B, H, S, D, cfg["causal"], inp.softmax_scale, dev["q"][0], dev["k"][0], dev["v"][0], o, lse, diag, fp8=f)
@@ -471,6 +477,13 @@ def test_attention_row_case_fp8_operands_exact(b):
     v = np.zeros((1, 1, S, D), np.float32); v[0, 0, :, 0] = np.where(np.arange(S) % 2 == 0, 1.0, 1.5)
     qd, kd, vd = up(q, "bf16"), up(k, "bf16"), up(v, "bf16")
     one = torch.ones(1, device="cuda")
+
+    def codes_of(x_dev, fmt):                                 # the values are on the grid: unit scale, nearest
+        cd = torch.zeros(S * D, dtype=torch.uint8, device="cuda")
+        b.bsp_round(x_dev.reshape(-1), S * D, b.quant(fmt, b.ROUND_NEAREST, 1.0), b.key(0, 1, 0), 0, cd)
+        return cd
+
+    qc, kc, vc = codes_of(qd, b.E4M3), codes_of(kd, b.E4M3), codes_of(vd, b.E4M3)
     f = b.attn_fp8(one, one, one, one, 256.0, 1.0)
     o = torch.zeros(S * D, device="cuda"); lse = torch.zeros(S, device="cuda")
     b.bsp_attn_fwd_stats(1, 1, S, D, True, c, qd, kd, vd, o, lse, fp8=f)
@@ -480,8 +493,10 @@ def test_attention_row_case_fp8_operands_exact(b):
         dO = np.zeros((1, 1, S, D), np.float32); dO[0, 0, 63, 0] = h
         saved = o.clone(); saved[63 * D] = x
         dq = torch.zeros(S * D, device="cuda"); d_out = torch.zeros(S, device="cuda")
-        b.bsp_attn_bwd(1, 1, S, D, True, c, 1, qd, kd, vd, up(dO, "bf16"), lse, saved, None, None, fp8.E4M3, 0,
-                       b.key(0, 2, 4, 0), dq, None, None, d_out, fp8=f)
+        dOd = up(dO, "bf16")
+        fb = b.attn_fp8(one, one, one, one, 256.0, 1.0, qc, kc, vc, codes_of(dOd, b.E5M2))
+        b.bsp_attn_bwd(1, 1, S, D, True, c, 1, qd, kd, vd, dOd, lse, saved, None, None, fp8.E4M3, 0,
+                       b.key(0, 2, 4, 0), dq, None, None, d_out, fp8=fb)
         return float(dq.cpu().numpy().reshape(S, D)[63, 0])
 
     for sig, tau, t_dev, t_fixed in cells:
