@@ -499,6 +499,11 @@ def test_attention_row_case_fp8_operands_exact(b):
                        b.key(0, 2, 4, 0), dq, None, None, d_out, fp8=fb)
         return float(dq.cpu().numpy().reshape(S, D)[63, 0])
 
+    # the backward of this mode reads the codes: without them it refuses before any launch
+    with pytest.raises(b.BspError):
+        dq0 = torch.zeros(S * D, device="cuda")
+        b.bsp_attn_bwd(1, 1, S, D, True, c, 1, qd, kd, vd, qd, lse, o, None, None, fp8.E4M3, 0, b.key(0, 2, 4, 0), dq0, None,
+                       None, torch.zeros(S, device="cuda"), fp8=f)
     for sig, tau, t_dev, t_fixed in cells:
         sig, tau = float(sig), float(tau)
         for h, want in ((sig * a, float(t_dev)), (a, float(t_fixed))):
