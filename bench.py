@@ -578,6 +578,50 @@ def kernel_table(b, peaks, g):
                 kernels=rows, compute_kernels=compute, diag_status=b.read_diag(diag)["status"])
 
 
+def sharded_draws_line(args, b, torch, dist, world, rank):
+    """The fresh reads of config 5 (gain use and weight use, K = 16) with the draws split over the ranks:
+    every rank prepares the same workload, evaluates its share of the draws, one all-reduce adds the
+    shifted sums, every rank finishes the statistics.  Total work is fixed: strong scaling."""
+    from paper_2609_39813_b200 import workloads
+    from paper_2609_39813_b200.harness import NormLinearGpu, max_over_ranks
+    from paper_2609_39813_b200.sharded import ShardedFreshReads
+    inp = workloads.config5()
+    g = NormLinearGpu(inp)
+    sh = ShardedFreshReads(g, inp.K, rank, world, draw_buffer_draws=16)
+    sh.prepare()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        res = sh.step()
+    barrier()
+    a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        res = sh.step()
+    c.record(stream)
+    barrier()
+    ms = max_over_ranks(a.elapsed_time(c), device="cuda")
+    if rank != 0:
+        return
+    elements = inp.T * inp.C * 2 * inp.K                      # the fresh reads of both uses
+    print(json.dumps(dict(metric=METRIC, value=elements * args.steps / (ms * 1e-3), unit=UNIT, n_gpus=world,
+                          steps=args.steps, warmup=max(args.warmup, 3), ms_per_step=ms / args.steps, higher_is_better=True,
+                          scaling="strong", vs_baseline=None, dtype="f8e4m3/f8e5m2 operands, f32 accumulate",
+                          data="synthetic",
+                          config=dict(workload=WORKLOAD, T=inp.T, C=inp.C, O=inp.O, K=inp.K,
+                                      policies="gain{N} x weight{N}", parallelism="draws/%d" % world,
+                                      draws_per_rank=sh.nd, exchange="one all-reduce (sum) of S1, S2 per step: %d bytes"
+                                      % (4 * 2 * (inp.C + inp.O * inp.C)),
+                                      l2="working set larger than L2"),
+                          verdicts=[int(r.verdict) for r in res], diag_status=b.read_diag(g.diag)["status"])), flush=True)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -604,6 +648,11 @@ def run_ours(args):
     if args.widened_only:
         if rank == 0:
             print(json.dumps(dict(widened=widened_section(b, torch))), flush=True)
+        return
+    if args.shard_draws:
+        sharded_draws_line(args, b, torch, dist, world, rank)
+        if world > 1:
+            dist.destroy_process_group()
         return
 
     inp = workloads.config5()
@@ -800,6 +849,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the sub-objects for configs 2, 3 and 4")
     ap.add_argument("--attention-only", action="store_true", help="run only the config-3 attention section")
     ap.add_argument("--attention-steps", type=int, default=3)
+    ap.add_argument("--shard-draws", action="store_true",
+                    help="instead of replicas: the K draws of the fresh reads split over the ranks, one all-reduce of "
+                         "the shifted sums per step (strong scaling)")
     ap.add_argument("--widened-only", action="store_true",
                     help="run only the b-bit store, coupling, rounded-probabilities and log-softmax checks")
     ap.add_argument("--kernel-table", action="store_true",
