@@ -425,6 +425,7 @@ def test_fp8_operand_mode(b, name):
                    lse, o, None, None, fp8.E4M3, 0, key, dq, dk, dv, d_out, diag, fp8=f)
     assert b.read_diag(diag)["status"] == 0
     oh = o.cpu().numpy().reshape(BH, S, D)
+    worst = {}
     for idx in range(BH):
         want_o, want_lse = attention.forward_output(hat["q"][idx], hat["k"][idx], hat["v"][idx], inp.softmax_scale, cfg["causal"])
         assert _rel(oh[idx], want_o) <= TOL_TC
@@ -433,7 +434,10 @@ def test_fp8_operand_mode(b, name):
                                   oh[idx].astype(np.float64), cfg["causal"], True, 256.0, ds_scale)
         assert _rel(d_out.cpu().numpy().reshape(BH, S)[idx], want["D"]) <= TOL_FP32
         for nm, t in (("dq", dq), ("dk", dk), ("dv", dv)):
-            assert _rel(t.cpu().numpy().reshape(BH, S, D)[idx], want[nm]) <= TOL_TC, (nm, idx)
+            dist_ = _rel(t.cpu().numpy().reshape(BH, S, D)[idx], want[nm])
+            worst[nm] = max(worst.get(nm, 0.0), dist_)
+            assert dist_ <= TOL_TC, (nm, idx, dist_)
+    print("FP8-operand backward, largest relative distance to the oracle per output:", worst)
 
 
 def test_attention_row_case_of_the_paper(b):
