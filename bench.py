@@ -649,6 +649,12 @@ def run_ours(args):
         if rank == 0:
             print(json.dumps(dict(widened=widened_section(b, torch))), flush=True)
         return
+    if args.config2_only:
+        if rank == 0:
+            side2 = torch.cuda.Stream()
+            print(json.dumps(dict(config2=norm_linear_check(b, torch, workloads.config2(), steps=args.steps, side=side2))),
+                  flush=True)
+        return
     if args.shard_draws:
         sharded_draws_line(args, b, torch, dist, world, rank)
         if world > 1:
@@ -852,6 +858,8 @@ def main():
     ap.add_argument("--shard-draws", action="store_true",
                     help="instead of replicas: the K draws of the fresh reads split over the ranks, one all-reduce of "
                          "the shifted sums per step (strong scaling)")
+    ap.add_argument("--config2-only", action="store_true",
+                    help="run only the check of config 2 (the small case: 0.6 GB on the device), --steps times")
     ap.add_argument("--widened-only", action="store_true",
                     help="run only the b-bit store, coupling, rounded-probabilities and log-softmax checks")
     ap.add_argument("--kernel-table", action="store_true",
