@@ -76,6 +76,21 @@ def test_against_the_oracle_on_the_same_draws(b, name):
     assert rel_l2(got["X"], want["X"]) <= 2e-3
 
 
+def test_at_the_390m_shape(b):
+    """Config 2's tensors (T = 4096, C = 1024, O = 4096, bf16, outlier channels), two pairs of forwards:
+    the contractions at the size the benchmark times them, against the oracle on the same draws."""
+    inp = workloads.config2()
+    pairs = 2
+    got, rstd, _ = _run(b, inp, pairs)
+    prep = coupling.prepare(inp.x, inp.gamma, None, inp.W, norm.RMS, inp.eps, rstd32=rstd)
+    want = coupling.run(prep, inp.seed, pairs)
+    assert np.allclose(got["T"], want["T"], rtol=5e-4)
+    assert np.max(np.abs(got["control"] - want["control"])) <= 5e-4 * np.max(np.abs(want["T"]))
+    assert rel_l2(got["gain_total"], want["gain_total"]) <= 5e-4
+    assert rel_l2(got["gain_fresh"], want["gain_fresh"]) <= 5e-4
+    assert rel_l2(got["X"], want["X"]) <= 2e-3
+
+
 def test_closed_forms_and_round_to_nearest(b):
     inp = workloads.config2(T=256, C=128, O=128, K=4, seed=23)
     pairs = 200
