@@ -45,7 +45,8 @@ def _run(b, p, V, law, param, seed, draw0, K):
 @pytest.mark.parametrize("R,n,d,law,param", [(7, 4, 3, 0, 0.125), (5, 3, 2, 1, 0.125), (33, 48, 16, 0, 1.0 / 64),
                                             (9, 200, 64, 1, 1.0 / 512), (3, 256, 64, 0, 1.0 / 256),
                                             # 128 x 64 takes the kernel of its own (eight draws at a time: K = 9 leaves one over)
-                                            (11, 128, 64, 0, 1.0 / 64), (6, 128, 64, 1, 1.0 / 512)])
+                                            (11, 128, 64, 0, 1.0 / 64), (6, 128, 64, 1, 1.0 / 512),
+                                            (600, 128, 64, 0, 1.0 / 64)])       # more blocks than the GPU holds at once
 def test_sums_match_the_oracle_draw_for_draw(b, R, n, d, law, param):
     p, V = _rows(R, n, d, 5 + n)
     K, draw0 = 9, 3
