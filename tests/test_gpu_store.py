@@ -63,6 +63,26 @@ def test_store_codes_and_steps_bit_exact(b, case):
     assert not np.array_equal(want, prep["codes"])
 
 
+def test_store_forward_on_a_width_that_is_no_multiple_of_16(b):
+    """C = 200: a row that does not fill whole groups of 16 columns."""
+    inp = workloads.config2(T=37, C=200, O=16, K=4, seed=31)
+    kind = norm.RMS
+    fw = norm.forward(inp.x, inp.gamma, None, kind, inp.eps)
+    x = up(inp.x, inp.dtype)
+    gamma = up(inp.gamma)
+    rstd = up(fw["rstd"].astype(np.float32))
+    u32 = norm.store_value_fp32(inp.x, inp.gamma, None, kind, fw["rstd"].astype(np.float32), None, None)
+    for bits in (6, 5):
+        s32 = store.steps(u32, bits)
+        codes = torch.zeros(inp.T * inp.C, dtype=torch.int8, device="cuda")
+        steps = torch.zeros(inp.T, device="cuda")
+        b.bsp_store_fwd(b.RMSNORM, x, inp.T, inp.C, gamma, None, rstd, None, bits, b.key(inp.seed, store.TENSOR_U, b.STREAM_FORWARD, 0),
+                        codes, steps)
+        assert np.array_equal(down(steps), s32)
+        want = store.store_codes(u32, s32, inp.seed, philox.STREAM_FORWARD, 0)
+        assert np.array_equal(codes.cpu().numpy().reshape(inp.T, inp.C).astype(np.int64), want)
+
+
 @pytest.mark.parametrize("read", [0, 1, 2, 3])
 def test_copies_and_weight_gradient(b, case, read):
     inp, g, kind, prep, bits, codes, steps = case
