@@ -47,16 +47,23 @@ cp_resid_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ sca
   }
 }
 
-// out[row][0 .. n) = hi(in[row]), out[row][n .. 2n) = lo(in[row]) as bf16; sum (may be NULL) += in.
+// out[row][0 .. n) = hi(in[row]), out[row][n .. 2n) = lo(in[row]) as bf16.  n a multiple of 4: a thread
+// takes four consecutive columns of row blockIdx.x.
 __global__ void __launch_bounds__(256)
 cp_split_rows_kernel(const float* __restrict__ in, int64_t rows, int64_t n, uint16_t* __restrict__ out) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)rows * n) return;
-  const size_t row = i / n, c = i % n;
-  const float v = in[i];
-  const uint32_t hi = float_to_bf16_bits(v);
-  out[row * 2 * n + c] = (uint16_t)hi;
-  out[row * 2 * n + n + c] = (uint16_t)float_to_bf16_bits(v - bf16_bits_to_float(hi));
+  const int64_t c = 4 * ((int64_t)blockIdx.y * blockDim.x + threadIdx.x), row = blockIdx.x;
+  if (c >= n || row >= rows) return;
+  const float4 v = __ldg(reinterpret_cast<const float4*>(in + (size_t)row * n + c));
+  const float f[4] = {v.x, v.y, v.z, v.w};
+  uint32_t hi[4], lo[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    hi[e] = float_to_bf16_bits(f[e]);
+    lo[e] = float_to_bf16_bits(f[e] - bf16_bits_to_float(hi[e]));
+  }
+  uint16_t* o = out + (size_t)row * 2 * n + c;
+  *reinterpret_cast<uint2*>(o) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+  *reinterpret_cast<uint2*>(o + n) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
 }
 
 // Wt2[c][o] = Wt2[c][O + o] = bf16(W[o][c]) and Wb[o][c] = bf16(W[o][c]).
@@ -329,7 +336,7 @@ int bsp_coupling_check(const bsp_coupling_desc_t* op, int pairs, double* T_out, 
     g.sa = 1.f; g.sa_dev = b.scale; g.sb = 1.f; g.mode = EPI_STORE_F32; g.C = b.y[slot]; g.ldc = O; g.diag = diag;
     BSP_TRY(gemm_run(g, st));
     // du = dy W with dy split into hi + lo against [W^T | W^T]
-    cp_split_rows_kernel<<<(unsigned)((no + 255) / 256), 256, 0, st>>>(b.y[slot], T, O, b.ysplit);
+    cp_split_rows_kernel<<<dim3((unsigned)T, (unsigned)((O / 4 + 255) / 256)), 256, 0, st>>>(b.y[slot], T, O, b.ysplit);
     BSP_LAUNCH_CHECK();
     GemmArgs h;
     h.M = T; h.N = C; h.K = 2 * O; h.nb = 1; h.fp8 = false;
