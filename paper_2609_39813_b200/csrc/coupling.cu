@@ -117,23 +117,38 @@ cp_gain_kernel(const float* __restrict__ r, const uint8_t* __restrict__ codes, c
 
 __global__ void __launch_bounds__(256)
 cp_gain_final_kernel(const float* __restrict__ partial, int nslabs, const float* __restrict__ gamma, int64_t C,
-                     float* __restrict__ out) {
+                     float* __restrict__ out, float scale = 1.f, bool accumulate = true) {
   const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= C) return;
   float t = 0.f;
   for (int y = 0; y < nslabs; ++y) t += partial[(size_t)y * C + c];
-  out[c] += t / gamma[c];
+  const float v = t * scale / gamma[c];
+  out[c] = accumulate ? out[c] + v : v;
 }
 
 // partial[b] = { sum (ra - rb)(dua - dub), sum dua * rb } over the block's grid-stride share, in double.
 __global__ void __launch_bounds__(256)
 cp_dots_kernel(const float* __restrict__ ra, const float* __restrict__ rb, const float* __restrict__ dua,
                const float* __restrict__ dub, size_t n, double* __restrict__ partial) {
-  double a = 0.0, b = 0.0;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-    a += (double)(ra[i] - rb[i]) * (double)(dua[i] - dub[i]);
-    b += (double)dua[i] * (double)rb[i];
+  // a thread's share (a few dozen groups of four) in FP32, four chains each; everything above a thread
+  // in double (double arithmetic is scarce on this part: the per-element work stays out of it)
+  float a4[4] = {0.f, 0.f, 0.f, 0.f}, b4[4] = {0.f, 0.f, 0.f, 0.f};
+  const size_t n4 = n / 4;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 xa = __ldg(reinterpret_cast<const float4*>(ra) + i), xb = __ldg(reinterpret_cast<const float4*>(rb) + i);
+    const float4 ya = __ldg(reinterpret_cast<const float4*>(dua) + i), yb = __ldg(reinterpret_cast<const float4*>(dub) + i);
+    a4[0] = fmaf(xa.x - xb.x, ya.x - yb.x, a4[0]); a4[1] = fmaf(xa.y - xb.y, ya.y - yb.y, a4[1]);
+    a4[2] = fmaf(xa.z - xb.z, ya.z - yb.z, a4[2]); a4[3] = fmaf(xa.w - xb.w, ya.w - yb.w, a4[3]);
+    b4[0] = fmaf(ya.x, xb.x, b4[0]); b4[1] = fmaf(ya.y, xb.y, b4[1]);
+    b4[2] = fmaf(ya.z, xb.z, b4[2]); b4[3] = fmaf(ya.w, xb.w, b4[3]);
   }
+  double a = ((double)a4[0] + (double)a4[1]) + ((double)a4[2] + (double)a4[3]);
+  double b = ((double)b4[0] + (double)b4[1]) + ((double)b4[2] + (double)b4[3]);
+  if (blockIdx.x == 0 && threadIdx.x == 0)
+    for (size_t i = n4 * 4; i < n; ++i) {                      // a tail of fewer than four
+      a += (double)(ra[i] - rb[i]) * (double)(dua[i] - dub[i]);
+      b += (double)dua[i] * (double)rb[i];
+    }
   __shared__ double sa[256], sb[256];
   sa[threadIdx.x] = a; sb[threadIdx.x] = b;
   __syncthreads();
@@ -194,26 +209,6 @@ __global__ void cp_accumulate_kernel(const float* __restrict__ a, size_t n, floa
 __global__ void cp_scale_kernel(float* __restrict__ a, size_t n, float f) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) a[i] *= f;
-}
-
-// mean part of the gain error: out[c] = sum_t (sum_r[t][c] / n) (sum_du[t][c] / n) / gamma[c].
-__global__ void __launch_bounds__(256)
-cp_mean_part_kernel(const float* __restrict__ sum_r, const float* __restrict__ sum_du, const float* __restrict__ gamma,
-                    int64_t T, int64_t C, float inv_n2, float* __restrict__ out) {
-  __shared__ float sm[8][33];
-  const int cl = threadIdx.x & 31, rl = threadIdx.x >> 5;
-  const int64_t c = (int64_t)blockIdx.x * 32 + cl;
-  float s = 0.f;
-  if (c < C)
-    for (int64_t t = rl; t < T; t += 8) s = fmaf(sum_r[(size_t)t * C + c], sum_du[(size_t)t * C + c], s);
-  sm[rl][cl] = s;
-  __syncthreads();
-  if (rl == 0 && c < C) {
-    float t = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) t += sm[w][cl];
-    out[c] = t * inv_n2 / gamma[c];
-  }
 }
 
 constexpr int kCpDotBlocks = 296;
@@ -385,7 +380,10 @@ int bsp_coupling_check(const bsp_coupling_desc_t* op, int pairs, double* T_out, 
     BSP_LAUNCH_CHECK();
   }
   const float inv_n = 1.0f / (float)(2 * pairs);
-  cp_mean_part_kernel<<<gcol, 256, 0, st>>>(b.sum_r, b.sum_du, op->gamma, T, C, inv_n * inv_n, b.gain_mean_part);
+  // mean part of the gain error, sum_t (sum_r / n) (sum_du / n) / gamma: the same column sums over row slabs
+  cp_gain_kernel<BSP_E4M3><<<ggain, 256, 0, st>>>(b.sum_r, nullptr, b.scale, b.u, b.sum_du, T, C, slab_rows, b.gain_partial, nullptr);
+  cp_gain_final_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(b.gain_partial, nslabs, op->gamma, C, b.gain_mean_part,
+                                                                     inv_n * inv_n, false);
   BSP_LAUNCH_CHECK();
   // sums over the forwards / pairs to averages
   cp_scale_kernel<<<(unsigned)((C + 255) / 256), 256, 0, st>>>(b.gain_total, (size_t)C, inv_n);
