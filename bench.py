@@ -302,6 +302,8 @@ def attention_section(b, peaks, steps=3):
     b.bsp_attn_dterm(B, H, S, D, dO, o, None, None, b.E4M3, b.READ_ORIGINAL, b.key(0, 2, 4), 0, 1, dterm)
     ms_dkv = timed(torch, stream, lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, c, q, k, v, dO, lse, dterm, None, dk, dv, diag))
     ms_dq = timed(torch, stream, lambda: b.bsp_attn_bwd_dterm(B, H, S, D, True, c, q, k, v, dO, lse, dterm, dq, None, None, diag))
+    # the one-kernel form: S, dP and the exponentials once per score tile, dQ by reduce-adds (its clearing included)
+    ms_one = timed(torch, stream, lambda: b.bsp_attn_bwd_dterm_fused(B, H, S, D, True, c, q, k, v, dO, lse, dterm, dq, dk, dv, diag))
     # the D pre-pass alone under its three reads (HBM-bound for U and R: dO read once, the copy of O
     # read once; the fresh read is bound by the generator: one word per element and draw)
     amax_o, scales_o = torch.zeros(B * H, device="cuda"), torch.zeros(B * H, device="cuda")
@@ -345,7 +347,8 @@ def attention_section(b, peaks, steps=3):
     return dict(workload="cfg3_causal_attention_bwd", B=B, H=H, S=S, D=D, K=K, data="seeded host recipe",
                 ms_per_check=mode_b["ms_per_check"], check_elements_per_s=mode_b["check_elements_per_s"],
                 verdicts=mode_b["verdicts"], bf16_operands=mode_b, fp8_operands=mode_a,
-                bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3, dterm=dterm_rows,
+                bwd_dkv_us=ms_dkv * 1e3, bwd_dq_us=ms_dq * 1e3, bwd_one_kernel_us=ms_one * 1e3,
+                bwd_one_kernel_algorithmic_frac=5 * prod / (ms_one * 1e-3) / 1e12 / peak, dterm=dterm_rows,
                 fwd_stats_us=ms_fwd * 1e3, quantize_one_tensor_us=ms_quant * 1e3,
                 bwd_fp8_operands_us=ms_fp8 * 1e3,   # D pre-pass + dK/dV + dQ kernels, FP8-operand mode
                 roofline=dict(bound="tensor", kernel="attn_kernel<dK/dV> + attn_kernel<dQ> (bf16 operands)",

@@ -406,6 +406,15 @@ int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_sc
                        const float* lse, const float* dterm, float* dq, float* dk, float* dv,
                        bsp_diag_t* diag, void* stream);
 
+/* The same backward (BF16 operands, all three gradients required) in one kernel: every score tile's
+ * S, dP and exponentials are formed once and serve dV, dK and dQ; the tile's share of dQ is added to
+ * dq in device memory, which this call clears first.  dk and dv are bit-reproducible; dq is up to the
+ * order of its FP32 additions (S/128 shares per element).  Arguments as bsp_attn_bwd_dterm. */
+int bsp_attn_bwd_dterm_fused(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q,
+                             const void* k, const void* v, const void* dO, int dt, const float* lse,
+                             const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag,
+                             void* stream);
+
 /* Backward under a read policy at the D use: bsp_attn_dterm (draw key.draw) into d_out[B,H,S]
  * (required), then bsp_attn_bwd_dterm.  fp8_operands = 0: fp8 must be NULL; fp8_operands = 1: fp8
  * gives the operand scales (BSP_ERR_ARG when the flag and the pointer disagree). */

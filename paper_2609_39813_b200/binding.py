@@ -147,6 +147,7 @@ _SIGNATURES = {
     "bsp_attn_dterm": (_I, [_I, _I, _I, _I, _P, _I, _P, _P, _P, _P, _I, _I, Key, _I, _I, _P, _P, _P]),
     "bsp_attn_bwd_dterm": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _P,
                                 _P, _P]),
+    "bsp_attn_bwd_dterm_fused": (_I, [_I, _I, _I, _I, _I, _F, _P, _P, _P, _P, _I, _P, _P, _P, _P, _P, _P, _P]),
     "bsp_attn_bwd": (_I, [_I, _I, _I, _I, _I, _F, _I, _P, _P, _P, _P, _I, C.POINTER(AttnFp8), _P, _P, _P, _P, _I, _I,
                           Key, _P, _P, _P, _P, _P, _P]),
     "bsp_attn_quantize": (_I, [_P, _I, _SZ, _I, _P, _P, _P, _P, _P, _P]),
@@ -421,6 +422,13 @@ def bsp_attn_bwd_dterm(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, lse, dte
     check(lib().bsp_attn_bwd_dterm(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), ptr(dO),
                                    dtype_code(q), _fp8ref(fp8), ptr(lse), ptr(dterm), ptr(dq), ptr(dk), ptr(dv),
                                    ptr(diag), _st(stream)), "bsp_attn_bwd_dterm")
+
+
+def bsp_attn_bwd_dterm_fused(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, lse, dterm, dq, dk, dv, diag=None,
+                             stream=None):
+    check(lib().bsp_attn_bwd_dterm_fused(B, H, S, Dh, int(causal), softmax_scale, ptr(q), ptr(k), ptr(v), ptr(dO),
+                                         dtype_code(q), ptr(lse), ptr(dterm), ptr(dq), ptr(dk), ptr(dv), ptr(diag),
+                                         _st(stream)), "bsp_attn_bwd_dterm_fused")
 
 
 def bsp_attn_bwd(B, H, S, Dh, causal, softmax_scale, fp8_operands, q, k, v, dO, lse, o_orig, o_codes, o_scales,

@@ -49,6 +49,7 @@ struct AttnParams {
   const float* dterm;            // [BH*S]  (DKV, DQ)
   float* out0;                   // DKV: dV   DQ: dQ   FWD: O      [BH*S*64]
   float* out1;                   // DKV: dK                         [BH*S*64]
+  float* out2;                   // DKV with the fused dQ: dQ (zero at launch), else NULL
   float* lse_out;                // FWD
   // Monte-Carlo epilogue (DQ, and DKV without dV): instead of storing the gradient g, the kernel adds
   // g - mc_ref to out0 and (g - mc_ref)^2 to out1 (the running sums S1, S2 of that gradient)
@@ -89,11 +90,19 @@ __device__ __forceinline__ uint32_t f8_grid_bf16x2(float lo, float hi) {
 // ND (Monte-Carlo dQ and dK kernels only): draws per launch.  S, dP and P do not depend on the correction
 // term, so with ND = 2 a step forms them once and builds two dS operands, one per draw's D (at
 // p.dterm and p.dterm + BH*S), into two accumulators; the epilogue adds both draws to the sums.
-template <int MODE, bool FP8, bool DV, bool MC, int ND>
+// DQF (dK/dV mode, BF16 operands only): the same CTA also forms the step's share of dQ, dS_ij K_j, and
+// adds it to dQ in global memory (one tiled bulk reduce-add per step and column half), so S, dP and
+// the exponentials are formed once per score tile for all three gradients.  dS^T then goes to
+// shared memory instead of tensor memory (K-major A operand of dK, MN-major A operand of dQ) and
+// the tile ring has two stages.  dQ must hold zeros at launch; the order of its FP32 additions is
+// not fixed, so dQ is not bit-reproducible in this form.
+template <int MODE, bool FP8, bool DV, bool MC, int ND, bool DQF = false>
 __global__ void __launch_bounds__(kAtThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-            const __grid_constant__ CUtensorMap tm_o0, const __grid_constant__ CUtensorMap tm_o1, AttnParams p) {
+            const __grid_constant__ CUtensorMap tm_o0, const __grid_constant__ CUtensorMap tm_o1,
+            const __grid_constant__ CUtensorMap tm_o2, AttnParams p) {
+  static_assert(!DQF || (MODE == AT_DKV && !FP8 && DV && !MC && ND == 1), "fused dQ: plain BF16 dK/dV kernel only");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -111,7 +120,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // streamed-tile ring: the backward modes have no P / dS buffers in shared memory (those operands
   // live in tensor memory), so their ring takes a third stage there, and the last 32 KB of that
   // space stage the second output of the dK/dV epilogue
-  constexpr uint32_t kStg = MODE == AT_FWD ? 2u : 3u;
+  constexpr uint32_t kStg = (MODE == AT_FWD || DQF) ? 2u : 3u;
+  const uint32_t dst_buf = str0 + 2u * 2u * kAtTile;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
+  const uint32_t dst_buf_unused = 0;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
   const uint32_t stage2 = str0 + 3u * 2u * kAtTile;
   uint8_t* gen = smem_raw + (base - raw);
   uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
@@ -132,6 +143,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // needs, per query (a column of S^T), delta = D_first - D_second, kept as FP32 in three buffers of
   // 128 values that the threads writing the X tiles fill alongside them
   const uint32_t delta0 = bars + 2304;
+  // DQF: the step's dQ share is complete / has been read out of tensor memory
+  const uint32_t b_dq_full = bars + 3848, b_dq_free = bars + 3856;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Persistent CTA: work items w = item_at(0), item_at(1), ... of nblk * BH, heavy blocks first
@@ -172,6 +185,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     for (uint32_t s = 0; s < kStg; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
     for (uint32_t s = 0; s < 3; ++s) mbar_init(b_bias + 8 * s, 8);
     mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
+    mbar_init(b_dq_full, 1); mbar_init(b_dq_free, 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -188,12 +202,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // two draws (dQ kernel): the second draw's dS operand takes the P columns (no product reads P
   // there) and its accumulator the second half of the accumulator buffer
   const uint32_t t_ds2 = tmem + 256;
+  const uint32_t t_dq = tmem + 320;                           // DQF: the step's dQ share (dS^T is in shared memory)
   const uint32_t t_accbase = MODE == AT_FWD ? tmem + 256 : tmem + 384;
   constexpr bool kAccDouble = MODE == AT_FWD;   // accumulators double-buffered across items
 
   // instruction descriptors (bf16 operands, FP32 accumulation)
   const uint32_t id_sdp = make_idesc(1u, 1u, 128, 128);                                   // A, B K-major
   const uint32_t id_kmn = make_idesc(1u, 1u, 128, 64) | (1u << 16);                       // A K-major, B MN-major
+  const uint32_t id_mn = make_idesc(1u, 1u, 128, 64) | (1u << 15) | (1u << 16);           // A, B MN-major
   // FP8-operand mode of the backward: every product is an FP8 tensor-core product (kind::f8f6f4) on the
   // codes themselves.  The streamed and resident tiles are 128 rows of 64 bytes (64-byte swizzle), a
   // K step is 32 elements, and P (E4M3) and dS (E5M2) go back into tensor memory four codes per column.
@@ -340,6 +356,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
             for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
           }
+        } else if (DQF) {
+          // dV += P^T dO with P^T from tensor memory; dK += dS^T Q with dS^T K-major from shared memory
+          // (two halves of 64 queries, four K = 16 steps each); then the step's dQ share = dS K_j: the same
+          // buffer read MN-major (128 queries wide, 16 keys per step), K_j = the resident tile, MN-major
+          const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t a = make_smem_desc(dst_buf + (k >> 2) * 16384u + (k & 3) * 32u);
+            tc_mma<false>(t_acc1, a, bq + 128u * k, id_kmn, first | (k != 0));
+          }
+          // the share of the step before has left tensor memory
+          if (!mbar_wait(b_dq_free, (jg & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t ads = make_smem_desc_mn(dst_buf, 16384u), bk = make_smem_desc_mn(res0, 16384u);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) tc_mma<false>(t_dq, ads + 128u * k, bk + 128u * k, id_mn, k != 0);
+          tc_commit(b_dq_full);
         } else if (MODE == AT_DKV) {
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
           // queries), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
@@ -406,6 +441,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     bool ok = true;
     uint32_t bias_written = 0;                                // DKV: rows of the X tiles written so far (global steps)
     bool store_pending = false;                               // warp 2, lane 0: an epilogue's bulk stores are in flight
+    bool red_pending = false;                                 // warp 2, lane 0 (DQF): a dQ share's reduce-adds are in flight
     uint32_t itg = 0;                                         // step counter across items
     int item = 0;
     for (int w = item_at(0); w < nitems && ok; w = item_at(++item)) {
@@ -504,6 +540,37 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     // FWD: the shift in use (log2 units) and the sum of exp2(c2 s - shift) of this row and column half
     float run_m = lse_known ? lse2 : -INFINITY, run_l = 0.f;
+    // DQF: the dQ share of global step jd (queries of block qblk): tensor memory -> registers (rows =
+    // queries, this thread's 32 columns of half h) -> scaled by c into the swizzled staging boxes ->
+    // two tiled bulk reduce-adds into dQ.  The staging buffer is the one the epilogue uses for dK.
+    auto drain_dq = [&](uint32_t jd, int qblk) -> bool {
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(b_dq_full, jd & 1u, abort_flag))) return false;
+      tc_fence_after();
+      uint32_t a[32];
+      tmem_ld32(t_dq + lane_off + h * 32, a);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_dq_free);
+      // the bulk operations that last read the staging buffer (the share before, or an epilogue) are done with it
+      if (warp == kAtSoftWarp0 && lane == 0 && (store_pending || red_pending)) tma_store_wait_read();
+      named_bar_sync(2, 256);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stage2 + off), "f"(__uint_as_float(a[4 * t]) * p.c),
+                     "f"(__uint_as_float(a[4 * t + 1]) * p.c), "f"(__uint_as_float(a[4 * t + 2]) * p.c),
+                     "f"(__uint_as_float(a[4 * t + 3]) * p.c) : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      named_bar_sync(4, 256);
+      if (warp == kAtSoftWarp0 && lane == 0) {
+        tma_reduce_add_3d(&tm_o2, stage2, 0, qblk * AT_BLK, bh);
+        tma_reduce_add_3d(&tm_o2, stage2 + 16384u, 32, qblk * AT_BLK, bh);
+        tma_store_commit();
+        red_pending = true;
+      }
+      return true;
+    };
     for (int it = 0; it < total && ok; ++it) {
       const int step = it_begin + (it % nsteps);
       const uint32_t ip = (itg + (uint32_t)it) & 1u;
@@ -789,8 +856,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
+          // DQF: 32 of the row's 64 dS^T values (four 16-byte chunks of eight queries) into row r of
+          // half h of the shared dS^T buffer, 128-byte swizzle: chunk index t ^ (r & 7)
+          auto st_half_smem = [&](int half, const uint32_t (&wv)[16]) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)((half * 4 + t) ^ (r & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst_buf + off), "r"(wv[4 * t]), "r"(wv[4 * t + 1]),
+                           "r"(wv[4 * t + 2]), "r"(wv[4 * t + 3]) : "memory");
+            }
+          };
           if (DV) st_half(t_p, 0, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
-          st_half(t_ds, 0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
+          if (DQF) st_half_smem(0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
+          else st_half(t_ds, 0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
           if (!edge) {
 #pragma unroll
             for (int j = 32; j < 64; j += 2) pair_at(j, false);
@@ -799,14 +877,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             for (int j = 32; j < 64; j += 2) pair_at(j, true);
           }
           if (DV) st_half(t_p, 1, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
-          st_half(t_ds, 1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
+          if (DQF) st_half_smem(1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
+          else st_half(t_ds, 1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
           tmem_wait_st();
           tc_fence_before();
         }
       }
-      if (MODE == AT_FWD) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (MODE == AT_FWD || DQF) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(b_pds_ready);
+      // DQF: the dQ share of the step before, now complete (its products were committed ahead of the
+      // operands' release that this step has already waited for), goes out while this step's products run
+      if (DQF && it > 0) {
+        ok = drain_dq(itg + (uint32_t)it - 1u, it_begin + it - 1);
+        if (!ok) break;
+      }
       if (it == 0 && warp == kAtSoftWarp0 && lane == 0 && store_pending) {
         // the previous item's output has left its staging buffer by now: hand the resident-tile
         // buffer it used back to the TMA producer
@@ -821,6 +906,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         ++bias_written;
       }
     }
+    if (DQF && ok) ok = drain_dq(itg + (uint32_t)total - 1u, it_begin + total - 1);   // the last step's share
     itg += (uint32_t)total;
     float fwd_w0 = 1.f, fwd_w1 = 1.f;                         // FWD: weights of the two halves' accumulators
     if (MODE == AT_FWD) {
@@ -867,6 +953,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tma_store_wait_read();
         mbar_arrive(b_res_empty + 8 * (rbi ^ 1u));
         store_pending = false;
+      }
+      if (DQF && warp == kAtSoftWarp0 && lane == 0 && red_pending) {
+        tma_store_wait_read();                                // the last share's reduce-adds have read the staging buffer
+        red_pending = false;
       }
       if (MODE == AT_DKV || mc) named_bar_sync(3, 256);       // ... before anyone writes the second staging buffer again
       float rv[32];                                           // this thread's 32 reference values
@@ -1090,12 +1180,14 @@ attn_dterm_kernel(const void* __restrict__ dO, const float* __restrict__ o_orig,
 
 // ------------------------------------------------------------------------------- host side
 
-template <int MODE, bool FP8, bool DV, bool MC = false, int ND = 1>
+template <int MODE, bool FP8, bool DV, bool MC = false, int ND = 1, bool DQF = false>
 static int launch_attn_mode(const void* q, const void* k, const void* v, const void* dO, AttnParams p, cudaStream_t st) {
-  CUtensorMap mq, mk, mv, mdo, mo0, mo1;
+  CUtensorMap mq, mk, mv, mdo, mo0, mo1, mo2;
   int rc;
+  if (DQF && !p.out2) return BSP_ERR_ARG;
   if ((rc = make_out_map(&mo0, p.out0 ? p.out0 : p.out1, p.BH, p.S)) != BSP_OK) return rc;
   if ((rc = make_out_map(&mo1, p.out1 ? p.out1 : p.out0, p.BH, p.S)) != BSP_OK) return rc;
+  if ((rc = make_out_map(&mo2, DQF ? p.out2 : (p.out0 ? p.out0 : p.out1), p.BH, p.S)) != BSP_OK) return rc;
   if (FP8 && MODE != AT_FWD) {
     // the backward of the FP8-operand mode loads the codes
     if (!p.cq || !p.ck || !p.cv || !p.cdo) return BSP_ERR_ARG;
@@ -1113,7 +1205,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
   static std::atomic<bool> attr_set_dev[kMaxDevices];       // per kernel instantiation and device
   std::atomic<bool>& attr_set = attr_set_dev[device_slot()];
   if (!attr_set.load(std::memory_order_acquire)) {
-    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC, ND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
+    BSP_CHECK_CUDA(cudaFuncSetAttribute(attn_kernel<MODE, FP8, DV, MC, ND, DQF>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmem));
     attr_set.store(true, std::memory_order_release);
   }
   // persistent: one CTA per SM walks the (block, head) items, heaviest first
@@ -1123,7 +1215,7 @@ static int launch_attn_mode(const void* q, const void* k, const void* v, const v
     nsm = sm_count;
   const int64_t nitems = (int64_t)p.nblk * p.BH;
   const unsigned grid = (unsigned)(nitems < nsm ? nitems : nsm);
-  attn_kernel<MODE, FP8, DV, MC, ND><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, p);
+  attn_kernel<MODE, FP8, DV, MC, ND, DQF><<<grid, kAtThreads, kAtSmem, st>>>(mq, mk, mv, mdo, mo0, mo1, mo2, p);
   BSP_LAUNCH_CHECK();
   return BSP_OK;
 }
@@ -1163,7 +1255,7 @@ int attn_fwd_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, 
   if (rc != BSP_OK) return rc;
   if (!q || !k || !v || !o || (!lse && !lse_known)) return BSP_ERR_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BSP_ERR_ALIGN;
-  AttnParams p;
+  AttnParams p{};
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
   p.lse = lse_known; p.dterm = nullptr; p.out0 = o; p.out1 = nullptr; p.lse_out = lse; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
@@ -1242,7 +1334,7 @@ int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_s
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) ||
       !aligned16(dv))
     return BSP_ERR_ALIGN;
-  AttnParams p;
+  AttnParams p{};
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
   p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
@@ -1256,6 +1348,27 @@ int attn_bwd_dterm_impl(int B, int H, int S, int Dh, int causal, float softmax_s
     if ((rc = launch_attn<AT_DQ>(q, k, v, dO, p, st)) != BSP_OK) return rc;
   }
   return BSP_OK;
+}
+
+// The same backward in one kernel: the dK/dV kernel also forms each score tile's share of dQ and adds
+// it to dQ in global memory (BF16 operands, all three gradients).  dQ is cleared here first.
+int attn_bwd_fused_impl(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                        const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq, float* dk,
+                        float* dv, bsp_diag_t* diag, void* stream) {
+  int rc = check_attn_shape(B, H, S, Dh, dt);
+  if (rc != BSP_OK) return rc;
+  if (!q || !k || !v || !dO || !lse || !dterm || !dq || !dk || !dv) return BSP_ERR_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dO) || !aligned16(dq) || !aligned16(dk) ||
+      !aligned16(dv))
+    return BSP_ERR_ALIGN;
+  AttnParams p{};
+  p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
+  p.lse = lse; p.dterm = dterm; p.lse_out = nullptr; p.diag = diag; p.mc_ref = nullptr; p.nd = 1;
+  if ((rc = set_fp8(p, nullptr)) != BSP_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  BSP_CHECK_CUDA(cudaMemsetAsync(dq, 0, (size_t)B * H * S * AT_D * sizeof(float), st));
+  p.out0 = dv; p.out1 = dk; p.out2 = dq;
+  return launch_attn_mode<AT_DKV, false, true, false, 1, true>(q, k, v, dO, p, st);
 }
 
 // nd (1 or 2) draws of the D use for dQ and dK with the Monte-Carlo epilogue: the kernels add g - ref
@@ -1273,7 +1386,7 @@ int attn_bwd_dterm_mc(int B, int H, int S, int Dh, int causal, float softmax_sca
   if (nd < 1 || nd > 2) return BSP_ERR_ARG;
   if (!aligned16(ref_dq) || !aligned16(ref_dk) || !aligned16(S1q) || !aligned16(S2q) || !aligned16(S1k) || !aligned16(S2k))
     return BSP_ERR_ALIGN;
-  AttnParams p;
+  AttnParams p{};
   p.BH = B * H; p.S = S; p.nblk = (S + AT_BLK - 1) / AT_BLK; p.causal = causal ? 1 : 0; p.c = softmax_scale;
   p.lse = lse; p.lse_out = nullptr; p.diag = diag;
   if ((rc = set_fp8(p, f)) != BSP_OK) return rc;
@@ -1320,6 +1433,12 @@ int bsp_attn_bwd_dterm(int B, int H, int S, int Dh, int causal, float softmax_sc
                        const float* dterm, float* dq, float* dk, float* dv, bsp_diag_t* diag, void* stream) {
   return attn_bwd_dterm_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, fp8, lse, dterm, dq, dk, dv, diag,
                              stream);
+}
+
+int bsp_attn_bwd_dterm_fused(int B, int H, int S, int Dh, int causal, float softmax_scale, const void* q, const void* k,
+                             const void* v, const void* dO, int dt, const float* lse, const float* dterm, float* dq,
+                             float* dk, float* dv, bsp_diag_t* diag, void* stream) {
+  return attn_bwd_fused_impl(B, H, S, Dh, causal, softmax_scale, q, k, v, dO, dt, lse, dterm, dq, dk, dv, diag, stream);
 }
 
 int bsp_attn_bwd(int B, int H, int S, int Dh, int causal, float softmax_scale, int fp8_operands, const void* q,

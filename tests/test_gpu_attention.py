@@ -230,6 +230,44 @@ def test_backward_is_deterministic_and_dv_ignores_the_read(b, case):
     assert not torch.equal(outs[0][0], outs[2][0])                         # dQ does
 
 
+def test_one_kernel_backward(b, case):
+    """The one-kernel form of the backward (every score tile's S, dP and exponentials formed once,
+    the tile's share of dQ added to dQ in device memory) against the plain float64 oracle, and against
+    the two-kernel form: dK and dV come from the same arithmetic in the same order; dQ is the same
+    sum of per-key-block shares taken in another order (each share rounded to FP32 on its way out)."""
+    inp, g = case
+    B, H, S, D = inp.B, inp.H, inp.S, inp.D
+    n = B * H * S * D
+    dterm = torch.zeros(B * H * S, device="cuda")
+    b.bsp_attn_dterm(B, H, S, D, g.dO, g.o, None, None, fp8.E4M3, b.READ_ORIGINAL,
+                     b.key(inp.seed, check.TENSOR_O, b.STREAM_ATTN_D, 0), 0, 1, dterm)
+    two = [torch.zeros(n, device="cuda") for _ in range(3)]
+    b.bsp_attn_bwd_dterm(B, H, S, D, g.causal, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, dterm, *two)
+    for rep in range(2):
+        one = [torch.full((n,), float("nan"), device="cuda") for _ in range(3)]
+        diag = b.new_diag()
+        b.bsp_attn_bwd_dterm_fused(B, H, S, D, g.causal, inp.softmax_scale, g.q, g.k, g.v, g.dO, g.lse, dterm, *one,
+                                   diag=diag)
+        assert b.read_diag(diag)["status"] == 0
+        assert torch.isfinite(one[0]).all()
+        assert _rel(one[1].cpu().numpy(), two[1].cpu().numpy()) <= 1e-6       # dK
+        assert torch.equal(one[2], two[2])                                     # dV: same products, same order
+        # dQ: the two-kernel form takes its dS from S = Q K^T with LSE subtracted in FP32, this one from
+        # S^T with LSE entering through the product; where the bf16 rounding of dS falls the other way
+        # an element moves by 2^-9 of itself
+        assert _rel(one[0].cpu().numpy(), two[0].cpu().numpy()) <= 2e-4
+    o = g.o.cpu().numpy().reshape(B * H, S, D)
+    got = {n_: t.cpu().numpy().reshape(B * H, S, D) for n_, t in zip(("dq", "dk", "dv"), one)}
+    for idx, q, k, v, dO in _slices(inp):
+        prep = check.prepare_attention_slice(q, k, v, dO, inp.softmax_scale, inp.seed, idx, g.causal, o32=o[idx])
+        copy = check.attention_d_copy(prep, 0, inp.seed, 0)
+        want = attention.backward(q, k, v, dO, inp.softmax_scale, copy, g.causal)
+        for name in ("dq", "dk", "dv"):
+            dist = _rel(got[name][idx], want[name])
+            print("one-kernel backward vs plain oracle: %s slice %d rel-L2 %.3e" % (name, idx, dist))
+            assert dist <= TOL_TC_BF16_OPERANDS, (name, idx, dist)
+
+
 def _attn_desc(b, g, inp, K, mask, fp8_operands=0, p_scale=256.0, ds_scale=1.0):
     d = b.AttnDesc()
     d.B, d.H, d.S, d.Dh, d.causal, d.softmax_scale, d.dtype = inp.B, inp.H, inp.S, inp.D, 1, inp.softmax_scale, b.BF16
