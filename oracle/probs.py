@@ -189,10 +189,15 @@ OPERATORS = ("J(q)", "J(f)", "K(f)", "J2(f,b)", "J2(q,b)")        # read at the 
 V_READS = ("u", "f")                                               # read at the gradient of V (p_q is exact)
 
 
-def rounded(p32, law: int, param: float, seed: int, stream: int, draw: int) -> np.ndarray:
-    """One rounding of every entry of p32[R, n] (float64 result)."""
+def rounded(p32, law: int, param: float, seed: int, stream: int, draw: int, first_row: int = 0) -> np.ndarray:
+    """One rounding of every entry of p32[R, n] (float64 result).  The rows are rows first_row ..
+    first_row + R - 1 of the whole tensor: an entry's word is keyed by its index there."""
     p32 = np.asarray(p32, dtype=np.float32)
-    w = philox.tensor_words(seed, TENSOR_P, stream, draw, p32.size).reshape(p32.shape)
+    if first_row == 0:
+        w = philox.tensor_words(seed, TENSOR_P, stream, draw, p32.size).reshape(p32.shape)
+    else:
+        idx = np.arange(first_row * p32.shape[1], (first_row + p32.shape[0]) * p32.shape[1], dtype=np.uint64)
+        w = philox.element_words(seed, TENSOR_P, stream, draw, idx).reshape(p32.shape)
     if law == LAW_SIGN:
         return p32.astype(np.float64) + np.where((w >> np.uint64(31)) & np.uint64(1), param, -param)
     g = np.float32(param)
@@ -215,9 +220,10 @@ def apply_J2(a, b, dp):
     return 0.5 * (a + b) * dp - 0.5 * (a * np.sum(b * dp, axis=1, keepdims=True) + b * np.sum(a * dp, axis=1, keepdims=True))
 
 
-def mc_sums(p32, V, law: int, param: float, seed: int, K: int, draw0: int = 0):
+def mc_sums(p32, V, law: int, param: float, seed: int, K: int, draw0: int = 0, first_row: int = 0):
     """Sums over draws draw0 .. draw0 + K - 1 of the errors Delta_s (per operator of OPERATORS,
-    [5, R, n]) and Delta_V (per read of V_READS, [2, R, n, d]), and of the squares of Delta_s."""
+    [5, R, n]) and Delta_V (per read of V_READS, [2, R, n, d]), and of the squares of Delta_s.
+    first_row: where these rows sit in the whole tensor (rows are independent but for their keys)."""
     p = np.asarray(p32, dtype=np.float32).astype(np.float64)
     V = np.asarray(V, dtype=np.float64)
     R, n = p.shape
@@ -225,9 +231,9 @@ def mc_sums(p32, V, law: int, param: float, seed: int, K: int, draw0: int = 0):
     ds2 = np.zeros_like(ds)
     dV = np.zeros((len(V_READS), R, n, V.shape[1]))
     for k in range(draw0, draw0 + K):
-        pq = rounded(p32, law, param, seed, 0, k)
-        pf = rounded(p32, law, param, seed, 1, k)
-        pb = rounded(p32, law, param, seed, 2, k)
+        pq = rounded(p32, law, param, seed, 0, k, first_row)
+        pf = rounded(p32, law, param, seed, 1, k, first_row)
+        pb = rounded(p32, law, param, seed, 2, k, first_row)
         h = pq @ V                                  # o = V^T p_q row by row; h = o
         dp = h @ V.T
         ref = apply_J(p, dp)

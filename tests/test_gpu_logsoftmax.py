@@ -68,6 +68,30 @@ def test_registered_statements(b, eps):
         assert abs(s[0].mean / (eps * eps / 2) - 1) >= 0.01 and abs(s[2].mean / (-eps * eps) - 1) >= 0.02
 
 
+def test_vocabulary_sized_rows_on_sampled_trials(b):
+    """The size `bench.py` times beside the paper's (256 rows of 8192 classes, 256 trials, eps 0.1,
+    seeded inputs of the same law): sampled trials against the oracle's per-trial statistics, and the
+    summary against the oracle's summary of the GPU's own per-trial values."""
+    rows, classes, trials, eps = 256, 8192, 256, 0.1
+    rng = np.random.default_rng(1926)
+    logits = rng.standard_normal((rows, classes)).astype(np.float32)
+    target = rng.integers(0, classes, rows).astype(np.int32)
+    pt = torch.zeros(trials * 6, device="cuda")
+    ws = b.workspace(b.bsp_lsm_check_workspace_bytes(rows, classes, trials))
+    stats = b.bsp_lsm_check(torch.from_numpy(logits).cuda(), torch.from_numpy(target).cuda(), rows, classes, eps, trials,
+                            1926, ls.TENSOR_S, pt, ws)
+    got = pt.cpu().numpy().reshape(trials, 6).astype(np.float64)
+    for t in (0, 1, 100, 255):
+        want = ls.trial_statistics(logits, target, eps, 1926, t)
+        scale = np.maximum(np.abs(want), eps * eps)
+        assert np.max(np.abs(got[t] - want) / scale) <= 2e-4, (t, got[t], want)
+    full = np.concatenate([got, (got[:, 0] - got[:, 1])[:, None], (got[:, 2] - got[:, 3])[:, None]], axis=1)
+    mean, se, z = ls.summarise(full)
+    for c in range(8):
+        assert abs(stats[c].mean - mean[c]) <= 1e-5 * max(abs(mean[c]), eps * eps)
+        assert abs(stats[c].se - se[c]) <= 1e-3 * se[c] + 1e-12
+
+
 def test_argument_errors(b):
     x, y = torch.zeros(8 * 6, device="cuda"), torch.zeros(8, dtype=torch.int32, device="cuda")
     ws = b.workspace(4096)

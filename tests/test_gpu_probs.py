@@ -62,6 +62,36 @@ def test_sums_match_the_oracle_draw_for_draw(b, R, n, d, law, param):
         assert np.max(np.abs(dV[i] - want_dV[i])) <= 2e-5 * scale
 
 
+def test_bench_size_on_sampled_rows(b):
+    """The size `bench.py` times (16384 rows of 128 probabilities, d = 64, grid 1/64, 256 draws; rows
+    drawn by the same recipe): blocks of rows from the start, the middle and the end of the tensor
+    against the oracle on those rows alone, keyed by their place in the whole tensor."""
+    R, n, d, K = 16384, 128, 64, 256
+    rng = np.random.default_rng(3003)
+    sc = rng.standard_normal((R, n)) * 1.5
+    p = np.exp(sc - sc.max(1, keepdims=True))
+    p = (p / p.sum(1, keepdims=True)).astype(np.float32)
+    V = (rng.standard_normal((n, d)) / np.sqrt(d)).astype(np.float32)
+    ds = torch.zeros(5 * R * n, device="cuda")
+    sq = torch.zeros(5 * R * n, device="cuda")
+    dV = torch.zeros(2 * R * n * d, device="cuda")
+    b.bsp_probs_mc(torch.from_numpy(p).cuda(), torch.from_numpy(V).cuda(), R, n, d, 0, 1.0 / 64, 3003, probs.TENSOR_P, 0, K,
+                   ds, sq, dV)
+    torch.cuda.synchronize()
+    ds, sq, dV = ds.view(5, R, n), sq.view(5, R, n), dV.view(2, R, n, d)
+    for r0, m in ((0, 3), (8191, 3), (R - 2, 2)):
+        want_ds, want_sq, want_dV = probs.mc_sums(p[r0:r0 + m], V, 0, 1.0 / 64, 3003, K, 0, first_row=r0)
+        got_ds = ds[:, r0:r0 + m].cpu().numpy().astype(np.float64)
+        got_sq = sq[:, r0:r0 + m].cpu().numpy().astype(np.float64)
+        got_dV = dV[:, r0:r0 + m].cpu().numpy().astype(np.float64)
+        for i in range(5):
+            # FP32 sums of 256 errors
+            assert np.max(np.abs(got_ds[i] - want_ds[i])) <= 1e-4 * (np.max(np.abs(want_ds[i])) + 1e-30), (r0, i)
+            assert np.max(np.abs(got_sq[i] - want_sq[i])) <= 3e-4 * (np.max(np.abs(want_sq[i])) + 1e-30), (r0, i)
+        for i in range(2):
+            assert np.max(np.abs(got_dV[i] - want_dV[i])) <= 1e-4 * (np.max(np.abs(want_dV[i])) + 1e-30), (r0, i)
+
+
 def test_cells_of_the_paper_on_the_gpu(b):
     """Cells A and B as rows of the kernel: the averages over 40 000 draws against the exact
     enumeration (every operator, both reads), within five standard errors."""

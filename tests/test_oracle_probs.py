@@ -4,6 +4,7 @@ outcome in cells A and B under both rounding laws, against the paper's closed fo
 operators built from new roundings; planted errors must change the outcome."""
 from fractions import Fraction as Fr
 
+import numpy as np
 import pytest
 
 from oracle import probs
@@ -211,3 +212,21 @@ def test_monte_carlo_form_agrees_with_the_enumeration():
             assert np.allclose(cf["minus_SGp"][0], [float(x) for x in ex["minus_SGp"]], rtol=1e-5, atol=1e-7)
             assert np.allclose(cf["half_replay"][0], [float(x) for x in ex["half_replay"]], rtol=1e-5, atol=1e-7)
             assert np.allclose(cf["dV_rows"][0], [[float(x) for x in row] for row in ex["dV_rows"]], rtol=1e-5, atol=1e-7)
+
+
+def test_rows_are_keyed_by_their_place_in_the_whole_tensor():
+    """A block of rows rounded alone, told where it sits, gets the whole tensor's words; told
+    nothing, it gets other words (so the argument is not ignored)."""
+    rng = np.random.default_rng(5)
+    p = rng.dirichlet(np.ones(12), size=9).astype(np.float32)
+    V = rng.standard_normal((12, 4))
+    for law, param in ((probs.LAW_GRID, 1.0 / 16), (probs.LAW_SIGN, 1.0 / 256)):
+        whole = probs.rounded(p, law, param, 31, 1, 6)
+        part = probs.rounded(p[4:7], law, param, 31, 1, 6, first_row=4)
+        assert np.array_equal(part, whole[4:7])
+        assert not np.array_equal(probs.rounded(p[4:7], law, param, 31, 1, 6), whole[4:7])
+        a = probs.mc_sums(p, V, law, param, 31, 3, 2)
+        c = probs.mc_sums(p[4:7], V, law, param, 31, 3, 2, first_row=4)
+        for x, y in zip(a, c):
+            assert np.array_equal(x[:, 4:7], y)
+
