@@ -120,7 +120,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // streamed-tile ring: the backward modes have no P / dS buffers in shared memory (those operands
   // live in tensor memory), so their ring takes a third stage there, and the last 32 KB of that
   // space stage the second output of the dK/dV epilogue
-  constexpr uint32_t kStg = (MODE == AT_FWD || DQF) ? 2u : 3u;
+  constexpr uint32_t kStg = DQF ? 2u : 3u;
+  // stage s of the ring; the forward's third stage sits behind its P buffer (where the backward's dS would be)
+  auto stage_at = [&](uint32_t s) -> uint32_t { return (MODE == AT_FWD && s == 2u) ? base + 10u * kAtTile : str0 + s * 2u * kAtTile; };
   const uint32_t dst_buf = str0 + 2u * 2u * kAtTile;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
   const uint32_t dst_buf_unused = 0;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
   const uint32_t stage2 = str0 + 3u * 2u * kAtTile;
@@ -248,7 +250,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           const int step = it_begin + (it % nsteps);
           const uint32_t s = itg % kStg, ph = (itg / kStg) & 1u;
           if (!mbar_wait(b_sempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t d0 = str0 + s * 2 * kAtTile, d1 = d0 + kAtTile;
+          const uint32_t d0 = stage_at(s), d1 = d0 + kAtTile;
           mbar_expect_tx(b_sfull + 8 * s, 2 * kTileB);
           if (MODE == AT_DKV) {
             tma_load_3d(d0, &tm_q, b_sfull + 8 * s, 0, step * AT_BLK, bh);
@@ -289,7 +291,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) return false;
         if (!mbar_wait(b_sdp_free, (jt & 1u) ^ 1u, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
+        const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
         const uint32_t q_t = MODE == AT_DKV ? st0 : res0, k_t = MODE == AT_DKV ? res0 : st0;
         const uint32_t do_t = MODE == AT_DKV ? st1 : res1, v_t = MODE == AT_DKV ? res1 : st1;
         // DKV forms the transposes, S^T = K Q^T and dP^T = V dO^T (rows = keys), so that P^T and dS^T
@@ -329,7 +331,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       for (int it = 0; it < total && ok; ++it) {
         const uint32_t jg = itg + (uint32_t)it;
         const uint32_t s = jg % kStg, ip = jg & 1u;
-        const uint32_t st0 = str0 + s * 2 * kAtTile, st1 = st0 + kAtTile;
+        const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
         if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
         if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
         tc_fence_after();
