@@ -124,7 +124,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // stage s of the ring; the forward's third stage sits behind its P buffer (where the backward's dS would be)
   auto stage_at = [&](uint32_t s) -> uint32_t { return (MODE == AT_FWD && s == 2u) ? base + 10u * kAtTile : str0 + s * 2u * kAtTile; };
   const uint32_t dst_buf = str0 + 2u * 2u * kAtTile;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
-  const uint32_t dst_buf_unused = 0;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
   const uint32_t stage2 = str0 + 3u * 2u * kAtTile;
   uint8_t* gen = smem_raw + (base - raw);
   uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
@@ -265,7 +264,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {
+      // the whole warp walks the loop (loop control and descriptor arithmetic stay warp-uniform); one
+      // lane issues.  Measured: a 128 x 64 x 16 product with A in tensor memory issues every 32 cycles
+      // this way, every 45 from a single-lane branch.
+      const uint32_t leader = elect_one() ? 1u : 0u;
+      auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag));
+      };
       bool ok = true;
       uint32_t itg = 0;                                       // step counter across items
       int item = 0;
@@ -278,18 +284,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       const uint32_t ab = kAccDouble ? rb : 0u, aph = kAccDouble ? iph : ((uint32_t)item & 1u);
       const uint32_t res0 = res_base + rb * 2 * kAtTile, res1 = res0 + kAtTile;
       const uint32_t t_acc0 = t_accbase + ab * 128, t_acc1 = t_acc0 + 64;
-      if (!mbar_wait(b_res + 8 * rb, iph, abort_flag)) { ok = false; break; }
+      if (!wait_all(b_res + 8 * rb, iph)) { ok = false; break; }
       // the accumulators are free once the epilogue that last used them is done: with two buffers
       // that is checked here, with one just before the item's first accumulating product, so the
       // first S and dP of this item already run under the epilogue of the item before
-      if (kAccDouble && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
+      if (kAccDouble && !wait_all(b_acc_free + 8 * ab, aph ^ 1u)) { ok = false; break; }
       // S = Q K^T (and dP = dO V^T) of global step `jt`: both operands K-major, 64 = 4 x 16 along K.
       // Issued one step ahead: the softmax warps release the S / dP columns as soon as they hold
       // them in registers, so these products overlap the softmax arithmetic of the step before.
       auto issue_sdp = [&](uint32_t jt) -> bool {
         const uint32_t s = jt % kStg, ph = (jt / kStg) & 1u;
-        if (!mbar_wait(b_sfull + 8 * s, ph, abort_flag)) return false;
-        if (!mbar_wait(b_sdp_free, (jt & 1u) ^ 1u, abort_flag)) return false;
+        if (!wait_all(b_sfull + 8 * s, ph)) return false;
+        if (!wait_all(b_sdp_free, (jt & 1u) ^ 1u)) return false;
         tc_fence_after();
         const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
         const uint32_t q_t = MODE == AT_DKV ? st0 : res0, k_t = MODE == AT_DKV ? res0 : st0;
@@ -300,31 +306,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // 64 bytes of K per row: two steps of 32 elements
           const uint64_t a = make_smem_desc_sw64(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc_sw64(MODE == AT_DKV ? q_t : k_t);
 #pragma unroll
-          for (int k = 0; k < 2; ++k) tc_mma<true>(t_s, a + 2u * k, b + 2u * k, id8_s, k != 0);
+          for (int k = 0; k < 2; ++k) tc_mma_l<true>(leader, t_s, a + 2u * k, b + 2u * k, id8_s, k != 0);
           const uint64_t a2 = make_smem_desc_sw64(MODE == AT_DKV ? v_t : do_t), b2 = make_smem_desc_sw64(MODE == AT_DKV ? do_t : v_t);
 #pragma unroll
-          for (int k = 0; k < 2; ++k) tc_mma<true>(t_dp, a2 + 2u * k, b2 + 2u * k, id8_dp, k != 0);
+          for (int k = 0; k < 2; ++k) tc_mma_l<true>(leader, t_dp, a2 + 2u * k, b2 + 2u * k, id8_dp, k != 0);
         } else {
           {
             const uint64_t a = make_smem_desc(MODE == AT_DKV ? k_t : q_t), b = make_smem_desc(MODE == AT_DKV ? q_t : k_t);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma<false>(t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+            for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_s, a + 2u * k, b + 2u * k, id_sdp, k != 0);
           }
           if (MODE != AT_FWD) {
             const uint64_t a = make_smem_desc(MODE == AT_DKV ? v_t : do_t), b = make_smem_desc(MODE == AT_DKV ? do_t : v_t);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma<false>(t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
+            for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_dp, a + 2u * k, b + 2u * k, id_sdp, k != 0);
           }
         }
         if (MODE == AT_DKV) {
           // the extra K = 16 step: minus LSE/c into S^T, minus D into dP^T (see the X tiles)
           const uint32_t bb = jt % 3u;
-          if (!mbar_wait(b_bias + 8 * bb, (jt / 3u) & 1u, abort_flag)) return false;
+          if (!wait_all(b_bias + 8 * bb, (jt / 3u) & 1u)) return false;
           const uint64_t ones = make_smem_desc_k16(bias0);
-          tc_mma<false>(t_s, ones, make_smem_desc_k16(bias0 + (1u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
-          tc_mma<false>(t_dp, ones, make_smem_desc_k16(bias0 + (2u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
+          tc_mma_l<false>(leader, t_s, ones, make_smem_desc_k16(bias0 + (1u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
+          tc_mma_l<false>(leader, t_dp, ones, make_smem_desc_k16(bias0 + (2u + 2u * bb) * kAtBiasTile), id_sdp, 1u);
         }
-        tc_commit(b_sdp_full);
+        tc_commit_l(leader, b_sdp_full);
         return true;
       };
       if (ok && total > 0) ok = issue_sdp(itg);
@@ -333,30 +339,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const uint32_t s = jg % kStg, ip = jg & 1u;
         const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
         if (it + 1 < total && !issue_sdp(jg + 1)) { ok = false; break; }
-        if (!mbar_wait(b_pds_ready, ip, abort_flag)) { ok = false; break; }
+        if (!wait_all(b_pds_ready, ip)) { ok = false; break; }
         tc_fence_after();
         const uint32_t first = it == 0 ? 0u : 1u;             // overwrite on the first product
-        if (!kAccDouble && it == 0 && !mbar_wait(b_acc_free + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!kAccDouble && it == 0 && !wait_all(b_acc_free + 8 * ab, aph ^ 1u)) { ok = false; break; }
         if (F8K && MODE == AT_DKV) {
           // the same products on the codes: eight columns per 32 queries, 128 queries = 4 x 32 along K
           const uint64_t bdo = make_smem_desc_mn_sw64(st1), bq = make_smem_desc_mn_sw64(st0);
           if (DV) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_p + 8u * k, bdo + 128u * k, id8_pdo, first | (k != 0));
+            for (int k = 0; k < 4; ++k) tc_mma_ts_l<true>(leader, t_acc0, t_p + 8u * k, bdo + 128u * k, id8_pdo, first | (k != 0));
           }
 #pragma unroll
-          for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc1, t_ds + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
+          for (int k = 0; k < 4; ++k) tc_mma_ts_l<true>(leader, t_acc1, t_ds + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
           if (ND == 2 && !DV) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_ds2 + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
+            for (int k = 0; k < 4; ++k) tc_mma_ts_l<true>(leader, t_acc0, t_ds2 + 8u * k, bq + 128u * k, id8_ds, first | (k != 0));
           }
         } else if (F8K && MODE == AT_DQ) {
           const uint64_t bk = make_smem_desc_mn_sw64(st0);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc0, t_ds + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
+          for (int k = 0; k < 4; ++k) tc_mma_ts_l<true>(leader, t_acc0, t_ds + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
           if (ND == 2) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) tc_mma_ts_f8(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
+            for (int k = 0; k < 4; ++k) tc_mma_ts_l<true>(leader, t_acc1, t_ds2 + 8u * k, bk + 128u * k, id8_ds, first | (k != 0));
           }
         } else if (DQF) {
           // dV += P^T dO with P^T from tensor memory; dK += dS^T Q with dS^T K-major from shared memory
@@ -364,42 +370,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // buffer read MN-major (128 queries wide, 16 keys per step), K_j = the resident tile, MN-major
           const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
+          for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint64_t a = make_smem_desc(dst_buf + (k >> 2) * 16384u + (k & 3) * 32u);
-            tc_mma<false>(t_acc1, a, bq + 128u * k, id_kmn, first | (k != 0));
+            tc_mma_l<false>(leader, t_acc1, a, bq + 128u * k, id_kmn, first | (k != 0));
           }
           // the share of the step before has left tensor memory
-          if (!mbar_wait(b_dq_free, (jg & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          if (!wait_all(b_dq_free, (jg & 1u) ^ 1u)) { ok = false; break; }
           tc_fence_after();
           const uint64_t ads = make_smem_desc_mn(dst_buf, 16384u), bk = make_smem_desc_mn(res0, 16384u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma<false>(t_dq, ads + 128u * k, bk + 128u * k, id_mn, k != 0);
-          tc_commit(b_dq_full);
+          for (int k = 0; k < 8; ++k) tc_mma_l<false>(leader, t_dq, ads + 128u * k, bk + 128u * k, id_mn, k != 0);
+          tc_commit_l(leader, b_dq_full);
         } else if (MODE == AT_DKV) {
           // dV += P^T dO, dK += dS^T Q : A from tensor memory (row = key, eight columns per 16
           // queries), B MN-major = the streamed 128 x 64 tiles; 128 queries = 8 x 16 along K
           const uint64_t bdo = make_smem_desc_mn(st1, 16384u), bq = make_smem_desc_mn(st0, 16384u);
           if (DV) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
+            for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc0, t_p + 8u * k, bdo + 128u * k, id_kmn, first | (k != 0));
           }
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
+          for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc1, t_ds + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
           if (ND == 2 && !DV) {
             // second draw: its dS^T operand sits in the P columns, its dK in the dV accumulator
 #pragma unroll
-            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_ds2 + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
+            for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc0, t_ds2 + 8u * k, bq + 128u * k, id_kmn, first | (k != 0));
           }
         } else if (MODE == AT_DQ) {
           // dQ += dS K : A from tensor memory (row = query, eight columns per 16 keys), B MN-major = streamed K
           const uint64_t bk = make_smem_desc_mn(st0, 16384u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc0, t_ds + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
+          for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc0, t_ds + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
           if (ND == 2) {
 #pragma unroll
-            for (int k = 0; k < 8; ++k) tc_mma_ts(t_acc1, t_ds2 + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
+            for (int k = 0; k < 8; ++k) tc_mma_ts_l<false>(leader, t_acc1, t_ds2 + 8u * k, bk + 128u * k, id_kmn, first | (k != 0));
           }
         } else {
           // O_h += P_h V_h for the two halves of 64 keys, each into its own accumulator (its own running
@@ -408,17 +414,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint64_t a = make_smem_desc(pbuf + (k >> 2) * 16384u + (k & 3) * 32u);
-            tc_mma<false>(k < 4 ? t_acc0 : t_acc1, a, bk + 128u * k, id_kmn, first | ((k & 3) != 0));
+            tc_mma_l<false>(leader, k < 4 ? t_acc0 : t_acc1, a, bk + 128u * k, id_kmn, first | ((k & 3) != 0));
           }
         }
-        tc_commit(b_pds_free);
-        tc_commit(b_sempty + 8 * s);
+        tc_commit_l(leader, b_pds_free);
+        tc_commit_l(leader, b_sempty + 8 * s);
       }
       itg += (uint32_t)total;
       if (ok) {
         // this item's accumulators are complete (and its resident tiles no longer read: the epilogue
         // stages the output through their buffer and releases it)
-        tc_commit(b_acc + 8 * ab);
+        tc_commit_l(leader, b_acc + 8 * ab);
       }
       }  // items
     }
