@@ -146,6 +146,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   const uint32_t delta0 = bars + 2304;
   // DQF: the step's dQ share is complete / has been read out of tensor memory
   const uint32_t b_dq_full = bars + 3848, b_dq_free = bars + 3856;
+  // Plain dQ kernel: the two halves of 64 keys of a step are two pipelines (their own S and dP
+  // products, 128 x 64 each, their own hand-over barriers with the four softmax warps that own those
+  // columns, their own share of the dQ product), issued in turn by the one MMA warp, so that one half's
+  // hand-overs run under the other half's work.
+  constexpr bool PP = MODE == AT_DQ && !FP8 && !MC && ND == 1;
+  const uint32_t b_sdp_full1 = bars + 3864, b_sdp_free1 = bars + 3872, b_pds_ready1 = bars + 3880, b_pds_free1 = bars + 3888;
+  const uint32_t id_sdp64 = make_idesc(1u, 1u, 128, 64);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Persistent CTA: work items w = item_at(0), item_at(1), ... of nblk * BH, heavy blocks first
@@ -185,7 +192,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     }
     for (uint32_t s = 0; s < kStg; ++s) { mbar_init(b_sfull + 8 * s, 1); mbar_init(b_sempty + 8 * s, 1); }
     for (uint32_t s = 0; s < 3; ++s) mbar_init(b_bias + 8 * s, 8);
-    mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, 8); mbar_init(b_pds_ready, 8); mbar_init(b_pds_free, 1);
+    mbar_init(b_sdp_full, 1); mbar_init(b_sdp_free, PP ? 4 : 8); mbar_init(b_pds_ready, PP ? 4 : 8); mbar_init(b_pds_free, 1);
+    mbar_init(b_sdp_full1, 1); mbar_init(b_sdp_free1, 4); mbar_init(b_pds_ready1, 4); mbar_init(b_pds_free1, 1);
     mbar_init(b_dq_full, 1); mbar_init(b_dq_free, 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -333,6 +341,47 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         tc_commit_l(leader, b_sdp_full);
         return true;
       };
+      // PP: S and dP of half hh (keys 64 hh .. 64 hh + 63 of the step's tiles) of global step jt
+      auto issue_half = [&](uint32_t jt, uint32_t hh) -> bool {
+        const uint32_t s = jt % kStg, ph = (jt / kStg) & 1u;
+        if (!wait_all(b_sfull + 8 * s, ph)) return false;
+        if (!wait_all(hh ? b_sdp_free1 : b_sdp_free, (jt & 1u) ^ 1u)) return false;
+        tc_fence_after();
+        const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
+        const uint64_t a = make_smem_desc(res0), b = make_smem_desc(st0 + hh * 8192u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_s + 64u * hh, a + 2u * k, b + 2u * k, id_sdp64, k != 0);
+        const uint64_t a2 = make_smem_desc(res1), b2 = make_smem_desc(st1 + hh * 8192u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_dp + 64u * hh, a2 + 2u * k, b2 + 2u * k, id_sdp64, k != 0);
+        tc_commit_l(leader, hh ? b_sdp_full1 : b_sdp_full);
+        return true;
+      };
+      if (PP) {
+        if (ok && total > 0) ok = issue_half(itg, 0u) && issue_half(itg, 1u);
+        for (int it = 0; it < total && ok; ++it) {
+          const uint32_t jg = itg + (uint32_t)it;
+          const uint32_t s = jg % kStg, ip = jg & 1u;
+          const uint64_t bk = make_smem_desc_mn(stage_at(s), 16384u);
+          // in turn: the next step's S and dP of a half, then this step's dQ share of that half (taking
+          // both halves' S and dP first, or giving each half an MMA warp of its own, measured slower)
+#pragma unroll
+          for (uint32_t hh = 0; hh < 2; ++hh) {
+            if (it + 1 < total && !issue_half(jg + 1, hh)) { ok = false; break; }
+            if (!wait_all(hh ? b_pds_ready1 : b_pds_ready, ip)) { ok = false; break; }
+            tc_fence_after();
+            if (it == 0 && hh == 0 && !wait_all(b_acc_free + 8 * ab, aph ^ 1u)) { ok = false; break; }
+            // dQ += dS_hh K_hh: 64 keys = 4 x 16 along K
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k)
+              tc_mma_ts_l<false>(leader, t_acc0, t_ds + 32u * hh + 8u * k, bk + 128u * (4u * hh + k), id_kmn,
+                                 (it != 0 || hh != 0 || k != 0) ? 1u : 0u);
+            tc_commit_l(leader, hh ? b_pds_free1 : b_pds_free);
+          }
+          if (!ok) break;
+          tc_commit_l(leader, b_sempty + 8 * s);
+        }
+      } else {
       if (ok && total > 0) ok = issue_sdp(itg);
       for (int it = 0; it < total && ok; ++it) {
         const uint32_t jg = itg + (uint32_t)it;
@@ -419,6 +468,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         }
         tc_commit_l(leader, b_pds_free);
         tc_commit_l(leader, b_sempty + 8 * s);
+      }
       }
       itg += (uint32_t)total;
       if (ok) {
@@ -592,7 +642,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         kblk = step;
       }
       const int qb0 = (MODE == AT_DKV ? step : blk) * AT_BLK;  // first query of this step's score tile
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sdp_full, ip, abort_flag));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait((PP && h) ? b_sdp_full1 : b_sdp_full, ip, abort_flag));
       if (!ok) break;
       tc_fence_after();
       // this thread's 64 scores (and 64 dP values) into registers, then hand the TMEM columns back
@@ -607,7 +657,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(b_sdp_free);
+      if (lane == 0) mbar_arrive((PP && h) ? b_sdp_free1 : b_sdp_free);
       if (bias_due) {                                         // lands under this step's arithmetic
         bias_next = bias_fetch(bias_bh, bias_step);
         bias_next2 = bias_fetch2(bias_bh, bias_step);
@@ -803,7 +853,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
           // the dS operand is free once the product of the previous step has read it; then the row's
           // 64 columns go back into tensor memory as 32 packed pairs (columns h*32 .. h*32+31)
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait((PP && h) ? b_pds_free1 : b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
           st_half(t_ds, 0, *reinterpret_cast<const uint32_t(*)[16]>(&dk[0]));
           st_half(t_ds, 1, *reinterpret_cast<const uint32_t(*)[16]>(&dk[16]));
@@ -893,7 +943,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       }
       if (MODE == AT_FWD || DQF) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(b_pds_ready);
+      if (lane == 0) mbar_arrive((PP && h) ? b_pds_ready1 : b_pds_ready);
       // DQF: the dQ share of the step before, now complete (its products were committed ahead of the
       // operands' release that this step has already waited for), goes out while this step's products run
       if (DQF && it > 0) {
