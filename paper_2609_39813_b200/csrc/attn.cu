@@ -344,7 +344,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
       // PP: S and dP of half hh (keys 64 hh .. 64 hh + 63 of the step's tiles) of global step jt
       auto issue_half = [&](uint32_t jt, uint32_t hh) -> bool {
         const uint32_t s = jt % kStg, ph = (jt / kStg) & 1u;
-        if (!wait_all(b_sfull + 8 * s, ph)) return false;
+        if (hh == 0 && !wait_all(b_sfull + 8 * s, ph)) return false;   // (the second half follows the first: the tiles have landed)
         if (!wait_all(hh ? b_sdp_free1 : b_sdp_free, (jt & 1u) ^ 1u)) return false;
         tc_fence_after();
         const uint32_t st0 = stage_at(s), st1 = st0 + kAtTile;
