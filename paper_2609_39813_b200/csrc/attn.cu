@@ -732,9 +732,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
                              uint32_t& dso) {
           float s0 = 0.f, s1 = 0.f;
           if (MODE == AT_FWD) run_l += p0 + p1;             // the row's normaliser, from the unrounded values
-          if (MODE != AT_FWD) {
-            s0 = p0 * (__uint_as_float(dp0) * dp_mul - d0);
-            s1 = p1 * (__uint_as_float(dp1) * dp_mul - d1);
+          if (MODE == AT_DKV && !FP8) {
+            // (the accumulators already hold dP - D): both products in one packed instruction
+            mul_f32x2(s0, s1, p0, p1, __uint_as_float(dp0), __uint_as_float(dp1));
+          } else if (MODE != AT_FWD) {
+            float t0, t1;
+            fma_f32x2(t0, t1, __uint_as_float(dp0), __uint_as_float(dp1), dp_mul, dp_mul, -d0, -d1);
+            mul_f32x2(s0, s1, p0, p1, t0, t1);
           }
           if (FP8 && MODE != AT_FWD) {                      // the forward keeps P unrounded
             if (F8K) {                                      // the codes themselves (two per word for now)
@@ -764,7 +768,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // DKV: the accumulators already hold s - LSE/c and dP - D (see the X tiles)
           const float l0 = MODE == AT_DKV ? 0.f : lse2, d0 = MODE == AT_DKV ? 0.f : dq;
           const float l1 = l0, d1 = d0;
-          float a0 = fmaf(__uint_as_float(sv[j]), c2, -l0), a1 = fmaf(__uint_as_float(sv[j + 1]), c2, -l1);
+          float a0, a1;
+          if (MODE == AT_DKV) {
+            mul_f32x2(a0, a1, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]), c2, c2);
+          } else {
+            fma_f32x2(a0, a1, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]), c2, c2, -l0, -l1);
+          }
           if (masked) {
             if (!valid_at(j)) a0 = -INFINITY;
             if (!valid_at(j + 1)) a1 = -INFINITY;
@@ -811,15 +820,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           // packed operands of both draws stay within the register budget
           uint32_t da[16], db[16];
           auto pair2_at = [&](int j, bool masked) {
-            float a0 = fmaf(__uint_as_float(sv[j]), c2, -lse2), a1 = fmaf(__uint_as_float(sv[j + 1]), c2, -lse2);
+            float a0, a1;
+            fma_f32x2(a0, a1, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]), c2, c2, -lse2, -lse2);
             if (masked) {
               if (!valid_at(j)) a0 = -INFINITY;
               if (!valid_at(j + 1)) a1 = -INFINITY;
             }
             const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-            const float x0 = __uint_as_float(dv[j]) * dp_mul, x1 = __uint_as_float(dv[j + 1]) * dp_mul;
-            da[(j & 31) >> 1] = pack_ds(p0 * (x0 - dq), p1 * (x1 - dq));
-            db[(j & 31) >> 1] = pack_ds(p0 * (x0 - dq2), p1 * (x1 - dq2));
+            float t0, t1, u0, u1, s0, s1, r0, r1;
+            fma_f32x2(t0, t1, __uint_as_float(dv[j]), __uint_as_float(dv[j + 1]), dp_mul, dp_mul, -dq, -dq);
+            fma_f32x2(u0, u1, __uint_as_float(dv[j]), __uint_as_float(dv[j + 1]), dp_mul, dp_mul, -dq2, -dq2);
+            mul_f32x2(s0, s1, p0, p1, t0, t1);
+            mul_f32x2(r0, r1, p0, p1, u0, u1);
+            da[(j & 31) >> 1] = pack_ds(s0, s1);
+            db[(j & 31) >> 1] = pack_ds(r0, r1);
           };
           if (!edge) {
 #pragma unroll
@@ -865,6 +879,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           uint32_t da[16], db[16];
           const uint32_t dbase = delta0 + (((itg + (uint32_t)it) % 3u) * 128u + (uint32_t)h * 64u) * 4u;
           auto pair2_at = [&](int j, bool masked) {
+            // (scalar arithmetic here: the packed forms cost this variant registers it does not have)
             float a0 = __uint_as_float(sv[j]) * c2, a1 = __uint_as_float(sv[j + 1]) * c2;
             if (masked) {
               if (!valid_at(j)) a0 = -INFINITY;
