@@ -298,7 +298,8 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         };
         uint32_t pk[32];
         auto pair_at = [&](int j, bool masked) {
-          float a0 = __uint_as_float(sv[j]) * c2, a1 = __uint_as_float(sv[j + 1]) * c2;
+          float a0, a1;
+          mul_f32x2(a0, a1, __uint_as_float(sv[j]), __uint_as_float(sv[j + 1]), c2, c2);
           if (masked) {
             if (!valid_at(j)) a0 = -INFINITY;
             if (!valid_at(j + 1)) a1 = -INFINITY;
