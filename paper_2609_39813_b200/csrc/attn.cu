@@ -13,13 +13,15 @@
 //           running maximum m_h (moved lazily, only past 2^8) and O_h += exp(S - m_h) V in an
 //           accumulator of its own, rescaled when m_h moves; the halves meet in the epilogue,
 //           O_i = (w_0 O_0 + w_1 O_1), which also gives the row's log-sum-exp.
-// No cross-CTA reduction exists in any mode, so results are bit-reproducible.
+// No cross-CTA reduction exists in these modes, so results are bit-reproducible (the one-kernel
+// form of the backward, further down, is the exception).
 //
-// Per inner step: S = Q K^T and dP = dO V^T (128x128x64 each) land in TMEM columns [0,128) and
-// [128,256); eight softmax warps (two per TMEM lane quarter, 64 keys each) turn them into P and dS,
-// written as bf16 into shared memory in the 128-byte-swizzle layout; the products with P / dS then
-// read those buffers directly (MN-major A for dV and dK, K-major A for dQ and O) and the TMA-loaded
-// 128 x 64 tiles as MN-major B.  320 threads: warp 0 TMA, warp 1 MMA, warps 2..9 softmax + epilogue.
+// Per inner step: S = Q K^T and dP = dO V^T (128x128x64 each; the dK/dV mode forms the transposes) land
+// in TMEM columns [0,128) and [128,256); eight softmax warps (two per TMEM lane quarter, 64 columns
+// each) turn them into P and dS and write those back into tensor memory as packed bf16 pairs (FP8-
+// operand mode: as codes), where the accumulating products read them as their A operand, row per
+// lane; the TMA-loaded 128 x 64 tiles are the MN-major B operands.  320 threads: warp 0 TMA, warp 1
+// MMA (the whole warp walks the loop, one elected lane issues), warps 2..9 softmax + epilogue.
 // Head dimension 64, bf16 inputs, FP32 outputs.  Every wait is bounded.
 #include <string.h>
 
@@ -458,13 +460,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           }
         } else {
           // O_h += P_h V_h for the two halves of 64 keys, each into its own accumulator (its own running
-          // maximum): A K-major from the P buffer in shared memory, B MN-major = streamed V
+          // maximum): A = P from tensor memory (eight columns per 16 keys), B MN-major = streamed V
           const uint64_t bk = make_smem_desc_mn(st1, 16384u);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint64_t a = make_smem_desc(pbuf + (k >> 2) * 16384u + (k & 3) * 32u);
-            tc_mma_l<false>(leader, k < 4 ? t_acc0 : t_acc1, a, bk + 128u * k, id_kmn, first | ((k & 3) != 0));
-          }
+          for (int k = 0; k < 8; ++k)
+            tc_mma_ts_l<false>(leader, k < 4 ? t_acc0 : t_acc1, t_dp + 8u * k, bk + 128u * k, id_kmn, first | ((k & 3) != 0));
         }
         tc_commit_l(leader, b_pds_free);
         tc_commit_l(leader, b_sempty + 8 * s);
@@ -808,13 +808,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             tmem_wait_st();
             tc_fence_before();
           }
-          // 64 keys = 8 chunks of 16 bytes in row r of half h of the shared P buffer: chunk index t ^ (r & 7)
-#pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            const uint32_t off = (uint32_t)h * 16384u + (uint32_t)r * 128u + ((uint32_t)(t ^ (r & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pbuf + off), "r"(pk[4 * t]), "r"(pk[4 * t + 1]),
-                         "r"(pk[4 * t + 2]), "r"(pk[4 * t + 3]) : "memory");
-          }
+          // the row's 64 probabilities go back into tensor memory as 32 packed pairs (columns h*32 .. h*32+31
+          // of the P operand, which sits where the backward modes keep dP)
+          st_half(t_dp, 0, *reinterpret_cast<const uint32_t(*)[16]>(&pk[0]));
+          st_half(t_dp, 1, *reinterpret_cast<const uint32_t(*)[16]>(&pk[16]));
+          tmem_wait_st();
+          tc_fence_before();
         } else if (MODE == AT_DQ && ND == 2) {
           // two draws: one exponential per element, two dS values; 32 columns at a time so that the
           // packed operands of both draws stay within the register budget
@@ -956,7 +955,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
           tc_fence_before();
         }
       }
-      if (MODE == AT_FWD || DQF) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (DQF) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive((PP && h) ? b_pds_ready1 : b_pds_ready);
       // DQF: the dQ share of the step before, now complete (its products were committed ahead of the
