@@ -152,7 +152,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   // products, 128 x 64 each, their own hand-over barriers with the four softmax warps that own those
   // columns, their own share of the dQ product), issued in turn by the one MMA warp, so that one half's
   // hand-overs run under the other half's work.
-  constexpr bool PP = MODE == AT_DQ && !FP8 && !MC && ND == 1;
+  constexpr bool PP = (MODE == AT_DQ || MODE == AT_FWD) && !FP8 && !MC && ND == 1;
   const uint32_t b_sdp_full1 = bars + 3864, b_sdp_free1 = bars + 3872, b_pds_ready1 = bars + 3880, b_pds_free1 = bars + 3888;
   const uint32_t id_sdp64 = make_idesc(1u, 1u, 128, 64);
 
@@ -353,9 +353,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         const uint64_t a = make_smem_desc(res0), b = make_smem_desc(st0 + hh * 8192u);
 #pragma unroll
         for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_s + 64u * hh, a + 2u * k, b + 2u * k, id_sdp64, k != 0);
-        const uint64_t a2 = make_smem_desc(res1), b2 = make_smem_desc(st1 + hh * 8192u);
+        if (MODE != AT_FWD) {
+          const uint64_t a2 = make_smem_desc(res1), b2 = make_smem_desc(st1 + hh * 8192u);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_dp + 64u * hh, a2 + 2u * k, b2 + 2u * k, id_sdp64, k != 0);
+          for (int k = 0; k < 4; ++k) tc_mma_l<false>(leader, t_dp + 64u * hh, a2 + 2u * k, b2 + 2u * k, id_sdp64, k != 0);
+        }
         tc_commit_l(leader, hh ? b_sdp_full1 : b_sdp_full);
         return true;
       };
@@ -364,7 +366,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
         for (int it = 0; it < total && ok; ++it) {
           const uint32_t jg = itg + (uint32_t)it;
           const uint32_t s = jg % kStg, ip = jg & 1u;
-          const uint64_t bk = make_smem_desc_mn(stage_at(s), 16384u);
+          const uint64_t bk = make_smem_desc_mn(stage_at(s) + (MODE == AT_FWD ? kAtTile : 0u), 16384u);   // dQ: K; forward: V
           // in turn: the next step's S and dP of a half, then this step's dQ share of that half (taking
           // both halves' S and dP first, or giving each half an MMA warp of its own, measured slower)
 #pragma unroll
@@ -372,12 +374,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             if (it + 1 < total && !issue_half(jg + 1, hh)) { ok = false; break; }
             if (!wait_all(hh ? b_pds_ready1 : b_pds_ready, ip)) { ok = false; break; }
             tc_fence_after();
-            if (it == 0 && hh == 0 && !wait_all(b_acc_free + 8 * ab, aph ^ 1u)) { ok = false; break; }
-            // dQ += dS_hh K_hh: 64 keys = 4 x 16 along K
+            if (!kAccDouble && it == 0 && hh == 0 && !wait_all(b_acc_free + 8 * ab, aph ^ 1u)) { ok = false; break; }
+            if (MODE == AT_FWD) {
+              // O_hh += P_hh V_hh into the half's own accumulator
 #pragma unroll
-            for (uint32_t k = 0; k < 4; ++k)
-              tc_mma_ts_l<false>(leader, t_acc0, t_ds + 32u * hh + 8u * k, bk + 128u * (4u * hh + k), id_kmn,
-                                 (it != 0 || hh != 0 || k != 0) ? 1u : 0u);
+              for (uint32_t k = 0; k < 4; ++k)
+                tc_mma_ts_l<false>(leader, hh ? t_acc1 : t_acc0, t_dp + 32u * hh + 8u * k, bk + 128u * (4u * hh + k), id_kmn,
+                                   (it != 0 || k != 0) ? 1u : 0u);
+            } else {
+              // dQ += dS_hh K_hh: 64 keys = 4 x 16 along K
+#pragma unroll
+              for (uint32_t k = 0; k < 4; ++k)
+                tc_mma_ts_l<false>(leader, t_acc0, t_ds + 32u * hh + 8u * k, bk + 128u * (4u * hh + k), id_kmn,
+                                   (it != 0 || hh != 0 || k != 0) ? 1u : 0u);
+            }
             tc_commit_l(leader, hh ? b_pds_free1 : b_pds_free);
           }
           if (!ok) break;
@@ -789,7 +799,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
             for (int j = 0; j < 64; j += 2) pair_at(j, true);
           }
           // the P buffer is free once the product of the previous step has read it
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_pds_free, ip ^ 1u, abort_flag));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait((PP && h) ? b_pds_free1 : b_pds_free, ip ^ 1u, abort_flag));
           if (!ok) break;
           if (__any_sync(0xFFFFFFFFu, resc != 1.f)) {
             // that product was also the last one to add to this half's accumulator: rescale the row
