@@ -358,7 +358,8 @@ def attention_section(b, peaks, steps=3):
                               algorithmic_tflops=5 * prod / bwd / 1e12, algorithmic_frac=5 * prod / bwd / 1e12 / peak,
                               peak_nominal=NOMINAL_BF16_TFLOPS, frac_of_nominal=(4 + 3) * prod / bwd / 1e12 / NOMINAL_BF16_TFLOPS,
                               note="achieved counts the 7 causal products of 2*S*S*d/2 flop per head that the two "
-                                   "kernels compute, algorithmic_* the 5 a backward needs; exp on the SFU co-bounds it"),
+                                   "kernels compute, algorithmic_* the 5 a backward needs; measured: paced by the hand-overs between "
+                                   "the MMA warp and the softmax warps, tensor pipe 39-48 % and exp2/convert unit 46-52 % busy"),
                 diag_status=b.read_diag(diag)["status"])
 
 
