@@ -33,14 +33,13 @@
 
 namespace bsp {
 
-constexpr int kAtPBytes = AT_BLK * AT_BLK * 2;    // 32 KB: P or dS, two 64-key halves of 16 KB
 constexpr int kAtThreads = 320;
 constexpr int kAtSoftWarp0 = 2;                   // first softmax warp
 constexpr int kAtSoftThread0 = kAtSoftWarp0 * 32;
-// shared memory: res0, res1, str[2][2], P, dS, barriers
+// shared memory: 12 tiles of 16 KB (resident, ring, staging), barriers and small buffers, the extra-step tiles
 constexpr int kAtBiasTile = AT_BLK * 16 * 2;      // 4 KB: one 128 x 16 bf16 tile of the extra K = 16 step (DKV)
 constexpr int kAtBias = 7 * kAtBiasTile;          // a tile of ones, then three buffers of (LSE tile, D tile)
-constexpr int kAtSmem = 4 * kAtTile + 4 * kAtTile + 2 * kAtPBytes + 1024 /*alignment*/ + 4096 /*barriers, exchange*/ +
+constexpr int kAtSmem = 12 * kAtTile + 1024 /*alignment*/ + 4096 /*barriers, exchange*/ +
                         kAtBias;
 
 struct AttnParams {
@@ -108,27 +107,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
-  // shared memory: resident tiles [2 buffers][2 tiles]; then FWD: streamed tiles [2 stages][2 tiles]
-  // and the P buffer; DKV / DQ: streamed tiles [4 stages][2 tiles] over the same 128 KB
+  // shared memory, in 16 KB tiles: resident tiles [2 buffers][2 tiles]; the ring of streamed tiles
+  // [3 stages][2 tiles] (the one-kernel form: 2 stages, the third's space holds dS^T); 32 KB of staging
+  // (second output of the dK/dV epilogue, dQ shares of the one-kernel form); barriers and small buffers
   const uint32_t res_base = base;
   const uint32_t str0 = base + 4 * kAtTile;                 // stage s: str0 + s*2*kAtTile (+kAtTile for the 2nd tile)
-  const uint32_t pbuf = base + 8 * kAtTile, dsbuf = pbuf + kAtPBytes;
-  const uint32_t bars = dsbuf + kAtPBytes;
+  const uint32_t bars = base + 12 * kAtTile;
   // barriers (8 bytes each): res_full[2], res_empty[2], str_full[2], str_empty[2], sdp_full, sdp_free,
   // pds_ready, pds_free, acc_full[2], acc_free[2]
   const uint32_t b_res = bars, b_res_empty = bars + 16, b_sfull = bars + 32, b_sempty = bars + 64,
                  b_sdp_full = bars + 96, b_sdp_free = bars + 104, b_pds_ready = bars + 112, b_pds_free = bars + 120,
                  b_acc = bars + 128, b_acc_free = bars + 144;
-  // streamed-tile ring: the backward modes have no P / dS buffers in shared memory (those operands
-  // live in tensor memory), so their ring takes a third stage there, and the last 32 KB of that
-  // space stage the second output of the dK/dV epilogue
   constexpr uint32_t kStg = DQF ? 2u : 3u;
-  // stage s of the ring; the forward's third stage sits behind its P buffer (where the backward's dS would be)
-  auto stage_at = [&](uint32_t s) -> uint32_t { return (MODE == AT_FWD && s == 2u) ? base + 10u * kAtTile : str0 + s * 2u * kAtTile; };
+  auto stage_at = [&](uint32_t s) -> uint32_t { return str0 + s * 2u * kAtTile; };
   const uint32_t dst_buf = str0 + 2u * 2u * kAtTile;         // DQF: dS^T [128 keys][2 halves of 64 queries], 32 KB
   const uint32_t stage2 = str0 + 3u * 2u * kAtTile;
   uint8_t* gen = smem_raw + (base - raw);
-  uint8_t* bars_gen = gen + 8 * kAtTile + 2 * kAtPBytes;
+  uint8_t* bars_gen = gen + 12 * kAtTile;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars_gen + 160);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars_gen + 164);
   float* xchg = reinterpret_cast<float*>(bars_gen + 176);   // FWD: row max / sum exchange between column halves
