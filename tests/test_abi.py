@@ -101,3 +101,8 @@ def test_host_side_argument_errors_need_no_gpu(built):
                           None, 0, None, None) == b.ERR_ARG                          # dx_read out of range
     assert l.bsp_linear_wgrad(8, 16, 16, 16, q, b.READ_FORWARD, 16, q, 8, 16, None, None, None, None, 0,
                               None, None) == b.ERR_ALIGN                             # ld_t not a multiple of 16
+    # the one-kernel attention backward: head width, missing gradient, misaligned operand (in that order)
+    args = lambda Dh, q_, dq_: (1, 1, 128, Dh, 1, 0.125, q_, 32, 48, 64, b.BF16, 80, 96, dq_, 112, 128, None, None)
+    assert l.bsp_attn_bwd_dterm_fused(*args(128, 16, 144)) == b.ERR_UNSUPPORTED
+    assert l.bsp_attn_bwd_dterm_fused(*args(64, 16, None)) == b.ERR_ARG
+    assert l.bsp_attn_bwd_dterm_fused(*args(64, 24, 144)) == b.ERR_ALIGN
