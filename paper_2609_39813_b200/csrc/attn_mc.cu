@@ -284,6 +284,9 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         uint32_t sv[64];
         tmem_ld32_nowait(t_s + lane_off + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
         tmem_ld32_nowait(t_s + lane_off + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+        // the step's Q tile has landed long ago (S^T read it); this thread still has to see its barrier
+        // before it reads the tile further down: the test goes out here, under the tensor-memory load
+        const uint32_t q_seen = mbar_try_wait(b_sfull + 8 * (jt % kDkStages), (jt / kDkStages) & 1u);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
@@ -337,8 +340,10 @@ attn_dk_diff_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         {
           const uint32_t s = jt % kDkStages, ph = (jt / kDkStages) & 1u;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sfull + 8 * s, ph, abort_flag));   // (long complete: S^T read the tile)
-          if (!ok) break;
+          if (!__all_sync(0xFFFFFFFFu, q_seen)) {
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(b_sfull + 8 * s, ph, abort_flag));
+            if (!ok) break;
+          }
           // the row factors -c (D_k - D*) of the draws (zero for a draw this launch does not have)
           uint32_t f2[kDkND];
           asm volatile("" : "+f"(dref_raw));
